@@ -1,0 +1,267 @@
+/*
+ * kvp.h -- C ABI of libkvp: KV-cache placement bound search on one NVIDIA B200.
+ *
+ * The library scores and searches placement schedules for the problem posed in
+ * "Accelerating LLM Inference via Dynamic KV Cache Placement in Heterogeneous
+ * Memory System" (arXiv 2508.13231), Section III:
+ *
+ *   - a KV cache of `units` equally sized blocks, `steps` decode steps, and for
+ *     every step the set of blocks that sparse attention reads (access bitmap);
+ *   - a placement schedule P: for every step the set of blocks that are resident
+ *     in HBM while that step reads (all other blocks are in off-package DRAM);
+ *   - the latency model of Eq. 1-4 and the capacity constraint of Eq. 5.
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ * Bitmaps. A bitmap has `steps` rows of W32 = ceil(units/32) uint32 words,
+ *   row-major ("step-major"). Unit u of step s is bit (u & 31) of word
+ *   [s*W32 + (u >> 5)]. Pad bits (u >= units) of the last word are ignored on
+ *   input and written as 0 on output.
+ * Time. All costs are exact integers ("ticks"). With g = gcd(B_h, B_k, B_d),
+ *   B'_x = B_x / g and L = lcm(B'_h, B'_k, B'_d), the weights are
+ *   kappa_h = L/B'_h, kappa_k = L/B'_k, kappa_d = L/B'_d,
+ *   kappa_e = max(kappa_k, kappa_d)  (the 1/min{B_k,B_d} of Eq. 4),
+ *   and one tick lasts bytes_per_unit / (L*g) seconds.
+ * Step cost (Eq. 2-4) for step s with previous row P[s-1] (P[-1] := P[0]):
+ *   hr = |A[s] & P[s]|, er = |A[s]| - hr, mi = |P[s] & ~P[s-1]|,
+ *   mo = |~P[s] & P[s-1]|, Fh/Fe = 1 when KVP_MIG_HBM/KVP_MIG_EXT is set,
+ *   th = kappa_h*(hr + hw[s] + Fh*(mi+mo))                              (Eq. 3)
+ *   te = kappa_e*er + max(kappa_k*(ew[s] + Fe*mo), kappa_k*Fe*mi,
+ *                         kappa_d*(ew[s] + Fe*(mi+mo)))                 (Eq. 4)
+ *   f_s = max(th, te)  (Eq. 2);   T = sum_s f_s  (Eq. 1);
+ *   feasible iff |P[s]| <= hbm_capacity_units for every s  (Eq. 5).
+ * Pointers. Every pointer argument is marked (host) or (device). Device
+ *   buffers are owned by the caller, must be 16-byte aligned and must stay
+ *   valid until the work queued on `stream` has finished. `stream` is a
+ *   cudaStream_t passed as void* (NULL = the legacy default stream).
+ * Errors. Every function returns KVP_OK or a negative code; there are no
+ *   exceptions, no abort, no output on stdout. On error, outputs are
+ *   unspecified but no memory outside the documented buffers is touched.
+ *   There is no CPU fallback: without a usable CUDA device every compute
+ *   call returns KVP_ERR_CUDA.
+ */
+#ifndef KVP_H_
+#define KVP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KVP_OK             0
+#define KVP_ERR_ARG       -1  /* null pointer, zero size, cap > units, bad enum, ...           */
+#define KVP_ERR_CAPACITY  -2  /* an initial schedule violates Eq. 5                              */
+#define KVP_ERR_RANGE     -3  /* tick weights or sizes outside the supported integer ranges     */
+#define KVP_ERR_CUDA      -4  /* a CUDA runtime call failed (see kvp_last_cuda_error)           */
+#define KVP_ERR_NOMEM     -5  /* device or host allocation failed                                */
+#define KVP_ERR_TIMEOUT   -6  /* a bounded device-side wait expired                              */
+#define KVP_ERR_INTERNAL  -7  /* self-check failed: re-scored winner differs from tracked ticks */
+
+#define KVP_MIG_HBM 1u  /* migrations occupy HBM bandwidth: the |M^i|+|M^o| terms of Eq. 3   */
+#define KVP_MIG_EXT 2u  /* migrations occupy link/DRAM bandwidth: the M terms of Eq. 4      */
+#define KVP_MIG_PAPER (KVP_MIG_HBM | KVP_MIG_EXT)
+
+/* Bandwidths of Eq. 3-4 in bytes per second (Table I gives 4.9e12 / 9e11 / 5e11). */
+typedef struct {
+    uint64_t bw_hbm;    /* B_h */
+    uint64_t bw_link;   /* B_k, uni-directional bandwidth of the full-duplex link */
+    uint64_t bw_dram;   /* B_d, off-package DRAM channel bandwidth */
+    uint32_t mig_flags; /* KVP_MIG_*; 0 = migrations are free (test mode with a closed-form optimum) */
+    uint32_t reserved;  /* must be 0 */
+} kvp_memsys;
+
+typedef struct kvp_problem kvp_problem; /* opaque; owns device copies of everything it needs */
+
+/* Derived integer weights of a problem (see "Time" above). */
+typedef struct {
+    uint64_t kappa_h, kappa_k, kappa_d, kappa_e;
+    uint64_t lcm, gcd;
+    double   seconds_per_tick;
+    uint32_t units, steps, words_per_row, capacity;
+} kvp_info;
+
+/*
+ * kvp_create -- build a problem instance (Section III-A: units, access pattern
+ * known a priori, capacity P_H <= 100% of `hbm_capacity_units`, bandwidths).
+ *   out              (host)   receives the handle.
+ *   access_bitmaps   (device) [steps][W32], copied; the caller may free it after
+ *                             the stream work finished.
+ *   hw_units/ew_units (host)  [steps] or NULL (= all zero): |H^w|, |E^w| of
+ *                             Eq. 3-4 in units, caller-supplied constants.
+ * Limits: 1 <= units < 2^26, 1 <= steps <= 32768, hbm_capacity_units <= units,
+ * kappa_max * (2*units + max hw + max ew) < 2^31 (else KVP_ERR_RANGE).
+ * Synchronises `stream` before returning.
+ */
+int kvp_create(kvp_problem** out, uint32_t units, uint64_t bytes_per_unit, uint32_t steps,
+               const uint32_t* access_bitmaps, uint32_t hbm_capacity_units,
+               const kvp_memsys* mem, const uint32_t* hw_units, const uint32_t* ew_units,
+               void* stream);
+
+/* Frees the handle and every device buffer it owns. NULL is allowed. */
+void kvp_destroy(kvp_problem* p);
+
+/* Fills *info (host). */
+int kvp_get_info(const kvp_problem* p, kvp_info* info);
+
+/*
+ * kvp_eval -- score `n` schedules with Eq. 1-4 and test Eq. 5.
+ *   schedules     (device) [n][steps][W32]
+ *   step_ticks    (device) [n][steps] uint64 or NULL : f_s
+ *   total_ticks   (device) [n] uint64                : T
+ *   step_seconds  (device) [n][steps] double or NULL : f_s * seconds_per_tick
+ *   total_seconds (device) [n] double or NULL        : T * seconds_per_tick
+ *   bad_step      (device) [n] int32 or NULL : first step whose row holds more
+ *                 than hbm_capacity_units units, or -1 when the schedule is feasible
+ *                 (an infeasible schedule is still scored).
+ * Asynchronous on `stream`; uses scratch owned by the problem, so calls on the
+ * same problem must be issued on one stream at a time.
+ */
+int kvp_eval(kvp_problem* p, const uint32_t* schedules, uint32_t n,
+             uint64_t* step_ticks, uint64_t* total_ticks,
+             double* step_seconds, double* total_seconds, int32_t* bad_step, void* stream);
+
+/*
+ * kvp_eval_counts -- the four per-step cardinalities the cost model is built on.
+ *   counts (device) [n][steps][4] uint32 = {hr, mi, mo, occ} with occ = |P[s]|.
+ */
+int kvp_eval_counts(kvp_problem* p, const uint32_t* schedules, uint32_t n,
+                    uint32_t* counts, void* stream);
+
+/* Initial placement of a chain. */
+#define KVP_INIT_STATIC_FIRST 0u /* units 0..cap-1 at every step: the Static Placement baseline (Section IV-A) */
+#define KVP_INIT_STATIC_FREQ  1u /* the cap units with most accesses over all steps (ties: lower index)     */
+#define KVP_INIT_USER         2u /* init_schedule */
+
+#define KVP_TABLE_Q 1024u        /* entries per temperature level of the acceptance table */
+
+/*
+ * Simulated-annealing parameters (Section III-B: Metropolis rule exp(-dT/C),
+ * initial acceptance ratio p0 = 0.8, geometric cooling alpha = 0.9, stop when the
+ * best improves by < 0.1% across successive temperature levels or the budget ends).
+ * The state that is annealed is the schedule itself: each move either swaps the
+ * placement of two units or flips one unit over a run of consecutive steps.
+ */
+typedef struct {
+    uint32_t chains;            /* independent chains, >= 1                                         */
+    uint32_t levels;            /* temperature levels, 1..4096; level(m) = min(levels-1, m/(moves/levels)) */
+    uint64_t moves;             /* proposals per chain, >= 1                                        */
+    uint64_t seed;              /* Philox key                                                       */
+    double   p0;                /* target initial acceptance of an average uphill move, in (0,1)    */
+    double   alpha;             /* geometric cooling factor, in (0,1]                               */
+    const double* temps;        /* (host) [levels] temperatures in ticks, or NULL = derive from p0, alpha */
+    uint32_t early_stop_permille;   /* stop a chain at a level boundary when its best improved by less
+                                       than this many 1/1000 since the previous boundary; 0 = never    */
+    uint32_t early_stop_from_level; /* the rule is not applied at boundaries entering levels below this */
+    uint32_t init_mode;         /* KVP_INIT_*                                                        */
+    uint32_t p_swap_256;        /* P(swap move) * 256, 0..256; the rest are flip moves              */
+    uint32_t max_len_log2;      /* run lengths are min(2^k, 31), k uniform in 0..max_len_log2 (<= 5) */
+    uint32_t reserved;          /* must be 0                                                         */
+    const uint32_t* init_schedule;  /* (device) [steps][W32], only for KVP_INIT_USER                */
+} kvp_anneal_params;
+
+/* Per-chain outcome. All fields are exact functions of (problem, params, chain). */
+typedef struct {
+    uint64_t best_ticks;    /* lowest T the chain visited                                          */
+    uint64_t best_move;     /* index of the first move after which T == best_ticks;
+                               UINT64_MAX when the initial state was never improved               */
+    uint64_t final_ticks;   /* T of the state after the last executed move                         */
+    uint64_t moves_done;    /* proposals executed (less than `moves` only after an early stop)     */
+    uint64_t n_accepted;    /* proposals that passed the Metropolis test (including no-op moves)   */
+    uint64_t n_changed;     /* accepted proposals that changed at least one placement bit          */
+    uint64_t n_infeasible;  /* flip proposals rejected because they would violate Eq. 5            */
+    uint64_t traj_hash;     /* running hash over (move index, T after move) of every changing move */
+} kvp_chain_result;
+
+typedef struct {
+    uint64_t init_ticks;        /* T of the initial placement                                      */
+    uint64_t best_ticks;        /* the bound: min over chains                                      */
+    uint32_t best_chain;        /* lowest chain index that reached it                              */
+    uint32_t levels;            /* number of levels actually used                                  */
+    uint64_t best_move;
+    uint64_t moves_total;       /* sum of moves_done over chains                                   */
+    uint64_t calib_mean_delta;  /* mean positive delta of the calibration proposals (0 if temps given) */
+    double   temp0;             /* temperature of level 0 in ticks                                 */
+    uint64_t winner_hits, winner_accessed; /* sum_s hr and sum_s |A[s]| of the winner: HBM hit rate */
+    float    ms_init, ms_chains, ms_finish;   /* device time of the three phases (CUDA events)     */
+    uint32_t kernel_launches;   /* kernels this call launched                                      */
+    kvp_chain_result* per_chain; /* (host) [chains] or NULL                                        */
+} kvp_anneal_stats;
+
+/*
+ * kvp_accept_table -- the quantised Metropolis thresholds kvp_anneal uses.
+ * For level j with temperature C_j (ticks; values below 1 are raised to 1):
+ *   shift_j = smallest sh >= 0 with 1024 * 2^sh >= 23 * C_j,
+ *   table[j][q] = min(2^32 - 1, floor(2^32 * exp(-((q + 0.5) * 2^shift_j) / C_j))).
+ * An uphill move with delta > 0 is accepted iff q = delta >> shift_j < 1024 and
+ * the move's 32-bit uniform w satisfies w < table[j][q].
+ *   temps  (host) [levels]         table (host) [levels][1024]     shifts (host) [levels]
+ * Pure host arithmetic; no device work.
+ */
+int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint32_t* shifts);
+
+/*
+ * kvp_anneal -- run `chains` independent annealing chains, reduce to the best
+ * schedule found (the bound of Section III-B) and re-score it with kvp_eval.
+ *   best_schedule (device) [steps][W32] or NULL
+ *   best_ticks, best_seconds (host) or NULL
+ *   stats (host) or NULL; stats->per_chain must be NULL or a host array [chains]
+ * Synchronises `stream` before returning.
+ */
+int kvp_anneal(kvp_problem* p, const kvp_anneal_params* params, uint32_t* best_schedule,
+               uint64_t* best_ticks, double* best_seconds, kvp_anneal_stats* stats, void* stream);
+
+/*
+ * kvp_anneal_chain_state -- replay one chain for its first `upto_moves` proposals
+ * and return the schedule it then holds (trajectories are pure functions of
+ * (seed, chain, move index), so this reproduces any state kvp_anneal went through).
+ *   schedule (device) [steps][W32];  result (host) or NULL.
+ */
+int kvp_anneal_chain_state(kvp_problem* p, const kvp_anneal_params* params, uint32_t chain,
+                           uint64_t upto_moves, uint32_t* schedule, kvp_chain_result* result,
+                           void* stream);
+
+/*
+ * Synthetic access traces: the stand-in for recorded attention scores
+ * (Section IV-A) in the spirit of the synthesised low/high-variation traces of
+ * Section IV-B. Units are arranged as `groups` (layer, kv-head) pairs of
+ * `units_per_group` blocks; every step each group reads its `topk` most
+ * important blocks. Importance of unit u at step t is the integer (Q16.16)
+ *   score = x_t(u) + base[u],  x_0 = (sigma_q*e_0) >> 16,
+ *   x_t = (rho_q*x_{t-1} + c_q*e_t) >> 16  [+ burst_jump with probability burst_thr/2^32],
+ * where e_t is a unit-variance Irwin-Hall(8) variate built from the eight 16-bit
+ * halves of Philox4x32-10(counter = (u, t, 0, 3), key = seed):
+ *   e = ((sum of halves - 262140) * 80265) >> 16.
+ * Ties are broken towards the lower unit index.
+ */
+typedef struct {
+    uint32_t groups, units_per_group, steps, topk;
+    uint64_t seed;
+    int32_t  rho_q;       /* AR(1) coefficient * 2^16, 0..65536                      */
+    int32_t  c_q;         /* innovation scale * 2^16, 0..2^20                        */
+    int32_t  sigma_q;     /* std of x_0 * 2^16, 0..2^20                              */
+    int32_t  burst_jump;  /* Q16.16 jump added to x_t when a burst fires             */
+    uint32_t burst_thr;   /* burst probability * 2^32 (0 = no bursts)                */
+    uint32_t reserved;    /* must be 0                                               */
+    const int32_t* base;  /* (device) [groups*units_per_group] static log-importance, or NULL = 0;
+                             |base| <= 2^29                                          */
+} kvp_trace_params;
+
+/*
+ * kvp_trace_generate -- fill access_bitmaps (device) [steps][ceil(U/32)] with the
+ * top-k sets described above. Asynchronous on `stream`.
+ */
+int kvp_trace_generate(const kvp_trace_params* params, uint32_t* access_bitmaps, void* stream);
+
+/* Philox4x32-10 (Salmon et al., SC'11) on the host; exposed so that callers can
+ * reproduce which proposal a given (seed, chain, move) pair is. */
+void kvp_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
+
+const char* kvp_strerror(int code);
+/* Text of the last CUDA error seen by the calling thread ("" if none). */
+const char* kvp_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVP_H_ */

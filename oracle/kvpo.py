@@ -1,0 +1,242 @@
+"""ctypes front end of the CPU oracle (oracle/kvpo.c).
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: only the tests, the smoke check and the
+benchmark's CPU-baseline leg may import this module. It never touches the
+CUDA library, and the CUDA library never touches it.
+
+All arrays are numpy arrays on the host; bitmaps are uint32 [steps][ceil(units/32)].
+"""
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "kvpo.c")
+_LIB = os.path.join(_HERE, "libkvpo.so")
+_lib = None
+
+OK = 0
+TABLE_Q = 1024
+INIT_STATIC_FIRST, INIT_STATIC_FREQ, INIT_USER = 0, 1, 2
+MIG_HBM, MIG_EXT, MIG_PAPER = 1, 2, 3
+
+
+def build(force=False):
+    """Compile kvpo.c into libkvpo.so with gcc (plain -O2, no contraction of a*b+c)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-ffp-contract=off", "-fPIC", "-shared",
+             "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+class AnnealParams(C.Structure):
+    _fields_ = [
+        ("chains", C.c_uint32), ("levels", C.c_uint32),
+        ("moves", C.c_uint64), ("seed", C.c_uint64),
+        ("p0", C.c_double), ("alpha", C.c_double),
+        ("temps", C.POINTER(C.c_double)),
+        ("early_stop_permille", C.c_uint32), ("early_stop_from_level", C.c_uint32),
+        ("init_mode", C.c_uint32), ("p_swap_256", C.c_uint32),
+        ("max_len_log2", C.c_uint32), ("reserved", C.c_uint32),
+        ("init_schedule", C.POINTER(C.c_uint32)),
+    ]
+
+
+class ChainResult(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in (
+        "best_ticks", "best_move", "final_ticks", "moves_done",
+        "n_accepted", "n_changed", "n_infeasible", "traj_hash")]
+
+    def astuple(self):
+        return tuple(int(getattr(self, n)) for n, _ in self._fields_)
+
+
+class TraceParams(C.Structure):
+    _fields_ = [
+        ("groups", C.c_uint32), ("units_per_group", C.c_uint32), ("steps", C.c_uint32), ("topk", C.c_uint32),
+        ("seed", C.c_uint64),
+        ("rho_q", C.c_int32), ("c_q", C.c_int32), ("sigma_q", C.c_int32), ("burst_jump", C.c_int32),
+        ("burst_thr", C.c_uint32), ("reserved", C.c_uint32),
+        ("base", C.POINTER(C.c_int32)),
+    ]
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = C.CDLL(_LIB)
+        _lib.kvpo_get_weights.restype = C.c_double
+    return _lib
+
+
+def _u32p(a):
+    return a.ctypes.data_as(C.POINTER(C.c_uint32)) if a is not None else None
+
+
+def _u64p(a):
+    return a.ctypes.data_as(C.POINTER(C.c_uint64)) if a is not None else None
+
+
+def _chk(rc, what):
+    if rc != OK:
+        raise RuntimeError(f"oracle {what} failed with code {rc}")
+
+
+def philox(ctr, key):
+    c = (C.c_uint32 * 4)(*ctr)
+    k = (C.c_uint32 * 2)(*key)
+    o = (C.c_uint32 * 4)()
+    lib().kvpo_philox4x32_10(c, k, o)
+    return tuple(int(x) for x in o)
+
+
+def tick_weights(bw_hbm, bw_link, bw_dram):
+    """-> dict(kh, kk, kd, ke, lcm, gcd)"""
+    o = (C.c_uint64 * 6)()
+    _chk(lib().kvpo_tick_weights(C.c_uint64(bw_hbm), C.c_uint64(bw_link), C.c_uint64(bw_dram), o), "tick_weights")
+    return dict(zip(("kh", "kk", "kd", "ke", "lcm", "gcd"), (int(x) for x in o)))
+
+
+class Problem:
+    def __init__(self, units, bytes_per_unit, steps, access, cap, bw_hbm, bw_link, bw_dram,
+                 mig_flags=MIG_PAPER, hw=None, ew=None):
+        access = np.ascontiguousarray(access, dtype=np.uint32)
+        self.units, self.steps, self.cap = int(units), int(steps), int(cap)
+        self.w32 = (self.units + 31) // 32
+        assert access.size == self.steps * self.w32
+        self.access = access.reshape(self.steps, self.w32)
+        hw = None if hw is None else np.ascontiguousarray(hw, dtype=np.uint32)
+        ew = None if ew is None else np.ascontiguousarray(ew, dtype=np.uint32)
+        self._h = C.c_void_p()
+        rc = lib().kvpo_create(C.byref(self._h), C.c_uint32(units), C.c_uint64(bytes_per_unit), C.c_uint32(steps),
+                               _u32p(self.access), C.c_uint32(cap), C.c_uint64(bw_hbm), C.c_uint64(bw_link),
+                               C.c_uint64(bw_dram), C.c_uint32(mig_flags), _u32p(hw), _u32p(ew))
+        _chk(rc, "create")
+        o = (C.c_uint64 * 6)()
+        self.seconds_per_tick = float(lib().kvpo_get_weights(self._h, o))
+        self.weights = dict(zip(("kh", "kk", "kd", "ke", "lcm", "gcd"), (int(x) for x in o)))
+
+    def __del__(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            lib().kvpo_destroy(self._h)
+            self._h = None
+
+    def _sched(self, P):
+        P = np.ascontiguousarray(P, dtype=np.uint32)
+        assert P.size == self.steps * self.w32
+        return P
+
+    def eval(self, P):
+        """-> dict(step_ticks, total_ticks, step_seconds, total_seconds, bad_step, counts[S][4])"""
+        P = self._sched(P)
+        st = np.zeros(self.steps, np.uint64)
+        ss = np.zeros(self.steps, np.float64)
+        cnt = np.zeros((self.steps, 4), np.uint32)
+        tt = C.c_uint64(); ts = C.c_double(); bad = C.c_int32()
+        _chk(lib().kvpo_eval(self._h, _u32p(P), _u64p(st), C.byref(tt), ss.ctypes.data_as(C.POINTER(C.c_double)),
+                             C.byref(ts), C.byref(bad), _u32p(cnt)), "eval")
+        return dict(step_ticks=st, total_ticks=int(tt.value), step_seconds=ss, total_seconds=float(ts.value),
+                    bad_step=int(bad.value), counts=cnt)
+
+    def init_placement(self, mode):
+        P = np.zeros((self.steps, self.w32), np.uint32)
+        _chk(lib().kvpo_init_placement(self._h, C.c_uint32(mode), _u32p(P)), "init_placement")
+        return P
+
+    def make_params(self, chains, moves, seed=0, levels=64, p0=0.8, alpha=0.9, temps=None,
+                    early_stop_permille=0, early_stop_from_level=0, init_mode=INIT_STATIC_FREQ,
+                    p_swap_256=128, max_len_log2=5, init_schedule=None):
+        ap = AnnealParams()
+        ap.chains, ap.levels, ap.moves, ap.seed = chains, levels, moves, seed
+        ap.p0, ap.alpha = p0, alpha
+        keep = []
+        if temps is not None:
+            t = np.ascontiguousarray(temps, dtype=np.float64)
+            assert t.size == levels
+            keep.append(t)
+            ap.temps = t.ctypes.data_as(C.POINTER(C.c_double))
+        ap.early_stop_permille, ap.early_stop_from_level = early_stop_permille, early_stop_from_level
+        ap.init_mode, ap.p_swap_256, ap.max_len_log2 = init_mode, p_swap_256, max_len_log2
+        if init_schedule is not None:
+            s = self._sched(init_schedule)
+            keep.append(s)
+            ap.init_schedule = _u32p(s)
+        ap._keep = keep
+        return ap
+
+    def temps(self, ap):
+        """Temperature ladder the parameters imply -> (temps[levels], calibration mean delta)."""
+        if ap.temps:
+            return np.ctypeslib.as_array(ap.temps, shape=(ap.levels,)).copy(), 0
+        t = np.zeros(ap.levels, np.float64)
+        mean = C.c_uint64()
+        _chk(lib().kvpo_default_temps(self._h, C.byref(ap), t.ctypes.data_as(C.POINTER(C.c_double)), C.byref(mean)),
+             "default_temps")
+        return t, int(mean.value)
+
+    def anneal_chains(self, ap, chain_begin, chain_count, upto_moves=None, want_final=False, want_best=False,
+                      table=None, shifts=None):
+        """-> (list of ChainResult, final_states or None, best_states or None)"""
+        if table is None:
+            t, _ = self.temps(ap)
+            table, shifts = accept_table(t)
+        res = (ChainResult * chain_count)()
+        fin = np.zeros((chain_count, self.steps, self.w32), np.uint32) if want_final else None
+        bst = np.zeros((chain_count, self.steps, self.w32), np.uint32) if want_best else None
+        upto = ap.moves if upto_moves is None else upto_moves
+        _chk(lib().kvpo_anneal_chains(self._h, C.byref(ap), _u32p(table), _u32p(shifts), C.c_uint32(chain_begin),
+                                      C.c_uint32(chain_count), C.c_uint64(upto), res, _u32p(fin), _u32p(bst)),
+             "anneal_chains")
+        return list(res), fin, bst
+
+    def anneal(self, ap, table=None, shifts=None):
+        """-> dict(best_schedule, best_ticks, best_seconds, best_chain, per_chain)"""
+        if table is None:
+            t, _ = self.temps(ap)
+            table, shifts = accept_table(t)
+        res = (ChainResult * ap.chains)()
+        best = np.zeros((self.steps, self.w32), np.uint32)
+        bt = C.c_uint64(); bc = C.c_uint32()
+        _chk(lib().kvpo_anneal(self._h, C.byref(ap), _u32p(table), _u32p(shifts), _u32p(best), C.byref(bt),
+                               C.byref(bc), res), "anneal")
+        return dict(best_schedule=best, best_ticks=int(bt.value), best_seconds=int(bt.value) * self.seconds_per_tick,
+                    best_chain=int(bc.value), per_chain=list(res))
+
+    def check_total(self, P, ticks):
+        return lib().kvpo_check_total(self._h, _u32p(self._sched(P)), C.c_uint64(ticks)) == 0
+
+
+def accept_table(temps):
+    temps = np.ascontiguousarray(temps, dtype=np.float64)
+    levels = temps.size
+    table = np.zeros((levels, TABLE_Q), np.uint32)
+    shifts = np.zeros(levels, np.uint32)
+    _chk(lib().kvpo_accept_table(temps.ctypes.data_as(C.POINTER(C.c_double)), C.c_uint32(levels),
+                                 _u32p(table), _u32p(shifts)), "accept_table")
+    return table, shifts
+
+
+def trace_generate(groups, units_per_group, steps, topk, seed, rho_q, c_q, sigma_q, burst_jump=0, burst_thr=0,
+                   base=None, group_begin=0, group_count=None, want_scores=False):
+    """-> access [steps][W32] (and scores [steps][U] int32 when want_scores)."""
+    tp = TraceParams()
+    tp.groups, tp.units_per_group, tp.steps, tp.topk, tp.seed = groups, units_per_group, steps, topk, seed
+    tp.rho_q, tp.c_q, tp.sigma_q, tp.burst_jump, tp.burst_thr = rho_q, c_q, sigma_q, burst_jump, burst_thr
+    if base is not None:
+        base = np.ascontiguousarray(base, dtype=np.int32)
+        assert base.size == groups * units_per_group
+        tp.base = base.ctypes.data_as(C.POINTER(C.c_int32))
+    U = groups * units_per_group
+    w32 = (U + 31) // 32
+    acc = np.zeros((steps, w32), np.uint32)
+    sc = np.zeros((steps, U), np.int32) if want_scores else None
+    if group_count is None:
+        group_count = groups - group_begin
+    _chk(lib().kvpo_trace_generate(C.byref(tp), C.c_uint32(group_begin), C.c_uint32(group_count), _u32p(acc),
+                                   sc.ctypes.data_as(C.POINTER(C.c_int32)) if want_scores else None),
+         "trace_generate")
+    return (acc, sc) if want_scores else acc

@@ -1,0 +1,193 @@
+// Host side of the C ABI: problem construction, integer time base, acceptance table, error text.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <vector>
+
+#include "kvp_common.cuh"
+
+namespace kvp {
+
+static thread_local char g_cuda_err[256] = "";
+
+int set_cuda_error(cudaError_t e, const char* what)
+{
+    snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", what, cudaGetErrorString(e));
+    cudaGetLastError();  // clear the sticky-free error state
+    return e == cudaErrorMemoryAllocation ? KVP_ERR_NOMEM : KVP_ERR_CUDA;
+}
+
+static int grow(void** ptr, size_t* have, size_t want)
+{
+    if (*have >= want) return KVP_OK;
+    if (*ptr) { KVP_CUDA(cudaFree(*ptr)); *ptr = nullptr; *have = 0; }
+    size_t bytes = (want + 255) & ~(size_t)255;
+    KVP_CUDA(cudaMalloc(ptr, bytes));
+    *have = bytes;
+    return KVP_OK;
+}
+
+int ensure_scratch(kvp_problem* p, size_t bytes) { return grow(&p->d_scratch, &p->scratch_bytes, bytes); }
+int ensure_chain_ws(kvp_problem* p, size_t bytes) { return grow(&p->d_chain_ws, &p->chain_ws_bytes, bytes); }
+
+static uint64_t gcd_u64(uint64_t a, uint64_t b)
+{
+    while (b) { const uint64_t t = a % b; a = b; b = t; }
+    return a;
+}
+
+// kappa_x = L / (B_x / g): the smallest integers inversely proportional to the bandwidths of Eq. 3-4.
+static int derive_weights(const kvp_memsys* m, kvp_problem* p)
+{
+    const uint64_t g = gcd_u64(gcd_u64(m->bw_hbm, m->bw_link), m->bw_dram);
+    const uint64_t rh = m->bw_hbm / g, rk = m->bw_link / g, rd = m->bw_dram / g;
+    const uint64_t limit = 1ull << 40;
+    uint64_t L = rh / gcd_u64(rh, rk);
+    if (L > limit / rk) return KVP_ERR_RANGE;
+    L *= rk;
+    const uint64_t Lq = L / gcd_u64(L, rd);
+    if (Lq > limit / rd) return KVP_ERR_RANGE;
+    L = Lq * rd;
+    p->gcd = g; p->lcm = L;
+    p->kh = L / rh; p->kk = L / rk; p->kd = L / rd;
+    p->ke = p->kk > p->kd ? p->kk : p->kd;
+    return KVP_OK;
+}
+
+}  // namespace kvp
+
+using namespace kvp;
+
+extern "C" void kvp_destroy(kvp_problem* p)
+{
+    if (!p) return;
+    cudaSetDevice(p->device);
+    cudaFree(p->dA); cudaFree(p->dAcol); cudaFree(p->d_a); cudaFree(p->d_stepc); cudaFree(p->d_ucnt);
+    cudaFree(p->d_row_freq); cudaFree(p->d_scratch); cudaFree(p->d_chain_ws);
+    delete p;
+}
+
+static int create_impl(kvp_problem* p, const uint32_t* access, const uint32_t* hw, const uint32_t* ew, cudaStream_t st)
+{
+    const size_t nw = (size_t)p->S * p->W32;
+    KVP_CUDA(cudaMalloc(&p->dA, nw * 4));
+    KVP_CUDA(cudaMalloc(&p->dAcol, (size_t)p->U * p->S32 * 4));
+    KVP_CUDA(cudaMalloc(&p->d_a, (size_t)p->S * 4));
+    KVP_CUDA(cudaMalloc(&p->d_stepc, (size_t)p->S * sizeof(StepC)));
+    KVP_CUDA(cudaMalloc(&p->d_ucnt, (size_t)p->U * 4));
+    KVP_CUDA(cudaMalloc(&p->d_row_freq, (size_t)p->W32 * 4));
+    int rc = ensure_scratch(p, (size_t)(p->S + 1) * 16);
+    if (rc) return rc;
+    if ((rc = launch_clean_copy(access, p->dA, p->S, p->W32, p->pad_mask, st))) return rc;
+    if ((rc = launch_row_popcount(p->dA, p->S, p->W32, p->d_a, st))) return rc;
+    if ((rc = launch_bit_transpose(p->dA, p->S, p->W32, p->U, p->dAcol, p->S32, st))) return rc;
+    if ((rc = launch_unit_counts(p->dAcol, p->U, p->S32, p->d_ucnt, st))) return rc;
+    if ((rc = launch_static_freq_row(p, p->d_row_freq, st))) return rc;
+    std::vector<uint32_t> a(p->S);
+    KVP_CUDA(cudaMemcpyAsync(a.data(), p->d_a, (size_t)p->S * 4, cudaMemcpyDeviceToHost, st));
+    KVP_CUDA(cudaStreamSynchronize(st));
+    // Per-step constants of the cost function; everything must stay below 2^31 so that the
+    // annealer can work in 32-bit arithmetic.
+    uint64_t wmax = 0;
+    for (uint32_t s = 0; s < p->S; ++s) {
+        const uint64_t e = (uint64_t)(hw ? hw[s] : 0) + (ew ? ew[s] : 0);
+        if (e > wmax) wmax = e;
+    }
+    const uint64_t kmax = p->kh > p->ke ? p->kh : p->ke;
+    if (kmax * (2ull * p->U + wmax) >= (1ull << 31)) return KVP_ERR_RANGE;
+    std::vector<StepC> sc(p->S);
+    p->total_accessed = 0;
+    for (uint32_t s = 0; s < p->S; ++s) {
+        const uint64_t h = hw ? hw[s] : 0, e = ew ? ew[s] : 0;
+        sc[s] = make_uint4((uint32_t)(p->kh * h), (uint32_t)(p->kk * e), (uint32_t)(p->kd * e), (uint32_t)(p->ke * a[s]));
+        p->total_accessed += a[s];
+    }
+    KVP_CUDA(cudaMemcpyAsync(p->d_stepc, sc.data(), (size_t)p->S * sizeof(StepC), cudaMemcpyHostToDevice, st));
+    KVP_CUDA(cudaStreamSynchronize(st));
+    return KVP_OK;
+}
+
+extern "C" int kvp_create(kvp_problem** out, uint32_t units, uint64_t bytes_per_unit, uint32_t steps,
+                          const uint32_t* access_bitmaps, uint32_t hbm_capacity_units, const kvp_memsys* mem,
+                          const uint32_t* hw_units, const uint32_t* ew_units, void* stream)
+{
+    if (!out || !access_bitmaps || !mem || !units || !steps || !bytes_per_unit) return KVP_ERR_ARG;
+    if (hbm_capacity_units > units || mem->reserved || (mem->mig_flags & ~KVP_MIG_PAPER)) return KVP_ERR_ARG;
+    if (!mem->bw_hbm || !mem->bw_link || !mem->bw_dram) return KVP_ERR_ARG;
+    if (units >= (1u << 26) || steps > 32768) return KVP_ERR_RANGE;
+    int dev = 0;
+    KVP_CUDA(cudaGetDevice(&dev));
+    kvp_problem* p = new (std::nothrow) kvp_problem();
+    if (!p) return KVP_ERR_NOMEM;
+    memset(p, 0, sizeof *p);
+    p->device = dev;
+    p->U = units; p->S = steps; p->cap = hbm_capacity_units;
+    p->W32 = (units + 31) / 32; p->S32 = (steps + 31) / 32;
+    p->pad_mask = units % 32 ? (1u << (units % 32)) - 1u : 0xFFFFFFFFu;
+    p->tail_mask = steps % 32 ? (1u << (steps % 32)) - 1u : 0xFFFFFFFFu;
+    p->bytes_per_unit = bytes_per_unit;
+    p->mig_flags = mem->mig_flags;
+    int rc = derive_weights(mem, p);
+    if (rc) { delete p; return rc; }
+    p->spt = (double)bytes_per_unit / ((double)p->lcm * (double)p->gcd);
+    const uint32_t Fh = (mem->mig_flags & KVP_MIG_HBM) ? 1u : 0u, Fe = (mem->mig_flags & KVP_MIG_EXT) ? 1u : 0u;
+    if (p->kh >= (1ull << 31) || p->ke >= (1ull << 31)) { delete p; return KVP_ERR_RANGE; }
+    p->K.kh = (uint32_t)p->kh; p->K.ke = (uint32_t)p->ke;
+    p->K.khF = (uint32_t)p->kh * Fh; p->K.kkF = (uint32_t)p->kk * Fe; p->K.kdF = (uint32_t)p->kd * Fe;
+    rc = create_impl(p, access_bitmaps, hw_units, ew_units, static_cast<cudaStream_t>(stream));
+    if (rc) { kvp_destroy(p); return rc; }
+    *out = p;
+    return KVP_OK;
+}
+
+extern "C" int kvp_get_info(const kvp_problem* p, kvp_info* info)
+{
+    if (!p || !info) return KVP_ERR_ARG;
+    info->kappa_h = p->kh; info->kappa_k = p->kk; info->kappa_d = p->kd; info->kappa_e = p->ke;
+    info->lcm = p->lcm; info->gcd = p->gcd; info->seconds_per_tick = p->spt;
+    info->units = p->U; info->steps = p->S; info->words_per_row = p->W32; info->capacity = p->cap;
+    return KVP_OK;
+}
+
+extern "C" int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint32_t* shifts)
+{
+    if (!temps || !table || !shifts || !levels) return KVP_ERR_ARG;
+    for (uint32_t j = 0; j < levels; ++j) {
+        const double C = temps[j] >= 1.0 ? temps[j] : 1.0;     // also maps NaN to 1
+        uint32_t sh = 0;
+        while ((double)KVP_TABLE_Q * (double)(1ull << sh) < 23.0 * C)
+            if (++sh > 40) return KVP_ERR_RANGE;
+        shifts[j] = sh;
+        const double bin = (double)(1ull << sh);
+        for (uint32_t q = 0; q < KVP_TABLE_Q; ++q) {
+            const double x = ((double)q + 0.5) * bin;
+            const double thr = 4294967296.0 * exp(-x / C);
+            table[(size_t)j * KVP_TABLE_Q + q] = thr >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)thr;
+        }
+    }
+    return KVP_OK;
+}
+
+extern "C" void kvp_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    philox4x32_10(ctr[0], ctr[1], ctr[2], ctr[3], key[0], key[1], out);
+}
+
+extern "C" const char* kvp_strerror(int code)
+{
+    switch (code) {
+        case KVP_OK: return "ok";
+        case KVP_ERR_ARG: return "invalid argument";
+        case KVP_ERR_CAPACITY: return "schedule exceeds the HBM capacity (Eq. 5)";
+        case KVP_ERR_RANGE: return "size or weight outside the supported integer range";
+        case KVP_ERR_CUDA: return "CUDA runtime error";
+        case KVP_ERR_NOMEM: return "out of memory";
+        case KVP_ERR_TIMEOUT: return "device-side wait timed out";
+        case KVP_ERR_INTERNAL: return "internal self-check failed";
+        default: return "unknown error";
+    }
+}
+
+extern "C" const char* kvp_last_cuda_error(void) { return kvp::g_cuda_err; }

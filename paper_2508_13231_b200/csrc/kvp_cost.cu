@@ -1,0 +1,279 @@
+// Cost kernels: per-step cardinalities of a schedule (popc over mask AND placement words) and Eq. 1-5.
+//
+// The counting pass is the HBM-bound part: every word of A and of P is read once, P[s-1] is carried
+// in registers from the previous iteration. Two shapes:
+//   wide rows   (>= 17 vectors per row): a warp owns 32 consecutive 16-byte vectors of every row of a
+//               step chunk; a CTA of 8 warps therefore reads 4 KB contiguous per row and array.
+//   narrow rows (<= 16 vectors per row): a sub-warp group of LPR lanes owns whole rows, consecutive
+//               groups own consecutive rows, so a warp still reads contiguous memory.
+#include "kvp_common.cuh"
+
+namespace kvp {
+
+namespace {
+
+template <int VEC>
+__device__ __forceinline__ uint4 load_vec(const uint32_t* __restrict__ base, size_t row_words, uint32_t row, uint32_t cv)
+{
+    if (VEC == 4) {
+        return __ldg(reinterpret_cast<const uint4*>(base + (size_t)row * row_words) + cv);
+    } else {
+        return make_uint4(__ldg(base + (size_t)row * row_words + cv), 0u, 0u, 0u);
+    }
+}
+
+template <int VEC>
+__device__ __forceinline__ uint4 mask_last(uint4 v, uint32_t cv, uint32_t WV, uint32_t pad_mask)
+{
+    if (cv == WV - 1) {
+        if (VEC == 4) v.w &= pad_mask; else v.x &= pad_mask;
+    }
+    return v;
+}
+
+__device__ __forceinline__ uint32_t popc4(uint4 v) { return __popc(v.x) + __popc(v.y) + __popc(v.z) + __popc(v.w); }
+__device__ __forceinline__ uint4 and4(uint4 a, uint4 b) { return make_uint4(a.x & b.x, a.y & b.y, a.z & b.z, a.w & b.w); }
+__device__ __forceinline__ uint4 andn4(uint4 a, uint4 b) { return make_uint4(a.x & ~b.x, a.y & ~b.y, a.z & ~b.z, a.w & ~b.w); }
+
+// counts of one vector: x = hr | mi << 16, y = mo | occ << 16 (each at most 128)
+__device__ __forceinline__ uint2 vec_counts(uint4 a, uint4 p, uint4 prev)
+{
+    const uint32_t hr = popc4(and4(a, p));
+    const uint32_t mi = popc4(andn4(p, prev));
+    const uint32_t mo = popc4(andn4(prev, p));
+    const uint32_t occ = popc4(p);
+    return make_uint2(hr | (mi << 16), mo | (occ << 16));
+}
+
+constexpr int WIDE_WARPS = 8;
+
+template <int VEC>
+__global__ void __launch_bounds__(WIDE_WARPS * 32)
+count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ Ps, uint32_t S, uint32_t W32,
+                  uint32_t WV, uint32_t pad_mask, uint32_t SC, uint32_t* __restrict__ counts)
+{
+    extern __shared__ uint2 acc[];                       // [WIDE_WARPS][SC]
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cv = (blockIdx.x * WIDE_WARPS + warp) * 32 + lane;
+    const bool valid = cv < WV;
+    const uint32_t sb = blockIdx.y * SC;
+    const uint32_t se = min(S, sb + SC);
+    const uint32_t* __restrict__ P = Ps + (size_t)blockIdx.z * S * W32;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    uint4 prev = valid ? mask_last<VEC>(load_vec<VEC>(P, W32, sb ? sb - 1 : 0, cv), cv, WV, pad_mask) : zero;
+#pragma unroll 4
+    for (uint32_t s = sb; s < se; ++s) {
+        const uint4 a = valid ? load_vec<VEC>(A, W32, s, cv) : zero;
+        const uint4 p = valid ? mask_last<VEC>(load_vec<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
+        uint2 c = vec_counts(a, p, prev);
+        c.x = __reduce_add_sync(0xFFFFFFFFu, c.x);       // 16-bit fields: 32 lanes * 128 < 65536
+        c.y = __reduce_add_sync(0xFFFFFFFFu, c.y);
+        if (lane == 0) acc[warp * SC + (s - sb)] = c;
+        prev = p;
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < se - sb; i += blockDim.x) {
+        uint32_t hr = 0, mi = 0, mo = 0, occ = 0;
+#pragma unroll
+        for (int w = 0; w < WIDE_WARPS; ++w) {
+            const uint2 c = acc[w * SC + i];
+            hr += c.x & 0xFFFFu; mi += c.x >> 16; mo += c.y & 0xFFFFu; occ += c.y >> 16;
+        }
+        uint32_t* dst = counts + ((size_t)blockIdx.z * S + sb + i) * 4;
+        if (hr) atomicAdd(dst + 0, hr);
+        if (mi) atomicAdd(dst + 1, mi);
+        if (mo) atomicAdd(dst + 2, mo);
+        if (occ) atomicAdd(dst + 3, occ);
+    }
+}
+
+constexpr int NARROW_ITERS = 8;
+
+template <int VEC, int LPR>
+__global__ void __launch_bounds__(256)
+count_narrow_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ Ps, uint32_t S, uint32_t W32,
+                    uint32_t WV, uint32_t pad_mask, uint32_t* __restrict__ counts)
+{
+    constexpr uint32_t GROUPS = 256 / LPR;               // rows in flight per CTA
+    const uint32_t g = threadIdx.x / LPR, cv = threadIdx.x % LPR;
+    const bool col_ok = cv < WV;
+    const uint32_t* __restrict__ P = Ps + (size_t)blockIdx.y * S * W32;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 2
+    for (int it = 0; it < NARROW_ITERS; ++it) {
+        const uint32_t s = (blockIdx.x * NARROW_ITERS + it) * GROUPS + g;
+        const bool ok = col_ok && s < S;
+        const uint4 a = ok ? load_vec<VEC>(A, W32, s, cv) : zero;
+        const uint4 p = ok ? mask_last<VEC>(load_vec<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
+        const uint4 q = ok ? mask_last<VEC>(load_vec<VEC>(P, W32, s ? s - 1 : 0, cv), cv, WV, pad_mask) : zero;
+        uint2 c = vec_counts(a, p, q);
+#pragma unroll
+        for (int off = LPR / 2; off > 0; off >>= 1) {
+            c.x += __shfl_xor_sync(0xFFFFFFFFu, c.x, off);
+            c.y += __shfl_xor_sync(0xFFFFFFFFu, c.y, off);
+        }
+        if (cv == 0 && s < S)
+            reinterpret_cast<uint4*>(counts)[(size_t)blockIdx.y * S + s] =
+                make_uint4(c.x & 0xFFFFu, c.x >> 16, c.y & 0xFFFFu, c.y >> 16);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+finish_kernel(const uint4* __restrict__ counts, const StepC* __restrict__ stepc, CostK K, uint32_t S, uint32_t cap,
+              double spt, uint64_t* __restrict__ step_ticks, uint64_t* __restrict__ total_ticks,
+              double* __restrict__ step_seconds, double* __restrict__ total_seconds, int32_t* __restrict__ bad_step,
+              uint64_t* __restrict__ hits)
+{
+    __shared__ uint64_t s_sum[8], s_hit[8];
+    __shared__ uint32_t s_bad[8];
+    const uint32_t i = blockIdx.x;
+    uint64_t sum = 0, hit = 0;
+    uint32_t bad = 0xFFFFFFFFu;
+    for (uint32_t s = threadIdx.x; s < S; s += blockDim.x) {
+        const uint4 c = counts[(size_t)i * S + s];
+        const uint32_t f = step_cost(c.x, c.y, c.z, __ldg(&stepc[s]), K);
+        if (step_ticks) step_ticks[(size_t)i * S + s] = f;
+        if (step_seconds) step_seconds[(size_t)i * S + s] = (double)f * spt;
+        sum += f;
+        hit += c.x;
+        if (c.w > cap) bad = min(bad, s);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, off);
+        hit += __shfl_xor_sync(0xFFFFFFFFu, hit, off);
+        bad = min(bad, __shfl_xor_sync(0xFFFFFFFFu, bad, off));
+    }
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { s_sum[warp] = sum; s_hit[warp] = hit; s_bad[warp] = bad; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) { sum += s_sum[w]; hit += s_hit[w]; bad = min(bad, s_bad[w]); }
+        if (total_ticks) total_ticks[i] = sum;
+        if (total_seconds) total_seconds[i] = (double)sum * spt;
+        if (bad_step) bad_step[i] = bad == 0xFFFFFFFFu ? -1 : (int32_t)bad;
+        if (hits) hits[i] = hit;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+row_popcount_kernel(const uint32_t* __restrict__ rows, uint32_t S, uint32_t W32, uint32_t* __restrict__ out)
+{
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= S) return;
+    uint32_t c = 0;
+    for (uint32_t w = lane; w < W32; w += 32) c += __popc(__ldg(rows + (size_t)warp * W32 + w));
+    c = __reduce_add_sync(0xFFFFFFFFu, c);
+    if (lane == 0) out[warp] = c;
+}
+
+template <int VEC>
+int launch_narrow(uint32_t WV, dim3 grid_rows, uint32_t n, const uint32_t* A, const uint32_t* P, uint32_t S, uint32_t W32,
+                  uint32_t pad_mask, uint32_t* counts, cudaStream_t st)
+{
+    (void)grid_rows;
+#define KVP_NARROW(LPR)                                                                          \
+    {                                                                                            \
+        const uint32_t rows_per_cta = (256 / LPR) * NARROW_ITERS;                                \
+        dim3 grid((S + rows_per_cta - 1) / rows_per_cta, n);                                     \
+        count_narrow_kernel<VEC, LPR><<<grid, 256, 0, st>>>(A, P, S, W32, WV, pad_mask, counts); \
+    }
+    if (WV <= 1) KVP_NARROW(1)
+    else if (WV <= 2) KVP_NARROW(2)
+    else if (WV <= 4) KVP_NARROW(4)
+    else if (WV <= 8) KVP_NARROW(8)
+    else KVP_NARROW(16)
+#undef KVP_NARROW
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+}  // namespace
+
+int launch_row_popcount(const uint32_t* rows, uint32_t S, uint32_t W32, uint32_t* out, cudaStream_t st)
+{
+    row_popcount_kernel<<<(S + 7) / 8, 256, 0, st>>>(rows, S, W32, out);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+// counts [n][S][4] = {hr, mi, mo, occ}
+int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, uint32_t* counts, cudaStream_t st,
+                  uint32_t* launches)
+{
+    const bool vec4 = (p->W32 % 4 == 0) && ((reinterpret_cast<uintptr_t>(schedules) & 15) == 0);
+    const uint32_t WV = vec4 ? p->W32 / 4 : p->W32;
+    if (WV <= 16) {
+        if (launches) *launches += 1;
+        return vec4 ? launch_narrow<4>(WV, dim3(), n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, st)
+                    : launch_narrow<1>(WV, dim3(), n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, st);
+    }
+    KVP_CUDA(cudaMemsetAsync(counts, 0, (size_t)n * p->S * 16, st));
+    const uint32_t col_ctas = (WV + WIDE_WARPS * 32 - 1) / (WIDE_WARPS * 32);
+    // Split the steps so that the grid fills the 148 SMs a few times over; every chunk re-reads one halo row.
+    uint32_t SC = p->S;
+    while (SC > 8 && (uint64_t)col_ctas * ((p->S + SC - 1) / SC) * n < 148u * 6u) SC = (SC + 1) / 2;
+    if (SC > 512) SC = 512;
+    dim3 grid(col_ctas, (p->S + SC - 1) / SC, n);
+    const size_t smem = (size_t)WIDE_WARPS * SC * sizeof(uint2);
+    if (vec4)
+        count_wide_kernel<4><<<grid, WIDE_WARPS * 32, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts);
+    else
+        count_wide_kernel<1><<<grid, WIDE_WARPS * 32, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts);
+    KVP_CUDA(cudaGetLastError());
+    if (launches) *launches += 1;
+    return KVP_OK;
+}
+
+int launch_finish(const kvp_problem* p, const uint32_t* counts, uint32_t n, uint64_t* step_ticks, uint64_t* total_ticks,
+                  double* step_seconds, double* total_seconds, int32_t* bad_step, uint64_t* hits, cudaStream_t st)
+{
+    finish_kernel<<<n, 256, 0, st>>>(reinterpret_cast<const uint4*>(counts), p->d_stepc, p->K, p->S, p->cap, p->spt,
+                                      step_ticks, total_ticks, step_seconds, total_seconds, bad_step, hits);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+}  // namespace kvp
+
+// The schedule index is a grid dimension limited to 65535: larger batches go in slices.
+static const uint32_t kBatchSlice = 32768;
+
+extern "C" int kvp_eval_counts(kvp_problem* p, const uint32_t* schedules, uint32_t n, uint32_t* counts, void* stream)
+{
+    if (!p || !schedules || !counts || !n) return KVP_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(counts) & 15) != 0) return KVP_ERR_ARG;
+    KVP_CUDA(cudaSetDevice(p->device));
+    const size_t sched_words = (size_t)p->S * p->W32;
+    for (uint32_t i = 0; i < n; i += kBatchSlice) {
+        const uint32_t m = n - i < kBatchSlice ? n - i : kBatchSlice;
+        int rc = kvp::launch_counts(p, schedules + i * sched_words, m, counts + (size_t)i * p->S * 4,
+                                    static_cast<cudaStream_t>(stream), nullptr);
+        if (rc) return rc;
+    }
+    return KVP_OK;
+}
+
+extern "C" int kvp_eval(kvp_problem* p, const uint32_t* schedules, uint32_t n, uint64_t* step_ticks, uint64_t* total_ticks,
+                        double* step_seconds, double* total_seconds, int32_t* bad_step, void* stream)
+{
+    if (!p || !schedules || !total_ticks || !n) return KVP_ERR_ARG;
+    KVP_CUDA(cudaSetDevice(p->device));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t slice = n < kBatchSlice ? n : kBatchSlice;
+    int rc = kvp::ensure_scratch(p, (size_t)slice * p->S * 16);
+    if (rc) return rc;
+    uint32_t* counts = static_cast<uint32_t*>(p->d_scratch);
+    const size_t sched_words = (size_t)p->S * p->W32;
+    for (uint32_t i = 0; i < n; i += kBatchSlice) {
+        const uint32_t m = n - i < kBatchSlice ? n - i : kBatchSlice;
+        if ((rc = kvp::launch_counts(p, schedules + i * sched_words, m, counts, st, nullptr))) return rc;
+        const size_t so = (size_t)i * p->S;
+        if ((rc = kvp::launch_finish(p, counts, m, step_ticks ? step_ticks + so : nullptr, total_ticks + i,
+                                     step_seconds ? step_seconds + so : nullptr,
+                                     total_seconds ? total_seconds + i : nullptr, bad_step ? bad_step + i : nullptr,
+                                     nullptr, st)))
+            return rc;
+    }
+    return KVP_OK;
+}

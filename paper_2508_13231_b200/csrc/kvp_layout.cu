@@ -1,0 +1,199 @@
+// Layout kernels: bit-matrix transposes between the step-major API layout and the time-packed layout
+// the annealer works on, pad-bit cleaning, per-unit access counts and the static initial placements.
+#include "kvp_common.cuh"
+
+namespace kvp {
+
+namespace {
+
+// in: [rows][in_words] words, bit c of row r = bit (c & 31) of in[r][c >> 5].
+// out: [cols][out_words], bit r of row c. Bits beyond `rows` in the last out word are 0.
+// One CTA transposes a tile of 32 rows x 32 words (1024 columns); warp w owns word column w.
+__global__ void __launch_bounds__(1024)
+bit_transpose_kernel(const uint32_t* __restrict__ in, uint32_t rows, uint32_t in_words, uint32_t cols,
+                     uint32_t* __restrict__ out, uint32_t out_words)
+{
+    __shared__ uint32_t tile[32][33];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t r0 = blockIdx.x * 32, w0 = blockIdx.y * 32;   // row blocks can be millions: they go in x
+    // coalesced load: warp `warp` reads row r0 + warp, lanes read consecutive words
+    {
+        const uint32_t r = r0 + warp, w = w0 + lane;
+        tile[warp][lane] = (r < rows && w < in_words) ? __ldg(in + (size_t)r * in_words + w) : 0u;
+    }
+    __syncthreads();
+    // warp `warp` now transposes word column w0 + warp: lane l holds row r0 + l
+    const uint32_t word = tile[lane][warp];
+    uint32_t mine = 0;
+#pragma unroll
+    for (int b = 0; b < 32; ++b) {
+        const uint32_t col_bits = __ballot_sync(0xFFFFFFFFu, (word >> b) & 1u);
+        if (lane == (uint32_t)b) mine = col_bits;
+    }
+    const uint32_t c = (w0 + warp) * 32 + lane;
+    if (c < cols) out[(size_t)c * out_words + blockIdx.x] = mine;
+}
+
+__global__ void clean_copy_kernel(const uint32_t* __restrict__ in, uint32_t* __restrict__ out, size_t total,
+                                  uint32_t W32, uint32_t pad_mask)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        uint32_t v = in[i];
+        if (i % W32 == W32 - 1) v &= pad_mask;
+        out[i] = v;
+    }
+}
+
+__global__ void unit_counts_kernel(const uint32_t* __restrict__ Acol, uint32_t U, uint32_t S32, uint32_t* __restrict__ ucnt)
+{
+    const uint32_t u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= U) return;
+    uint32_t c = 0;
+    for (uint32_t j = 0; j < S32; ++j) c += __popc(__ldg(Acol + (size_t)u * S32 + j));
+    ucnt[u] = c;
+}
+
+__global__ void histogram_kernel(const uint32_t* __restrict__ ucnt, uint32_t U, uint32_t* __restrict__ hist)
+{
+    const uint32_t u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u < U) atomicAdd(hist + ucnt[u], 1u);
+}
+
+// The `cap` most accessed units, ties to the lower index. One CTA: find the count threshold from the
+// histogram, then walk the units in index order with a running count of the ties already taken.
+// sel = {threshold count, number of ties to take}.
+__global__ void __launch_bounds__(1024)
+static_freq_kernel(const uint32_t* __restrict__ ucnt, const uint32_t* __restrict__ hist, uint32_t U, uint32_t S,
+                   uint32_t cap, uint32_t* __restrict__ row, uint32_t W32)
+{
+    __shared__ uint32_t s_thr, s_take, s_base;
+    __shared__ uint32_t s_warp[32];
+    if (threadIdx.x == 0) {
+        uint32_t above = 0, thr = S + 1, take = 0;
+        // counts run 0..S; descend until the capacity is reached
+        for (int64_t c = S; c >= 0; --c) {
+            const uint32_t h = hist[c];
+            if (above + h >= cap) { thr = (uint32_t)c; take = cap - above; break; }
+            above += h;
+        }
+        if (cap == 0) { thr = S + 1; take = 0; }
+        s_thr = thr; s_take = take; s_base = 0;
+    }
+    __syncthreads();
+    const uint32_t thr = s_thr, take = s_take;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t Upad = W32 * 32;
+    for (uint32_t u0 = 0; u0 < Upad; u0 += 1024) {
+        const uint32_t u = u0 + threadIdx.x;
+        const uint32_t c = u < U ? ucnt[u] : 0xFFFFFFFFu;
+        const bool tie = u < U && c == thr;
+        const uint32_t tie_bits = __ballot_sync(0xFFFFFFFFu, tie);
+        if (lane == 0) s_warp[warp] = __popc(tie_bits);
+        __syncthreads();
+        uint32_t before = s_base;
+        for (uint32_t w = 0; w < warp; ++w) before += s_warp[w];
+        before += __popc(tie_bits & ((1u << lane) - 1u));
+        const bool pick = u < U && (c > thr || (tie && before < take));
+        const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
+        if (lane == 0 && u < Upad) row[u >> 5] = bits;
+        __syncthreads();
+        if (threadIdx.x == 0) { uint32_t t = 0; for (int w = 0; w < 32; ++w) t += s_warp[w]; s_base += t; }
+        __syncthreads();
+    }
+}
+
+__global__ void static_first_kernel(uint32_t* __restrict__ row, uint32_t W32, uint32_t cap)
+{
+    const uint32_t w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (w >= W32) return;
+    const uint32_t lo = w * 32;
+    row[w] = cap >= lo + 32 ? 0xFFFFFFFFu : (cap > lo ? (1u << (cap - lo)) - 1u : 0u);
+}
+
+__global__ void broadcast_row_kernel(const uint32_t* __restrict__ row, uint32_t W32, size_t total, uint32_t* __restrict__ sched)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+        sched[i] = __ldg(row + i % W32);
+}
+
+// time-packed columns of a schedule whose every row equals `row`
+__global__ void row_to_columns_kernel(const uint32_t* __restrict__ row, uint32_t U, uint32_t S, uint32_t S32,
+                                      uint32_t* __restrict__ Pcol)
+{
+    const size_t total = (size_t)U * S32;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const uint32_t u = (uint32_t)(i / S32), j = (uint32_t)(i % S32);
+        const uint32_t on = (__ldg(row + (u >> 5)) >> (u & 31)) & 1u;
+        const uint32_t valid = (j + 1) * 32 <= S ? 0xFFFFFFFFu : ((1u << (S - j * 32)) - 1u);
+        Pcol[i] = on ? valid : 0u;
+    }
+}
+
+inline uint32_t grid_for(size_t total, uint32_t block)
+{
+    size_t g = (total + block - 1) / block;
+    return (uint32_t)(g > 148 * 16 ? 148 * 16 : (g ? g : 1));
+}
+
+}  // namespace
+
+int launch_bit_transpose(const uint32_t* in, uint32_t rows, uint32_t in_words, uint32_t cols, uint32_t* out,
+                         uint32_t out_words, cudaStream_t st)
+{
+    dim3 grid((rows + 31) / 32, (in_words + 31) / 32);
+    bit_transpose_kernel<<<grid, 1024, 0, st>>>(in, rows, in_words, cols, out, out_words);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_clean_copy(const uint32_t* in, uint32_t* out, uint32_t S, uint32_t W32, uint32_t pad_mask, cudaStream_t st)
+{
+    const size_t total = (size_t)S * W32;
+    clean_copy_kernel<<<grid_for(total, 256), 256, 0, st>>>(in, out, total, W32, pad_mask);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_unit_counts(const uint32_t* Acol, uint32_t U, uint32_t S32, uint32_t* ucnt, cudaStream_t st)
+{
+    unit_counts_kernel<<<(U + 255) / 256, 256, 0, st>>>(Acol, U, S32, ucnt);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+// needs (S + 1) * 4 bytes of zeroed scratch for the histogram; uses p->d_scratch
+int launch_static_freq_row(const kvp_problem* p, uint32_t* row, cudaStream_t st)
+{
+    uint32_t* hist = static_cast<uint32_t*>(p->d_scratch);
+    KVP_CUDA(cudaMemsetAsync(hist, 0, (size_t)(p->S + 1) * 4, st));
+    histogram_kernel<<<(p->U + 255) / 256, 256, 0, st>>>(p->d_ucnt, p->U, hist);
+    KVP_CUDA(cudaGetLastError());
+    static_freq_kernel<<<1, 1024, 0, st>>>(p->d_ucnt, hist, p->U, p->S, p->cap, row, p->W32);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_static_first_row(const kvp_problem* p, uint32_t* row, cudaStream_t st)
+{
+    static_first_kernel<<<(p->W32 + 255) / 256, 256, 0, st>>>(row, p->W32, p->cap);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_broadcast_row(const uint32_t* row, uint32_t S, uint32_t W32, uint32_t* sched, cudaStream_t st)
+{
+    const size_t total = (size_t)S * W32;
+    broadcast_row_kernel<<<grid_for(total, 256), 256, 0, st>>>(row, W32, total, sched);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_row_to_columns(const uint32_t* row, uint32_t U, uint32_t S, uint32_t S32, uint32_t* Pcol, cudaStream_t st)
+{
+    const size_t total = (size_t)U * S32;
+    row_to_columns_kernel<<<grid_for(total, 256), 256, 0, st>>>(row, U, S, S32, Pcol);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+}  // namespace kvp

@@ -1,0 +1,179 @@
+// Trace kernel: synthetic importance per unit and step, top-k per (layer, kv-head) group, packed into uint32
+// bitmaps. One CTA per group walks the steps in order (the AR(1) recurrence is sequential in time); the
+// importance state of a unit lives in a register of the thread that owns it. The k-th largest score of a step
+// is found by a 32-round bitwise binary search with block-wide counts, ties go to the lower unit index.
+#include "kvp_common.cuh"
+
+namespace kvp {
+
+namespace {
+
+struct TraceK {
+    uint32_t groups, n, steps, topk, W32;
+    uint32_t seed_lo, seed_hi;
+    int32_t rho_q, c_q, sigma_q, burst_jump;
+    uint32_t burst_thr;
+    const int32_t* base;
+    uint32_t* out;
+    int aligned;             // n % 32 == 0: whole output words belong to one group
+};
+
+__device__ __forceinline__ int64_t noise_q16(uint32_t seed_lo, uint32_t seed_hi, uint32_t u, uint32_t t)
+{
+    uint32_t r[4];
+    philox4x32_10(u, t, 0u, TAG_NOISE, seed_lo, seed_hi, r);
+    int64_t sum = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) sum += (int64_t)(r[i] & 0xFFFFu) + (int64_t)(r[i] >> 16);
+    return ((sum - 262140) * 80265) >> 16;     // Irwin-Hall(8), unit variance in Q16.16 (arithmetic shift = floor)
+}
+
+// Sum of a per-thread value over the CTA; every thread gets the result. slot: one of 32 shared counters.
+__device__ __forceinline__ uint32_t block_sum(uint32_t v, uint32_t* slot)
+{
+    v = __reduce_add_sync(0xFFFFFFFFu, v);
+    if ((threadIdx.x & 31) == 0 && v) atomicAdd(slot, v);
+    __syncthreads();
+    return *slot;
+}
+
+template <int UPT>
+__global__ void __launch_bounds__(1024)
+trace_kernel(const TraceK k)
+{
+    __shared__ uint32_t s_cnt[36];           // 32 search rounds + 2 extra counts
+    __shared__ uint32_t s_warp[32];
+    __shared__ uint32_t s_run;
+    const uint32_t g = blockIdx.x, T = blockDim.x, tid = threadIdx.x;
+    const uint32_t lane = tid & 31, warp = tid >> 5;
+    const uint32_t gbase = g * k.n;
+    int32_t x[UPT], b[UPT];
+#pragma unroll
+    for (int j = 0; j < UPT; ++j) {
+        const uint32_t i = j * T + tid;
+        x[j] = 0;
+        b[j] = (i < k.n && k.base) ? __ldg(k.base + gbase + i) : 0;
+    }
+    for (uint32_t t = 0; t < k.steps; ++t) {
+        for (uint32_t i = tid; i < 36; i += T) s_cnt[i] = 0;
+        uint32_t key[UPT];
+#pragma unroll
+        for (int j = 0; j < UPT; ++j) {
+            const uint32_t i = j * T + tid;
+            key[j] = 0;
+            if (i < k.n) {
+                const uint32_t u = gbase + i;
+                const int64_t e = noise_q16(k.seed_lo, k.seed_hi, u, t);
+                int64_t xn = t == 0 ? ((int64_t)k.sigma_q * e) >> 16
+                                    : ((int64_t)k.rho_q * (int64_t)x[j] + (int64_t)k.c_q * e) >> 16;
+                if (k.burst_thr) {
+                    uint32_t r[4];
+                    philox4x32_10(u, t, 0u, TAG_BURST, k.seed_lo, k.seed_hi, r);
+                    if (r[0] < k.burst_thr) xn += k.burst_jump;
+                }
+                x[j] = (int32_t)xn;
+                key[j] = (uint32_t)(x[j] + b[j]) ^ 0x80000000u;       // order-preserving map int32 -> uint32
+            }
+        }
+        __syncthreads();
+        // largest K with |{key >= K}| >= topk, bit by bit from the top
+        uint32_t K = 0;
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t cand = K | (1u << bit);
+            uint32_t c = 0;
+#pragma unroll
+            for (int j = 0; j < UPT; ++j) c += (j * T + tid < k.n && key[j] >= cand) ? 1u : 0u;
+            if (block_sum(c, &s_cnt[31 - bit]) >= k.topk) K = cand;
+        }
+        uint32_t cg = 0, ce = 0;
+#pragma unroll
+        for (int j = 0; j < UPT; ++j) {
+            const bool ok = j * T + tid < k.n;
+            cg += (ok && key[j] > K) ? 1u : 0u;
+            ce += (ok && key[j] == K) ? 1u : 0u;
+        }
+        const uint32_t above = block_sum(cg, &s_cnt[32]);
+        const uint32_t equal = block_sum(ce, &s_cnt[33]);
+        const uint32_t take = k.topk - above;                // ties to admit, lowest unit index first
+        const bool rank_ties = equal != take;
+        if (tid == 0) s_run = 0;
+        __syncthreads();
+        uint32_t* row = k.out + (size_t)t * k.W32;
+#pragma unroll
+        for (int j = 0; j < UPT; ++j) {
+            const uint32_t i = j * T + tid;
+            const bool ok = i < k.n;
+            const bool tie = ok && key[j] == K;
+            bool pick = ok && key[j] > K;
+            if (!rank_ties) {
+                pick = pick || tie;
+            } else {
+                // units of round j are consecutive over the CTA, so index order = (round, thread) order
+                const uint32_t tb = __ballot_sync(0xFFFFFFFFu, tie);
+                if (lane == 0) s_warp[warp] = __popc(tb);
+                __syncthreads();
+                uint32_t before = s_run;
+                for (uint32_t w = 0; w < warp; ++w) before += s_warp[w];
+                before += __popc(tb & ((1u << lane) - 1u));
+                pick = pick || (tie && before < take);
+                __syncthreads();
+                if (tid == 0) { uint32_t s = 0; for (uint32_t w = 0; w < (T >> 5); ++w) s += s_warp[w]; s_run += s; }
+                __syncthreads();
+            }
+            if (k.aligned) {
+                const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
+                if (lane == 0 && j * T + (tid & ~31u) < k.n) row[(gbase + j * T + tid) >> 5] = bits;
+            } else if (pick) {
+                atomicOr(row + ((gbase + i) >> 5), 1u << ((gbase + i) & 31));
+            }
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+}  // namespace kvp
+
+using namespace kvp;
+
+extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_bitmaps, void* stream)
+{
+    if (!tp || !access_bitmaps || !tp->groups || !tp->units_per_group || !tp->steps || tp->reserved) return KVP_ERR_ARG;
+    if (!tp->topk || tp->topk > tp->units_per_group) return KVP_ERR_ARG;
+    if (tp->rho_q < 0 || tp->rho_q > 65536 || tp->c_q < 0 || tp->c_q > (1 << 20) || tp->sigma_q < 0 ||
+        tp->sigma_q > (1 << 20))
+        return KVP_ERR_ARG;
+    const uint64_t U64 = (uint64_t)tp->groups * tp->units_per_group;
+    if (U64 >= (1ull << 26) || tp->units_per_group > 8192 || tp->steps > 32768) return KVP_ERR_RANGE;
+    // |score| must stay below 2^31: bound |x_t| by its worst case, step by step (|base| <= 2^29 is the caller's)
+    {
+        const int64_t emax = (((int64_t)262140 * 80265) >> 16) + 1;
+        const int64_t jump = tp->burst_thr ? (tp->burst_jump < 0 ? -(int64_t)tp->burst_jump : tp->burst_jump) : 0;
+        int64_t bound = (((int64_t)tp->sigma_q * emax) >> 16) + 1 + jump;
+        for (uint32_t t = 1; t < tp->steps && bound < (1ll << 30); ++t)
+            bound = (((int64_t)tp->rho_q * bound + (int64_t)tp->c_q * emax) >> 16) + 1 + jump;
+        if (bound >= (1ll << 30)) return KVP_ERR_RANGE;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    TraceK k;
+    k.groups = tp->groups; k.n = tp->units_per_group; k.steps = tp->steps; k.topk = tp->topk;
+    k.W32 = (uint32_t)((U64 + 31) / 32);
+    k.seed_lo = (uint32_t)tp->seed; k.seed_hi = (uint32_t)(tp->seed >> 32);
+    k.rho_q = tp->rho_q; k.c_q = tp->c_q; k.sigma_q = tp->sigma_q; k.burst_jump = tp->burst_jump;
+    k.burst_thr = tp->burst_thr; k.base = tp->base; k.out = access_bitmaps;
+    k.aligned = tp->units_per_group % 32 == 0;
+    if (!k.aligned) KVP_CUDA(cudaMemsetAsync(access_bitmaps, 0, (size_t)tp->steps * k.W32 * 4, st));
+    const uint32_t n = tp->units_per_group;
+    const int upt = n <= 1024 ? 1 : n <= 2048 ? 2 : n <= 4096 ? 4 : 8;
+    uint32_t T = (n + upt - 1) / upt;
+    T = (T + 31) / 32 * 32;
+    switch (upt) {
+        case 1: trace_kernel<1><<<tp->groups, T, 0, st>>>(k); break;
+        case 2: trace_kernel<2><<<tp->groups, T, 0, st>>>(k); break;
+        case 4: trace_kernel<4><<<tp->groups, T, 0, st>>>(k); break;
+        default: trace_kernel<8><<<tp->groups, T, 0, st>>>(k); break;
+    }
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}

@@ -1,0 +1,169 @@
+"""Annealing kernels vs oracle: per-chain trajectories, bound and winner schedule, all bit-exact."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2508_13231_b200 import workloads as wl
+from gpu_util import both_problems, named_problem, to_dev, to_np, trace_on_gpu
+from oracle_pool import oracle_chains_parallel
+
+pytestmark = pytest.mark.gpu
+GB = 10 ** 9
+NEVER = 2 ** 64 - 1
+
+
+@pytest.fixture(scope="module")
+def kvp():
+    from paper_2508_13231_b200 import kvp
+    return kvp
+
+
+def _params(g, o, **kw):
+    return g.make_params(**kw), o.make_params(**kw)
+
+
+def _check_against_oracle(g, o, gp, op, chains_to_check=None, check_schedule=True):
+    out = g.anneal(gp, want_per_chain=True)
+    stats = out["stats"]
+    temps, mean = o.temps(op)
+    assert stats.calib_mean_delta == mean and stats.temp0 == temps[0]
+    chains = range(gp.chains) if chains_to_check is None else chains_to_check
+    for c in chains:
+        want, _, _ = o.anneal_chains(op, c, 1)
+        assert out["per_chain"][c].astuple() == want[0].astuple(), c
+    if check_schedule and chains_to_check is None:
+        ref = o.anneal(op)
+        assert out["best_ticks"] == ref["best_ticks"] and stats.best_chain == ref["best_chain"]
+        assert np.array_equal(to_np(out["best_schedule"]), ref["best_schedule"])
+        assert out["best_seconds"] == pytest.approx(ref["best_seconds"], rel=1e-9)
+    assert stats.moves_total == sum(r.moves_done for r in out["per_chain"])
+    assert stats.best_ticks == min(r.best_ticks for r in out["per_chain"])
+    return out
+
+
+def test_anneal_tiny_all_chains(kvp, oracle):
+    g, o, cfg, A = named_problem(kvp, oracle, "tiny")
+    for p0 in (0.8, 1e-3):
+        gp, op = _params(g, o, chains=cfg["chains"], moves=cfg["moves"], seed=0, p0=p0)
+        out = _check_against_oracle(g, o, gp, op)
+        assert out["stats"].init_ticks == o.eval(o.init_placement(1))["total_ticks"]
+
+
+@pytest.mark.parametrize("U,S,cap,bw,flags", [
+    (45, 40, 12, (4900, 900, 500), 3),      # odd sizes, ragged words both ways, Table I weights
+    (33, 1, 5, (8000, 900, 900), 3),        # a single step: no migration can ever be charged
+    (1, 7, 1, (8000, 900, 900), 3),         # a single unit
+    (64, 95, 0, (8000, 900, 900), 3),       # nothing fits in HBM: every flip-in is infeasible
+    (64, 64, 64, (8000, 900, 900), 3),      # everything fits
+    (200, 130, 37, (4900, 500, 900), 2),    # link slower than DRAM, migrations free on the HBM side
+    (90, 33, 20, (3, 1, 1), 0),             # free migration
+])
+def test_anneal_small_shapes(kvp, oracle, U, S, cap, bw, flags):
+    A = wl.random_access(U, S, 0.3, seed=U + S)
+    hw = (np.arange(S) % 2).astype(np.uint32)
+    ew = (np.arange(S) % 3).astype(np.uint32)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, tuple(b * GB for b in bw), mig_flags=flags, hw=hw, ew=ew)
+    for init in (kvp.INIT_STATIC_FIRST, kvp.INIT_STATIC_FREQ):
+        gp, op = _params(g, o, chains=9, moves=3001, seed=12345678901234, levels=7, init_mode=init, p_swap_256=100,
+                         max_len_log2=4)
+        _check_against_oracle(g, o, gp, op)
+
+
+def test_anneal_options(kvp, oracle):
+    U, S, cap = 120, 70, 30
+    A = wl.random_access(U, S, 0.25, seed=3)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    # caller-supplied temperature ladder, only flips / only swaps, a single level, fewer moves than levels
+    for kw in (dict(chains=5, moves=2000, levels=4, temps=[900.0, 90.0, 9.0, 0.5]),
+               dict(chains=5, moves=2000, levels=3, p_swap_256=0), dict(chains=5, moves=2000, levels=3, p_swap_256=256),
+               dict(chains=3, moves=500, levels=1), dict(chains=3, moves=5, levels=16), dict(chains=1, moves=1),
+               dict(chains=4, moves=64000, levels=64, early_stop_permille=1),
+               dict(chains=4, moves=64000, levels=64, early_stop_permille=5, early_stop_from_level=30, p0=0.01),
+               dict(chains=40, moves=777, levels=5, max_len_log2=0, seed=2 ** 63 + 5)):
+        gp, op = _params(g, o, **kw)
+        _check_against_oracle(g, o, gp, op)
+    # user-supplied initial schedule
+    init = wl.random_schedules(U, S, cap, 1, seed=4, churn=0.1)[0]
+    gp = g.make_params(chains=6, moves=1500, levels=5, init_mode=kvp.INIT_USER, init_schedule=to_dev(init))
+    op = o.make_params(chains=6, moves=1500, levels=5, init_mode=oracle.INIT_USER, init_schedule=init)
+    _check_against_oracle(g, o, gp, op)
+    # an infeasible initial schedule is refused (Eq. 5)
+    bits = wl.unpack_bits(init, U); bits[10, :cap + 1] = 1
+    gp = g.make_params(chains=2, moves=10, init_mode=kvp.INIT_USER, init_schedule=to_dev(wl.pack_bits(bits)))
+    with pytest.raises(kvp.KvpError) as e:
+        g.anneal(gp)
+    assert e.value.code == kvp.ERR_CAPACITY
+    for bad in (dict(chains=0, moves=10), dict(chains=1, moves=0), dict(chains=1, moves=1, max_len_log2=6),
+                dict(chains=1, moves=1, p0=1.5), dict(chains=1, moves=1, levels=0)):
+        with pytest.raises(kvp.KvpError) as e:
+            g.anneal(g.make_params(**bad))
+        assert e.value.code == kvp.ERR_ARG
+
+
+def test_chain_state_replay(kvp, oracle):
+    U, S, cap = 150, 100, 40
+    A = wl.random_access(U, S, 0.25, seed=8)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (4900 * GB, 900 * GB, 500 * GB))
+    gp, op = _params(g, o, chains=4, moves=5000, levels=10, seed=99)
+    for chain, upto in [(0, 0), (1, 1), (2, 31), (3, 33), (2, 1234), (3, 5000), (0, 99999)]:
+        sched, res = g.chain_state(gp, chain, upto)
+        want, fin, _ = o.anneal_chains(op, chain, 1, upto_moves=min(upto, 5000), want_final=True)
+        assert np.array_equal(to_np(sched), fin[0]), (chain, upto)
+        assert res.astuple() == want[0].astuple()
+        assert int(g.eval(sched)["total_ticks"][0]) == want[0].final_ticks
+
+
+def test_anneal_single_head_benchmark_configuration(kvp, oracle):
+    # the configuration the benchmark times: 1024 chains x 100k moves, schedule resident in shared memory.
+    # The oracle replays chains on the host cores (as many as the time allows) plus the winner.
+    g, o, cfg, A = named_problem(kvp, oracle, "single_head")
+    kw = dict(chains=cfg["chains"], moves=cfg["moves"], seed=0, p0=cfg.get("p0", 0.8))
+    gp, op = _params(g, o, **kw)
+    out = g.anneal(gp, want_per_chain=True)
+    cores = os.cpu_count() or 1
+    n_check = 1024 if cores >= 32 else (256 if cores >= 8 else 64)
+    want = oracle_chains_parallel("single_head", kw, n_check)
+    got = [r.astuple() for r in out["per_chain"][:n_check]]
+    assert got == want
+    st = out["stats"]
+    w = st.best_chain
+    ref, _, bst = o.anneal_chains(op, w, 1, want_best=True)
+    assert ref[0].astuple() == out["per_chain"][w].astuple()
+    assert np.array_equal(to_np(out["best_schedule"]), bst[0])
+    assert out["best_ticks"] == ref[0].best_ticks == min(r.best_ticks for r in out["per_chain"])
+    assert o.eval(bst[0])["total_ticks"] == out["best_ticks"] and o.eval(bst[0])["bad_step"] == -1
+    assert st.moves_total == 1024 * 100_000
+
+
+def test_anneal_layer_8b_global_state(kvp, oracle):
+    # schedule too large for shared memory: chain state lives in global scratch
+    g, o, cfg, A = named_problem(kvp, oracle, "layer_8b")
+    kw = dict(chains=64, moves=20_000, seed=0, p0=1e-3)
+    gp, op = _params(g, o, **kw)
+    out = _check_against_oracle(g, o, gp, op, chains_to_check=[0, 1, 31, 63], check_schedule=False)
+    w = out["stats"].best_chain
+    ref, _, bst = o.anneal_chains(op, w, 1, want_best=True)
+    assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
+
+
+@pytest.mark.parametrize("name,chains,moves", [("full_8b", 128, 20_000), ("long_70b", 96, 20_000)])
+def test_anneal_full_size_sampled_chains(kvp, oracle, name, chains, moves):
+    # full-size problems, reduced chain count and budget; the oracle recomputes a sample of the chains
+    cfg = wl.CONFIGS[name]
+    U, S, cap = wl.units(cfg), cfg["steps"], cfg["cap"]
+    A = to_np(trace_on_gpu(kvp, wl.trace_params(name, seed=0)))
+    g, o = both_problems(kvp, oracle, U, cfg["bytes_per_unit"], S, A, cap, cfg["bw"])
+    kw = dict(chains=chains, moves=moves, seed=0, p0=1e-3)
+    gp, op = _params(g, o, **kw)
+    out = g.anneal(gp, want_per_chain=True)
+    temps, mean = o.temps(op)
+    assert out["stats"].calib_mean_delta == mean
+    for c in (0, chains // 2, chains - 1):
+        want, _, _ = o.anneal_chains(op, c, 1)
+        assert out["per_chain"][c].astuple() == want[0].astuple(), c
+    # properties at full size: the winner's schedule re-scores to the bound and respects Eq. 5
+    ev = g.eval(out["best_schedule"])
+    assert int(ev["total_ticks"][0]) == out["best_ticks"] and int(ev["bad_step"][0]) == -1
+    assert out["best_ticks"] <= out["stats"].init_ticks

@@ -156,7 +156,8 @@ typedef struct {
     uint32_t init_mode;         /* KVP_INIT_*                                                        */
     uint32_t p_swap_256;        /* P(swap move) * 256, 0..256; the rest are flip moves              */
     uint32_t max_len_log2;      /* run lengths are min(2^k, 31), k uniform in 0..max_len_log2 (<= 5) */
-    uint32_t reserved;          /* must be 0                                                         */
+    uint32_t first_chain;       /* index of the first chain: the call runs chains first_chain ..
+                                   first_chain+chains-1, so that a job can be split over GPUs or calls */
     const uint32_t* init_schedule;  /* (device) [steps][W32], only for KVP_INIT_USER                */
 } kvp_anneal_params;
 
@@ -176,7 +177,7 @@ typedef struct {
 typedef struct {
     uint64_t init_ticks;        /* T of the initial placement                                      */
     uint64_t best_ticks;        /* the bound: min over chains                                      */
-    uint32_t best_chain;        /* lowest chain index that reached it                              */
+    uint32_t best_chain;        /* lowest chain index that reached it (absolute: includes first_chain) */
     uint32_t levels;            /* number of levels actually used                                  */
     uint64_t best_move;
     uint64_t moves_total;       /* sum of moves_done over chains                                   */
@@ -206,6 +207,7 @@ int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint
  *   best_schedule (device) [steps][W32] or NULL
  *   best_ticks, best_seconds (host) or NULL
  *   stats (host) or NULL; stats->per_chain must be NULL or a host array [chains]
+ *   (entry i belongs to chain first_chain + i)
  * Synchronises `stream` before returning.
  */
 int kvp_anneal(kvp_problem* p, const kvp_anneal_params* params, uint32_t* best_schedule,

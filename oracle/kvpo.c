@@ -292,7 +292,7 @@ typedef struct {
     double p0, alpha;
     const double *temps;
     uint32_t early_stop_permille, early_stop_from_level;
-    uint32_t init_mode, p_swap_256, max_len_log2, reserved;
+    uint32_t init_mode, p_swap_256, max_len_log2, first_chain;
     const uint32_t *init_schedule;
 } kvpo_anneal_params;
 
@@ -564,7 +564,7 @@ int kvpo_anneal_chains(const kvpo_problem *p, const kvpo_anneal_params *ap,
 }
 
 /*
- * The whole search: every chain in index order, the bound = the lowest
+ * The whole search: chains first_chain .. first_chain+chains-1 in index order, the bound = the lowest
  * best_ticks, ties to the lower chain index; best_schedule [S][W32] receives the
  * winner's schedule at the moment it reached the bound. per_chain [chains] or NULL.
  */
@@ -577,11 +577,12 @@ int kvpo_anneal(const kvpo_problem *p, const kvpo_anneal_params *ap, const uint3
     uint32_t *tmp = (uint32_t *)malloc(nw * 4);
     if (!tmp) return KVPO_ERR_NOMEM;
     uint64_t bt = UINT64_MAX; uint32_t bc = 0;
-    for (uint32_t c = 0; c < ap->chains; ++c) {
+    for (uint32_t i = 0; i < ap->chains; ++i) {
+        uint32_t c = ap->first_chain + i;
         kvpo_chain_result r;
         int rc = kvpo_anneal_chains(p, ap, table, shifts, c, 1, ap->moves, &r, NULL, tmp);
         if (rc) { free(tmp); return rc; }
-        if (per_chain) per_chain[c] = r;
+        if (per_chain) per_chain[i] = r;
         if (r.best_ticks < bt) {
             bt = r.best_ticks; bc = c;
             if (best_schedule) memcpy(best_schedule, tmp, nw * 4);

@@ -40,7 +40,7 @@ class AnnealParams(C.Structure):
         ("temps", C.POINTER(C.c_double)),
         ("early_stop_permille", C.c_uint32), ("early_stop_from_level", C.c_uint32),
         ("init_mode", C.c_uint32), ("p_swap_256", C.c_uint32),
-        ("max_len_log2", C.c_uint32), ("reserved", C.c_uint32),
+        ("max_len_log2", C.c_uint32), ("first_chain", C.c_uint32),
         ("init_schedule", C.POINTER(C.c_uint32)),
     ]
 
@@ -149,7 +149,7 @@ class Problem:
 
     def make_params(self, chains, moves, seed=0, levels=64, p0=0.8, alpha=0.9, temps=None,
                     early_stop_permille=0, early_stop_from_level=0, init_mode=INIT_STATIC_FREQ,
-                    p_swap_256=128, max_len_log2=5, init_schedule=None):
+                    p_swap_256=128, max_len_log2=5, init_schedule=None, first_chain=0):
         ap = AnnealParams()
         ap.chains, ap.levels, ap.moves, ap.seed = chains, levels, moves, seed
         ap.p0, ap.alpha = p0, alpha
@@ -161,6 +161,7 @@ class Problem:
             ap.temps = t.ctypes.data_as(C.POINTER(C.c_double))
         ap.early_stop_permille, ap.early_stop_from_level = early_stop_permille, early_stop_from_level
         ap.init_mode, ap.p_swap_256, ap.max_len_log2 = init_mode, p_swap_256, max_len_log2
+        ap.first_chain = first_chain
         if init_schedule is not None:
             s = self._sched(init_schedule)
             keep.append(s)

@@ -306,11 +306,11 @@ struct Ctx {
 int validate(const kvp_problem* p, const kvp_anneal_params* a)
 {
     if (!p || !a) return KVP_ERR_ARG;
-    if (!a->chains || !a->moves || !a->levels || a->levels > 4096 || a->reserved) return KVP_ERR_ARG;
+    if (!a->chains || !a->moves || !a->levels || a->levels > 4096) return KVP_ERR_ARG;
     if (a->p_swap_256 > 256 || a->max_len_log2 > 5 || a->init_mode > KVP_INIT_USER) return KVP_ERR_ARG;
     if (a->init_mode == KVP_INIT_USER && !a->init_schedule) return KVP_ERR_ARG;
     if (!a->temps && (!(a->p0 > 0.0 && a->p0 < 1.0) || !(a->alpha > 0.0 && a->alpha <= 1.0))) return KVP_ERR_ARG;
-    if (a->chains >= (1u << 24)) return KVP_ERR_RANGE;
+    if (a->chains >= (1u << 24) || (uint64_t)a->first_chain + a->chains > (1ull << 31)) return KVP_ERR_RANGE;
     return KVP_OK;
 }
 
@@ -504,7 +504,9 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     // the chains, one wave of resident chains after the other
     for (uint32_t first = 0; first < a->chains; first += c.resident) {
         const uint32_t count = a->chains - first < c.resident ? a->chains - first : c.resident;
-        if ((rc = run_chains(c, first, count, 0, c.results, a->moves, nullptr))) { cleanup(); return rc; }
+        if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr))) {
+            cleanup(); return rc;
+        }
     }
     KVP_CUDA(cudaEventRecord(ev[2], st));
 
@@ -517,6 +519,7 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
     KVP_CUDA(cudaStreamSynchronize(st));
     const uint64_t upto = red.best_move == ~0ull ? 0 : red.best_move + 1;
+    red.best_chain += a->first_chain;                      // the reduction works on call-local indices
     if ((rc = replay_to_sched(p, c, red.best_chain, upto, c.results + a->chains))) { cleanup(); return rc; }
     if ((rc = launch_counts(p, c.sched, 1, c.counts0, st, &c.launches))) { cleanup(); return rc; }
     if ((rc = launch_finish(p, c.counts0, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2), c.small + 1, st))) {

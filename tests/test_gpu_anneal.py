@@ -84,6 +84,15 @@ def test_anneal_options(kvp, oracle):
                dict(chains=40, moves=777, levels=5, max_len_log2=0, seed=2 ** 63 + 5)):
         gp, op = _params(g, o, **kw)
         _check_against_oracle(g, o, gp, op)
+    # a slice of a larger job: chains 5..9 behave exactly as in a run of chains 0..15
+    gp16, op16 = _params(g, o, chains=16, moves=1500, levels=5)
+    gp5, _ = _params(g, o, chains=5, moves=1500, levels=5, first_chain=5)
+    whole, part = g.anneal(gp16, want_per_chain=True), g.anneal(gp5, want_per_chain=True)
+    assert [r.astuple() for r in part["per_chain"]] == [r.astuple() for r in whole["per_chain"][5:10]]
+    assert 5 <= part["stats"].best_chain < 10
+    ref = o.anneal(o.make_params(chains=5, moves=1500, levels=5, first_chain=5))
+    assert (part["best_ticks"], part["stats"].best_chain) == (ref["best_ticks"], ref["best_chain"])
+    assert np.array_equal(to_np(part["best_schedule"]), ref["best_schedule"])
     # user-supplied initial schedule
     init = wl.random_schedules(U, S, cap, 1, seed=4, churn=0.1)[0]
     gp = g.make_params(chains=6, moves=1500, levels=5, init_mode=kvp.INIT_USER, init_schedule=to_dev(init))

@@ -128,6 +128,33 @@ int kvp_eval(kvp_problem* p, const uint32_t* schedules, uint32_t n,
 int kvp_eval_counts(kvp_problem* p, const uint32_t* schedules, uint32_t n,
                     uint32_t* counts, void* stream);
 
+/*
+ * kvp_eval_noalloc -- kvp_eval for callers that must not allocate device memory. (The paper has no
+ * counterpart; this is a service of this library.)
+ *
+ * kvp_eval keeps its per-step cardinalities in a scratch buffer that it grows with cudaFree/cudaMalloc
+ * whenever a batch is larger than any before. That is unwelcome in three situations: inside a serving or
+ * control loop where an allocation would stall the whole device for a moment; in a process whose
+ * framework has claimed all device memory for its own pool, so that a raw cudaMalloc fails; and in code
+ * that is not allowed to call the allocator at all at that point. This variant takes the same arguments
+ * and gives the same results, but its scratch is a fixed array that is part of the library image:
+ * KVP_NOALLOC_SCRATCH_BYTES (1 MiB) of device memory on every GPU that loads the library, held until the
+ * process exits. It calls no allocating routine, neither of CUDA nor of any other library.
+ *
+ * Limit: n * steps * 16 bytes <= KVP_NOALLOC_SCRATCH_BYTES, i.e. n * steps <= 65536; a larger batch is
+ * refused with KVP_ERR_RANGE and nothing is launched (split it, or use kvp_eval).
+ * First call on a device: looks up the device address of the array (once per device, with that device
+ * current). Make that first call outside any stream capture.
+ * Sharing: every call on a device uses the same array and overwrites what the previous call left there
+ * (everything that must start from zero is cleared by the call itself). Two calls whose kernels can
+ * overlap on the GPU -- different streams, or different host threads -- race on it; order them.
+ * Otherwise as kvp_eval: asynchronous on `stream`, all pointers (device), `p` from kvp_create.
+ */
+#define KVP_NOALLOC_SCRATCH_BYTES (1u << 20)
+int kvp_eval_noalloc(kvp_problem* p, const uint32_t* schedules, uint32_t n,
+                     uint64_t* step_ticks, uint64_t* total_ticks,
+                     double* step_seconds, double* total_seconds, int32_t* bad_step, void* stream);
+
 /* Initial placement of a chain. */
 #define KVP_INIT_STATIC_FIRST 0u /* units 0..cap-1 at every step: the Static Placement baseline (Section IV-A) */
 #define KVP_INIT_STATIC_FREQ  1u /* the cap units with most accesses over all steps (ties: lower index)     */

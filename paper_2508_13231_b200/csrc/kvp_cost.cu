@@ -277,3 +277,46 @@ extern "C" int kvp_eval(kvp_problem* p, const uint32_t* schedules, uint32_t n, u
     }
     return KVP_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------
+// kvp_eval without any allocation: the per-step cardinalities go to a fixed array in the library image.
+// Meant for callers that cannot afford or are not allowed a cudaMalloc at this point (a latency-bound
+// loop, a process whose memory pool owns the whole device, allocator-free code). See include/kvp.h.
+static __device__ __align__(256) uint32_t g_noalloc_counts[KVP_NOALLOC_SCRATCH_BYTES / 4];
+
+namespace {
+constexpr int kMaxDevices = 64;
+uint32_t* g_noalloc_addr[kMaxDevices];   // device address of g_noalloc_counts, per device; null until looked up
+}
+
+// In host code `g_noalloc_counts` names a host-side shadow of the symbol, not device memory: the address a
+// kernel may use has to be asked for, once per device and with that device current.
+static int noalloc_scratch(int device, uint32_t** out)
+{
+    if (device < 0 || device >= kMaxDevices) return KVP_ERR_RANGE;
+    uint32_t* ptr = __atomic_load_n(&g_noalloc_addr[device], __ATOMIC_ACQUIRE);
+    if (!ptr) {
+        KVP_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_counts));
+        if (!ptr) return KVP_ERR_CUDA;
+        __atomic_store_n(&g_noalloc_addr[device], ptr, __ATOMIC_RELEASE);   // racing threads store the same value
+    }
+    *out = ptr;
+    return KVP_OK;
+}
+
+extern "C" int kvp_eval_noalloc(kvp_problem* p, const uint32_t* schedules, uint32_t n, uint64_t* step_ticks,
+                                uint64_t* total_ticks, double* step_seconds, double* total_seconds, int32_t* bad_step,
+                                void* stream)
+{
+    if (!p || !schedules || !total_ticks || !n) return KVP_ERR_ARG;
+    if ((uint64_t)n * p->S * 16ull > (uint64_t)KVP_NOALLOC_SCRATCH_BYTES) return KVP_ERR_RANGE;   // batch too large
+    KVP_CUDA(cudaSetDevice(p->device));
+    uint32_t* counts = nullptr;
+    int rc = noalloc_scratch(p->device, &counts);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array still holds the previous call's numbers. launch_counts either overwrites every entry it
+    // owns (narrow rows) or clears them on the stream before accumulating (wide rows).
+    if ((rc = kvp::launch_counts(p, schedules, n, counts, st, nullptr))) return rc;
+    return kvp::launch_finish(p, counts, n, step_ticks, total_ticks, step_seconds, total_seconds, bad_step, nullptr, st);
+}

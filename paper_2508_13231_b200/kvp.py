@@ -18,8 +18,10 @@ MIG_HBM, MIG_EXT, MIG_PAPER = 1, 2, 3
 INIT_STATIC_FIRST, INIT_STATIC_FREQ, INIT_USER = 0, 1, 2
 TABLE_Q = 1024
 
+NOALLOC_SCRATCH_BYTES = 1 << 20
+
 EXPORTS = [
-    "kvp_create", "kvp_destroy", "kvp_get_info", "kvp_eval", "kvp_eval_counts", "kvp_accept_table", "kvp_anneal",
+    "kvp_create", "kvp_destroy", "kvp_get_info", "kvp_eval", "kvp_eval_counts", "kvp_eval_noalloc", "kvp_accept_table", "kvp_anneal",
     "kvp_anneal_chain_state", "kvp_trace_generate", "kvp_philox4x32_10", "kvp_strerror", "kvp_last_cuda_error",
 ]
 
@@ -204,6 +206,17 @@ class Problem:
         _chk(_lib().kvp_eval(self._h, _ptr(schedules, torch.int32), C.c_uint32(n), _ptr(st), _ptr(tt), _ptr(ss),
                              _ptr(ts), _ptr(bad), _stream(stream)), "kvp_eval")
         return dict(step_ticks=st, total_ticks=tt, step_seconds=ss, total_seconds=ts, bad_step=bad)
+
+    def eval_noalloc(self, schedules, step_ticks, total_ticks, step_seconds, total_seconds, bad_step, stream=None):
+        """kvp_eval_noalloc: like eval(), but the library allocates nothing. The caller passes every output
+        tensor (CUDA; any but total_ticks may be None) so that this wrapper allocates nothing either.
+        For code that cannot call the allocator here: a latency-bound loop, or a process whose memory pool
+        owns the device. Batches are limited to n * steps <= 65536; calls share one scratch array per GPU,
+        so do not let two of them run concurrently."""
+        n = self._n(schedules)
+        _chk(_lib().kvp_eval_noalloc(self._h, _ptr(schedules, torch.int32), C.c_uint32(n), _ptr(step_ticks),
+                                     _ptr(total_ticks), _ptr(step_seconds), _ptr(total_seconds), _ptr(bad_step),
+                                     _stream(stream)), "kvp_eval_noalloc")
 
     def eval_counts(self, schedules, stream=None):
         n = self._n(schedules)

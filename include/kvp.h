@@ -182,7 +182,7 @@ typedef struct {
     uint32_t early_stop_from_level; /* the rule is not applied at boundaries entering levels below this */
     uint32_t init_mode;         /* KVP_INIT_*                                                        */
     uint32_t p_swap_256;        /* P(swap move) * 256, 0..256; the rest are flip moves              */
-    uint32_t max_len_log2;      /* run lengths are min(2^k, 31), k uniform in 0..max_len_log2 (<= 5) */
+    uint32_t max_len_log2;      /* run lengths are min(2^k, 30), k uniform in 0..max_len_log2 (<= 5) */
     uint32_t first_chain;       /* index of the first chain: the call runs chains first_chain ..
                                    first_chain+chains-1, so that a job can be split over GPUs or calls */
     const uint32_t* init_schedule;  /* (device) [steps][W32], only for KVP_INIT_USER                */

@@ -317,7 +317,7 @@ static move_t decode_move(const kvpo_problem *p, const kvpo_anneal_params *ap,
     move_t mv;
     mv.swap = (r[0] & 255u) < ap->p_swap_256;
     uint32_t k = (((r[0] >> 8) & 255u) * (ap->max_len_log2 + 1u)) >> 8;
-    mv.len = (1u << k) < 31u ? (1u << k) : 31u;
+    mv.len = (1u << k) < 30u ? (1u << k) : 30u;
     mv.s0 = ((r[0] >> 16) * p->S) >> 16;
     mv.u = (uint32_t)(((uint64_t)r[1] * p->U) >> 32);
     mv.v = (uint32_t)(((uint64_t)r[2] * p->U) >> 32);

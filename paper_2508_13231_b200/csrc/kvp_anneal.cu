@@ -30,6 +30,8 @@ struct ChainParams {
     uint32_t* ws;                // global scratch: [slots][U*S32] (only the global-state variant)
     kvp_chain_result* results;   // indexed by chain - result_base
     uint32_t* dump;              // if set, slot 0 writes its final schedule here (time-packed)
+    const uint32_t* full0;       // [S32] full-step bitmap of the initial schedule
+    uint32_t* snap;              // if set: [slots][U*S32], each chain's schedule when it reached its best
     CostK K;
     uint32_t U, S, S32, cap;
     uint32_t chain_first, chain_count, result_base;
@@ -39,102 +41,173 @@ struct ChainParams {
     uint64_t per_level, upto, init_ticks;
 };
 
-// What a lane needs to remember between evaluating and applying a proposal.
-struct LaneDelta {
-    uint4 ctr;                   // counters of the lane's step before the move
-    int dhr, dmi, dmo, docc;
-    uint32_t t;                  // the lane's step (valid when active)
-    bool active;
+// A proposal as one lane sees it: the Philox words, and after evaluation the placement windows of its one
+// or two units before (W) and after (N) the move, their access windows (A) and the verdict.
+// Window convention: bit k of a window belongs to step s0 - 1 + k, so bit 0 is the step before the run (for
+// s0 == 0 it repeats step 0, because P[-1] := P[0]), bits 1..run are the run, and the affected steps
+// s0..last are bits 1..nl <= 31. Run lengths stop at 30 so that every vector fits one 32-bit register.
+struct LaneMove {
+    uint32_t pk, u, v, w;        // packed (swap | len << 1 | s0 << 8), units, Metropolis uniform
+    uint32_t Wu, Wv, Nu, Nv, Au, Av;
+    int delta;
+    bool inf, acc, chg;
 };
 
 __device__ __forceinline__ void decode_move(const uint32_t r[4], uint32_t p_swap_256, uint32_t len_choices, uint32_t S,
-                                            uint32_t U, uint32_t& pk, uint32_t& u, uint32_t& v)
+                                            uint32_t U, LaneMove& mv)
 {
     const uint32_t swap = (r[0] & 255u) < p_swap_256 ? 1u : 0u;
     const uint32_t k = (((r[0] >> 8) & 255u) * len_choices) >> 8;
-    const uint32_t len = min(1u << k, 31u);
+    const uint32_t len = min(1u << k, 30u);
     const uint32_t s0 = ((r[0] >> 16) * S) >> 16;
-    pk = swap | (len << 1) | (s0 << 8);
-    u = __umulhi(r[1], U);
-    v = __umulhi(r[2], U);
+    mv.pk = swap | (len << 1) | (s0 << 8);
+    mv.u = __umulhi(r[1], U);
+    mv.v = __umulhi(r[2], U);
+    mv.w = r[3];
 }
 
-// Evaluate a proposal against the current state. All 32 lanes call this with identical arguments.
-// Returns the summed cost change; `infeasible` (a flip would break Eq. 5) and `changed` are warp-uniform.
-template <typename CtrPtr>
-__device__ __forceinline__ int eval_move(const uint32_t* P, const uint32_t* __restrict__ Acol, CtrPtr ctr,
-                                         const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
-                                         uint32_t cap, uint32_t lane, uint32_t pk, uint32_t u, uint32_t v,
-                                         LaneDelta& ld, bool& infeasible, bool& changed)
+// 32 consecutive bits of a time-packed column starting at step s0 - 1 (see LaneMove). Bits that belong to
+// steps beyond the horizon are arbitrary; every user masks them.
+template <typename Ptr>
+__device__ __forceinline__ uint32_t window(Ptr col, uint32_t S32, uint32_t s0)
 {
-    const bool swap = pk & 1u;
-    const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
-    const uint32_t last = min(s0 + len, S - 1);
-    const uint32_t t = s0 + lane;
-    const bool active = t <= last;
-    const uint32_t tt = active ? t : s0;
-    const bool in_run = active && lane < len;                      // the placement bit of step t changes hands
-    const bool prev_in_run = active && (tt == 0 ? in_run : lane >= 1);  // step 0 has no predecessor: P[-1] := P[0]
-    const uint32_t tp = tt ? tt - 1 : 0;
-    const size_t ub = (size_t)u * S32, vb = (size_t)v * S32;
-    const uint32_t wi = tt >> 5, bi = tt & 31, wpi = tp >> 5, bpi = tp & 31;
-
-    const uint32_t pu = (P[ub + wi] >> bi) & 1u, qu = (P[ub + wpi] >> bpi) & 1u;
-    const uint32_t au = (__ldg(Acol + ub + wi) >> bi) & 1u;
-    uint32_t pv = 0, qv = 0, av = 0;
-    if (swap) {
-        pv = (P[vb + wi] >> bi) & 1u; qv = (P[vb + wpi] >> bpi) & 1u;
-        av = (__ldg(Acol + vb + wi) >> bi) & 1u;
+    if (s0 == 0) {
+        const uint32_t raw = col[0];
+        return (raw << 1) | (raw & 1u);
     }
-    uint32_t npu, nqu, npv, nqv;
-    if (swap) {
-        npu = in_run ? pv : pu; npv = in_run ? pu : pv;
-        nqu = prev_in_run ? qv : qu; nqv = prev_in_run ? qu : qv;
-    } else {
-        npu = pu ^ (in_run ? 1u : 0u); nqu = qu ^ (prev_in_run ? 1u : 0u);
-        npv = 0; nqv = 0;
-    }
-    ld.dhr = (int)(au & npu) - (int)(au & pu) + (int)(av & npv) - (int)(av & pv);
-    ld.dmi = (int)(npu & ~nqu & 1u) - (int)(pu & ~qu & 1u) + (int)(npv & ~nqv & 1u) - (int)(pv & ~qv & 1u);
-    ld.dmo = (int)(~npu & nqu & 1u) - (int)(~pu & qu & 1u) + (int)(~npv & nqv & 1u) - (int)(~pv & qv & 1u);
-    ld.docc = (int)npu - (int)pu + (int)npv - (int)pv;
-    ld.active = active;
-    ld.t = tt;
-    ld.ctr = ctr[tt];
-    const StepC c = __ldg(stepc + tt);
-    const uint32_t f_old = step_cost(ld.ctr.x, ld.ctr.y, ld.ctr.z, c, K);
-    const uint32_t f_new = step_cost(ld.ctr.x + ld.dhr, ld.ctr.y + ld.dmi, ld.ctr.z + ld.dmo, c, K);
-    const int dl = active ? (int)(f_new - f_old) : 0;
-    infeasible = __any_sync(0xFFFFFFFFu, active && ld.docc > 0 && ld.ctr.w + (uint32_t)ld.docc > cap);
-    changed = __any_sync(0xFFFFFFFFu, active && (npu != pu || npv != pv));
-    return __reduce_add_sync(0xFFFFFFFFu, dl);
+    const uint32_t b0 = s0 - 1, w = b0 >> 5;
+    const uint32_t lo = col[w], hi = col[min(w + 1, S32 - 1)];
+    return __funnelshift_r(lo, hi, b0 & 31u);
 }
 
-__device__ __forceinline__ void apply_move(uint32_t* P, uint4* ctr, uint32_t S, uint32_t S32, uint32_t lane,
-                                           uint32_t pk, uint32_t u, uint32_t v, const LaneDelta& ld)
+struct ChainView {               // where a chain's state lives
+    uint32_t* P;                 // [U][S32] schedule, time-packed (shared or global)
+    uint4* ctr;                  // [S] {hr, mi, mo, occ} (shared)
+    uint32_t* full;              // [S32] bit t set iff occ[t] == cap (shared)
+};
+
+// Evaluate one proposal against the current state, all in the calling lane. Word-parallel over the <= 31
+// affected steps for everything that is a bit; Eq. 2-4 are re-evaluated only at steps whose cardinalities change.
+template <typename PPtr, typename CPtr, typename FPtr>
+__device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ Acol, CPtr ctr, FPtr full,
+                                          const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
+                                          const uint32_t* __restrict__ trow, uint32_t shift, LaneMove& mv)
 {
+    const bool swap = mv.pk & 1u;
+    const uint32_t len = (mv.pk >> 1) & 63u, s0 = mv.pk >> 8;
+    const uint32_t run = min(s0 + len, S) - s0;                   // steps whose placement bits change hands
+    const uint32_t nl = min(s0 + len, S - 1) - s0 + 1;            // affected steps: the run and the step after it
+    const uint32_t M = ((1u << run) - 1u) << 1;
+    const uint32_t Sb = ((1u << nl) - 1u) << 1;
+    const size_t ub = (size_t)mv.u * S32;
+    const uint32_t Wu = window(P + ub, S32, s0);
+    const uint32_t Au = window(Acol + ub, S32, s0);
+    uint32_t Wv = 0, Av = 0;
+    if (swap) {
+        const size_t vb = (size_t)mv.v * S32;
+        Wv = window(P + vb, S32, s0);
+        Av = window(Acol + vb, S32, s0);
+    }
+    const uint32_t D = swap ? ((Wu ^ Wv) & M) : M;                // bits that toggle
+    uint32_t Nu = Wu ^ D, Nv = swap ? (Wv ^ D) : 0u;
+    if (s0 == 0) {                                                // the virtual step -1 follows step 0
+        Nu = (Nu & ~1u) | ((Nu >> 1) & 1u);
+        Nv = (Nv & ~1u) | ((Nv >> 1) & 1u);
+    }
+    mv.Wu = Wu; mv.Wv = Wv; mv.Nu = Nu; mv.Nv = Nv; mv.Au = Au; mv.Av = Av;
+    mv.chg = D != 0;
+    mv.inf = false;
+    mv.delta = 0;
+    if (!swap) {                                                  // a flip may not raise a full step (Eq. 5)
+        const uint32_t Fw = window(full, S32, s0);
+        mv.inf = (~Wu & M & Fw) != 0;
+    }
+    const uint32_t up = Nu & ~Wu, um = Wu & ~Nu;                  // bits u gains / loses (v: the reverse)
+    const uint32_t hrP = (Au & ~Av & up) | (Av & ~Au & um);       // steps whose HBM hit count rises / falls by one
+    const uint32_t hrN = (Au & ~Av & um) | (Av & ~Au & up);
+    const uint32_t miuo = Wu & ~(Wu << 1), miun = Nu & ~(Nu << 1), mivo = Wv & ~(Wv << 1), mivn = Nv & ~(Nv << 1);
+    const uint32_t mouo = ~Wu & (Wu << 1), moun = ~Nu & (Nu << 1), movo = ~Wv & (Wv << 1), movn = ~Nv & (Nv << 1);
+    uint32_t todo = ((miuo ^ miun) | (mivo ^ mivn) | (mouo ^ moun) | (movo ^ movn) | hrP | hrN) & Sb;
+    if (mv.inf) todo = 0;
+    int delta = 0;
+    while (todo) {
+        const uint32_t k = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const uint32_t t = s0 + k - 1;
+        const uint4 c4 = ctr[t];
+        const StepC c = __ldg(stepc + t);
+        const int dhr = (int)((hrP >> k) & 1u) - (int)((hrN >> k) & 1u);
+        const int dmi = (int)(((miun >> k) & 1u) + ((mivn >> k) & 1u)) - (int)(((miuo >> k) & 1u) + ((mivo >> k) & 1u));
+        const int dmo = (int)(((moun >> k) & 1u) + ((movn >> k) & 1u)) - (int)(((mouo >> k) & 1u) + ((movo >> k) & 1u));
+        delta += (int)(step_cost(c4.x + dhr, c4.y + dmi, c4.z + dmo, c, K) - step_cost(c4.x, c4.y, c4.z, c, K));
+    }
+    mv.delta = delta;
+    bool acc = delta <= 0;
+    if (!acc) {
+        const uint32_t q = (uint32_t)delta >> shift;
+        acc = q < KVP_TABLE_Q && mv.w < __ldg(trow + q);          // Metropolis, quantised exp(-delta/C)
+    }
+    mv.acc = acc;
+}
+
+// Apply the proposal held by lane `b`: all lanes take part, lane j updates the counters of window bit j.
+__device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
+                                           uint32_t b, const LaneMove& mine)
+{
+    const uint32_t pk = __shfl_sync(0xFFFFFFFFu, mine.pk, b);
+    const uint32_t u = __shfl_sync(0xFFFFFFFFu, mine.u, b), v = __shfl_sync(0xFFFFFFFFu, mine.v, b);
+    const uint32_t Wu = __shfl_sync(0xFFFFFFFFu, mine.Wu, b), Wv = __shfl_sync(0xFFFFFFFFu, mine.Wv, b);
+    const uint32_t Nu = __shfl_sync(0xFFFFFFFFu, mine.Nu, b), Nv = __shfl_sync(0xFFFFFFFFu, mine.Nv, b);
+    const uint32_t Au = __shfl_sync(0xFFFFFFFFu, mine.Au, b), Av = __shfl_sync(0xFFFFFFFFu, mine.Av, b);
     const bool swap = pk & 1u;
     const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
-    if (ld.active)
-        ctr[ld.t] = make_uint4(ld.ctr.x + ld.dhr, ld.ctr.y + ld.dmi, ld.ctr.z + ld.dmo, ld.ctr.w + ld.docc);
+    const uint32_t run = min(s0 + len, S) - s0;
+    const uint32_t nl = min(s0 + len, S - 1) - s0 + 1;
+    const bool valid = lane >= 1 && lane <= nl;
+    const uint32_t j = valid ? lane : 1u, t = s0 + j - 1;
+    const uint32_t pu = (Wu >> j) & 1u, qu = (Wu >> (j - 1)) & 1u, npu = (Nu >> j) & 1u, nqu = (Nu >> (j - 1)) & 1u;
+    const uint32_t pv = (Wv >> j) & 1u, qv = (Wv >> (j - 1)) & 1u, npv = (Nv >> j) & 1u, nqv = (Nv >> (j - 1)) & 1u;
+    const uint32_t au = (Au >> j) & 1u, av = (Av >> j) & 1u;
+    uint4 c = cv.ctr[t];
+    c.x += (au & npu) - (au & pu) + (av & npv) - (av & pv);
+    c.y += (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
+    c.z += (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
+    c.w += npu - pu + npv - pv;
+    if (valid) cv.ctr[t] = c;
+    uint32_t F = __ballot_sync(0xFFFFFFFFu, valid && c.w == cap);   // bit j <-> window bit j
+    uint32_t V = __ballot_sync(0xFFFFFFFFu, valid);
     if (lane < 2) {
-        const uint32_t end = min(s0 + len, S);
-        const uint32_t wj = (s0 >> 5) + lane;
-        const uint32_t lo = max(s0, wj * 32u), hi = min(end, wj * 32u + 32u);
-        if (hi > lo) {                                   // run lengths are at most 31, so never a full word
-            const uint32_t mask = ((1u << (hi - lo)) - 1u) << (lo - wj * 32u);
-            const size_t iu = (size_t)u * S32 + wj;
-            if (swap) {
-                const size_t iv = (size_t)v * S32 + wj;
-                const uint32_t a = P[iu], b = P[iv];
-                const uint32_t d = (a ^ b) & mask;
-                if (d) { P[iu] = a ^ d; P[iv] = b ^ d; }
-            } else {
-                P[iu] ^= mask;
+        uint32_t M = ((1u << run) - 1u) << 1, NU = Nu, NV = Nv, sbit = s0 - 1;
+        if (s0 == 0) { F >>= 1; V >>= 1; M >>= 1; NU >>= 1; NV >>= 1; sbit = 0; }
+        const uint32_t wj = (sbit >> 5) + lane, sh = sbit & 31u;
+        if (wj < S32 && (lane == 0 || sh != 0)) {
+            // lane 0 holds the part of the window that falls into the first word, lane 1 the spill-over
+            const uint32_t Vx = lane ? V >> (32 - sh) : V << sh, Fx = lane ? F >> (32 - sh) : F << sh;
+            const uint32_t Mx = lane ? M >> (32 - sh) : M << sh;
+            const uint32_t NUx = lane ? NU >> (32 - sh) : NU << sh, NVx = lane ? NV >> (32 - sh) : NV << sh;
+            if (Vx) cv.full[wj] = (cv.full[wj] & ~Vx) | (Fx & Vx);
+            if (Mx) {
+                const size_t iu = (size_t)u * S32 + wj;
+                cv.P[iu] = (cv.P[iu] & ~Mx) | (NUx & Mx);
+                if (swap) {
+                    const size_t iv = (size_t)v * S32 + wj;
+                    cv.P[iv] = (cv.P[iv] & ~Mx) | (NVx & Mx);
+                }
             }
         }
     }
     __syncwarp();
+}
+
+__device__ __forceinline__ void copy_words(uint32_t* dst, const uint32_t* src, size_t n, uint32_t lane)
+{
+    if ((n & 3) == 0 && ((reinterpret_cast<uintptr_t>(dst) | reinterpret_cast<uintptr_t>(src)) & 15) == 0) {
+        uint4* d4 = reinterpret_cast<uint4*>(dst);
+        const uint4* s4 = reinterpret_cast<const uint4*>(src);
+        for (size_t i = lane; i < n / 4; i += 32) d4[i] = s4[i];
+    } else {
+        for (size_t i = lane; i < n; i += 32) dst[i] = src[i];
+    }
 }
 
 template <bool PSMEM>
@@ -148,12 +221,17 @@ chain_kernel(const ChainParams prm)
     const uint32_t chain = prm.chain_first + slot;
     const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
     const size_t pwords = (size_t)U * S32;
-    uint4* ctr = smem4 + (size_t)warp * S;
-    uint32_t* P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)wpb * S) + (size_t)warp * pwords
-                        : prm.ws + (size_t)slot * pwords;
-    for (uint32_t i = lane; i < S; i += 32) ctr[i] = __ldg(prm.counters0 + i);
-    for (size_t i = lane; i < pwords; i += 32) P[i] = __ldg(prm.Pcol0 + i);
+    const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
+    ChainView cv;
+    cv.ctr = smem4 + (size_t)warp * (S + f4);
+    cv.full = reinterpret_cast<uint32_t*>(cv.ctr + S);
+    cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)wpb * (S + f4)) + (size_t)warp * pwords
+                 : prm.ws + (size_t)slot * pwords;
+    for (uint32_t i = lane; i < S; i += 32) cv.ctr[i] = __ldg(prm.counters0 + i);
+    for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
+    copy_words(cv.P, prm.Pcol0, pwords, lane);
     __syncwarp();
+    uint32_t* snap = prm.snap ? prm.snap + (size_t)slot * pwords : nullptr;
 
     uint64_t cur = prm.init_ticks, best = cur, best_move = ~0ull, best_at_boundary = cur;
     uint64_t n_acc = 0, n_chg = 0, n_inf = 0, hash = 0;
@@ -161,52 +239,69 @@ chain_kernel(const ChainParams prm)
     const uint32_t* trow = prm.table;
     uint64_t next_boundary = prm.levels > 1 ? prm.per_level : ~0ull;
     uint64_t m = 0;
-    bool stop = false;
-    while (m < prm.upto && !stop) {
-        // one Philox block per lane: the proposals of moves m .. m+31
-        uint32_t r[4], my_pk, my_u, my_v;
-        const uint64_t mine = m + lane;
-        philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
-        decode_move(r, prm.p_swap_256, prm.len_choices, S, U, my_pk, my_u, my_v);
-        const uint32_t my_w = r[3];
-        const uint32_t nb = (uint32_t)min((uint64_t)32, prm.upto - m);
-        for (uint32_t i = 0; i < nb; ++i, ++m) {
-            if (m == next_boundary) {                    // a new temperature level starts at this move
-                ++level;
-                if (prm.early_permille && level >= prm.early_from &&
-                    (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille) {
-                    stop = true;
-                    break;
-                }
-                best_at_boundary = best;
-                shift = __ldg(prm.shifts + level);
-                trow = prm.table + (size_t)level * KVP_TABLE_Q;
-                next_boundary = level + 1 < prm.levels ? next_boundary + prm.per_level : ~0ull;
-            }
-            const uint32_t pk = __shfl_sync(0xFFFFFFFFu, my_pk, i);
-            const uint32_t u = __shfl_sync(0xFFFFFFFFu, my_u, i);
-            const uint32_t v = __shfl_sync(0xFFFFFFFFu, my_v, i);
-            const uint32_t w = __shfl_sync(0xFFFFFFFFu, my_w, i);
-            LaneDelta ld;
-            bool infeasible, changed;
-            const int delta = eval_move(P, prm.Acol, ctr, prm.stepc, prm.K, S, S32, prm.cap, lane, pk, u, v, ld,
-                                        infeasible, changed);
-            if (infeasible) { ++n_inf; continue; }
-            bool accept = delta <= 0;
-            if (!accept) {
-                const uint32_t q = (uint32_t)delta >> shift;
-                accept = q < KVP_TABLE_Q && w < __ldg(trow + q);      // Metropolis, quantised exp(-delta/C)
-            }
-            if (!accept) continue;
-            ++n_acc;
-            if (!changed) continue;
-            apply_move(P, ctr, S, S32, lane, pk, u, v, ld);
-            ++n_chg;
-            cur = (uint64_t)((int64_t)cur + delta);
-            hash = (hash ^ m) * 0x9E3779B97F4A7C15ull + cur;
-            if (cur < best) { best = cur; best_move = m; }
+    bool snap_dirty = false;                                      // the best state is the current one, not yet saved
+    while (m < prm.upto) {
+        if (m == next_boundary) {                                 // a new temperature level starts at this move
+            ++level;
+            if (prm.early_permille && level >= prm.early_from &&
+                (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille)
+                break;
+            best_at_boundary = best;
+            shift = __ldg(prm.shifts + level);
+            trow = prm.table + (size_t)level * KVP_TABLE_Q;
+            next_boundary = level + 1 < prm.levels ? next_boundary + prm.per_level : ~0ull;
         }
+        // A batch: up to 32 consecutive moves of one temperature level, one per lane. Every lane draws and
+        // evaluates its own proposal against the current state; the warp then commits them in move order.
+        // A move that changes the schedule invalidates only later moves whose step windows overlap its own;
+        // those are evaluated again before their turn comes, so the outcome is that of the sequential chain.
+        const uint32_t nb = (uint32_t)min(min((uint64_t)32, prm.upto - m), next_boundary - m);
+        LaneMove mv;
+        {
+            uint32_t r[4];
+            const uint64_t mine = m + lane;
+            philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
+            decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv);
+        }
+        mv.inf = false; mv.acc = false; mv.chg = false; mv.delta = 0;
+        mv.Wu = mv.Wv = mv.Nu = mv.Nv = mv.Au = mv.Av = 0;
+        uint32_t todo = nb == 32 ? 0xFFFFFFFFu : (1u << nb) - 1u;
+        uint32_t need = todo;
+        while (todo) {
+            if ((need >> lane) & 1u)
+                eval_lane(cv.P, prm.Acol, cv.ctr, cv.full, prm.stepc, prm.K, S, S32, trow, shift, mv);
+            __syncwarp();
+            const uint32_t infb = __ballot_sync(0xFFFFFFFFu, mv.inf);
+            const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !mv.inf && mv.acc);
+            const uint32_t blk = __ballot_sync(0xFFFFFFFFu, !mv.inf && mv.acc && mv.chg) & todo;
+            if (!blk) {
+                n_inf += __popc(infb & todo);
+                n_acc += __popc(accb & todo);
+                break;
+            }
+            const uint32_t b = __ffs(blk) - 1;
+            const uint32_t done = todo & (0xFFFFFFFFu >> (31 - b));   // the moves up to and including b
+            n_inf += __popc(infb & done);
+            n_acc += __popc(accb & done);
+            ++n_chg;
+            const int delta = __shfl_sync(0xFFFFFFFFu, mv.delta, b);
+            const uint64_t after = (uint64_t)((int64_t)cur + delta);
+            if (snap && snap_dirty && after >= best) {            // leaving the best state: save it first
+                copy_words(snap, cv.P, pwords, lane);
+                snap_dirty = false;
+            }
+            apply_move(cv, S, S32, prm.cap, lane, b, mv);
+            cur = after;
+            const uint64_t mb = m + b;
+            hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
+            if (cur < best) { best = cur; best_move = mb; snap_dirty = true; }
+            todo &= ~done;
+            const uint32_t s0b = __shfl_sync(0xFFFFFFFFu, mv.pk, b) >> 8, s0 = mv.pk >> 8;
+            need = __ballot_sync(0xFFFFFFFFu, s0 + 32 > s0b && s0b + 32 > s0) & todo;
+        }
+        m += nb;
     }
+    if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
     if (lane == 0) {
         kvp_chain_result res;
         res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m;
@@ -215,8 +310,16 @@ chain_kernel(const ChainParams prm)
     }
     if (prm.dump && slot == 0) {
         __syncwarp();
-        for (size_t i = lane; i < pwords; i += 32) prm.dump[i] = P[i];
+        copy_words(prm.dump, cv.P, pwords, lane);
     }
+}
+
+// bit t of full0 is set iff the initial schedule fills the HBM capacity at step t
+__global__ void full_mask_kernel(const uint4* __restrict__ counters0, uint32_t S, uint32_t cap, uint32_t* __restrict__ full0)
+{
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t bits = __ballot_sync(0xFFFFFFFFu, t < S && counters0[t < S ? t : 0].w == cap);
+    if ((threadIdx.x & 31) == 0 && t < ((S + 31) / 32) * 32) full0[t >> 5] = bits;
 }
 
 // Calibration of the temperature ladder: proposals (i, 0, 0, TAG_CALIB), i < 1024, are evaluated against the
@@ -224,18 +327,15 @@ chain_kernel(const ChainParams prm)
 __global__ void __launch_bounds__(256)
 calib_kernel(const ChainParams prm, unsigned long long* acc)
 {
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= CALIB_N) return;
-    uint32_t r[4], pk, u, v;
+    uint32_t r[4];
+    LaneMove mv;
     philox4x32_10(i, 0u, 0u, TAG_CALIB, prm.seed_lo, prm.seed_hi, r);
-    decode_move(r, prm.p_swap_256, prm.len_choices, prm.S, prm.U, pk, u, v);
-    LaneDelta ld;
-    bool infeasible, changed;
-    const int delta = eval_move(prm.Pcol0, prm.Acol, prm.counters0, prm.stepc, prm.K, prm.S, prm.S32, prm.cap, lane,
-                                pk, u, v, ld, infeasible, changed);
-    if (lane == 0 && !infeasible && delta > 0) {
-        atomicAdd(acc, (unsigned long long)delta);
+    decode_move(r, prm.p_swap_256, prm.len_choices, prm.S, prm.U, mv);
+    eval_lane(prm.Pcol0, prm.Acol, prm.counters0, prm.full0, prm.stepc, prm.K, prm.S, prm.S32, prm.table, 0u, mv);
+    if (!mv.inf && mv.delta > 0) {
+        atomicAdd(acc, (unsigned long long)mv.delta);
         atomicAdd(acc + 1, 1ull);
     }
 }
@@ -294,6 +394,8 @@ struct Ctx {
     uint32_t* dumpcol;       // [U][S32]
     uint32_t* sched;         // [S][W32]
     uint32_t* slots;         // chain state slices (global variant)
+    uint32_t* full0;         // [S32]
+    uint32_t* snap;          // best-state snapshots (shared-memory variant), or null
     bool psmem;
     uint32_t wpb;            // warps per CTA
     uint32_t resident;       // chains per wave
@@ -325,9 +427,10 @@ int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 }
 
 int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp_chain_result* results, uint64_t upto,
-               uint32_t* dump)
+               uint32_t* dump, uint32_t* snap)
 {
     ChainParams prm = c.prm;
+    prm.snap = snap;
     prm.chain_first = first; prm.chain_count = count; prm.result_base = result_base;
     prm.results = results; prm.upto = upto; prm.dump = dump;
     ++c.launches;
@@ -350,7 +453,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     KVP_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     KVP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const size_t budget = (size_t)smem_max - 1024;
-    const size_t ctr_bytes = (size_t)p->S * 16;
+    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4) * 16;    // counters and the full-step bitmap
     const size_t psmem_per_warp = ctr_bytes + (size_t)p->U * p->S32 * 4;
     c.psmem = psmem_per_warp <= budget / 2;
     if (c.psmem) {
@@ -394,6 +497,12 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const size_t o_res = take((size_t)(a->chains + 1) * sizeof(kvp_chain_result));
     const size_t o_dump = take(col_bytes), o_sched = take(sched_bytes);
     const size_t o_slots = take(c.psmem ? 0 : (size_t)c.resident * col_bytes);
+    const size_t o_full = take((size_t)p->S32 * 4);
+    // Chains whose schedule lives in shared memory save it to global memory whenever they leave their best state;
+    // chains in global scratch do not (a copy would cost as much as thousands of moves): their winner is replayed.
+    const size_t snap_bytes = (size_t)a->chains * p->U * p->S32 * 4;
+    const bool snapshots = c.psmem && snap_bytes <= ((size_t)2 << 30);
+    const size_t o_snap = take(snapshots ? snap_bytes : 0);
     rc = ensure_chain_ws(p, off);
     if (rc) return rc;
     char* base = static_cast<char*>(p->d_chain_ws);
@@ -401,6 +510,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     c.small = (uint64_t*)(base + o_small); c.table = (uint32_t*)(base + o_table); c.shifts = (uint32_t*)(base + o_shift);
     c.results = (kvp_chain_result*)(base + o_res); c.dumpcol = (uint32_t*)(base + o_dump);
     c.sched = (uint32_t*)(base + o_sched); c.slots = (uint32_t*)(base + o_slots);
+    c.full0 = (uint32_t*)(base + o_full); c.snap = snapshots ? (uint32_t*)(base + o_snap) : nullptr;
 
     // initial schedule in both layouts
     if (a->init_mode == KVP_INIT_USER) {
@@ -422,11 +532,14 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     if ((rc = launch_finish(p, c.counts0, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2), c.small + 1, st)))
         return rc;
     ++c.launches;
+    full_mask_kernel<<<(p->S32 * 32 + 255) / 256, 256, 0, st>>>((const uint4*)c.counts0, p->S, p->cap, c.full0);
+    KVP_CUDA(cudaGetLastError());
+    ++c.launches;
 
     ChainParams& prm = c.prm;
     memset(&prm, 0, sizeof prm);
     prm.Acol = p->dAcol; prm.stepc = p->d_stepc; prm.counters0 = (const uint4*)c.counts0; prm.Pcol0 = c.Pcol0;
-    prm.table = c.table; prm.shifts = c.shifts; prm.ws = c.slots; prm.K = p->K;
+    prm.table = c.table; prm.shifts = c.shifts; prm.ws = c.slots; prm.K = p->K; prm.full0 = c.full0;
     prm.U = p->U; prm.S = p->S; prm.S32 = p->S32; prm.cap = p->cap;
     prm.levels = a->levels; prm.p_swap_256 = a->p_swap_256; prm.len_choices = a->max_len_log2 + 1;
     prm.early_permille = a->early_stop_permille; prm.early_from = a->early_stop_from_level;
@@ -439,7 +552,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const bool calibrate = a->temps == nullptr;
     if (calibrate) {
         KVP_CUDA(cudaMemsetAsync(c.small + 4, 0, 16, st));
-        calib_kernel<<<CALIB_N / 8, 256, 0, st>>>(prm, (unsigned long long*)(c.small + 4));
+        calib_kernel<<<CALIB_N / 256, 256, 0, st>>>(prm, (unsigned long long*)(c.small + 4));
         KVP_CUDA(cudaGetLastError());
         ++c.launches;
     }
@@ -474,7 +587,7 @@ int replay_to_sched(kvp_problem* p, Ctx& c, uint32_t chain, uint64_t upto, kvp_c
         KVP_CUDA(cudaMemcpyAsync(c.sched, c.P0, (size_t)p->S * p->W32 * 4, cudaMemcpyDeviceToDevice, c.st));
         return KVP_OK;
     }
-    if ((rc = run_chains(c, chain, 1, chain, result_dev, upto, c.dumpcol))) return rc;
+    if ((rc = run_chains(c, chain, 1, chain, result_dev, upto, c.dumpcol, nullptr))) return rc;
     if ((rc = launch_bit_transpose(c.dumpcol, p->U, p->S32, p->S, c.sched, p->W32, c.st))) return rc;
     ++c.launches;
     return KVP_OK;
@@ -504,7 +617,7 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     // the chains, one wave of resident chains after the other
     for (uint32_t first = 0; first < a->chains; first += c.resident) {
         const uint32_t count = a->chains - first < c.resident ? a->chains - first : c.resident;
-        if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr))) {
+        if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr, c.snap))) {
             cleanup(); return rc;
         }
     }
@@ -519,8 +632,15 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
     KVP_CUDA(cudaStreamSynchronize(st));
     const uint64_t upto = red.best_move == ~0ull ? 0 : red.best_move + 1;
-    red.best_chain += a->first_chain;                      // the reduction works on call-local indices
-    if ((rc = replay_to_sched(p, c, red.best_chain, upto, c.results + a->chains))) { cleanup(); return rc; }
+    if (c.snap && upto) {                                  // the winner saved its best state itself
+        const uint32_t* col = c.snap + (size_t)red.best_chain * p->U * p->S32;
+        if ((rc = launch_bit_transpose(col, p->U, p->S32, p->S, c.sched, p->W32, st))) { cleanup(); return rc; }
+        ++c.launches;
+        red.best_chain += a->first_chain;                  // the reduction works on call-local indices
+    } else {
+        red.best_chain += a->first_chain;
+        if ((rc = replay_to_sched(p, c, red.best_chain, upto, c.results + a->chains))) { cleanup(); return rc; }
+    }
     if ((rc = launch_counts(p, c.sched, 1, c.counts0, st, &c.launches))) { cleanup(); return rc; }
     if ((rc = launch_finish(p, c.counts0, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2), c.small + 1, st))) {
         cleanup(); return rc;

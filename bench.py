@@ -26,35 +26,47 @@ WORKLOAD = "single_head"
 METRIC = "sa_move_evals_per_sec"
 UNIT = "move-evals/s"
 # Issue-slot roofline of the chain kernel: 148 SMs x 4 warp schedulers x 1.965 GHz, one warp instruction per
-# scheduler and cycle. Algorithmic work per move evaluation in the warp-per-chain form: 100 warp instructions
-# (Philox and decode amortised over 32 lanes ~3, 4 broadcasts, ~80 for the lane-per-step evaluation of
-# Eq. 2-4 twice plus bit extraction, ~5 Metropolis test, ~8 apply and bookkeeping).
+# scheduler and cycle. Algorithmic work per move evaluation with one proposal per lane: 16 warp instructions
+# (per 32 moves: Philox and decode ~105, window extraction and word-parallel bit logic ~100, work-queue scan
+# and push ~100, about 35 (lane, step) cost evaluations of ~70 thread instructions each in two warp rounds
+# ~150, Metropolis and in-order commit ~50).
 ISSUE_PEAK_GWIPS = 148 * 4 * 1.965
-ALG_WARP_INSTR_PER_MOVE = 100.0
+ALG_WARP_INSTR_PER_MOVE = 16.0
 
 
 def _clock_sampler(stop, samples):
-    q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-    idx = os.environ.get("LOCAL_RANK", "0")
+    """SM clock and throttle reasons of this rank's GPU through NVML, every 20 ms while the timed region runs."""
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+        idx = int(os.environ.get("LOCAL_RANK", "0"))
+        if visible:
+            idx = int(visible.split(",")[idx])
+        h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+        smax = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+    except Exception:
+        return
+    bits = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
     while not stop.is_set():
         try:
-            out = subprocess.run(["nvidia-smi", "-i", idx, f"--query-gpu={q}", "--format=csv,noheader,nounits"],
-                                 capture_output=True, text=True, timeout=5).stdout.strip().split("\n")[0]
-            f = [x.strip() for x in out.split(",")]
-            samples.append((float(f[0]), float(f[1]), f[2:6]))
+            sm = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+            try:
+                r = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+            except Exception:
+                r = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+            samples.append((float(sm), float(smax), [n for b, n in bits.items() if r & b]))
         except Exception:
             pass
-        stop.wait(0.2)
+        stop.wait(0.02)
 
 
 def _clock_summary(samples):
     if not samples:
         return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
     sm = sorted(s[0] for s in samples)
-    names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-    reasons = sorted({n for s in samples for n, v in zip(names, s[2]) if v.lower().startswith("active")})
-    return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": samples[0][1], "reasons": reasons}
+    return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": samples[0][1], "samples": len(samples),
+            "reasons": sorted({n for s in samples for n in s[2]})}
 
 
 def run_reference(args):
@@ -160,9 +172,9 @@ def main():
         prob.eval(scheds_dev, want_steps=False)
         prm = prob.make_params(chains=chains, moves=moves, seed=seed, p0=cfg["p0"], first_chain=rank * chains)
         out = prob.anneal(prm)
-        # kernels: 1 trace + 6 create (clean, popcount, transpose, unit counts, histogram, static row)
-        #          + 2 eval (count, finish) + those kvp_anneal reports
-        launches[0] = 1 + 6 + 2 + out["stats"].kernel_launches
+        # kernels: 2 trace (scores, select) + 6 create (clean, popcount, transpose, unit counts, histogram,
+        #          static row) + 2 eval (count, finish) + those kvp_anneal reports
+        launches[0] = 2 + 6 + 2 + out["stats"].kernel_launches
         prob.close()
         return out
 

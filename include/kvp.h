@@ -98,7 +98,9 @@ int kvp_create(kvp_problem** out, uint32_t units, uint64_t bytes_per_unit, uint3
                const kvp_memsys* mem, const uint32_t* hw_units, const uint32_t* ew_units,
                void* stream);
 
-/* Frees the handle and every device buffer it owns. NULL is allowed. */
+/* Frees the handle and every device buffer it owns, in stream order behind the last call made on the
+ * problem (that stream must still exist). NULL is allowed. Device memory comes from CUDA's stream-ordered
+ * allocator; the library sets the default pool's release threshold to 1 GiB on first use of a device. */
 void kvp_destroy(kvp_problem* p);
 
 /* Fills *info (host). */
@@ -132,8 +134,8 @@ int kvp_eval_counts(kvp_problem* p, const uint32_t* schedules, uint32_t n,
  * kvp_eval_noalloc -- kvp_eval for callers that must not allocate device memory. (The paper has no
  * counterpart; this is a service of this library.)
  *
- * kvp_eval keeps its per-step cardinalities in a scratch buffer that it grows with cudaFree/cudaMalloc
- * whenever a batch is larger than any before. That is unwelcome in three situations: inside a serving or
+ * kvp_eval keeps its per-step cardinalities in a scratch buffer that it re-allocates whenever a batch is
+ * larger than any before. That is unwelcome in three situations: inside a serving or
  * control loop where an allocation would stall the whole device for a moment; in a process whose
  * framework has claimed all device memory for its own pool, so that a raw cudaMalloc fails; and in code
  * that is not allowed to call the allocator at all at that point. This variant takes the same arguments
@@ -271,10 +273,13 @@ typedef struct {
     int32_t  sigma_q;     /* std of x_0 * 2^16, 0..2^20                              */
     int32_t  burst_jump;  /* Q16.16 jump added to x_t when a burst fires             */
     uint32_t burst_thr;   /* burst probability * 2^32 (0 = no bursts)                */
-    uint32_t reserved;    /* must be 0                                               */
+    uint32_t flags;       /* KVP_TRACE_*                                             */
     const int32_t* base;  /* (device) [groups*units_per_group] static log-importance, or NULL = 0;
                              |base| <= 2^29                                          */
 } kvp_trace_params;
+
+#define KVP_TRACE_SINGLE_PASS 1u /* never allocate the [steps][units] int32 score matrix (the default does when it
+                                    is at most 1 GiB, stream-ordered and freed on return); slower for few groups */
 
 /*
  * kvp_trace_generate -- fill access_bitmaps (device) [steps][ceil(U/32)] with the

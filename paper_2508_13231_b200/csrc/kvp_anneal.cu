@@ -80,18 +80,23 @@ __device__ __forceinline__ uint32_t window(Ptr col, uint32_t S32, uint32_t s0)
     return __funnelshift_r(lo, hi, b0 & 31u);
 }
 
+constexpr uint32_t kAccSlots4 = 8;       // 32 ints
+constexpr uint32_t kQueueSlots4 = 124;   // 32 * 31 uint16 items = 1984 bytes
+
 struct ChainView {               // where a chain's state lives
     uint32_t* P;                 // [U][S32] schedule, time-packed (shared or global)
     uint4* ctr;                  // [S] {hr, mi, mo, occ} (shared)
     uint32_t* full;              // [S32] bit t set iff occ[t] == cap (shared)
+    int* acc;                    // [32] per-lane cost change being summed (shared)
+    uint16_t* queue;             // [32 * 31] work items (lane << 5 | window bit) of the current batch (shared)
 };
 
-// Evaluate one proposal against the current state, all in the calling lane. Word-parallel over the <= 31
-// affected steps for everything that is a bit; Eq. 2-4 are re-evaluated only at steps whose cardinalities change.
-template <typename PPtr, typename CPtr, typename FPtr>
-__device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ Acol, CPtr ctr, FPtr full,
-                                          const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
-                                          const uint32_t* __restrict__ trow, uint32_t shift, LaneMove& mv)
+// First half of evaluating a proposal, all in the calling lane and word-parallel over the <= 31 affected
+// steps: the windows before and after the move, feasibility (Eq. 5), whether any bit changes, and the set
+// of window bits (steps) whose cardinalities, hence cost, change.
+template <typename PPtr, typename FPtr>
+__device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restrict__ Acol, FPtr full, uint32_t S,
+                                                 uint32_t S32, LaneMove& mv)
 {
     const bool swap = mv.pk & 1u;
     const uint32_t len = (mv.pk >> 1) & 63u, s0 = mv.pk >> 8;
@@ -117,37 +122,104 @@ __device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ A
     mv.Wu = Wu; mv.Wv = Wv; mv.Nu = Nu; mv.Nv = Nv; mv.Au = Au; mv.Av = Av;
     mv.chg = D != 0;
     mv.inf = false;
-    mv.delta = 0;
     if (!swap) {                                                  // a flip may not raise a full step (Eq. 5)
         const uint32_t Fw = window(full, S32, s0);
         mv.inf = (~Wu & M & Fw) != 0;
     }
-    const uint32_t up = Nu & ~Wu, um = Wu & ~Nu;                  // bits u gains / loses (v: the reverse)
-    const uint32_t hrP = (Au & ~Av & up) | (Av & ~Au & um);       // steps whose HBM hit count rises / falls by one
-    const uint32_t hrN = (Au & ~Av & um) | (Av & ~Au & up);
-    const uint32_t miuo = Wu & ~(Wu << 1), miun = Nu & ~(Nu << 1), mivo = Wv & ~(Wv << 1), mivn = Nv & ~(Nv << 1);
-    const uint32_t mouo = ~Wu & (Wu << 1), moun = ~Nu & (Nu << 1), movo = ~Wv & (Wv << 1), movn = ~Nv & (Nv << 1);
-    uint32_t todo = ((miuo ^ miun) | (mivo ^ mivn) | (mouo ^ moun) | (movo ^ movn) | hrP | hrN) & Sb;
-    if (mv.inf) todo = 0;
+    const uint32_t hr = (Au ^ Av) & (Wu ^ Nu);                    // a hit is won or lost (v mirrors u in a swap)
+    // migrations of a unit at step t are the edges p[t] != p[t-1] (into HBM when p[t] is set, out otherwise):
+    // the counts change where an edge appears, disappears or turns around
+    const uint32_t euo = Wu ^ (Wu << 1), eun = Nu ^ (Nu << 1), evo = Wv ^ (Wv << 1), evn = Nv ^ (Nv << 1);
+    const uint32_t mg = (euo ^ eun) | (euo & eun & (Wu ^ Nu)) | (evo ^ evn) | (evo & evn & (Wv ^ Nv));
+    return mv.inf ? 0u : ((hr | mg) & Sb);
+}
+
+// Cost change of the step at window bit k (Eq. 2-4 before and after), from the six windows of a proposal.
+__device__ __forceinline__ int item_delta(uint32_t Wu, uint32_t Wv, uint32_t Nu, uint32_t Nv, uint32_t Au, uint32_t Av,
+                                          uint32_t k, const uint4 c4, const StepC c, const CostK K)
+{
+    const uint32_t pu = (Wu >> k) & 1u, qu = (Wu >> (k - 1)) & 1u, npu = (Nu >> k) & 1u, nqu = (Nu >> (k - 1)) & 1u;
+    const uint32_t pv = (Wv >> k) & 1u, qv = (Wv >> (k - 1)) & 1u, npv = (Nv >> k) & 1u, nqv = (Nv >> (k - 1)) & 1u;
+    const uint32_t au = (Au >> k) & 1u, av = (Av >> k) & 1u;
+    const uint32_t hr = c4.x + (au & npu) - (au & pu) + (av & npv) - (av & pv);
+    const uint32_t mi = c4.y + (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
+    const uint32_t mo = c4.z + (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
+    return (int)(step_cost(hr, mi, mo, c, K) - step_cost(c4.x, c4.y, c4.z, c, K));
+}
+
+__device__ __forceinline__ bool metropolis(int delta, uint32_t w, const uint32_t* __restrict__ trow, uint32_t shift)
+{
+    if (delta <= 0) return true;
+    const uint32_t q = (uint32_t)delta >> shift;
+    return q < KVP_TABLE_Q && w < __ldg(trow + q);                // quantised exp(-delta/C)
+}
+
+// Whole evaluation in one lane (used where there is no warp to share the work with: calibration).
+template <typename PPtr, typename CPtr, typename FPtr>
+__device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ Acol, CPtr ctr, FPtr full,
+                                          const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
+                                          const uint32_t* __restrict__ trow, uint32_t shift, LaneMove& mv)
+{
+    uint32_t todo = lane_windows(P, Acol, full, S, S32, mv);
+    const uint32_t s0 = mv.pk >> 8;
     int delta = 0;
     while (todo) {
         const uint32_t k = __ffs(todo) - 1;
         todo &= todo - 1;
         const uint32_t t = s0 + k - 1;
-        const uint4 c4 = ctr[t];
-        const StepC c = __ldg(stepc + t);
-        const int dhr = (int)((hrP >> k) & 1u) - (int)((hrN >> k) & 1u);
-        const int dmi = (int)(((miun >> k) & 1u) + ((mivn >> k) & 1u)) - (int)(((miuo >> k) & 1u) + ((mivo >> k) & 1u));
-        const int dmo = (int)(((moun >> k) & 1u) + ((movn >> k) & 1u)) - (int)(((mouo >> k) & 1u) + ((movo >> k) & 1u));
-        delta += (int)(step_cost(c4.x + dhr, c4.y + dmi, c4.z + dmo, c, K) - step_cost(c4.x, c4.y, c4.z, c, K));
+        delta += item_delta(mv.Wu, mv.Wv, mv.Nu, mv.Nv, mv.Au, mv.Av, k, ctr[t], __ldg(stepc + t), K);
     }
     mv.delta = delta;
-    bool acc = delta <= 0;
-    if (!acc) {
-        const uint32_t q = (uint32_t)delta >> shift;
-        acc = q < KVP_TABLE_Q && mv.w < __ldg(trow + q);          // Metropolis, quantised exp(-delta/C)
+    mv.acc = metropolis(delta, mv.w, trow, shift);
+}
+
+// Evaluation of the proposals of the lanes in `need`, shared by the warp: every lane prepares its own
+// proposal, the (lane, step) pairs whose cost changes are queued in shared memory, and the warp works the
+// queue off 32 pairs at a time, so that lanes with short and long proposals carry the same load.
+__device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* __restrict__ Acol,
+                                           const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
+                                           const uint32_t* __restrict__ trow, uint32_t shift, uint32_t need,
+                                           uint32_t lane, LaneMove& mv)
+{
+    const bool mine = (need >> lane) & 1u;
+    uint32_t todo = 0;
+    if (mine) {
+        todo = lane_windows(cv.P, Acol, cv.full, S, S32, mv);
+        cv.acc[lane] = 0;
     }
-    mv.acc = acc;
+    const uint32_t cnt = __popc(todo);
+    uint32_t incl = cnt;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= (uint32_t)off) incl += o;
+    }
+    const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    uint32_t pos = incl - cnt;
+    while (todo) {
+        const uint32_t k = __ffs(todo) - 1;
+        todo &= todo - 1;
+        cv.queue[pos++] = (uint16_t)((lane << 5) | k);
+    }
+    __syncwarp();
+    for (uint32_t base = 0; base < total; base += 32) {
+        const uint32_t g = base + lane;
+        const bool live = g < total;
+        const uint32_t item = live ? cv.queue[g] : 1u;            // a dead lane works on (lane 0, bit 1) and drops it
+        const uint32_t o = item >> 5, k = item & 31u;
+        const uint32_t Wu = __shfl_sync(0xFFFFFFFFu, mv.Wu, o), Wv = __shfl_sync(0xFFFFFFFFu, mv.Wv, o);
+        const uint32_t Nu = __shfl_sync(0xFFFFFFFFu, mv.Nu, o), Nv = __shfl_sync(0xFFFFFFFFu, mv.Nv, o);
+        const uint32_t Au = __shfl_sync(0xFFFFFFFFu, mv.Au, o), Av = __shfl_sync(0xFFFFFFFFu, mv.Av, o);
+        const uint32_t s0 = __shfl_sync(0xFFFFFFFFu, mv.pk, o) >> 8;
+        const uint32_t t = min(s0 + k - 1, S - 1);
+        const int d = item_delta(Wu, Wv, Nu, Nv, Au, Av, k, cv.ctr[t], __ldg(stepc + t), K);
+        if (live && d) atomicAdd(cv.acc + o, d);
+    }
+    __syncwarp();
+    if (mine) {
+        mv.delta = cv.acc[lane];
+        mv.acc = metropolis(mv.delta, mv.w, trow, shift);
+    }
 }
 
 // Apply the proposal held by lane `b`: all lanes take part, lane j updates the counters of window bit j.
@@ -222,10 +294,13 @@ chain_kernel(const ChainParams prm)
     const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
     const size_t pwords = (size_t)U * S32;
     const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
+    const uint32_t fixed4 = S + f4 + kAccSlots4 + kQueueSlots4;   // per-warp shared state besides the schedule
     ChainView cv;
-    cv.ctr = smem4 + (size_t)warp * (S + f4);
+    cv.ctr = smem4 + (size_t)warp * fixed4;
     cv.full = reinterpret_cast<uint32_t*>(cv.ctr + S);
-    cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)wpb * (S + f4)) + (size_t)warp * pwords
+    cv.acc = reinterpret_cast<int*>(cv.ctr + S + f4);
+    cv.queue = reinterpret_cast<uint16_t*>(cv.ctr + S + f4 + kAccSlots4);
+    cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)wpb * fixed4) + (size_t)warp * pwords
                  : prm.ws + (size_t)slot * pwords;
     for (uint32_t i = lane; i < S; i += 32) cv.ctr[i] = __ldg(prm.counters0 + i);
     for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
@@ -268,9 +343,7 @@ chain_kernel(const ChainParams prm)
         uint32_t todo = nb == 32 ? 0xFFFFFFFFu : (1u << nb) - 1u;
         uint32_t need = todo;
         while (todo) {
-            if ((need >> lane) & 1u)
-                eval_lane(cv.P, prm.Acol, cv.ctr, cv.full, prm.stepc, prm.K, S, S32, trow, shift, mv);
-            __syncwarp();
+            if (need) eval_batch(cv, prm.Acol, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
             const uint32_t infb = __ballot_sync(0xFFFFFFFFu, mv.inf);
             const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !mv.inf && mv.acc);
             const uint32_t blk = __ballot_sync(0xFFFFFFFFu, !mv.inf && mv.acc && mv.chg) & todo;
@@ -453,7 +526,8 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     KVP_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     KVP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const size_t budget = (size_t)smem_max - 1024;
-    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4) * 16;    // counters and the full-step bitmap
+    // per warp: counters, full-step bitmap, 32 accumulators, the work queue
+    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4 + kAccSlots4 + kQueueSlots4) * 16;
     const size_t psmem_per_warp = ctr_bytes + (size_t)p->U * p->S32 * 4;
     c.psmem = psmem_per_warp <= budget / 2;
     if (c.psmem) {
@@ -479,6 +553,13 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
         size_t free_b = 0, total_b = 0;
         KVP_CUDA(cudaMemGetInfo(&free_b, &total_b));
         free_b += p->chain_ws_bytes;                               // what we already hold can be reused
+        {                                                          // and so can what the pool holds in reserve
+            cudaMemPool_t pool; uint64_t reserved = 0, used = 0;
+            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess &&
+                cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReservedMemCurrent, &reserved) == cudaSuccess &&
+                cudaMemPoolGetAttribute(pool, cudaMemPoolAttrUsedMemCurrent, &used) == cudaSuccess && reserved > used)
+                free_b += (size_t)(reserved - used);
+        }
         const size_t usable = free_b / 10 * 7;
         size_t fit = usable / col_bytes;
         if (fit < 1) return KVP_ERR_NOMEM;
@@ -503,7 +584,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const size_t snap_bytes = (size_t)a->chains * p->U * p->S32 * 4;
     const bool snapshots = c.psmem && snap_bytes <= ((size_t)2 << 30);
     const size_t o_snap = take(snapshots ? snap_bytes : 0);
-    rc = ensure_chain_ws(p, off);
+    rc = ensure_chain_ws(p, off, st);
     if (rc) return rc;
     char* base = static_cast<char*>(p->d_chain_ws);
     c.P0 = (uint32_t*)(base + o_P0); c.Pcol0 = (uint32_t*)(base + o_col0); c.counts0 = (uint32_t*)(base + o_cnt);

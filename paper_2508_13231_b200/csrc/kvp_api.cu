@@ -19,18 +19,40 @@ int set_cuda_error(cudaError_t e, const char* what)
     return e == cudaErrorMemoryAllocation ? KVP_ERR_NOMEM : KVP_ERR_CUDA;
 }
 
-static int grow(void** ptr, size_t* have, size_t want)
+// All device memory comes from the stream-ordered allocator: a create/anneal/destroy cycle then costs no
+// device-wide synchronisation. The default pool is told once per device to keep up to 1 GiB of freed memory.
+static int prepare_pool(int device)
+{
+    static bool done[64];
+    if (device < 0 || device >= 64 || done[device]) return KVP_OK;
+    cudaMemPool_t pool;
+    KVP_CUDA(cudaDeviceGetDefaultMemPool(&pool, device));
+    uint64_t keep = 1ull << 30;
+    KVP_CUDA(cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep));
+    done[device] = true;
+    return KVP_OK;
+}
+
+static int grow(void** ptr, size_t* have, size_t want, cudaStream_t st)
 {
     if (*have >= want) return KVP_OK;
-    if (*ptr) { KVP_CUDA(cudaFree(*ptr)); *ptr = nullptr; *have = 0; }
+    if (*ptr) { KVP_CUDA(cudaFreeAsync(*ptr, st)); *ptr = nullptr; *have = 0; }
     size_t bytes = (want + 255) & ~(size_t)255;
-    KVP_CUDA(cudaMalloc(ptr, bytes));
+    KVP_CUDA(cudaMallocAsync(ptr, bytes, st));
     *have = bytes;
     return KVP_OK;
 }
 
-int ensure_scratch(kvp_problem* p, size_t bytes) { return grow(&p->d_scratch, &p->scratch_bytes, bytes); }
-int ensure_chain_ws(kvp_problem* p, size_t bytes) { return grow(&p->d_chain_ws, &p->chain_ws_bytes, bytes); }
+int ensure_scratch(kvp_problem* p, size_t bytes, cudaStream_t st)
+{
+    p->last_stream = st;
+    return grow(&p->d_scratch, &p->scratch_bytes, bytes, st);
+}
+int ensure_chain_ws(kvp_problem* p, size_t bytes, cudaStream_t st)
+{
+    p->last_stream = st;
+    return grow(&p->d_chain_ws, &p->chain_ws_bytes, bytes, st);
+}
 
 static uint64_t gcd_u64(uint64_t a, uint64_t b)
 {
@@ -64,22 +86,29 @@ extern "C" void kvp_destroy(kvp_problem* p)
 {
     if (!p) return;
     cudaSetDevice(p->device);
-    cudaFree(p->dA); cudaFree(p->dAcol); cudaFree(p->d_a); cudaFree(p->d_stepc); cudaFree(p->d_ucnt);
-    cudaFree(p->d_row_freq); cudaFree(p->d_scratch); cudaFree(p->d_chain_ws);
+    // freed in stream order behind the last work queued for this problem
+    if (p->d_block) cudaFreeAsync(p->d_block, p->last_stream);
+    if (p->d_scratch) cudaFreeAsync(p->d_scratch, p->last_stream);
+    if (p->d_chain_ws) cudaFreeAsync(p->d_chain_ws, p->last_stream);
     delete p;
 }
 
 static int create_impl(kvp_problem* p, const uint32_t* access, const uint32_t* hw, const uint32_t* ew, cudaStream_t st)
 {
     const size_t nw = (size_t)p->S * p->W32;
-    KVP_CUDA(cudaMalloc(&p->dA, nw * 4));
-    KVP_CUDA(cudaMalloc(&p->dAcol, (size_t)p->U * p->S32 * 4));
-    KVP_CUDA(cudaMalloc(&p->d_a, (size_t)p->S * 4));
-    KVP_CUDA(cudaMalloc(&p->d_stepc, (size_t)p->S * sizeof(StepC)));
-    KVP_CUDA(cudaMalloc(&p->d_ucnt, (size_t)p->U * 4));
-    KVP_CUDA(cudaMalloc(&p->d_row_freq, (size_t)p->W32 * 4));
-    int rc = ensure_scratch(p, (size_t)(p->S + 1) * 16);
+    int rc = prepare_pool(p->device);
     if (rc) return rc;
+    p->last_stream = st;
+    // one block for everything the problem keeps
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) & ~(size_t)255; return o; };
+    const size_t oA = take(nw * 4), oAcol = take((size_t)p->U * p->S32 * 4), oa = take((size_t)p->S * 4);
+    const size_t osc = take((size_t)p->S * sizeof(StepC)), ouc = take((size_t)p->U * 4), orf = take((size_t)p->W32 * 4);
+    KVP_CUDA(cudaMallocAsync(&p->d_block, off, st));
+    char* base = static_cast<char*>(p->d_block);
+    p->dA = (uint32_t*)(base + oA); p->dAcol = (uint32_t*)(base + oAcol); p->d_a = (uint32_t*)(base + oa);
+    p->d_stepc = (StepC*)(base + osc); p->d_ucnt = (uint32_t*)(base + ouc); p->d_row_freq = (uint32_t*)(base + orf);
+    if ((rc = ensure_scratch(p, (size_t)(p->S + 1) * 16, st))) return rc;
     if ((rc = launch_clean_copy(access, p->dA, p->S, p->W32, p->pad_mask, st))) return rc;
     if ((rc = launch_row_popcount(p->dA, p->S, p->W32, p->d_a, st))) return rc;
     if ((rc = launch_bit_transpose(p->dA, p->S, p->W32, p->U, p->dAcol, p->S32, st))) return rc;

@@ -77,6 +77,8 @@ struct kvp_problem {
     uint32_t* d_ucnt;    // [U]        accesses per unit over all steps
     uint32_t* d_row_freq;// [W32]      STATIC_FREQ row
     uint64_t total_accessed;
+    void* d_block;             // one allocation behind the pointers above
+    cudaStream_t last_stream;  // stream of the most recent call; frees are ordered behind it
     // scratch owned by the problem, grown on demand
     void* d_scratch; size_t scratch_bytes;
     void* d_chain_ws; size_t chain_ws_bytes;
@@ -91,8 +93,8 @@ int set_cuda_error(cudaError_t e, const char* what);
         if (e_ != cudaSuccess) return kvp::set_cuda_error(e_, #call);    \
     } while (0)
 
-int ensure_scratch(kvp_problem* p, size_t bytes);
-int ensure_chain_ws(kvp_problem* p, size_t bytes);
+int ensure_scratch(kvp_problem* p, size_t bytes, cudaStream_t st);
+int ensure_chain_ws(kvp_problem* p, size_t bytes, cudaStream_t st);
 
 // kvp_cost.cu
 int launch_row_popcount(const uint32_t* rows, uint32_t S, uint32_t W32, uint32_t* out, cudaStream_t st);

@@ -261,7 +261,7 @@ extern "C" int kvp_eval(kvp_problem* p, const uint32_t* schedules, uint32_t n, u
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t slice = n < kBatchSlice ? n : kBatchSlice;
-    int rc = kvp::ensure_scratch(p, (size_t)slice * p->S * 16);
+    int rc = kvp::ensure_scratch(p, (size_t)slice * p->S * 16, st);
     if (rc) return rc;
     uint32_t* counts = static_cast<uint32_t*>(p->d_scratch);
     const size_t sched_words = (size_t)p->S * p->W32;

@@ -1,7 +1,8 @@
-// Trace kernel: synthetic importance per unit and step, top-k per (layer, kv-head) group, packed into uint32
-// bitmaps. One CTA per group walks the steps in order (the AR(1) recurrence is sequential in time); the
-// importance state of a unit lives in a register of the thread that owns it. The k-th largest score of a step
-// is found by a 32-round bitwise binary search with block-wide counts, ties go to the lower unit index.
+// Trace kernels: synthetic importance per unit and step, top-k per (layer, kv-head) group, packed into uint32
+// bitmaps. Two passes by default: one thread per unit runs the AR(1) recurrence over all steps (sequential in
+// time) and writes a score matrix; then one CTA per (group, step) finds the k-th largest score with a 32-round
+// bitwise binary search over block-wide counts, ties going to the lower unit index. A fused single-pass form
+// (one CTA per group, state in registers) serves traces whose score matrix would exceed the scratch budget.
 #include "kvp_common.cuh"
 
 namespace kvp {
@@ -37,15 +38,92 @@ __device__ __forceinline__ uint32_t block_sum(uint32_t v, uint32_t* slot)
     return *slot;
 }
 
+struct SelectSmem {
+    uint32_t cnt[36];            // 32 search rounds + 2 extra counts
+    uint32_t warp[32];
+    uint32_t run;
+};
+
+// Top-k of one (group, step): the CTA holds the n keys (UPT per thread, unit i = j*T + tid) and sets the
+// bits of the k largest, ties to the lower unit index. sm.cnt must be zero on entry (and a barrier passed).
+template <int UPT>
+__device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const TraceK& k, uint32_t gbase, uint32_t t,
+                                            SelectSmem& sm)
+{
+    const uint32_t T = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // largest K with |{key >= K}| >= topk, bit by bit from the top
+    uint32_t K = 0;
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t cand = K | (1u << bit);
+        uint32_t c = 0;
+#pragma unroll
+        for (int j = 0; j < UPT; ++j) c += (j * T + tid < k.n && key[j] >= cand) ? 1u : 0u;
+        if (block_sum(c, &sm.cnt[31 - bit]) >= k.topk) K = cand;
+    }
+    uint32_t cg = 0, ce = 0;
+#pragma unroll
+    for (int j = 0; j < UPT; ++j) {
+        const bool ok = j * T + tid < k.n;
+        cg += (ok && key[j] > K) ? 1u : 0u;
+        ce += (ok && key[j] == K) ? 1u : 0u;
+    }
+    const uint32_t above = block_sum(cg, &sm.cnt[32]);
+    const uint32_t equal = block_sum(ce, &sm.cnt[33]);
+    const uint32_t take = k.topk - above;                    // ties to admit, lowest unit index first
+    const bool rank_ties = equal != take;
+    if (tid == 0) sm.run = 0;
+    __syncthreads();
+    uint32_t* row = k.out + (size_t)t * k.W32;
+#pragma unroll
+    for (int j = 0; j < UPT; ++j) {
+        const uint32_t i = j * T + tid;
+        const bool ok = i < k.n;
+        const bool tie = ok && key[j] == K;
+        bool pick = ok && key[j] > K;
+        if (!rank_ties) {
+            pick = pick || tie;
+        } else {
+            // units of round j are consecutive over the CTA, so index order = (round, thread) order
+            const uint32_t tb = __ballot_sync(0xFFFFFFFFu, tie);
+            if (lane == 0) sm.warp[warp] = __popc(tb);
+            __syncthreads();
+            uint32_t before = sm.run;
+            for (uint32_t w = 0; w < warp; ++w) before += sm.warp[w];
+            before += __popc(tb & ((1u << lane) - 1u));
+            pick = pick || (tie && before < take);
+            __syncthreads();
+            if (tid == 0) { uint32_t s = 0; for (uint32_t w = 0; w < (T >> 5); ++w) s += sm.warp[w]; sm.run += s; }
+            __syncthreads();
+        }
+        if (k.aligned) {
+            const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
+            if (lane == 0 && j * T + (tid & ~31u) < k.n) row[(gbase + j * T + tid) >> 5] = bits;
+        } else if (pick) {
+            atomicOr(row + ((gbase + i) >> 5), 1u << ((gbase + i) & 31));
+        }
+    }
+}
+
+// importance of unit u at step t given its state at t-1 (Q16.16)
+__device__ __forceinline__ int32_t next_state(const TraceK& k, uint32_t u, uint32_t t, int32_t x)
+{
+    const int64_t e = noise_q16(k.seed_lo, k.seed_hi, u, t);
+    int64_t xn = t == 0 ? ((int64_t)k.sigma_q * e) >> 16 : ((int64_t)k.rho_q * (int64_t)x + (int64_t)k.c_q * e) >> 16;
+    if (k.burst_thr) {
+        uint32_t r[4];
+        philox4x32_10(u, t, 0u, TAG_BURST, k.seed_lo, k.seed_hi, r);
+        if (r[0] < k.burst_thr) xn += k.burst_jump;
+    }
+    return (int32_t)xn;
+}
+
+// Fused form: one CTA per group walks the steps; used when the score matrix would not fit the scratch budget.
 template <int UPT>
 __global__ void __launch_bounds__(1024)
 trace_kernel(const TraceK k)
 {
-    __shared__ uint32_t s_cnt[36];           // 32 search rounds + 2 extra counts
-    __shared__ uint32_t s_warp[32];
-    __shared__ uint32_t s_run;
+    __shared__ SelectSmem sm;
     const uint32_t g = blockIdx.x, T = blockDim.x, tid = threadIdx.x;
-    const uint32_t lane = tid & 31, warp = tid >> 5;
     const uint32_t gbase = g * k.n;
     int32_t x[UPT], b[UPT];
 #pragma unroll
@@ -55,80 +133,55 @@ trace_kernel(const TraceK k)
         b[j] = (i < k.n && k.base) ? __ldg(k.base + gbase + i) : 0;
     }
     for (uint32_t t = 0; t < k.steps; ++t) {
-        for (uint32_t i = tid; i < 36; i += T) s_cnt[i] = 0;
+        for (uint32_t i = tid; i < 36; i += T) sm.cnt[i] = 0;
         uint32_t key[UPT];
 #pragma unroll
         for (int j = 0; j < UPT; ++j) {
             const uint32_t i = j * T + tid;
             key[j] = 0;
             if (i < k.n) {
-                const uint32_t u = gbase + i;
-                const int64_t e = noise_q16(k.seed_lo, k.seed_hi, u, t);
-                int64_t xn = t == 0 ? ((int64_t)k.sigma_q * e) >> 16
-                                    : ((int64_t)k.rho_q * (int64_t)x[j] + (int64_t)k.c_q * e) >> 16;
-                if (k.burst_thr) {
-                    uint32_t r[4];
-                    philox4x32_10(u, t, 0u, TAG_BURST, k.seed_lo, k.seed_hi, r);
-                    if (r[0] < k.burst_thr) xn += k.burst_jump;
-                }
-                x[j] = (int32_t)xn;
+                x[j] = next_state(k, gbase + i, t, x[j]);
                 key[j] = (uint32_t)(x[j] + b[j]) ^ 0x80000000u;       // order-preserving map int32 -> uint32
             }
         }
         __syncthreads();
-        // largest K with |{key >= K}| >= topk, bit by bit from the top
-        uint32_t K = 0;
-        for (int bit = 31; bit >= 0; --bit) {
-            const uint32_t cand = K | (1u << bit);
-            uint32_t c = 0;
-#pragma unroll
-            for (int j = 0; j < UPT; ++j) c += (j * T + tid < k.n && key[j] >= cand) ? 1u : 0u;
-            if (block_sum(c, &s_cnt[31 - bit]) >= k.topk) K = cand;
-        }
-        uint32_t cg = 0, ce = 0;
-#pragma unroll
-        for (int j = 0; j < UPT; ++j) {
-            const bool ok = j * T + tid < k.n;
-            cg += (ok && key[j] > K) ? 1u : 0u;
-            ce += (ok && key[j] == K) ? 1u : 0u;
-        }
-        const uint32_t above = block_sum(cg, &s_cnt[32]);
-        const uint32_t equal = block_sum(ce, &s_cnt[33]);
-        const uint32_t take = k.topk - above;                // ties to admit, lowest unit index first
-        const bool rank_ties = equal != take;
-        if (tid == 0) s_run = 0;
-        __syncthreads();
-        uint32_t* row = k.out + (size_t)t * k.W32;
-#pragma unroll
-        for (int j = 0; j < UPT; ++j) {
-            const uint32_t i = j * T + tid;
-            const bool ok = i < k.n;
-            const bool tie = ok && key[j] == K;
-            bool pick = ok && key[j] > K;
-            if (!rank_ties) {
-                pick = pick || tie;
-            } else {
-                // units of round j are consecutive over the CTA, so index order = (round, thread) order
-                const uint32_t tb = __ballot_sync(0xFFFFFFFFu, tie);
-                if (lane == 0) s_warp[warp] = __popc(tb);
-                __syncthreads();
-                uint32_t before = s_run;
-                for (uint32_t w = 0; w < warp; ++w) before += s_warp[w];
-                before += __popc(tb & ((1u << lane) - 1u));
-                pick = pick || (tie && before < take);
-                __syncthreads();
-                if (tid == 0) { uint32_t s = 0; for (uint32_t w = 0; w < (T >> 5); ++w) s += s_warp[w]; s_run += s; }
-                __syncthreads();
-            }
-            if (k.aligned) {
-                const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
-                if (lane == 0 && j * T + (tid & ~31u) < k.n) row[(gbase + j * T + tid) >> 5] = bits;
-            } else if (pick) {
-                atomicOr(row + ((gbase + i) >> 5), 1u << ((gbase + i) & 31));
-            }
-        }
+        select_step<UPT>(key, k, gbase, t, sm);
         __syncthreads();
     }
+}
+
+// Two-pass form, pass 1: the AR(1) recurrence is sequential in time but independent across units, so one
+// thread per unit writes the whole score column; scores [steps][U].
+__global__ void __launch_bounds__(128)
+trace_scores_kernel(const TraceK k, uint32_t U, int32_t* __restrict__ scores)
+{
+    const uint32_t u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= U) return;
+    const int32_t b = k.base ? __ldg(k.base + u) : 0;
+    int32_t x = 0;
+    for (uint32_t t = 0; t < k.steps; ++t) {
+        x = next_state(k, u, t, x);
+        scores[(size_t)t * U + u] = x + b;
+    }
+}
+
+// Two-pass form, pass 2: the top-k selections of different steps are independent: one CTA per (group, step).
+template <int UPT>
+__global__ void __launch_bounds__(1024)
+trace_select_kernel(const TraceK k, uint32_t U, const int32_t* __restrict__ scores)
+{
+    __shared__ SelectSmem sm;
+    const uint32_t g = blockIdx.x, t = blockIdx.y, T = blockDim.x, tid = threadIdx.x;
+    const uint32_t gbase = g * k.n;
+    for (uint32_t i = tid; i < 36; i += T) sm.cnt[i] = 0;
+    uint32_t key[UPT];
+#pragma unroll
+    for (int j = 0; j < UPT; ++j) {
+        const uint32_t i = j * T + tid;
+        key[j] = i < k.n ? (uint32_t)__ldg(scores + (size_t)t * U + gbase + i) ^ 0x80000000u : 0u;
+    }
+    __syncthreads();
+    select_step<UPT>(key, k, gbase, t, sm);
 }
 
 }  // namespace
@@ -139,7 +192,8 @@ using namespace kvp;
 
 extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_bitmaps, void* stream)
 {
-    if (!tp || !access_bitmaps || !tp->groups || !tp->units_per_group || !tp->steps || tp->reserved) return KVP_ERR_ARG;
+    if (!tp || !access_bitmaps || !tp->groups || !tp->units_per_group || !tp->steps || (tp->flags & ~KVP_TRACE_SINGLE_PASS))
+        return KVP_ERR_ARG;
     if (!tp->topk || tp->topk > tp->units_per_group) return KVP_ERR_ARG;
     if (tp->rho_q < 0 || tp->rho_q > 65536 || tp->c_q < 0 || tp->c_q > (1 << 20) || tp->sigma_q < 0 ||
         tp->sigma_q > (1 << 20))
@@ -168,6 +222,25 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
     const int upt = n <= 1024 ? 1 : n <= 2048 ? 2 : n <= 4096 ? 4 : 8;
     uint32_t T = (n + upt - 1) / upt;
     T = (T + 31) / 32 * 32;
+    // Two passes (scores, then one CTA per (group, step)) whenever the score matrix fits a 1 GiB scratch:
+    // the fused kernel has only `groups` CTAs and walks the steps one after the other.
+    const size_t score_bytes = (size_t)U64 * tp->steps * 4;
+    if (score_bytes <= ((size_t)1 << 30) && !(tp->flags & KVP_TRACE_SINGLE_PASS)) {
+        int32_t* scores = nullptr;
+        KVP_CUDA(cudaMallocAsync(&scores, score_bytes, st));
+        trace_scores_kernel<<<(uint32_t)((U64 + 127) / 128), 128, 0, st>>>(k, (uint32_t)U64, scores);
+        dim3 grid(tp->groups, tp->steps);
+        switch (upt) {
+            case 1: trace_select_kernel<1><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
+            case 2: trace_select_kernel<2><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
+            case 4: trace_select_kernel<4><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
+            default: trace_select_kernel<8><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
+        }
+        cudaError_t le = cudaGetLastError();
+        KVP_CUDA(cudaFreeAsync(scores, st));
+        KVP_CUDA(le);
+        return KVP_OK;
+    }
     switch (upt) {
         case 1: trace_kernel<1><<<tp->groups, T, 0, st>>>(k); break;
         case 2: trace_kernel<2><<<tp->groups, T, 0, st>>>(k); break;

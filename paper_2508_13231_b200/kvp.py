@@ -78,7 +78,7 @@ class TraceParams(C.Structure):
     _fields_ = [
         ("groups", C.c_uint32), ("units_per_group", C.c_uint32), ("steps", C.c_uint32), ("topk", C.c_uint32),
         ("seed", C.c_uint64), ("rho_q", C.c_int32), ("c_q", C.c_int32), ("sigma_q", C.c_int32), ("burst_jump", C.c_int32),
-        ("burst_thr", C.c_uint32), ("reserved", C.c_uint32), ("base", C.c_void_p),
+        ("burst_thr", C.c_uint32), ("flags", C.c_uint32), ("base", C.c_void_p),
     ]
 
 
@@ -137,12 +137,16 @@ def accept_table(temps):
     return table, shifts
 
 
+TRACE_SINGLE_PASS = 1
+
+
 def trace_generate(groups, units_per_group, steps, topk, seed, rho_q, c_q, sigma_q, burst_jump=0, burst_thr=0,
-                   base=None, out=None, stream=None):
+                   base=None, out=None, stream=None, flags=0):
     """Synthetic access bitmaps on the current CUDA device -> int32 tensor [steps][ceil(U/32)] (bit pattern uint32)."""
     tp = TraceParams()
     tp.groups, tp.units_per_group, tp.steps, tp.topk, tp.seed = groups, units_per_group, steps, topk, seed
     tp.rho_q, tp.c_q, tp.sigma_q, tp.burst_jump, tp.burst_thr = rho_q, c_q, sigma_q, burst_jump, burst_thr
+    tp.flags = flags
     if base is not None:
         if base.numel() != groups * units_per_group:
             raise ValueError("base must have one entry per unit")

@@ -26,10 +26,10 @@ def both_problems(kvp, oracle, U, bpu, S, A, cap, bw, mig_flags=3, hw=None, ew=N
     return g, o
 
 
-def trace_on_gpu(kvp, tp):
+def trace_on_gpu(kvp, tp, flags=0):
     base = None if tp["base"] is None else torch.from_numpy(tp["base"]).cuda()
     args = {k: v for k, v in tp.items() if k != "base"}
-    return kvp.trace_generate(**args, base=base)
+    return kvp.trace_generate(**args, base=base, flags=flags)
 
 
 def named_problem(kvp, oracle, name, A=None, seed=0):

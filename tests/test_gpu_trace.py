@@ -19,9 +19,9 @@ def kvp():
 @pytest.mark.parametrize("name", ["tiny", "single_head", "layer_8b"])
 def test_trace_named_configs_full(kvp, oracle, name):
     tp = wl.trace_params(name, seed=0)
-    got = to_np(trace_on_gpu(kvp, tp))
     want = oracle.trace_generate(**tp)
-    assert np.array_equal(got, want)
+    assert np.array_equal(to_np(trace_on_gpu(kvp, tp)), want)
+    assert np.array_equal(to_np(trace_on_gpu(kvp, tp, kvp.TRACE_SINGLE_PASS)), want)
 
 
 @pytest.mark.parametrize("name,groups", [("full_8b", [0, 101, 255]), ("long_70b", [0, 317, 639])])
@@ -41,12 +41,13 @@ def test_trace_full_size_sampled_groups(kvp, oracle, name, groups):
 
 @pytest.mark.parametrize("G,n,S,k", [(3, 40, 12, 7), (1, 16, 5, 16), (5, 100, 9, 1), (2, 1024, 6, 100),
                                      (2, 2048 + 64, 4, 33), (1, 8192, 3, 500), (7, 33, 40, 5)])
-def test_trace_ragged_shapes(kvp, oracle, G, n, S, k):
+@pytest.mark.parametrize("flags", [0, 1])          # two passes over a score matrix / single fused pass
+def test_trace_ragged_shapes(kvp, oracle, G, n, S, k, flags):
     rng = np.random.default_rng(G * 1000 + n)
     base = (rng.integers(-3 * Q16, 3 * Q16, size=G * n)).astype(np.int32)
     tp = dict(groups=G, units_per_group=n, steps=S, topk=k, seed=77, rho_q=int(0.9 * Q16), c_q=int(0.4 * Q16),
               sigma_q=Q16, burst_jump=3 * Q16, burst_thr=int(0.05 * 2 ** 32), base=base)
-    assert np.array_equal(to_np(trace_on_gpu(kvp, tp)), oracle.trace_generate(**tp))
+    assert np.array_equal(to_np(trace_on_gpu(kvp, tp, flags)), oracle.trace_generate(**tp))
 
 
 def test_trace_ties_go_to_lower_index(kvp, oracle):
@@ -57,8 +58,10 @@ def test_trace_ties_go_to_lower_index(kvp, oracle):
     tp = dict(groups=G, units_per_group=n, steps=S, topk=k, seed=1, rho_q=Q16, c_q=0, sigma_q=0, burst_jump=0,
               burst_thr=0, base=base)
     assert np.array_equal(to_np(trace_on_gpu(kvp, tp)), oracle.trace_generate(**tp))
+    assert np.array_equal(to_np(trace_on_gpu(kvp, tp, kvp.TRACE_SINGLE_PASS)), oracle.trace_generate(**tp))
     tp = dict(tp, units_per_group=50, groups=3, topk=20, base=base[:150])
     assert np.array_equal(to_np(trace_on_gpu(kvp, tp)), oracle.trace_generate(**tp))
+    assert np.array_equal(to_np(trace_on_gpu(kvp, tp, kvp.TRACE_SINGLE_PASS)), oracle.trace_generate(**tp))
 
 
 def test_trace_argument_errors(kvp):

@@ -41,14 +41,21 @@ struct ChainParams {
     uint64_t per_level, upto, init_ticks;
 };
 
-// A proposal as one lane sees it: the Philox words, and after evaluation the placement windows of its one
-// or two units before (W) and after (N) the move, their access windows (A) and the verdict.
-// Window convention: bit k of a window belongs to step s0 - 1 + k, so bit 0 is the step before the run (for
-// s0 == 0 it repeats step 0, because P[-1] := P[0]), bits 1..run are the run, and the affected steps
-// s0..last are bits 1..nl <= 31. Run lengths stop at 30 so that every vector fits one 32-bit register.
+// Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
+constexpr int kMPL = 1;
+constexpr uint32_t kBatch = 32 * kMPL;
+constexpr uint32_t kWinSlots4 = kBatch * 2;                        // 8 words of windows per proposal
+constexpr uint32_t kAccSlots4 = kBatch / 4;                        // one int per proposal
+constexpr uint32_t kQueueSlots4 = (kBatch * 31 * 2 + 15) / 16;     // uint16 work items, worst case 31 per proposal
+
+// A proposal as its lane keeps it in registers: the Philox words and, after evaluation, the verdict.
+// The placement windows live in shared memory (ChainView::win), 8 words per proposal:
+//   {Wu, Wv, Nu, Nv} = placement of units u, v before (W) and after (N) the move, {Au, Av} = access bits,
+//   then s0. Window convention: bit k belongs to step s0 - 1 + k, so bit 0 is the step before the run (for
+//   s0 == 0 it repeats step 0, because P[-1] := P[0]), bits 1..run are the run, and the affected steps
+//   s0..last are bits 1..nl <= 31. Run lengths stop at 30 so that every vector fits one 32-bit register.
 struct LaneMove {
     uint32_t pk, u, v, w;        // packed (swap | len << 1 | s0 << 8), units, Metropolis uniform
-    uint32_t Wu, Wv, Nu, Nv, Au, Av;
     int delta;
     bool inf, acc, chg;
 };
@@ -71,32 +78,29 @@ __device__ __forceinline__ void decode_move(const uint32_t r[4], uint32_t p_swap
 template <typename Ptr>
 __device__ __forceinline__ uint32_t window(Ptr col, uint32_t S32, uint32_t s0)
 {
-    if (s0 == 0) {
-        const uint32_t raw = col[0];
-        return (raw << 1) | (raw & 1u);
-    }
-    const uint32_t b0 = s0 - 1, w = b0 >> 5;
+    const uint32_t b0 = s0 ? s0 - 1 : 0u, w = b0 >> 5;
     const uint32_t lo = col[w], hi = col[min(w + 1, S32 - 1)];
-    return __funnelshift_r(lo, hi, b0 & 31u);
+    const uint32_t slid = __funnelshift_r(lo, hi, b0 & 31u);
+    return s0 ? slid : ((lo << 1) | (lo & 1u));                  // s0 == 0: bit 0 repeats step 0
 }
-
-constexpr uint32_t kAccSlots4 = 8;       // 32 ints
-constexpr uint32_t kQueueSlots4 = 124;   // 32 * 31 uint16 items = 1984 bytes
 
 struct ChainView {               // where a chain's state lives
     uint32_t* P;                 // [U][S32] schedule, time-packed (shared or global)
     uint4* ctr;                  // [S] {hr, mi, mo, occ} (shared)
     uint32_t* full;              // [S32] bit t set iff occ[t] == cap (shared)
-    int* acc;                    // [32] per-lane cost change being summed (shared)
-    uint16_t* queue;             // [32 * 31] work items (lane << 5 | window bit) of the current batch (shared)
+    uint4* win;                  // [kBatch][2] windows of the batch's proposals (shared)
+    int* acc;                    // [kBatch] cost change of each proposal being summed (shared)
+    uint16_t* queue;             // [kBatch * 31] work items (proposal slot << 5 | window bit) (shared)
 };
+
+struct Windows { uint32_t Wu, Wv, Nu, Nv, Au, Av, s0; };
 
 // First half of evaluating a proposal, all in the calling lane and word-parallel over the <= 31 affected
 // steps: the windows before and after the move, feasibility (Eq. 5), whether any bit changes, and the set
 // of window bits (steps) whose cardinalities, hence cost, change.
 template <typename PPtr, typename FPtr>
 __device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restrict__ Acol, FPtr full, uint32_t S,
-                                                 uint32_t S32, LaneMove& mv)
+                                                 uint32_t S32, LaneMove& mv, Windows& wn)
 {
     const bool swap = mv.pk & 1u;
     const uint32_t len = (mv.pk >> 1) & 63u, s0 = mv.pk >> 8;
@@ -104,28 +108,21 @@ __device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restr
     const uint32_t nl = min(s0 + len, S - 1) - s0 + 1;            // affected steps: the run and the step after it
     const uint32_t M = ((1u << run) - 1u) << 1;
     const uint32_t Sb = ((1u << nl) - 1u) << 1;
-    const size_t ub = (size_t)mv.u * S32;
-    const uint32_t Wu = window(P + ub, S32, s0);
-    const uint32_t Au = window(Acol + ub, S32, s0);
-    uint32_t Wv = 0, Av = 0;
-    if (swap) {
-        const size_t vb = (size_t)mv.v * S32;
-        Wv = window(P + vb, S32, s0);
-        Av = window(Acol + vb, S32, s0);
-    }
+    // branch-free: a flip reads unit u twice and ignores the second copy, a swap ignores the full-step window
+    const size_t ub = (size_t)mv.u * S32, vb = (size_t)(swap ? mv.v : mv.u) * S32;
+    const uint32_t Wu = window(P + ub, S32, s0), Au = window(Acol + ub, S32, s0);
+    const uint32_t wv = window(P + vb, S32, s0), av = window(Acol + vb, S32, s0);
+    const uint32_t Wv = swap ? wv : 0u, Av = swap ? av : 0u;
+    const uint32_t Fw = window(full, S32, s0);
     const uint32_t D = swap ? ((Wu ^ Wv) & M) : M;                // bits that toggle
     uint32_t Nu = Wu ^ D, Nv = swap ? (Wv ^ D) : 0u;
     if (s0 == 0) {                                                // the virtual step -1 follows step 0
         Nu = (Nu & ~1u) | ((Nu >> 1) & 1u);
         Nv = (Nv & ~1u) | ((Nv >> 1) & 1u);
     }
-    mv.Wu = Wu; mv.Wv = Wv; mv.Nu = Nu; mv.Nv = Nv; mv.Au = Au; mv.Av = Av;
+    wn.Wu = Wu; wn.Wv = Wv; wn.Nu = Nu; wn.Nv = Nv; wn.Au = Au; wn.Av = Av; wn.s0 = s0;
     mv.chg = D != 0;
-    mv.inf = false;
-    if (!swap) {                                                  // a flip may not raise a full step (Eq. 5)
-        const uint32_t Fw = window(full, S32, s0);
-        mv.inf = (~Wu & M & Fw) != 0;
-    }
+    mv.inf = !swap && (~Wu & M & Fw) != 0;                        // a flip may not raise a full step (Eq. 5)
     const uint32_t hr = (Au ^ Av) & (Wu ^ Nu);                    // a hit is won or lost (v mirrors u in a swap)
     // migrations of a unit at step t are the edges p[t] != p[t-1] (into HBM when p[t] is set, out otherwise):
     // the counts change where an edge appears, disappears or turns around
@@ -134,13 +131,12 @@ __device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restr
     return mv.inf ? 0u : ((hr | mg) & Sb);
 }
 
-// Cost change of the step at window bit k (Eq. 2-4 before and after), from the six windows of a proposal.
-__device__ __forceinline__ int item_delta(uint32_t Wu, uint32_t Wv, uint32_t Nu, uint32_t Nv, uint32_t Au, uint32_t Av,
-                                          uint32_t k, const uint4 c4, const StepC c, const CostK K)
+// Cost change of the step at window bit k (Eq. 2-4 before and after), from the windows of a proposal.
+__device__ __forceinline__ int item_delta(const Windows& wn, uint32_t k, const uint4 c4, const StepC c, const CostK K)
 {
-    const uint32_t pu = (Wu >> k) & 1u, qu = (Wu >> (k - 1)) & 1u, npu = (Nu >> k) & 1u, nqu = (Nu >> (k - 1)) & 1u;
-    const uint32_t pv = (Wv >> k) & 1u, qv = (Wv >> (k - 1)) & 1u, npv = (Nv >> k) & 1u, nqv = (Nv >> (k - 1)) & 1u;
-    const uint32_t au = (Au >> k) & 1u, av = (Av >> k) & 1u;
+    const uint32_t pu = (wn.Wu >> k) & 1u, qu = (wn.Wu >> (k - 1)) & 1u, npu = (wn.Nu >> k) & 1u, nqu = (wn.Nu >> (k - 1)) & 1u;
+    const uint32_t pv = (wn.Wv >> k) & 1u, qv = (wn.Wv >> (k - 1)) & 1u, npv = (wn.Nv >> k) & 1u, nqv = (wn.Nv >> (k - 1)) & 1u;
+    const uint32_t au = (wn.Au >> k) & 1u, av = (wn.Av >> k) & 1u;
     const uint32_t hr = c4.x + (au & npu) - (au & pu) + (av & npv) - (av & pv);
     const uint32_t mi = c4.y + (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
     const uint32_t mo = c4.z + (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
@@ -160,34 +156,42 @@ __device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ A
                                           const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
                                           const uint32_t* __restrict__ trow, uint32_t shift, LaneMove& mv)
 {
-    uint32_t todo = lane_windows(P, Acol, full, S, S32, mv);
-    const uint32_t s0 = mv.pk >> 8;
+    Windows wn;
+    uint32_t todo = lane_windows(P, Acol, full, S, S32, mv, wn);
     int delta = 0;
     while (todo) {
         const uint32_t k = __ffs(todo) - 1;
         todo &= todo - 1;
-        const uint32_t t = s0 + k - 1;
-        delta += item_delta(mv.Wu, mv.Wv, mv.Nu, mv.Nv, mv.Au, mv.Av, k, ctr[t], __ldg(stepc + t), K);
+        const uint32_t t = wn.s0 + k - 1;
+        delta += item_delta(wn, k, ctr[t], __ldg(stepc + t), K);
     }
     mv.delta = delta;
     mv.acc = metropolis(delta, mv.w, trow, shift);
 }
 
-// Evaluation of the proposals of the lanes in `need`, shared by the warp: every lane prepares its own
-// proposal, the (lane, step) pairs whose cost changes are queued in shared memory, and the warp works the
-// queue off 32 pairs at a time, so that lanes with short and long proposals carry the same load.
+// Evaluation of the proposals named by `need` (one mask per proposal row), shared by the warp: every lane
+// prepares its own proposals, the (proposal, step) pairs whose cost changes are queued in shared memory, and
+// the warp works the queue off 32 pairs at a time, so that lanes with short and long proposals carry the
+// same load.
 __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* __restrict__ Acol,
                                            const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
-                                           const uint32_t* __restrict__ trow, uint32_t shift, uint32_t need,
-                                           uint32_t lane, LaneMove& mv)
+                                           const uint32_t* __restrict__ trow, uint32_t shift,
+                                           const uint32_t (&need)[kMPL], uint32_t lane, LaneMove (&mv)[kMPL])
 {
-    const bool mine = (need >> lane) & 1u;
-    uint32_t todo = 0;
-    if (mine) {
-        todo = lane_windows(cv.P, Acol, cv.full, S, S32, mv);
-        cv.acc[lane] = 0;
+    uint32_t todo[kMPL], cnt = 0;
+#pragma unroll
+    for (int h = 0; h < kMPL; ++h) {
+        todo[h] = 0;
+        if ((need[h] >> lane) & 1u) {
+            const uint32_t slot = h * 32 + lane;
+            Windows wn;
+            todo[h] = lane_windows(cv.P, Acol, cv.full, S, S32, mv[h], wn);
+            cv.win[slot * 2] = make_uint4(wn.Wu, wn.Wv, wn.Nu, wn.Nv);
+            cv.win[slot * 2 + 1] = make_uint4(wn.Au, wn.Av, wn.s0, 0u);
+            cv.acc[slot] = 0;
+        }
+        cnt += __popc(todo[h]);
     }
-    const uint32_t cnt = __popc(todo);
     uint32_t incl = cnt;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -196,41 +200,47 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
     }
     const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
     uint32_t pos = incl - cnt;
-    while (todo) {
-        const uint32_t k = __ffs(todo) - 1;
-        todo &= todo - 1;
-        cv.queue[pos++] = (uint16_t)((lane << 5) | k);
+    // queue the set bits of every mask; all 31 positions are tried so that no lane waits on a serial bit scan
+#pragma unroll
+    for (int h = 0; h < kMPL; ++h) {
+        const uint32_t td = todo[h];
+        if (__any_sync(0xFFFFFFFFu, td != 0)) {
+#pragma unroll
+            for (uint32_t k = 1; k < 32; ++k)
+                if ((td >> k) & 1u)
+                    cv.queue[pos + __popc(td & ((1u << k) - 1u))] = (uint16_t)(((h * 32 + lane) << 5) | k);
+            pos += __popc(td);
+        }
     }
     __syncwarp();
     for (uint32_t base = 0; base < total; base += 32) {
         const uint32_t g = base + lane;
         const bool live = g < total;
-        const uint32_t item = live ? cv.queue[g] : 1u;            // a dead lane works on (lane 0, bit 1) and drops it
-        const uint32_t o = item >> 5, k = item & 31u;
-        const uint32_t Wu = __shfl_sync(0xFFFFFFFFu, mv.Wu, o), Wv = __shfl_sync(0xFFFFFFFFu, mv.Wv, o);
-        const uint32_t Nu = __shfl_sync(0xFFFFFFFFu, mv.Nu, o), Nv = __shfl_sync(0xFFFFFFFFu, mv.Nv, o);
-        const uint32_t Au = __shfl_sync(0xFFFFFFFFu, mv.Au, o), Av = __shfl_sync(0xFFFFFFFFu, mv.Av, o);
-        const uint32_t s0 = __shfl_sync(0xFFFFFFFFu, mv.pk, o) >> 8;
-        const uint32_t t = min(s0 + k - 1, S - 1);
-        const int d = item_delta(Wu, Wv, Nu, Nv, Au, Av, k, cv.ctr[t], __ldg(stepc + t), K);
-        if (live && d) atomicAdd(cv.acc + o, d);
+        const uint32_t item = live ? cv.queue[g] : 1u;            // a dead lane works on (proposal 0, bit 1) and drops it
+        const uint32_t slot = item >> 5, k = item & 31u;
+        const uint4 w0 = cv.win[slot * 2], w1 = cv.win[slot * 2 + 1];
+        Windows wn;
+        wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
+        const uint32_t t = min(wn.s0 + k - 1, S - 1);
+        const int d = item_delta(wn, k, cv.ctr[t], __ldg(stepc + t), K);
+        if (live && d) atomicAdd(cv.acc + slot, d);
     }
     __syncwarp();
-    if (mine) {
-        mv.delta = cv.acc[lane];
-        mv.acc = metropolis(mv.delta, mv.w, trow, shift);
-    }
+#pragma unroll
+    for (int h = 0; h < kMPL; ++h)
+        if ((need[h] >> lane) & 1u) {
+            mv[h].delta = cv.acc[h * 32 + lane];
+            mv[h].acc = metropolis(mv[h].delta, mv[h].w, trow, shift);
+        }
 }
 
-// Apply the proposal held by lane `b`: all lanes take part, lane j updates the counters of window bit j.
+// Apply the proposal in window slot `slot` (pk, u, v given): all lanes take part, lane j updates the counters
+// of window bit j, lanes 0 and 1 rewrite the words of the schedule and of the full-step bitmap.
 __device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
-                                           uint32_t b, const LaneMove& mine)
+                                           uint32_t slot, uint32_t pk, uint32_t u, uint32_t v)
 {
-    const uint32_t pk = __shfl_sync(0xFFFFFFFFu, mine.pk, b);
-    const uint32_t u = __shfl_sync(0xFFFFFFFFu, mine.u, b), v = __shfl_sync(0xFFFFFFFFu, mine.v, b);
-    const uint32_t Wu = __shfl_sync(0xFFFFFFFFu, mine.Wu, b), Wv = __shfl_sync(0xFFFFFFFFu, mine.Wv, b);
-    const uint32_t Nu = __shfl_sync(0xFFFFFFFFu, mine.Nu, b), Nv = __shfl_sync(0xFFFFFFFFu, mine.Nv, b);
-    const uint32_t Au = __shfl_sync(0xFFFFFFFFu, mine.Au, b), Av = __shfl_sync(0xFFFFFFFFu, mine.Av, b);
+    const uint4 w0 = cv.win[slot * 2], w1 = cv.win[slot * 2 + 1];
+    const uint32_t Wu = w0.x, Wv = w0.y, Nu = w0.z, Nv = w0.w, Au = w1.x, Av = w1.y;
     const bool swap = pk & 1u;
     const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
     const uint32_t run = min(s0 + len, S) - s0;
@@ -294,16 +304,18 @@ chain_kernel(const ChainParams prm)
     const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
     const size_t pwords = (size_t)U * S32;
     const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
-    const uint32_t fixed4 = S + f4 + kAccSlots4 + kQueueSlots4;   // per-warp shared state besides the schedule
+    const uint32_t fixed4 = S + f4 + kWinSlots4 + kAccSlots4 + kQueueSlots4;   // per-warp shared state besides the schedule
     ChainView cv;
     cv.ctr = smem4 + (size_t)warp * fixed4;
     cv.full = reinterpret_cast<uint32_t*>(cv.ctr + S);
-    cv.acc = reinterpret_cast<int*>(cv.ctr + S + f4);
-    cv.queue = reinterpret_cast<uint16_t*>(cv.ctr + S + f4 + kAccSlots4);
+    cv.win = cv.ctr + S + f4;
+    cv.acc = reinterpret_cast<int*>(cv.win + kWinSlots4);
+    cv.queue = reinterpret_cast<uint16_t*>(cv.win + kWinSlots4 + kAccSlots4);
     cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)wpb * fixed4) + (size_t)warp * pwords
                  : prm.ws + (size_t)slot * pwords;
     for (uint32_t i = lane; i < S; i += 32) cv.ctr[i] = __ldg(prm.counters0 + i);
     for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
+    for (uint32_t i = lane; i < kWinSlots4; i += 32) cv.win[i] = make_uint4(0u, 0u, 0u, 0u);
     copy_words(cv.P, prm.Pcol0, pwords, lane);
     __syncwarp();
     uint32_t* snap = prm.snap ? prm.snap + (size_t)slot * pwords : nullptr;
@@ -326,51 +338,73 @@ chain_kernel(const ChainParams prm)
             trow = prm.table + (size_t)level * KVP_TABLE_Q;
             next_boundary = level + 1 < prm.levels ? next_boundary + prm.per_level : ~0ull;
         }
-        // A batch: up to 32 consecutive moves of one temperature level, one per lane. Every lane draws and
-        // evaluates its own proposal against the current state; the warp then commits them in move order.
-        // A move that changes the schedule invalidates only later moves whose step windows overlap its own;
-        // those are evaluated again before their turn comes, so the outcome is that of the sequential chain.
-        const uint32_t nb = (uint32_t)min(min((uint64_t)32, prm.upto - m), next_boundary - m);
-        LaneMove mv;
-        {
+        // A batch: up to 32 * kMPL consecutive moves of one temperature level, move m + 32 h + lane in row h of
+        // its lane. Every lane draws and evaluates its own proposals against the current state; the warp then
+        // commits them in move order. A move that changes the schedule invalidates only later moves whose step
+        // windows overlap its own; those are evaluated again before their turn comes, so the outcome is that
+        // of the sequential chain.
+        const uint32_t nb = (uint32_t)min(min((uint64_t)kBatch, prm.upto - m), next_boundary - m);
+        LaneMove mv[kMPL];
+        uint32_t todo[kMPL], need[kMPL];
+#pragma unroll
+        for (int h = 0; h < kMPL; ++h) {
             uint32_t r[4];
-            const uint64_t mine = m + lane;
+            const uint64_t mine = m + 32u * h + lane;
             philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
-            decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv);
+            decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv[h]);
+            mv[h].inf = false; mv[h].acc = false; mv[h].chg = false; mv[h].delta = 0;
+            const uint32_t left = nb > 32u * h ? nb - 32u * h : 0u;
+            todo[h] = left >= 32 ? 0xFFFFFFFFu : (1u << left) - 1u;
+            need[h] = todo[h];
         }
-        mv.inf = false; mv.acc = false; mv.chg = false; mv.delta = 0;
-        mv.Wu = mv.Wv = mv.Nu = mv.Nv = mv.Au = mv.Av = 0;
-        uint32_t todo = nb == 32 ? 0xFFFFFFFFu : (1u << nb) - 1u;
-        uint32_t need = todo;
-        while (todo) {
-            if (need) eval_batch(cv, prm.Acol, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
-            const uint32_t infb = __ballot_sync(0xFFFFFFFFu, mv.inf);
-            const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !mv.inf && mv.acc);
-            const uint32_t blk = __ballot_sync(0xFFFFFFFFu, !mv.inf && mv.acc && mv.chg) & todo;
-            if (!blk) {
-                n_inf += __popc(infb & todo);
-                n_acc += __popc(accb & todo);
-                break;
+        for (;;) {
+            uint32_t any_need = 0;
+#pragma unroll
+            for (int h = 0; h < kMPL; ++h) any_need |= need[h];
+            if (any_need) eval_batch(cv, prm.Acol, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+            bool applied = false;
+#pragma unroll
+            for (int h = 0; h < kMPL; ++h) need[h] = 0;
+#pragma unroll
+            for (int h = 0; h < kMPL; ++h) {
+                if (applied || !todo[h]) continue;
+                const uint32_t infb = __ballot_sync(0xFFFFFFFFu, mv[h].inf);
+                const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !mv[h].inf && mv[h].acc);
+                const uint32_t blk = __ballot_sync(0xFFFFFFFFu, !mv[h].inf && mv[h].acc && mv[h].chg) & todo[h];
+                if (!blk) {                                       // nothing in this row changes the schedule
+                    n_inf += __popc(infb & todo[h]);
+                    n_acc += __popc(accb & todo[h]);
+                    todo[h] = 0;
+                    continue;
+                }
+                const uint32_t b = __ffs(blk) - 1;
+                const uint32_t done = todo[h] & (0xFFFFFFFFu >> (31 - b));   // the row's moves up to and including b
+                n_inf += __popc(infb & done);
+                n_acc += __popc(accb & done);
+                ++n_chg;
+                const int delta = __shfl_sync(0xFFFFFFFFu, mv[h].delta, b);
+                const uint32_t pk = __shfl_sync(0xFFFFFFFFu, mv[h].pk, b);
+                const uint32_t bu = __shfl_sync(0xFFFFFFFFu, mv[h].u, b), bv = __shfl_sync(0xFFFFFFFFu, mv[h].v, b);
+                const uint64_t after = (uint64_t)((int64_t)cur + delta);
+                if (snap && snap_dirty && after >= best) {        // leaving the best state: save it first
+                    copy_words(snap, cv.P, pwords, lane);
+                    snap_dirty = false;
+                }
+                apply_move(cv, S, S32, prm.cap, lane, h * 32 + b, pk, bu, bv);
+                cur = after;
+                const uint64_t mb = m + 32u * h + b;
+                hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
+                if (cur < best) { best = cur; best_move = mb; snap_dirty = true; }
+                todo[h] &= ~done;
+                const uint32_t s0b = pk >> 8;
+#pragma unroll
+                for (int h2 = 0; h2 < kMPL; ++h2) {
+                    const uint32_t s0 = mv[h2].pk >> 8;
+                    need[h2] = __ballot_sync(0xFFFFFFFFu, s0 + 32 > s0b && s0b + 32 > s0) & todo[h2];
+                }
+                applied = true;
             }
-            const uint32_t b = __ffs(blk) - 1;
-            const uint32_t done = todo & (0xFFFFFFFFu >> (31 - b));   // the moves up to and including b
-            n_inf += __popc(infb & done);
-            n_acc += __popc(accb & done);
-            ++n_chg;
-            const int delta = __shfl_sync(0xFFFFFFFFu, mv.delta, b);
-            const uint64_t after = (uint64_t)((int64_t)cur + delta);
-            if (snap && snap_dirty && after >= best) {            // leaving the best state: save it first
-                copy_words(snap, cv.P, pwords, lane);
-                snap_dirty = false;
-            }
-            apply_move(cv, S, S32, prm.cap, lane, b, mv);
-            cur = after;
-            const uint64_t mb = m + b;
-            hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
-            if (cur < best) { best = cur; best_move = mb; snap_dirty = true; }
-            todo &= ~done;
-            const uint32_t s0b = __shfl_sync(0xFFFFFFFFu, mv.pk, b) >> 8, s0 = mv.pk >> 8;
-            need = __ballot_sync(0xFFFFFFFFu, s0 + 32 > s0b && s0b + 32 > s0) & todo;
+            if (!applied) break;
         }
         m += nb;
     }
@@ -526,8 +560,8 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     KVP_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     KVP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const size_t budget = (size_t)smem_max - 1024;
-    // per warp: counters, full-step bitmap, 32 accumulators, the work queue
-    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4 + kAccSlots4 + kQueueSlots4) * 16;
+    // per warp: counters, full-step bitmap, the batch's windows, accumulators and work queue
+    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4 + kWinSlots4 + kAccSlots4 + kQueueSlots4) * 16;
     const size_t psmem_per_warp = ctr_bytes + (size_t)p->U * p->S32 * 4;
     c.psmem = psmem_per_warp <= budget / 2;
     if (c.psmem) {

@@ -396,11 +396,13 @@ chain_kernel(const ChainParams prm)
                 hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
                 if (cur < best) { best = cur; best_move = mb; snap_dirty = true; }
                 todo[h] &= ~done;
-                const uint32_t s0b = pk >> 8;
+                // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later proposal
+                // read steps s0 - 1 .. s0 + len: it has to be evaluated again iff the two ranges meet.
+                const uint32_t s0b = pk >> 8, endb = s0b + ((pk >> 1) & 63u);
 #pragma unroll
                 for (int h2 = 0; h2 < kMPL; ++h2) {
-                    const uint32_t s0 = mv[h2].pk >> 8;
-                    need[h2] = __ballot_sync(0xFFFFFFFFu, s0 + 32 > s0b && s0b + 32 > s0) & todo[h2];
+                    const uint32_t s0 = mv[h2].pk >> 8, end = s0 + ((mv[h2].pk >> 1) & 63u);
+                    need[h2] = __ballot_sync(0xFFFFFFFFu, s0 <= endb + 1 && s0b <= end) & todo[h2];
                 }
                 applied = true;
             }

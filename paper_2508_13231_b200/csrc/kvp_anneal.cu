@@ -206,10 +206,11 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         const uint32_t td = todo[h];
         if (__any_sync(0xFFFFFFFFu, td != 0)) {
 #pragma unroll
-            for (uint32_t k = 1; k < 32; ++k)
-                if ((td >> k) & 1u)
-                    cv.queue[pos + __popc(td & ((1u << k) - 1u))] = (uint16_t)(((h * 32 + lane) << 5) | k);
-            pos += __popc(td);
+            for (uint32_t k = 1; k < 32; ++k) {
+                const uint32_t bit = (td >> k) & 1u;
+                if (bit) cv.queue[pos] = (uint16_t)(((h * 32 + lane) << 5) | k);
+                pos += bit;
+            }
         }
     }
     __syncwarp();

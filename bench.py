@@ -129,6 +129,63 @@ def cpu_baseline(cfg, tp):
                       f"and set-up; {dt:.1f} s on one thread"}
 
 
+def run_cost_kernel(args):
+    """The cost kernel alone on the rows of the largest configuration: HBM roofline.
+
+    A batch of schedules of long_70b (81,920 words per row, 64 rows, 20 MB each) is scored by kvp_eval; the
+    batch plus the access bitmap is larger than L2. Algorithmic bytes: every placement word once and the access
+    bitmap once per batch (it stays in L2 across the batch), (n + 1) * S * W32 * 4.
+    """
+    import numpy as np
+    import torch
+    from paper_2508_13231_b200 import kvp, workloads as wl
+    torch.cuda.set_device(0)
+    name, n = "long_70b", 96
+    cfg = wl.CONFIGS[name]
+    tp = wl.trace_params(name, seed=0)
+    U, S, W32 = wl.units(cfg), cfg["steps"], wl.words_per_row(cfg)
+    A = kvp.trace_generate(**{k: v for k, v in tp.items() if k != "base"}, base=None)
+    prob = kvp.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"])
+    g = torch.Generator(device="cuda"); g.manual_seed(1)
+    # random words thinned to ~6% density (three ANDed draws halve it each time; 1/8 would exceed the capacity check,
+    # which only sets a flag and costs nothing)
+    sched = torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, W32), dtype=torch.int32, device="cuda", generator=g)
+    for _ in range(3):
+        sched &= torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, W32), dtype=torch.int32, device="cuda", generator=g)
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    for _ in range(max(3, args.warmup)):
+        prob.eval(sched, want_steps=False, want_seconds=False)
+    torch.cuda.synchronize()
+    total_ms = 0.0
+    for k in range(args.steps):
+        flush.fill_(k & 255)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        prob.eval(sched, want_steps=False, want_seconds=False)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        total_ms += e0.elapsed_time(e1)
+    ms = total_ms / args.steps
+    alg_bytes = (n + 1) * S * W32 * 4
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak, src = (peaks["hbm_gbs"], "measured copy bandwidth (MEASURED_PEAKS.json)") if "hbm_gbs" in peaks else \
+        (6650.0, "fallback 6.65 TB/s")
+    achieved = alg_bytes / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "kernel": "count_wide_kernel+finish_kernel (kvp_eval)", "metric": "schedules_scored_per_sec",
+        "value": n / (ms * 1e-3), "unit": "schedules/s", "ms_per_call": ms, "steps": args.steps,
+        "config": {"workload": name, "batch": n, "words_per_row": W32, "rows": S,
+                   "l2": "flushed with a 256 MB write between timed iterations"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "algorithmic_bytes": alg_bytes, "peak_source": src}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -136,9 +193,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="kvp", choices=["kvp", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", default="path", choices=["path", "cost"],
+                    help="path: the whole hot path (the benchmark line); cost: the cost kernel alone on full-size rows")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.kernel == "cost":
+        return run_cost_kernel(args)
 
     import numpy as np
     import torch

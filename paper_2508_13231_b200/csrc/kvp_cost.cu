@@ -2,8 +2,8 @@
 //
 // The counting pass is the HBM-bound part: every word of A and of P is read once, P[s-1] is carried
 // in registers from the previous iteration. Two shapes:
-//   wide rows   (>= 17 vectors per row): a warp owns 32 consecutive 16-byte vectors of every row of a
-//               step chunk; a CTA of 8 warps therefore reads 4 KB contiguous per row and array.
+//   wide rows   (>= 17 vectors per row): a warp owns 64 consecutive 16-byte vectors of every row of a
+//               step chunk; a CTA of 8 warps therefore reads 8 KB contiguous per row and array.
 //   narrow rows (<= 16 vectors per row): a sub-warp group of LPR lanes owns whole rows, consecutive
 //               groups own consecutive rows, so a warp still reads contiguous memory.
 #include "kvp_common.cuh"
@@ -46,7 +46,33 @@ __device__ __forceinline__ uint2 vec_counts(uint4 a, uint4 p, uint4 prev)
 }
 
 constexpr int WIDE_WARPS = 8;
+constexpr int WIDE_VEC = 2;              // 16-byte vectors per lane and row
 
+// Carry-save adder: three bit-vectors in, (carry, sum) out; each bit position is added independently.
+__device__ __forceinline__ void csa(uint32_t& carry, uint32_t& sum, uint32_t a, uint32_t b, uint32_t c)
+{
+    sum = a ^ b ^ c;
+    carry = (a & b) | (c & (a ^ b));
+}
+
+// Number of set bits in eight words with four popc instead of eight (Harley-Seal): the words are first added
+// bit-position-wise into a 4-bit counter held as four bit-vectors. popc is the scarce instruction of this kernel.
+__device__ __forceinline__ uint32_t popc8(const uint32_t (&w)[8])
+{
+    uint32_t ones, twos, fours, eights, ta, tb, tc, td, fa, fb;
+    csa(ta, ones, w[0], w[1], w[2]);
+    csa(tb, ones, ones, w[3], w[4]);
+    csa(tc, ones, ones, w[5], w[6]);
+    td = ones & w[7]; ones ^= w[7];
+    csa(fa, twos, ta, tb, tc);
+    fb = twos & td; twos ^= td;
+    eights = fa & fb; fours = fa ^ fb;
+    return __popc(ones) + 2 * __popc(twos) + 4 * __popc(fours) + 8 * __popc(eights);
+}
+
+// Wide rows: a warp owns 64 consecutive 16-byte vectors (1 KB) of every row of a step chunk, two per lane.
+// Per lane and step only three cardinalities are counted, hits |A&P|, occupancy |P| and stayers |P&Pprev|;
+// migrations follow as mi = occ - stay and mo = occ_prev - stay.
 template <int VEC>
 __global__ void __launch_bounds__(WIDE_WARPS * 32)
 count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ Ps, uint32_t S, uint32_t W32,
@@ -54,22 +80,44 @@ count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ P
 {
     extern __shared__ uint2 acc[];                       // [WIDE_WARPS][SC]
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t cv = (blockIdx.x * WIDE_WARPS + warp) * 32 + lane;
-    const bool valid = cv < WV;
+    const uint32_t cv0 = (blockIdx.x * WIDE_WARPS + warp) * (32 * WIDE_VEC) + lane;
     const uint32_t sb = blockIdx.y * SC;
     const uint32_t se = min(S, sb + SC);
     const uint32_t* __restrict__ P = Ps + (size_t)blockIdx.z * S * W32;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    uint4 prev = valid ? mask_last<VEC>(load_vec<VEC>(P, W32, sb ? sb - 1 : 0, cv), cv, WV, pad_mask) : zero;
-#pragma unroll 4
+    uint4 prev[WIDE_VEC];
+    uint32_t occ_prev;
+    {
+        uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < WIDE_VEC; ++j) {
+            const uint32_t cv = cv0 + 32 * j;
+            prev[j] = cv < WV ? mask_last<VEC>(load_vec<VEC>(P, W32, sb ? sb - 1 : 0, cv), cv, WV, pad_mask) : zero;
+            w[4 * j] = prev[j].x; w[4 * j + 1] = prev[j].y; w[4 * j + 2] = prev[j].z; w[4 * j + 3] = prev[j].w;
+        }
+        occ_prev = popc8(w);
+    }
+#pragma unroll 2
     for (uint32_t s = sb; s < se; ++s) {
-        const uint4 a = valid ? load_vec<VEC>(A, W32, s, cv) : zero;
-        const uint4 p = valid ? mask_last<VEC>(load_vec<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
-        uint2 c = vec_counts(a, p, prev);
-        c.x = __reduce_add_sync(0xFFFFFFFFu, c.x);       // 16-bit fields: 32 lanes * 128 < 65536
+        uint32_t wp[8], wh[8], ws[8];
+#pragma unroll
+        for (int j = 0; j < WIDE_VEC; ++j) {
+            const uint32_t cv = cv0 + 32 * j;
+            const bool valid = cv < WV;
+            const uint4 a = valid ? load_vec<VEC>(A, W32, s, cv) : zero;
+            const uint4 p = valid ? mask_last<VEC>(load_vec<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
+            wp[4 * j] = p.x; wp[4 * j + 1] = p.y; wp[4 * j + 2] = p.z; wp[4 * j + 3] = p.w;
+            wh[4 * j] = a.x & p.x; wh[4 * j + 1] = a.y & p.y; wh[4 * j + 2] = a.z & p.z; wh[4 * j + 3] = a.w & p.w;
+            ws[4 * j] = p.x & prev[j].x; ws[4 * j + 1] = p.y & prev[j].y;
+            ws[4 * j + 2] = p.z & prev[j].z; ws[4 * j + 3] = p.w & prev[j].w;
+            prev[j] = p;
+        }
+        const uint32_t occ = popc8(wp), hr = popc8(wh), stay = popc8(ws);
+        uint2 c = make_uint2(hr | ((occ - stay) << 16), (occ_prev - stay) | (occ << 16));
+        occ_prev = occ;
+        c.x = __reduce_add_sync(0xFFFFFFFFu, c.x);       // 16-bit fields: 32 lanes * 256 < 65536
         c.y = __reduce_add_sync(0xFFFFFFFFu, c.y);
         if (lane == 0) acc[warp * SC + (s - sb)] = c;
-        prev = p;
     }
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < se - sb; i += blockDim.x) {
@@ -209,10 +257,11 @@ int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, u
                     : launch_narrow<1>(WV, dim3(), n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, st);
     }
     KVP_CUDA(cudaMemsetAsync(counts, 0, (size_t)n * p->S * 16, st));
-    const uint32_t col_ctas = (WV + WIDE_WARPS * 32 - 1) / (WIDE_WARPS * 32);
-    // Split the steps so that the grid fills the 148 SMs a few times over; every chunk re-reads one halo row.
+    const uint32_t col_ctas = (WV + WIDE_WARPS * 32 * WIDE_VEC - 1) / (WIDE_WARPS * 32 * WIDE_VEC);
+    // Split the steps until the grid is at least four full waves (148 SMs x 8 resident CTAs), so that the last,
+    // partial wave costs little; every chunk re-reads one halo row (1/SC more traffic, mostly from L2).
     uint32_t SC = p->S;
-    while (SC > 8 && (uint64_t)col_ctas * ((p->S + SC - 1) / SC) * n < 148u * 6u) SC = (SC + 1) / 2;
+    while (SC > 8 && (uint64_t)col_ctas * ((p->S + SC - 1) / SC) * n < 148u * 8u * 4u) SC = (SC + 1) / 2;
     if (SC > 512) SC = 512;
     dim3 grid(col_ctas, (p->S + SC - 1) / SC, n);
     const size_t smem = (size_t)WIDE_WARPS * SC * sizeof(uint2);

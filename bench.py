@@ -204,7 +204,7 @@ def main():
     import numpy as np
     import torch
     import torch.distributed as dist
-    from paper_2508_13231_b200 import kvp, workloads as wl
+    from paper_2508_13231_b200 import kvp, sharding, workloads as wl
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -231,7 +231,8 @@ def main():
         A = kvp.trace_generate(**targs, seed=seed, base=base_dev)
         prob = kvp.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"])
         prob.eval(scheds_dev, want_steps=False)
-        prm = prob.make_params(chains=chains, moves=moves, seed=seed, p0=cfg["p0"], first_chain=rank * chains)
+        first, count = sharding.chain_range(rank, world, world * chains)
+        prm = prob.make_params(chains=count, moves=moves, seed=seed, p0=cfg["p0"], first_chain=first)
         out = prob.anneal(prm)
         # kernels: 2 trace (scores, select) + 6 create (clean, popcount, transpose, unit counts, histogram,
         #          static row) + 2 eval (count, finish) + those kvp_anneal reports
@@ -287,10 +288,9 @@ def main():
     barrier()
     stop.set(); th.join()
     total_ms = max_over_ranks(total_ms)
-    # the cross-rank part of the reduction: minimum of (ticks, chain) keys, 8 bytes per rank
+    # the cross-rank part of the reduction: two 8-byte MIN reductions over (ticks, chain)
     if world > 1:
-        key = torch.tensor([(out["best_ticks"] << 21) | out["stats"].best_chain], dtype=torch.int64, device="cuda")
-        dist.all_reduce(key, op=dist.ReduceOp.MIN)
+        sharding.combine_best(dist, out["best_ticks"], out["stats"].best_chain, device="cuda")
     barrier()
     e2e_ms, _, (out2, sched_host) = timed(args.steps, e2e=True)
     barrier()

@@ -22,6 +22,17 @@ __device__ __forceinline__ uint4 load_vec(const uint32_t* __restrict__ base, siz
     }
 }
 
+// placement words are read once and never again: stream them through L2 (evict first)
+template <int VEC>
+__device__ __forceinline__ uint4 load_stream(const uint32_t* __restrict__ base, size_t row_words, uint32_t row, uint32_t cv)
+{
+    if (VEC == 4) {
+        return __ldcs(reinterpret_cast<const uint4*>(base + (size_t)row * row_words) + cv);
+    } else {
+        return make_uint4(__ldcs(base + (size_t)row * row_words + cv), 0u, 0u, 0u);
+    }
+}
+
 template <int VEC>
 __device__ __forceinline__ uint4 mask_last(uint4 v, uint32_t cv, uint32_t WV, uint32_t pad_mask)
 {
@@ -97,7 +108,7 @@ count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ P
         }
         occ_prev = popc8(w);
     }
-#pragma unroll 2
+#pragma unroll 4
     for (uint32_t s = sb; s < se; ++s) {
         uint32_t wp[8], wh[8], ws[8];
 #pragma unroll
@@ -105,7 +116,7 @@ count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ P
             const uint32_t cv = cv0 + 32 * j;
             const bool valid = cv < WV;
             const uint4 a = valid ? load_vec<VEC>(A, W32, s, cv) : zero;
-            const uint4 p = valid ? mask_last<VEC>(load_vec<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
+            const uint4 p = valid ? mask_last<VEC>(load_stream<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
             wp[4 * j] = p.x; wp[4 * j + 1] = p.y; wp[4 * j + 2] = p.z; wp[4 * j + 3] = p.w;
             wh[4 * j] = a.x & p.x; wh[4 * j + 1] = a.y & p.y; wh[4 * j + 2] = a.z & p.z; wh[4 * j + 3] = a.w & p.w;
             ws[4 * j] = p.x & prev[j].x; ws[4 * j + 1] = p.y & prev[j].y;

@@ -192,14 +192,15 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         }
         cnt += __popc(todo[h]);
     }
-    uint32_t incl = cnt;
+    // exclusive prefix sum of cnt over the lanes, bit-sliced: the five ballots do not depend on one another
+    uint32_t pos = 0, total = 0;
+    const uint32_t below = (1u << lane) - 1u;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-        if (lane >= (uint32_t)off) incl += o;
+    for (int bit = 0; bit < 5 + (kMPL > 1 ? 1 : 0) + (kMPL > 2 ? 1 : 0); ++bit) {
+        const uint32_t has = __ballot_sync(0xFFFFFFFFu, (cnt >> bit) & 1u);
+        pos += __popc(has & below) << bit;
+        total += __popc(has) << bit;
     }
-    const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-    uint32_t pos = incl - cnt;
     // queue the set bits of every mask; all 31 positions are tried so that no lane waits on a serial bit scan
 #pragma unroll
     for (int h = 0; h < kMPL; ++h) {
@@ -214,17 +215,27 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         }
     }
     __syncwarp();
-    for (uint32_t base = 0; base < total; base += 32) {
-        const uint32_t g = base + lane;
-        const bool live = g < total;
-        const uint32_t item = live ? cv.queue[g] : 1u;            // a dead lane works on (proposal 0, bit 1) and drops it
-        const uint32_t slot = item >> 5, k = item & 31u;
-        const uint4 w0 = cv.win[slot * 2], w1 = cv.win[slot * 2 + 1];
-        Windows wn;
-        wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
-        const uint32_t t = min(wn.s0 + k - 1, S - 1);
-        const int d = item_delta(wn, k, cv.ctr[t], __ldg(stepc + t), K);
-        if (live && d) atomicAdd(cv.acc + slot, d);
+    // two items per lane and trip: the two evaluations are independent and overlap
+    for (uint32_t base = 0; base < total; base += 64) {
+        int d[2];
+        uint32_t slot[2];
+        bool live[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const uint32_t g = base + 32 * r + lane;
+            live[r] = g < total;
+            const uint32_t item = live[r] ? cv.queue[g] : 1u;     // a dead lane works on (proposal 0, bit 1) and drops it
+            slot[r] = item >> 5;
+            const uint32_t k = item & 31u;
+            const uint4 w0 = cv.win[slot[r] * 2], w1 = cv.win[slot[r] * 2 + 1];
+            Windows wn;
+            wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
+            const uint32_t t = min(wn.s0 + k - 1, S - 1);
+            d[r] = item_delta(wn, k, cv.ctr[t], __ldg(stepc + t), K);
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r)
+            if (live[r] && d[r]) atomicAdd(cv.acc + slot[r], d[r]);
     }
     __syncwarp();
 #pragma unroll

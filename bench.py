@@ -186,6 +186,39 @@ def run_cost_kernel(args):
                      "traffic": None, "algorithmic_bytes": alg_bytes, "peak_source": src}}))
 
 
+def time_to_bound(kvp, cfg, targs, base_dev, U, S):
+    """Outside the timed region: wall time of kvp_anneal (all of its kernels, warm) to reach the bound.
+
+    full: the whole budget, the stop rule off. early_stop: the same call with the paper's rule on (a chain stops at
+    a level boundary when its best improved by less than 0.1% since the previous one). smallest_budget: the smallest
+    of moves/16, /8, /4, /2, moves whose bound is within 0.1% of the full-budget bound, and its wall time.
+    """
+    import torch
+    A = kvp.trace_generate(**targs, seed=0, base=base_dev)
+    prob = kvp.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"])
+
+    def run(moves, permille=0):
+        prm = prob.make_params(chains=cfg["chains"], moves=moves, seed=0, p0=cfg["p0"], early_stop_permille=permille)
+        prob.anneal(prm, want_schedule=False)                       # warm
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        out = prob.anneal(prm, want_schedule=False)
+        torch.cuda.synchronize()
+        return out["best_ticks"], 1e3 * (time.perf_counter() - t0), out["stats"].moves_total
+
+    full_ticks, full_ms, _ = run(cfg["moves"])
+    es_ticks, es_ms, es_moves = run(cfg["moves"], permille=1)
+    res = {"full_budget": {"moves_per_chain": cfg["moves"], "bound_ticks": full_ticks, "ms": full_ms},
+           "early_stop_0.1pct": {"bound_ticks": es_ticks, "ms": es_ms, "moves_executed": es_moves}}
+    for div in (16, 8, 4, 2, 1):
+        ticks, ms, _ = run(cfg["moves"] // div)
+        if (ticks - full_ticks) * 1000 <= full_ticks:
+            res["smallest_budget_within_0.1pct"] = {"moves_per_chain": cfg["moves"] // div, "bound_ticks": ticks, "ms": ms}
+            break
+    prob.close()
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -319,6 +352,8 @@ def main():
                          "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"},
             "bound_ticks": out["best_ticks"], "init_ticks": out["stats"].init_ticks,
         }
+        if world == 1:
+            line["time_to_bound"] = time_to_bound(kvp, cfg, targs, base_dev, U, S)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(cfg, tp)
         print(json.dumps(line))

@@ -278,8 +278,9 @@ typedef struct {
                              |base| <= 2^29                                          */
 } kvp_trace_params;
 
-#define KVP_TRACE_SINGLE_PASS 1u /* never allocate the [steps][units] int32 score matrix (the default does when it
-                                    is at most 1 GiB, stream-ordered and freed on return); slower for few groups */
+#define KVP_TRACE_SINGLE_PASS 1u /* never allocate the [steps][units] int32 score matrix (the default does for traces
+                                    of fewer than 148 groups when it is at most 1 GiB; stream-ordered, freed on
+                                    return); much slower for few groups */
 
 /*
  * kvp_trace_generate -- fill access_bitmaps (device) [steps][ceil(U/32)] with the

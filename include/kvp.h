@@ -288,6 +288,63 @@ typedef struct {
  */
 int kvp_trace_generate(const kvp_trace_params* params, uint32_t* access_bitmaps, void* stream);
 
+/*
+ * The look-ahead placement policy that the paper's annealer tunes (Section III-B), as a schedule generator.
+ * Window W (steps, 1..64) and migration ratio R = ratio_permille / 1000. Starting from the static placement
+ * `init_mode` (KVP_INIT_STATIC_FIRST or KVP_INIT_STATIC_FREQ), before every step s:
+ *   - the frequency of a unit is the number of its accesses in steps s .. s+W-1;
+ *   - candidates are the units outside HBM with frequency > 0, ranked by frequency (ties: lower index); only the
+ *     best floor(R * candidates) may migrate;
+ *   - they first take free HBM capacity; then the j-th remaining candidate replaces the j-th resident in order of
+ *     rising frequency (ties: lower index) as long as that resident is accessed less often than the candidate.
+ * The placement decided before step s is the one step s reads (row s of the schedule); the cost model charges the
+ * migrations to step s (none at s = 0).
+ *   windows, ratios_permille (host) [n];  schedules (device) [n][steps][W32]: one schedule per (W, R) pair.
+ * Limit: units <= 32768 (KVP_ERR_RANGE). Synchronises `stream` before returning.
+ */
+int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const uint32_t* windows,
+                         const uint32_t* ratios_permille, uint32_t n, uint32_t* schedules, void* stream);
+
+/*
+ * kvp_wr_grid -- T(W, R) of the look-ahead policy on the whole grid W = 1..w_max, R = r / (n_ratio - 1),
+ * r = 0..n_ratio-1: runs kvp_policy_lookahead and kvp_eval on every grid point.
+ *   table (device) [w_max][n_ratio] uint64 total ticks.
+ */
+int kvp_wr_grid(kvp_problem* p, uint32_t init_mode, uint32_t w_max, uint32_t n_ratio, uint64_t* table, void* stream);
+
+/*
+ * The paper's own annealer (Section III-B): state (W, R), objective T(W, R) from a kvp_wr_grid table. Each
+ * iteration draws one of three operators with probabilities (0.4, 0.4, 0.2): a window move (W +- 1 or 2), a ratio
+ * move (R +- one grid step, 0.1 for n_ratio = 11), or both at once; a proposal that leaves the grid is discarded.
+ * Metropolis acceptance exp(-dT/C) with the quantised table of kvp_accept_table; C_0 accepts the mean uphill step
+ * between grid neighbours with probability p0 and C_{j+1} = alpha * C_j over `levels` levels of iters/levels
+ * iterations; with early_stop_permille a chain stops at a level boundary when its best improved by less than that
+ * many 1/1000 since the previous boundary. Iteration i of chain c uses Philox4x32-10(counter (i_lo, i_hi, c, 5), key
+ * seed): operator from the low byte of word 0 (< 102: window, < 204: ratio, else both), the W step from bits 8-9
+ * ({-2, -1, +1, +2}), the R direction from bit 10, the Metropolis uniform is word 3.
+ */
+typedef struct {
+    uint32_t chains, levels;
+    uint64_t iters, seed;
+    double   p0, alpha;             /* the paper: 0.8, 0.9 */
+    uint32_t early_stop_permille;   /* the paper: 1 (0.1%); 0 = never */
+    uint32_t w0, r0;                /* start: W = w0 (1..w_max), R = r0 / (n_ratio - 1) */
+    uint32_t reserved;              /* must be 0 */
+} kvp_wr_params;
+
+typedef struct {
+    uint64_t best_ticks, final_ticks, iters_done, n_accepted;
+    uint32_t best_w, best_r, final_w, final_r;
+} kvp_wr_result;
+
+/*
+ * kvp_wr_anneal -- run `chains` independent (W, R) chains on a table.
+ *   table (device) [w_max][n_ratio];  results (host) [chains] or NULL;  best (host) or NULL: the chain with the
+ *   lowest best_ticks (ties: lower chain index). Synchronises `stream`.
+ */
+int kvp_wr_anneal(const uint64_t* table, uint32_t w_max, uint32_t n_ratio, const kvp_wr_params* params,
+                  kvp_wr_result* results, kvp_wr_result* best, void* stream);
+
 /* Philox4x32-10 (Salmon et al., SC'11) on the host; exposed so that callers can
  * reproduce which proposal a given (seed, chain, move) pair is. */
 void kvp_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);

@@ -691,3 +691,208 @@ int kvpo_trace_generate(const kvpo_trace_params *tp, uint32_t group_begin, uint3
     free(x); free(score); free(picked);
     return KVPO_OK;
 }
+
+/* ------------------------------------------------------------------ */
+/* Placement policies that produce a schedule from the access pattern (Section IV-A's comparison strategies and
+ * the look-ahead policy of Section III-B that the paper's annealer tunes). Each starts from the static placement
+ * named by init_mode (0: units 0..cap-1, the paper's Static Placement; 1: the cap most accessed units) and
+ * writes P [S][W32]. Migrations decided "at step s" are in place when step s reads (they are charged to step s by
+ * the cost model; at s = 0 they are free because P[-1] := P[0]). */
+
+typedef struct { uint32_t f, u; } fu_t;
+
+static int by_freq_desc(const void *a, const void *b)
+{
+    const fu_t *x = (const fu_t *)a, *y = (const fu_t *)b;
+    if (x->f != y->f) return x->f > y->f ? -1 : 1;
+    return x->u < y->u ? -1 : (x->u > y->u ? 1 : 0);
+}
+
+static int by_freq_asc(const void *a, const void *b)
+{
+    const fu_t *x = (const fu_t *)a, *y = (const fu_t *)b;
+    if (x->f != y->f) return x->f < y->f ? -1 : 1;
+    return x->u < y->u ? -1 : (x->u > y->u ? 1 : 0);
+}
+
+/*
+ * Look-ahead policy with window W (steps) and migration ratio R = ratio_permille / 1000 (Section III-B).
+ * Before step s: every unit's frequency is the number of its accesses in steps s .. s+W-1. The units that are
+ * not in HBM and will be accessed are the candidates, ranked by frequency (ties: lower index); only the top
+ * floor(R * candidates) of them may migrate. They first fill free HBM capacity; after that the j-th remaining
+ * candidate replaces the j-th resident in order of rising frequency (ties: lower index), as long as that resident
+ * is accessed less often than the candidate.
+ */
+int kvpo_policy_lookahead(const kvpo_problem *p, uint32_t init_mode, uint32_t W, uint32_t ratio_permille, uint32_t *P)
+{
+    if (!p || !P || init_mode > 1 || W < 1 || W > 64 || ratio_permille > 1000) return KVPO_ERR_ARG;
+    int rc = kvpo_init_placement(p, init_mode, P);
+    if (rc) return rc;
+    uint8_t *in = (uint8_t *)calloc(p->U, 1);
+    fu_t *cand = (fu_t *)malloc(sizeof(fu_t) * p->U), *res = (fu_t *)malloc(sizeof(fu_t) * p->U);
+    if (!in || !cand || !res) { free(in); free(cand); free(res); return KVPO_ERR_NOMEM; }
+    for (uint32_t u = 0; u < p->U; ++u) in[u] = (uint8_t)bit_of(P, u);
+    for (uint32_t s = 0; s < p->S; ++s) {
+        uint32_t nc = 0, nr = 0;
+        for (uint32_t u = 0; u < p->U; ++u) {
+            uint32_t f = 0;
+            for (uint32_t t = s; t < s + W && t < p->S; ++t) f += (uint32_t)bit_of(p->A + (size_t)t * p->W32, u);
+            if (in[u]) { res[nr].f = f; res[nr].u = u; ++nr; }
+            else if (f > 0) { cand[nc].f = f; cand[nc].u = u; ++nc; }
+        }
+        qsort(cand, nc, sizeof(fu_t), by_freq_desc);
+        qsort(res, nr, sizeof(fu_t), by_freq_asc);
+        uint32_t k = (uint32_t)(((uint64_t)nc * ratio_permille) / 1000u);
+        uint32_t ci = 0, vi = 0, occ = nr;
+        for (; ci < k; ++ci) {
+            if (occ < p->cap) { in[cand[ci].u] = 1; ++occ; continue; }          /* free capacity */
+            if (vi >= nr || !(res[vi].f < cand[ci].f)) break;                     /* no resident worth replacing */
+            in[res[vi].u] = 0; in[cand[ci].u] = 1; ++vi;
+        }
+        uint32_t *row = P + (size_t)s * p->W32;
+        memset(row, 0, (size_t)p->W32 * 4);
+        for (uint32_t u = 0; u < p->U; ++u) if (in[u]) set_bit(row, u, 1);
+    }
+    free(in); free(cand); free(res);
+    return KVPO_OK;
+}
+
+/*
+ * Reactive Scheduling (Section IV-A): a unit that is accessed while it is not in HBM is promoted, the least
+ * recently used resident makes room when HBM is full. The promotion follows the miss: the miss of step s is served
+ * from off-package DRAM and the unit is resident from step s+1 on. Per step: the accessed residents become most
+ * recently used; the missed units, in index order and at most `cap` of them, first take free capacity, then replace
+ * the residents in order of last use (ties: lower index).
+ */
+int kvpo_policy_reactive(const kvpo_problem *p, uint32_t init_mode, uint32_t *P)
+{
+    if (!p || !P || init_mode > 1) return KVPO_ERR_ARG;
+    int rc = kvpo_init_placement(p, init_mode, P);
+    if (rc) return rc;
+    uint8_t *in = (uint8_t *)calloc(p->U, 1);
+    uint32_t *stamp = (uint32_t *)calloc(p->U, 4);        /* 0 = never used, else step of last use + 1 */
+    fu_t *res = (fu_t *)malloc(sizeof(fu_t) * p->U);
+    if (!in || !stamp || !res) { free(in); free(stamp); free(res); return KVPO_ERR_NOMEM; }
+    for (uint32_t u = 0; u < p->U; ++u) in[u] = (uint8_t)bit_of(P, u);
+    for (uint32_t s = 0; s + 1 < p->S; ++s) {                        /* row s is final; build row s+1 */
+        const uint32_t *acc = p->A + (size_t)s * p->W32;
+        uint32_t nr = 0, occ = 0;
+        for (uint32_t u = 0; u < p->U; ++u) {
+            if (in[u] && bit_of(acc, u)) stamp[u] = s + 1;
+            if (in[u]) { res[nr].f = stamp[u]; res[nr].u = u; ++nr; ++occ; }
+        }
+        qsort(res, nr, sizeof(fu_t), by_freq_asc);                   /* least recently used first */
+        uint32_t vi = 0, promoted = 0;
+        for (uint32_t u = 0; u < p->U && promoted < p->cap; ++u) {
+            if (in[u] || !bit_of(acc, u)) continue;
+            if (occ < p->cap) ++occ;
+            else { if (vi >= nr) break; in[res[vi].u] = 0; ++vi; }
+            in[u] = 1; stamp[u] = s + 1; ++promoted;
+        }
+        uint32_t *row = P + (size_t)(s + 1) * p->W32;
+        memset(row, 0, (size_t)p->W32 * 4);
+        for (uint32_t u = 0; u < p->U; ++u) if (in[u]) set_bit(row, u, 1);
+    }
+    free(in); free(stamp); free(res);
+    return KVPO_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* The paper's own annealer (Section III-B): the state is the pair (W, R) of the look-ahead policy, the objective
+ * T(W, R) the total latency of the schedule that policy produces. Here the objective comes from a table
+ * T[(W-1) * n_ratio + r] (W = 1..w_max, R = r / (n_ratio - 1)) filled beforehand by running the policy and the cost
+ * model on every grid point. Proposal operators and their probabilities (0.4, 0.4, 0.2), the steps {+-1, +-2} of W
+ * and +-0.1 of R, the Metropolis rule, p0, alpha and the 0.1% stop rule are the paper's; a proposal that leaves the
+ * grid is discarded. */
+#define TAG_WR 5u
+
+typedef struct {
+    uint32_t chains, levels;
+    uint64_t iters, seed;
+    double p0, alpha;
+    uint32_t early_stop_permille, w0, r0, reserved;
+} kvpo_wr_params;
+
+typedef struct {
+    uint64_t best_ticks, final_ticks, iters_done, n_accepted;
+    uint32_t best_w, best_r, final_w, final_r;
+} kvpo_wr_result;
+
+static const int WR_DW[4] = { -2, -1, 1, 2 };
+
+/* Temperature ladder: C_0 accepts the mean uphill step between grid neighbours with probability p0. */
+int kvpo_wr_temps(const uint64_t *table, uint32_t w_max, uint32_t n_ratio, const kvpo_wr_params *wp, double *temps,
+                  uint64_t *mean_out)
+{
+    if (!table || !wp || !temps || !w_max || n_ratio < 2 || !wp->levels) return KVPO_ERR_ARG;
+    if (!(wp->p0 > 0.0 && wp->p0 < 1.0) || !(wp->alpha > 0.0 && wp->alpha <= 1.0)) return KVPO_ERR_ARG;
+    uint64_t sum = 0, cnt = 0;
+    for (uint32_t w = 1; w <= w_max; ++w)
+        for (uint32_t r = 0; r < n_ratio; ++r)
+            for (int op = 0; op < 3; ++op)
+                for (int a = 0; a < 4; ++a)
+                    for (int b = 0; b < 2; ++b) {
+                        if (op == 0 && b) continue;              /* a window move has no ratio part */
+                        if (op == 1 && a) continue;              /* a ratio move has no window part */
+                        int64_t nw = (int64_t)w + (op != 1 ? WR_DW[a] : 0);
+                        int64_t nr = (int64_t)r + (op != 0 ? (b ? 1 : -1) : 0);
+                        if (nw < 1 || nw > (int64_t)w_max || nr < 0 || nr >= (int64_t)n_ratio) continue;
+                        uint64_t t0 = table[(size_t)(w - 1) * n_ratio + r], t1 = table[(size_t)(nw - 1) * n_ratio + nr];
+                        if (t1 > t0) { sum += t1 - t0; ++cnt; }
+                    }
+    uint64_t mean = cnt ? sum / cnt : 1;
+    if (!mean) mean = 1;
+    if (mean_out) *mean_out = mean;
+    double C = -(double)mean / log(wp->p0);
+    for (uint32_t j = 0; j < wp->levels; ++j) { temps[j] = C; C = C * wp->alpha; }
+    return KVPO_OK;
+}
+
+int kvpo_wr_anneal(const uint64_t *table, uint32_t w_max, uint32_t n_ratio, const kvpo_wr_params *wp,
+                   const uint32_t *acc_table, const uint32_t *shifts, kvpo_wr_result *results)
+{
+    if (!table || !wp || !acc_table || !shifts || !results || !w_max || n_ratio < 2) return KVPO_ERR_ARG;
+    if (!wp->chains || !wp->levels || !wp->iters || wp->w0 < 1 || wp->w0 > w_max || wp->r0 >= n_ratio) return KVPO_ERR_ARG;
+    uint64_t per_level = wp->iters / wp->levels;
+    if (!per_level) per_level = 1;
+    for (uint32_t c = 0; c < wp->chains; ++c) {
+        uint32_t w = wp->w0, r = wp->r0;
+        uint64_t cur = table[(size_t)(w - 1) * n_ratio + r];
+        kvpo_wr_result res;
+        memset(&res, 0, sizeof res);
+        res.best_ticks = cur; res.best_w = w; res.best_r = r;
+        uint64_t best_at_boundary = cur, i = 0;
+        for (; i < wp->iters; ++i) {
+            uint64_t lev = i / per_level;
+            if (lev > wp->levels - 1) lev = wp->levels - 1;
+            if (i > 0 && i % per_level == 0 && i / per_level <= wp->levels - 1) {
+                if (wp->early_stop_permille &&
+                    (best_at_boundary - res.best_ticks) * 1000ull < best_at_boundary * (uint64_t)wp->early_stop_permille)
+                    break;
+                best_at_boundary = res.best_ticks;
+            }
+            uint32_t x[4];
+            philox(wp->seed, (uint32_t)i, (uint32_t)(i >> 32), c, TAG_WR, x);
+            uint32_t sel = x[0] & 255u;
+            int op = sel < 102u ? 0 : (sel < 204u ? 1 : 2);       /* window, ratio, diagonal: 0.4, 0.4, 0.2 */
+            int dw = op != 1 ? WR_DW[(x[0] >> 8) & 3u] : 0;
+            int dr = op != 0 ? (((x[0] >> 10) & 1u) ? 1 : -1) : 0;
+            int64_t nw = (int64_t)w + dw, nr = (int64_t)r + dr;
+            if (nw < 1 || nw > (int64_t)w_max || nr < 0 || nr >= (int64_t)n_ratio) continue;
+            uint64_t cand = table[(size_t)(nw - 1) * n_ratio + nr];
+            int accept;
+            if (cand <= cur) accept = 1;
+            else {
+                uint64_t q = (cand - cur) >> shifts[lev];
+                accept = q < TABLE_Q && x[3] < acc_table[lev * TABLE_Q + q];
+            }
+            if (!accept) continue;
+            ++res.n_accepted;
+            w = (uint32_t)nw; r = (uint32_t)nr; cur = cand;
+            if (cur < res.best_ticks) { res.best_ticks = cur; res.best_w = w; res.best_r = r; }
+        }
+        res.iters_done = i; res.final_ticks = cur; res.final_w = w; res.final_r = r;
+        results[c] = res;
+    }
+    return KVPO_OK;
+}

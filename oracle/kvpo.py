@@ -241,3 +241,69 @@ def trace_generate(groups, units_per_group, steps, topk, seed, rho_q, c_q, sigma
                                    sc.ctypes.data_as(C.POINTER(C.c_int32)) if want_scores else None),
          "trace_generate")
     return (acc, sc) if want_scores else acc
+
+
+class WRParams(C.Structure):
+    _fields_ = [("chains", C.c_uint32), ("levels", C.c_uint32), ("iters", C.c_uint64), ("seed", C.c_uint64),
+                ("p0", C.c_double), ("alpha", C.c_double), ("early_stop_permille", C.c_uint32),
+                ("w0", C.c_uint32), ("r0", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class WRResult(C.Structure):
+    _fields_ = [("best_ticks", C.c_uint64), ("final_ticks", C.c_uint64), ("iters_done", C.c_uint64),
+                ("n_accepted", C.c_uint64), ("best_w", C.c_uint32), ("best_r", C.c_uint32),
+                ("final_w", C.c_uint32), ("final_r", C.c_uint32)]
+
+    def astuple(self):
+        return tuple(int(getattr(self, n)) for n, _ in self._fields_)
+
+
+def policy_lookahead(prob, window, ratio_permille, init_mode=INIT_STATIC_FIRST):
+    """Schedule of the look-ahead policy (W = window steps, R = ratio_permille / 1000) -> uint32 [S][W32]."""
+    P = np.zeros((prob.steps, prob.w32), np.uint32)
+    _chk(lib().kvpo_policy_lookahead(prob._h, C.c_uint32(init_mode), C.c_uint32(window), C.c_uint32(ratio_permille),
+                                     _u32p(P)), "policy_lookahead")
+    return P
+
+
+def policy_reactive(prob, init_mode=INIT_STATIC_FIRST):
+    """Schedule of promote-on-miss with LRU eviction -> uint32 [S][W32]."""
+    P = np.zeros((prob.steps, prob.w32), np.uint32)
+    _chk(lib().kvpo_policy_reactive(prob._h, C.c_uint32(init_mode), _u32p(P)), "policy_reactive")
+    return P
+
+
+def wr_grid(prob, w_max, n_ratio=11, init_mode=INIT_STATIC_FIRST):
+    """T(W, R) in ticks for W = 1..w_max, R = r / (n_ratio - 1) -> uint64 [w_max][n_ratio]."""
+    T = np.zeros((w_max, n_ratio), np.uint64)
+    for w in range(1, w_max + 1):
+        for r in range(n_ratio):
+            T[w - 1, r] = prob.eval(policy_lookahead(prob, w, (1000 * r) // (n_ratio - 1), init_mode))["total_ticks"]
+    return T
+
+
+def wr_params(chains, iters, seed=0, levels=16, p0=0.8, alpha=0.9, early_stop_permille=0, w0=1, r0=0):
+    wp = WRParams()
+    wp.chains, wp.levels, wp.iters, wp.seed = chains, levels, iters, seed
+    wp.p0, wp.alpha, wp.early_stop_permille, wp.w0, wp.r0 = p0, alpha, early_stop_permille, w0, r0
+    return wp
+
+
+def wr_temps(table, wp):
+    table = np.ascontiguousarray(table, dtype=np.uint64)
+    t = np.zeros(wp.levels, np.float64)
+    mean = C.c_uint64()
+    _chk(lib().kvpo_wr_temps(_u64p(table), C.c_uint32(table.shape[0]), C.c_uint32(table.shape[1]), C.byref(wp),
+                             t.ctypes.data_as(C.POINTER(C.c_double)), C.byref(mean)), "wr_temps")
+    return t, int(mean.value)
+
+
+def wr_anneal(table, wp):
+    """The paper's (W, R) annealer on a latency table -> list of WRResult, one per chain."""
+    table = np.ascontiguousarray(table, dtype=np.uint64)
+    temps, _ = wr_temps(table, wp)
+    acc, shifts = accept_table(temps)
+    res = (WRResult * wp.chains)()
+    _chk(lib().kvpo_wr_anneal(_u64p(table), C.c_uint32(table.shape[0]), C.c_uint32(table.shape[1]), C.byref(wp),
+                              _u32p(acc), _u32p(shifts), res), "wr_anneal")
+    return list(res)

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvp.so")
-SOURCES = ["kvp_api.cu", "kvp_cost.cu", "kvp_layout.cu", "kvp_anneal.cu", "kvp_trace.cu"]
+SOURCES = ["kvp_api.cu", "kvp_cost.cu", "kvp_layout.cu", "kvp_anneal.cu", "kvp_trace.cu", "kvp_policy.cu"]
 
 
 def _nvcc():

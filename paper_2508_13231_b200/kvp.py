@@ -23,6 +23,7 @@ NOALLOC_SCRATCH_BYTES = 1 << 20
 EXPORTS = [
     "kvp_create", "kvp_destroy", "kvp_get_info", "kvp_eval", "kvp_eval_counts", "kvp_eval_noalloc", "kvp_accept_table", "kvp_anneal",
     "kvp_anneal_chain_state", "kvp_trace_generate", "kvp_philox4x32_10", "kvp_strerror", "kvp_last_cuda_error",
+    "kvp_policy_lookahead", "kvp_wr_grid", "kvp_wr_anneal",
 ]
 
 
@@ -72,6 +73,21 @@ class AnnealStats(C.Structure):
         ("ms_init", C.c_float), ("ms_chains", C.c_float), ("ms_finish", C.c_float), ("kernel_launches", C.c_uint32),
         ("per_chain", C.POINTER(ChainResult)),
     ]
+
+
+class WRParams(C.Structure):
+    _fields_ = [("chains", C.c_uint32), ("levels", C.c_uint32), ("iters", C.c_uint64), ("seed", C.c_uint64),
+                ("p0", C.c_double), ("alpha", C.c_double), ("early_stop_permille", C.c_uint32),
+                ("w0", C.c_uint32), ("r0", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class WRResult(C.Structure):
+    _fields_ = [("best_ticks", C.c_uint64), ("final_ticks", C.c_uint64), ("iters_done", C.c_uint64),
+                ("n_accepted", C.c_uint64), ("best_w", C.c_uint32), ("best_r", C.c_uint32),
+                ("final_w", C.c_uint32), ("final_r", C.c_uint32)]
+
+    def astuple(self):
+        return tuple(int(getattr(self, n)) for n, _ in self._fields_)
 
 
 class TraceParams(C.Structure):
@@ -270,3 +286,36 @@ class Problem:
                                            _ptr(sched, torch.int32), C.byref(res), _stream(stream)),
              "kvp_anneal_chain_state")
         return sched, res
+
+    def policy_lookahead(self, windows, ratios_permille, init_mode=INIT_STATIC_FIRST, stream=None):
+        """kvp_policy_lookahead -> CUDA int32 [n][S][W32], one schedule per (W, R) pair."""
+        n = len(windows)
+        w = (C.c_uint32 * n)(*[int(x) for x in windows])
+        r = (C.c_uint32 * n)(*[int(x) for x in ratios_permille])
+        out = torch.empty((n, self.steps, self.w32), dtype=torch.int32, device="cuda")
+        _chk(_lib().kvp_policy_lookahead(self._h, C.c_uint32(init_mode), w, r, C.c_uint32(n), _ptr(out), _stream(stream)),
+             "kvp_policy_lookahead")
+        return out
+
+    def wr_grid(self, w_max, n_ratio=11, init_mode=INIT_STATIC_FIRST, stream=None):
+        """kvp_wr_grid -> CUDA int64 [w_max][n_ratio]: total ticks of the look-ahead policy on the (W, R) grid."""
+        table = torch.empty((w_max, n_ratio), dtype=torch.int64, device="cuda")
+        _chk(_lib().kvp_wr_grid(self._h, C.c_uint32(init_mode), C.c_uint32(w_max), C.c_uint32(n_ratio), _ptr(table),
+                                _stream(stream)), "kvp_wr_grid")
+        return table
+
+
+def wr_params(chains, iters, seed=0, levels=16, p0=0.8, alpha=0.9, early_stop_permille=0, w0=1, r0=0):
+    wp = WRParams()
+    wp.chains, wp.levels, wp.iters, wp.seed = chains, levels, iters, seed
+    wp.p0, wp.alpha, wp.early_stop_permille, wp.w0, wp.r0 = p0, alpha, early_stop_permille, w0, r0
+    return wp
+
+
+def wr_anneal(table, wp, stream=None):
+    """kvp_wr_anneal on a CUDA int64 table [w_max][n_ratio] -> (list of WRResult per chain, best WRResult)."""
+    res = (WRResult * wp.chains)()
+    best = WRResult()
+    _chk(_lib().kvp_wr_anneal(_ptr(table, torch.int64), C.c_uint32(table.shape[0]), C.c_uint32(table.shape[1]),
+                              C.byref(wp), res, C.byref(best), _stream(stream)), "kvp_wr_anneal")
+    return list(res), best

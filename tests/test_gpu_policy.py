@@ -1,0 +1,78 @@
+"""Look-ahead policy kernel, (W, R) grid and the paper-literal annealer vs the oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2508_13231_b200 import workloads as wl
+from gpu_util import both_problems, named_problem, to_np, u64
+
+pytestmark = pytest.mark.gpu
+GB = 10 ** 9
+
+
+@pytest.fixture(scope="module")
+def kvp():
+    from paper_2508_13231_b200 import kvp
+    return kvp
+
+
+@pytest.mark.parametrize("U,S,cap", [(4, 3, 1), (70, 40, 15), (33, 1, 5), (1, 9, 1), (300, 65, 0), (1000, 130, 1000),
+                                     (2085, 77, 400)])
+def test_lookahead_small_shapes(kvp, oracle, U, S, cap):
+    A = wl.random_access(U, S, 0.15, seed=U + S)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    pairs = [(1, 0), (1, 1000), (2, 500), (5, 300), (31, 100), (32, 1000), (33, 700), (64, 1000), (64, 1)]
+    for init in (kvp.INIT_STATIC_FIRST, kvp.INIT_STATIC_FREQ):
+        got = to_np(g.policy_lookahead([w for w, _ in pairs], [r for _, r in pairs], init_mode=init))
+        for i, (w, r) in enumerate(pairs):
+            assert np.array_equal(got[i], oracle.policy_lookahead(o, w, r, init_mode=init)), (w, r, init)
+
+
+@pytest.mark.parametrize("name,pairs", [("tiny", [(1, 1000), (4, 500), (40, 1000)]),
+                                        ("single_head", [(1, 100), (16, 100), (8, 1000), (64, 300)]),
+                                        ("layer_8b", [(4, 300), (64, 1000)])])
+def test_lookahead_named_configs(kvp, oracle, name, pairs):
+    g, o, cfg, A = named_problem(kvp, oracle, name)
+    got = to_np(g.policy_lookahead([w for w, _ in pairs], [r for _, r in pairs]))
+    for i, (w, r) in enumerate(pairs):
+        assert np.array_equal(got[i], oracle.policy_lookahead(o, w, r)), (w, r)
+    ev = g.eval(torch.from_numpy(got.view(np.int32)).cuda())
+    assert int(ev["bad_step"].max()) == -1
+
+
+def test_lookahead_limits(kvp, oracle):
+    g, o, cfg, A = named_problem(kvp, oracle, "tiny")
+    for w, r in [(0, 100), (65, 100), (3, 1001)]:
+        with pytest.raises(kvp.KvpError) as e:
+            g.policy_lookahead([w], [r])
+        assert e.value.code == kvp.ERR_ARG
+    U, S = 32768 + 32, 2
+    big = kvp.Problem(U, 8192, S, torch.zeros((S, (U + 31) // 32), dtype=torch.int32, device="cuda"), 10,
+                      8000 * GB, 900 * GB, 900 * GB)
+    with pytest.raises(kvp.KvpError) as e:
+        big.policy_lookahead([1], [100])
+    assert e.value.code == kvp.ERR_RANGE
+
+
+def test_wr_grid_and_annealer(kvp, oracle):
+    g, o, cfg, A = named_problem(kvp, oracle, "single_head")
+    w_max, n_ratio = 20, 11
+    table = g.wr_grid(w_max, n_ratio)
+    want = oracle.wr_grid(o, w_max, n_ratio)
+    assert np.array_equal(u64(table), want)
+    for kw in (dict(chains=64, iters=3000, seed=5, levels=16),
+               dict(chains=7, iters=64000, seed=1, levels=64, early_stop_permille=1),
+               dict(chains=3, iters=10, seed=2, levels=16, w0=20, r0=10),
+               dict(chains=5, iters=2000, seed=2 ** 40 + 1, levels=1, p0=0.3, alpha=1.0)):
+        res, best = kvp.wr_anneal(table, kvp.wr_params(**kw))
+        ref = oracle.wr_anneal(want, oracle.wr_params(**kw))
+        assert [r.astuple() for r in res] == [r.astuple() for r in ref]
+        low = min(r.best_ticks for r in ref)
+        assert best.astuple() == next(r for r in ref if r.best_ticks == low).astuple()
+    # the walk finds the grid minimum, which beats Static Placement (R = 0 column) by the paper's kind of factor
+    res, best = kvp.wr_anneal(table, kvp.wr_params(chains=256, iters=4000, seed=0, levels=32))
+    assert best.best_ticks == int(want.min())
+    assert int(want[0, 0]) / best.best_ticks > 4.0
+    with pytest.raises(kvp.KvpError) as e:
+        kvp.wr_anneal(table, kvp.wr_params(chains=1, iters=10, w0=21))
+    assert e.value.code == kvp.ERR_ARG

@@ -98,3 +98,45 @@ def test_eval_full_size(kvp, oracle, name):
         bits[s:, idx] ^= 1
     sched = wl.pack_bits(bits)[None]
     _compare(g, o, sched)
+
+
+def test_eval_batches_beyond_one_grid_slice(kvp, oracle):
+    # more schedules than fit one launch's grid dimension (slices of 32768): every slice lands in the right place
+    U, S, cap = 40, 3, 12
+    A = wl.random_access(U, S, 0.3, seed=77)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    base = wl.random_schedules(U, S, cap, 7, seed=78, churn=0.3)
+    n = 70001
+    idx = np.arange(n) % 7
+    scheds = base[idx]
+    out = g.eval(to_dev(scheds))
+    want = np.array([o.eval(P)["total_ticks"] for P in base], np.uint64)
+    assert np.array_equal(u64(out["total_ticks"]), want[idx])
+    st = u64(out["step_ticks"])
+    assert np.array_equal(st[-1], o.eval(base[idx[-1]])["step_ticks"])
+    assert np.array_equal(st[32768], o.eval(base[idx[32768]])["step_ticks"])
+
+
+def test_long_horizons(kvp, oracle):
+    # the scoring side takes the maximum horizon; the annealer keeps per-step state in shared memory and says so
+    U, S, cap = 40, 32768, 10
+    A = wl.random_access(U, S, 0.1, seed=79)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    P = wl.random_schedules(U, S, cap, 1, seed=80, churn=0.3)
+    out = g.eval(to_dev(P))
+    assert int(u64(out["total_ticks"])[0]) == o.eval(P[0])["total_ticks"]
+    with pytest.raises(kvp.KvpError) as e:
+        g.anneal(g.make_params(chains=2, moves=100))
+    assert e.value.code == kvp.ERR_RANGE
+    with pytest.raises(kvp.KvpError) as e:
+        kvp.Problem(U, 8192, 32769, to_dev(np.zeros((32769, 2), np.uint32)), cap, 8000 * GB, 900 * GB, 900 * GB)
+    assert e.value.code == kvp.ERR_RANGE
+    # a horizon the annealer can still hold: 8192 steps
+    S2 = 8192
+    A2 = wl.random_access(U, S2, 0.1, seed=81)
+    g2, o2 = both_problems(kvp, oracle, U, 8192, S2, A2, cap, (8000 * GB, 900 * GB, 900 * GB))
+    kw = dict(chains=3, moves=4000, levels=8, seed=4)
+    got = g2.anneal(g2.make_params(**kw), want_per_chain=True)
+    ref = o2.anneal(o2.make_params(**kw))
+    assert [r.astuple() for r in got["per_chain"]] == [r.astuple() for r in ref["per_chain"]]
+    assert np.array_equal(to_np(got["best_schedule"]), ref["best_schedule"])

@@ -306,6 +306,26 @@ int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const uint32_t* win
                          const uint32_t* ratios_permille, uint32_t n, uint32_t* schedules, void* stream);
 
 /*
+ * Reactive Scheduling (Section IV-A) as a schedule generator: a unit read while it is outside HBM is promoted, the
+ * least recently used resident makes room. The miss of step s is served off-package; the unit is resident from
+ * step s+1. Per step the hit units become most recently used; the missed units, in index order and at most
+ * `capacity` of them, first take free capacity and then replace residents in order of (last use, index).
+ *   schedule (device) [steps][W32]. Limit: units <= 32768. Asynchronous on `stream`.
+ */
+int kvp_policy_reactive(kvp_problem* p, uint32_t init_mode, uint32_t* schedule, void* stream);
+
+/*
+ * Page Granularity Scheduling (Section IV-A) as a schedule generator: placement in pages of page_units consecutive
+ * units (a power of two, 2..32, dividing `units`; the paper uses pages of 16 tokens) with perfect foresight of the
+ * current step. Before step s a page's score is the number of its units that step s reads; non-resident pages with
+ * a positive score, ranked by score (ties: lower index), first take free page slots (floor(capacity / page_units)
+ * pages), then the j-th remaining one replaces the j-th resident page in order of rising score while that score is
+ * lower. Initial placement: the first pages up to capacity.
+ *   schedule (device) [steps][W32]. Limit: units <= 32768. Asynchronous on `stream`.
+ */
+int kvp_policy_page(kvp_problem* p, uint32_t page_units, uint32_t* schedule, void* stream);
+
+/*
  * kvp_wr_grid -- T(W, R) of the look-ahead policy on the whole grid W = 1..w_max, R = r / (n_ratio - 1),
  * r = 0..n_ratio-1: runs kvp_policy_lookahead and kvp_eval on every grid point.
  *   table (device) [w_max][n_ratio] uint64 total ticks.

@@ -783,8 +783,10 @@ int kvpo_policy_reactive(const kvpo_problem *p, uint32_t init_mode, uint32_t *P)
         }
         qsort(res, nr, sizeof(fu_t), by_freq_asc);                   /* least recently used first */
         uint32_t vi = 0, promoted = 0;
+        const uint32_t *was = P + (size_t)s * p->W32;                /* who was resident while step s read */
         for (uint32_t u = 0; u < p->U && promoted < p->cap; ++u) {
-            if (in[u] || !bit_of(acc, u)) continue;
+            if (bit_of(was, u) || !bit_of(acc, u)) continue;        /* a miss is judged against row s, not against
+                                                                        evictions made a moment ago */
             if (occ < p->cap) ++occ;
             else { if (vi >= nr) break; in[res[vi].u] = 0; ++vi; }
             in[u] = 1; stamp[u] = s + 1; ++promoted;
@@ -894,5 +896,47 @@ int kvpo_wr_anneal(const uint64_t *table, uint32_t w_max, uint32_t n_ratio, cons
         res.iters_done = i; res.final_ticks = cur; res.final_w = w; res.final_r = r;
         results[c] = res;
     }
+    return KVPO_OK;
+}
+
+/*
+ * Page Granularity Scheduling (Section IV-A): placement is managed in pages of page_units consecutive units with
+ * perfect foresight of the current step's accesses. Before step s a page's score is the number of its units that
+ * step s reads; non-resident pages with a positive score, ranked by score (ties: lower page index), first take free
+ * page slots (capacity floor(cap / page_units) pages), then the j-th remaining one replaces the j-th resident page in
+ * order of rising score (ties: lower index) while that page's score is lower. Whole pages move, so the unaccessed
+ * units of a page ride along. Initial placement: the first pages up to capacity.
+ */
+int kvpo_policy_page(const kvpo_problem *p, uint32_t page_units, uint32_t *P)
+{
+    if (!p || !P || !page_units || page_units > 32 || (page_units & (page_units - 1)) || p->U % page_units)
+        return KVPO_ERR_ARG;
+    const uint32_t np = p->U / page_units, cap_pages = p->cap / page_units;
+    uint8_t *in = (uint8_t *)calloc(np, 1);
+    fu_t *cand = (fu_t *)malloc(sizeof(fu_t) * np), *res = (fu_t *)malloc(sizeof(fu_t) * np);
+    if (!in || !cand || !res) { free(in); free(cand); free(res); return KVPO_ERR_NOMEM; }
+    for (uint32_t g = 0; g < cap_pages; ++g) in[g] = 1;
+    for (uint32_t s = 0; s < p->S; ++s) {
+        uint32_t nc = 0, nr = 0;
+        for (uint32_t g = 0; g < np; ++g) {
+            uint32_t f = 0;
+            for (uint32_t i = 0; i < page_units; ++i) f += (uint32_t)bit_of(p->A + (size_t)s * p->W32, g * page_units + i);
+            if (in[g]) { res[nr].f = f; res[nr].u = g; ++nr; }
+            else if (f > 0) { cand[nc].f = f; cand[nc].u = g; ++nc; }
+        }
+        qsort(cand, nc, sizeof(fu_t), by_freq_desc);
+        qsort(res, nr, sizeof(fu_t), by_freq_asc);
+        uint32_t vi = 0, occ = nr;
+        for (uint32_t ci = 0; ci < nc; ++ci) {
+            if (occ < cap_pages) { in[cand[ci].u] = 1; ++occ; continue; }
+            if (vi >= nr || !(res[vi].f < cand[ci].f)) break;
+            in[res[vi].u] = 0; in[cand[ci].u] = 1; ++vi;
+        }
+        uint32_t *row = P + (size_t)s * p->W32;
+        memset(row, 0, (size_t)p->W32 * 4);
+        for (uint32_t g = 0; g < np; ++g)
+            if (in[g]) for (uint32_t i = 0; i < page_units; ++i) set_bit(row, g * page_units + i, 1);
+    }
+    free(in); free(cand); free(res);
     return KVPO_OK;
 }

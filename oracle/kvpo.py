@@ -307,3 +307,10 @@ def wr_anneal(table, wp):
     _chk(lib().kvpo_wr_anneal(_u64p(table), C.c_uint32(table.shape[0]), C.c_uint32(table.shape[1]), C.byref(wp),
                               _u32p(acc), _u32p(shifts), res), "wr_anneal")
     return list(res)
+
+
+def policy_page(prob, page_units):
+    """Schedule of page-granularity placement with perfect foresight of the current step -> uint32 [S][W32]."""
+    P = np.zeros((prob.steps, prob.w32), np.uint32)
+    _chk(lib().kvpo_policy_page(prob._h, C.c_uint32(page_units), _u32p(P)), "policy_page")
+    return P

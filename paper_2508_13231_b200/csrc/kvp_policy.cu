@@ -40,14 +40,18 @@ __device__ __forceinline__ uint32_t window_freq(const uint32_t* __restrict__ col
     return __popc(lo) + __popc(hi);
 }
 
+// The kernel also serves Page Granularity Scheduling: then an "entity" is a page of `page` consecutive units (a power
+// of two <= 32), its frequency is the number of its units the current step reads (W = 1), R = 1, the capacity is in
+// pages, the initial placement is the first pages, and each row is expanded from the page bitmap.
+// E entities, EW32 = ceil(E/32); for page == 1 entities are units and EW32 == W32.
 __global__ void __launch_bounds__(1024)
-lookahead_kernel(const uint32_t* __restrict__ Acol, const uint32_t* __restrict__ row0, uint32_t U, uint32_t S,
-                 uint32_t S32, uint32_t W32, uint32_t cap, const uint32_t* __restrict__ windows,
-                 const uint32_t* __restrict__ ratios, uint32_t* __restrict__ out)
+lookahead_kernel(const uint32_t* __restrict__ Acol, const uint32_t* __restrict__ Arows, const uint32_t* __restrict__ row0,
+                 uint32_t E, uint32_t page, uint32_t S, uint32_t S32, uint32_t W32, uint32_t EW32, uint32_t cap,
+                 const uint32_t* __restrict__ windows, const uint32_t* __restrict__ ratios, uint32_t* __restrict__ out)
 {
     extern __shared__ uint32_t sm[];
-    uint32_t* H = sm;                                    // [W32] resident bitmap
-    uint32_t* histC = H + W32;                           // [66] candidates by frequency
+    uint32_t* H = sm;                                    // [EW32] resident bitmap over entities
+    uint32_t* histC = H + EW32;                           // [66] candidates by frequency
     uint32_t* histR = histC + 66;                        // [66] residents by frequency
     uint32_t* warpC = histR + 66;                        // [32]
     uint32_t* warpR = warpC + 32;                        // [32]
@@ -56,10 +60,15 @@ lookahead_kernel(const uint32_t* __restrict__ Acol, const uint32_t* __restrict__
     uint8_t* fb = reinterpret_cast<uint8_t*>(ctl + 1);   // [rounds * T] frequency of every unit at this step
 
     const uint32_t T = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
-    const uint32_t W = windows[blockIdx.x], permille = ratios[blockIdx.x];
-    const uint32_t rounds = (W32 * 32 + T - 1) / T;
+    const uint32_t W = page > 1 ? page : windows[blockIdx.x];          // W doubles as the largest frequency class
+    const uint32_t permille = page > 1 ? 1000u : ratios[blockIdx.x];
+    const uint32_t U = E;                                              // entities are indexed like units below
+    const uint32_t rounds = (EW32 * 32 + T - 1) / T;
     uint32_t* mine = out + (size_t)blockIdx.x * S * W32;
-    for (uint32_t i = tid; i < W32; i += T) H[i] = __ldg(row0 + i);
+    for (uint32_t i = tid; i < EW32; i += T) {
+        if (row0) H[i] = __ldg(row0 + i);
+        else H[i] = cap >= i * 32 + 32 ? 0xFFFFFFFFu : (cap > i * 32 ? (1u << (cap - i * 32)) - 1u : 0u);
+    }
     __syncthreads();
     for (uint32_t s = 0; s < S; ++s) {
         for (uint32_t i = tid; i < 132; i += T) histC[i] = 0;          // both histograms
@@ -70,7 +79,13 @@ lookahead_kernel(const uint32_t* __restrict__ Acol, const uint32_t* __restrict__
             const uint32_t u = j * T + tid;
             uint32_t f = 0, in = 0;
             if (u < U) {
-                f = window_freq(Acol + (size_t)u * S32, S32, s, W);
+                if (page > 1) {
+                    const uint32_t first = u * page;                   // the page's units share one row word
+                    const uint32_t word = __ldg(Arows + (size_t)s * W32 + (first >> 5)) >> (first & 31);
+                    f = __popc(page == 32 ? word : word & ((1u << page) - 1u));
+                } else {
+                    f = window_freq(Acol + (size_t)u * S32, S32, s, W);
+                }
                 in = (H[u >> 5] >> (u & 31)) & 1u;
             }
             fb[u] = (uint8_t)f;
@@ -143,11 +158,122 @@ lookahead_kernel(const uint32_t* __restrict__ Acol, const uint32_t* __restrict__
             const bool leave = in && (f < c.frs || (tieR && rankR < c.takeR));
             const uint32_t bits = __ballot_sync(0xFFFFFFFFu, (in && !leave) || enter);
             __syncthreads();                             // every thread has read H and the warp counts of this round
-            if (lane == 0 && (u >> 5) < W32) { H[u >> 5] = bits; mine[(size_t)s * W32 + (u >> 5)] = bits; }
+            if (lane == 0 && (u >> 5) < EW32) {
+                H[u >> 5] = bits;
+                if (page == 1) mine[(size_t)s * W32 + (u >> 5)] = bits;
+            }
             if (tid == 0) {
                 uint32_t a = 0, b = 0;
                 for (uint32_t w = 0; w < nwarps; ++w) { a += warpC[w]; b += warpR[w]; }
                 run[0] += a; run[1] += b;
+            }
+            __syncthreads();
+        }
+        if (page > 1) {                                  // every resident page contributes `page` ones to the row
+            const uint32_t per_word = 32 / page;
+            for (uint32_t w = tid; w < W32; w += T) {
+                const uint32_t e0 = w * per_word;
+                uint32_t eb = H[e0 >> 5] >> (e0 & 31), word = 0;
+                const uint32_t ones = page == 32 ? 0xFFFFFFFFu : (1u << page) - 1u;
+                for (uint32_t i = 0; i < per_word; ++i)
+                    if ((eb >> i) & 1u) word |= ones << (i * page);
+                mine[(size_t)s * W32 + w] = word;
+            }
+        }
+    }
+}
+
+// Sum of a per-thread value over the CTA; every thread gets the result. Needs a zeroed shared counter per call.
+__device__ __forceinline__ uint32_t cta_sum(uint32_t v, uint32_t* slot)
+{
+    v = __reduce_add_sync(0xFFFFFFFFu, v);
+    if ((threadIdx.x & 31) == 0 && v) atomicAdd(slot, v);
+    __syncthreads();
+    return *slot;
+}
+
+// Reactive Scheduling (Section IV-A): promote on miss, evict the least recently used. One CTA walks the steps; row
+// s+1 follows from row s and the accesses of step s. Per step: hits refresh their stamp; the first min(misses, cap)
+// missed units in index order are promoted; they take free capacity first and then the places of the residents with
+// the smallest (stamp, index), found by a bitwise search for the stamp threshold and a ballot ranking of the ties.
+__global__ void __launch_bounds__(1024)
+reactive_kernel(const uint32_t* __restrict__ Arows, const uint32_t* __restrict__ row0, uint32_t U, uint32_t S,
+                uint32_t W32, uint32_t cap, uint32_t* __restrict__ out)
+{
+    extern __shared__ uint32_t sm[];
+    uint32_t* H = sm;                                    // [W32]
+    uint32_t* cnt = H + W32;                             // [24] block counters of one step
+    uint32_t* warpV = cnt + 24;                          // [32]
+    uint32_t* warpM = warpV + 32;                        // [32]
+    uint32_t* run = warpM + 32;                          // [2]
+    uint16_t* stamp = reinterpret_cast<uint16_t*>(run + 2);   // [rounds * T] step of last use + 1, 0 = never
+    const uint32_t T = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = T >> 5;
+    const uint32_t rounds = (W32 * 32 + T - 1) / T;
+    for (uint32_t i = tid; i < W32; i += T) { H[i] = __ldg(row0 + i); out[i] = H[i]; }
+    for (uint32_t i = tid; i < rounds * T; i += T) stamp[i] = 0;
+    __syncthreads();
+    for (uint32_t s = 0; s + 1 < S; ++s) {
+        for (uint32_t i = tid; i < 24; i += T) cnt[i] = 0;
+        if (tid == 0) { run[0] = 0; run[1] = 0; }
+        __syncthreads();
+        uint32_t my_miss = 0, my_res = 0;
+        for (uint32_t j = 0; j < rounds; ++j) {
+            const uint32_t u = j * T + tid;
+            if (u < U) {
+                const uint32_t a = (__ldg(Arows + (size_t)s * W32 + (u >> 5)) >> (u & 31)) & 1u;
+                const uint32_t in = (H[u >> 5] >> (u & 31)) & 1u;
+                if (a & in) stamp[u] = (uint16_t)(s + 1);
+                my_miss += a & ~in & 1u;
+                my_res += in;
+            }
+        }
+        const uint32_t nM = cta_sum(my_miss, cnt + 0), nR = cta_sum(my_res, cnt + 1);
+        const uint32_t promoted = min(nM, cap), free_slots = cap - nR;
+        const uint32_t evict = promoted > free_slots ? promoted - free_slots : 0u;
+        // smallest stamp value tau with |{resident, stamp <= tau}| >= evict, bit by bit from the top (stamps < 2^16)
+        uint32_t tau = 0, takeV = 0;
+        if (evict) {
+            for (int bit = 15; bit >= 0; --bit) {
+                const uint32_t probe = tau | (1u << bit);             // is the answer >= probe?  <=> count(stamp < probe) < evict
+                uint32_t c = 0;
+                for (uint32_t j = 0; j < rounds; ++j) {
+                    const uint32_t u = j * T + tid;
+                    if (u < U && ((H[u >> 5] >> (u & 31)) & 1u) && stamp[u] < probe) ++c;
+                }
+                if (cta_sum(c, cnt + 2 + (15 - bit)) < evict) tau = probe;
+            }
+            uint32_t c = 0;
+            for (uint32_t j = 0; j < rounds; ++j) {
+                const uint32_t u = j * T + tid;
+                if (u < U && ((H[u >> 5] >> (u & 31)) & 1u) && stamp[u] < tau) ++c;
+            }
+            takeV = evict - cta_sum(c, cnt + 18);
+        }
+        __syncthreads();
+        for (uint32_t j = 0; j < rounds; ++j) {
+            const uint32_t u = j * T + tid;
+            const bool ok = u < U;
+            const bool in = ok && ((H[u >> 5] >> (u & 31)) & 1u);
+            const bool a = ok && ((__ldg(Arows + (size_t)s * W32 + (u >> 5)) >> (u & 31)) & 1u);
+            const uint32_t st = ok ? stamp[u] : 0u;
+            const bool miss = a && !in, tieV = in && evict && st == tau;
+            const uint32_t bv = __ballot_sync(0xFFFFFFFFu, tieV), bm = __ballot_sync(0xFFFFFFFFu, miss);
+            if (lane == 0) { warpV[warp] = __popc(bv); warpM[warp] = __popc(bm); }
+            __syncthreads();
+            uint32_t rankV = run[0], rankM = run[1];
+            for (uint32_t w = 0; w < warp; ++w) { rankV += warpV[w]; rankM += warpM[w]; }
+            rankV += __popc(bv & ((1u << lane) - 1u));
+            rankM += __popc(bm & ((1u << lane) - 1u));
+            const bool leave = in && evict && (st < tau || (tieV && rankV < takeV));
+            const bool enter = miss && rankM < promoted;
+            if (enter) stamp[u] = (uint16_t)(s + 1);
+            const uint32_t bits = __ballot_sync(0xFFFFFFFFu, (in && !leave) || enter);
+            __syncthreads();
+            if (lane == 0 && (u >> 5) < W32) { H[u >> 5] = bits; out[(size_t)(s + 1) * W32 + (u >> 5)] = bits; }
+            if (tid == 0) {
+                uint32_t x = 0, y = 0;
+                for (uint32_t w = 0; w < nwarps; ++w) { x += warpV[w]; y += warpM[w]; }
+                run[0] += x; run[1] += y;
             }
             __syncthreads();
         }
@@ -209,6 +335,53 @@ __global__ void wr_anneal_kernel(const WRK k, kvp_wr_result* __restrict__ result
 
 using namespace kvp;
 
+static size_t policy_smem(uint32_t EW32, uint32_t rounds, uint32_t T)
+{
+    return ((size_t)EW32 + 66 + 66 + 32 + 32 + 2 + 4) * 4 + (size_t)rounds * T;
+}
+
+extern "C" int kvp_policy_reactive(kvp_problem* p, uint32_t init_mode, uint32_t* schedule, void* stream)
+{
+    if (!p || !schedule || init_mode > KVP_INIT_STATIC_FREQ) return KVP_ERR_ARG;
+    if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;        // stamps are 16 bits and live in shared memory
+    KVP_CUDA(cudaSetDevice(p->device));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t T = (p->U + 31) / 32 * 32;
+    if (T > 1024) T = 1024;
+    const uint32_t rounds = (p->W32 * 32 + T - 1) / T;
+    const size_t smem = ((size_t)p->W32 + 24 + 32 + 32 + 2) * 4 + (size_t)rounds * T * 2;
+    const uint32_t* row = p->d_row_freq;
+    if (init_mode == KVP_INIT_STATIC_FIRST) {
+        int rc = ensure_scratch(p, (size_t)p->W32 * 4, st);
+        if (rc) return rc;
+        if ((rc = launch_static_first_row(p, static_cast<uint32_t*>(p->d_scratch), st))) return rc;
+        row = static_cast<uint32_t*>(p->d_scratch);
+    }
+    KVP_CUDA(cudaFuncSetAttribute(reactive_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    reactive_kernel<<<1, T, smem, st>>>(p->dA, row, p->U, p->S, p->W32, p->cap, schedule);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+extern "C" int kvp_policy_page(kvp_problem* p, uint32_t page_units, uint32_t* schedule, void* stream)
+{
+    if (!p || !schedule || page_units < 2 || page_units > 32 || (page_units & (page_units - 1)) || p->U % page_units)
+        return KVP_ERR_ARG;
+    if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;
+    KVP_CUDA(cudaSetDevice(p->device));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t E = p->U / page_units, EW32 = (E + 31) / 32;
+    uint32_t T = (E + 31) / 32 * 32;
+    if (T > 1024) T = 1024;
+    const uint32_t rounds = (EW32 * 32 + T - 1) / T;
+    const size_t smem = policy_smem(EW32, rounds, T);
+    KVP_CUDA(cudaFuncSetAttribute(lookahead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    lookahead_kernel<<<1, T, smem, st>>>(p->dAcol, p->dA, nullptr, E, page_units, p->S, p->S32, p->W32, EW32,
+                                         p->cap / page_units, nullptr, nullptr, schedule);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
 extern "C" int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const uint32_t* windows, const uint32_t* ratios_permille,
                                     uint32_t n, uint32_t* schedules, void* stream)
 {
@@ -221,7 +394,7 @@ extern "C" int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const ui
     uint32_t T = (p->U + 31) / 32 * 32;
     if (T > 1024) T = 1024;
     const uint32_t rounds = (p->W32 * 32 + T - 1) / T;
-    const size_t smem = ((size_t)p->W32 + 66 + 66 + 32 + 32 + 2 + 4) * 4 + (size_t)rounds * T;
+    const size_t smem = policy_smem(p->W32, rounds, T);
     // per-call parameters and, for the first-come placement, its row
     int rc = ensure_scratch(p, ((size_t)2 * n + p->W32) * 4 + 256, st);
     if (rc) return rc;
@@ -236,7 +409,8 @@ extern "C" int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const ui
         row = d_row;
     }
     KVP_CUDA(cudaFuncSetAttribute(lookahead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    lookahead_kernel<<<n, T, smem, st>>>(p->dAcol, row, p->U, p->S, p->S32, p->W32, p->cap, d_w, d_r, schedules);
+    lookahead_kernel<<<n, T, smem, st>>>(p->dAcol, p->dA, row, p->U, 1u, p->S, p->S32, p->W32, p->W32, p->cap, d_w, d_r,
+                                         schedules);
     KVP_CUDA(cudaGetLastError());
     KVP_CUDA(cudaStreamSynchronize(st));                             // the host arrays may go away
     return KVP_OK;

@@ -23,7 +23,7 @@ NOALLOC_SCRATCH_BYTES = 1 << 20
 EXPORTS = [
     "kvp_create", "kvp_destroy", "kvp_get_info", "kvp_eval", "kvp_eval_counts", "kvp_eval_noalloc", "kvp_accept_table", "kvp_anneal",
     "kvp_anneal_chain_state", "kvp_trace_generate", "kvp_philox4x32_10", "kvp_strerror", "kvp_last_cuda_error",
-    "kvp_policy_lookahead", "kvp_wr_grid", "kvp_wr_anneal",
+    "kvp_policy_lookahead", "kvp_policy_reactive", "kvp_policy_page", "kvp_wr_grid", "kvp_wr_anneal",
 ]
 
 
@@ -295,6 +295,18 @@ class Problem:
         out = torch.empty((n, self.steps, self.w32), dtype=torch.int32, device="cuda")
         _chk(_lib().kvp_policy_lookahead(self._h, C.c_uint32(init_mode), w, r, C.c_uint32(n), _ptr(out), _stream(stream)),
              "kvp_policy_lookahead")
+        return out
+
+    def policy_reactive(self, init_mode=INIT_STATIC_FIRST, stream=None):
+        """kvp_policy_reactive -> CUDA int32 [S][W32]."""
+        out = torch.empty((self.steps, self.w32), dtype=torch.int32, device="cuda")
+        _chk(_lib().kvp_policy_reactive(self._h, C.c_uint32(init_mode), _ptr(out), _stream(stream)), "kvp_policy_reactive")
+        return out
+
+    def policy_page(self, page_units, stream=None):
+        """kvp_policy_page -> CUDA int32 [S][W32]."""
+        out = torch.empty((self.steps, self.w32), dtype=torch.int32, device="cuda")
+        _chk(_lib().kvp_policy_page(self._h, C.c_uint32(page_units), _ptr(out), _stream(stream)), "kvp_policy_page")
         return out
 
     def wr_grid(self, w_max, n_ratio=11, init_mode=INIT_STATIC_FIRST, stream=None):

@@ -76,3 +76,30 @@ def test_wr_grid_and_annealer(kvp, oracle):
     with pytest.raises(kvp.KvpError) as e:
         kvp.wr_anneal(table, kvp.wr_params(chains=1, iters=10, w0=21))
     assert e.value.code == kvp.ERR_ARG
+
+
+@pytest.mark.parametrize("U,S,cap", [(4, 4, 2), (60, 50, 12), (33, 1, 5), (1, 9, 1), (300, 65, 0), (1000, 130, 1000),
+                                     (2085, 77, 400), (4096, 200, 100)])
+def test_reactive_parity(kvp, oracle, U, S, cap):
+    A = wl.random_access(U, S, 0.15, seed=U + S + 1)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    for init in (kvp.INIT_STATIC_FIRST, kvp.INIT_STATIC_FREQ):
+        assert np.array_equal(to_np(g.policy_reactive(init_mode=init)), oracle.policy_reactive(o, init_mode=init)), init
+
+
+@pytest.mark.parametrize("U,S,cap,page", [(8, 2, 2, 2), (128, 30, 40, 8), (4096, 64, 1024, 16), (4096, 64, 1000, 32),
+                                          (64, 5, 64, 4), (96, 7, 0, 16), (32768, 12, 5000, 16)])
+def test_page_parity(kvp, oracle, U, S, cap, page):
+    A = wl.random_access(U, S, 0.1, seed=U + S + page)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    assert np.array_equal(to_np(g.policy_page(page)), oracle.policy_page(o, page))
+    for bad in (1, 3, 64):
+        with pytest.raises(kvp.KvpError) as e:
+            g.policy_page(bad)
+        assert e.value.code == kvp.ERR_ARG
+
+
+def test_named_policies(kvp, oracle):
+    g, o, cfg, A = named_problem(kvp, oracle, "layer_8b")
+    assert np.array_equal(to_np(g.policy_reactive()), oracle.policy_reactive(o))
+    assert np.array_equal(to_np(g.policy_page(16)), oracle.policy_page(o, 16))

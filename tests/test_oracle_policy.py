@@ -35,11 +35,16 @@ def test_hand_worked_policies(oracle):
             W, R = int(f[1][2:]), int(f[2][2:])
             got = wl.unpack_bits(oracle.policy_lookahead(look, W, R), 4)
             assert np.array_equal(got, _bits(_rows(f[4]), 4)), line
-        else:
+        elif f[0] == "reactive":
             got = wl.unpack_bits(oracle.policy_reactive(react), 4)
             assert np.array_equal(got, _bits(_rows(f[2]), 4)), line
+        else:
+            A_pg = wl.pack_bits(_bits([[2, 3, 5], [4, 5, 6]], 8))
+            pg = oracle.Problem(8, 8192, 2, A_pg, 2, 8000 * GB, 900 * GB, 900 * GB)
+            got = wl.unpack_bits(oracle.policy_page(pg, 2), 8)
+            assert np.array_equal(got, _bits(_rows(f[2]), 8)), line
         n += 1
-    assert n == 5
+    assert n == 6
 
 
 def test_lookahead_invariants(oracle):
@@ -80,6 +85,20 @@ def test_reactive_invariants(oracle):
             assert np.all(bits[s + 1, hit] == 1)                 # what was just used is not the LRU victim
         if missed.size == 0:
             assert np.array_equal(bits[s + 1], bits[s])          # no miss, no migration
+
+
+def test_page_invariants(oracle):
+    U, S, cap, page = 128, 30, 40, 8
+    A = wl.random_access(U, S, 0.1, seed=43)
+    prob = oracle.Problem(U, 8192, S, A, cap, 8000 * GB, 900 * GB, 900 * GB)
+    bits = wl.unpack_bits(oracle.policy_page(prob, page), U).reshape(S, U // page, page)
+    assert np.all((bits.sum(axis=2) == 0) | (bits.sum(axis=2) == page))          # whole pages only
+    assert np.all((bits.sum(axis=2) > 0).sum(axis=1) <= cap // page)              # capacity in pages
+    a = wl.unpack_bits(A, U).reshape(S, U // page, page).sum(axis=2)
+    res = bits[:, :, 0].astype(bool)
+    for s in range(S):                                                            # no resident page scores less than
+        if (~res[s]).any() and res[s].any() and (a[s][~res[s]] > 0).any():        # a page left outside
+            assert a[s][res[s]].min() >= a[s][~res[s]].max()
 
 
 def test_policies_reproduce_the_papers_ordering_on_a_synthetic_trace(oracle):

@@ -88,6 +88,22 @@ def trace_params(name, seed=0):
         burst_thr=int(cfg["burst_p"] * 2 ** 32), base=base)
 
 
+def custom_trace_params(groups, units_per_group, steps, topk, rho, sigma=1.0, zipf=None, seed=0):
+    """Trace parameters for an ad-hoc shape (same recipe as the named configurations, no recency, no bursts)."""
+    rng = np.random.Generator(np.random.PCG64([seed, 0x637573]))
+    base = None
+    if zipf is not None:
+        lo, hi = zipf
+        base = np.zeros((groups, units_per_group), np.int64)
+        for g in range(groups):
+            s_g = lo if lo == hi else rng.uniform(lo, hi)
+            base[g] = -np.rint(s_g * np.log(rng.permutation(units_per_group) + 1.0) * Q16).astype(np.int64)
+        base = base.reshape(-1).astype(np.int32)
+    return dict(groups=groups, units_per_group=units_per_group, steps=steps, topk=topk, seed=seed,
+                rho_q=int(round(rho * Q16)), c_q=int(round(sigma * math.sqrt(1.0 - rho * rho) * Q16)),
+                sigma_q=int(round(sigma * Q16)), burst_jump=0, burst_thr=0, base=base)
+
+
 def random_schedules(num_units, steps, cap, count, seed, churn=0.02):
     """`count` random feasible schedules, uint32 [count][steps][ceil(U/32)].
 

@@ -42,7 +42,7 @@ struct ChainParams {
 };
 
 // Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
-// Measured on 256 units x 512 steps, 1024 chains: kMPL = 2 is slower (7.1 ms vs 5.25 ms per 10^8 moves): a move that
+// Measured on 256 units x 512 steps, 1024 chains: kMPL = 2 is slower (6.0 ms vs 5.25 ms per 10^8 moves): a move that
 // changes the schedule then costs a re-evaluation pass over twice as many proposals. Serving a chain with two warps
 // that evaluate side by side and commit in turn was tried as well and was no faster (5.9 ms).
 constexpr int kMPL = 1;

@@ -31,6 +31,9 @@ UNIT = "move-evals/s"
 # and push ~100, about 35 (lane, step) cost evaluations of ~70 thread instructions each in two warp rounds
 # ~150, Metropolis and in-order commit ~50).
 ISSUE_PEAK_GWIPS = 148 * 4 * 1.965
+# dram__bytes_read.sum + dram__bytes_write.sum of one chain-kernel launch on this workload (ncu capture summarised in
+# profiles/chain_kernel_single_head.md; set to None whenever the kernel changes until it is captured again)
+CHAIN_KERNEL_DRAM_BYTES = 354304
 ALG_WARP_INSTR_PER_MOVE = 16.0
 
 
@@ -117,7 +120,7 @@ def cpu_baseline(cfg, tp):
     from oracle import kvpo
     from paper_2508_13231_b200 import workloads as wl
     kvpo.build()
-    sample_chains = 256
+    sample_chains = 768
     t0 = time.perf_counter()
     A = kvpo.trace_generate(**tp)
     o = kvpo.Problem(wl.units(cfg), cfg["bytes_per_unit"], cfg["steps"], A, cfg["cap"], *cfg["bw"])
@@ -348,7 +351,7 @@ def main():
             "gpu_launches": launches[0] * args.steps,
             "roofline": {"bound": "alu", "kernel": "chain_kernel<smem>", "achieved": achieved,
                          "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
-                         "traffic": None, "ms_per_launch": per_launch_ms,
+                         "traffic": CHAIN_KERNEL_DRAM_BYTES, "ms_per_launch": per_launch_ms,
                          "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"},
             "bound_ticks": out["best_ticks"], "init_ticks": out["stats"].init_ticks,
         }

@@ -32,6 +32,9 @@ struct ChainParams {
     uint32_t* dump;              // if set, slot 0 writes its final schedule here (time-packed)
     const uint32_t* full0;       // [S32] full-step bitmap of the initial schedule
     uint32_t* snap;              // if set: [slots][U*S32], each chain's schedule when it reached its best
+    uint64_t* undo_log;          // if set: [slots][undo_cap] indices of the moves applied since the best state
+    uint32_t* undo_len;          // [slots] how many there were (more than undo_cap: the log overflowed)
+    uint32_t undo_cap;
     CostK K;
     uint32_t U, S, S32, cap;
     uint32_t chain_first, chain_count, result_base;
@@ -342,6 +345,8 @@ chain_kernel(const ChainParams prm)
     uint64_t next_boundary = prm.levels > 1 ? prm.per_level : ~0ull;
     uint64_t m = 0;
     bool snap_dirty = false;                                      // the best state is the current one, not yet saved
+    uint64_t* ulog = prm.undo_log ? prm.undo_log + (size_t)slot * prm.undo_cap : nullptr;
+    uint32_t ulen = 0;                                            // moves applied since the best state
     while (m < prm.upto) {
         if (m == next_boundary) {                                 // a new temperature level starts at this move
             ++level;
@@ -409,7 +414,11 @@ chain_kernel(const ChainParams prm)
                 cur = after;
                 const uint64_t mb = m + 32u * h + b;
                 hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
-                if (cur < best) { best = cur; best_move = mb; snap_dirty = true; }
+                if (cur < best) { best = cur; best_move = mb; snap_dirty = true; ulen = 0; }
+                else if (ulog) {                                  // every move is its own inverse: remember it
+                    if (ulen < prm.undo_cap && lane == 0) ulog[ulen] = mb;
+                    if (ulen <= prm.undo_cap) ++ulen;
+                }
                 todo[h] &= ~done;
                 // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later proposal
                 // read steps s0 - 1 .. s0 + len: it has to be evaluated again iff the two ranges meet.
@@ -426,6 +435,7 @@ chain_kernel(const ChainParams prm)
         m += nb;
     }
     if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
+    if (ulog && lane == 0) prm.undo_len[slot] = ulen;
     if (lane == 0) {
         kvp_chain_result res;
         res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m;
@@ -436,6 +446,45 @@ chain_kernel(const ChainParams prm)
         __syncwarp();
         copy_words(prm.dump, cv.P, pwords, lane);
     }
+}
+
+// Takes a finished chain's schedule back to its best state: the moves applied after the best were logged, each
+// swap or flip is its own inverse, so applying them again in reverse order undoes them. One warp; only the
+// schedule words are touched (the counters are not needed any more).
+__global__ void __launch_bounds__(32)
+undo_kernel(const ChainParams prm, uint32_t slot, uint32_t* __restrict__ dst)
+{
+    const uint32_t lane = threadIdx.x, S = prm.S, S32 = prm.S32;
+    const size_t pwords = (size_t)prm.U * S32;
+    uint32_t* P = prm.ws + (size_t)slot * pwords;
+    const uint64_t* ulog = prm.undo_log + (size_t)slot * prm.undo_cap;
+    const uint32_t n = prm.undo_len[slot], chain = prm.chain_first + slot;
+    for (uint32_t i = n; i-- > 0;) {
+        const uint64_t m = ulog[i];
+        uint32_t r[4];
+        LaneMove mv;
+        philox4x32_10((uint32_t)m, (uint32_t)(m >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
+        decode_move(r, prm.p_swap_256, prm.len_choices, S, prm.U, mv);
+        const bool swap = mv.pk & 1u;
+        const uint32_t len = (mv.pk >> 1) & 63u, s0 = mv.pk >> 8, end = min(s0 + len, S);
+        if (lane < 2) {
+            const uint32_t wj = (s0 >> 5) + lane;
+            const uint32_t lo = max(s0, wj * 32u), hi = min(end, wj * 32u + 32u);
+            if (hi > lo) {                               // run lengths are at most 30, so never a full word
+                const uint32_t mask = ((1u << (hi - lo)) - 1u) << (lo - wj * 32u);
+                const size_t iu = (size_t)mv.u * S32 + wj, iv = (size_t)mv.v * S32 + wj;
+                if (swap) {
+                    const uint32_t a = P[iu], b = P[iv], d = (a ^ b) & mask;
+                    if (d) { P[iu] = a ^ d; P[iv] = b ^ d; }
+                } else {
+                    P[iu] ^= mask;
+                }
+            }
+        }
+        __syncwarp();
+    }
+    __syncwarp();
+    copy_words(dst, P, pwords, lane);
 }
 
 // bit t of full0 is set iff the initial schedule fills the HBM capacity at step t
@@ -520,6 +569,9 @@ struct Ctx {
     uint32_t* slots;         // chain state slices (global variant)
     uint32_t* full0;         // [S32]
     uint32_t* snap;          // best-state snapshots (shared-memory variant), or null
+    uint64_t* undo_log;      // undo logs (global variant), or null
+    uint32_t* undo_len;
+    uint32_t undo_cap;
     bool psmem;
     uint32_t wpb;            // warps per CTA
     uint32_t resident;       // chains per wave
@@ -551,10 +603,11 @@ int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 }
 
 int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp_chain_result* results, uint64_t upto,
-               uint32_t* dump, uint32_t* snap)
+               uint32_t* dump, uint32_t* snap, bool with_undo = false)
 {
     ChainParams prm = c.prm;
     prm.snap = snap;
+    prm.undo_log = with_undo ? c.undo_log : nullptr; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
     prm.chain_first = first; prm.chain_count = count; prm.result_base = result_base;
     prm.results = results; prm.upto = upto; prm.dump = dump;
     ++c.launches;
@@ -635,6 +688,10 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const size_t snap_bytes = (size_t)a->chains * p->U * p->S32 * 4;
     const bool snapshots = c.psmem && snap_bytes <= ((size_t)2 << 30);
     const size_t o_snap = take(snapshots ? snap_bytes : 0);
+    // Chains in global scratch log the moves they apply after their best state (8 bytes each, up to 4096), so that
+    // the winner can be walked back instead of replayed from its first move.
+    c.undo_cap = c.psmem ? 0u : 4096u;
+    const size_t o_ulog = take((size_t)c.resident * c.undo_cap * 8), o_ulen = take(c.psmem ? 0 : (size_t)c.resident * 4);
     rc = ensure_chain_ws(p, off, st);
     if (rc) return rc;
     char* base = static_cast<char*>(p->d_chain_ws);
@@ -643,6 +700,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     c.results = (kvp_chain_result*)(base + o_res); c.dumpcol = (uint32_t*)(base + o_dump);
     c.sched = (uint32_t*)(base + o_sched); c.slots = (uint32_t*)(base + o_slots);
     c.full0 = (uint32_t*)(base + o_full); c.snap = snapshots ? (uint32_t*)(base + o_snap) : nullptr;
+    c.undo_log = c.psmem ? nullptr : (uint64_t*)(base + o_ulog); c.undo_len = c.psmem ? nullptr : (uint32_t*)(base + o_ulen);
 
     // initial schedule in both layouts
     if (a->init_mode == KVP_INIT_USER) {
@@ -747,25 +805,55 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     KVP_CUDA(cudaEventRecord(ev[1], st));
 
     // the chains, one wave of resident chains after the other
-    for (uint32_t first = 0; first < a->chains; first += c.resident) {
+    ReduceOut* red_dev = reinterpret_cast<ReduceOut*>(c.small + 8);
+    ReduceOut red;
+    memset(&red, 0, sizeof red);
+    uint32_t dumped_chain = 0xFFFFFFFFu;                  // call-local index of the chain whose best state is in dumpcol
+    uint32_t waves = 0;
+    for (uint32_t first = 0; first < a->chains; first += c.resident, ++waves) {
         const uint32_t count = a->chains - first < c.resident ? a->chains - first : c.resident;
-        if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr, c.snap))) {
+        if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr, c.snap,
+                             c.undo_log != nullptr))) {
             cleanup(); return rc;
+        }
+        if (c.undo_log) {
+            // Best so far over the chains that have finished; if it belongs to this wave, walk that chain back to
+            // its best state while its scratch slice still holds its final state.
+            reduce_kernel<<<1, 1024, 0, st>>>(c.results, first + count, red_dev);
+            KVP_CUDA(cudaGetLastError());
+            ++c.launches;
+            KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
+            KVP_CUDA(cudaStreamSynchronize(st));
+            if (red.best_chain >= first && red.best_move != ~0ull) {
+                uint32_t len = 0;
+                KVP_CUDA(cudaMemcpyAsync(&len, c.undo_len + (red.best_chain - first), 4, cudaMemcpyDeviceToHost, st));
+                KVP_CUDA(cudaStreamSynchronize(st));
+                if (len <= c.undo_cap) {
+                    ChainParams prm = c.prm;
+                    prm.chain_first = a->first_chain + first;
+                    prm.undo_log = c.undo_log; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
+                    undo_kernel<<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
+                    KVP_CUDA(cudaGetLastError());
+                    ++c.launches;
+                    dumped_chain = red.best_chain;
+                }
+            }
         }
     }
     KVP_CUDA(cudaEventRecord(ev[2], st));
 
-    // cross-chain reduction, then the winner's schedule by deterministic replay and a re-score
-    ReduceOut* red_dev = reinterpret_cast<ReduceOut*>(c.small + 8);
-    reduce_kernel<<<1, 1024, 0, st>>>(c.results, a->chains, red_dev);
-    KVP_CUDA(cudaGetLastError());
-    ++c.launches;
-    ReduceOut red;
-    KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
-    KVP_CUDA(cudaStreamSynchronize(st));
+    // cross-chain reduction, then the winner's schedule (its own snapshot, its walked-back state, or a replay) and a
+    // re-score
+    if (!c.undo_log) {
+        reduce_kernel<<<1, 1024, 0, st>>>(c.results, a->chains, red_dev);
+        KVP_CUDA(cudaGetLastError());
+        ++c.launches;
+        KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
+        KVP_CUDA(cudaStreamSynchronize(st));
+    }
     const uint64_t upto = red.best_move == ~0ull ? 0 : red.best_move + 1;
-    if (c.snap && upto) {                                  // the winner saved its best state itself
-        const uint32_t* col = c.snap + (size_t)red.best_chain * p->U * p->S32;
+    if (upto && (c.snap || dumped_chain == red.best_chain)) {
+        const uint32_t* col = c.snap ? c.snap + (size_t)red.best_chain * p->U * p->S32 : c.dumpcol;
         if ((rc = launch_bit_transpose(col, p->U, p->S32, p->S, c.sched, p->W32, st))) { cleanup(); return rc; }
         ++c.launches;
         red.best_chain += a->first_chain;                  // the reduction works on call-local indices

@@ -176,3 +176,19 @@ def test_anneal_full_size_sampled_chains(kvp, oracle, name, chains, moves):
     ev = g.eval(out["best_schedule"])
     assert int(ev["total_ticks"][0]) == out["best_ticks"] and int(ev["bad_step"][0]) == -1
     assert out["best_ticks"] <= out["stats"].init_ticks
+
+
+def test_global_state_winner_paths(kvp, oracle):
+    # chains in global scratch rebuild the winner by walking its logged moves back; check the three ways this can go:
+    # a short log, a log that overflows (hot start: thousands of applied moves after the best; falls back to a replay),
+    # and a winner from an earlier wave of a run with more chains than are resident at once
+    g, o, cfg, A = named_problem(kvp, oracle, "layer_8b")
+    for kw in (dict(chains=8, moves=30_000, seed=3, p0=1e-3), dict(chains=8, moves=40_000, seed=3, p0=0.8, levels=4),
+               dict(chains=2500, moves=600, seed=5, p0=1e-3, levels=4)):
+        gp, op = _params(g, o, **kw)
+        out = g.anneal(gp, want_per_chain=True)
+        w = out["stats"].best_chain
+        assert w == min(range(kw["chains"]), key=lambda c: (out["per_chain"][c].best_ticks, c))
+        ref, _, bst = o.anneal_chains(op, w, 1, want_best=True)
+        assert ref[0].astuple() == out["per_chain"][w].astuple()
+        assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks

@@ -25,28 +25,28 @@ CONFIGS = {
     "tiny": dict(groups=1, units_per_group=16, steps=32, topk=4, bytes_per_unit=8192, cap=6,
                  bw=(8 * TB, 1 * TB, 1 * TB), rho=0.9, sigma=1.0, zipf=None,
                  recency_blocks=2, recency_boost=2.0, burst_p=0.0, burst_jump=0.0,
-                 chains=64, moves=10_000, p0=1e-3),
+                 chains=64, moves=10_000, p0=1e-6),
     "single_head": dict(groups=1, units_per_group=256, steps=512, topk=26, bytes_per_unit=8192, cap=64,
                         bw=(8 * TB, 9 * TB // 10, 9 * TB // 10), rho=0.95, sigma=1.0, zipf=(1.1, 1.1),
                         recency_blocks=0, recency_boost=0.0, burst_p=0.0, burst_jump=0.0,
-                        chains=1024, moves=100_000, p0=1e-3),
+                        chains=1024, moves=100_000, p0=1e-6),
     "layer_8b": dict(groups=8, units_per_group=2048, steps=256, topk=256, bytes_per_unit=8192, cap=4915,
                      bw=(8 * TB, 9 * TB // 10, 9 * TB // 10), rho=0.98, sigma=1.0, zipf=(0.8, 1.4),
                      recency_blocks=0, recency_boost=0.0, burst_p=0.0, burst_jump=0.0,
-                     chains=1024, moves=200_000, p0=1e-3),
+                     chains=1024, moves=200_000, p0=1e-6),
     "full_8b": dict(groups=256, units_per_group=2048, steps=128, topk=205, bytes_per_unit=8192, cap=104857,
                     bw=(8 * TB, 9 * TB // 10, 9 * TB // 10), rho=0.97, sigma=1.0, zipf=None,
                     recency_blocks=16, recency_boost=16.0, burst_p=0.0, burst_jump=0.0,
-                    chains=4096, moves=250_000, p0=1e-3),
+                    chains=4096, moves=250_000, p0=1e-6),
     "long_70b": dict(groups=640, units_per_group=4096, steps=64, topk=205, bytes_per_unit=16384, cap=262144,
                      bw=(8 * TB, 45 * TB // 100, 45 * TB // 100), rho=0.95, sigma=1.0, zipf=None,
                      recency_blocks=0, recency_boost=0.0, burst_p=0.01, burst_jump=4.0,
-                     chains=8192, moves=1_000_000, p0=1e-3),
+                     chains=8192, moves=1_000_000, p0=1e-6),
     # Table I bandwidths (4.9 TB/s HBM, 900 GB/s link, 500 GB/s DRAM) on the layer_8b shape
     "gh200": dict(groups=8, units_per_group=2048, steps=256, topk=256, bytes_per_unit=8192, cap=4915,
                   bw=(49 * TB // 10, 9 * TB // 10, 5 * TB // 10), rho=0.98, sigma=1.0, zipf=(0.8, 1.4),
                   recency_blocks=0, recency_boost=0.0, burst_p=0.0, burst_jump=0.0,
-                  chains=1024, moves=200_000, p0=1e-3),
+                  chains=1024, moves=200_000, p0=1e-6),
 }
 ORDER = ["tiny", "single_head", "layer_8b", "full_8b", "long_70b"]
 

@@ -17,3 +17,10 @@ def oracle():
     from oracle import kvpo
     kvpo.build()
     return kvpo
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The CUDA library is built in-tree (nvcc, sm_100a) if it is missing or older than its sources."""
+    from paper_2508_13231_b200 import build
+    build.build_library()

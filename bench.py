@@ -189,6 +189,59 @@ def run_cost_kernel(args):
                      "traffic": None, "algorithmic_bytes": alg_bytes, "peak_source": src}}))
 
 
+# Algorithmic thread instructions of the trace kernels per (unit, step): one Philox4x32-10 for the noise (10 rounds
+# of two wide multiplies, four xors and two key additions: 60 with 3-input logic ops), the 8-term Irwin-Hall sum
+# and the AR(1) update 22, a second Philox and a compare for the burst draw 62 when bursts are on, and the top-k
+# search, 32 rounds of one compare and one count per unit plus the selection compares: 68.
+def trace_alg_thread_instr(bursts):
+    return 60 + 22 + (62 if bursts else 0) + 68
+
+
+def run_trace_kernel(args):
+    """The trace kernel alone on the largest configuration: plain-ALU (issue-slot) roofline.
+
+    long_70b: 640 groups of 4096 units, 64 steps, k = 205, bursts on; the fused single-pass kernel (one CTA per
+    group). The output (S * W32 * 4 = 21 MB, plus 4 bytes per unit where a configuration has base scores) is the
+    only memory traffic, reported as GB/s beside the instruction rate.
+    """
+    import torch
+    from paper_2508_13231_b200 import kvp, workloads as wl
+    torch.cuda.set_device(0)
+    name = "long_70b"
+    cfg = wl.CONFIGS[name]
+    tp = wl.trace_params(name, seed=0)
+    U, S, W32 = wl.units(cfg), cfg["steps"], wl.words_per_row(cfg)
+    base = torch.from_numpy(tp["base"]).cuda() if tp["base"] is not None else None
+    targs = {k: v for k, v in tp.items() if k not in ("base", "seed")}
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    for w in range(max(3, args.warmup)):
+        kvp.trace_generate(**targs, seed=100 + w, base=base)
+    torch.cuda.synchronize()
+    total_ms = 0.0
+    for k in range(args.steps):
+        flush.fill_(k & 255)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        kvp.trace_generate(**targs, seed=k, base=base)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        total_ms += e0.elapsed_time(e1)
+    ms = total_ms / args.steps
+    alg = trace_alg_thread_instr(bool(tp.get("burst_thr"))) / 32.0 * U * S           # warp instructions
+    achieved = alg / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "kernel": "trace_kernel (kvp_trace_generate)", "metric": "unit_steps_per_sec", "value": U * S / (ms * 1e-3),
+        "unit": "unit-steps/s", "ms_per_call": ms, "steps": args.steps,
+        "config": {"workload": name, "groups": cfg["groups"], "units_per_group": cfg["units_per_group"], "rows": S,
+                   "topk": cfg["topk"], "l2": "flushed with a 256 MB write between timed iterations"},
+        "roofline": {"bound": "alu", "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s",
+                     "frac": achieved / ISSUE_PEAK_GWIPS, "traffic": None,
+                     "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)",
+                     "memory_gbs": (S * W32 * 4 + (U * 4 if base is not None else 0)) / (ms * 1e-3) / 1e9}}))
+
+
 def time_to_bound(kvp, cfg, targs, base_dev, U, S):
     """Outside the timed region: wall time of kvp_anneal (all of its kernels, warm) to reach the bound.
 
@@ -229,13 +282,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="kvp", choices=["kvp", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel", default="path", choices=["path", "cost"],
-                    help="path: the whole hot path (the benchmark line); cost: the cost kernel alone on full-size rows")
+    ap.add_argument("--kernel", default="path", choices=["path", "cost", "trace"],
+                    help="path: the whole hot path (the benchmark line); cost / trace: that kernel alone on full-size rows")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
     if args.kernel == "cost":
         return run_cost_kernel(args)
+    if args.kernel == "trace":
+        return run_trace_kernel(args)
 
     import numpy as np
     import torch

@@ -19,14 +19,17 @@ struct TraceK {
     int aligned;             // n % 32 == 0: whole output words belong to one group
 };
 
-__device__ __forceinline__ int64_t noise_q16(uint32_t seed_lo, uint32_t seed_hi, uint32_t u, uint32_t t)
+// Irwin-Hall(8) noise with unit variance in Q16.16: the sum of the eight 16-bit halves of one Philox block, centred
+// and scaled by floor(). |result| <= 321,057, so 32 bits hold it; only the product needs 64.
+__device__ __forceinline__ int32_t noise_q16(uint32_t seed_lo, uint32_t seed_hi, uint32_t u, uint32_t t)
 {
     uint32_t r[4];
     philox4x32_10(u, t, 0u, TAG_NOISE, seed_lo, seed_hi, r);
-    int64_t sum = 0;
+    uint32_t sum = 0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) sum += (int64_t)(r[i] & 0xFFFFu) + (int64_t)(r[i] >> 16);
-    return ((sum - 262140) * 80265) >> 16;     // Irwin-Hall(8), unit variance in Q16.16 (arithmetic shift = floor)
+    for (int i = 0; i < 4; ++i) sum = __dp2a_lo(r[i], 0x0101u, sum);      // + low half + high half
+    const int64_t scaled = (int64_t)((int32_t)sum - 262140) * 80265;
+    return (int32_t)(scaled >> 16);                                       // arithmetic shift = floor
 }
 
 // Sum of a per-thread value over the CTA; every thread gets the result. slot: one of 32 shared counters.
@@ -42,22 +45,41 @@ struct SelectSmem {
     uint32_t cnt[36];            // 32 search rounds + 2 extra counts
     uint32_t warp[32];
     uint32_t run;
+    uint32_t hi, lo;             // largest and smallest key of the step
 };
 
-// Top-k of one (group, step): the CTA holds the n keys (UPT per thread, unit i = j*T + tid) and sets the
-// bits of the k largest, ties to the lower unit index. sm.cnt must be zero on entry (and a barrier passed).
+// State of one selection; a barrier must follow before select_step.
+__device__ __forceinline__ void select_reset(SelectSmem& sm)
+{
+    for (uint32_t i = threadIdx.x; i < 36; i += blockDim.x) sm.cnt[i] = 0;
+    if (threadIdx.x == 0) { sm.hi = 0u; sm.lo = ~0u; }
+}
+
+// Top-k of one (group, step): the CTA holds the n keys (UPT per thread, unit i = j*T + tid, 0 past n) and sets the
+// bits of the k largest, ties to the lower unit index. select_reset and a barrier come first.
 template <int UPT>
 __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const TraceK& k, uint32_t gbase, uint32_t t,
                                             SelectSmem& sm)
 {
     const uint32_t T = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // The k-th largest key lies between the smallest and the largest, so it shares every bit above the highest one
+    // in which those two differ: the search starts below that bit.
+    uint32_t mx = 0u, mn = ~0u;
+#pragma unroll
+    for (int j = 0; j < UPT; ++j)
+        if (j * T + tid < k.n) { mx = max(mx, key[j]); mn = min(mn, key[j]); }
+    mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+    mn = __reduce_min_sync(0xFFFFFFFFu, mn);
+    if (lane == 0) { atomicMax(&sm.hi, mx); atomicMin(&sm.lo, mn); }
+    __syncthreads();
+    const int low_bits = 32 - __clz(sm.hi ^ sm.lo);          // 0 when all keys are equal
     // largest K with |{key >= K}| >= topk, bit by bit from the top
-    uint32_t K = 0;
-    for (int bit = 31; bit >= 0; --bit) {
+    uint32_t K = low_bits >= 32 ? 0u : sm.hi & ~((1u << low_bits) - 1u);
+    for (int bit = low_bits - 1; bit >= 0; --bit) {
         const uint32_t cand = K | (1u << bit);
         uint32_t c = 0;
 #pragma unroll
-        for (int j = 0; j < UPT; ++j) c += (j * T + tid < k.n && key[j] >= cand) ? 1u : 0u;
+        for (int j = 0; j < UPT; ++j) c += key[j] >= cand ? 1u : 0u;      // slots past n hold key 0 < cand
         if (block_sum(c, &sm.cnt[31 - bit]) >= k.topk) K = cand;
     }
     uint32_t cg = 0, ce = 0;
@@ -104,22 +126,25 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
     }
 }
 
-// importance of unit u at step t given its state at t-1 (Q16.16)
+// importance of unit u at step t given its state at t-1 (Q16.16). The 64-bit sum of the two 32x32 products is
+// shifted and then cut to 32 bits (the range check on the host keeps the true value inside them).
 __device__ __forceinline__ int32_t next_state(const TraceK& k, uint32_t u, uint32_t t, int32_t x)
 {
-    const int64_t e = noise_q16(k.seed_lo, k.seed_hi, u, t);
-    int64_t xn = t == 0 ? ((int64_t)k.sigma_q * e) >> 16 : ((int64_t)k.rho_q * (int64_t)x + (int64_t)k.c_q * e) >> 16;
+    const int32_t e = noise_q16(k.seed_lo, k.seed_hi, u, t);
+    const int64_t acc = t == 0 ? (int64_t)k.sigma_q * e : (int64_t)k.rho_q * x + (int64_t)k.c_q * e;
+    int32_t xn = (int32_t)(acc >> 16);
     if (k.burst_thr) {
         uint32_t r[4];
         philox4x32_10(u, t, 0u, TAG_BURST, k.seed_lo, k.seed_hi, r);
         if (r[0] < k.burst_thr) xn += k.burst_jump;
     }
-    return (int32_t)xn;
+    return xn;
 }
 
 // Fused form: one CTA per group walks the steps; used when the score matrix would not fit the scratch budget.
+// Two CTAs per SM (at most 32 registers per thread): one CTA's barriers in the search hide behind the other's work.
 template <int UPT>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(1024, 2)
 trace_kernel(const TraceK k)
 {
     __shared__ SelectSmem sm;
@@ -133,7 +158,7 @@ trace_kernel(const TraceK k)
         b[j] = (i < k.n && k.base) ? __ldg(k.base + gbase + i) : 0;
     }
     for (uint32_t t = 0; t < k.steps; ++t) {
-        for (uint32_t i = tid; i < 36; i += T) sm.cnt[i] = 0;
+        select_reset(sm);
         uint32_t key[UPT];
 #pragma unroll
         for (int j = 0; j < UPT; ++j) {
@@ -173,7 +198,7 @@ trace_select_kernel(const TraceK k, uint32_t U, const int32_t* __restrict__ scor
     __shared__ SelectSmem sm;
     const uint32_t g = blockIdx.x, t = blockIdx.y, T = blockDim.x, tid = threadIdx.x;
     const uint32_t gbase = g * k.n;
-    for (uint32_t i = tid; i < 36; i += T) sm.cnt[i] = 0;
+    select_reset(sm);
     uint32_t key[UPT];
 #pragma unroll
     for (int j = 0; j < UPT; ++j) {

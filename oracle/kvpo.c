@@ -16,6 +16,11 @@
  * bound, the free-migration per-step optimum, brute force over every static
  * placement and over every dynamic schedule of tiny instances, the published
  * Philox4x32-10 known-answer vectors, incremental-vs-full cost agreement.
+ * Growing cache (kvpo_set_births; tests/test_oracle_growing.py): a hand-worked
+ * instance with H^w / E^w decided by the schedule, the all-HBM and all-DRAM
+ * closed forms, the exact reduction to the fixed-population model with the
+ * written entries handed over as per-step constants, exhaustive search on
+ * tiny instances; the layered trace against the single-layer generator.
  * Parity unpinned: the synthetic trace generator beyond its structural
  * properties (exactly k bits per group and step, lag-1 autocorrelation), and
  * the quality of the annealed bound on large instances (it is only bracketed
@@ -111,6 +116,8 @@ typedef struct kvpo_problem {
     uint32_t *A;           /* [S][W32] */
     uint32_t *a;           /* [S] accessed units per step */
     uint32_t *hw, *ew;     /* [S] */
+    uint32_t *birth;       /* [U] or NULL: growing cache, see kvpo_set_births */
+    uint32_t *nb;          /* [S] units written (born) during step s */
     double spt;            /* seconds per tick */
 } kvpo_problem;
 
@@ -123,7 +130,7 @@ static void set_bit(uint32_t *row, uint32_t u, int b)
 void kvpo_destroy(kvpo_problem *p)
 {
     if (!p) return;
-    free(p->A); free(p->a); free(p->hw); free(p->ew); free(p);
+    free(p->A); free(p->a); free(p->hw); free(p->ew); free(p->birth); free(p->nb); free(p);
 }
 
 int kvpo_create(kvpo_problem **out, uint32_t units, uint64_t bytes_per_unit, uint32_t steps,
@@ -173,34 +180,81 @@ double kvpo_get_weights(const kvpo_problem *p, uint64_t out[6])
     return p->spt;
 }
 
-/* Eq. 2-4 for one step, in ticks. hr: accessed units resident in HBM,
- * mi / mo: units migrated into / out of HBM before this step. */
-static uint64_t step_cost(const kvpo_problem *p, uint32_t s, uint64_t hr, uint64_t mi, uint64_t mo)
+/*
+ * Growing cache (Section III-A lists the newly written entries H^w and E^w among
+ * the scheduling decisions). birth[u] = 0: unit u exists before the first step
+ * (written by the prefill, outside the model). birth[u] = b >= 1: unit u is
+ * written during step b; before b it is nowhere, so its placement bits of
+ * earlier steps are ignored and it may not be accessed there. At step b the
+ * placement bit decides where the new entry goes: set = written to HBM (it
+ * counts in |H^w_b|), clear = written to off-package DRAM (|E^w_b|). Being
+ * written is not a migration. The caller's hw/ew constants still add.
+ */
+int kvpo_set_births(kvpo_problem *p, const uint32_t *birth)
 {
+    if (!p || !birth || p->birth) return KVPO_ERR_ARG;
+    uint32_t *b = (uint32_t *)malloc((size_t)p->U * 4);
+    uint32_t *nb = (uint32_t *)calloc(p->S, 4);
+    if (!b || !nb) { free(b); free(nb); return KVPO_ERR_NOMEM; }
+    for (uint32_t u = 0; u < p->U; ++u) {
+        if (birth[u] >= p->S) { free(b); free(nb); return KVPO_ERR_ARG; }
+        b[u] = birth[u];
+        if (birth[u]) ++nb[birth[u]];
+        for (uint32_t s = 0; s < birth[u]; ++s)
+            if (bit_of(p->A + (size_t)s * p->W32, u)) { free(b); free(nb); return KVPO_ERR_ARG; }
+    }
+    uint64_t mx = 0;
+    for (uint32_t s = 0; s < p->S; ++s) {
+        uint64_t e = (uint64_t)p->hw[s] + p->ew[s] + nb[s];
+        if (e > mx) mx = e;
+    }
+    uint64_t kmax = p->kh > p->ke ? p->kh : p->ke;
+    if (kmax * (2ull * p->U + mx) >= (1ull << 31)) { free(b); free(nb); return KVPO_ERR_RANGE; }
+    p->birth = b; p->nb = nb;
+    return KVPO_OK;
+}
+
+static int alive(const kvpo_problem *p, uint32_t u, uint32_t s) { return !p->birth || p->birth[u] <= s; }
+static int born_at(const kvpo_problem *p, uint32_t u, uint32_t s) { return p->birth && s > 0 && p->birth[u] == s; }
+
+/* Eq. 2-4 for one step, in ticks. hr: accessed units resident in HBM,
+ * mi / mo: units migrated into / out of HBM before this step, hb: units
+ * written to HBM at birth during this step (0 without kvpo_set_births). */
+static uint64_t step_cost(const kvpo_problem *p, uint32_t s, uint64_t hr, uint64_t mi, uint64_t mo, uint64_t hb)
+{
+    uint64_t hw = p->hw[s] + hb;                                             /* |H^w| */
+    uint64_t ew = p->ew[s] + (p->nb ? p->nb[s] - hb : 0);                    /* |E^w| */
     uint64_t er = (uint64_t)p->a[s] - hr;                                    /* |E^r| */
-    uint64_t th = p->kh * (hr + p->hw[s] + p->fh * (mi + mo));               /* Eq. 3 */
-    uint64_t w1 = p->kk * (p->ew[s] + p->fe * mo);                           /* link, outbound  */
+    uint64_t th = p->kh * (hr + hw + p->fh * (mi + mo));                     /* Eq. 3 */
+    uint64_t w1 = p->kk * (ew + p->fe * mo);                                 /* link, outbound  */
     uint64_t w2 = p->kk * (p->fe * mi);                                      /* link, inbound   */
-    uint64_t w3 = p->kd * (p->ew[s] + p->fe * (mi + mo));                    /* DRAM channels   */
+    uint64_t w3 = p->kd * (ew + p->fe * (mi + mo));                          /* DRAM channels   */
     uint64_t wm = w1 > w2 ? w1 : w2;
     if (w3 > wm) wm = w3;
     uint64_t te = p->ke * er + wm;                                           /* Eq. 4 */
     return th > te ? th : te;                                                /* Eq. 2 */
 }
 
-/* The four cardinalities of step s of schedule P (rows of W32 words). */
-static void step_counts(const kvpo_problem *p, const uint32_t *P, uint32_t s, uint32_t c[4])
+/* The cardinalities of step s of schedule P (rows of W32 words): hr, mi, mo, occ and, for a growing cache, hb.
+ * A unit that does not exist yet counts as absent whatever its bit says. */
+static void step_counts(const kvpo_problem *p, const uint32_t *P, uint32_t s, uint32_t c[5])
 {
     const uint32_t *row = P + (size_t)s * p->W32;
     const uint32_t *prev = s ? row - p->W32 : row;                           /* P[-1] := P[0] */
     const uint32_t *acc = p->A + (size_t)s * p->W32;
-    c[0] = c[1] = c[2] = c[3] = 0;
+    c[0] = c[1] = c[2] = c[3] = c[4] = 0;
     for (uint32_t u = 0; u < p->U; ++u) {
-        int pb = bit_of(row, u), qb = bit_of(prev, u), ab = bit_of(acc, u);
-        c[0] += (uint32_t)(pb & ab);          /* hr  */
-        c[1] += (uint32_t)(pb & (1 - qb));         /* mi  */
-        c[2] += (uint32_t)((1 - pb) & qb);         /* mo  */
-        c[3] += (uint32_t)pb;                 /* occ */
+        int pb = bit_of(row, u) & alive(p, u, s);
+        int qb = s ? (bit_of(prev, u) & alive(p, u, s - 1)) : pb;
+        int ab = bit_of(acc, u);
+        c[0] += (uint32_t)(pb & ab);               /* hr  */
+        c[3] += (uint32_t)pb;                      /* occ */
+        if (born_at(p, u, s)) {
+            c[4] += (uint32_t)pb;                  /* hb: written to HBM, not migrated */
+        } else {
+            c[1] += (uint32_t)(pb & (1 - qb));     /* mi  */
+            c[2] += (uint32_t)((1 - pb) & qb);     /* mo  */
+        }
     }
 }
 
@@ -216,13 +270,13 @@ int kvpo_eval(const kvpo_problem *p, const uint32_t *P, uint64_t *step_ticks, ui
     uint64_t T = 0;
     int32_t bad = -1;
     for (uint32_t s = 0; s < p->S; ++s) {
-        uint32_t c[4];
+        uint32_t c[5];
         step_counts(p, P, s, c);
-        uint64_t f = step_cost(p, s, c[0], c[1], c[2]);
+        uint64_t f = step_cost(p, s, c[0], c[1], c[2], c[4]);
         if (c[3] > p->cap && bad < 0) bad = (int32_t)s;                      /* Eq. 5 */
         if (step_ticks) step_ticks[s] = f;
         if (step_seconds) step_seconds[s] = (double)f * p->spt;
-        if (counts) memcpy(counts + 4 * (size_t)s, c, sizeof c);
+        if (counts) memcpy(counts + 4 * (size_t)s, c, 4 * sizeof c[0]);
         T += f;                                                              /* Eq. 1 */
     }
     if (total_ticks) *total_ticks = T;
@@ -231,10 +285,23 @@ int kvpo_eval(const kvpo_problem *p, const uint32_t *P, uint64_t *step_ticks, ui
     return KVPO_OK;
 }
 
+/* hb [S]: units written to HBM at birth in every step (all 0 for a fixed population). */
+int kvpo_eval_hb(const kvpo_problem *p, const uint32_t *P, uint32_t *hb)
+{
+    if (!p || !P || !hb) return KVPO_ERR_ARG;
+    for (uint32_t s = 0; s < p->S; ++s) {
+        uint32_t c[5];
+        step_counts(p, P, s, c);
+        hb[s] = c[4];
+    }
+    return KVPO_OK;
+}
+
 /* ------------------------------------------------------------------ */
 /* Initial placements. mode 0: units 0..cap-1 (Static Placement: fill HBM in
  * arrival order, never migrate). mode 1: the cap most accessed units, ties to
- * the lower index. The same row is used at every step. */
+ * the lower index. The same row is used at every step; in a growing cache a
+ * unit of the row enters HBM when it is written. */
 int kvpo_init_placement(const kvpo_problem *p, uint32_t mode, uint32_t *P)
 {
     if (!p || !P || mode > 1) return KVPO_ERR_ARG;
@@ -257,7 +324,11 @@ int kvpo_init_placement(const kvpo_problem *p, uint32_t mode, uint32_t *P)
                 if (cnt[u] == (uint32_t)c) { set_bit(row, u, 1); ++placed; }
         free(cnt);
     }
-    for (uint32_t s = 0; s < p->S; ++s) memcpy(P + (size_t)s * p->W32, row, (size_t)p->W32 * 4);
+    for (uint32_t s = 0; s < p->S; ++s) {
+        memset(P + (size_t)s * p->W32, 0, (size_t)p->W32 * 4);
+        for (uint32_t u = 0; u < p->U; ++u)
+            set_bit(P + (size_t)s * p->W32, u, bit_of(row, u) & alive(p, u, s));
+    }
     free(row);
     return KVPO_OK;
 }
@@ -326,16 +397,18 @@ static move_t decode_move(const kvpo_problem *p, const kvpo_anneal_params *ap,
 }
 
 typedef struct {
-    uint32_t *P;                    /* [S][W32] current schedule */
+    uint32_t *P;                    /* [S][W32] current schedule (bits of unborn units stay clear) */
     uint32_t *hr, *mi, *mo, *occ;   /* [S] */
+    uint32_t *hb;                   /* [S] units written to HBM at birth */
     uint64_t cur;
 } chain_state;
 
-/* Placement bit unit x would have at step t if the move were applied. */
+/* Placement bit unit x would have at step t if the move were applied. A move
+ * acts on a step only if the units it names exist there. */
 static int proposed_bit(const kvpo_problem *p, const chain_state *st, const move_t *mv, uint32_t t, uint32_t x)
 {
     const uint32_t *row = st->P + (size_t)t * p->W32;
-    int in_range = t >= mv->s0 && t < mv->s0 + mv->len;
+    int in_range = t >= mv->s0 && t < mv->s0 + mv->len && alive(p, mv->u, t) && (!mv->swap || alive(p, mv->v, t));
     if (!in_range) return bit_of(row, x);
     if (!mv->swap) return x == mv->u ? !bit_of(row, x) : bit_of(row, x);
     if (x == mv->u) return bit_of(row, mv->v);
@@ -346,13 +419,13 @@ static int proposed_bit(const kvpo_problem *p, const chain_state *st, const move
 /*
  * Evaluate a proposal against the current state without applying it.
  * Returns 0 = evaluated, 1 = infeasible (a flip would exceed capacity).
- * d[t - s0][0..3] receive the changes of hr, mi, mo, occ of every affected
+ * d[t - s0][0..4] receive the changes of hr, mi, mo, occ, hb of every affected
  * step t = s0 .. last, where last = min(s0 + len, S - 1): the step after the
  * run is affected too because its migration counts compare against the run's
  * last row.
  */
 static int evaluate_move(const kvpo_problem *p, const chain_state *st, const move_t *mv,
-                         int64_t *delta, int32_t d[32][4], uint32_t *last_out, int *changed)
+                         int64_t *delta, int32_t d[32][5], uint32_t *last_out, int *changed)
 {
     uint32_t last = mv->s0 + mv->len;
     if (last > p->S - 1) last = p->S - 1;
@@ -363,7 +436,7 @@ static int evaluate_move(const kvpo_problem *p, const chain_state *st, const mov
     int64_t dsum = 0;
     for (uint32_t t = mv->s0; t <= last; ++t) {
         int32_t *dt = d[t - mv->s0];
-        dt[0] = dt[1] = dt[2] = dt[3] = 0;
+        dt[0] = dt[1] = dt[2] = dt[3] = dt[4] = 0;
         for (int i = 0; i < nx; ++i) {
             uint32_t x = xs[i];
             int po = bit_of(st->P + (size_t)t * p->W32, x);
@@ -372,16 +445,21 @@ static int evaluate_move(const kvpo_problem *p, const chain_state *st, const mov
             int qn = t ? proposed_bit(p, st, mv, t - 1, x) : pn;
             int ab = bit_of(p->A + (size_t)t * p->W32, x);
             dt[0] += ab * (pn - po);
-            dt[1] += (pn & (1 - qn)) - (po & (1 - qo));
-            dt[2] += ((1 - pn) & qn) - ((1 - po) & qo);
             dt[3] += pn - po;
+            if (born_at(p, x, t)) {
+                dt[4] += pn - po;                     /* written to HBM instead of DRAM, or back */
+            } else {
+                dt[1] += (pn & (1 - qn)) - (po & (1 - qo));
+                dt[2] += ((1 - pn) & qn) - ((1 - po) & qo);
+            }
             if (pn != po) *changed = 1;
         }
         if (!mv->swap && (int64_t)st->occ[t] + dt[3] > (int64_t)p->cap && dt[3] > 0) return 1;
-        uint64_t f_old = step_cost(p, t, st->hr[t], st->mi[t], st->mo[t]);
+        uint64_t f_old = step_cost(p, t, st->hr[t], st->mi[t], st->mo[t], st->hb[t]);
         uint64_t f_new = step_cost(p, t, (uint64_t)((int64_t)st->hr[t] + dt[0]),
                                    (uint64_t)((int64_t)st->mi[t] + dt[1]),
-                                   (uint64_t)((int64_t)st->mo[t] + dt[2]));
+                                   (uint64_t)((int64_t)st->mo[t] + dt[2]),
+                                   (uint64_t)((int64_t)st->hb[t] + dt[4]));
         dsum += (int64_t)f_new - (int64_t)f_old;
     }
     *delta = dsum;
@@ -389,17 +467,14 @@ static int evaluate_move(const kvpo_problem *p, const chain_state *st, const mov
 }
 
 static void apply_move(const kvpo_problem *p, chain_state *st, const move_t *mv,
-                       int32_t d[32][4], uint32_t last, int64_t delta)
+                       int32_t d[32][5], uint32_t last, int64_t delta)
 {
     for (uint32_t t = mv->s0; t < mv->s0 + mv->len && t < p->S; ++t) {
         uint32_t *row = st->P + (size_t)t * p->W32;
-        if (mv->swap) {
-            int bu = bit_of(row, mv->u), bv = bit_of(row, mv->v);
-            set_bit(row, mv->u, bv);
-            set_bit(row, mv->v, bu);
-        } else {
-            set_bit(row, mv->u, !bit_of(row, mv->u));
-        }
+        int bu = proposed_bit(p, st, mv, t, mv->u);
+        int bv = mv->swap ? proposed_bit(p, st, mv, t, mv->v) : 0;
+        set_bit(row, mv->u, bu);
+        if (mv->swap) set_bit(row, mv->v, bv);
     }
     for (uint32_t t = mv->s0; t <= last; ++t) {
         int32_t *dt = d[t - mv->s0];
@@ -407,6 +482,7 @@ static void apply_move(const kvpo_problem *p, chain_state *st, const move_t *mv,
         st->mi[t] = (uint32_t)((int32_t)st->mi[t] + dt[1]);
         st->mo[t] = (uint32_t)((int32_t)st->mo[t] + dt[2]);
         st->occ[t] = (uint32_t)((int32_t)st->occ[t] + dt[3]);
+        st->hb[t] = (uint32_t)((int32_t)st->hb[t] + dt[4]);
     }
     st->cur = (uint64_t)((int64_t)st->cur + delta);
 }
@@ -419,22 +495,23 @@ static int state_init(const kvpo_problem *p, chain_state *st, const uint32_t *P0
     st->mi = (uint32_t *)malloc((size_t)p->S * 4);
     st->mo = (uint32_t *)malloc((size_t)p->S * 4);
     st->occ = (uint32_t *)malloc((size_t)p->S * 4);
-    if (!st->P || !st->hr || !st->mi || !st->mo || !st->occ) return KVPO_ERR_NOMEM;
+    st->hb = (uint32_t *)malloc((size_t)p->S * 4);
+    if (!st->P || !st->hr || !st->mi || !st->mo || !st->occ || !st->hb) return KVPO_ERR_NOMEM;
     memcpy(st->P, P0, nw * 4);
     st->cur = 0;
     for (uint32_t s = 0; s < p->S; ++s) {
-        uint32_t c[4];
+        uint32_t c[5];
         step_counts(p, st->P, s, c);
-        st->hr[s] = c[0]; st->mi[s] = c[1]; st->mo[s] = c[2]; st->occ[s] = c[3];
+        st->hr[s] = c[0]; st->mi[s] = c[1]; st->mo[s] = c[2]; st->occ[s] = c[3]; st->hb[s] = c[4];
         if (c[3] > p->cap) return KVPO_ERR_CAPACITY;
-        st->cur += step_cost(p, s, c[0], c[1], c[2]);
+        st->cur += step_cost(p, s, c[0], c[1], c[2], c[4]);
     }
     return KVPO_OK;
 }
 
 static void state_free(chain_state *st)
 {
-    free(st->P); free(st->hr); free(st->mi); free(st->mo); free(st->occ);
+    free(st->P); free(st->hr); free(st->mi); free(st->mo); free(st->occ); free(st->hb);
 }
 
 /* Resolve the initial schedule named by the parameters into P0 [S][W32]. */
@@ -445,7 +522,7 @@ static int resolve_init(const kvpo_problem *p, const kvpo_anneal_params *ap, uin
         memset(P0, 0, (size_t)p->S * p->W32 * 4);
         for (uint32_t s = 0; s < p->S; ++s)
             for (uint32_t u = 0; u < p->U; ++u)
-                set_bit(P0 + (size_t)s * p->W32, u, bit_of(ap->init_schedule + (size_t)s * p->W32, u));
+                set_bit(P0 + (size_t)s * p->W32, u, bit_of(ap->init_schedule + (size_t)s * p->W32, u) & alive(p, u, s));
         return KVPO_OK;
     }
     return kvpo_init_placement(p, ap->init_mode, P0);
@@ -472,7 +549,7 @@ int kvpo_default_temps(const kvpo_problem *p, const kvpo_anneal_params *ap, doub
     uint64_t sum = 0, cnt = 0;
     for (uint32_t i = 0; i < CALIB_N; ++i) {
         move_t mv = decode_move(p, ap, i, 0, TAG_CALIB);
-        int64_t delta; int32_t d[32][4]; uint32_t last; int changed;
+        int64_t delta; int32_t d[32][5]; uint32_t last; int changed;
         if (evaluate_move(p, &st, &mv, &delta, d, &last, &changed)) continue;
         if (delta > 0) { sum += (uint64_t)delta; ++cnt; }
     }
@@ -533,7 +610,7 @@ int kvpo_anneal_chains(const kvpo_problem *p, const kvpo_anneal_params *ap,
                 best_at_boundary = r.best_ticks;
             }
             move_t mv = decode_move(p, ap, m, chain, TAG_MOVE);
-            int64_t delta; int32_t d[32][4]; uint32_t last; int changed;
+            int64_t delta; int32_t d[32][5]; uint32_t last; int changed;
             if (evaluate_move(p, &st, &mv, &delta, d, &last, &changed)) { ++r.n_infeasible; continue; }
             int accept;
             if (delta <= 0) accept = 1;                                 /* downhill or level: always */
@@ -612,6 +689,8 @@ typedef struct {
     int32_t rho_q, c_q, sigma_q, burst_jump;
     uint32_t burst_thr, reserved;
     const int32_t *base;
+    uint32_t layers, reserved2;   /* 0 or 1: every group reads at every step */
+    const uint32_t *birth;        /* [U] or NULL: step from which a unit can be read */
 } kvpo_trace_params;
 
 static int64_t floor_shift16(int64_t v)
@@ -626,6 +705,13 @@ static int64_t floor_shift16(int64_t v)
  * Groups group_begin .. group_begin+group_count-1 only (groups are independent);
  * bits of other groups are left 0. scores_out: [steps][U] int32 or NULL (for
  * statistical tests; only the selected groups are written).
+ *
+ * layers = L > 1: the steps are the (token n, layer l) pairs of Section III-A in
+ * the order s = n * L + l. The groups are split into L consecutive blocks, one
+ * per layer; a group reads only at the steps of its layer, and the importance
+ * of its units advances once per token (the noise counter is (u, n)). With
+ * birth given, a group reads its min(topk, existing) most important existing
+ * units (birth[u] <= s).
  */
 int kvpo_trace_generate(const kvpo_trace_params *tp, uint32_t group_begin, uint32_t group_count,
                         uint32_t *access, int32_t *scores_out)
@@ -633,6 +719,7 @@ int kvpo_trace_generate(const kvpo_trace_params *tp, uint32_t group_begin, uint3
     if (!tp || !access || !tp->groups || !tp->units_per_group || !tp->steps) return KVPO_ERR_ARG;
     if (!tp->topk || tp->topk > tp->units_per_group) return KVPO_ERR_ARG;
     if (group_begin > tp->groups || group_count > tp->groups - group_begin) return KVPO_ERR_ARG;
+    if (tp->layers > 1 && tp->groups % tp->layers) return KVPO_ERR_ARG;
     if (tp->rho_q < 0 || tp->rho_q > 65536 || tp->c_q < 0 || tp->c_q > (1 << 20) ||
         tp->sigma_q < 0 || tp->sigma_q > (1 << 20)) return KVPO_ERR_ARG;
     uint64_t U64 = (uint64_t)tp->groups * tp->units_per_group;
@@ -657,29 +744,37 @@ int kvpo_trace_generate(const kvpo_trace_params *tp, uint32_t group_begin, uint3
     uint8_t *picked = (uint8_t *)calloc(n, 1);
     if (!x || !score || !picked) { free(x); free(score); free(picked); return KVPO_ERR_NOMEM; }
     memset(access, 0, (size_t)tp->steps * W32 * 4);
+    uint32_t L = tp->layers ? tp->layers : 1;
+    uint32_t per_layer = tp->groups / L;
     for (uint32_t t = 0; t < tp->steps; ++t) {
-        for (uint32_t u = group_begin * n; u < (group_begin + group_count) * n; ++u) {
-            uint32_t r[4];
-            philox(tp->seed, u, t, 0, TAG_NOISE, r);
-            int64_t sum = 0;
-            for (int i = 0; i < 4; ++i) sum += (int64_t)(r[i] & 0xFFFFu) + (int64_t)(r[i] >> 16);
-            int64_t e = floor_shift16((sum - 262140) * 80265);
-            if (t == 0) x[u] = floor_shift16((int64_t)tp->sigma_q * e);
-            else x[u] = floor_shift16((int64_t)tp->rho_q * x[u] + (int64_t)tp->c_q * e);
-            if (tp->burst_thr) {
-                philox(tp->seed, u, t, 0, TAG_BURST, r);
-                if (r[0] < tp->burst_thr) x[u] += tp->burst_jump;
-            }
-        }
+        uint32_t tok = t / L, layer = t % L;
         for (uint32_t g = group_begin; g < group_begin + group_count; ++g) {
+            if (g / per_layer != layer) continue;
+            for (uint32_t i = 0; i < n; ++i) {
+                uint32_t u = g * n + i;
+                uint32_t r[4];
+                philox(tp->seed, u, tok, 0, TAG_NOISE, r);
+                int64_t sum = 0;
+                for (int k = 0; k < 4; ++k) sum += (int64_t)(r[k] & 0xFFFFu) + (int64_t)(r[k] >> 16);
+                int64_t e = floor_shift16((sum - 262140) * 80265);
+                if (tok == 0) x[u] = floor_shift16((int64_t)tp->sigma_q * e);
+                else x[u] = floor_shift16((int64_t)tp->rho_q * x[u] + (int64_t)tp->c_q * e);
+                if (tp->burst_thr) {
+                    philox(tp->seed, u, tok, 0, TAG_BURST, r);
+                    if (r[0] < tp->burst_thr) x[u] += tp->burst_jump;
+                }
+            }
+            uint32_t existing = 0;
             for (uint32_t i = 0; i < n; ++i) {
                 uint32_t u = g * n + i;
                 score[i] = x[u] + (tp->base ? tp->base[u] : 0);
-                picked[i] = 0;
+                picked[i] = (uint8_t)(tp->birth && tp->birth[u] > t);    /* not there yet: never chosen */
+                existing += !picked[i];
                 if (scores_out) scores_out[(size_t)t * U + u] = (int32_t)score[i];
             }
             /* k rounds of "largest remaining score, lowest index among equals" */
-            for (uint32_t r = 0; r < tp->topk; ++r) {
+            uint32_t k = tp->topk < existing ? tp->topk : existing;
+            for (uint32_t r = 0; r < k; ++r) {
                 uint32_t arg = n;
                 for (uint32_t i = 0; i < n; ++i)
                     if (!picked[i] && (arg == n || score[i] > score[arg])) arg = i;
@@ -725,6 +820,7 @@ static int by_freq_asc(const void *a, const void *b)
  */
 int kvpo_policy_lookahead(const kvpo_problem *p, uint32_t init_mode, uint32_t W, uint32_t ratio_permille, uint32_t *P)
 {
+    if (p && p->birth) return KVPO_ERR_ARG;       /* the policies are defined on a fixed population */
     if (!p || !P || init_mode > 1 || W < 1 || W > 64 || ratio_permille > 1000) return KVPO_ERR_ARG;
     int rc = kvpo_init_placement(p, init_mode, P);
     if (rc) return rc;
@@ -766,6 +862,7 @@ int kvpo_policy_lookahead(const kvpo_problem *p, uint32_t init_mode, uint32_t W,
  */
 int kvpo_policy_reactive(const kvpo_problem *p, uint32_t init_mode, uint32_t *P)
 {
+    if (p && p->birth) return KVPO_ERR_ARG;       /* the policies are defined on a fixed population */
     if (!p || !P || init_mode > 1) return KVPO_ERR_ARG;
     int rc = kvpo_init_placement(p, init_mode, P);
     if (rc) return rc;
@@ -909,6 +1006,7 @@ int kvpo_wr_anneal(const uint64_t *table, uint32_t w_max, uint32_t n_ratio, cons
  */
 int kvpo_policy_page(const kvpo_problem *p, uint32_t page_units, uint32_t *P)
 {
+    if (p && p->birth) return KVPO_ERR_ARG;       /* the policies are defined on a fixed population */
     if (!p || !P || !page_units || page_units > 32 || (page_units & (page_units - 1)) || p->U % page_units)
         return KVPO_ERR_ARG;
     const uint32_t np = p->U / page_units, cap_pages = p->cap / page_units;

@@ -61,6 +61,8 @@ class TraceParams(C.Structure):
         ("rho_q", C.c_int32), ("c_q", C.c_int32), ("sigma_q", C.c_int32), ("burst_jump", C.c_int32),
         ("burst_thr", C.c_uint32), ("reserved", C.c_uint32),
         ("base", C.POINTER(C.c_int32)),
+        ("layers", C.c_uint32), ("reserved2", C.c_uint32),
+        ("birth", C.POINTER(C.c_uint32)),
     ]
 
 
@@ -103,7 +105,7 @@ def tick_weights(bw_hbm, bw_link, bw_dram):
 
 class Problem:
     def __init__(self, units, bytes_per_unit, steps, access, cap, bw_hbm, bw_link, bw_dram,
-                 mig_flags=MIG_PAPER, hw=None, ew=None):
+                 mig_flags=MIG_PAPER, hw=None, ew=None, birth=None):
         access = np.ascontiguousarray(access, dtype=np.uint32)
         self.units, self.steps, self.cap = int(units), int(steps), int(cap)
         self.w32 = (self.units + 31) // 32
@@ -119,6 +121,11 @@ class Problem:
         o = (C.c_uint64 * 6)()
         self.seconds_per_tick = float(lib().kvpo_get_weights(self._h, o))
         self.weights = dict(zip(("kh", "kk", "kd", "ke", "lcm", "gcd"), (int(x) for x in o)))
+        self.birth = None
+        if birth is not None:
+            self.birth = np.ascontiguousarray(birth, dtype=np.uint32)
+            assert self.birth.size == self.units
+            _chk(lib().kvpo_set_births(self._h, _u32p(self.birth)), "set_births")
 
     def __del__(self):
         if getattr(self, "_h", None) is not None and self._h:
@@ -139,8 +146,10 @@ class Problem:
         tt = C.c_uint64(); ts = C.c_double(); bad = C.c_int32()
         _chk(lib().kvpo_eval(self._h, _u32p(P), _u64p(st), C.byref(tt), ss.ctypes.data_as(C.POINTER(C.c_double)),
                              C.byref(ts), C.byref(bad), _u32p(cnt)), "eval")
+        hb = np.zeros(self.steps, np.uint32)
+        _chk(lib().kvpo_eval_hb(self._h, _u32p(P), _u32p(hb)), "eval_hb")
         return dict(step_ticks=st, total_ticks=int(tt.value), step_seconds=ss, total_seconds=float(ts.value),
-                    bad_step=int(bad.value), counts=cnt)
+                    bad_step=int(bad.value), counts=cnt, hb=hb)
 
     def init_placement(self, mode):
         P = np.zeros((self.steps, self.w32), np.uint32)
@@ -222,9 +231,14 @@ def accept_table(temps):
 
 
 def trace_generate(groups, units_per_group, steps, topk, seed, rho_q, c_q, sigma_q, burst_jump=0, burst_thr=0,
-                   base=None, group_begin=0, group_count=None, want_scores=False):
+                   base=None, group_begin=0, group_count=None, want_scores=False, layers=0, birth=None):
     """-> access [steps][W32] (and scores [steps][U] int32 when want_scores)."""
     tp = TraceParams()
+    tp.layers = layers
+    if birth is not None:
+        birth = np.ascontiguousarray(birth, dtype=np.uint32)
+        assert birth.size == groups * units_per_group
+        tp.birth = birth.ctypes.data_as(C.POINTER(C.c_uint32))
     tp.groups, tp.units_per_group, tp.steps, tp.topk, tp.seed = groups, units_per_group, steps, topk, seed
     tp.rho_q, tp.c_q, tp.sigma_q, tp.burst_jump, tp.burst_thr = rho_q, c_q, sigma_q, burst_jump, burst_thr
     if base is not None:

@@ -157,6 +157,27 @@ int kvp_eval_noalloc(kvp_problem* p, const uint32_t* schedules, uint32_t n,
                      uint64_t* step_ticks, uint64_t* total_ticks,
                      double* step_seconds, double* total_seconds, int32_t* bad_step, void* stream);
 
+/*
+ * kvp_set_births -- make the problem a growing cache: the newly written entries H^w and E^w of the scheduling
+ * decision S_(n,l) (Section III-A) become part of the schedule.
+ *   birth (device) [units] uint32: 0 = the unit exists before the first step (written by the prefill, outside the
+ *   model); b >= 1 = the unit is written during step b, b < steps.
+ * Meaning for every later call on `p`:
+ *   - before step birth[u] the unit is nowhere: its placement bits there are ignored (by kvp_eval) and never set
+ *     (by kvp_anneal, whose moves act only on the steps at which the units they name exist), it does not count
+ *     towards Eq. 5, and it must not be accessed (KVP_ERR_ARG otherwise);
+ *   - at step b the placement bit decides where the new entry is written: set = HBM, it adds to |H^w_b| of
+ *     Eq. 3; clear = off-package DRAM, it adds to |E^w_b| of Eq. 4. Being written is not a migration;
+ *   - hw_units / ew_units of kvp_create still add to both sets;
+ *   - the static initial placements hold a unit of their row from the step it is written.
+ * Call it once, directly after kvp_create. Supported afterwards: kvp_eval, kvp_anneal, kvp_anneal_chain_state,
+ * kvp_get_info. kvp_eval_counts, kvp_eval_noalloc, the policies and kvp_wr_grid are defined for fixed populations
+ * and return KVP_ERR_ARG. Copies `birth`; synchronises `stream`. Errors: KVP_ERR_ARG (null, called twice, a birth
+ * >= steps, an access before birth), KVP_ERR_RANGE (the tick range check of kvp_create with the births added to
+ * the written units), KVP_ERR_NOMEM, KVP_ERR_CUDA; on error the problem is unchanged.
+ */
+int kvp_set_births(kvp_problem* p, const uint32_t* birth, void* stream);
+
 /* Initial placement of a chain. */
 #define KVP_INIT_STATIC_FIRST 0u /* units 0..cap-1 at every step: the Static Placement baseline (Section IV-A) */
 #define KVP_INIT_STATIC_FREQ  1u /* the cap units with most accesses over all steps (ties: lower index)     */
@@ -264,6 +285,13 @@ int kvp_anneal_chain_state(kvp_problem* p, const kvp_anneal_params* params, uint
  * halves of Philox4x32-10(counter = (u, t, 0, 3), key = seed):
  *   e = ((sum of halves - 262140) * 80265) >> 16.
  * Ties are broken towards the lower unit index.
+ *
+ * layers = L > 1: the steps are the (token n, layer l) pairs of Section III-A in the order s = n*L + l. The groups
+ * are split into L consecutive blocks of groups/L, one per layer; a group reads only at the steps of its layer
+ * (its bits are 0 elsewhere) and the importance of its units advances once per token: the noise counter is
+ * (u, n, 0, 3) and x_n follows x_{n-1}. groups must be a multiple of L.
+ * birth != NULL (growing cache, see kvp_set_births): at step s a group reads its min(topk, existing) most
+ * important existing units, a unit existing from step birth[u] on.
  */
 typedef struct {
     uint32_t groups, units_per_group, steps, topk;
@@ -276,6 +304,9 @@ typedef struct {
     uint32_t flags;       /* KVP_TRACE_*                                             */
     const int32_t* base;  /* (device) [groups*units_per_group] static log-importance, or NULL = 0;
                              |base| <= 2^29                                          */
+    uint32_t layers;      /* 0 or 1: every group reads at every step                 */
+    uint32_t reserved;    /* must be 0                                               */
+    const uint32_t* birth;/* (device) [groups*units_per_group] or NULL               */
 } kvp_trace_params;
 
 #define KVP_TRACE_SINGLE_PASS 1u /* never allocate the [steps][units] int32 score matrix (the default does for traces

@@ -35,6 +35,8 @@ struct ChainParams {
     uint64_t* undo_log;          // if set: [slots][undo_cap] indices of the moves applied since the best state
     uint32_t* undo_len;          // [slots] how many there were (more than undo_cap: the log overflowed)
     uint32_t undo_cap;
+    const uint32_t* birth;       // growing cache: [U] step at which a unit is written (0 = there from the start)
+    const uint32_t* hb0;         // growing cache: [S] units written to HBM at birth under the initial schedule
     CostK K;
     uint32_t U, S, S32, cap;
     uint32_t chain_first, chain_count, result_base;
@@ -97,16 +99,30 @@ struct ChainView {               // where a chain's state lives
     uint4* win;                  // [kBatch][2] windows of the batch's proposals (shared)
     int* acc;                    // [kBatch] cost change of each proposal being summed (shared)
     uint16_t* queue;             // [kBatch * 31] work items (proposal slot << 5 | window bit) (shared)
+    uint32_t* hb;                // growing cache: [S] units written to HBM at birth (shared)
 };
 
-struct Windows { uint32_t Wu, Wv, Nu, Nv, Au, Av, s0; };
+// born: window bit of the step in which u (low byte) and v (next byte) are written, 0 = not among bits 1..31
+struct Windows { uint32_t Wu, Wv, Nu, Nv, Au, Av, s0, born; };
+
+// Growing cache, unit with birth step b seen through the window that starts at step s0 - 1 (-1 for s0 == 0):
+// the bits of steps at which it exists, and the bit of the step in which it is written.
+__device__ __forceinline__ void alive_born(uint32_t b, uint32_t s0, uint32_t& alive, uint32_t& born)
+{
+    const int off = (int)b - ((int)s0 - 1);
+    alive = (b == 0 || off <= 0) ? 0xFFFFFFFFu : (off >= 32 ? 0u : 0xFFFFFFFFu << off);
+    born = (b != 0 && off >= 1 && off < 32) ? 1u << off : 0u;
+}
 
 // First half of evaluating a proposal, all in the calling lane and word-parallel over the <= 31 affected
 // steps: the windows before and after the move, feasibility (Eq. 5), whether any bit changes, and the set
 // of window bits (steps) whose cardinalities, hence cost, change.
-template <typename PPtr, typename FPtr>
-__device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restrict__ Acol, FPtr full, uint32_t S,
-                                                 uint32_t S32, LaneMove& mv, Windows& wn)
+// GROW: a move acts only on the steps at which the units it names exist, and a unit that enters HBM in the step
+// it is written was written there (it counts in hb), not migrated.
+template <bool GROW, typename PPtr, typename FPtr>
+__device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restrict__ Acol, FPtr full,
+                                                 const uint32_t* __restrict__ birth, uint32_t S, uint32_t S32,
+                                                 LaneMove& mv, Windows& wn)
 {
     const bool swap = mv.pk & 1u;
     const uint32_t len = (mv.pk >> 1) & 63u, s0 = mv.pk >> 8;
@@ -120,30 +136,53 @@ __device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restr
     const uint32_t wv = window(P + vb, S32, s0), av = window(Acol + vb, S32, s0);
     const uint32_t Wv = swap ? wv : 0u, Av = swap ? av : 0u;
     const uint32_t Fw = window(full, S32, s0);
-    const uint32_t D = swap ? ((Wu ^ Wv) & M) : M;                // bits that toggle
+    uint32_t Bu = 0u, Bv = 0u, live = 0xFFFFFFFFu;
+    if (GROW) {
+        uint32_t Lu, Lv;
+        alive_born(__ldg(birth + mv.u), s0, Lu, Bu);
+        alive_born(__ldg(birth + (swap ? mv.v : mv.u)), s0, Lv, Bv);
+        live = Lu & Lv;
+        if (!swap) Bv = 0u;
+    }
+    const uint32_t D = (swap ? (Wu ^ Wv) : 0xFFFFFFFFu) & M & live;      // bits that toggle
     uint32_t Nu = Wu ^ D, Nv = swap ? (Wv ^ D) : 0u;
     if (s0 == 0) {                                                // the virtual step -1 follows step 0
         Nu = (Nu & ~1u) | ((Nu >> 1) & 1u);
         Nv = (Nv & ~1u) | ((Nv >> 1) & 1u);
     }
     wn.Wu = Wu; wn.Wv = Wv; wn.Nu = Nu; wn.Nv = Nv; wn.Au = Au; wn.Av = Av; wn.s0 = s0;
+    wn.born = GROW ? ((Bu ? 31u - __clz(Bu) : 0u) | ((Bv ? 31u - __clz(Bv) : 0u) << 8)) : 0u;
     mv.chg = D != 0;
-    mv.inf = !swap && (~Wu & M & Fw) != 0;                        // a flip may not raise a full step (Eq. 5)
+    mv.inf = !swap && (~Wu & D & Fw) != 0;                        // a flip may not raise a full step (Eq. 5)
     const uint32_t hr = (Au ^ Av) & (Wu ^ Nu);                    // a hit is won or lost (v mirrors u in a swap)
     // migrations of a unit at step t are the edges p[t] != p[t-1] (into HBM when p[t] is set, out otherwise):
     // the counts change where an edge appears, disappears or turns around
-    const uint32_t euo = Wu ^ (Wu << 1), eun = Nu ^ (Nu << 1), evo = Wv ^ (Wv << 1), evn = Nv ^ (Nv << 1);
+    // (the edge into the step of birth is no migration; there the placement bit moves a write between H^w and E^w)
+    const uint32_t euo = (Wu ^ (Wu << 1)) & ~Bu, eun = (Nu ^ (Nu << 1)) & ~Bu;
+    const uint32_t evo = (Wv ^ (Wv << 1)) & ~Bv, evn = (Nv ^ (Nv << 1)) & ~Bv;
     const uint32_t mg = (euo ^ eun) | (euo & eun & (Wu ^ Nu)) | (evo ^ evn) | (evo & evn & (Wv ^ Nv));
-    return mv.inf ? 0u : ((hr | mg) & Sb);
+    const uint32_t wr = ((Wu ^ Nu) & Bu) | ((Wv ^ Nv) & Bv);
+    return mv.inf ? 0u : ((hr | mg | wr) & Sb);
 }
 
 // Cost change of the step at window bit k (Eq. 2-4 before and after), from the windows of a proposal.
-__device__ __forceinline__ int item_delta(const Windows& wn, uint32_t k, const uint4 c4, const StepC c, const CostK K)
+// hb: the step's count of units written to HBM at birth (GROW only).
+template <bool GROW>
+__device__ __forceinline__ int item_delta(const Windows& wn, uint32_t k, const uint4 c4, uint32_t hb, const StepC c,
+                                          const CostK K)
 {
     const uint32_t pu = (wn.Wu >> k) & 1u, qu = (wn.Wu >> (k - 1)) & 1u, npu = (wn.Nu >> k) & 1u, nqu = (wn.Nu >> (k - 1)) & 1u;
     const uint32_t pv = (wn.Wv >> k) & 1u, qv = (wn.Wv >> (k - 1)) & 1u, npv = (wn.Nv >> k) & 1u, nqv = (wn.Nv >> (k - 1)) & 1u;
     const uint32_t au = (wn.Au >> k) & 1u, av = (wn.Av >> k) & 1u;
     const uint32_t hr = c4.x + (au & npu) - (au & pu) + (av & npv) - (av & pv);
+    if (GROW) {
+        // mu / mv: 1 when the step is an ordinary one for the unit, 0 when it is the step the unit is written in
+        const uint32_t mu = (wn.born & 255u) == k ? 0u : 1u, mw = ((wn.born >> 8) & 255u) == k ? 0u : 1u;
+        const uint32_t mi = c4.y + mu * ((npu & ~nqu) - (pu & ~qu)) + mw * ((npv & ~nqv) - (pv & ~qv));
+        const uint32_t mo = c4.z + (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
+        const uint32_t hn = hb + (1u - mu) * (npu - pu) + (1u - mw) * (npv - pv);
+        return (int)(step_cost_g(hr, mi, mo, hn, c, K) - step_cost_g(c4.x, c4.y, c4.z, hb, c, K));
+    }
     const uint32_t mi = c4.y + (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
     const uint32_t mo = c4.z + (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
     return (int)(step_cost(hr, mi, mo, c, K) - step_cost(c4.x, c4.y, c4.z, c, K));
@@ -157,19 +196,20 @@ __device__ __forceinline__ bool metropolis(int delta, uint32_t w, const uint32_t
 }
 
 // Whole evaluation in one lane (used where there is no warp to share the work with: calibration).
-template <typename PPtr, typename CPtr, typename FPtr>
+template <bool GROW, typename PPtr, typename CPtr, typename FPtr>
 __device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ Acol, CPtr ctr, FPtr full,
+                                          const uint32_t* __restrict__ birth, const uint32_t* __restrict__ hb,
                                           const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
                                           const uint32_t* __restrict__ trow, uint32_t shift, LaneMove& mv)
 {
     Windows wn;
-    uint32_t todo = lane_windows(P, Acol, full, S, S32, mv, wn);
+    uint32_t todo = lane_windows<GROW>(P, Acol, full, birth, S, S32, mv, wn);
     int delta = 0;
     while (todo) {
         const uint32_t k = __ffs(todo) - 1;
         todo &= todo - 1;
         const uint32_t t = wn.s0 + k - 1;
-        delta += item_delta(wn, k, ctr[t], __ldg(stepc + t), K);
+        delta += item_delta<GROW>(wn, k, ctr[t], GROW ? hb[t] : 0u, __ldg(stepc + t), K);
     }
     mv.delta = delta;
     mv.acc = metropolis(delta, mv.w, trow, shift);
@@ -179,7 +219,9 @@ __device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ A
 // prepares its own proposals, the (proposal, step) pairs whose cost changes are queued in shared memory, and
 // the warp works the queue off 32 pairs at a time, so that lanes with short and long proposals carry the
 // same load.
+template <bool GROW>
 __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* __restrict__ Acol,
+                                           const uint32_t* __restrict__ birth,
                                            const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
                                            const uint32_t* __restrict__ trow, uint32_t shift,
                                            const uint32_t (&need)[kMPL], uint32_t lane, LaneMove (&mv)[kMPL])
@@ -191,9 +233,9 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         if ((need[h] >> lane) & 1u) {
             const uint32_t slot = h * 32 + lane;
             Windows wn;
-            todo[h] = lane_windows(cv.P, Acol, cv.full, S, S32, mv[h], wn);
+            todo[h] = lane_windows<GROW>(cv.P, Acol, cv.full, birth, S, S32, mv[h], wn);
             cv.win[slot * 2] = make_uint4(wn.Wu, wn.Wv, wn.Nu, wn.Nv);
-            cv.win[slot * 2 + 1] = make_uint4(wn.Au, wn.Av, wn.s0, 0u);
+            cv.win[slot * 2 + 1] = make_uint4(wn.Au, wn.Av, wn.s0, wn.born);
             cv.acc[slot] = 0;
         }
         cnt += __popc(todo[h]);
@@ -236,8 +278,9 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
             const uint4 w0 = cv.win[slot[r] * 2], w1 = cv.win[slot[r] * 2 + 1];
             Windows wn;
             wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
+            wn.born = w1.w;
             const uint32_t t = min(wn.s0 + k - 1, S - 1);
-            d[r] = item_delta(wn, k, cv.ctr[t], __ldg(stepc + t), K);
+            d[r] = item_delta<GROW>(wn, k, cv.ctr[t], GROW ? cv.hb[t] : 0u, __ldg(stepc + t), K);
         }
 #pragma unroll
         for (int r = 0; r < 2; ++r)
@@ -254,6 +297,7 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
 
 // Apply the proposal in window slot `slot` (pk, u, v given): all lanes take part, lane j updates the counters
 // of window bit j, lanes 0 and 1 rewrite the words of the schedule and of the full-step bitmap.
+template <bool GROW>
 __device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
                                            uint32_t slot, uint32_t pk, uint32_t u, uint32_t v)
 {
@@ -270,7 +314,14 @@ __device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint3
     const uint32_t au = (Au >> j) & 1u, av = (Av >> j) & 1u;
     uint4 c = cv.ctr[t];
     c.x += (au & npu) - (au & pu) + (av & npv) - (av & pv);
-    c.y += (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
+    if (GROW) {
+        const uint32_t mu = (w1.w & 255u) == j ? 0u : 1u, mw = ((w1.w >> 8) & 255u) == j ? 0u : 1u;
+        c.y += mu * ((npu & ~nqu) - (pu & ~qu)) + mw * ((npv & ~nqv) - (pv & ~qv));
+        const uint32_t dh = (1u - mu) * (npu - pu) + (1u - mw) * (npv - pv);
+        if (valid && dh) cv.hb[t] += dh;
+    } else {
+        c.y += (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
+    }
     c.z += (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
     c.w += npu - pu + npv - pv;
     if (valid) cv.ctr[t] = c;
@@ -310,7 +361,7 @@ __device__ __forceinline__ void copy_words(uint32_t* dst, const uint32_t* src, s
     }
 }
 
-template <bool PSMEM>
+template <bool PSMEM, bool GROW>
 __global__ void __launch_bounds__(512)
 chain_kernel(const ChainParams prm)
 {
@@ -322,17 +373,21 @@ chain_kernel(const ChainParams prm)
     const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
     const size_t pwords = (size_t)U * S32;
     const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
-    const uint32_t fixed4 = S + f4 + kWinSlots4 + kAccSlots4 + kQueueSlots4;   // per-warp shared state besides the schedule
+    const uint32_t h4 = GROW ? (S + 3) / 4 : 0u;                  // uint4 slots of the written-to-HBM counts
+    const uint32_t fixed4 = S + f4 + kWinSlots4 + kAccSlots4 + kQueueSlots4 + h4;   // per-warp shared state besides the schedule
     ChainView cv;
     cv.ctr = smem4 + (size_t)warp * fixed4;
     cv.full = reinterpret_cast<uint32_t*>(cv.ctr + S);
     cv.win = cv.ctr + S + f4;
     cv.acc = reinterpret_cast<int*>(cv.win + kWinSlots4);
     cv.queue = reinterpret_cast<uint16_t*>(cv.win + kWinSlots4 + kAccSlots4);
+    cv.hb = reinterpret_cast<uint32_t*>(cv.win + kWinSlots4 + kAccSlots4 + kQueueSlots4);
     cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)wpb * fixed4) + (size_t)warp * pwords
                  : prm.ws + (size_t)slot * pwords;
     for (uint32_t i = lane; i < S; i += 32) cv.ctr[i] = __ldg(prm.counters0 + i);
     for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
+    if (GROW)
+        for (uint32_t i = lane; i < S; i += 32) cv.hb[i] = __ldg(prm.hb0 + i);
     for (uint32_t i = lane; i < kWinSlots4; i += 32) cv.win[i] = make_uint4(0u, 0u, 0u, 0u);
     copy_words(cv.P, prm.Pcol0, pwords, lane);
     __syncwarp();
@@ -381,7 +436,7 @@ chain_kernel(const ChainParams prm)
             uint32_t any_need = 0;
 #pragma unroll
             for (int h = 0; h < kMPL; ++h) any_need |= need[h];
-            if (any_need) eval_batch(cv, prm.Acol, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+            if (any_need) eval_batch<GROW>(cv, prm.Acol, prm.birth, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
             bool applied = false;
 #pragma unroll
             for (int h = 0; h < kMPL; ++h) need[h] = 0;
@@ -410,7 +465,7 @@ chain_kernel(const ChainParams prm)
                     copy_words(snap, cv.P, pwords, lane);
                     snap_dirty = false;
                 }
-                apply_move(cv, S, S32, prm.cap, lane, h * 32 + b, pk, bu, bv);
+                apply_move<GROW>(cv, S, S32, prm.cap, lane, h * 32 + b, pk, bu, bv);
                 cur = after;
                 const uint64_t mb = m + 32u * h + b;
                 hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
@@ -451,6 +506,7 @@ chain_kernel(const ChainParams prm)
 // Takes a finished chain's schedule back to its best state: the moves applied after the best were logged, each
 // swap or flip is its own inverse, so applying them again in reverse order undoes them. One warp; only the
 // schedule words are touched (the counters are not needed any more).
+template <bool GROW>
 __global__ void __launch_bounds__(32)
 undo_kernel(const ChainParams prm, uint32_t slot, uint32_t* __restrict__ dst)
 {
@@ -471,7 +527,12 @@ undo_kernel(const ChainParams prm, uint32_t slot, uint32_t* __restrict__ dst)
             const uint32_t wj = (s0 >> 5) + lane;
             const uint32_t lo = max(s0, wj * 32u), hi = min(end, wj * 32u + 32u);
             if (hi > lo) {                               // run lengths are at most 30, so never a full word
-                const uint32_t mask = ((1u << (hi - lo)) - 1u) << (lo - wj * 32u);
+                uint32_t mask = ((1u << (hi - lo)) - 1u) << (lo - wj * 32u);
+                if (GROW) {                              // only the steps at which the units exist were touched
+                    const uint32_t b = max(__ldg(prm.birth + mv.u), swap ? __ldg(prm.birth + mv.v) : 0u);
+                    if (b >= wj * 32u + 32u) mask = 0u;
+                    else if (b > wj * 32u) mask &= 0xFFFFFFFFu << (b - wj * 32u);
+                }
                 const size_t iu = (size_t)mv.u * S32 + wj, iv = (size_t)mv.v * S32 + wj;
                 if (swap) {
                     const uint32_t a = P[iu], b = P[iv], d = (a ^ b) & mask;
@@ -497,6 +558,7 @@ __global__ void full_mask_kernel(const uint4* __restrict__ counters0, uint32_t S
 
 // Calibration of the temperature ladder: proposals (i, 0, 0, TAG_CALIB), i < 1024, are evaluated against the
 // initial schedule and never applied; acc = {sum of positive deltas, their number}.
+template <bool GROW>
 __global__ void __launch_bounds__(256)
 calib_kernel(const ChainParams prm, unsigned long long* acc)
 {
@@ -506,7 +568,8 @@ calib_kernel(const ChainParams prm, unsigned long long* acc)
     LaneMove mv;
     philox4x32_10(i, 0u, 0u, TAG_CALIB, prm.seed_lo, prm.seed_hi, r);
     decode_move(r, prm.p_swap_256, prm.len_choices, prm.S, prm.U, mv);
-    eval_lane(prm.Pcol0, prm.Acol, prm.counters0, prm.full0, prm.stepc, prm.K, prm.S, prm.S32, prm.table, 0u, mv);
+    eval_lane<GROW>(prm.Pcol0, prm.Acol, prm.counters0, prm.full0, prm.birth, prm.hb0, prm.stepc, prm.K, prm.S, prm.S32,
+                    prm.table, 0u, mv);
     if (!mv.inf && mv.delta > 0) {
         atomicAdd(acc, (unsigned long long)mv.delta);
         atomicAdd(acc + 1, 1ull);
@@ -568,6 +631,9 @@ struct Ctx {
     uint32_t* sched;         // [S][W32]
     uint32_t* slots;         // chain state slices (global variant)
     uint32_t* full0;         // [S32]
+    uint32_t* hb0;           // growing cache: [S] written-to-HBM counts of the initial schedule
+    uint32_t* hb_tmp;        // growing cache: [S] the same for the winner's re-score
+    bool grow;
     uint32_t* snap;          // best-state snapshots (shared-memory variant), or null
     uint64_t* undo_log;      // undo logs (global variant), or null
     uint32_t* undo_len;
@@ -592,12 +658,19 @@ int validate(const kvp_problem* p, const kvp_anneal_params* a)
     return KVP_OK;
 }
 
-template <bool PSMEM>
+typedef void (*ChainKernel)(const ChainParams);
+
+ChainKernel chain_kernel_for(bool psmem, bool grow)
+{
+    return psmem ? (grow ? chain_kernel<true, true> : chain_kernel<true, false>)
+                 : (grow ? chain_kernel<false, true> : chain_kernel<false, false>);
+}
+
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 {
     const uint32_t grid = (count + c.wpb - 1) / c.wpb;
     const size_t smem = (size_t)c.wpb * c.smem_per_warp;
-    chain_kernel<PSMEM><<<grid, c.wpb * 32, smem, c.st>>>(prm);
+    chain_kernel_for(c.psmem, c.grow)<<<grid, c.wpb * 32, smem, c.st>>>(prm);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }
@@ -611,7 +684,7 @@ int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp
     prm.chain_first = first; prm.chain_count = count; prm.result_base = result_base;
     prm.results = results; prm.upto = upto; prm.dump = dump;
     ++c.launches;
-    return c.psmem ? launch_chains<true>(c, prm, count) : launch_chains<false>(c, prm, count);
+    return launch_chains(c, prm, count);
 }
 
 // Initial schedule, its counters and cost, the temperature ladder and the acceptance table.
@@ -631,7 +704,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     KVP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const size_t budget = (size_t)smem_max - 1024;
     // per warp: counters, full-step bitmap, the batch's windows, accumulators and work queue
-    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4 + kWinSlots4 + kAccSlots4 + kQueueSlots4) * 16;
+    c.grow = p->dL != nullptr;
+    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4 + kWinSlots4 + kAccSlots4 + kQueueSlots4 +
+                              (c.grow ? (p->S + 3) / 4 : 0)) * 16;
     const size_t psmem_per_warp = ctr_bytes + (size_t)p->U * p->S32 * 4;
     c.psmem = psmem_per_warp <= budget / 2;
     if (c.psmem) {
@@ -641,15 +716,15 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
         uint32_t want = (a->chains + sms - 1) / sms;
         c.wpb = want < 1 ? 1 : (want > wmax ? wmax : want);
         c.resident = a->chains;
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.grow), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
         if (ctr_bytes > budget) return KVP_ERR_RANGE;
         c.smem_per_warp = ctr_bytes;
         uint32_t wmax = (uint32_t)(budget / 2 / ctr_bytes);
         c.wpb = wmax < 1 ? 1 : (wmax > 16 ? 16 : wmax);
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, c.grow), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
         int ctas = 0;
-        KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel<false>, (int)c.wpb * 32,
+        KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, c.grow), (int)c.wpb * 32,
                                                                c.wpb * c.smem_per_warp));
         if (ctas < 1) return KVP_ERR_RANGE;
         uint32_t per_sm = (uint32_t)ctas * c.wpb;                  // resident chains per SM, at most 32
@@ -683,6 +758,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const size_t o_dump = take(col_bytes), o_sched = take(sched_bytes);
     const size_t o_slots = take(c.psmem ? 0 : (size_t)c.resident * col_bytes);
     const size_t o_full = take((size_t)p->S32 * 4);
+    const size_t o_hb0 = take(c.grow ? (size_t)p->S * 4 : 0), o_hbt = take(c.grow ? (size_t)p->S * 4 : 0);
     // Chains whose schedule lives in shared memory save it to global memory whenever they leave their best state;
     // chains in global scratch do not (a copy would cost as much as thousands of moves): their winner is replayed.
     const size_t snap_bytes = (size_t)a->chains * p->U * p->S32 * 4;
@@ -699,6 +775,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     c.small = (uint64_t*)(base + o_small); c.table = (uint32_t*)(base + o_table); c.shifts = (uint32_t*)(base + o_shift);
     c.results = (kvp_chain_result*)(base + o_res); c.dumpcol = (uint32_t*)(base + o_dump);
     c.sched = (uint32_t*)(base + o_sched); c.slots = (uint32_t*)(base + o_slots);
+    c.hb0 = c.grow ? (uint32_t*)(base + o_hb0) : nullptr; c.hb_tmp = c.grow ? (uint32_t*)(base + o_hbt) : nullptr;
     c.full0 = (uint32_t*)(base + o_full); c.snap = snapshots ? (uint32_t*)(base + o_snap) : nullptr;
     c.undo_log = c.psmem ? nullptr : (uint64_t*)(base + o_ulog); c.undo_len = c.psmem ? nullptr : (uint32_t*)(base + o_ulen);
 
@@ -715,11 +792,18 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             ++c.launches;
         }
         if ((rc = launch_broadcast_row(row, p->S, p->W32, c.P0, st))) return rc;
-        if ((rc = launch_row_to_columns(row, p->U, p->S, p->S32, c.Pcol0, st))) return rc;
+        if (!c.grow && (rc = launch_row_to_columns(row, p->U, p->S, p->S32, c.Pcol0, st))) return rc;
         c.launches += 2;
     }
-    if ((rc = launch_counts(p, c.P0, 1, c.counts0, st, &c.launches))) return rc;
-    if ((rc = launch_finish(p, c.counts0, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2), c.small + 1, st)))
+    if (c.grow) {
+        // a unit of the initial placement enters HBM when it is written; the chains keep the bits before that clear
+        if ((rc = launch_and_rows(c.P0, p->dL, (size_t)p->S * p->W32, st))) return rc;
+        if ((rc = launch_bit_transpose(c.P0, p->S, p->W32, p->U, c.Pcol0, p->S32, st))) return rc;
+        c.launches += a->init_mode == KVP_INIT_USER ? 2 : 1;
+    }
+    if ((rc = launch_counts(p, c.P0, 1, c.counts0, c.hb0, st, &c.launches))) return rc;
+    if ((rc = launch_finish(p, c.counts0, c.hb0, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2), c.small + 1,
+                            st)))
         return rc;
     ++c.launches;
     full_mask_kernel<<<(p->S32 * 32 + 255) / 256, 256, 0, st>>>((const uint4*)c.counts0, p->S, p->cap, c.full0);
@@ -730,6 +814,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     memset(&prm, 0, sizeof prm);
     prm.Acol = p->dAcol; prm.stepc = p->d_stepc; prm.counters0 = (const uint4*)c.counts0; prm.Pcol0 = c.Pcol0;
     prm.table = c.table; prm.shifts = c.shifts; prm.ws = c.slots; prm.K = p->K; prm.full0 = c.full0;
+    prm.birth = p->d_birth; prm.hb0 = c.hb0;
     prm.U = p->U; prm.S = p->S; prm.S32 = p->S32; prm.cap = p->cap;
     prm.levels = a->levels; prm.p_swap_256 = a->p_swap_256; prm.len_choices = a->max_len_log2 + 1;
     prm.early_permille = a->early_stop_permille; prm.early_from = a->early_stop_from_level;
@@ -742,7 +827,8 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const bool calibrate = a->temps == nullptr;
     if (calibrate) {
         KVP_CUDA(cudaMemsetAsync(c.small + 4, 0, 16, st));
-        calib_kernel<<<CALIB_N / 256, 256, 0, st>>>(prm, (unsigned long long*)(c.small + 4));
+        if (c.grow) calib_kernel<true><<<CALIB_N / 256, 256, 0, st>>>(prm, (unsigned long long*)(c.small + 4));
+        else calib_kernel<false><<<CALIB_N / 256, 256, 0, st>>>(prm, (unsigned long long*)(c.small + 4));
         KVP_CUDA(cudaGetLastError());
         ++c.launches;
     }
@@ -832,7 +918,8 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
                     ChainParams prm = c.prm;
                     prm.chain_first = a->first_chain + first;
                     prm.undo_log = c.undo_log; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
-                    undo_kernel<<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
+                    if (c.grow) undo_kernel<true><<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
+                    else undo_kernel<false><<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
                     KVP_CUDA(cudaGetLastError());
                     ++c.launches;
                     dumped_chain = red.best_chain;
@@ -861,8 +948,9 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
         red.best_chain += a->first_chain;
         if ((rc = replay_to_sched(p, c, red.best_chain, upto, c.results + a->chains))) { cleanup(); return rc; }
     }
-    if ((rc = launch_counts(p, c.sched, 1, c.counts0, st, &c.launches))) { cleanup(); return rc; }
-    if ((rc = launch_finish(p, c.counts0, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2), c.small + 1, st))) {
+    if ((rc = launch_counts(p, c.sched, 1, c.counts0, c.hb_tmp, st, &c.launches))) { cleanup(); return rc; }
+    if ((rc = launch_finish(p, c.counts0, c.hb_tmp, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2),
+                            c.small + 1, st))) {
         cleanup(); return rc;
     }
     ++c.launches;

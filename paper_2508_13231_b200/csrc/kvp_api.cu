@@ -90,6 +90,8 @@ extern "C" void kvp_destroy(kvp_problem* p)
     if (p->d_block) cudaFreeAsync(p->d_block, p->last_stream);
     if (p->d_scratch) cudaFreeAsync(p->d_scratch, p->last_stream);
     if (p->d_chain_ws) cudaFreeAsync(p->d_chain_ws, p->last_stream);
+    if (p->d_grow_block) cudaFreeAsync(p->d_grow_block, p->last_stream);
+    free(p->h_writes);
     delete p;
 }
 
@@ -120,8 +122,12 @@ static int create_impl(kvp_problem* p, const uint32_t* access, const uint32_t* h
     // Per-step constants of the cost function; everything must stay below 2^31 so that the
     // annealer can work in 32-bit arithmetic.
     uint64_t wmax = 0;
+    p->h_writes = static_cast<uint32_t*>(malloc((size_t)p->S * 4));
+    if (!p->h_writes) return KVP_ERR_NOMEM;
     for (uint32_t s = 0; s < p->S; ++s) {
         const uint64_t e = (uint64_t)(hw ? hw[s] : 0) + (ew ? ew[s] : 0);
+        if (e >= (1ull << 31)) return KVP_ERR_RANGE;
+        p->h_writes[s] = (uint32_t)e;
         if (e > wmax) wmax = e;
     }
     const uint64_t kmax = p->kh > p->ke ? p->kh : p->ke;
@@ -165,9 +171,50 @@ extern "C" int kvp_create(kvp_problem** out, uint32_t units, uint64_t bytes_per_
     if (p->kh >= (1ull << 31) || p->ke >= (1ull << 31)) { delete p; return KVP_ERR_RANGE; }
     p->K.kh = (uint32_t)p->kh; p->K.ke = (uint32_t)p->ke;
     p->K.khF = (uint32_t)p->kh * Fh; p->K.kkF = (uint32_t)p->kk * Fe; p->K.kdF = (uint32_t)p->kd * Fe;
+    p->K.kk = (uint32_t)p->kk; p->K.kd = (uint32_t)p->kd;
     rc = create_impl(p, access_bitmaps, hw_units, ew_units, static_cast<cudaStream_t>(stream));
     if (rc) { kvp_destroy(p); return rc; }
     *out = p;
+    return KVP_OK;
+}
+
+extern "C" int kvp_set_births(kvp_problem* p, const uint32_t* birth, void* stream)
+{
+    if (!p || !birth || p->dL) return KVP_ERR_ARG;
+    KVP_CUDA(cudaSetDevice(p->device));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
+    const size_t nw = (size_t)p->S * p->W32;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) & ~(size_t)255; return o; };
+    const size_t ob = take((size_t)p->U * 4), oL = take(nw * 4), onb = take((size_t)p->S * 4 + 4);
+    void* block = nullptr;
+    KVP_CUDA(cudaMallocAsync(&block, off, st));
+    char* base = static_cast<char*>(block);
+    uint32_t* d_birth = (uint32_t*)(base + ob);
+    uint32_t* dL = (uint32_t*)(base + oL);
+    uint32_t* d_nb = (uint32_t*)(base + onb);            // [S] births per step, then the check flags
+    std::vector<uint32_t> nb((size_t)p->S + 1);
+    int rc = KVP_OK;
+    auto fail = [&](int code) { cudaFreeAsync(block, st); return code; };
+    if (cudaMemcpyAsync(d_birth, birth, (size_t)p->U * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+        cudaMemsetAsync(d_nb, 0, (size_t)p->S * 4 + 4, st) != cudaSuccess)
+        return fail(set_cuda_error(cudaGetLastError(), "kvp_set_births copy"));
+    if ((rc = launch_birth_stats(d_birth, p->U, p->S, p->dAcol, p->S32, d_nb, d_nb + p->S, st))) return fail(rc);
+    if ((rc = launch_alive_rows(d_birth, p->U, p->S, p->W32, dL, st))) return fail(rc);
+    if (cudaMemcpyAsync(nb.data(), d_nb, (size_t)p->S * 4 + 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return fail(set_cuda_error(cudaGetLastError(), "kvp_set_births read-back"));
+    if (nb[p->S]) return fail(KVP_ERR_ARG);              // a birth beyond the horizon, or an access before birth
+    uint64_t wmax = 0;
+    for (uint32_t s = 0; s < p->S; ++s) {
+        const uint64_t e = (uint64_t)p->h_writes[s] + nb[s];
+        if (e > wmax) wmax = e;
+    }
+    const uint64_t kmax = p->kh > p->ke ? p->kh : p->ke;
+    if (kmax * (2ull * p->U + wmax) >= (1ull << 31)) return fail(KVP_ERR_RANGE);
+    if ((rc = launch_stepc_births(p->d_stepc, d_nb, p->S, p->K.kk, p->K.kd, st))) return fail(rc);
+    p->d_grow_block = block; p->d_birth = d_birth; p->dL = dL;
     return KVP_OK;
 }
 

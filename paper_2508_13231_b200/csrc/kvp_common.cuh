@@ -17,6 +17,7 @@ struct CostK {
     uint32_t kh, ke;      // kappa_h, kappa_e
     uint32_t khF;         // kappa_h * Fh
     uint32_t kkF, kdF;    // kappa_k * Fe, kappa_d * Fe
+    uint32_t kk, kd;      // kappa_k, kappa_d (writes are charged whatever the migration flags say)
 };
 
 // Per-step constants: x = kappa_h*hw, y = kappa_k*ew, z = kappa_d*ew, w = kappa_e*|A[s]|.
@@ -57,6 +58,20 @@ __host__ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1,
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// The same with a growing cache: hb units are written to HBM at birth during this step. c.y and c.z count every
+// unit born in the step as written to DRAM; each one that goes to HBM instead moves from |E^w| to |H^w|.
+__device__ __forceinline__ uint32_t step_cost_g(uint32_t hr, uint32_t mi, uint32_t mo, uint32_t hb, const StepC c,
+                                                const CostK k)
+{
+    const uint32_t mm = mi + mo;
+    const uint32_t th = c.x + k.kh * (hr + hb) + k.khF * mm;          // Eq. 3
+    const uint32_t e1 = c.y - k.kk * hb + k.kkF * mo;
+    const uint32_t e2 = k.kkF * mi;
+    const uint32_t e3 = c.z - k.kd * hb + k.kdF * mm;
+    const uint32_t te = c.w - k.ke * hr + max(max(e1, e2), e3);       // Eq. 4
+    return max(th, te);                                               // Eq. 2
+}
+
 }  // namespace kvp
 
 // Host-side problem object behind the opaque handle.
@@ -77,6 +92,11 @@ struct kvp_problem {
     uint32_t* d_ucnt;    // [U]        accesses per unit over all steps
     uint32_t* d_row_freq;// [W32]      STATIC_FREQ row
     uint64_t total_accessed;
+    // growing cache (kvp_set_births); all null for a fixed population
+    uint32_t* d_birth;   // [U]        step at which a unit is written, 0 = there from the start
+    uint32_t* dL;        // [S][W32]   bit u of row s set iff unit u exists at step s
+    void* d_grow_block;  // the allocation behind the two
+    uint32_t* h_writes;  // (host) [S] hw + ew of kvp_create, for the range check of kvp_set_births
     void* d_block;             // one allocation behind the pointers above
     cudaStream_t last_stream;  // stream of the most recent call; frees are ordered behind it
     // scratch owned by the problem, grown on demand
@@ -98,10 +118,12 @@ int ensure_chain_ws(kvp_problem* p, size_t bytes, cudaStream_t st);
 
 // kvp_cost.cu
 int launch_row_popcount(const uint32_t* rows, uint32_t S, uint32_t W32, uint32_t* out, cudaStream_t st);
-int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, uint32_t* counts, cudaStream_t st,
-                  uint32_t* launches);
-int launch_finish(const kvp_problem* p, const uint32_t* counts, uint32_t n, uint64_t* step_ticks, uint64_t* total_ticks,
-                  double* step_seconds, double* total_seconds, int32_t* bad_step, uint64_t* hits, cudaStream_t st);
+// hbc: [n][S] units written to HBM at birth; needed (and only used) when the problem has births
+int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, uint32_t* counts, uint32_t* hbc,
+                  cudaStream_t st, uint32_t* launches);
+int launch_finish(const kvp_problem* p, const uint32_t* counts, const uint32_t* hbc, uint32_t n, uint64_t* step_ticks,
+                  uint64_t* total_ticks, double* step_seconds, double* total_seconds, int32_t* bad_step, uint64_t* hits,
+                  cudaStream_t st);
 
 // kvp_layout.cu
 int launch_bit_transpose(const uint32_t* in, uint32_t rows, uint32_t in_words, uint32_t cols, uint32_t* out,
@@ -112,5 +134,10 @@ int launch_static_freq_row(const kvp_problem* p, uint32_t* row, cudaStream_t st)
 int launch_static_first_row(const kvp_problem* p, uint32_t* row, cudaStream_t st);
 int launch_broadcast_row(const uint32_t* row, uint32_t S, uint32_t W32, uint32_t* sched, cudaStream_t st);
 int launch_row_to_columns(const uint32_t* row, uint32_t U, uint32_t S, uint32_t S32, uint32_t* Pcol, cudaStream_t st);
+int launch_alive_rows(const uint32_t* birth, uint32_t U, uint32_t S, uint32_t W32, uint32_t* L, cudaStream_t st);
+int launch_birth_stats(const uint32_t* birth, uint32_t U, uint32_t S, const uint32_t* Acol, uint32_t S32, uint32_t* nb,
+                       uint32_t* flag, cudaStream_t st);
+int launch_stepc_births(StepC* stepc, const uint32_t* nb, uint32_t S, uint32_t kk, uint32_t kd, cudaStream_t st);
+int launch_and_rows(uint32_t* sched, const uint32_t* L, size_t total, cudaStream_t st);
 
 }  // namespace kvp

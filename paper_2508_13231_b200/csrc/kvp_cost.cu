@@ -84,19 +84,24 @@ __device__ __forceinline__ uint32_t popc8(const uint32_t (&w)[8])
 // Wide rows: a warp owns 64 consecutive 16-byte vectors (1 KB) of every row of a step chunk, two per lane.
 // Per lane and step only three cardinalities are counted, hits |A&P|, occupancy |P| and stayers |P&Pprev|;
 // migrations follow as mi = occ - stay and mo = occ_prev - stay.
-template <int VEC>
+// GROW (growing cache): L holds the rows of existing units. Placement bits of units that do not exist yet are
+// dropped, and the units born in a step (in L[s], not in L[s-1]) that are placed in HBM are a fourth cardinality
+// hb: they were written there, not migrated, so mi = occ - stay - hb.
+template <int VEC, bool GROW>
 __global__ void __launch_bounds__(WIDE_WARPS * 32)
 count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ Ps, uint32_t S, uint32_t W32,
-                  uint32_t WV, uint32_t pad_mask, uint32_t SC, uint32_t* __restrict__ counts)
+                  uint32_t WV, uint32_t pad_mask, uint32_t SC, uint32_t* __restrict__ counts,
+                  const uint32_t* __restrict__ L, uint32_t* __restrict__ hbc)
 {
-    extern __shared__ uint2 acc[];                       // [WIDE_WARPS][SC]
+    extern __shared__ uint2 acc[];                       // [WIDE_WARPS][SC], then GROW: uint32 [WIDE_WARPS][SC]
+    uint32_t* acc_hb = reinterpret_cast<uint32_t*>(acc + WIDE_WARPS * SC);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cv0 = (blockIdx.x * WIDE_WARPS + warp) * (32 * WIDE_VEC) + lane;
     const uint32_t sb = blockIdx.y * SC;
     const uint32_t se = min(S, sb + SC);
     const uint32_t* __restrict__ P = Ps + (size_t)blockIdx.z * S * W32;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    uint4 prev[WIDE_VEC];
+    uint4 prev[WIDE_VEC], lprev[WIDE_VEC];
     uint32_t occ_prev;
     {
         uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -104,19 +109,30 @@ count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ P
         for (int j = 0; j < WIDE_VEC; ++j) {
             const uint32_t cv = cv0 + 32 * j;
             prev[j] = cv < WV ? mask_last<VEC>(load_vec<VEC>(P, W32, sb ? sb - 1 : 0, cv), cv, WV, pad_mask) : zero;
+            if (GROW) {
+                lprev[j] = cv < WV ? load_vec<VEC>(L, W32, sb ? sb - 1 : 0, cv) : zero;
+                prev[j] = and4(prev[j], lprev[j]);
+            }
             w[4 * j] = prev[j].x; w[4 * j + 1] = prev[j].y; w[4 * j + 2] = prev[j].z; w[4 * j + 3] = prev[j].w;
         }
         occ_prev = popc8(w);
     }
 #pragma unroll 4
     for (uint32_t s = sb; s < se; ++s) {
-        uint32_t wp[8], wh[8], ws[8];
+        uint32_t wp[8], wh[8], ws[8], wb[8];
 #pragma unroll
         for (int j = 0; j < WIDE_VEC; ++j) {
             const uint32_t cv = cv0 + 32 * j;
             const bool valid = cv < WV;
             const uint4 a = valid ? load_vec<VEC>(A, W32, s, cv) : zero;
-            const uint4 p = valid ? mask_last<VEC>(load_stream<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
+            uint4 p = valid ? mask_last<VEC>(load_stream<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
+            if (GROW) {
+                const uint4 l = valid ? load_vec<VEC>(L, W32, s, cv) : zero;
+                p = and4(p, l);
+                const uint4 born = andn4(p, lprev[j]);               // placed in HBM in the step it is written
+                wb[4 * j] = born.x; wb[4 * j + 1] = born.y; wb[4 * j + 2] = born.z; wb[4 * j + 3] = born.w;
+                lprev[j] = l;
+            }
             wp[4 * j] = p.x; wp[4 * j + 1] = p.y; wp[4 * j + 2] = p.z; wp[4 * j + 3] = p.w;
             wh[4 * j] = a.x & p.x; wh[4 * j + 1] = a.y & p.y; wh[4 * j + 2] = a.z & p.z; wh[4 * j + 3] = a.w & p.w;
             ws[4 * j] = p.x & prev[j].x; ws[4 * j + 1] = p.y & prev[j].y;
@@ -124,11 +140,17 @@ count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ P
             prev[j] = p;
         }
         const uint32_t occ = popc8(wp), hr = popc8(wh), stay = popc8(ws);
-        uint2 c = make_uint2(hr | ((occ - stay) << 16), (occ_prev - stay) | (occ << 16));
+        uint32_t hb = 0;
+        if (GROW) hb = popc8(wb);
+        uint2 c = make_uint2(hr | ((occ - stay - hb) << 16), (occ_prev - stay) | (occ << 16));
         occ_prev = occ;
         c.x = __reduce_add_sync(0xFFFFFFFFu, c.x);       // 16-bit fields: 32 lanes * 256 < 65536
         c.y = __reduce_add_sync(0xFFFFFFFFu, c.y);
-        if (lane == 0) acc[warp * SC + (s - sb)] = c;
+        if (GROW) hb = __reduce_add_sync(0xFFFFFFFFu, hb);
+        if (lane == 0) {
+            acc[warp * SC + (s - sb)] = c;
+            if (GROW) acc_hb[warp * SC + (s - sb)] = hb;
+        }
     }
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < se - sb; i += blockDim.x) {
@@ -143,15 +165,22 @@ count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ P
         if (mi) atomicAdd(dst + 1, mi);
         if (mo) atomicAdd(dst + 2, mo);
         if (occ) atomicAdd(dst + 3, occ);
+        if (GROW) {
+            uint32_t hb = 0;
+#pragma unroll
+            for (int w = 0; w < WIDE_WARPS; ++w) hb += acc_hb[w * SC + i];
+            if (hb) atomicAdd(hbc + (size_t)blockIdx.z * S + sb + i, hb);
+        }
     }
 }
 
 constexpr int NARROW_ITERS = 8;
 
-template <int VEC, int LPR>
+template <int VEC, int LPR, bool GROW>
 __global__ void __launch_bounds__(256)
 count_narrow_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ Ps, uint32_t S, uint32_t W32,
-                    uint32_t WV, uint32_t pad_mask, uint32_t* __restrict__ counts)
+                    uint32_t WV, uint32_t pad_mask, uint32_t* __restrict__ counts, const uint32_t* __restrict__ L,
+                    uint32_t* __restrict__ hbc)
 {
     constexpr uint32_t GROUPS = 256 / LPR;               // rows in flight per CTA
     const uint32_t g = threadIdx.x / LPR, cv = threadIdx.x % LPR;
@@ -163,22 +192,35 @@ count_narrow_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__
         const uint32_t s = (blockIdx.x * NARROW_ITERS + it) * GROUPS + g;
         const bool ok = col_ok && s < S;
         const uint4 a = ok ? load_vec<VEC>(A, W32, s, cv) : zero;
-        const uint4 p = ok ? mask_last<VEC>(load_vec<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
-        const uint4 q = ok ? mask_last<VEC>(load_vec<VEC>(P, W32, s ? s - 1 : 0, cv), cv, WV, pad_mask) : zero;
+        uint4 p = ok ? mask_last<VEC>(load_vec<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
+        uint4 q = ok ? mask_last<VEC>(load_vec<VEC>(P, W32, s ? s - 1 : 0, cv), cv, WV, pad_mask) : zero;
+        uint32_t hb = 0;
+        if (GROW) {                                      // see count_wide_kernel
+            const uint4 l = ok ? load_vec<VEC>(L, W32, s, cv) : zero;
+            const uint4 lq = ok ? load_vec<VEC>(L, W32, s ? s - 1 : 0, cv) : zero;
+            p = and4(p, l);
+            q = and4(q, lq);
+            hb = popc4(andn4(p, lq));
+        }
         uint2 c = vec_counts(a, p, q);
+        if (GROW) c.x -= hb << 16;                       // born in HBM: written, not migrated in
 #pragma unroll
         for (int off = LPR / 2; off > 0; off >>= 1) {
             c.x += __shfl_xor_sync(0xFFFFFFFFu, c.x, off);
             c.y += __shfl_xor_sync(0xFFFFFFFFu, c.y, off);
+            if (GROW) hb += __shfl_xor_sync(0xFFFFFFFFu, hb, off);
         }
-        if (cv == 0 && s < S)
+        if (cv == 0 && s < S) {
             reinterpret_cast<uint4*>(counts)[(size_t)blockIdx.y * S + s] =
                 make_uint4(c.x & 0xFFFFu, c.x >> 16, c.y & 0xFFFFu, c.y >> 16);
+            if (GROW) hbc[(size_t)blockIdx.y * S + s] = hb;
+        }
     }
 }
 
 __global__ void __launch_bounds__(256)
-finish_kernel(const uint4* __restrict__ counts, const StepC* __restrict__ stepc, CostK K, uint32_t S, uint32_t cap,
+finish_kernel(const uint4* __restrict__ counts, const uint32_t* __restrict__ hbc, const StepC* __restrict__ stepc, CostK K,
+              uint32_t S, uint32_t cap,
               double spt, uint64_t* __restrict__ step_ticks, uint64_t* __restrict__ total_ticks,
               double* __restrict__ step_seconds, double* __restrict__ total_seconds, int32_t* __restrict__ bad_step,
               uint64_t* __restrict__ hits)
@@ -190,7 +232,8 @@ finish_kernel(const uint4* __restrict__ counts, const StepC* __restrict__ stepc,
     uint32_t bad = 0xFFFFFFFFu;
     for (uint32_t s = threadIdx.x; s < S; s += blockDim.x) {
         const uint4 c = counts[(size_t)i * S + s];
-        const uint32_t f = step_cost(c.x, c.y, c.z, __ldg(&stepc[s]), K);
+        const uint32_t f = hbc ? step_cost_g(c.x, c.y, c.z, hbc[(size_t)i * S + s], __ldg(&stepc[s]), K)
+                               : step_cost(c.x, c.y, c.z, __ldg(&stepc[s]), K);
         if (step_ticks) step_ticks[(size_t)i * S + s] = f;
         if (step_seconds) step_seconds[(size_t)i * S + s] = (double)f * spt;
         sum += f;
@@ -226,16 +269,15 @@ row_popcount_kernel(const uint32_t* __restrict__ rows, uint32_t S, uint32_t W32,
     if (lane == 0) out[warp] = c;
 }
 
-template <int VEC>
-int launch_narrow(uint32_t WV, dim3 grid_rows, uint32_t n, const uint32_t* A, const uint32_t* P, uint32_t S, uint32_t W32,
-                  uint32_t pad_mask, uint32_t* counts, cudaStream_t st)
+template <int VEC, bool GROW>
+int launch_narrow(uint32_t WV, uint32_t n, const uint32_t* A, const uint32_t* P, uint32_t S, uint32_t W32,
+                  uint32_t pad_mask, uint32_t* counts, const uint32_t* L, uint32_t* hbc, cudaStream_t st)
 {
-    (void)grid_rows;
-#define KVP_NARROW(LPR)                                                                          \
-    {                                                                                            \
-        const uint32_t rows_per_cta = (256 / LPR) * NARROW_ITERS;                                \
-        dim3 grid((S + rows_per_cta - 1) / rows_per_cta, n);                                     \
-        count_narrow_kernel<VEC, LPR><<<grid, 256, 0, st>>>(A, P, S, W32, WV, pad_mask, counts); \
+#define KVP_NARROW(LPR)                                                                                          \
+    {                                                                                                            \
+        const uint32_t rows_per_cta = (256 / LPR) * NARROW_ITERS;                                                \
+        dim3 grid((S + rows_per_cta - 1) / rows_per_cta, n);                                                     \
+        count_narrow_kernel<VEC, LPR, GROW><<<grid, 256, 0, st>>>(A, P, S, W32, WV, pad_mask, counts, L, hbc);   \
     }
     if (WV <= 1) KVP_NARROW(1)
     else if (WV <= 2) KVP_NARROW(2)
@@ -256,18 +298,24 @@ int launch_row_popcount(const uint32_t* rows, uint32_t S, uint32_t W32, uint32_t
     return KVP_OK;
 }
 
-// counts [n][S][4] = {hr, mi, mo, occ}
-int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, uint32_t* counts, cudaStream_t st,
-                  uint32_t* launches)
+// counts [n][S][4] = {hr, mi, mo, occ}; hbc [n][S] for a problem with births
+int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, uint32_t* counts, uint32_t* hbc,
+                  cudaStream_t st, uint32_t* launches)
 {
+    const bool grow = p->dL != nullptr;
+    if (grow && !hbc) return KVP_ERR_ARG;
     const bool vec4 = (p->W32 % 4 == 0) && ((reinterpret_cast<uintptr_t>(schedules) & 15) == 0);
     const uint32_t WV = vec4 ? p->W32 / 4 : p->W32;
     if (WV <= 16) {
         if (launches) *launches += 1;
-        return vec4 ? launch_narrow<4>(WV, dim3(), n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, st)
-                    : launch_narrow<1>(WV, dim3(), n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, st);
+        if (grow)
+            return vec4 ? launch_narrow<4, true>(WV, n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, p->dL, hbc, st)
+                        : launch_narrow<1, true>(WV, n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, p->dL, hbc, st);
+        return vec4 ? launch_narrow<4, false>(WV, n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, nullptr, nullptr, st)
+                    : launch_narrow<1, false>(WV, n, p->dA, schedules, p->S, p->W32, p->pad_mask, counts, nullptr, nullptr, st);
     }
     KVP_CUDA(cudaMemsetAsync(counts, 0, (size_t)n * p->S * 16, st));
+    if (grow) KVP_CUDA(cudaMemsetAsync(hbc, 0, (size_t)n * p->S * 4, st));
     const uint32_t col_ctas = (WV + WIDE_WARPS * 32 * WIDE_VEC - 1) / (WIDE_WARPS * 32 * WIDE_VEC);
     // Split the steps until the grid is at least four full waves (148 SMs x 8 resident CTAs), so that the last,
     // partial wave costs little; every chunk re-reads one halo row (1/SC more traffic, mostly from L2).
@@ -275,21 +323,31 @@ int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, u
     while (SC > 8 && (uint64_t)col_ctas * ((p->S + SC - 1) / SC) * n < 148u * 8u * 4u) SC = (SC + 1) / 2;
     if (SC > 512) SC = 512;
     dim3 grid(col_ctas, (p->S + SC - 1) / SC, n);
-    const size_t smem = (size_t)WIDE_WARPS * SC * sizeof(uint2);
-    if (vec4)
-        count_wide_kernel<4><<<grid, WIDE_WARPS * 32, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts);
-    else
-        count_wide_kernel<1><<<grid, WIDE_WARPS * 32, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts);
+    const size_t smem = (size_t)WIDE_WARPS * SC * (sizeof(uint2) + (grow ? 4 : 0));
+    const int T = WIDE_WARPS * 32;
+    if (grow) {
+        if (vec4)
+            count_wide_kernel<4, true><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, p->dL, hbc);
+        else
+            count_wide_kernel<1, true><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, p->dL, hbc);
+    } else {
+        if (vec4)
+            count_wide_kernel<4, false><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, nullptr, nullptr);
+        else
+            count_wide_kernel<1, false><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, nullptr, nullptr);
+    }
     KVP_CUDA(cudaGetLastError());
     if (launches) *launches += 1;
     return KVP_OK;
 }
 
-int launch_finish(const kvp_problem* p, const uint32_t* counts, uint32_t n, uint64_t* step_ticks, uint64_t* total_ticks,
-                  double* step_seconds, double* total_seconds, int32_t* bad_step, uint64_t* hits, cudaStream_t st)
+int launch_finish(const kvp_problem* p, const uint32_t* counts, const uint32_t* hbc, uint32_t n, uint64_t* step_ticks,
+                  uint64_t* total_ticks, double* step_seconds, double* total_seconds, int32_t* bad_step, uint64_t* hits,
+                  cudaStream_t st)
 {
-    finish_kernel<<<n, 256, 0, st>>>(reinterpret_cast<const uint4*>(counts), p->d_stepc, p->K, p->S, p->cap, p->spt,
-                                      step_ticks, total_ticks, step_seconds, total_seconds, bad_step, hits);
+    if (p->dL && !hbc) return KVP_ERR_ARG;
+    finish_kernel<<<n, 256, 0, st>>>(reinterpret_cast<const uint4*>(counts), p->dL ? hbc : nullptr, p->d_stepc, p->K, p->S,
+                                      p->cap, p->spt, step_ticks, total_ticks, step_seconds, total_seconds, bad_step, hits);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }
@@ -302,12 +360,13 @@ static const uint32_t kBatchSlice = 32768;
 extern "C" int kvp_eval_counts(kvp_problem* p, const uint32_t* schedules, uint32_t n, uint32_t* counts, void* stream)
 {
     if (!p || !schedules || !counts || !n) return KVP_ERR_ARG;
+    if (p->dL) return KVP_ERR_ARG;                       // four cardinalities do not describe a growing cache
     if ((reinterpret_cast<uintptr_t>(counts) & 15) != 0) return KVP_ERR_ARG;
     KVP_CUDA(cudaSetDevice(p->device));
     const size_t sched_words = (size_t)p->S * p->W32;
     for (uint32_t i = 0; i < n; i += kBatchSlice) {
         const uint32_t m = n - i < kBatchSlice ? n - i : kBatchSlice;
-        int rc = kvp::launch_counts(p, schedules + i * sched_words, m, counts + (size_t)i * p->S * 4,
+        int rc = kvp::launch_counts(p, schedules + i * sched_words, m, counts + (size_t)i * p->S * 4, nullptr,
                                     static_cast<cudaStream_t>(stream), nullptr);
         if (rc) return rc;
     }
@@ -321,15 +380,16 @@ extern "C" int kvp_eval(kvp_problem* p, const uint32_t* schedules, uint32_t n, u
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t slice = n < kBatchSlice ? n : kBatchSlice;
-    int rc = kvp::ensure_scratch(p, (size_t)slice * p->S * 16, st);
+    int rc = kvp::ensure_scratch(p, (size_t)slice * p->S * 20, st);
     if (rc) return rc;
     uint32_t* counts = static_cast<uint32_t*>(p->d_scratch);
+    uint32_t* hbc = counts + (size_t)slice * p->S * 4;   // used by problems with births only
     const size_t sched_words = (size_t)p->S * p->W32;
     for (uint32_t i = 0; i < n; i += kBatchSlice) {
         const uint32_t m = n - i < kBatchSlice ? n - i : kBatchSlice;
-        if ((rc = kvp::launch_counts(p, schedules + i * sched_words, m, counts, st, nullptr))) return rc;
+        if ((rc = kvp::launch_counts(p, schedules + i * sched_words, m, counts, hbc, st, nullptr))) return rc;
         const size_t so = (size_t)i * p->S;
-        if ((rc = kvp::launch_finish(p, counts, m, step_ticks ? step_ticks + so : nullptr, total_ticks + i,
+        if ((rc = kvp::launch_finish(p, counts, hbc, m, step_ticks ? step_ticks + so : nullptr, total_ticks + i,
                                      step_seconds ? step_seconds + so : nullptr,
                                      total_seconds ? total_seconds + i : nullptr, bad_step ? bad_step + i : nullptr,
                                      nullptr, st)))
@@ -368,7 +428,7 @@ extern "C" int kvp_eval_noalloc(kvp_problem* p, const uint32_t* schedules, uint3
                                 uint64_t* total_ticks, double* step_seconds, double* total_seconds, int32_t* bad_step,
                                 void* stream)
 {
-    if (!p || !schedules || !total_ticks || !n) return KVP_ERR_ARG;
+    if (!p || !schedules || !total_ticks || !n || p->dL) return KVP_ERR_ARG;
     if ((uint64_t)n * p->S * 16ull > (uint64_t)KVP_NOALLOC_SCRATCH_BYTES) return KVP_ERR_RANGE;   // batch too large
     KVP_CUDA(cudaSetDevice(p->device));
     uint32_t* counts = nullptr;
@@ -377,6 +437,7 @@ extern "C" int kvp_eval_noalloc(kvp_problem* p, const uint32_t* schedules, uint3
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array still holds the previous call's numbers. launch_counts either overwrites every entry it
     // owns (narrow rows) or clears them on the stream before accumulating (wide rows).
-    if ((rc = kvp::launch_counts(p, schedules, n, counts, st, nullptr))) return rc;
-    return kvp::launch_finish(p, counts, n, step_ticks, total_ticks, step_seconds, total_seconds, bad_step, nullptr, st);
+    if ((rc = kvp::launch_counts(p, schedules, n, counts, nullptr, st, nullptr))) return rc;
+    return kvp::launch_finish(p, counts, nullptr, n, step_ticks, total_ticks, step_seconds, total_seconds, bad_step, nullptr,
+                              st);
 }

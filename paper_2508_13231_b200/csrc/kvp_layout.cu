@@ -129,6 +129,54 @@ __global__ void row_to_columns_kernel(const uint32_t* __restrict__ row, uint32_t
     }
 }
 
+// Growing cache: row s of L has bit u set iff unit u exists at step s (birth[u] <= s). One thread per word.
+__global__ void alive_rows_kernel(const uint32_t* __restrict__ birth, uint32_t U, uint32_t W32, size_t total,
+                                  uint32_t* __restrict__ L)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const uint32_t s = (uint32_t)(i / W32), u0 = (uint32_t)(i % W32) * 32;
+        uint32_t bits = 0;
+        for (uint32_t b = 0; b < 32 && u0 + b < U; ++b) bits |= (__ldg(birth + u0 + b) <= s ? 1u : 0u) << b;
+        L[i] = bits;
+    }
+}
+
+// Births per step, and the checks of kvp_set_births: flag bit 0 = a birth beyond the horizon, bit 1 = a unit
+// that is accessed before it exists.
+__global__ void birth_stats_kernel(const uint32_t* __restrict__ birth, uint32_t U, uint32_t S,
+                                   const uint32_t* __restrict__ Acol, uint32_t S32, uint32_t* __restrict__ nb,
+                                   uint32_t* __restrict__ flag)
+{
+    const uint32_t u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= U) return;
+    const uint32_t b = birth[u];
+    if (b >= S) { atomicOr(flag, 1u); return; }
+    if (b == 0) return;
+    atomicAdd(nb + b, 1u);
+    uint32_t early = 0;
+    for (uint32_t j = 0; j < (b >> 5); ++j) early |= __ldg(Acol + (size_t)u * S32 + j);
+    if (b & 31u) early |= __ldg(Acol + (size_t)u * S32 + (b >> 5)) & ((1u << (b & 31u)) - 1u);
+    if (early) atomicOr(flag, 2u);
+}
+
+// every unit born in a step is first counted as written to DRAM (see step_cost_g)
+__global__ void stepc_births_kernel(StepC* __restrict__ stepc, const uint32_t* __restrict__ nb, uint32_t S, uint32_t kk,
+                                    uint32_t kd)
+{
+    const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    StepC c = stepc[s];
+    c.y += kk * nb[s];
+    c.z += kd * nb[s];
+    stepc[s] = c;
+}
+
+__global__ void and_rows_kernel(uint32_t* __restrict__ sched, const uint32_t* __restrict__ L, size_t total)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+        sched[i] &= __ldg(L + i);
+}
+
 inline uint32_t grid_for(size_t total, uint32_t block)
 {
     size_t g = (total + block - 1) / block;
@@ -192,6 +240,36 @@ int launch_row_to_columns(const uint32_t* row, uint32_t U, uint32_t S, uint32_t 
 {
     const size_t total = (size_t)U * S32;
     row_to_columns_kernel<<<grid_for(total, 256), 256, 0, st>>>(row, U, S, S32, Pcol);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_alive_rows(const uint32_t* birth, uint32_t U, uint32_t S, uint32_t W32, uint32_t* L, cudaStream_t st)
+{
+    const size_t total = (size_t)S * W32;
+    alive_rows_kernel<<<grid_for(total, 256), 256, 0, st>>>(birth, U, W32, total, L);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_birth_stats(const uint32_t* birth, uint32_t U, uint32_t S, const uint32_t* Acol, uint32_t S32, uint32_t* nb,
+                       uint32_t* flag, cudaStream_t st)
+{
+    birth_stats_kernel<<<(U + 255) / 256, 256, 0, st>>>(birth, U, S, Acol, S32, nb, flag);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_stepc_births(StepC* stepc, const uint32_t* nb, uint32_t S, uint32_t kk, uint32_t kd, cudaStream_t st)
+{
+    stepc_births_kernel<<<(S + 255) / 256, 256, 0, st>>>(stepc, nb, S, kk, kd);
+    KVP_CUDA(cudaGetLastError());
+    return KVP_OK;
+}
+
+int launch_and_rows(uint32_t* sched, const uint32_t* L, size_t total, cudaStream_t st)
+{
+    and_rows_kernel<<<grid_for(total, 256), 256, 0, st>>>(sched, L, total);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }

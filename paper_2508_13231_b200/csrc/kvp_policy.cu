@@ -342,7 +342,7 @@ static size_t policy_smem(uint32_t EW32, uint32_t rounds, uint32_t T)
 
 extern "C" int kvp_policy_reactive(kvp_problem* p, uint32_t init_mode, uint32_t* schedule, void* stream)
 {
-    if (!p || !schedule || init_mode > KVP_INIT_STATIC_FREQ) return KVP_ERR_ARG;
+    if (!p || !schedule || init_mode > KVP_INIT_STATIC_FREQ || p->dL) return KVP_ERR_ARG;   // fixed populations only
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;        // stamps are 16 bits and live in shared memory
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -365,6 +365,7 @@ extern "C" int kvp_policy_reactive(kvp_problem* p, uint32_t init_mode, uint32_t*
 
 extern "C" int kvp_policy_page(kvp_problem* p, uint32_t page_units, uint32_t* schedule, void* stream)
 {
+    if (p && p->dL) return KVP_ERR_ARG;                      // fixed populations only
     if (!p || !schedule || page_units < 2 || page_units > 32 || (page_units & (page_units - 1)) || p->U % page_units)
         return KVP_ERR_ARG;
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;
@@ -386,6 +387,7 @@ extern "C" int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const ui
                                     uint32_t n, uint32_t* schedules, void* stream)
 {
     if (!p || !windows || !ratios_permille || !schedules || !n || init_mode > KVP_INIT_STATIC_FREQ) return KVP_ERR_ARG;
+    if (p->dL) return KVP_ERR_ARG;                           // fixed populations only
     for (uint32_t i = 0; i < n; ++i)
         if (windows[i] < 1 || windows[i] > kMaxWindow || ratios_permille[i] > 1000) return KVP_ERR_ARG;
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;
@@ -418,7 +420,7 @@ extern "C" int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const ui
 
 extern "C" int kvp_wr_grid(kvp_problem* p, uint32_t init_mode, uint32_t w_max, uint32_t n_ratio, uint64_t* table, void* stream)
 {
-    if (!p || !table || w_max < 1 || w_max > kMaxWindow || n_ratio < 2 || n_ratio > 1001) return KVP_ERR_ARG;
+    if (!p || !table || w_max < 1 || w_max > kMaxWindow || n_ratio < 2 || n_ratio > 1001 || p->dL) return KVP_ERR_ARG;
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -17,6 +17,9 @@ struct TraceK {
     const int32_t* base;
     uint32_t* out;
     int aligned;             // n % 32 == 0: whole output words belong to one group
+    uint32_t layers;         // >= 1; step t belongs to token t / layers and layer t % layers
+    uint32_t per_layer;      // groups per layer
+    const uint32_t* birth;   // or null: unit u can be read from step birth[u] on
 };
 
 // Irwin-Hall(8) noise with unit variance in Q16.16: the sum of the eight 16-bit halves of one Philox block, centred
@@ -57,9 +60,10 @@ __device__ __forceinline__ void select_reset(SelectSmem& sm)
 
 // Top-k of one (group, step): the CTA holds the n keys (UPT per thread, unit i = j*T + tid, 0 past n) and sets the
 // bits of the k largest, ties to the lower unit index. select_reset and a barrier come first.
+// topk: how many to pick (at most the number of non-zero keys when zero marks a unit that is not there yet).
 template <int UPT>
-__device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const TraceK& k, uint32_t gbase, uint32_t t,
-                                            SelectSmem& sm)
+__device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const TraceK& k, uint32_t topk, uint32_t gbase,
+                                            uint32_t t, SelectSmem& sm)
 {
     const uint32_t T = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // The k-th largest key lies between the smallest and the largest, so it shares every bit above the highest one
@@ -80,7 +84,7 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
         uint32_t c = 0;
 #pragma unroll
         for (int j = 0; j < UPT; ++j) c += key[j] >= cand ? 1u : 0u;      // slots past n hold key 0 < cand
-        if (block_sum(c, &sm.cnt[31 - bit]) >= k.topk) K = cand;
+        if (block_sum(c, &sm.cnt[31 - bit]) >= topk) K = cand;
     }
     uint32_t cg = 0, ce = 0;
 #pragma unroll
@@ -91,7 +95,7 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
     }
     const uint32_t above = block_sum(cg, &sm.cnt[32]);
     const uint32_t equal = block_sum(ce, &sm.cnt[33]);
-    const uint32_t take = k.topk - above;                    // ties to admit, lowest unit index first
+    const uint32_t take = topk - above;                      // ties to admit, lowest unit index first
     const bool rank_ties = equal != take;
     if (tid == 0) sm.run = 0;
     __syncthreads();
@@ -143,7 +147,8 @@ __device__ __forceinline__ int32_t next_state(const TraceK& k, uint32_t u, uint3
 
 // Fused form: one CTA per group walks the steps; used when the score matrix would not fit the scratch budget.
 // Two CTAs per SM (at most 32 registers per thread): one CTA's barriers in the search hide behind the other's work.
-template <int UPT>
+// GROW: units have birth steps; one that is not there yet gets key 0 and is never picked.
+template <int UPT, bool GROW>
 __global__ void __launch_bounds__(1024, 2)
 trace_kernel(const TraceK k)
 {
@@ -157,20 +162,35 @@ trace_kernel(const TraceK k)
         x[j] = 0;
         b[j] = (i < k.n && k.base) ? __ldg(k.base + gbase + i) : 0;
     }
-    for (uint32_t t = 0; t < k.steps; ++t) {
+    // the group reads at the steps of its layer, one per token
+    const uint32_t layer = g / k.per_layer;
+    uint32_t born[GROW ? UPT : 1];
+    if (GROW) {
+#pragma unroll
+        for (int j = 0; j < (GROW ? UPT : 1); ++j) {
+            const uint32_t i = j * T + tid;
+            born[j] = i < k.n ? __ldg(k.birth + gbase + i) : 0u;
+        }
+    }
+    for (uint32_t tok = 0, t = layer; t < k.steps; ++tok, t += k.layers) {
         select_reset(sm);
-        uint32_t key[UPT];
+        uint32_t key[UPT], here = 0;
 #pragma unroll
         for (int j = 0; j < UPT; ++j) {
             const uint32_t i = j * T + tid;
             key[j] = 0;
             if (i < k.n) {
-                x[j] = next_state(k, gbase + i, t, x[j]);
-                key[j] = (uint32_t)(x[j] + b[j]) ^ 0x80000000u;       // order-preserving map int32 -> uint32
+                x[j] = next_state(k, gbase + i, tok, x[j]);
+                if (!GROW || born[GROW ? j : 0] <= t) {
+                    key[j] = (uint32_t)(x[j] + b[j]) ^ 0x80000000u;   // order-preserving map int32 -> uint32, never 0
+                    ++here;
+                }
             }
         }
         __syncthreads();
-        select_step<UPT>(key, k, gbase, t, sm);
+        uint32_t topk = k.topk;
+        if (GROW) topk = min(topk, block_sum(here, &sm.cnt[34]));
+        select_step<UPT>(key, k, topk, gbase, t, sm);
         __syncthreads();
     }
 }
@@ -206,7 +226,7 @@ trace_select_kernel(const TraceK k, uint32_t U, const int32_t* __restrict__ scor
         key[j] = i < k.n ? (uint32_t)__ldg(scores + (size_t)t * U + gbase + i) ^ 0x80000000u : 0u;
     }
     __syncthreads();
-    select_step<UPT>(key, k, gbase, t, sm);
+    select_step<UPT>(key, k, k.topk, gbase, t, sm);
 }
 
 }  // namespace
@@ -220,6 +240,7 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
     if (!tp || !access_bitmaps || !tp->groups || !tp->units_per_group || !tp->steps || (tp->flags & ~KVP_TRACE_SINGLE_PASS))
         return KVP_ERR_ARG;
     if (!tp->topk || tp->topk > tp->units_per_group) return KVP_ERR_ARG;
+    if (tp->reserved || (tp->layers > 1 && tp->groups % tp->layers)) return KVP_ERR_ARG;
     if (tp->rho_q < 0 || tp->rho_q > 65536 || tp->c_q < 0 || tp->c_q > (1 << 20) || tp->sigma_q < 0 ||
         tp->sigma_q > (1 << 20))
         return KVP_ERR_ARG;
@@ -242,7 +263,11 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
     k.rho_q = tp->rho_q; k.c_q = tp->c_q; k.sigma_q = tp->sigma_q; k.burst_jump = tp->burst_jump;
     k.burst_thr = tp->burst_thr; k.base = tp->base; k.out = access_bitmaps;
     k.aligned = tp->units_per_group % 32 == 0;
-    if (!k.aligned) KVP_CUDA(cudaMemsetAsync(access_bitmaps, 0, (size_t)tp->steps * k.W32 * 4, st));
+    k.layers = tp->layers ? tp->layers : 1u;
+    k.per_layer = tp->groups / k.layers;
+    k.birth = tp->birth;
+    const bool layered = k.layers > 1 || k.birth;        // rows of other layers' steps stay zero
+    if (!k.aligned || layered) KVP_CUDA(cudaMemsetAsync(access_bitmaps, 0, (size_t)tp->steps * k.W32 * 4, st));
     const uint32_t n = tp->units_per_group;
     const int upt = n <= 1024 ? 1 : n <= 2048 ? 2 : n <= 4096 ? 4 : 8;
     uint32_t T = (n + upt - 1) / upt;
@@ -251,7 +276,7 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
     // walks the steps one after the other, could not fill the 148 SMs, and the score matrix fits a 1 GiB scratch.
     // With many groups the fused form is faster (measured: 1.9 vs 3.0 ms on 256 groups, 3.9 vs 6.5 ms on 640).
     const size_t score_bytes = (size_t)U64 * tp->steps * 4;
-    if (tp->groups < 148 && score_bytes <= ((size_t)1 << 30) && !(tp->flags & KVP_TRACE_SINGLE_PASS)) {
+    if (tp->groups < 148 && score_bytes <= ((size_t)1 << 30) && !(tp->flags & KVP_TRACE_SINGLE_PASS) && !layered) {
         int32_t* scores = nullptr;
         KVP_CUDA(cudaMallocAsync(&scores, score_bytes, st));
         trace_scores_kernel<<<(uint32_t)((U64 + 127) / 128), 128, 0, st>>>(k, (uint32_t)U64, scores);
@@ -267,11 +292,20 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
         KVP_CUDA(le);
         return KVP_OK;
     }
-    switch (upt) {
-        case 1: trace_kernel<1><<<tp->groups, T, 0, st>>>(k); break;
-        case 2: trace_kernel<2><<<tp->groups, T, 0, st>>>(k); break;
-        case 4: trace_kernel<4><<<tp->groups, T, 0, st>>>(k); break;
-        default: trace_kernel<8><<<tp->groups, T, 0, st>>>(k); break;
+    if (k.birth) {
+        switch (upt) {
+            case 1: trace_kernel<1, true><<<tp->groups, T, 0, st>>>(k); break;
+            case 2: trace_kernel<2, true><<<tp->groups, T, 0, st>>>(k); break;
+            case 4: trace_kernel<4, true><<<tp->groups, T, 0, st>>>(k); break;
+            default: trace_kernel<8, true><<<tp->groups, T, 0, st>>>(k); break;
+        }
+    } else {
+        switch (upt) {
+            case 1: trace_kernel<1, false><<<tp->groups, T, 0, st>>>(k); break;
+            case 2: trace_kernel<2, false><<<tp->groups, T, 0, st>>>(k); break;
+            case 4: trace_kernel<4, false><<<tp->groups, T, 0, st>>>(k); break;
+            default: trace_kernel<8, false><<<tp->groups, T, 0, st>>>(k); break;
+        }
     }
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;

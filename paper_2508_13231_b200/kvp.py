@@ -23,7 +23,7 @@ NOALLOC_SCRATCH_BYTES = 1 << 20
 EXPORTS = [
     "kvp_create", "kvp_destroy", "kvp_get_info", "kvp_eval", "kvp_eval_counts", "kvp_eval_noalloc", "kvp_accept_table", "kvp_anneal",
     "kvp_anneal_chain_state", "kvp_trace_generate", "kvp_philox4x32_10", "kvp_strerror", "kvp_last_cuda_error",
-    "kvp_policy_lookahead", "kvp_policy_reactive", "kvp_policy_page", "kvp_wr_grid", "kvp_wr_anneal",
+    "kvp_policy_lookahead", "kvp_policy_reactive", "kvp_policy_page", "kvp_wr_grid", "kvp_wr_anneal", "kvp_set_births",
 ]
 
 
@@ -95,6 +95,7 @@ class TraceParams(C.Structure):
         ("groups", C.c_uint32), ("units_per_group", C.c_uint32), ("steps", C.c_uint32), ("topk", C.c_uint32),
         ("seed", C.c_uint64), ("rho_q", C.c_int32), ("c_q", C.c_int32), ("sigma_q", C.c_int32), ("burst_jump", C.c_int32),
         ("burst_thr", C.c_uint32), ("flags", C.c_uint32), ("base", C.c_void_p),
+        ("layers", C.c_uint32), ("reserved", C.c_uint32), ("birth", C.c_void_p),
     ]
 
 
@@ -157,9 +158,16 @@ TRACE_SINGLE_PASS = 1
 
 
 def trace_generate(groups, units_per_group, steps, topk, seed, rho_q, c_q, sigma_q, burst_jump=0, burst_thr=0,
-                   base=None, out=None, stream=None, flags=0):
-    """Synthetic access bitmaps on the current CUDA device -> int32 tensor [steps][ceil(U/32)] (bit pattern uint32)."""
+                   base=None, out=None, stream=None, flags=0, layers=0, birth=None):
+    """Synthetic access bitmaps on the current CUDA device -> int32 tensor [steps][ceil(U/32)] (bit pattern uint32).
+
+    layers: the steps are (token, layer) pairs; birth: int32 CUDA tensor [U] of the steps at which units appear."""
     tp = TraceParams()
+    tp.layers = layers
+    if birth is not None:
+        if birth.numel() != groups * units_per_group:
+            raise ValueError("birth must have one entry per unit")
+        tp.birth = _ptr(birth, torch.int32)
     tp.groups, tp.units_per_group, tp.steps, tp.topk, tp.seed = groups, units_per_group, steps, topk, seed
     tp.rho_q, tp.c_q, tp.sigma_q, tp.burst_jump, tp.burst_thr = rho_q, c_q, sigma_q, burst_jump, burst_thr
     tp.flags = flags
@@ -178,7 +186,7 @@ class Problem:
     """A problem instance (kvp_create). Bitmaps are int32 CUDA tensors holding the uint32 words."""
 
     def __init__(self, units, bytes_per_unit, steps, access, cap, bw_hbm, bw_link, bw_dram, mig_flags=MIG_PAPER,
-                 hw=None, ew=None, stream=None):
+                 hw=None, ew=None, stream=None, birth=None):
         self.units, self.steps, self.cap = int(units), int(steps), int(cap)
         self.w32 = (self.units + 31) // 32
         if access.numel() != self.steps * self.w32:
@@ -190,6 +198,14 @@ class Problem:
         _chk(_lib().kvp_create(C.byref(self._h), C.c_uint32(units), C.c_uint64(bytes_per_unit), C.c_uint32(steps),
                                _ptr(access, torch.int32), C.c_uint32(cap), C.byref(ms), hw_a, ew_a, _stream(stream)),
              "kvp_create")
+        if birth is not None:                                # growing cache (kvp_set_births)
+            if birth.numel() != self.units:
+                self.close()
+                raise ValueError("birth must have one entry per unit")
+            rc = _lib().kvp_set_births(self._h, _ptr(birth, torch.int32), _stream(stream))
+            if rc:
+                self.close()
+                _chk(rc, "kvp_set_births")
         info = Info()
         _chk(_lib().kvp_get_info(self._h, C.byref(info)), "kvp_get_info")
         self.info = info

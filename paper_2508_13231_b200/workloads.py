@@ -50,6 +50,48 @@ CONFIGS = {
 }
 ORDER = ["tiny", "single_head", "layer_8b", "full_8b", "long_70b"]
 
+# Growing caches with (token, layer) steps: `layers` x `heads` groups of `units_per_group` units (one unit = the KV
+# entry of one token in one (layer, kv-head)); the first `prompt` units of every group exist from the start, unit
+# prompt + j is written by decoded token j + 1 at the step of its layer. steps = layers * (units_per_group - prompt + 1).
+GROWING = {
+    "growing_tiny": dict(layers=2, heads=1, units_per_group=12, prompt=4, topk=3, bytes_per_unit=512, cap=6,
+                         bw=(49 * TB // 10, 9 * TB // 10, 5 * TB // 10), rho=0.9, zipf=None,
+                         chains=32, moves=4_000, p0=1e-6),
+    "growing_small": dict(layers=4, heads=2, units_per_group=64, prompt=32, topk=8, bytes_per_unit=512, cap=96,
+                          bw=(8 * TB, 9 * TB // 10, 9 * TB // 10), rho=0.95, zipf=(0.8, 1.4),
+                          chains=256, moves=20_000, p0=1e-6),
+    # the shape of LLaMA-3.1-8B (32 layers, 8 KV heads): 480 prompt tokens, 32 decoded ones
+    "growing_8b": dict(layers=32, heads=8, units_per_group=512, prompt=480, topk=51, bytes_per_unit=512, cap=26214,
+                       bw=(8 * TB, 9 * TB // 10, 9 * TB // 10), rho=0.97, zipf=(0.8, 1.4),
+                       chains=1024, moves=100_000, p0=1e-6),
+}
+
+
+def growing_shape(cfg):
+    """-> (groups, units, steps) of a GROWING configuration."""
+    groups = cfg["layers"] * cfg["heads"]
+    tokens = cfg["units_per_group"] - cfg["prompt"] + 1
+    return groups, groups * cfg["units_per_group"], cfg["layers"] * tokens
+
+
+def growing_births(cfg):
+    """uint32 [U]: 0 for the prompt's units, else the step (token * layers + layer) at which the unit is written."""
+    groups, _, _ = growing_shape(cfg)
+    n, L = cfg["units_per_group"], cfg["layers"]
+    birth = np.zeros((groups, n), np.uint32)
+    for g in range(groups):
+        layer = g // cfg["heads"]
+        j = np.arange(n - cfg["prompt"])
+        birth[g, cfg["prompt"]:] = (j + 1) * L + layer
+    return birth.reshape(-1)
+
+
+def growing_trace_params(name, seed=0):
+    """Trace parameters of a GROWING configuration (pass layers=cfg['layers'] and the births to the generator too)."""
+    cfg = GROWING[name]
+    groups, _, steps = growing_shape(cfg)
+    return custom_trace_params(groups, cfg["units_per_group"], steps, cfg["topk"], cfg["rho"], zipf=cfg["zipf"], seed=seed)
+
 
 def units(cfg):
     return cfg["groups"] * cfg["units_per_group"]

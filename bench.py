@@ -242,6 +242,80 @@ def run_trace_kernel(args):
                      "memory_gbs": (S * W32 * 4 + (U * 4 if base is not None else 0)) / (ms * 1e-3) / 1e9}}))
 
 
+def run_growing(args):
+    """The whole path on a growing cache with (token, layer) steps, configuration growing_8b:
+    layered trace with births -> kvp_create + kvp_set_births -> kvp_eval of 4 schedules -> kvp_anneal.
+
+    The chains' schedules (17 MB each) live in global memory; the oracle is timed on a few chains beside it.
+    """
+    import numpy as np
+    import torch
+    from paper_2508_13231_b200 import kvp, workloads as wl
+    torch.cuda.set_device(0)
+    name = "growing_8b"
+    cfg = wl.GROWING[name]
+    groups, U, S = wl.growing_shape(cfg)
+    birth_np = wl.growing_births(cfg)
+    birth = torch.from_numpy(birth_np.view(np.int32)).cuda()
+    tp = wl.growing_trace_params(name, seed=0)
+    base = torch.from_numpy(tp["base"]).cuda()
+    targs = {k: v for k, v in tp.items() if k not in ("base", "seed")}
+    chains, moves = cfg["chains"], cfg["moves"]
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    g = torch.Generator(device="cuda"); g.manual_seed(3)
+    w32 = (U + 31) // 32
+    scheds = torch.randint(-2 ** 31, 2 ** 31 - 1, (4, S, w32), dtype=torch.int32, device="cuda", generator=g)
+    for _ in range(3):                                        # ~6% density, below the capacity
+        scheds &= torch.randint(-2 ** 31, 2 ** 31 - 1, (4, S, w32), dtype=torch.int32, device="cuda", generator=g)
+
+    def step(seed):
+        A = kvp.trace_generate(**targs, seed=seed, base=base, layers=cfg["layers"], birth=birth)
+        prob = kvp.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"], birth=birth)
+        prob.eval(scheds, want_steps=False)
+        out = prob.anneal(prob.make_params(chains=chains, moves=moves, seed=seed, p0=cfg["p0"]), want_schedule=False)
+        prob.close()
+        return out
+
+    for w in range(max(3, args.warmup)):
+        step(1000 + w)
+    torch.cuda.synchronize()
+    total_ms = chain_ms = 0.0
+    for k in range(args.steps):
+        flush.fill_(k & 255)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        out = step(k)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        total_ms += e0.elapsed_time(e1)
+        chain_ms += out["stats"].ms_chains
+    ms, cms = total_ms / args.steps, chain_ms / args.steps
+    achieved = ALG_WARP_INSTR_PER_MOVE * chains * moves / (cms * 1e-3) / 1e9
+    line = {"metric": METRIC, "value": chains * moves / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": args.steps,
+            "config": {"workload": name, "units": U, "steps": S, "layers": cfg["layers"], "chains": chains, "moves": moves,
+                       "p0": cfg["p0"], "l2": "flushed with a 256 MB write between timed iterations"},
+            "roofline": {"bound": "alu", "kernel": "chain_kernel<global, growing>", "achieved": achieved,
+                         "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
+                         "traffic": None, "ms_per_launch": cms,
+                         "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"},
+            "anneal_ms": {"init": out["stats"].ms_init, "chains": out["stats"].ms_chains, "finish": out["stats"].ms_finish},
+            "bound_ticks": out["best_ticks"], "init_ticks": out["stats"].init_ticks}
+    if not args.no_cpu_baseline:
+        from oracle import kvpo
+        t0 = time.perf_counter()
+        A = kvpo.trace_generate(**targs, seed=0, base=tp["base"], layers=cfg["layers"], birth=birth_np)
+        o = kvpo.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"], birth=birth_np)
+        n = 2
+        res, _, _ = o.anneal_chains(o.make_params(chains=chains, moves=moves, seed=0, p0=cfg["p0"]), 0, n)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": sum(r.moves_done for r in res) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"chains 0..{n - 1} of {chains}, all {moves} moves each, plus trace and "
+                                          f"set-up; {dt:.1f} s on one thread"}
+    print(json.dumps(line))
+
+
 def time_to_bound(kvp, cfg, targs, base_dev, U, S):
     """Outside the timed region: wall time of kvp_anneal (all of its kernels, warm) to reach the bound.
 
@@ -282,8 +356,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="kvp", choices=["kvp", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel", default="path", choices=["path", "cost", "trace"],
-                    help="path: the whole hot path (the benchmark line); cost / trace: that kernel alone on full-size rows")
+    ap.add_argument("--kernel", default="path", choices=["path", "cost", "trace", "growing"],
+                    help="path: the whole hot path (the benchmark line); cost / trace: that kernel alone on full-size rows; "
+                         "growing: the whole path on a growing cache with (token, layer) steps")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -291,6 +366,8 @@ def main():
         return run_cost_kernel(args)
     if args.kernel == "trace":
         return run_trace_kernel(args)
+    if args.kernel == "growing":
+        return run_growing(args)
 
     import numpy as np
     import torch

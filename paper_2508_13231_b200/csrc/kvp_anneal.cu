@@ -350,12 +350,24 @@ __device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint3
     __syncwarp();
 }
 
-__device__ __forceinline__ void copy_words(uint32_t* dst, const uint32_t* src, size_t n, uint32_t lane)
+// One warp copies n words. A chain in global scratch starts by copying tens of megabytes with this one warp, so
+// eight 16-byte loads per lane are in flight before the first store (4 KB per trip instead of 512 bytes).
+__device__ __forceinline__ void copy_words(uint32_t* __restrict__ dst, const uint32_t* __restrict__ src, size_t n,
+                                           uint32_t lane)
 {
     if ((n & 3) == 0 && ((reinterpret_cast<uintptr_t>(dst) | reinterpret_cast<uintptr_t>(src)) & 15) == 0) {
-        uint4* d4 = reinterpret_cast<uint4*>(dst);
-        const uint4* s4 = reinterpret_cast<const uint4*>(src);
-        for (size_t i = lane; i < n / 4; i += 32) d4[i] = s4[i];
+        uint4* __restrict__ d4 = reinterpret_cast<uint4*>(dst);
+        const uint4* __restrict__ s4 = reinterpret_cast<const uint4*>(src);
+        const size_t n4 = n / 4;
+        size_t i = lane;
+        for (; i + 7 * 32 < n4; i += 8 * 32) {
+            uint4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = s4[i + 32 * j];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) d4[i + 32 * j] = v[j];
+        }
+        for (; i < n4; i += 32) d4[i] = s4[i];
     } else {
         for (size_t i = lane; i < n; i += 32) dst[i] = src[i];
     }

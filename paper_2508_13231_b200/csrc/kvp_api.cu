@@ -20,24 +20,35 @@ int set_cuda_error(cudaError_t e, const char* what)
 }
 
 // All device memory comes from the stream-ordered allocator: a create/anneal/destroy cycle then costs no
-// device-wide synchronisation. The default pool is told once per device to keep up to 1 GiB of freed memory.
-static int prepare_pool(int device)
+// device-wide synchronisation. The default pool is told to keep freed memory up to the largest block this
+// library has asked for on the device so far (at least 1 GiB), so that the next problem of the same size
+// gets its workspace back without a trip to the driver.
+static int retain_in_pool(int device, size_t bytes)
 {
-    static bool done[64];
-    if (device < 0 || device >= 64 || done[device]) return KVP_OK;
+    static uint64_t kept[64];                // racing threads may both raise the threshold; either value is fine
+    if (device < 0 || device >= 64) return KVP_OK;
+    uint64_t want = (uint64_t)bytes + (1ull << 30);
+    if (__atomic_load_n(&kept[device], __ATOMIC_RELAXED) >= want) return KVP_OK;
     cudaMemPool_t pool;
     KVP_CUDA(cudaDeviceGetDefaultMemPool(&pool, device));
-    uint64_t keep = 1ull << 30;
-    KVP_CUDA(cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep));
-    done[device] = true;
+    uint64_t now = 0;
+    KVP_CUDA(cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &now));
+    if (now < want) KVP_CUDA(cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &want));
+    __atomic_store_n(&kept[device], want, __ATOMIC_RELAXED);
     return KVP_OK;
 }
+
+static int prepare_pool(int device) { return retain_in_pool(device, 0); }
 
 static int grow(void** ptr, size_t* have, size_t want, cudaStream_t st)
 {
     if (*have >= want) return KVP_OK;
     if (*ptr) { KVP_CUDA(cudaFreeAsync(*ptr, st)); *ptr = nullptr; *have = 0; }
     size_t bytes = (want + 255) & ~(size_t)255;
+    int dev = 0;
+    KVP_CUDA(cudaGetDevice(&dev));
+    int rc = retain_in_pool(dev, bytes);
+    if (rc) return rc;
     KVP_CUDA(cudaMallocAsync(ptr, bytes, st));
     *have = bytes;
     return KVP_OK;

@@ -259,6 +259,11 @@ int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint
  *   stats (host) or NULL; stats->per_chain must be NULL or a host array [chains]
  *   (entry i belongs to chain first_chain + i)
  * Synchronises `stream` before returning.
+ * A job of few chains (at most 8 per SM) is served by two warps per chain that take the chain's batches of 32
+ * proposals in turn; the results are those of the sequential chain either way. The environment variable
+ * KVP_WARPS_PER_CHAIN=1|2 overrides the choice (tuning and tests). The only device-side wait of the library is a
+ * warp's wait for its turn; it is bounded, and a chain whose wait runs out makes the call return KVP_ERR_TIMEOUT
+ * (the outputs are then undefined).
  */
 int kvp_anneal(kvp_problem* p, const kvp_anneal_params* params, uint32_t* best_schedule,
                uint64_t* best_ticks, double* best_seconds, kvp_anneal_stats* stats, void* stream);

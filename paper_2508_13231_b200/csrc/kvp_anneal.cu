@@ -1,15 +1,17 @@
-// Annealing kernels: one chain per warp, lanes spread over the steps a proposal touches.
+// Annealing kernels: one or two warps per chain, one proposal per lane.
 //
 // State of a chain: the schedule in time-packed form (for every unit a bit string over the steps), either
 // in shared memory (small problems) or in a private slice of global scratch, plus the four per-step
-// cardinalities {hr, mi, mo, occ} in shared memory and the running total T in registers.
+// cardinalities {hr, mi, mo, occ} in shared memory and the running total T.
 //
 // A proposal (one Philox4x32-10 block, a pure function of seed, chain and move index) names a run of at most
-// 31 consecutive steps and one or two units. Only the run's steps and the step after it change cost, so
-// lane j re-evaluates step s0 + j with Eq. 2-4 from the counters and a handful of bit reads, the warp sums
-// the differences with one redux, and one thread-uniform Metropolis test against the quantised
-// exp(-delta/C) table decides. Philox blocks are drawn 32 moves at a time, one per lane.
+// 30 consecutive steps and one or two units. Only the run's steps and the step after it change cost. Proposals
+// are drawn and evaluated 32 at a time, one per lane, against the state the batch starts from; the (proposal,
+// step) pairs whose cost changes go through a work queue shared by the warp; the warp then commits the batch in
+// move order with a Metropolis test against the quantised exp(-delta/C) table, evaluating again only what an
+// applied move could have touched. With two warps per chain the warps take the batches in turn (see ChainShare).
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <vector>
@@ -35,6 +37,7 @@ struct ChainParams {
     uint64_t* undo_log;          // if set: [slots][undo_cap] indices of the moves applied since the best state
     uint32_t* undo_len;          // [slots] how many there were (more than undo_cap: the log overflowed)
     uint32_t undo_cap;
+    uint32_t* err;               // set to 1 by a warp that gave up waiting for its turn
     const uint32_t* birth;       // growing cache: [U] step at which a unit is written (0 = there from the start)
     const uint32_t* hb0;         // growing cache: [S] units written to HBM at birth under the initial schedule
     CostK K;
@@ -350,168 +353,346 @@ __device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint3
     __syncwarp();
 }
 
-// One warp copies n words. A chain in global scratch starts by copying tens of megabytes with this one warp, so
-// eight 16-byte loads per lane are in flight before the first store (4 KB per trip instead of 512 bytes).
+// A group of nthr threads (one or more whole warps, this thread being number tid) copies n words. A chain in global
+// scratch starts by copying tens of megabytes this way, so eight 16-byte loads per thread are in flight before the
+// first store.
 __device__ __forceinline__ void copy_words(uint32_t* __restrict__ dst, const uint32_t* __restrict__ src, size_t n,
-                                           uint32_t lane)
+                                           uint32_t tid, uint32_t nthr = 32)
 {
     if ((n & 3) == 0 && ((reinterpret_cast<uintptr_t>(dst) | reinterpret_cast<uintptr_t>(src)) & 15) == 0) {
         uint4* __restrict__ d4 = reinterpret_cast<uint4*>(dst);
         const uint4* __restrict__ s4 = reinterpret_cast<const uint4*>(src);
         const size_t n4 = n / 4;
-        size_t i = lane;
-        for (; i + 7 * 32 < n4; i += 8 * 32) {
+        size_t i = tid;
+        for (; i + 7 * (size_t)nthr < n4; i += 8 * (size_t)nthr) {
             uint4 v[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = s4[i + 32 * j];
+            for (int j = 0; j < 8; ++j) v[j] = s4[i + (size_t)nthr * j];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) d4[i + 32 * j] = v[j];
+            for (int j = 0; j < 8; ++j) d4[i + (size_t)nthr * j] = v[j];
         }
-        for (; i < n4; i += 32) d4[i] = s4[i];
+        for (; i < n4; i += nthr) d4[i] = s4[i];
     } else {
-        for (size_t i = lane; i < n; i += 32) dst[i] = src[i];
+        for (size_t i = tid; i < n; i += nthr) dst[i] = src[i];
     }
 }
 
-template <bool PSMEM, bool GROW>
+// Hand-over block of a chain that is served by more than one warp (shared memory, one per chain).
+// The warps of a chain take the batches in turn: warp w owns batches w, w + W, w + 2W, ... It evaluates a batch
+// against whatever state it finds (another warp may be committing an earlier batch meanwhile), then waits for its
+// turn, evaluates again the proposals that a move applied in the meantime could have touched, and commits. `turn`
+// is the index of the batch whose owner may commit; `napplied` counts the state-changing moves of the chain and
+// `applog` keeps the step ranges of the latest kLog of them. The chain-wide scalars are read and written back only
+// in a turn that applies a move, starts a temperature level or ends the chain; the two counters that change in
+// nearly every batch are kept per warp and added up at the end.
+constexpr uint32_t kLog = 16;
+constexpr int kMaxW = 2;
+struct ChainShare {
+    uint64_t cur, best, best_move, best_at_boundary, n_chg, hash;
+    uint64_t n_acc[kMaxW], n_inf[kMaxW];
+    uint32_t ulen, snap_dirty, stopped, pad;
+    uint32_t turn, napplied, pad2[2];
+    uint32_t applog[kLog];       // s0 | (s0 + len) << 16 of an applied move
+};
+constexpr uint32_t kShareSlots4 = (sizeof(ChainShare) + 15) / 16;
+constexpr uint32_t kPrivSlots4 = kWinSlots4 + kAccSlots4 + kQueueSlots4;   // per warp: windows, sums, work queue
+// A wait for the turn gives up after this many polls (each at least some tens of nanoseconds apart): the chain then
+// reports KVP_ERR_TIMEOUT instead of holding the GPU. A turn lasts microseconds.
+constexpr uint32_t kTurnPolls = 1u << 24;
+
+__device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p) { return *reinterpret_cast<const volatile uint32_t*>(p); }
+__device__ __forceinline__ void st_volatile_u32(uint32_t* p, uint32_t v) { *reinterpret_cast<volatile uint32_t*>(p) = v; }
+
+// shared-memory words (as uint4 slots) of one chain besides its schedule
+__host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool grow, uint32_t W)
+{
+    return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (W > 1 ? kShareSlots4 : 0u) + W * kPrivSlots4;
+}
+
+template <bool PSMEM, bool GROW, int W>
 __global__ void __launch_bounds__(512)
 chain_kernel(const ChainParams prm)
 {
+    static_assert(W >= 1 && W <= kMaxW && (W & (W - 1)) == 0, "warps per chain");
     extern __shared__ uint4 smem4[];
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
-    const uint32_t slot = blockIdx.x * wpb + warp;
-    if (slot >= prm.chain_count) return;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t cpb = (blockDim.x >> 5) / W;                   // chains per CTA
+    const uint32_t cic = warp / W, sub = warp % W;                // chain within the CTA, warp within the chain
+    const uint32_t tid = sub * 32 + lane;                         // thread within the chain
+    const uint32_t slot = blockIdx.x * cpb + cic;
+    const bool active = slot < prm.chain_count;
+    if (W == 1 && !active) return;
     const uint32_t chain = prm.chain_first + slot;
     const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
     const size_t pwords = (size_t)U * S32;
     const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
     const uint32_t h4 = GROW ? (S + 3) / 4 : 0u;                  // uint4 slots of the written-to-HBM counts
-    const uint32_t fixed4 = S + f4 + kWinSlots4 + kAccSlots4 + kQueueSlots4 + h4;   // per-warp shared state besides the schedule
+    const uint32_t fixed4 = chain_fixed4(S, S32, GROW, W);
+    uint4* const mine4 = smem4 + (size_t)cic * fixed4;
     ChainView cv;
-    cv.ctr = smem4 + (size_t)warp * fixed4;
-    cv.full = reinterpret_cast<uint32_t*>(cv.ctr + S);
-    cv.win = cv.ctr + S + f4;
-    cv.acc = reinterpret_cast<int*>(cv.win + kWinSlots4);
-    cv.queue = reinterpret_cast<uint16_t*>(cv.win + kWinSlots4 + kAccSlots4);
-    cv.hb = reinterpret_cast<uint32_t*>(cv.win + kWinSlots4 + kAccSlots4 + kQueueSlots4);
-    cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)wpb * fixed4) + (size_t)warp * pwords
+    cv.ctr = mine4;
+    cv.full = reinterpret_cast<uint32_t*>(mine4 + S);
+    cv.hb = reinterpret_cast<uint32_t*>(mine4 + S + f4);
+    ChainShare* const sh = reinterpret_cast<ChainShare*>(mine4 + S + f4 + h4);
+    uint4* const priv4 = mine4 + S + f4 + h4 + (W > 1 ? kShareSlots4 : 0u) + sub * kPrivSlots4;
+    cv.win = priv4;
+    cv.acc = reinterpret_cast<int*>(priv4 + kWinSlots4);
+    cv.queue = reinterpret_cast<uint16_t*>(priv4 + kWinSlots4 + kAccSlots4);
+    cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)cpb * fixed4) + (size_t)cic * pwords
                  : prm.ws + (size_t)slot * pwords;
-    for (uint32_t i = lane; i < S; i += 32) cv.ctr[i] = __ldg(prm.counters0 + i);
-    for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
-    if (GROW)
-        for (uint32_t i = lane; i < S; i += 32) cv.hb[i] = __ldg(prm.hb0 + i);
-    for (uint32_t i = lane; i < kWinSlots4; i += 32) cv.win[i] = make_uint4(0u, 0u, 0u, 0u);
-    copy_words(cv.P, prm.Pcol0, pwords, lane);
-    __syncwarp();
+    if (active) {
+        for (uint32_t i = tid; i < S; i += 32 * W) cv.ctr[i] = __ldg(prm.counters0 + i);
+        for (uint32_t i = tid; i < S32; i += 32 * W) cv.full[i] = __ldg(prm.full0 + i);
+        if (GROW)
+            for (uint32_t i = tid; i < S; i += 32 * W) cv.hb[i] = __ldg(prm.hb0 + i);
+        for (uint32_t i = lane; i < kWinSlots4; i += 32) cv.win[i] = make_uint4(0u, 0u, 0u, 0u);
+        copy_words(cv.P, prm.Pcol0, pwords, tid, 32 * W);
+        if (W > 1 && tid == 0) {
+            sh->cur = sh->best = sh->best_at_boundary = prm.init_ticks;
+            sh->best_move = ~0ull; sh->n_chg = 0; sh->hash = 0;
+            for (int w = 0; w < kMaxW; ++w) { sh->n_acc[w] = 0; sh->n_inf[w] = 0; }
+            sh->ulen = 0u; sh->snap_dirty = 0u; sh->stopped = 0u; sh->turn = 0u; sh->napplied = 0u;
+        }
+    }
+    if (W > 1) {
+        __syncthreads();
+        if (!active) return;
+    } else {
+        __syncwarp();
+    }
     uint32_t* snap = prm.snap ? prm.snap + (size_t)slot * pwords : nullptr;
-
-    uint64_t cur = prm.init_ticks, best = cur, best_move = ~0ull, best_at_boundary = cur;
-    uint64_t n_acc = 0, n_chg = 0, n_inf = 0, hash = 0;
-    uint32_t level = 0, shift = __ldg(prm.shifts);
-    const uint32_t* trow = prm.table;
-    uint64_t next_boundary = prm.levels > 1 ? prm.per_level : ~0ull;
-    uint64_t m = 0;
-    bool snap_dirty = false;                                      // the best state is the current one, not yet saved
     uint64_t* ulog = prm.undo_log ? prm.undo_log + (size_t)slot * prm.undo_cap : nullptr;
+
+    // Chain-wide scalars. One warp: they live in registers. Several warps: the master copy is in `sh`; a warp
+    // fetches it (`have`) in a turn that needs it and writes it back before it passes the turn on.
+    uint64_t cur = prm.init_ticks, best = cur, best_move = ~0ull, best_at_boundary = cur;
+    uint64_t n_chg = 0, hash = 0;
+    bool snap_dirty = false;                                      // the best state is the current one, not yet saved
     uint32_t ulen = 0;                                            // moves applied since the best state
-    while (m < prm.upto) {
-        if (m == next_boundary) {                                 // a new temperature level starts at this move
-            ++level;
+    uint64_t n_acc = 0, n_inf = 0;                                // this warp's share of the two counters
+    uint32_t napp = 0;                                            // state-changing moves so far (W > 1)
+    bool have = W == 1;
+    auto fetch = [&]() {
+        if (W > 1 && !have) {
+            cur = sh->cur; best = sh->best; best_move = sh->best_move; best_at_boundary = sh->best_at_boundary;
+            n_chg = sh->n_chg; hash = sh->hash; ulen = sh->ulen; snap_dirty = sh->snap_dirty != 0;
+            have = true;
+        }
+    };
+    // Ends this warp's turn for batch b: scalars back to `sh` if they were fetched, then the next batch may commit.
+    auto pass_turn = [&](uint32_t b) {
+        __syncwarp();
+        if (lane == 0) {
+            if (have) {
+                sh->cur = cur; sh->best = best; sh->best_move = best_move; sh->best_at_boundary = best_at_boundary;
+                sh->n_chg = n_chg; sh->hash = hash; sh->ulen = ulen; sh->snap_dirty = snap_dirty ? 1u : 0u;
+            }
+            sh->n_acc[sub] = n_acc; sh->n_inf[sub] = n_inf;
+            __threadfence_block();
+            st_volatile_u32(&sh->turn, b + 1u);
+        }
+        have = false;
+    };
+
+    uint64_t lvl_start = 0, m_end = 0;                            // m_end: moves done when the chain ended
+    uint32_t base = 0;                                            // index of the level's first batch (mod 2^32)
+    bool stop = false;
+    for (uint32_t level = 0; level < prm.levels && lvl_start < prm.upto; ++level) {
+        // a temperature level: its moves in batches of up to 32 * kMPL consecutive moves
+        const uint64_t lvl_end = level + 1 < prm.levels ? min(lvl_start + prm.per_level, prm.upto) : prm.upto;
+        const uint64_t nbat = (lvl_end - lvl_start + kBatch - 1) / kBatch;
+        const uint32_t shift = __ldg(prm.shifts + level);
+        const uint32_t* trow = prm.table + (size_t)level * KVP_TABLE_Q;
+        if (W == 1 && level > 0) {
             if (prm.early_permille && level >= prm.early_from &&
-                (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille)
+                (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille) {
+                stop = true;
+                m_end = lvl_start;
                 break;
+            }
             best_at_boundary = best;
-            shift = __ldg(prm.shifts + level);
-            trow = prm.table + (size_t)level * KVP_TABLE_Q;
-            next_boundary = level + 1 < prm.levels ? next_boundary + prm.per_level : ~0ull;
         }
-        // A batch: up to 32 * kMPL consecutive moves of one temperature level, move m + 32 h + lane in row h of
-        // its lane. Every lane draws and evaluates its own proposals against the current state; the warp then
-        // commits them in move order. A move that changes the schedule invalidates only later moves whose step
-        // windows overlap its own; those are evaluated again before their turn comes, so the outcome is that
-        // of the sequential chain.
-        const uint32_t nb = (uint32_t)min(min((uint64_t)kBatch, prm.upto - m), next_boundary - m);
-        LaneMove mv[kMPL];
-        uint32_t todo[kMPL], need[kMPL];
-#pragma unroll
-        for (int h = 0; h < kMPL; ++h) {
-            uint32_t r[4];
-            const uint64_t mine = m + 32u * h + lane;
-            philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
-            decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv[h]);
-            mv[h].inf = false; mv[h].acc = false; mv[h].chg = false; mv[h].delta = 0;
-            const uint32_t left = nb > 32u * h ? nb - 32u * h : 0u;
-            todo[h] = left >= 32 ? 0xFFFFFFFFu : (1u << left) - 1u;
-            need[h] = todo[h];
-        }
-        for (;;) {
-            uint32_t any_need = 0;
-#pragma unroll
-            for (int h = 0; h < kMPL; ++h) any_need |= need[h];
-            if (any_need) eval_batch<GROW>(cv, prm.Acol, prm.birth, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
-            bool applied = false;
-#pragma unroll
-            for (int h = 0; h < kMPL; ++h) need[h] = 0;
+        // A batch: move m + 32 h + lane in row h of its lane. Every lane draws and evaluates its own proposals
+        // against the current state; the warp then commits them in move order. A move that changes the schedule
+        // invalidates only later moves whose step windows overlap its own; those are evaluated again before their
+        // turn comes, so the outcome is that of the sequential chain.
+        for (uint64_t bi = (sub - base) & (W - 1); bi < nbat; bi += W) {
+            const uint64_t m = lvl_start + bi * kBatch;
+            const uint32_t nb = (uint32_t)min((uint64_t)kBatch, lvl_end - m);
+            const uint32_t b = base + (uint32_t)bi;
+            uint32_t n0 = 0;
+            if (W > 1) {
+                // Moves applied from now on may be half visible to the reads below: they are checked for at the turn.
+                n0 = __shfl_sync(0xFFFFFFFFu, ld_volatile_u32(&sh->napplied), 0);
+                __threadfence_block();
+            }
+            LaneMove mv[kMPL];
+            uint32_t todo[kMPL], need[kMPL];
 #pragma unroll
             for (int h = 0; h < kMPL; ++h) {
-                if (applied || !todo[h]) continue;
-                const uint32_t infb = __ballot_sync(0xFFFFFFFFu, mv[h].inf);
-                const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !mv[h].inf && mv[h].acc);
-                const uint32_t blk = __ballot_sync(0xFFFFFFFFu, !mv[h].inf && mv[h].acc && mv[h].chg) & todo[h];
-                if (!blk) {                                       // nothing in this row changes the schedule
-                    n_inf += __popc(infb & todo[h]);
-                    n_acc += __popc(accb & todo[h]);
-                    todo[h] = 0;
-                    continue;
-                }
-                const uint32_t b = __ffs(blk) - 1;
-                const uint32_t done = todo[h] & (0xFFFFFFFFu >> (31 - b));   // the row's moves up to and including b
-                n_inf += __popc(infb & done);
-                n_acc += __popc(accb & done);
-                ++n_chg;
-                const int delta = __shfl_sync(0xFFFFFFFFu, mv[h].delta, b);
-                const uint32_t pk = __shfl_sync(0xFFFFFFFFu, mv[h].pk, b);
-                const uint32_t bu = __shfl_sync(0xFFFFFFFFu, mv[h].u, b), bv = __shfl_sync(0xFFFFFFFFu, mv[h].v, b);
-                const uint64_t after = (uint64_t)((int64_t)cur + delta);
-                if (snap && snap_dirty && after >= best) {        // leaving the best state: save it first
-                    copy_words(snap, cv.P, pwords, lane);
-                    snap_dirty = false;
-                }
-                apply_move<GROW>(cv, S, S32, prm.cap, lane, h * 32 + b, pk, bu, bv);
-                cur = after;
-                const uint64_t mb = m + 32u * h + b;
-                hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
-                if (cur < best) { best = cur; best_move = mb; snap_dirty = true; ulen = 0; }
-                else if (ulog) {                                  // every move is its own inverse: remember it
-                    if (ulen < prm.undo_cap && lane == 0) ulog[ulen] = mb;
-                    if (ulen <= prm.undo_cap) ++ulen;
-                }
-                todo[h] &= ~done;
-                // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later proposal
-                // read steps s0 - 1 .. s0 + len: it has to be evaluated again iff the two ranges meet.
-                const uint32_t s0b = pk >> 8, endb = s0b + ((pk >> 1) & 63u);
-#pragma unroll
-                for (int h2 = 0; h2 < kMPL; ++h2) {
-                    const uint32_t s0 = mv[h2].pk >> 8, end = s0 + ((mv[h2].pk >> 1) & 63u);
-                    need[h2] = __ballot_sync(0xFFFFFFFFu, s0 <= endb + 1 && s0b <= end) & todo[h2];
-                }
-                applied = true;
+                uint32_t r[4];
+                const uint64_t mine = m + 32u * h + lane;
+                philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
+                decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv[h]);
+                mv[h].inf = false; mv[h].acc = false; mv[h].chg = false; mv[h].delta = 0;
+                const uint32_t left = nb > 32u * h ? nb - 32u * h : 0u;
+                todo[h] = left >= 32 ? 0xFFFFFFFFu : (1u << left) - 1u;
+                need[h] = todo[h];
             }
-            if (!applied) break;
+            eval_batch<GROW>(cv, prm.Acol, prm.birth, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+#pragma unroll
+            for (int h = 0; h < kMPL; ++h) need[h] = 0;
+            if (W > 1) {
+                // wait for the turn
+                uint32_t polls = 0, t;
+                for (;;) {
+                    t = __shfl_sync(0xFFFFFFFFu, ld_volatile_u32(&sh->turn), 0);
+                    if (t == b || ++polls > kTurnPolls) break;
+                    __nanosleep(64);
+                }
+                __threadfence_block();
+                if (t != b) {                                     // gave up: flag it, let the others pass, leave
+                    if (lane == 0) {
+                        atomicExch(prm.err, 1u);
+                        st_volatile_u32(&sh->stopped, 2u);
+                        __threadfence_block();
+                        st_volatile_u32(&sh->turn, b + 1u);
+                    }
+                    return;
+                }
+                if (ld_volatile_u32(&sh->stopped)) {              // the chain has ended: pass the turn on and leave
+                    __syncwarp();
+                    if (lane == 0) st_volatile_u32(&sh->turn, b + 1u);
+                    return;
+                }
+                napp = sh->napplied;
+                // proposals whose steps meet those of a move applied since this batch was evaluated
+                if (napp - n0 > kLog) {
+#pragma unroll
+                    for (int h = 0; h < kMPL; ++h) need[h] = todo[h];
+                } else {
+                    for (uint32_t k = n0; k != napp; ++k) {
+                        const uint32_t e = sh->applog[k % kLog], s0b = e & 0xFFFFu, endb = e >> 16;
+#pragma unroll
+                        for (int h = 0; h < kMPL; ++h) {
+                            const uint32_t s0 = mv[h].pk >> 8, end = s0 + ((mv[h].pk >> 1) & 63u);
+                            need[h] |= __ballot_sync(0xFFFFFFFFu, s0 <= endb + 1 && s0b <= end) & todo[h];
+                        }
+                    }
+                }
+                if (bi == 0 && level > 0) {                       // the level's first batch: stop rule, new reference
+                    fetch();
+                    if (prm.early_permille && level >= prm.early_from &&
+                        (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille) {
+                        stop = true;
+                        m_end = lvl_start;
+                        break;
+                    }
+                    best_at_boundary = best;
+                }
+            }
+            for (;;) {
+                uint32_t any_need = 0;
+#pragma unroll
+                for (int h = 0; h < kMPL; ++h) any_need |= need[h];
+                if (any_need)
+                    eval_batch<GROW>(cv, prm.Acol, prm.birth, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+                bool applied = false;
+#pragma unroll
+                for (int h = 0; h < kMPL; ++h) need[h] = 0;
+#pragma unroll
+                for (int h = 0; h < kMPL; ++h) {
+                    if (applied || !todo[h]) continue;
+                    const uint32_t infb = __ballot_sync(0xFFFFFFFFu, mv[h].inf);
+                    const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !mv[h].inf && mv[h].acc);
+                    const uint32_t blk = __ballot_sync(0xFFFFFFFFu, !mv[h].inf && mv[h].acc && mv[h].chg) & todo[h];
+                    if (!blk) {                                   // nothing in this row changes the schedule
+                        n_inf += __popc(infb & todo[h]);
+                        n_acc += __popc(accb & todo[h]);
+                        todo[h] = 0;
+                        continue;
+                    }
+                    const uint32_t bb = __ffs(blk) - 1;
+                    const uint32_t done = todo[h] & (0xFFFFFFFFu >> (31 - bb));  // the row's moves up to and including bb
+                    n_inf += __popc(infb & done);
+                    n_acc += __popc(accb & done);
+                    fetch();
+                    ++n_chg;
+                    const int delta = __shfl_sync(0xFFFFFFFFu, mv[h].delta, bb);
+                    const uint32_t pk = __shfl_sync(0xFFFFFFFFu, mv[h].pk, bb);
+                    const uint32_t bu = __shfl_sync(0xFFFFFFFFu, mv[h].u, bb), bv = __shfl_sync(0xFFFFFFFFu, mv[h].v, bb);
+                    const uint64_t after = (uint64_t)((int64_t)cur + delta);
+                    if (snap && snap_dirty && after >= best) {    // leaving the best state: save it first
+                        copy_words(snap, cv.P, pwords, lane);
+                        snap_dirty = false;
+                    }
+                    apply_move<GROW>(cv, S, S32, prm.cap, lane, h * 32 + bb, pk, bu, bv);
+                    // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later
+                    // proposal read steps s0 - 1 .. s0 + len: it has to be evaluated again iff the two ranges meet.
+                    const uint32_t s0b = pk >> 8, endb = s0b + ((pk >> 1) & 63u);
+                    if (W > 1) {                                  // tell the warps that are evaluating later batches
+                        if (lane == 0) {
+                            sh->applog[napp % kLog] = s0b | (endb << 16);
+                            __threadfence_block();
+                            st_volatile_u32(&sh->napplied, napp + 1u);
+                        }
+                        ++napp;
+                    }
+                    cur = after;
+                    const uint64_t mb = m + 32u * h + bb;
+                    hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
+                    if (cur < best) { best = cur; best_move = mb; snap_dirty = true; ulen = 0; }
+                    else if (ulog) {                              // every move is its own inverse: remember it
+                        if (ulen < prm.undo_cap && lane == 0) ulog[ulen] = mb;
+                        if (ulen <= prm.undo_cap) ++ulen;
+                    }
+                    todo[h] &= ~done;
+#pragma unroll
+                    for (int h2 = 0; h2 < kMPL; ++h2) {
+                        const uint32_t s0 = mv[h2].pk >> 8, end = s0 + ((mv[h2].pk >> 1) & 63u);
+                        need[h2] = __ballot_sync(0xFFFFFFFFu, s0 <= endb + 1 && s0b <= end) & todo[h2];
+                    }
+                    applied = true;
+                }
+                if (!applied) break;
+            }
+            m_end = m + nb;
+            if (W > 1 && m_end < prm.upto) pass_turn(b);          // hand the chain to the owner of the next batch
         }
-        m += nb;
+        if (stop) break;                                          // `base` stays the index of the batch that stopped
+        base += (uint32_t)nbat;
+        lvl_start = lvl_end;
+    }
+    // The warp that committed the last batch, or that ended the chain by the stop rule, reports.
+    if (W > 1) {
+        const bool writer = stop || (base ? ((base - 1u) & (W - 1)) == sub : sub == 0);
+        if (!writer) return;
+        fetch();
+        sh->n_acc[sub] = n_acc; sh->n_inf[sub] = n_inf;           // all lanes write the same values
+        __syncwarp();
+        n_acc = 0; n_inf = 0;
+        for (int w = 0; w < W; ++w) { n_acc += sh->n_acc[w]; n_inf += sh->n_inf[w]; }
+        if (!stop) m_end = prm.upto < lvl_start ? prm.upto : lvl_start;
     }
     if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
     if (ulog && lane == 0) prm.undo_len[slot] = ulen;
     if (lane == 0) {
         kvp_chain_result res;
-        res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m;
+        res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m_end;
         res.n_accepted = n_acc; res.n_changed = n_chg; res.n_infeasible = n_inf; res.traj_hash = hash;
         prm.results[chain - prm.result_base] = res;
     }
     if (prm.dump && slot == 0) {
         __syncwarp();
         copy_words(prm.dump, cv.P, pwords, lane);
+    }
+    if (W > 1 && stop) {                                          // ended by the stop rule: release the next owner
+        __syncwarp();
+        if (lane == 0) {
+            st_volatile_u32(&sh->stopped, 1u);
+            __threadfence_block();
+            st_volatile_u32(&sh->turn, base + 1u);
+        }
     }
 }
 
@@ -590,12 +771,12 @@ calib_kernel(const ChainParams prm, unsigned long long* acc)
 
 struct ReduceOut {
     uint64_t best_ticks, best_move, moves_total;
-    uint32_t best_chain, pad;
+    uint32_t best_chain, pad;    // pad: the chains' error word
 };
 
 // Cross-chain best-so-far: lexicographic minimum of (best_ticks, chain index), plus the executed-move total.
 __global__ void __launch_bounds__(1024)
-reduce_kernel(const kvp_chain_result* __restrict__ res, uint32_t chains, ReduceOut* out)
+reduce_kernel(const kvp_chain_result* __restrict__ res, uint32_t chains, const uint32_t* __restrict__ err, ReduceOut* out)
 {
     __shared__ uint64_t s_t[32], s_m[32];
     __shared__ uint32_t s_c[32];
@@ -623,7 +804,7 @@ reduce_kernel(const kvp_chain_result* __restrict__ res, uint32_t chains, ReduceO
         }
         out->best_ticks = bt; out->best_chain = bc; out->moves_total = moves;
         out->best_move = res[bc].best_move;
-        out->pad = 0;
+        out->pad = *err;                                  // a chain gave up waiting for its turn
     }
 }
 
@@ -651,7 +832,8 @@ struct Ctx {
     uint32_t* undo_len;
     uint32_t undo_cap;
     bool psmem;
-    uint32_t wpb;            // warps per CTA
+    uint32_t wpb;            // chains per CTA
+    uint32_t wpc;            // warps per chain
     uint32_t resident;       // chains per wave
     size_t smem_per_warp;
     std::vector<double> temps;
@@ -672,17 +854,20 @@ int validate(const kvp_problem* p, const kvp_anneal_params* a)
 
 typedef void (*ChainKernel)(const ChainParams);
 
-ChainKernel chain_kernel_for(bool psmem, bool grow)
+ChainKernel chain_kernel_for(bool psmem, bool grow, uint32_t W)
 {
-    return psmem ? (grow ? chain_kernel<true, true> : chain_kernel<true, false>)
-                 : (grow ? chain_kernel<false, true> : chain_kernel<false, false>);
+    if (W == 2)
+        return psmem ? (grow ? chain_kernel<true, true, 2> : chain_kernel<true, false, 2>)
+                     : (grow ? chain_kernel<false, true, 2> : chain_kernel<false, false, 2>);
+    return psmem ? (grow ? chain_kernel<true, true, 1> : chain_kernel<true, false, 1>)
+                 : (grow ? chain_kernel<false, true, 1> : chain_kernel<false, false, 1>);
 }
 
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 {
     const uint32_t grid = (count + c.wpb - 1) / c.wpb;
     const size_t smem = (size_t)c.wpb * c.smem_per_warp;
-    chain_kernel_for(c.psmem, c.grow)<<<grid, c.wpb * 32, smem, c.st>>>(prm);
+    chain_kernel_for(c.psmem, c.grow, c.wpc)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }
@@ -715,32 +900,44 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     KVP_CUDA(cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     KVP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const size_t budget = (size_t)smem_max - 1024;
-    // per warp: counters, full-step bitmap, the batch's windows, accumulators and work queue
+    // per chain: counters, full-step bitmap and, per warp, the batch's windows, accumulators and work queue
     c.grow = p->dL != nullptr;
-    const size_t ctr_bytes = ((size_t)p->S + (p->S32 + 3) / 4 + kWinSlots4 + kAccSlots4 + kQueueSlots4 +
-                              (c.grow ? (p->S + 3) / 4 : 0)) * 16;
-    const size_t psmem_per_warp = ctr_bytes + (size_t)p->U * p->S32 * 4;
-    c.psmem = psmem_per_warp <= budget / 2;
+    auto fixed_bytes = [&](uint32_t W) { return (size_t)chain_fixed4(p->S, p->S32, c.grow, W) * 16; };
+    const size_t pbytes = (size_t)p->U * p->S32 * 4;
+    // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
+    // chains then keeps twice as many warps in flight. KVP_WARPS_PER_CHAIN=1|2 overrides the choice (for tuning).
+    const uint32_t chains_per_sm = (a->chains + sms - 1) / sms;
+    uint32_t W = chains_per_sm <= 8 ? 2u : 1u;
+    if (const char* e = getenv("KVP_WARPS_PER_CHAIN")) {
+        if (e[0] == '1' && !e[1]) W = 1;
+        if (e[0] == '2' && !e[1]) W = 2;
+    }
+    c.psmem = fixed_bytes(1) + pbytes <= budget / 2;
     if (c.psmem) {
-        c.smem_per_warp = psmem_per_warp;
-        uint32_t wmax = (uint32_t)(budget / psmem_per_warp);
-        if (wmax > 16) wmax = 16;
-        uint32_t want = (a->chains + sms - 1) / sms;
-        c.wpb = want < 1 ? 1 : (want > wmax ? wmax : want);
+        uint32_t want = chains_per_sm < 1 ? 1 : chains_per_sm;
+        if (W == 2 && (want > 8 || (fixed_bytes(2) + pbytes) * want > budget) && (fixed_bytes(1) + pbytes) * want <= budget)
+            W = 1;                                                 // the second warp's work area does not fit
+        c.smem_per_warp = fixed_bytes(W) + pbytes;
+        uint32_t wmax = (uint32_t)(budget / c.smem_per_warp);
+        if (wmax > 16 / W) wmax = 16 / W;
+        c.wpb = want > wmax ? wmax : want;
+        c.wpc = W;
         c.resident = a->chains;
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.grow), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
+        const size_t ctr_bytes = fixed_bytes(W);
         if (ctr_bytes > budget) return KVP_ERR_RANGE;
         c.smem_per_warp = ctr_bytes;
-        uint32_t wmax = (uint32_t)(budget / 2 / ctr_bytes);
-        c.wpb = wmax < 1 ? 1 : (wmax > 16 ? 16 : wmax);
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, c.grow), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        c.wpc = W;
+        uint32_t wcap = (uint32_t)(budget / ctr_bytes);            // chains per CTA at most
+        if (wcap > 16 / W) wcap = 16 / W;
+        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
         int ctas = 0;
-        KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, c.grow), (int)c.wpb * 32,
-                                                               c.wpb * c.smem_per_warp));
+        KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, c.grow, W), (int)(wcap * W * 32),
+                                                               wcap * c.smem_per_warp));
         if (ctas < 1) return KVP_ERR_RANGE;
-        uint32_t per_sm = (uint32_t)ctas * c.wpb;                  // resident chains per SM, at most 32
-        if (per_sm > 32) per_sm = 32 / c.wpb ? 32 / c.wpb * c.wpb : c.wpb;
+        uint32_t per_sm = (uint32_t)ctas * wcap;                   // resident chains per SM, at most 32 warps
+        if (per_sm * W > 32) per_sm = 32 / W / wcap ? 32 / W / wcap * wcap : wcap;
         size_t free_b = 0, total_b = 0;
         KVP_CUDA(cudaMemGetInfo(&free_b, &total_b));
         free_b += p->chain_ws_bytes;                               // what we already hold can be reused
@@ -759,6 +956,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
         if (r > fit) r = fit;
         const uint32_t waves = (uint32_t)((a->chains + r - 1) / r);
         c.resident = (a->chains + waves - 1) / waves;              // equal waves
+        // a wave is spread over all SMs: CTAs of ceil(resident / SMs) chains where one CTA per SM holds them
+        const uint32_t even = (c.resident + sms - 1) / sms;
+        c.wpb = even < wcap ? even : wcap;
     }
 
     // workspace layout
@@ -827,6 +1027,8 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     prm.Acol = p->dAcol; prm.stepc = p->d_stepc; prm.counters0 = (const uint4*)c.counts0; prm.Pcol0 = c.Pcol0;
     prm.table = c.table; prm.shifts = c.shifts; prm.ws = c.slots; prm.K = p->K; prm.full0 = c.full0;
     prm.birth = p->d_birth; prm.hb0 = c.hb0;
+    prm.err = reinterpret_cast<uint32_t*>(c.small + 16);
+    KVP_CUDA(cudaMemsetAsync(prm.err, 0, 4, st));
     prm.U = p->U; prm.S = p->S; prm.S32 = p->S32; prm.cap = p->cap;
     prm.levels = a->levels; prm.p_swap_256 = a->p_swap_256; prm.len_choices = a->max_len_log2 + 1;
     prm.early_permille = a->early_stop_permille; prm.early_from = a->early_stop_from_level;
@@ -917,11 +1119,12 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
         if (c.undo_log) {
             // Best so far over the chains that have finished; if it belongs to this wave, walk that chain back to
             // its best state while its scratch slice still holds its final state.
-            reduce_kernel<<<1, 1024, 0, st>>>(c.results, first + count, red_dev);
+            reduce_kernel<<<1, 1024, 0, st>>>(c.results, first + count, c.prm.err, red_dev);
             KVP_CUDA(cudaGetLastError());
             ++c.launches;
             KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
             KVP_CUDA(cudaStreamSynchronize(st));
+            if (red.pad) { cleanup(); return KVP_ERR_TIMEOUT; }
             if (red.best_chain >= first && red.best_move != ~0ull) {
                 uint32_t len = 0;
                 KVP_CUDA(cudaMemcpyAsync(&len, c.undo_len + (red.best_chain - first), 4, cudaMemcpyDeviceToHost, st));
@@ -944,11 +1147,12 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     // cross-chain reduction, then the winner's schedule (its own snapshot, its walked-back state, or a replay) and a
     // re-score
     if (!c.undo_log) {
-        reduce_kernel<<<1, 1024, 0, st>>>(c.results, a->chains, red_dev);
+        reduce_kernel<<<1, 1024, 0, st>>>(c.results, a->chains, c.prm.err, red_dev);
         KVP_CUDA(cudaGetLastError());
         ++c.launches;
         KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
         KVP_CUDA(cudaStreamSynchronize(st));
+        if (red.pad) { cleanup(); return KVP_ERR_TIMEOUT; }
     }
     const uint64_t upto = red.best_move == ~0ull ? 0 : red.best_move + 1;
     if (upto && (c.snap || dumped_chain == red.best_chain)) {
@@ -1014,6 +1218,8 @@ extern "C" int kvp_anneal_chain_state(kvp_problem* p, const kvp_anneal_params* a
     if ((rc = replay_to_sched(p, c, chain, upto_moves, res_dev))) return rc;
     KVP_CUDA(cudaMemcpyAsync(schedule, c.sched, (size_t)p->S * p->W32 * 4, cudaMemcpyDeviceToDevice, st));
     if (result) KVP_CUDA(cudaMemcpyAsync(result, res_dev, sizeof *result, cudaMemcpyDeviceToHost, st));
+    uint32_t gave_up = 0;
+    KVP_CUDA(cudaMemcpyAsync(&gave_up, c.prm.err, 4, cudaMemcpyDeviceToHost, st));
     KVP_CUDA(cudaStreamSynchronize(st));
-    return KVP_OK;
+    return gave_up ? KVP_ERR_TIMEOUT : KVP_OK;
 }

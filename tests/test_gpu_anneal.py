@@ -20,6 +20,13 @@ def kvp():
     return kvp
 
 
+@pytest.fixture(params=["1", "2"])
+def warps_per_chain(request, monkeypatch):
+    """Both forms of the chain kernel: one warp per chain, and two warps that take a chain's batches in turn."""
+    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", request.param)
+    return int(request.param)
+
+
 def _params(g, o, **kw):
     return g.make_params(**kw), o.make_params(**kw)
 
@@ -43,7 +50,7 @@ def _check_against_oracle(g, o, gp, op, chains_to_check=None, check_schedule=Tru
     return out
 
 
-def test_anneal_tiny_all_chains(kvp, oracle):
+def test_anneal_tiny_all_chains(kvp, oracle, warps_per_chain):
     g, o, cfg, A = named_problem(kvp, oracle, "tiny")
     for p0 in (0.8, 1e-3):
         gp, op = _params(g, o, chains=cfg["chains"], moves=cfg["moves"], seed=0, p0=p0)
@@ -60,7 +67,7 @@ def test_anneal_tiny_all_chains(kvp, oracle):
     (200, 130, 37, (4900, 500, 900), 2),    # link slower than DRAM, migrations free on the HBM side
     (90, 33, 20, (3, 1, 1), 0),             # free migration
 ])
-def test_anneal_small_shapes(kvp, oracle, U, S, cap, bw, flags):
+def test_anneal_small_shapes(kvp, oracle, U, S, cap, bw, flags, warps_per_chain):
     A = wl.random_access(U, S, 0.3, seed=U + S)
     hw = (np.arange(S) % 2).astype(np.uint32)
     ew = (np.arange(S) % 3).astype(np.uint32)
@@ -71,7 +78,7 @@ def test_anneal_small_shapes(kvp, oracle, U, S, cap, bw, flags):
         _check_against_oracle(g, o, gp, op)
 
 
-def test_anneal_options(kvp, oracle):
+def test_anneal_options(kvp, oracle, warps_per_chain):
     U, S, cap = 120, 70, 30
     A = wl.random_access(U, S, 0.25, seed=3)
     g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
@@ -178,7 +185,7 @@ def test_anneal_full_size_sampled_chains(kvp, oracle, name, chains, moves):
     assert out["best_ticks"] <= out["stats"].init_ticks
 
 
-def test_global_state_winner_paths(kvp, oracle):
+def test_global_state_winner_paths(kvp, oracle, warps_per_chain):
     # chains in global scratch rebuild the winner by walking its logged moves back; check the three ways this can go:
     # a short log, a log that overflows (hot start: thousands of applied moves after the best; falls back to a replay),
     # and a winner from an earlier wave of a run with more chains than are resident at once

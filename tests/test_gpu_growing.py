@@ -17,6 +17,13 @@ def kvp():
     return kvp
 
 
+@pytest.fixture(params=["1", "2"])
+def warps_per_chain(request, monkeypatch):
+    """Both forms of the chain kernel: one warp per chain, and two warps that take a chain's batches in turn."""
+    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", request.param)
+    return int(request.param)
+
+
 def _birth_dev(birth):
     return torch.from_numpy(np.ascontiguousarray(birth, np.uint32).view(np.int32)).cuda()
 
@@ -174,7 +181,7 @@ def test_anneal_growing_named(kvp, oracle, name):
         assert out["stats"].init_ticks == o.eval(o.init_placement(init))["total_ticks"]
 
 
-def test_anneal_growing_odd_shapes_and_options(kvp, oracle):
+def test_anneal_growing_odd_shapes_and_options(kvp, oracle, warps_per_chain):
     cfg, groups, U, S, birth = _shape(3, 1, 45, 20)
     rng = np.random.default_rng(4)
     alive = birth[None, :] <= np.arange(S)[:, None]
@@ -196,7 +203,7 @@ def test_anneal_growing_odd_shapes_and_options(kvp, oracle):
     assert res.astuple() == want[0].astuple() and np.array_equal(to_np(sched), fin[0])
 
 
-def test_anneal_growing_global_state(kvp, oracle):
+def test_anneal_growing_global_state(kvp, oracle, warps_per_chain):
     """A schedule too large for shared memory: chains in global scratch, the winner walked back through its undo log."""
     cfg, groups, U, S, birth = _shape(4, 4, 256, 200)
     tp = wl.custom_trace_params(groups, 256, S, 24, rho=0.95, zipf=(0.8, 1.4), seed=2)

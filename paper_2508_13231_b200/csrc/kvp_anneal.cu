@@ -57,7 +57,10 @@ constexpr int kMPL = 1;
 constexpr uint32_t kBatch = 32 * kMPL;
 constexpr uint32_t kWinSlots4 = kBatch * 2;                        // 8 words of windows per proposal
 constexpr uint32_t kAccSlots4 = kBatch / 4;                        // one int per proposal
-constexpr uint32_t kQueueSlots4 = (kBatch * 31 * 2 + 15) / 16;     // uint16 work items, worst case 31 per proposal
+// uint16 work items; 31 per proposal in the worst case, so the queue holds the worst case of half a warp's proposals
+// and a batch with more items than that is worked off in two halves
+constexpr uint32_t kQueueCap = kBatch * 31 / 2;
+constexpr uint32_t kQueueSlots4 = (kQueueCap * 2 + 15) / 16;
 
 // A proposal as its lane keeps it in registers: the Philox words and, after evaluation, the verdict.
 // The placement windows live in shared memory (ChainView::win), 8 words per proposal:
@@ -222,7 +225,7 @@ __device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ A
 // prepares its own proposals, the (proposal, step) pairs whose cost changes are queued in shared memory, and
 // the warp works the queue off 32 pairs at a time, so that lanes with short and long proposals carry the
 // same load.
-template <bool GROW>
+template <bool GROW, bool ASMEM>
 __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* __restrict__ Acol,
                                            const uint32_t* __restrict__ birth,
                                            const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
@@ -252,42 +255,53 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         pos += __popc(has & below) << bit;
         total += __popc(has) << bit;
     }
-    // queue the set bits of every mask; all 31 positions are tried so that no lane waits on a serial bit scan
+    // The queue holds kQueueCap items, the worst case of 16 lanes. A batch with more (rare) goes in two halves,
+    // lanes 0..15 first.
+    const uint32_t halves = total > kQueueCap ? 2u : 1u;
+    const uint32_t mid = halves > 1 ? __shfl_sync(0xFFFFFFFFu, pos, 16) : 0u;   // items of lanes 0..15
+    for (uint32_t half = 0; half < halves; ++half) {
+        const bool pushing = halves == 1 || (lane >> 4) == half;
+        const uint32_t first = half ? mid : 0u;                                  // queue position 0 is item `first`
+        const uint32_t count = halves == 1 ? total : (half ? total - mid : mid);
+        if (half) __syncwarp();
+        // queue the set bits of every mask; all 31 positions are tried so that no lane waits on a serial bit scan
 #pragma unroll
-    for (int h = 0; h < kMPL; ++h) {
-        const uint32_t td = todo[h];
-        if (__any_sync(0xFFFFFFFFu, td != 0)) {
+        for (int h = 0; h < kMPL; ++h) {
+            const uint32_t td = pushing ? todo[h] : 0u;
+            if (__any_sync(0xFFFFFFFFu, td != 0)) {
 #pragma unroll
-            for (uint32_t k = 1; k < 32; ++k) {
-                const uint32_t bit = (td >> k) & 1u;
-                if (bit) cv.queue[pos] = (uint16_t)(((h * 32 + lane) << 5) | k);
-                pos += bit;
+                for (uint32_t k = 1; k < 32; ++k) {
+                    const uint32_t bit = (td >> k) & 1u;
+                    if (bit) cv.queue[pos - first] = (uint16_t)(((h * 32 + lane) << 5) | k);
+                    pos += bit;
+                }
             }
         }
-    }
-    __syncwarp();
-    // two items per lane and trip: the two evaluations are independent and overlap
-    for (uint32_t base = 0; base < total; base += 64) {
-        int d[2];
-        uint32_t slot[2];
-        bool live[2];
+        __syncwarp();
+        // two items per lane and trip: the two evaluations are independent and overlap
+        for (uint32_t base = 0; base < count; base += 64) {
+            int d[2];
+            uint32_t slot[2];
+            bool live[2];
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const uint32_t g = base + 32 * r + lane;
-            live[r] = g < total;
-            const uint32_t item = live[r] ? cv.queue[g] : 1u;     // a dead lane works on (proposal 0, bit 1) and drops it
-            slot[r] = item >> 5;
-            const uint32_t k = item & 31u;
-            const uint4 w0 = cv.win[slot[r] * 2], w1 = cv.win[slot[r] * 2 + 1];
-            Windows wn;
-            wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
-            wn.born = w1.w;
-            const uint32_t t = min(wn.s0 + k - 1, S - 1);
-            d[r] = item_delta<GROW>(wn, k, cv.ctr[t], GROW ? cv.hb[t] : 0u, __ldg(stepc + t), K);
+            for (int r = 0; r < 2; ++r) {
+                const uint32_t g = base + 32 * r + lane;
+                live[r] = g < count;
+                const uint32_t item = live[r] ? cv.queue[g] : 1u; // a dead lane works on (proposal 0, bit 1) and drops it
+                slot[r] = item >> 5;
+                const uint32_t k = item & 31u;
+                const uint4 w0 = cv.win[slot[r] * 2], w1 = cv.win[slot[r] * 2 + 1];
+                Windows wn;
+                wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
+                wn.born = w1.w;
+                const uint32_t t = min(wn.s0 + k - 1, S - 1);
+                const StepC sc = ASMEM ? stepc[t] : __ldg(stepc + t);
+                d[r] = item_delta<GROW>(wn, k, cv.ctr[t], GROW ? cv.hb[t] : 0u, sc, K);
+            }
+#pragma unroll
+            for (int r = 0; r < 2; ++r)
+                if (live[r] && d[r]) atomicAdd(cv.acc + slot[r], d[r]);
         }
-#pragma unroll
-        for (int r = 0; r < 2; ++r)
-            if (live[r] && d[r]) atomicAdd(cv.acc + slot[r], d[r]);
     }
     __syncwarp();
 #pragma unroll
@@ -409,11 +423,15 @@ __host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool 
     return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (W > 1 ? kShareSlots4 : 0u) + W * kPrivSlots4;
 }
 
-template <bool PSMEM, bool GROW, int W>
+// ASMEM (only with PSMEM): the access bitmap and the per-step constants, which every chain of the CTA reads, are
+// staged in shared memory once per CTA. With the schedules in shared memory the L1 cache is down to its minimum and
+// cannot hold them.
+template <bool PSMEM, bool GROW, int W, bool ASMEM>
 __global__ void __launch_bounds__(512)
 chain_kernel(const ChainParams prm)
 {
     static_assert(W >= 1 && W <= kMaxW && (W & (W - 1)) == 0, "warps per chain");
+    static_assert(PSMEM || !ASMEM, "shared access bitmap only beside shared schedules");
     extern __shared__ uint4 smem4[];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t cpb = (blockDim.x >> 5) / W;                   // chains per CTA
@@ -421,7 +439,7 @@ chain_kernel(const ChainParams prm)
     const uint32_t tid = sub * 32 + lane;                         // thread within the chain
     const uint32_t slot = blockIdx.x * cpb + cic;
     const bool active = slot < prm.chain_count;
-    if (W == 1 && !active) return;
+    if (W == 1 && !ASMEM && !active) return;
     const uint32_t chain = prm.chain_first + slot;
     const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
     const size_t pwords = (size_t)U * S32;
@@ -438,8 +456,19 @@ chain_kernel(const ChainParams prm)
     cv.win = priv4;
     cv.acc = reinterpret_cast<int*>(priv4 + kWinSlots4);
     cv.queue = reinterpret_cast<uint16_t*>(priv4 + kWinSlots4 + kAccSlots4);
-    cv.P = PSMEM ? reinterpret_cast<uint32_t*>(smem4 + (size_t)cpb * fixed4) + (size_t)cic * pwords
-                 : prm.ws + (size_t)slot * pwords;
+    uint32_t* const pool = reinterpret_cast<uint32_t*>(smem4 + (size_t)cpb * fixed4);   // schedules, then A, then constants
+    cv.P = PSMEM ? pool + (size_t)cic * pwords : prm.ws + (size_t)slot * pwords;
+    const uint32_t* Acol = prm.Acol;
+    const StepC* stepc = prm.stepc;
+    if (ASMEM) {
+        const size_t a_off = ((size_t)cpb * pwords + 3) & ~(size_t)3, c_off = (a_off + pwords + 3) & ~(size_t)3;
+        uint32_t* const a_s = pool + a_off;
+        StepC* const c_s = reinterpret_cast<StepC*>(pool + c_off);
+        copy_words(a_s, prm.Acol, pwords, threadIdx.x, blockDim.x);
+        for (uint32_t i = threadIdx.x; i < S; i += blockDim.x) c_s[i] = __ldg(prm.stepc + i);
+        Acol = a_s;
+        stepc = c_s;
+    }
     if (active) {
         for (uint32_t i = tid; i < S; i += 32 * W) cv.ctr[i] = __ldg(prm.counters0 + i);
         for (uint32_t i = tid; i < S32; i += 32 * W) cv.full[i] = __ldg(prm.full0 + i);
@@ -454,7 +483,7 @@ chain_kernel(const ChainParams prm)
             sh->ulen = 0u; sh->snap_dirty = 0u; sh->stopped = 0u; sh->turn = 0u; sh->napplied = 0u;
         }
     }
-    if (W > 1) {
+    if (W > 1 || ASMEM) {
         __syncthreads();
         if (!active) return;
     } else {
@@ -539,7 +568,7 @@ chain_kernel(const ChainParams prm)
                 todo[h] = left >= 32 ? 0xFFFFFFFFu : (1u << left) - 1u;
                 need[h] = todo[h];
             }
-            eval_batch<GROW>(cv, prm.Acol, prm.birth, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+            eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, lane, mv);
 #pragma unroll
             for (int h = 0; h < kMPL; ++h) need[h] = 0;
             if (W > 1) {
@@ -596,7 +625,7 @@ chain_kernel(const ChainParams prm)
 #pragma unroll
                 for (int h = 0; h < kMPL; ++h) any_need |= need[h];
                 if (any_need)
-                    eval_batch<GROW>(cv, prm.Acol, prm.birth, prm.stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+                    eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, lane, mv);
                 bool applied = false;
 #pragma unroll
                 for (int h = 0; h < kMPL; ++h) need[h] = 0;
@@ -835,7 +864,9 @@ struct Ctx {
     uint32_t wpb;            // chains per CTA
     uint32_t wpc;            // warps per chain
     uint32_t resident;       // chains per wave
-    size_t smem_per_warp;
+    size_t smem_per_warp;    // shared memory per chain
+    size_t smem_shared;      // shared memory of the CTA beside its chains (access bitmap and step constants)
+    bool asmem;              // the access bitmap and the step constants are staged in shared memory
     std::vector<double> temps;
     uint64_t init_ticks, calib_mean;
     uint32_t launches;
@@ -854,20 +885,24 @@ int validate(const kvp_problem* p, const kvp_anneal_params* a)
 
 typedef void (*ChainKernel)(const ChainParams);
 
-ChainKernel chain_kernel_for(bool psmem, bool grow, uint32_t W)
+template <bool PSMEM, bool ASMEM>
+ChainKernel chain_kernel_pick(bool grow, uint32_t W)
 {
-    if (W == 2)
-        return psmem ? (grow ? chain_kernel<true, true, 2> : chain_kernel<true, false, 2>)
-                     : (grow ? chain_kernel<false, true, 2> : chain_kernel<false, false, 2>);
-    return psmem ? (grow ? chain_kernel<true, true, 1> : chain_kernel<true, false, 1>)
-                 : (grow ? chain_kernel<false, true, 1> : chain_kernel<false, false, 1>);
+    if (W == 2) return grow ? chain_kernel<PSMEM, true, 2, ASMEM> : chain_kernel<PSMEM, false, 2, ASMEM>;
+    return grow ? chain_kernel<PSMEM, true, 1, ASMEM> : chain_kernel<PSMEM, false, 1, ASMEM>;
+}
+
+ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W)
+{
+    if (!psmem) return chain_kernel_pick<false, false>(grow, W);
+    return asmem ? chain_kernel_pick<true, true>(grow, W) : chain_kernel_pick<true, false>(grow, W);
 }
 
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 {
     const uint32_t grid = (count + c.wpb - 1) / c.wpb;
-    const size_t smem = (size_t)c.wpb * c.smem_per_warp;
-    chain_kernel_for(c.psmem, c.grow, c.wpc)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
+    const size_t smem = (size_t)c.wpb * c.smem_per_warp + c.smem_shared;
+    chain_kernel_for(c.psmem, c.asmem, c.grow, c.wpc)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }
@@ -923,17 +958,24 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
         c.wpb = want > wmax ? wmax : want;
         c.wpc = W;
         c.resident = a->chains;
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        // the access bitmap and the step constants beside the schedules, if there is room (the offsets are the kernel's)
+        const size_t a_off = ((size_t)c.wpb * (pbytes / 4) + 3) & ~(size_t)3, c_off = (a_off + pbytes / 4 + 3) & ~(size_t)3;
+        const size_t with_a = (size_t)c.wpb * fixed_bytes(W) + c_off * 4 + (size_t)p->S * 16;
+        c.asmem = with_a <= budget;
+        c.smem_shared = c.asmem ? with_a - (size_t)c.wpb * c.smem_per_warp : 0;
+        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.asmem, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
         const size_t ctr_bytes = fixed_bytes(W);
         if (ctr_bytes > budget) return KVP_ERR_RANGE;
         c.smem_per_warp = ctr_bytes;
+        c.smem_shared = 0;
+        c.asmem = false;
         c.wpc = W;
         uint32_t wcap = (uint32_t)(budget / ctr_bytes);            // chains per CTA at most
         if (wcap > 16 / W) wcap = 16 / W;
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, false, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
         int ctas = 0;
-        KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, c.grow, W), (int)(wcap * W * 32),
+        KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, false, c.grow, W), (int)(wcap * W * 32),
                                                                wcap * c.smem_per_warp));
         if (ctas < 1) return KVP_ERR_RANGE;
         uint32_t per_sm = (uint32_t)ctas * wcap;                   // resident chains per SM, at most 32 warps

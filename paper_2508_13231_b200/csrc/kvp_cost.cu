@@ -87,89 +87,116 @@ __device__ __forceinline__ uint32_t popc8(const uint32_t (&w)[8])
 // GROW (growing cache): L holds the rows of existing units. Placement bits of units that do not exist yet are
 // dropped, and the units born in a step (in L[s], not in L[s-1]) that are placed in HBM are a fourth cardinality
 // hb: they were written there, not migrated, so mi = occ - stay - hb.
-template <int VEC, bool GROW>
+// NS schedules of a batch share a thread: the access words are loaded once and used for all of them, which halves
+// the L2 traffic of a batch (A is the half of the bytes that comes from L2, not DRAM).
+template <int VEC, bool GROW, int NS>
 __global__ void __launch_bounds__(WIDE_WARPS * 32)
 count_wide_kernel(const uint32_t* __restrict__ A, const uint32_t* __restrict__ Ps, uint32_t S, uint32_t W32,
-                  uint32_t WV, uint32_t pad_mask, uint32_t SC, uint32_t* __restrict__ counts,
+                  uint32_t WV, uint32_t pad_mask, uint32_t SC, uint32_t n, uint32_t* __restrict__ counts,
                   const uint32_t* __restrict__ L, uint32_t* __restrict__ hbc)
 {
-    extern __shared__ uint2 acc[];                       // [WIDE_WARPS][SC], then GROW: uint32 [WIDE_WARPS][SC]
-    uint32_t* acc_hb = reinterpret_cast<uint32_t*>(acc + WIDE_WARPS * SC);
+    extern __shared__ uint2 acc[];                       // [NS][WIDE_WARPS][SC], then GROW: uint32 [NS][WIDE_WARPS][SC]
+    uint32_t* acc_hb = reinterpret_cast<uint32_t*>(acc + NS * WIDE_WARPS * SC);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cv0 = (blockIdx.x * WIDE_WARPS + warp) * (32 * WIDE_VEC) + lane;
     const uint32_t sb = blockIdx.y * SC;
     const uint32_t se = min(S, sb + SC);
-    const uint32_t* __restrict__ P = Ps + (size_t)blockIdx.z * S * W32;
+    const uint32_t* __restrict__ P[NS];
+#pragma unroll
+    for (int q = 0; q < NS; ++q)                         // a schedule past the batch re-reads the last one; its counts are dropped
+        P[q] = Ps + (size_t)min(blockIdx.z * NS + q, n - 1) * S * W32;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-    uint4 prev[WIDE_VEC], lprev[WIDE_VEC];
-    uint32_t occ_prev;
-    {
+    uint4 prev[NS][WIDE_VEC], lprev[WIDE_VEC];
+    uint32_t occ_prev[NS];
+#pragma unroll
+    for (int j = 0; j < WIDE_VEC; ++j) {
+        const uint32_t cv = cv0 + 32 * j;
+        if (GROW) lprev[j] = cv < WV ? load_vec<VEC>(L, W32, sb ? sb - 1 : 0, cv) : zero;
+    }
+#pragma unroll
+    for (int q = 0; q < NS; ++q) {
         uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
         for (int j = 0; j < WIDE_VEC; ++j) {
             const uint32_t cv = cv0 + 32 * j;
-            prev[j] = cv < WV ? mask_last<VEC>(load_vec<VEC>(P, W32, sb ? sb - 1 : 0, cv), cv, WV, pad_mask) : zero;
-            if (GROW) {
-                lprev[j] = cv < WV ? load_vec<VEC>(L, W32, sb ? sb - 1 : 0, cv) : zero;
-                prev[j] = and4(prev[j], lprev[j]);
-            }
-            w[4 * j] = prev[j].x; w[4 * j + 1] = prev[j].y; w[4 * j + 2] = prev[j].z; w[4 * j + 3] = prev[j].w;
+            prev[q][j] = cv < WV ? mask_last<VEC>(load_vec<VEC>(P[q], W32, sb ? sb - 1 : 0, cv), cv, WV, pad_mask) : zero;
+            if (GROW) prev[q][j] = and4(prev[q][j], lprev[j]);
+            w[4 * j] = prev[q][j].x; w[4 * j + 1] = prev[q][j].y; w[4 * j + 2] = prev[q][j].z; w[4 * j + 3] = prev[q][j].w;
         }
-        occ_prev = popc8(w);
+        occ_prev[q] = popc8(w);
     }
 #pragma unroll 4
     for (uint32_t s = sb; s < se; ++s) {
-        uint32_t wp[8], wh[8], ws[8], wb[8];
+        uint4 a[WIDE_VEC], l[WIDE_VEC], p[NS][WIDE_VEC];
 #pragma unroll
         for (int j = 0; j < WIDE_VEC; ++j) {
             const uint32_t cv = cv0 + 32 * j;
             const bool valid = cv < WV;
-            const uint4 a = valid ? load_vec<VEC>(A, W32, s, cv) : zero;
-            uint4 p = valid ? mask_last<VEC>(load_stream<VEC>(P, W32, s, cv), cv, WV, pad_mask) : zero;
-            if (GROW) {
-                const uint4 l = valid ? load_vec<VEC>(L, W32, s, cv) : zero;
-                p = and4(p, l);
-                const uint4 born = andn4(p, lprev[j]);               // placed in HBM in the step it is written
-                wb[4 * j] = born.x; wb[4 * j + 1] = born.y; wb[4 * j + 2] = born.z; wb[4 * j + 3] = born.w;
-                lprev[j] = l;
-            }
-            wp[4 * j] = p.x; wp[4 * j + 1] = p.y; wp[4 * j + 2] = p.z; wp[4 * j + 3] = p.w;
-            wh[4 * j] = a.x & p.x; wh[4 * j + 1] = a.y & p.y; wh[4 * j + 2] = a.z & p.z; wh[4 * j + 3] = a.w & p.w;
-            ws[4 * j] = p.x & prev[j].x; ws[4 * j + 1] = p.y & prev[j].y;
-            ws[4 * j + 2] = p.z & prev[j].z; ws[4 * j + 3] = p.w & prev[j].w;
-            prev[j] = p;
+            a[j] = valid ? load_vec<VEC>(A, W32, s, cv) : zero;
+            if (GROW) l[j] = valid ? load_vec<VEC>(L, W32, s, cv) : zero;
+#pragma unroll
+            for (int q = 0; q < NS; ++q)
+                p[q][j] = valid ? mask_last<VEC>(load_stream<VEC>(P[q], W32, s, cv), cv, WV, pad_mask) : zero;
         }
-        const uint32_t occ = popc8(wp), hr = popc8(wh), stay = popc8(ws);
-        uint32_t hb = 0;
-        if (GROW) hb = popc8(wb);
-        uint2 c = make_uint2(hr | ((occ - stay - hb) << 16), (occ_prev - stay) | (occ << 16));
-        occ_prev = occ;
-        c.x = __reduce_add_sync(0xFFFFFFFFu, c.x);       // 16-bit fields: 32 lanes * 256 < 65536
-        c.y = __reduce_add_sync(0xFFFFFFFFu, c.y);
-        if (GROW) hb = __reduce_add_sync(0xFFFFFFFFu, hb);
-        if (lane == 0) {
-            acc[warp * SC + (s - sb)] = c;
-            if (GROW) acc_hb[warp * SC + (s - sb)] = hb;
+#pragma unroll
+        for (int q = 0; q < NS; ++q) {
+            uint32_t wp[8], wh[8], ws[8], wb[8];
+#pragma unroll
+            for (int j = 0; j < WIDE_VEC; ++j) {
+                uint4 pj = p[q][j];
+                if (GROW) {
+                    pj = and4(pj, l[j]);
+                    const uint4 born = andn4(pj, lprev[j]);          // placed in HBM in the step it is written
+                    wb[4 * j] = born.x; wb[4 * j + 1] = born.y; wb[4 * j + 2] = born.z; wb[4 * j + 3] = born.w;
+                }
+                wp[4 * j] = pj.x; wp[4 * j + 1] = pj.y; wp[4 * j + 2] = pj.z; wp[4 * j + 3] = pj.w;
+                wh[4 * j] = a[j].x & pj.x; wh[4 * j + 1] = a[j].y & pj.y;
+                wh[4 * j + 2] = a[j].z & pj.z; wh[4 * j + 3] = a[j].w & pj.w;
+                ws[4 * j] = pj.x & prev[q][j].x; ws[4 * j + 1] = pj.y & prev[q][j].y;
+                ws[4 * j + 2] = pj.z & prev[q][j].z; ws[4 * j + 3] = pj.w & prev[q][j].w;
+                prev[q][j] = pj;
+            }
+            const uint32_t occ = popc8(wp), hr = popc8(wh), stay = popc8(ws);
+            uint32_t hb = 0;
+            if (GROW) hb = popc8(wb);
+            uint2 c = make_uint2(hr | ((occ - stay - hb) << 16), (occ_prev[q] - stay) | (occ << 16));
+            occ_prev[q] = occ;
+            c.x = __reduce_add_sync(0xFFFFFFFFu, c.x);   // 16-bit fields: 32 lanes * 256 < 65536
+            c.y = __reduce_add_sync(0xFFFFFFFFu, c.y);
+            if (GROW) hb = __reduce_add_sync(0xFFFFFFFFu, hb);
+            if (lane == 0) {
+                acc[(q * WIDE_WARPS + warp) * SC + (s - sb)] = c;
+                if (GROW) acc_hb[(q * WIDE_WARPS + warp) * SC + (s - sb)] = hb;
+            }
+        }
+        if (GROW) {
+#pragma unroll
+            for (int j = 0; j < WIDE_VEC; ++j) lprev[j] = l[j];
         }
     }
     __syncthreads();
-    for (uint32_t i = threadIdx.x; i < se - sb; i += blockDim.x) {
-        uint32_t hr = 0, mi = 0, mo = 0, occ = 0;
 #pragma unroll
-        for (int w = 0; w < WIDE_WARPS; ++w) {
-            const uint2 c = acc[w * SC + i];
-            hr += c.x & 0xFFFFu; mi += c.x >> 16; mo += c.y & 0xFFFFu; occ += c.y >> 16;
-        }
-        uint32_t* dst = counts + ((size_t)blockIdx.z * S + sb + i) * 4;
-        if (hr) atomicAdd(dst + 0, hr);
-        if (mi) atomicAdd(dst + 1, mi);
-        if (mo) atomicAdd(dst + 2, mo);
-        if (occ) atomicAdd(dst + 3, occ);
-        if (GROW) {
-            uint32_t hb = 0;
+    for (int q = 0; q < NS; ++q) {
+        const uint32_t sched = blockIdx.z * NS + q;
+        if (sched >= n) break;
+        for (uint32_t i = threadIdx.x; i < se - sb; i += blockDim.x) {
+            uint32_t hr = 0, mi = 0, mo = 0, occ = 0;
 #pragma unroll
-            for (int w = 0; w < WIDE_WARPS; ++w) hb += acc_hb[w * SC + i];
-            if (hb) atomicAdd(hbc + (size_t)blockIdx.z * S + sb + i, hb);
+            for (int w = 0; w < WIDE_WARPS; ++w) {
+                const uint2 c = acc[(q * WIDE_WARPS + w) * SC + i];
+                hr += c.x & 0xFFFFu; mi += c.x >> 16; mo += c.y & 0xFFFFu; occ += c.y >> 16;
+            }
+            uint32_t* dst = counts + ((size_t)sched * S + sb + i) * 4;
+            if (hr) atomicAdd(dst + 0, hr);
+            if (mi) atomicAdd(dst + 1, mi);
+            if (mo) atomicAdd(dst + 2, mo);
+            if (occ) atomicAdd(dst + 3, occ);
+            if (GROW) {
+                uint32_t hb = 0;
+#pragma unroll
+                for (int w = 0; w < WIDE_WARPS; ++w) hb += acc_hb[(q * WIDE_WARPS + w) * SC + i];
+                if (hb) atomicAdd(hbc + (size_t)sched * S + sb + i, hb);
+            }
         }
     }
 }
@@ -317,25 +344,28 @@ int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, u
     KVP_CUDA(cudaMemsetAsync(counts, 0, (size_t)n * p->S * 16, st));
     if (grow) KVP_CUDA(cudaMemsetAsync(hbc, 0, (size_t)n * p->S * 4, st));
     const uint32_t col_ctas = (WV + WIDE_WARPS * 32 * WIDE_VEC - 1) / (WIDE_WARPS * 32 * WIDE_VEC);
+    // two schedules per thread once a batch is large enough to fill the GPU that way
+    const uint32_t NS = n >= 8 ? 2u : 1u;
+    const uint32_t nz = (n + NS - 1) / NS;
     // Split the steps until the grid is at least four full waves (148 SMs x 8 resident CTAs), so that the last,
     // partial wave costs little; every chunk re-reads one halo row (1/SC more traffic, mostly from L2).
     uint32_t SC = p->S;
-    while (SC > 8 && (uint64_t)col_ctas * ((p->S + SC - 1) / SC) * n < 148u * 8u * 4u) SC = (SC + 1) / 2;
+    while (SC > 8 && (uint64_t)col_ctas * ((p->S + SC - 1) / SC) * nz < 148u * 8u * 4u) SC = (SC + 1) / 2;
     if (SC > 512) SC = 512;
-    dim3 grid(col_ctas, (p->S + SC - 1) / SC, n);
-    const size_t smem = (size_t)WIDE_WARPS * SC * (sizeof(uint2) + (grow ? 4 : 0));
+    dim3 grid(col_ctas, (p->S + SC - 1) / SC, nz);
+    const size_t smem = (size_t)NS * WIDE_WARPS * SC * (sizeof(uint2) + (grow ? 4 : 0));
     const int T = WIDE_WARPS * 32;
-    if (grow) {
-        if (vec4)
-            count_wide_kernel<4, true><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, p->dL, hbc);
-        else
-            count_wide_kernel<1, true><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, p->dL, hbc);
+#define KVP_WIDE(VEC, GROW, NSCH)                                                                                  \
+    count_wide_kernel<VEC, GROW, NSCH><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, n, \
+                                                              counts, GROW ? p->dL : nullptr, GROW ? hbc : nullptr)
+    if (NS == 2) {
+        if (grow) { if (vec4) KVP_WIDE(4, true, 2); else KVP_WIDE(1, true, 2); }
+        else { if (vec4) KVP_WIDE(4, false, 2); else KVP_WIDE(1, false, 2); }
     } else {
-        if (vec4)
-            count_wide_kernel<4, false><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, nullptr, nullptr);
-        else
-            count_wide_kernel<1, false><<<grid, T, smem, st>>>(p->dA, schedules, p->S, p->W32, WV, p->pad_mask, SC, counts, nullptr, nullptr);
+        if (grow) { if (vec4) KVP_WIDE(4, true, 1); else KVP_WIDE(1, true, 1); }
+        else { if (vec4) KVP_WIDE(4, false, 1); else KVP_WIDE(1, false, 1); }
     }
+#undef KVP_WIDE
     KVP_CUDA(cudaGetLastError());
     if (launches) *launches += 1;
     return KVP_OK;

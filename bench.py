@@ -192,9 +192,10 @@ def run_cost_kernel(args):
 # Algorithmic thread instructions of the trace kernels per (unit, step): one Philox4x32-10 for the noise (10 rounds
 # of two wide multiplies, four xors and two key additions: 60 with 3-input logic ops), the 8-term Irwin-Hall sum
 # and the AR(1) update 22, a second Philox and a compare for the burst draw 62 when bursts are on, and the top-k
-# search, 32 rounds of one compare and one count per unit plus the selection compares: 68.
+# search: the range reduction (2), three histogram passes of a prefix compare, a digit and a shared-memory add per
+# unit (12) and the selection compares (4): 18.
 def trace_alg_thread_instr(bursts):
-    return 60 + 22 + (62 if bursts else 0) + 68
+    return 60 + 22 + (62 if bursts else 0) + 18
 
 
 def run_trace_kernel(args):

@@ -4,6 +4,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
+#include <thread>
 #include <vector>
 
 #include "kvp_common.cuh"
@@ -238,21 +240,57 @@ extern "C" int kvp_get_info(const kvp_problem* p, kvp_info* info)
     return KVP_OK;
 }
 
+namespace {
+
+// Rows [j0, j1) of the acceptance table. Entries whose exponent is beyond 22.5 > ln(2^32) are zero whatever the
+// last bits of exp() are, so exp() is not called for them.
+void accept_rows(const double* temps, const uint32_t* shifts, uint32_t j0, uint32_t j1, uint32_t* table)
+{
+    for (uint32_t j = j0; j < j1; ++j) {
+        const double C = temps[j] >= 1.0 ? temps[j] : 1.0;     // also maps NaN to 1
+        const double bin = (double)(1ull << shifts[j]);
+        for (uint32_t q = 0; q < KVP_TABLE_Q; ++q) {
+            const double x = ((double)q + 0.5) * bin;
+            const double y = x / C;
+            uint32_t v = 0u;
+            if (y <= 22.5) {
+                const double thr = 4294967296.0 * exp(-x / C);
+                v = thr >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)thr;
+            }
+            table[(size_t)j * KVP_TABLE_Q + q] = v;
+        }
+    }
+}
+
+}  // namespace
+
 extern "C" int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint32_t* shifts)
 {
     if (!temps || !table || !shifts || !levels) return KVP_ERR_ARG;
     for (uint32_t j = 0; j < levels; ++j) {
-        const double C = temps[j] >= 1.0 ? temps[j] : 1.0;     // also maps NaN to 1
+        const double C = temps[j] >= 1.0 ? temps[j] : 1.0;
         uint32_t sh = 0;
         while ((double)KVP_TABLE_Q * (double)(1ull << sh) < 23.0 * C)
             if (++sh > 40) return KVP_ERR_RANGE;
         shifts[j] = sh;
-        const double bin = (double)(1ull << sh);
-        for (uint32_t q = 0; q < KVP_TABLE_Q; ++q) {
-            const double x = ((double)q + 0.5) * bin;
-            const double thr = 4294967296.0 * exp(-x / C);
-            table[(size_t)j * KVP_TABLE_Q + q] = thr >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)thr;
+    }
+    // A ladder of 64 levels is 65,536 calls of exp(), about half a millisecond on one core and a tenth of an
+    // annealing call on a small problem: the rows are independent, so a few threads share them.
+    uint32_t nthr = levels >= 16 ? std::min<uint32_t>(8u, std::max(1u, std::thread::hardware_concurrency())) : 1u;
+    if (nthr > 1) {
+        std::vector<std::thread> pool;
+        const uint32_t per = (levels + nthr - 1) / nthr;
+        try {
+            for (uint32_t t = 1; t < nthr && t * per < levels; ++t)
+                pool.emplace_back(accept_rows, temps, shifts, t * per, std::min(levels, (t + 1) * per), table);
+        } catch (...) {                                        // no thread to be had: this one does the rest
+            const uint32_t done = (uint32_t)pool.size() + 1;
+            accept_rows(temps, shifts, std::min(levels, done * per), levels, table);
         }
+        accept_rows(temps, shifts, 0, std::min(levels, per), table);
+        for (auto& th : pool) th.join();
+    } else {
+        accept_rows(temps, shifts, 0, levels, table);
     }
     return KVP_OK;
 }

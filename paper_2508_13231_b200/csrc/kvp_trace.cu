@@ -1,8 +1,9 @@
 // Trace kernels: synthetic importance per unit and step, top-k per (layer, kv-head) group, packed into uint32
-// bitmaps. Two passes by default: one thread per unit runs the AR(1) recurrence over all steps (sequential in
-// time) and writes a score matrix; then one CTA per (group, step) finds the k-th largest score with a 32-round
-// bitwise binary search over block-wide counts, ties going to the lower unit index. A fused single-pass form
-// (one CTA per group, state in registers) serves traces whose score matrix would exceed the scratch budget.
+// bitmaps. Two passes when there are few groups: one thread per unit runs the AR(1) recurrence over all steps
+// (sequential in time) and writes a score matrix; then one CTA per (group, step) finds the k-th largest score
+// digit by digit with shared-memory histograms, ties going to the lower unit index. A fused single-pass form
+// (one CTA per group walking the steps, state in registers) serves traces with many groups, layered or growing
+// traces and those whose score matrix would exceed the scratch budget.
 #include "kvp_common.cuh"
 
 namespace kvp {
@@ -44,30 +45,40 @@ __device__ __forceinline__ uint32_t block_sum(uint32_t v, uint32_t* slot)
     return *slot;
 }
 
+constexpr int kDigitBits = 8;                        // the search fixes this many bits of the threshold per pass
+constexpr int kBins = 1 << kDigitBits;
+constexpr int kPasses = 32 / kDigitBits;
+
 struct SelectSmem {
-    uint32_t cnt[36];            // 32 search rounds + 2 extra counts
+    uint32_t hist[kPasses][kBins];   // per pass: how many keys with the threshold's higher bits have each digit
+    uint32_t cnt[4];                 // block-wide counts beside the search
     uint32_t warp[32];
     uint32_t run;
-    uint32_t hi, lo;             // largest and smallest key of the step
+    uint32_t hi, lo;                 // largest and smallest key of the step
+    uint32_t K, need, equal;         // threshold so far, how many keys are still to find at or below it, ties at it
 };
 
 // State of one selection; a barrier must follow before select_step.
 __device__ __forceinline__ void select_reset(SelectSmem& sm)
 {
-    for (uint32_t i = threadIdx.x; i < 36; i += blockDim.x) sm.cnt[i] = 0;
+    for (uint32_t i = threadIdx.x; i < kPasses * kBins; i += blockDim.x) (&sm.hist[0][0])[i] = 0;
+    if (threadIdx.x < 4) sm.cnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) { sm.hi = 0u; sm.lo = ~0u; }
 }
 
 // Top-k of one (group, step): the CTA holds the n keys (UPT per thread, unit i = j*T + tid, 0 past n) and sets the
 // bits of the k largest, ties to the lower unit index. select_reset and a barrier come first.
 // topk: how many to pick (at most the number of non-zero keys when zero marks a unit that is not there yet).
+//
+// The threshold K (the k-th largest key) is found digit by digit from the top, eight bits per pass: the keys that
+// agree with K in the bits fixed so far are counted per digit in a shared-memory histogram, and one warp walks
+// the histogram from the top until the counts reach what is still needed. The bits above the highest one in which
+// the largest and the smallest key differ are common to all keys and need no pass: three passes on these scores.
 template <int UPT>
 __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const TraceK& k, uint32_t topk, uint32_t gbase,
                                             uint32_t t, SelectSmem& sm)
 {
     const uint32_t T = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // The k-th largest key lies between the smallest and the largest, so it shares every bit above the highest one
-    // in which those two differ: the search starts below that bit.
     uint32_t mx = 0u, mn = ~0u;
 #pragma unroll
     for (int j = 0; j < UPT; ++j)
@@ -76,26 +87,49 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
     mn = __reduce_min_sync(0xFFFFFFFFu, mn);
     if (lane == 0) { atomicMax(&sm.hi, mx); atomicMin(&sm.lo, mn); }
     __syncthreads();
-    const int low_bits = 32 - __clz(sm.hi ^ sm.lo);          // 0 when all keys are equal
-    // largest K with |{key >= K}| >= topk, bit by bit from the top
-    uint32_t K = low_bits >= 32 ? 0u : sm.hi & ~((1u << low_bits) - 1u);
-    for (int bit = low_bits - 1; bit >= 0; --bit) {
-        const uint32_t cand = K | (1u << bit);
-        uint32_t c = 0;
+    int rem = 32 - __clz(sm.hi ^ sm.lo);                     // bits still open; 0 when all keys are equal
+    uint32_t K = rem >= 32 ? 0u : sm.hi & ~((1u << rem) - 1u);
+    uint32_t need = topk, equal = k.n;                       // all keys equal: every one ties at K
+    for (int pass = 0; rem > 0; ++pass) {
+        const int w = rem < kDigitBits ? rem : kDigitBits, sh = rem - w;
+        uint32_t* hist = sm.hist[pass];
 #pragma unroll
-        for (int j = 0; j < UPT; ++j) c += key[j] >= cand ? 1u : 0u;      // slots past n hold key 0 < cand
-        if (block_sum(c, &sm.cnt[31 - bit]) >= topk) K = cand;
-    }
-    uint32_t cg = 0, ce = 0;
+        for (int j = 0; j < UPT; ++j) {
+            const bool in = j * T + tid < k.n && (rem >= 32 || (key[j] >> rem) == (K >> rem));
+            if (in) atomicAdd(hist + ((key[j] >> sh) & ((1u << w) - 1u)), 1u);
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane l owns digits 8l .. 8l+7; suffix sums over the lanes, then over the owner's eight bins
+            uint32_t h[8], s = 0;
 #pragma unroll
-    for (int j = 0; j < UPT; ++j) {
-        const bool ok = j * T + tid < k.n;
-        cg += (ok && key[j] > K) ? 1u : 0u;
-        ce += (ok && key[j] == K) ? 1u : 0u;
+            for (int i = 0; i < 8; ++i) { h[i] = hist[8 * lane + i]; s += h[i]; }
+            uint32_t suf = s;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t v = __shfl_down_sync(0xFFFFFFFFu, suf, off);
+                if (lane + off < 32) suf += v;
+            }
+            const uint32_t reach = __ballot_sync(0xFFFFFFFFu, suf >= need);    // never empty: the counts add up to >= need
+            if (lane == 31u - __clz(reach)) {
+                uint32_t higher = suf - s;
+#pragma unroll
+                for (int i = 7; i >= 0; --i) {
+                    if (higher + h[i] >= need) {
+                        sm.K = K | ((uint32_t)(8 * lane + i) << sh);
+                        sm.need = need - higher;
+                        sm.equal = h[i];
+                        break;
+                    }
+                    higher += h[i];
+                }
+            }
+        }
+        __syncthreads();
+        K = sm.K; need = sm.need; equal = sm.equal;
+        rem = sh;
     }
-    const uint32_t above = block_sum(cg, &sm.cnt[32]);
-    const uint32_t equal = block_sum(ce, &sm.cnt[33]);
-    const uint32_t take = topk - above;                      // ties to admit, lowest unit index first
+    const uint32_t take = need;                              // ties to admit, lowest unit index first
     const bool rank_ties = equal != take;
     if (tid == 0) sm.run = 0;
     __syncthreads();
@@ -189,7 +223,7 @@ trace_kernel(const TraceK k)
         }
         __syncthreads();
         uint32_t topk = k.topk;
-        if (GROW) topk = min(topk, block_sum(here, &sm.cnt[34]));
+        if (GROW) topk = min(topk, block_sum(here, &sm.cnt[0]));
         select_step<UPT>(key, k, topk, gbase, t, sm);
         __syncthreads();
     }

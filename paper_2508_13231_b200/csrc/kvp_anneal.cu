@@ -57,10 +57,11 @@ constexpr int kMPL = 1;
 constexpr uint32_t kBatch = 32 * kMPL;
 constexpr uint32_t kWinSlots4 = kBatch * 2;                        // 8 words of windows per proposal
 constexpr uint32_t kAccSlots4 = kBatch / 4;                        // one int per proposal
-// uint16 work items; 31 per proposal in the worst case, so the queue holds the worst case of half a warp's proposals
-// and a batch with more items than that is worked off in two halves
-constexpr uint32_t kQueueCap = kBatch * 31 / 2;
+// uint16 work items, 31 per proposal in the worst case. Where shared memory is short (HALFQ) the queue holds the worst
+// case of half a warp's proposals and a batch with more items than that is worked off in two halves.
+constexpr uint32_t kQueueCap = kBatch * 31;
 constexpr uint32_t kQueueSlots4 = (kQueueCap * 2 + 15) / 16;
+constexpr uint32_t kHalfQueueSlots4 = (kQueueCap / 2 * 2 + 15) / 16;
 
 // A proposal as its lane keeps it in registers: the Philox words and, after evaluation, the verdict.
 // The placement windows live in shared memory (ChainView::win), 8 words per proposal:
@@ -221,6 +222,35 @@ __device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ A
     mv.acc = metropolis(delta, mv.w, trow, shift);
 }
 
+// N queue items per lane, items base + 32 r + lane: the cost change of one step of one proposal each, added to the
+// proposal's sum.
+template <bool GROW, bool ASMEM, int N>
+__device__ __forceinline__ void eval_items(const ChainView cv, const StepC* __restrict__ stepc, const CostK K, uint32_t S,
+                                           uint32_t base, uint32_t count, uint32_t lane)
+{
+    int d[N];
+    uint32_t slot[N];
+    bool live[N];
+#pragma unroll
+    for (int r = 0; r < N; ++r) {
+        const uint32_t g = base + 32 * r + lane;
+        live[r] = g < count;
+        const uint32_t item = live[r] ? cv.queue[g] : 1u;         // a dead lane works on (proposal 0, bit 1) and drops it
+        slot[r] = item >> 5;
+        const uint32_t k = item & 31u;
+        const uint4 w0 = cv.win[slot[r] * 2], w1 = cv.win[slot[r] * 2 + 1];
+        Windows wn;
+        wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
+        wn.born = w1.w;
+        const uint32_t t = min(wn.s0 + k - 1, S - 1);
+        const StepC sc = ASMEM ? stepc[t] : __ldg(stepc + t);
+        d[r] = item_delta<GROW>(wn, k, cv.ctr[t], GROW ? cv.hb[t] : 0u, sc, K);
+    }
+#pragma unroll
+    for (int r = 0; r < N; ++r)
+        if (live[r] && d[r]) atomicAdd(cv.acc + slot[r], d[r]);
+}
+
 // Evaluation of the proposals named by `need` (one mask per proposal row), shared by the warp: every lane
 // prepares its own proposals, the (proposal, step) pairs whose cost changes are queued in shared memory, and
 // the warp works the queue off 32 pairs at a time, so that lanes with short and long proposals carry the
@@ -255,9 +285,9 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         pos += __popc(has & below) << bit;
         total += __popc(has) << bit;
     }
-    // The queue holds kQueueCap items, the worst case of 16 lanes. A batch with more (rare) goes in two halves,
-    // lanes 0..15 first.
-    const uint32_t halves = total > kQueueCap ? 2u : 1u;
+    // ASMEM: the queue holds kQueueCap / 2 items, the worst case of 16 lanes. A batch with more (rare) goes in two
+    // halves, lanes 0..15 first.
+    const uint32_t halves = ASMEM && total > kQueueCap / 2 ? 2u : 1u;
     const uint32_t mid = halves > 1 ? __shfl_sync(0xFFFFFFFFu, pos, 16) : 0u;   // items of lanes 0..15
     for (uint32_t half = 0; half < halves; ++half) {
         const bool pushing = halves == 1 || (lane >> 4) == half;
@@ -278,29 +308,10 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
             }
         }
         __syncwarp();
-        // two items per lane and trip: the two evaluations are independent and overlap
+        // two items per lane and trip (the two evaluations are independent and overlap), one where 32 or fewer are left
         for (uint32_t base = 0; base < count; base += 64) {
-            int d[2];
-            uint32_t slot[2];
-            bool live[2];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const uint32_t g = base + 32 * r + lane;
-                live[r] = g < count;
-                const uint32_t item = live[r] ? cv.queue[g] : 1u; // a dead lane works on (proposal 0, bit 1) and drops it
-                slot[r] = item >> 5;
-                const uint32_t k = item & 31u;
-                const uint4 w0 = cv.win[slot[r] * 2], w1 = cv.win[slot[r] * 2 + 1];
-                Windows wn;
-                wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
-                wn.born = w1.w;
-                const uint32_t t = min(wn.s0 + k - 1, S - 1);
-                const StepC sc = ASMEM ? stepc[t] : __ldg(stepc + t);
-                d[r] = item_delta<GROW>(wn, k, cv.ctr[t], GROW ? cv.hb[t] : 0u, sc, K);
-            }
-#pragma unroll
-            for (int r = 0; r < 2; ++r)
-                if (live[r] && d[r]) atomicAdd(cv.acc + slot[r], d[r]);
+            if (base + 32 < count) eval_items<GROW, ASMEM, 2>(cv, stepc, K, S, base, count, lane);
+            else eval_items<GROW, ASMEM, 1>(cv, stepc, K, S, base, count, lane);
         }
     }
     __syncwarp();
@@ -409,7 +420,11 @@ struct ChainShare {
     uint32_t applog[kLog];       // s0 | (s0 + len) << 16 of an applied move
 };
 constexpr uint32_t kShareSlots4 = (sizeof(ChainShare) + 15) / 16;
-constexpr uint32_t kPrivSlots4 = kWinSlots4 + kAccSlots4 + kQueueSlots4;   // per warp: windows, sums, work queue
+// per warp: windows, sums, work queue
+__host__ __device__ constexpr uint32_t priv_slots4(bool halfq)
+{
+    return kWinSlots4 + kAccSlots4 + (halfq ? kHalfQueueSlots4 : kQueueSlots4);
+}
 // A wait for the turn gives up after this many polls (each at least some tens of nanoseconds apart): the chain then
 // reports KVP_ERR_TIMEOUT instead of holding the GPU. A turn lasts microseconds.
 constexpr uint32_t kTurnPolls = 1u << 24;
@@ -418,9 +433,9 @@ __device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p) { return 
 __device__ __forceinline__ void st_volatile_u32(uint32_t* p, uint32_t v) { *reinterpret_cast<volatile uint32_t*>(p) = v; }
 
 // shared-memory words (as uint4 slots) of one chain besides its schedule
-__host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool grow, uint32_t W)
+__host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool grow, uint32_t W, bool halfq)
 {
-    return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (W > 1 ? kShareSlots4 : 0u) + W * kPrivSlots4;
+    return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (W > 1 ? kShareSlots4 : 0u) + W * priv_slots4(halfq);
 }
 
 // ASMEM (only with PSMEM): the access bitmap and the per-step constants, which every chain of the CTA reads, are
@@ -445,14 +460,14 @@ chain_kernel(const ChainParams prm)
     const size_t pwords = (size_t)U * S32;
     const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
     const uint32_t h4 = GROW ? (S + 3) / 4 : 0u;                  // uint4 slots of the written-to-HBM counts
-    const uint32_t fixed4 = chain_fixed4(S, S32, GROW, W);
+    const uint32_t fixed4 = chain_fixed4(S, S32, GROW, W, ASMEM);
     uint4* const mine4 = smem4 + (size_t)cic * fixed4;
     ChainView cv;
     cv.ctr = mine4;
     cv.full = reinterpret_cast<uint32_t*>(mine4 + S);
     cv.hb = reinterpret_cast<uint32_t*>(mine4 + S + f4);
     ChainShare* const sh = reinterpret_cast<ChainShare*>(mine4 + S + f4 + h4);
-    uint4* const priv4 = mine4 + S + f4 + h4 + (W > 1 ? kShareSlots4 : 0u) + sub * kPrivSlots4;
+    uint4* const priv4 = mine4 + S + f4 + h4 + (W > 1 ? kShareSlots4 : 0u) + sub * priv_slots4(ASMEM);
     cv.win = priv4;
     cv.acc = reinterpret_cast<int*>(priv4 + kWinSlots4);
     cv.queue = reinterpret_cast<uint16_t*>(priv4 + kWinSlots4 + kAccSlots4);
@@ -523,20 +538,22 @@ chain_kernel(const ChainParams prm)
         have = false;
     };
 
-    uint64_t lvl_start = 0, m_end = 0;                            // m_end: moves done when the chain ended
+    uint64_t lvl_start = 0;                                       // first move of the level
     uint32_t base = 0;                                            // index of the level's first batch (mod 2^32)
     bool stop = false;
     for (uint32_t level = 0; level < prm.levels && lvl_start < prm.upto; ++level) {
-        // a temperature level: its moves in batches of up to 32 * kMPL consecutive moves
-        const uint64_t lvl_end = level + 1 < prm.levels ? min(lvl_start + prm.per_level, prm.upto) : prm.upto;
-        const uint64_t nbat = (lvl_end - lvl_start + kBatch - 1) / kBatch;
+        // a temperature level: its moves in batches of up to 32 * kMPL consecutive moves (fewer than 2^32 batches:
+        // the host refuses longer levels)
+        const uint64_t lvl_len = (level + 1 < prm.levels ? min(lvl_start + prm.per_level, prm.upto) : prm.upto) - lvl_start;
+        const uint32_t nbat = (uint32_t)((lvl_len + kBatch - 1) / kBatch);
+        const uint32_t last_nb = (uint32_t)(lvl_len - (uint64_t)(nbat - 1) * kBatch);
+        const bool last_level = lvl_start + lvl_len >= prm.upto;
         const uint32_t shift = __ldg(prm.shifts + level);
         const uint32_t* trow = prm.table + (size_t)level * KVP_TABLE_Q;
         if (W == 1 && level > 0) {
             if (prm.early_permille && level >= prm.early_from &&
                 (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille) {
                 stop = true;
-                m_end = lvl_start;
                 break;
             }
             best_at_boundary = best;
@@ -545,10 +562,10 @@ chain_kernel(const ChainParams prm)
         // against the current state; the warp then commits them in move order. A move that changes the schedule
         // invalidates only later moves whose step windows overlap its own; those are evaluated again before their
         // turn comes, so the outcome is that of the sequential chain.
-        for (uint64_t bi = (sub - base) & (W - 1); bi < nbat; bi += W) {
-            const uint64_t m = lvl_start + bi * kBatch;
-            const uint32_t nb = (uint32_t)min((uint64_t)kBatch, lvl_end - m);
-            const uint32_t b = base + (uint32_t)bi;
+        for (uint32_t bi = (sub - base) & (W - 1); bi < nbat; bi += W) {
+            const uint64_t m = lvl_start + (uint64_t)bi * kBatch;
+            const uint32_t nb = bi + 1 < nbat ? kBatch : last_nb;
+            const uint32_t b = base + bi;
             uint32_t n0 = 0;
             if (W > 1) {
                 // Moves applied from now on may be half visible to the reads below: they are checked for at the turn.
@@ -614,7 +631,6 @@ chain_kernel(const ChainParams prm)
                     if (prm.early_permille && level >= prm.early_from &&
                         (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille) {
                         stop = true;
-                        m_end = lvl_start;
                         break;
                     }
                     best_at_boundary = best;
@@ -685,13 +701,13 @@ chain_kernel(const ChainParams prm)
                 }
                 if (!applied) break;
             }
-            m_end = m + nb;
-            if (W > 1 && m_end < prm.upto) pass_turn(b);          // hand the chain to the owner of the next batch
+            if (W > 1 && !(last_level && bi + 1 == nbat)) pass_turn(b);   // hand the chain to the owner of the next batch
         }
         if (stop) break;                                          // `base` stays the index of the batch that stopped
-        base += (uint32_t)nbat;
-        lvl_start = lvl_end;
+        base += nbat;
+        lvl_start += lvl_len;
     }
+    const uint64_t m_end = stop ? lvl_start : prm.upto;           // moves done when the chain ended
     // The warp that committed the last batch, or that ended the chain by the stop rule, reports.
     if (W > 1) {
         const bool writer = stop || (base ? ((base - 1u) & (W - 1)) == sub : sub == 0);
@@ -701,7 +717,6 @@ chain_kernel(const ChainParams prm)
         __syncwarp();
         n_acc = 0; n_inf = 0;
         for (int w = 0; w < W; ++w) { n_acc += sh->n_acc[w]; n_inf += sh->n_inf[w]; }
-        if (!stop) m_end = prm.upto < lvl_start ? prm.upto : lvl_start;
     }
     if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
     if (ulog && lane == 0) prm.undo_len[slot] = ulen;
@@ -880,6 +895,7 @@ int validate(const kvp_problem* p, const kvp_anneal_params* a)
     if (a->init_mode == KVP_INIT_USER && !a->init_schedule) return KVP_ERR_ARG;
     if (!a->temps && (!(a->p0 > 0.0 && a->p0 < 1.0) || !(a->alpha > 0.0 && a->alpha <= 1.0))) return KVP_ERR_ARG;
     if (a->chains >= (1u << 24) || (uint64_t)a->first_chain + a->chains > (1ull << 31)) return KVP_ERR_RANGE;
+    if (a->moves / a->levels + a->levels >= (1ull << 36)) return KVP_ERR_RANGE;   // batches of a level are counted in 32 bits
     return KVP_OK;
 }
 
@@ -937,7 +953,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const size_t budget = (size_t)smem_max - 1024;
     // per chain: counters, full-step bitmap and, per warp, the batch's windows, accumulators and work queue
     c.grow = p->dL != nullptr;
-    auto fixed_bytes = [&](uint32_t W) { return (size_t)chain_fixed4(p->S, p->S32, c.grow, W) * 16; };
+    auto fixed_bytes = [&](uint32_t W, bool halfq = false) {
+        return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq) * 16;
+    };
     const size_t pbytes = (size_t)p->U * p->S32 * 4;
     // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
     // chains then keeps twice as many warps in flight. KVP_WARPS_PER_CHAIN=1|2 overrides the choice (for tuning).
@@ -960,9 +978,14 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
         c.resident = a->chains;
         // the access bitmap and the step constants beside the schedules, if there is room (the offsets are the kernel's)
         const size_t a_off = ((size_t)c.wpb * (pbytes / 4) + 3) & ~(size_t)3, c_off = (a_off + pbytes / 4 + 3) & ~(size_t)3;
-        const size_t with_a = (size_t)c.wpb * fixed_bytes(W) + c_off * 4 + (size_t)p->S * 16;
+        const size_t with_a = (size_t)c.wpb * fixed_bytes(W, true) + c_off * 4 + (size_t)p->S * 16;
         c.asmem = with_a <= budget;
-        c.smem_shared = c.asmem ? with_a - (size_t)c.wpb * c.smem_per_warp : 0;
+        if (c.asmem) {                                           // that kernel makes do with half the work queue
+            c.smem_per_warp = fixed_bytes(W, true) + pbytes;
+            c.smem_shared = with_a - (size_t)c.wpb * c.smem_per_warp;
+        } else {
+            c.smem_shared = 0;
+        }
         KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.asmem, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
         const size_t ctr_bytes = fixed_bytes(W);

@@ -45,7 +45,7 @@ struct ChainParams {
     uint32_t chain_first, chain_count, result_base;
     uint32_t levels, p_swap_256, len_choices;
     uint32_t early_permille, early_from;
-    uint32_t seed_lo, seed_hi;
+    PhiloxKeys keys;             // round keys of the seed
     uint64_t per_level, upto, init_ticks;
 };
 
@@ -578,7 +578,7 @@ chain_kernel(const ChainParams prm)
             for (int h = 0; h < kMPL; ++h) {
                 uint32_t r[4];
                 const uint64_t mine = m + 32u * h + lane;
-                philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
+                philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.keys, r);
                 decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv[h]);
                 mv[h].inf = false; mv[h].acc = false; mv[h].chg = false; mv[h].delta = 0;
                 const uint32_t left = nb > 32u * h ? nb - 32u * h : 0u;
@@ -756,7 +756,7 @@ undo_kernel(const ChainParams prm, uint32_t slot, uint32_t* __restrict__ dst)
         const uint64_t m = ulog[i];
         uint32_t r[4];
         LaneMove mv;
-        philox4x32_10((uint32_t)m, (uint32_t)(m >> 32), chain, TAG_MOVE, prm.seed_lo, prm.seed_hi, r);
+        philox4x32_10((uint32_t)m, (uint32_t)(m >> 32), chain, TAG_MOVE, prm.keys, r);
         decode_move(r, prm.p_swap_256, prm.len_choices, S, prm.U, mv);
         const bool swap = mv.pk & 1u;
         const uint32_t len = (mv.pk >> 1) & 63u, s0 = mv.pk >> 8, end = min(s0 + len, S);
@@ -803,7 +803,7 @@ calib_kernel(const ChainParams prm, unsigned long long* acc)
     if (i >= CALIB_N) return;
     uint32_t r[4];
     LaneMove mv;
-    philox4x32_10(i, 0u, 0u, TAG_CALIB, prm.seed_lo, prm.seed_hi, r);
+    philox4x32_10(i, 0u, 0u, TAG_CALIB, prm.keys, r);
     decode_move(r, prm.p_swap_256, prm.len_choices, prm.S, prm.U, mv);
     eval_lane<GROW>(prm.Pcol0, prm.Acol, prm.counters0, prm.full0, prm.birth, prm.hb0, prm.stepc, prm.K, prm.S, prm.S32,
                     prm.table, 0u, mv);
@@ -1097,7 +1097,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     prm.U = p->U; prm.S = p->S; prm.S32 = p->S32; prm.cap = p->cap;
     prm.levels = a->levels; prm.p_swap_256 = a->p_swap_256; prm.len_choices = a->max_len_log2 + 1;
     prm.early_permille = a->early_stop_permille; prm.early_from = a->early_stop_from_level;
-    prm.seed_lo = (uint32_t)a->seed; prm.seed_hi = (uint32_t)(a->seed >> 32);
+    prm.keys = philox_keys((uint32_t)a->seed, (uint32_t)(a->seed >> 32));
     prm.per_level = a->moves / a->levels ? a->moves / a->levels : 1;
 
     // temperature ladder

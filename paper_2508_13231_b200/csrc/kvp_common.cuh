@@ -58,6 +58,37 @@ __host__ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1,
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// The ten round keys of Philox4x32-10 for one seed (round r uses key + r * Weyl constant). A kernel that draws every
+// block with the same seed takes them as a launch parameter: the per-round additions then cost nothing on the device.
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+};
+
+inline PhiloxKeys philox_keys(uint32_t seed_lo, uint32_t seed_hi)
+{
+    PhiloxKeys k;
+    for (int r = 0; r < 10; ++r) {
+        k.k0[r] = seed_lo + (uint32_t)r * 0x9E3779B9u;
+        k.k1[r] = seed_hi + (uint32_t)r * 0xBB67AE85u;
+    }
+    return k;
+}
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys& k,
+                                              uint32_t out[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+        const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+        c0 = h1 ^ c1 ^ k.k0[r];
+        c1 = l1;
+        c2 = h0 ^ c3 ^ k.k1[r];
+        c3 = l0;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
 // The same with a growing cache: hb units are written to HBM at birth during this step. c.y and c.z count every
 // unit born in the step as written to DRAM; each one that goes to HBM instead moves from |E^w| to |H^w|.
 __device__ __forceinline__ uint32_t step_cost_g(uint32_t hr, uint32_t mi, uint32_t mo, uint32_t hb, const StepC c,

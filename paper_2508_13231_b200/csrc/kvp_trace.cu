@@ -12,7 +12,7 @@ namespace {
 
 struct TraceK {
     uint32_t groups, n, steps, topk, W32;
-    uint32_t seed_lo, seed_hi;
+    PhiloxKeys keys;         // round keys of the seed
     int32_t rho_q, c_q, sigma_q, burst_jump;
     uint32_t burst_thr;
     const int32_t* base;
@@ -25,10 +25,10 @@ struct TraceK {
 
 // Irwin-Hall(8) noise with unit variance in Q16.16: the sum of the eight 16-bit halves of one Philox block, centred
 // and scaled by floor(). |result| <= 321,057, so 32 bits hold it; only the product needs 64.
-__device__ __forceinline__ int32_t noise_q16(uint32_t seed_lo, uint32_t seed_hi, uint32_t u, uint32_t t)
+__device__ __forceinline__ int32_t noise_q16(const PhiloxKeys& keys, uint32_t u, uint32_t t)
 {
     uint32_t r[4];
-    philox4x32_10(u, t, 0u, TAG_NOISE, seed_lo, seed_hi, r);
+    philox4x32_10(u, t, 0u, TAG_NOISE, keys, r);
     uint32_t sum = 0;
 #pragma unroll
     for (int i = 0; i < 4; ++i) sum = __dp2a_lo(r[i], 0x0101u, sum);      // + low half + high half
@@ -168,12 +168,12 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
 // shifted and then cut to 32 bits (the range check on the host keeps the true value inside them).
 __device__ __forceinline__ int32_t next_state(const TraceK& k, uint32_t u, uint32_t t, int32_t x)
 {
-    const int32_t e = noise_q16(k.seed_lo, k.seed_hi, u, t);
+    const int32_t e = noise_q16(k.keys, u, t);
     const int64_t acc = t == 0 ? (int64_t)k.sigma_q * e : (int64_t)k.rho_q * x + (int64_t)k.c_q * e;
     int32_t xn = (int32_t)(acc >> 16);
     if (k.burst_thr) {
         uint32_t r[4];
-        philox4x32_10(u, t, 0u, TAG_BURST, k.seed_lo, k.seed_hi, r);
+        philox4x32_10(u, t, 0u, TAG_BURST, k.keys, r);
         if (r[0] < k.burst_thr) xn += k.burst_jump;
     }
     return xn;
@@ -293,7 +293,7 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
     TraceK k;
     k.groups = tp->groups; k.n = tp->units_per_group; k.steps = tp->steps; k.topk = tp->topk;
     k.W32 = (uint32_t)((U64 + 31) / 32);
-    k.seed_lo = (uint32_t)tp->seed; k.seed_hi = (uint32_t)(tp->seed >> 32);
+    k.keys = philox_keys((uint32_t)tp->seed, (uint32_t)(tp->seed >> 32));
     k.rho_q = tp->rho_q; k.c_q = tp->c_q; k.sigma_q = tp->sigma_q; k.burst_jump = tp->burst_jump;
     k.burst_thr = tp->burst_thr; k.base = tp->base; k.out = access_bitmaps;
     k.aligned = tp->units_per_group % 32 == 0;

@@ -33,7 +33,7 @@ UNIT = "move-evals/s"
 ISSUE_PEAK_GWIPS = 148 * 4 * 1.965
 # dram__bytes_read.sum + dram__bytes_write.sum of one chain-kernel launch on this workload (ncu capture summarised in
 # profiles/chain_kernel_single_head.md; set to None whenever the kernel changes until it is captured again)
-CHAIN_KERNEL_DRAM_BYTES = 360704
+CHAIN_KERNEL_DRAM_BYTES = 378368
 ALG_WARP_INSTR_PER_MOVE = 16.0
 
 

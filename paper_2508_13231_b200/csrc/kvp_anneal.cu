@@ -38,6 +38,7 @@ struct ChainParams {
     uint32_t* undo_len;          // [slots] how many there were (more than undo_cap: the log overflowed)
     uint32_t undo_cap;
     uint32_t* err;               // set to 1 by a warp that gave up waiting for its turn
+    uint32_t drop_first_turn;    // test hook: the owner of batch 0 never passes the turn on, so the next wait runs out
     const uint32_t* birth;       // growing cache: [U] step at which a unit is written (0 = there from the start)
     const uint32_t* hb0;         // growing cache: [S] units written to HBM at birth under the initial schedule
     CostK K;
@@ -533,7 +534,7 @@ chain_kernel(const ChainParams prm)
             }
             sh->n_acc[sub] = n_acc; sh->n_inf[sub] = n_inf;
             __threadfence_block();
-            st_volatile_u32(&sh->turn, b + 1u);
+            if (!(prm.drop_first_turn && b == 0)) st_volatile_u32(&sh->turn, b + 1u);
         }
         have = false;
     };
@@ -1093,6 +1094,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     prm.table = c.table; prm.shifts = c.shifts; prm.ws = c.slots; prm.K = p->K; prm.full0 = c.full0;
     prm.birth = p->d_birth; prm.hb0 = c.hb0;
     prm.err = reinterpret_cast<uint32_t*>(c.small + 16);
+    // KVP_TEST_DROP_TURN=1 (tests of the bounded wait only): one hand-over per chain is withheld, the waiting warp
+    // gives up after its poll limit (about a second) and the call returns KVP_ERR_TIMEOUT
+    if (const char* e = getenv("KVP_TEST_DROP_TURN")) prm.drop_first_turn = e[0] == '1' && !e[1];
     KVP_CUDA(cudaMemsetAsync(prm.err, 0, 4, st));
     prm.U = p->U; prm.S = p->S; prm.S32 = p->S32; prm.cap = p->cap;
     prm.levels = a->levels; prm.p_swap_256 = a->p_swap_256; prm.len_choices = a->max_len_log2 + 1;

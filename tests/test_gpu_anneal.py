@@ -199,3 +199,17 @@ def test_global_state_winner_paths(kvp, oracle, warps_per_chain):
         ref, _, bst = o.anneal_chains(op, w, 1, want_best=True)
         assert ref[0].astuple() == out["per_chain"][w].astuple()
         assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
+
+
+def test_turn_wait_is_bounded(kvp, oracle, monkeypatch):
+    """A hand-over that never comes: the waiting warp gives up after its poll limit (about a second), kvp_anneal
+    returns KVP_ERR_TIMEOUT instead of holding the GPU, and the next call on the same problem is exact again."""
+    g, o, cfg, A = named_problem(kvp, oracle, "tiny")
+    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", "2")
+    monkeypatch.setenv("KVP_TEST_DROP_TURN", "1")
+    with pytest.raises(kvp.KvpError) as e:
+        g.anneal(g.make_params(chains=4, moves=1000, seed=0))
+    assert e.value.code == kvp.ERR_TIMEOUT
+    monkeypatch.delenv("KVP_TEST_DROP_TURN")
+    gp, op = _params(g, o, chains=4, moves=1000, seed=0)
+    _check_against_oracle(g, o, gp, op)

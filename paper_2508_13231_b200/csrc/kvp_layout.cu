@@ -66,22 +66,41 @@ __global__ void __launch_bounds__(1024)
 static_freq_kernel(const uint32_t* __restrict__ ucnt, const uint32_t* __restrict__ hist, uint32_t U, uint32_t S,
                    uint32_t cap, uint32_t* __restrict__ row, uint32_t W32)
 {
-    __shared__ uint32_t s_thr, s_take, s_base;
+    __shared__ uint32_t s_thr, s_take, s_base, s_found;
     __shared__ uint32_t s_warp[32];
-    if (threadIdx.x == 0) {
-        uint32_t above = 0, thr = S + 1, take = 0;
-        // counts run 0..S; descend until the capacity is reached
-        for (int64_t c = S; c >= 0; --c) {
-            const uint32_t h = hist[c];
-            if (above + h >= cap) { thr = (uint32_t)c; take = cap - above; break; }
-            above += h;
-        }
-        if (cap == 0) { thr = S + 1; take = 0; }
-        s_thr = thr; s_take = take; s_base = 0;
-    }
-    __syncthreads();
-    const uint32_t thr = s_thr, take = s_take;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { s_thr = S + 1; s_take = 0; s_base = 0; s_found = 0; }
+    __syncthreads();
+    // counts run 0..S; descend, 1024 counts at a time (thread i looks at count top - i), until the capacity is reached
+    if (cap != 0) {
+        uint32_t above = 0;                               // units with a count above this chunk
+        for (int64_t top = S; top >= 0; top -= 1024) {
+            const int64_t c = top - (int64_t)threadIdx.x;
+            const uint32_t h = c >= 0 ? hist[c] : 0u;
+            uint32_t incl = h;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= (uint32_t)off) incl += v;
+            }
+            if (lane == 31) s_warp[warp] = incl;
+            __syncthreads();
+            uint32_t before = 0, total = 0;
+            for (uint32_t w = 0; w < 32; ++w) {
+                const uint32_t v = s_warp[w];
+                before += w < warp ? v : 0u;
+                total += v;
+            }
+            incl += before + above;
+            const uint32_t excl = incl - h;
+            if (c >= 0 && excl < cap && incl >= cap) { s_thr = (uint32_t)c; s_take = cap - excl; s_found = 1; }   // one thread at most
+            __syncthreads();
+            if (s_found) break;
+            above += total;
+            __syncthreads();
+        }
+    }
+    const uint32_t thr = s_thr, take = s_take;
     const uint32_t Upad = W32 * 32;
     for (uint32_t u0 = 0; u0 < Upad; u0 += 1024) {
         const uint32_t u = u0 + threadIdx.x;

@@ -229,18 +229,45 @@ trace_kernel(const TraceK k)
     }
 }
 
-// Two-pass form, pass 1: the AR(1) recurrence is sequential in time but independent across units, so one
-// thread per unit writes the whole score column; scores [steps][U].
-__global__ void __launch_bounds__(128)
+// Two-pass form, pass 1: scores [steps][U]. The random draws of a (unit, step) pair depend on nothing else, only the
+// AR(1) recurrence is sequential in time. A CTA owns 32 consecutive units and walks the steps in segments: all its
+// threads draw the segment's noise (and burst decisions) into shared memory, then one warp, a lane per unit, runs
+// the recurrence over the segment and writes 128 contiguous bytes per step.
+constexpr uint32_t kScoreSeg = 256, kScoreThreads = 512;
+
+__global__ void __launch_bounds__(kScoreThreads)
 trace_scores_kernel(const TraceK k, uint32_t U, int32_t* __restrict__ scores)
 {
-    const uint32_t u = blockIdx.x * blockDim.x + threadIdx.x;
-    if (u >= U) return;
-    const int32_t b = k.base ? __ldg(k.base + u) : 0;
-    int32_t x = 0;
-    for (uint32_t t = 0; t < k.steps; ++t) {
-        x = next_state(k, u, t, x);
-        scores[(size_t)t * U + u] = x + b;
+    __shared__ int32_t draw[kScoreSeg][32];              // noise << 1 | burst
+    const uint32_t u0 = blockIdx.x * 32, tid = threadIdx.x;
+    const uint32_t ul = tid & 31, u = u0 + ul;
+    int32_t x = 0, b = 0;
+    if (tid < 32 && u < U && k.base) b = __ldg(k.base + u);
+    for (uint32_t t0 = 0; t0 < k.steps; t0 += kScoreSeg) {
+        const uint32_t len = min(kScoreSeg, k.steps - t0);
+        for (uint32_t tt = tid >> 5; tt < len; tt += kScoreThreads / 32) {
+            if (u < U) {
+                int32_t d = noise_q16(k.keys, u, t0 + tt) * 2;
+                if (k.burst_thr) {
+                    uint32_t r[4];
+                    philox4x32_10(u, t0 + tt, 0u, TAG_BURST, k.keys, r);
+                    d |= r[0] < k.burst_thr ? 1 : 0;
+                }
+                draw[tt][ul] = d;
+            }
+        }
+        __syncthreads();
+        if (tid < 32 && u < U) {
+            for (uint32_t tt = 0; tt < len; ++tt) {
+                const int32_t d = draw[tt][ul], e = d >> 1;
+                const uint32_t t = t0 + tt;
+                const int64_t acc = t == 0 ? (int64_t)k.sigma_q * e : (int64_t)k.rho_q * x + (int64_t)k.c_q * e;
+                x = (int32_t)(acc >> 16);
+                if (d & 1) x += k.burst_jump;
+                scores[(size_t)t * U + u] = x + b;
+            }
+        }
+        __syncthreads();
     }
 }
 
@@ -313,7 +340,7 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
     if (tp->groups < 148 && score_bytes <= ((size_t)1 << 30) && !(tp->flags & KVP_TRACE_SINGLE_PASS) && !layered) {
         int32_t* scores = nullptr;
         KVP_CUDA(cudaMallocAsync(&scores, score_bytes, st));
-        trace_scores_kernel<<<(uint32_t)((U64 + 127) / 128), 128, 0, st>>>(k, (uint32_t)U64, scores);
+        trace_scores_kernel<<<(uint32_t)((U64 + 31) / 32), kScoreThreads, 0, st>>>(k, (uint32_t)U64, scores);
         dim3 grid(tp->groups, tp->steps);
         switch (upt) {
             case 1: trace_select_kernel<1><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;

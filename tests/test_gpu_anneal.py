@@ -213,3 +213,22 @@ def test_turn_wait_is_bounded(kvp, oracle, monkeypatch):
     monkeypatch.delenv("KVP_TEST_DROP_TURN")
     gp, op = _params(g, o, chains=4, moves=1000, seed=0)
     _check_against_oracle(g, o, gp, op)
+
+
+@pytest.mark.parametrize("name,p0", [("single_head", 1e-6), ("single_head", 0.3), ("layer_8b", 1e-6)])
+def test_two_warp_chains_repeat_exactly(kvp, oracle, monkeypatch, name, p0):
+    """Two warps per chain evaluate ahead of each other's commits, so their timing varies from run to run; the
+    results may not. All chains of the configuration, twenty runs, against one run with one warp per chain (which the
+    other tests compare with the oracle), at a cold and at a hot start (many applied moves, many re-evaluations)."""
+    g, o, cfg, A = named_problem(kvp, oracle, name)
+    moves = min(cfg["moves"], 50_000)
+    gp = g.make_params(chains=cfg["chains"], moves=moves, seed=3, p0=p0)
+    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", "1")
+    ref = g.anneal(gp, want_per_chain=True)
+    want = [r.astuple() for r in ref["per_chain"]]
+    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", "2")
+    for _ in range(20):
+        out = g.anneal(gp, want_per_chain=True)
+        assert [r.astuple() for r in out["per_chain"]] == want
+        assert out["best_ticks"] == ref["best_ticks"]
+        assert torch.equal(out["best_schedule"], ref["best_schedule"])

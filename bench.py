@@ -34,6 +34,8 @@ ISSUE_PEAK_GWIPS = 148 * 4 * 1.965
 # dram__bytes_read.sum + dram__bytes_write.sum of one chain-kernel launch on this workload (ncu capture summarised in
 # profiles/chain_kernel_single_head.md; set to None whenever the kernel changes until it is captured again)
 CHAIN_KERNEL_DRAM_BYTES = 378368
+# what that capture shows of the integer datapath (fractions of peak over the launch; context beside the timed figure)
+CHAIN_KERNEL_NCU = {"issue_active": 0.684, "alu_pipe": 0.575, "imad_pipe": 0.402, "warp_inst_per_move": 32.7}
 ALG_WARP_INSTR_PER_MOVE = 16.0
 
 
@@ -484,7 +486,7 @@ def main():
             "gpu_launches": launches[0] * args.steps,
             "roofline": {"bound": "alu", "kernel": "chain_kernel<smem>", "achieved": achieved,
                          "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
-                         "traffic": CHAIN_KERNEL_DRAM_BYTES, "ms_per_launch": per_launch_ms,
+                         "traffic": CHAIN_KERNEL_DRAM_BYTES, "ncu": CHAIN_KERNEL_NCU, "ms_per_launch": per_launch_ms,
                          "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"},
             "bound_ticks": out["best_ticks"], "init_ticks": out["stats"].init_ticks,
         }

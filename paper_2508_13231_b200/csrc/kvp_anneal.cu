@@ -39,6 +39,7 @@ struct ChainParams {
     uint32_t undo_cap;
     uint32_t* err;               // set to 1 by a warp that gave up waiting for its turn
     uint32_t drop_first_turn;    // test hook: the owner of batch 0 never passes the turn on, so the next wait runs out
+    uint32_t split_at;           // a batch with more queue items than this goes in two halves (kQueueCap / 2; less in tests)
     const uint32_t* birth;       // growing cache: [U] step at which a unit is written (0 = there from the start)
     const uint32_t* hb0;         // growing cache: [S] units written to HBM at birth under the initial schedule
     CostK K;
@@ -260,7 +261,7 @@ template <bool GROW, bool ASMEM>
 __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* __restrict__ Acol,
                                            const uint32_t* __restrict__ birth,
                                            const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
-                                           const uint32_t* __restrict__ trow, uint32_t shift,
+                                           const uint32_t* __restrict__ trow, uint32_t shift, uint32_t split_at,
                                            const uint32_t (&need)[kMPL], uint32_t lane, LaneMove (&mv)[kMPL])
 {
     uint32_t todo[kMPL], cnt = 0;
@@ -286,16 +287,9 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         pos += __popc(has & below) << bit;
         total += __popc(has) << bit;
     }
-    // ASMEM: the queue holds kQueueCap / 2 items, the worst case of 16 lanes. A batch with more (rare) goes in two
-    // halves, lanes 0..15 first.
-    const uint32_t halves = ASMEM && total > kQueueCap / 2 ? 2u : 1u;
-    const uint32_t mid = halves > 1 ? __shfl_sync(0xFFFFFFFFu, pos, 16) : 0u;   // items of lanes 0..15
-    for (uint32_t half = 0; half < halves; ++half) {
-        const bool pushing = halves == 1 || (lane >> 4) == half;
-        const uint32_t first = half ? mid : 0u;                                  // queue position 0 is item `first`
-        const uint32_t count = halves == 1 ? total : (half ? total - mid : mid);
-        if (half) __syncwarp();
-        // queue the set bits of every mask; all 31 positions are tried so that no lane waits on a serial bit scan
+    // queue the set bits of every mask of the lanes named by `pushing`; all 31 positions are tried so that no lane
+    // waits on a serial bit scan. Item `first` goes to queue position 0.
+    auto push = [&](bool pushing, uint32_t first) {
 #pragma unroll
         for (int h = 0; h < kMPL; ++h) {
             const uint32_t td = pushing ? todo[h] : 0u;
@@ -309,11 +303,26 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
             }
         }
         __syncwarp();
-        // two items per lane and trip (the two evaluations are independent and overlap), one where 32 or fewer are left
+    };
+    // two items per lane and trip (the two evaluations are independent and overlap), one where 32 or fewer are left
+    auto work_off = [&](uint32_t count) {
         for (uint32_t base = 0; base < count; base += 64) {
             if (base + 32 < count) eval_items<GROW, ASMEM, 2>(cv, stepc, K, S, base, count, lane);
             else eval_items<GROW, ASMEM, 1>(cv, stepc, K, S, base, count, lane);
         }
+    };
+    if (!ASMEM || total <= split_at) {
+        push(true, 0u);
+        work_off(total);
+    } else {
+        // ASMEM: the queue holds kQueueCap / 2 items, the worst case of 16 lanes. A batch with more (rare) goes in two
+        // halves, lanes 0..15 first.
+        const uint32_t mid = __shfl_sync(0xFFFFFFFFu, pos, 16);   // items of lanes 0..15
+        push(lane < 16, 0u);
+        work_off(mid);
+        __syncwarp();
+        push(lane >= 16, mid);
+        work_off(total - mid);
     }
     __syncwarp();
 #pragma unroll
@@ -586,7 +595,7 @@ chain_kernel(const ChainParams prm)
                 todo[h] = left >= 32 ? 0xFFFFFFFFu : (1u << left) - 1u;
                 need[h] = todo[h];
             }
-            eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+            eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv);
 #pragma unroll
             for (int h = 0; h < kMPL; ++h) need[h] = 0;
             if (W > 1) {
@@ -642,7 +651,7 @@ chain_kernel(const ChainParams prm)
 #pragma unroll
                 for (int h = 0; h < kMPL; ++h) any_need |= need[h];
                 if (any_need)
-                    eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+                    eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv);
                 bool applied = false;
 #pragma unroll
                 for (int h = 0; h < kMPL; ++h) need[h] = 0;
@@ -1097,6 +1106,13 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     // KVP_TEST_DROP_TURN=1 (tests of the bounded wait only): one hand-over per chain is withheld, the waiting warp
     // gives up after its poll limit (about a second) and the call returns KVP_ERR_TIMEOUT
     if (const char* e = getenv("KVP_TEST_DROP_TURN")) prm.drop_first_turn = e[0] == '1' && !e[1];
+    // KVP_TEST_SPLIT_QUEUE=n (tests only): batches with more than n < 496 queue items already take the two-halves
+    // path of the half-size work queue, which ordinary inputs almost never reach
+    prm.split_at = kQueueCap / 2;
+    if (const char* e = getenv("KVP_TEST_SPLIT_QUEUE")) {
+        const long v = atol(e);
+        if (v >= 0 && v < (long)(kQueueCap / 2)) prm.split_at = (uint32_t)v;
+    }
     KVP_CUDA(cudaMemsetAsync(prm.err, 0, 4, st));
     prm.U = p->U; prm.S = p->S; prm.S32 = p->S32; prm.cap = p->cap;
     prm.levels = a->levels; prm.p_swap_256 = a->p_swap_256; prm.len_choices = a->max_len_log2 + 1;

@@ -232,3 +232,21 @@ def test_two_warp_chains_repeat_exactly(kvp, oracle, monkeypatch, name, p0):
         assert [r.astuple() for r in out["per_chain"]] == want
         assert out["best_ticks"] == ref["best_ticks"]
         assert torch.equal(out["best_schedule"], ref["best_schedule"])
+
+
+@pytest.mark.parametrize("split", ["0", "20", "64"])
+def test_work_queue_in_two_halves(kvp, oracle, monkeypatch, split, warps_per_chain):
+    """Chains in shared memory with the access bitmap staged beside them keep half a work queue and work a batch
+    with more items than it holds off in two halves. Ordinary inputs never fill it, so the hook lowers the limit:
+    dense accesses, a churning initial schedule and a hot start give batches of a few hundred items."""
+    monkeypatch.setenv("KVP_TEST_SPLIT_QUEUE", split)
+    U, S, cap = 64, 200, 32
+    A = wl.random_access(U, S, 0.5, seed=9)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    init = wl.random_schedules(U, S, cap, 1, seed=4, churn=0.5)[0]
+    kw = dict(chains=6, moves=2500, levels=5, p0=0.5, p_swap_256=200)
+    gp = g.make_params(init_mode=kvp.INIT_USER, init_schedule=to_dev(init), **kw)
+    op = o.make_params(init_mode=oracle.INIT_USER, init_schedule=init, **kw)
+    _check_against_oracle(g, o, gp, op)
+    gp, op = _params(g, o, chains=6, moves=2500, levels=5, p0=1e-3)
+    _check_against_oracle(g, o, gp, op)

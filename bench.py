@@ -135,7 +135,7 @@ def cpu_baseline(cfg, tp):
 
 
 def run_cost_kernel(args):
-    """The cost kernel alone on the rows of the largest configuration: HBM roofline.
+    """The cost kernel alone (Eq. 1-5 over a batch of schedules) on the rows of the largest configuration: HBM roofline.
 
     A batch of schedules of long_70b (81,920 words per row, 64 rows, 20 MB each) is scored by kvp_eval; the
     batch plus the access bitmap is larger than L2. Algorithmic bytes: every placement word once and the access
@@ -201,7 +201,7 @@ def trace_alg_thread_instr(bursts):
 
 
 def run_trace_kernel(args):
-    """The trace kernel alone on the largest configuration: plain-ALU (issue-slot) roofline.
+    """The trace kernel alone (synthetic access sets) on the largest configuration: plain-ALU (issue-slot) roofline.
 
     long_70b: 640 groups of 4096 units, 64 steps, k = 205, bursts on; the fused single-pass kernel (one CTA per
     group). The output (S * W32 * 4 = 21 MB, plus 4 bytes per unit where a configuration has base scores) is the
@@ -246,7 +246,7 @@ def run_trace_kernel(args):
 
 
 def run_growing(args):
-    """The whole path on a growing cache with (token, layer) steps, configuration growing_8b:
+    """The whole path on a growing cache with (token, layer) steps (Section III-A), configuration growing_8b:
     layered trace with births -> kvp_create + kvp_set_births -> kvp_eval of 4 schedules -> kvp_anneal.
 
     The chains' schedules (17 MB each) live in global memory; the oracle is timed on a few chains beside it.

@@ -128,7 +128,7 @@ class Problem:
             _chk(lib().kvpo_set_births(self._h, _u32p(self.birth)), "set_births")
 
     def __del__(self):
-        if getattr(self, "_h", None) is not None and self._h:
+        if getattr(self, "_h", None) is not None and self._h and lib is not None:   # lib is None at interpreter exit
             lib().kvpo_destroy(self._h)
             self._h = None
 

@@ -43,6 +43,15 @@ def test_host_only_entry_points(lib, oracle):
     assert rc == 0
     otable, oshifts = oracle.accept_table(temps)
     assert np.array_equal(table, otable) and np.array_equal(shifts, oshifts)
+    # long ladders are built by several host threads, rows split unevenly when the level count is no multiple
+    for levels, c0, alpha in ((64, 54321.0, 0.9), (100, 7.5e6, 0.83), (17, 3.0, 0.5)):
+        temps = c0 * alpha ** np.arange(levels, dtype=np.float64)
+        table = np.zeros((levels, 1024), np.uint32)
+        shifts = np.zeros(levels, np.uint32)
+        assert lib.kvp_accept_table(temps.ctypes.data_as(ctypes.c_void_p), ctypes.c_uint32(levels),
+                                    table.ctypes.data_as(ctypes.c_void_p), shifts.ctypes.data_as(ctypes.c_void_p)) == 0
+        otable, oshifts = oracle.accept_table(temps)
+        assert np.array_equal(table, otable) and np.array_equal(shifts, oshifts)
     lib.kvp_strerror.restype = ctypes.c_char_p
     assert lib.kvp_strerror(0) == b"ok" and b"capacity" in lib.kvp_strerror(-2)
     assert lib.kvp_accept_table(None, 1, None, None) == -1

@@ -257,27 +257,34 @@ __device__ __forceinline__ void eval_items(const ChainView cv, const StepC* __re
 // prepares its own proposals, the (proposal, step) pairs whose cost changes are queued in shared memory, and
 // the warp works the queue off 32 pairs at a time, so that lanes with short and long proposals carry the
 // same load.
-template <bool GROW, bool ASMEM>
+// ALL: every lane prepares its proposal whether `need` names it or not (its items are dropped if not), so that this
+// part is straight-line code; `side_work` is then scheduled into it by the compiler (the draw of the next batch: a
+// long chain of dependent integer operations that fills the issue slots the window loads leave empty).
+template <bool GROW, bool ASMEM, bool ALL, typename SideWork>
 __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* __restrict__ Acol,
                                            const uint32_t* __restrict__ birth,
                                            const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
                                            const uint32_t* __restrict__ trow, uint32_t shift, uint32_t split_at,
-                                           const uint32_t (&need)[kMPL], uint32_t lane, LaneMove (&mv)[kMPL])
+                                           const uint32_t (&need)[kMPL], uint32_t lane, LaneMove (&mv)[kMPL],
+                                           SideWork&& side_work)
 {
     uint32_t todo[kMPL], cnt = 0;
 #pragma unroll
     for (int h = 0; h < kMPL; ++h) {
         todo[h] = 0;
-        if ((need[h] >> lane) & 1u) {
+        const bool named = (need[h] >> lane) & 1u;
+        if (ALL || named) {
             const uint32_t slot = h * 32 + lane;
             Windows wn;
-            todo[h] = lane_windows<GROW>(cv.P, Acol, cv.full, birth, S, S32, mv[h], wn);
+            const uint32_t tm = lane_windows<GROW>(cv.P, Acol, cv.full, birth, S, S32, mv[h], wn);
+            todo[h] = named ? tm : 0u;
             cv.win[slot * 2] = make_uint4(wn.Wu, wn.Wv, wn.Nu, wn.Nv);
             cv.win[slot * 2 + 1] = make_uint4(wn.Au, wn.Av, wn.s0, wn.born);
             cv.acc[slot] = 0;
         }
         cnt += __popc(todo[h]);
     }
+    side_work();
     // exclusive prefix sum of cnt over the lanes, bit-sliced: the five ballots do not depend on one another
     uint32_t pos = 0, total = 0;
     const uint32_t below = (1u << lane) - 1u;
@@ -572,6 +579,9 @@ chain_kernel(const ChainParams prm)
         // against the current state; the warp then commits them in move order. A move that changes the schedule
         // invalidates only later moves whose step windows overlap its own; those are evaluated again before their
         // turn comes, so the outcome is that of the sequential chain.
+        bool have_next = false;                                   // `next` holds the draw of the batch about to start
+        LaneMove next;
+        next.pk = next.u = next.v = next.w = 0u; next.delta = 0; next.inf = next.acc = next.chg = false;
         for (uint32_t bi = (sub - base) & (W - 1); bi < nbat; bi += W) {
             const uint64_t m = lvl_start + (uint64_t)bi * kBatch;
             const uint32_t nb = bi + 1 < nbat ? kBatch : last_nb;
@@ -582,20 +592,30 @@ chain_kernel(const ChainParams prm)
                 n0 = __shfl_sync(0xFFFFFFFFu, ld_volatile_u32(&sh->napplied), 0);
                 __threadfence_block();
             }
+            static_assert(kMPL == 1, "the draw of the next batch is carried in one LaneMove");
             LaneMove mv[kMPL];
             uint32_t todo[kMPL], need[kMPL];
-#pragma unroll
-            for (int h = 0; h < kMPL; ++h) {
+            if (have_next) {
+                mv[0] = next;
+            } else {
                 uint32_t r[4];
-                const uint64_t mine = m + 32u * h + lane;
+                const uint64_t mine = m + lane;
                 philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.keys, r);
-                decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv[h]);
-                mv[h].inf = false; mv[h].acc = false; mv[h].chg = false; mv[h].delta = 0;
-                const uint32_t left = nb > 32u * h ? nb - 32u * h : 0u;
-                todo[h] = left >= 32 ? 0xFFFFFFFFu : (1u << left) - 1u;
-                need[h] = todo[h];
+                decode_move(r, prm.p_swap_256, prm.len_choices, S, U, mv[0]);
             }
-            eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv);
+            mv[0].inf = false; mv[0].acc = false; mv[0].chg = false; mv[0].delta = 0;
+            todo[0] = nb >= 32 ? 0xFFFFFFFFu : (1u << nb) - 1u;
+            need[0] = todo[0];
+            // the proposals of this warp's next batch of the level are drawn while this batch's windows are loaded
+            // (drawn, and dropped, even where the level has no further batch for this warp)
+            eval_batch<GROW, ASMEM, true>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv,
+                                          [&]() {
+                                              uint32_t r[4];
+                                              const uint64_t mine = m + (uint64_t)W * kBatch + lane;
+                                              philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.keys, r);
+                                              decode_move(r, prm.p_swap_256, prm.len_choices, S, U, next);
+                                          });
+            have_next = bi + W < nbat;
 #pragma unroll
             for (int h = 0; h < kMPL; ++h) need[h] = 0;
             if (W > 1) {
@@ -651,7 +671,8 @@ chain_kernel(const ChainParams prm)
 #pragma unroll
                 for (int h = 0; h < kMPL; ++h) any_need |= need[h];
                 if (any_need)
-                    eval_batch<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv);
+                    eval_batch<GROW, ASMEM, false>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv,
+                                                   []() {});
                 bool applied = false;
 #pragma unroll
                 for (int h = 0; h < kMPL; ++h) need[h] = 0;

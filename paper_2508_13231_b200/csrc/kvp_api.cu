@@ -25,7 +25,7 @@ int set_cuda_error(cudaError_t e, const char* what)
 // device-wide synchronisation. The default pool is told to keep freed memory up to the largest block this
 // library has asked for on the device so far (at least 1 GiB), so that the next problem of the same size
 // gets its workspace back without a trip to the driver.
-static int retain_in_pool(int device, size_t bytes)
+int retain_in_pool(int device, size_t bytes)
 {
     static uint64_t kept[64];                // racing threads may both raise the threshold; either value is fine
     if (device < 0 || device >= 64) return KVP_OK;

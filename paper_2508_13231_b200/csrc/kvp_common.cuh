@@ -144,6 +144,8 @@ int set_cuda_error(cudaError_t e, const char* what);
         if (e_ != cudaSuccess) return kvp::set_cuda_error(e_, #call);    \
     } while (0)
 
+// keep freed blocks of up to `bytes` (+ 1 GiB) in the device's default memory pool
+int retain_in_pool(int device, size_t bytes);
 int ensure_scratch(kvp_problem* p, size_t bytes, cudaStream_t st);
 int ensure_chain_ws(kvp_problem* p, size_t bytes, cudaStream_t st);
 

@@ -1,9 +1,9 @@
 // Trace kernels: synthetic importance per unit and step, top-k per (layer, kv-head) group, packed into uint32
-// bitmaps. Two passes when there are few groups: one thread per unit runs the AR(1) recurrence over all steps
-// (sequential in time) and writes a score matrix; then one CTA per (group, step) finds the k-th largest score
-// digit by digit with shared-memory histograms, ties going to the lower unit index. A fused single-pass form
-// (one CTA per group walking the steps, state in registers) serves traces with many groups, layered or growing
-// traces and those whose score matrix would exceed the scratch budget.
+// bitmaps. Two passes by default: the first writes a score matrix (the draws in parallel over units and steps, the
+// AR(1) recurrence, sequential in time, by one lane per unit); then one CTA per (group, step) finds the k-th largest
+// score digit by digit with shared-memory histograms, ties going to the lower unit index. A fused single-pass form
+// (one CTA per group walking the steps, state in registers) serves layered or growing traces and those whose score
+// matrix would exceed the scratch budget.
 #include "kvp_common.cuh"
 
 namespace kvp {
@@ -333,20 +333,32 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
     const int upt = n <= 1024 ? 1 : n <= 2048 ? 2 : n <= 4096 ? 4 : 8;
     uint32_t T = (n + upt - 1) / upt;
     T = (T + 31) / 32 * 32;
-    // Two passes (scores, then one CTA per (group, step)) when the fused kernel, which has only `groups` CTAs and
-    // walks the steps one after the other, could not fill the 148 SMs, and the score matrix fits a 1 GiB scratch.
-    // With many groups the fused form is faster (measured: 1.9 vs 3.0 ms on 256 groups, 3.9 vs 6.5 ms on 640).
+    // Two passes (scores, then one CTA per (group, step)) whenever the score matrix fits a 1 GiB scratch: the work
+    // then comes in tens of thousands of equal pieces, while the fused kernel has only `groups` CTAs that walk the
+    // steps one after the other (measured: 0.84 vs 0.89 ms on 256 groups of 2048, 1.85 vs 2.11 ms on 640 of 4096,
+    // 0.05 vs 2.1 ms on one group of 256).
     const size_t score_bytes = (size_t)U64 * tp->steps * 4;
-    if (tp->groups < 148 && score_bytes <= ((size_t)1 << 30) && !(tp->flags & KVP_TRACE_SINGLE_PASS) && !layered) {
+    if (score_bytes <= ((size_t)1 << 30) && !(tp->flags & KVP_TRACE_SINGLE_PASS) && !layered) {
         int32_t* scores = nullptr;
+        int dev = 0;
+        KVP_CUDA(cudaGetDevice(&dev));
+        int prc = retain_in_pool(dev, score_bytes);          // the next call gets the block back from the pool
+        if (prc) return prc;
         KVP_CUDA(cudaMallocAsync(&scores, score_bytes, st));
         trace_scores_kernel<<<(uint32_t)((U64 + 31) / 32), kScoreThreads, 0, st>>>(k, (uint32_t)U64, scores);
         dim3 grid(tp->groups, tp->steps);
-        switch (upt) {
-            case 1: trace_select_kernel<1><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
-            case 2: trace_select_kernel<2><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
-            case 4: trace_select_kernel<4><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
-            default: trace_select_kernel<8><<<grid, T, 0, st>>>(k, (uint32_t)U64, scores); break;
+        // Small CTAs with many units per thread: a selection is a chain of barriers and a serial histogram walk, so
+        // what counts is how many of them an SM overlaps (whole call, 640 groups of 4096 units x 64 steps: 1.85 ms
+        // with 1024 threads, 1.70 ms with 256; 256 groups of 2048 x 128 steps: 0.84 against 0.61 ms with 128).
+        int su = 1;
+        while (su < 16 && (n + su - 1) / su > 128) su *= 2;
+        const uint32_t ST = ((n + su - 1) / su + 31) / 32 * 32;
+        switch (su) {
+            case 1: trace_select_kernel<1><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
+            case 2: trace_select_kernel<2><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
+            case 4: trace_select_kernel<4><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
+            case 8: trace_select_kernel<8><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
+            default: trace_select_kernel<16><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
         }
         cudaError_t le = cudaGetLastError();
         KVP_CUDA(cudaFreeAsync(scores, st));

@@ -203,9 +203,9 @@ def trace_alg_thread_instr(bursts):
 def run_trace_kernel(args):
     """The trace kernel alone (synthetic access sets) on the largest configuration: plain-ALU (issue-slot) roofline.
 
-    long_70b: 640 groups of 4096 units, 64 steps, k = 205, bursts on; the fused single-pass kernel (one CTA per
-    group). The output (S * W32 * 4 = 21 MB, plus 4 bytes per unit where a configuration has base scores) is the
-    only memory traffic, reported as GB/s beside the instruction rate.
+    long_70b: 640 groups of 4096 units, 64 steps, k = 205, bursts on; two passes (scores, then one selection per
+    group and step). Memory traffic: the int32 score matrix written once and read once (2 * U * S * 4 = 1.3 GB) and
+    the output (S * W32 * 4 = 21 MB), reported as GB/s beside the instruction rate.
     """
     import torch
     from paper_2508_13231_b200 import kvp, workloads as wl
@@ -235,14 +235,14 @@ def run_trace_kernel(args):
     alg = trace_alg_thread_instr(bool(tp.get("burst_thr"))) / 32.0 * U * S           # warp instructions
     achieved = alg / (ms * 1e-3) / 1e9
     print(json.dumps({
-        "kernel": "trace_kernel (kvp_trace_generate)", "metric": "unit_steps_per_sec", "value": U * S / (ms * 1e-3),
+        "kernel": "trace_scores_kernel + trace_select_kernel (kvp_trace_generate)", "metric": "unit_steps_per_sec", "value": U * S / (ms * 1e-3),
         "unit": "unit-steps/s", "ms_per_call": ms, "steps": args.steps,
         "config": {"workload": name, "groups": cfg["groups"], "units_per_group": cfg["units_per_group"], "rows": S,
                    "topk": cfg["topk"], "l2": "flushed with a 256 MB write between timed iterations"},
         "roofline": {"bound": "alu", "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s",
                      "frac": achieved / ISSUE_PEAK_GWIPS, "traffic": None,
                      "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)",
-                     "memory_gbs": (S * W32 * 4 + (U * 4 if base is not None else 0)) / (ms * 1e-3) / 1e9}}))
+                     "memory_gbs": (2 * U * S * 4 + S * W32 * 4 + (U * 4 if base is not None else 0)) / (ms * 1e-3) / 1e9}}))
 
 
 def run_growing(args):

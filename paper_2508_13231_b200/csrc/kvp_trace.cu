@@ -74,7 +74,8 @@ __device__ __forceinline__ void select_reset(SelectSmem& sm)
 // agree with K in the bits fixed so far are counted per digit in a shared-memory histogram, and one warp walks
 // the histogram from the top until the counts reach what is still needed. The bits above the highest one in which
 // the largest and the smallest key differ are common to all keys and need no pass: three passes on these scores.
-template <int UPT>
+// FULL: the CTA's UPT * T slots are exactly the n units, so no slot needs a bounds test.
+template <int UPT, bool FULL = false>
 __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const TraceK& k, uint32_t topk, uint32_t gbase,
                                             uint32_t t, SelectSmem& sm)
 {
@@ -82,7 +83,7 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
     uint32_t mx = 0u, mn = ~0u;
 #pragma unroll
     for (int j = 0; j < UPT; ++j)
-        if (j * T + tid < k.n) { mx = max(mx, key[j]); mn = min(mn, key[j]); }
+        if (FULL || j * T + tid < k.n) { mx = max(mx, key[j]); mn = min(mn, key[j]); }
     mx = __reduce_max_sync(0xFFFFFFFFu, mx);
     mn = __reduce_min_sync(0xFFFFFFFFu, mn);
     if (lane == 0) { atomicMax(&sm.hi, mx); atomicMin(&sm.lo, mn); }
@@ -95,7 +96,7 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
         uint32_t* hist = sm.hist[pass];
 #pragma unroll
         for (int j = 0; j < UPT; ++j) {
-            const bool in = j * T + tid < k.n && (rem >= 32 || (key[j] >> rem) == (K >> rem));
+            const bool in = (FULL || j * T + tid < k.n) && (rem >= 32 || (key[j] >> rem) == (K >> rem));
             if (in) atomicAdd(hist + ((key[j] >> sh) & ((1u << w) - 1u)), 1u);
         }
         __syncthreads();
@@ -137,7 +138,7 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
 #pragma unroll
     for (int j = 0; j < UPT; ++j) {
         const uint32_t i = j * T + tid;
-        const bool ok = i < k.n;
+        const bool ok = FULL || i < k.n;
         const bool tie = ok && key[j] == K;
         bool pick = ok && key[j] > K;
         if (!rank_ties) {
@@ -157,7 +158,7 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
         }
         if (k.aligned) {
             const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
-            if (lane == 0 && j * T + (tid & ~31u) < k.n) row[(gbase + j * T + tid) >> 5] = bits;
+            if (lane == 0 && (FULL || j * T + (tid & ~31u) < k.n)) row[(gbase + j * T + tid) >> 5] = bits;
         } else if (pick) {
             atomicOr(row + ((gbase + i) >> 5), 1u << ((gbase + i) & 31));
         }
@@ -272,7 +273,7 @@ trace_scores_kernel(const TraceK k, uint32_t U, int32_t* __restrict__ scores)
 }
 
 // Two-pass form, pass 2: the top-k selections of different steps are independent: one CTA per (group, step).
-template <int UPT>
+template <int UPT, bool FULL>
 __global__ void __launch_bounds__(1024)
 trace_select_kernel(const TraceK k, uint32_t U, const int32_t* __restrict__ scores)
 {
@@ -284,10 +285,10 @@ trace_select_kernel(const TraceK k, uint32_t U, const int32_t* __restrict__ scor
 #pragma unroll
     for (int j = 0; j < UPT; ++j) {
         const uint32_t i = j * T + tid;
-        key[j] = i < k.n ? (uint32_t)__ldg(scores + (size_t)t * U + gbase + i) ^ 0x80000000u : 0u;
+        key[j] = (FULL || i < k.n) ? (uint32_t)__ldg(scores + (size_t)t * U + gbase + i) ^ 0x80000000u : 0u;
     }
     __syncthreads();
-    select_step<UPT>(key, k, k.topk, gbase, t, sm);
+    select_step<UPT, FULL>(key, k, k.topk, gbase, t, sm);
 }
 
 }  // namespace
@@ -353,13 +354,18 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
         int su = 1;
         while (su < 16 && (n + su - 1) / su > 128) su *= 2;
         const uint32_t ST = ((n + su - 1) / su + 31) / 32 * 32;
+        const bool full = (uint64_t)su * ST == n;             // every slot of the CTA holds a unit
+#define KVP_SELECT(UPT)                                                                              \
+    if (full) trace_select_kernel<UPT, true><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores);         \
+    else trace_select_kernel<UPT, false><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores)
         switch (su) {
-            case 1: trace_select_kernel<1><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
-            case 2: trace_select_kernel<2><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
-            case 4: trace_select_kernel<4><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
-            case 8: trace_select_kernel<8><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
-            default: trace_select_kernel<16><<<grid, ST, 0, st>>>(k, (uint32_t)U64, scores); break;
+            case 1: KVP_SELECT(1); break;
+            case 2: KVP_SELECT(2); break;
+            case 4: KVP_SELECT(4); break;
+            case 8: KVP_SELECT(8); break;
+            default: KVP_SELECT(16); break;
         }
+#undef KVP_SELECT
         cudaError_t le = cudaGetLastError();
         KVP_CUDA(cudaFreeAsync(scores, st));
         KVP_CUDA(le);

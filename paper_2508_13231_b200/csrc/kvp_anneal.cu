@@ -49,6 +49,11 @@ struct ChainParams {
     uint32_t early_permille, early_from;
     PhiloxKeys keys;             // round keys of the seed
     uint64_t per_level, upto, init_ticks;
+    uint32_t* touch_log;         // if set: [slots][touch_cap] units whose schedule words the slot's chain has rewritten
+    uint32_t* touch_len;         // [slots] how many entries (more than touch_cap: the log overflowed)
+    uint32_t touch_cap;
+    uint32_t restore;            // the slices hold the final states of chains that started from the same initial
+                                 // schedule and logged what they touched: only those units are copied again
 };
 
 // Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
@@ -450,18 +455,22 @@ __device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p) { return 
 __device__ __forceinline__ void st_volatile_u32(uint32_t* p, uint32_t v) { *reinterpret_cast<volatile uint32_t*>(p) = v; }
 
 // shared-memory words (as uint4 slots) of one chain besides its schedule
-__host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool grow, uint32_t W, bool halfq)
+__host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool grow, uint32_t W, bool halfq, bool touch)
 {
-    return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (W > 1 ? kShareSlots4 : 0u) + W * priv_slots4(halfq);
+    return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (touch ? 1u : 0u) + (W > 1 ? kShareSlots4 : 0u) +
+           W * priv_slots4(halfq);
 }
 
 // ASMEM (only with PSMEM): the access bitmap and the per-step constants, which every chain of the CTA reads, are
 // staged in shared memory once per CTA. With the schedules in shared memory the L1 cache is down to its minimum and
 // cannot hold them.
-template <bool PSMEM, bool GROW, int W, bool ASMEM>
+// TOUCH (only without PSMEM): the chain logs the units it rewrites, and may start from a slice that holds the final
+// state of an earlier chain with such a log (ChainParams::restore).
+template <bool PSMEM, bool GROW, int W, bool ASMEM, bool TOUCH>
 __global__ void __launch_bounds__(512)
 chain_kernel(const ChainParams prm)
 {
+    static_assert(!TOUCH || !PSMEM, "touch logs only for schedules in global scratch");
     static_assert(W >= 1 && W <= kMaxW && (W & (W - 1)) == 0, "warps per chain");
     static_assert(PSMEM || !ASMEM, "shared access bitmap only beside shared schedules");
     extern __shared__ uint4 smem4[];
@@ -477,14 +486,16 @@ chain_kernel(const ChainParams prm)
     const size_t pwords = (size_t)U * S32;
     const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
     const uint32_t h4 = GROW ? (S + 3) / 4 : 0u;                  // uint4 slots of the written-to-HBM counts
-    const uint32_t fixed4 = chain_fixed4(S, S32, GROW, W, ASMEM);
+    const uint32_t fixed4 = chain_fixed4(S, S32, GROW, W, ASMEM, TOUCH);
+    constexpr uint32_t t4 = TOUCH ? 1u : 0u;
     uint4* const mine4 = smem4 + (size_t)cic * fixed4;
     ChainView cv;
     cv.ctr = mine4;
     cv.full = reinterpret_cast<uint32_t*>(mine4 + S);
     cv.hb = reinterpret_cast<uint32_t*>(mine4 + S + f4);
-    ChainShare* const sh = reinterpret_cast<ChainShare*>(mine4 + S + f4 + h4);
-    uint4* const priv4 = mine4 + S + f4 + h4 + (W > 1 ? kShareSlots4 : 0u) + sub * priv_slots4(ASMEM);
+    uint32_t* const touched = reinterpret_cast<uint32_t*>(mine4 + S + f4 + h4);   // TOUCH: entries in the chain's log
+    ChainShare* const sh = reinterpret_cast<ChainShare*>(mine4 + S + f4 + h4 + t4);
+    uint4* const priv4 = mine4 + S + f4 + h4 + t4 + (W > 1 ? kShareSlots4 : 0u) + sub * priv_slots4(ASMEM);
     cv.win = priv4;
     cv.acc = reinterpret_cast<int*>(priv4 + kWinSlots4);
     cv.queue = reinterpret_cast<uint16_t*>(priv4 + kWinSlots4 + kAccSlots4);
@@ -507,7 +518,20 @@ chain_kernel(const ChainParams prm)
         if (GROW)
             for (uint32_t i = tid; i < S; i += 32 * W) cv.hb[i] = __ldg(prm.hb0 + i);
         for (uint32_t i = lane; i < kWinSlots4; i += 32) cv.win[i] = make_uint4(0u, 0u, 0u, 0u);
-        copy_words(cv.P, prm.Pcol0, pwords, tid, 32 * W);
+        bool whole = true;
+        if (TOUCH && prm.restore) {
+            const uint32_t n = __ldcg(prm.touch_len + slot);
+            if (n <= prm.touch_cap) {
+                whole = false;
+                const uint32_t* tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
+                for (uint32_t i = tid; i < n; i += 32 * W) {
+                    const size_t o = (size_t)__ldcg(tlog + i) * S32;
+                    for (uint32_t w = 0; w < S32; ++w) cv.P[o + w] = __ldg(prm.Pcol0 + o + w);
+                }
+            }
+        }
+        if (whole) copy_words(cv.P, prm.Pcol0, pwords, tid, 32 * W);
+        if (TOUCH && tid == 0) *touched = 0u;
         if (W > 1 && tid == 0) {
             sh->cur = sh->best = sh->best_at_boundary = prm.init_ticks;
             sh->best_move = ~0ull; sh->n_chg = 0; sh->hash = 0;
@@ -706,6 +730,13 @@ chain_kernel(const ChainParams prm)
                     // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later
                     // proposal read steps s0 - 1 .. s0 + len: it has to be evaluated again iff the two ranges meet.
                     const uint32_t s0b = pk >> 8, endb = s0b + ((pk >> 1) & 63u);
+                    if (TOUCH && prm.touch_log && lane == 0) {   // the units whose words no longer are the initial ones
+                        uint32_t* const tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
+                        const uint32_t n = *touched, two = pk & 1u;
+                        if (n < prm.touch_cap) tlog[n] = bu;
+                        if (two && n + 1u < prm.touch_cap) tlog[n + 1u] = bv;
+                        *touched = min(n + 1u + two, prm.touch_cap + 1u);
+                    }
                     if (W > 1) {                                  // tell the warps that are evaluating later batches
                         if (lane == 0) {
                             sh->applog[napp % kLog] = s0b | (endb << 16);
@@ -751,6 +782,7 @@ chain_kernel(const ChainParams prm)
     }
     if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
     if (ulog && lane == 0) prm.undo_len[slot] = ulen;
+    if (TOUCH && prm.touch_log && lane == 0) prm.touch_len[slot] = *touched;
     if (lane == 0) {
         kvp_chain_result res;
         res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m_end;
@@ -906,6 +938,10 @@ struct Ctx {
     uint64_t* undo_log;      // undo logs (global variant), or null
     uint32_t* undo_len;
     uint32_t undo_cap;
+    uint32_t* touch_log;     // touched-unit logs (global variant), or null
+    uint32_t* touch_len;
+    uint32_t touch_cap;
+    bool touch;              // the chains come in several waves and log the units they rewrite
     bool psmem;
     uint32_t wpb;            // chains per CTA
     uint32_t wpc;            // warps per chain
@@ -932,34 +968,36 @@ int validate(const kvp_problem* p, const kvp_anneal_params* a)
 
 typedef void (*ChainKernel)(const ChainParams);
 
-template <bool PSMEM, bool ASMEM>
+template <bool PSMEM, bool ASMEM, bool TOUCH>
 ChainKernel chain_kernel_pick(bool grow, uint32_t W)
 {
-    if (W == 2) return grow ? chain_kernel<PSMEM, true, 2, ASMEM> : chain_kernel<PSMEM, false, 2, ASMEM>;
-    return grow ? chain_kernel<PSMEM, true, 1, ASMEM> : chain_kernel<PSMEM, false, 1, ASMEM>;
+    if (W == 2) return grow ? chain_kernel<PSMEM, true, 2, ASMEM, TOUCH> : chain_kernel<PSMEM, false, 2, ASMEM, TOUCH>;
+    return grow ? chain_kernel<PSMEM, true, 1, ASMEM, TOUCH> : chain_kernel<PSMEM, false, 1, ASMEM, TOUCH>;
 }
 
-ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W)
+ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W, bool touch)
 {
-    if (!psmem) return chain_kernel_pick<false, false>(grow, W);
-    return asmem ? chain_kernel_pick<true, true>(grow, W) : chain_kernel_pick<true, false>(grow, W);
+    if (!psmem) return touch ? chain_kernel_pick<false, false, true>(grow, W) : chain_kernel_pick<false, false, false>(grow, W);
+    return asmem ? chain_kernel_pick<true, true, false>(grow, W) : chain_kernel_pick<true, false, false>(grow, W);
 }
 
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 {
     const uint32_t grid = (count + c.wpb - 1) / c.wpb;
     const size_t smem = (size_t)c.wpb * c.smem_per_warp + c.smem_shared;
-    chain_kernel_for(c.psmem, c.asmem, c.grow, c.wpc)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
+    chain_kernel_for(c.psmem, c.asmem, c.grow, c.wpc, c.touch)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }
 
 int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp_chain_result* results, uint64_t upto,
-               uint32_t* dump, uint32_t* snap, bool with_undo = false)
+               uint32_t* dump, uint32_t* snap, bool with_undo = false, bool restore = false)
 {
     ChainParams prm = c.prm;
     prm.snap = snap;
     prm.undo_log = with_undo ? c.undo_log : nullptr; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
+    prm.touch_log = with_undo ? c.touch_log : nullptr; prm.touch_len = c.touch_len; prm.touch_cap = c.touch_cap;
+    prm.restore = with_undo && restore && c.touch_log ? 1u : 0u;
     prm.chain_first = first; prm.chain_count = count; prm.result_base = result_base;
     prm.results = results; prm.upto = upto; prm.dump = dump;
     ++c.launches;
@@ -984,9 +1022,10 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const size_t budget = (size_t)smem_max - 1024;
     // per chain: counters, full-step bitmap and, per warp, the batch's windows, accumulators and work queue
     c.grow = p->dL != nullptr;
-    auto fixed_bytes = [&](uint32_t W, bool halfq = false) {
-        return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq) * 16;
+    auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false) {
+        return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq, touch) * 16;
     };
+    c.touch = false;
     const size_t pbytes = (size_t)p->U * p->S32 * 4;
     // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
     // chains then keeps twice as many warps in flight. KVP_WARPS_PER_CHAIN=1|2 overrides the choice (for tuning).
@@ -1017,44 +1056,50 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
         } else {
             c.smem_shared = 0;
         }
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.asmem, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.asmem, c.grow, W, false), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
-        const size_t ctr_bytes = fixed_bytes(W);
-        if (ctr_bytes > budget) return KVP_ERR_RANGE;
-        c.smem_per_warp = ctr_bytes;
-        c.smem_shared = 0;
-        c.asmem = false;
-        c.wpc = W;
-        uint32_t wcap = (uint32_t)(budget / ctr_bytes);            // chains per CTA at most
-        if (wcap > 16 / W) wcap = 16 / W;
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, false, c.grow, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
-        int ctas = 0;
-        KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, false, c.grow, W), (int)(wcap * W * 32),
-                                                               wcap * c.smem_per_warp));
-        if (ctas < 1) return KVP_ERR_RANGE;
-        uint32_t per_sm = (uint32_t)ctas * wcap;                   // resident chains per SM, at most 32 warps
-        if (per_sm * W > 32) per_sm = 32 / W / wcap ? 32 / W / wcap * wcap : wcap;
-        size_t free_b = 0, total_b = 0;
-        KVP_CUDA(cudaMemGetInfo(&free_b, &total_b));
-        free_b += p->chain_ws_bytes;                               // what we already hold can be reused
-        {                                                          // and so can what the pool holds in reserve
-            cudaMemPool_t pool; uint64_t reserved = 0, used = 0;
-            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess &&
-                cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReservedMemCurrent, &reserved) == cudaSuccess &&
-                cudaMemPoolGetAttribute(pool, cudaMemPoolAttrUsedMemCurrent, &used) == cudaSuccess && reserved > used)
-                free_b += (size_t)(reserved - used);
+        // planned without the touch logs first; a job that then needs several waves is planned again with them (one
+        // more shared-memory slot per chain)
+        for (int pass = 0; pass < 2; ++pass) {
+            c.touch = pass == 1;
+            const size_t ctr_bytes = fixed_bytes(W, false, c.touch);
+            if (ctr_bytes > budget) return KVP_ERR_RANGE;
+            c.smem_per_warp = ctr_bytes;
+            c.smem_shared = 0;
+            c.asmem = false;
+            c.wpc = W;
+            uint32_t wcap = (uint32_t)(budget / ctr_bytes);            // chains per CTA at most
+            if (wcap > 16 / W) wcap = 16 / W;
+            KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, false, c.grow, W, c.touch), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+            int ctas = 0;
+            KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, false, c.grow, W, c.touch), (int)(wcap * W * 32),
+                                                                   wcap * c.smem_per_warp));
+            if (ctas < 1) return KVP_ERR_RANGE;
+            uint32_t per_sm = (uint32_t)ctas * wcap;                   // resident chains per SM, at most 32 warps
+            if (per_sm * W > 32) per_sm = 32 / W / wcap ? 32 / W / wcap * wcap : wcap;
+            size_t free_b = 0, total_b = 0;
+            KVP_CUDA(cudaMemGetInfo(&free_b, &total_b));
+            free_b += p->chain_ws_bytes;                               // what we already hold can be reused
+            {                                                          // and so can what the pool holds in reserve
+                cudaMemPool_t pool; uint64_t reserved = 0, used = 0;
+                if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess &&
+                    cudaMemPoolGetAttribute(pool, cudaMemPoolAttrReservedMemCurrent, &reserved) == cudaSuccess &&
+                    cudaMemPoolGetAttribute(pool, cudaMemPoolAttrUsedMemCurrent, &used) == cudaSuccess && reserved > used)
+                    free_b += (size_t)(reserved - used);
+            }
+            const size_t usable = free_b / 10 * 7;
+            size_t fit = usable / col_bytes;
+            if (fit < 1) return KVP_ERR_NOMEM;
+            size_t cap_r = (size_t)per_sm * sms;
+            size_t r = a->chains < cap_r ? a->chains : cap_r;
+            if (r > fit) r = fit;
+            const uint32_t waves = (uint32_t)((a->chains + r - 1) / r);
+            c.resident = (a->chains + waves - 1) / waves;              // equal waves
+            // a wave is spread over all SMs: CTAs of ceil(resident / SMs) chains where one CTA per SM holds them
+            const uint32_t even = (c.resident + sms - 1) / sms;
+            c.wpb = even < wcap ? even : wcap;
+            if (a->chains <= c.resident) break;
         }
-        const size_t usable = free_b / 10 * 7;
-        size_t fit = usable / col_bytes;
-        if (fit < 1) return KVP_ERR_NOMEM;
-        size_t cap_r = (size_t)per_sm * sms;
-        size_t r = a->chains < cap_r ? a->chains : cap_r;
-        if (r > fit) r = fit;
-        const uint32_t waves = (uint32_t)((a->chains + r - 1) / r);
-        c.resident = (a->chains + waves - 1) / waves;              // equal waves
-        // a wave is spread over all SMs: CTAs of ceil(resident / SMs) chains where one CTA per SM holds them
-        const uint32_t even = (c.resident + sms - 1) / sms;
-        c.wpb = even < wcap ? even : wcap;
     }
 
     // workspace layout
@@ -1076,6 +1121,11 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     // the winner can be walked back instead of replayed from its first move.
     c.undo_cap = c.psmem ? 0u : 4096u;
     const size_t o_ulog = take((size_t)c.resident * c.undo_cap * 8), o_ulen = take(c.psmem ? 0 : (size_t)c.resident * 4);
+    // Where the chains come in several waves they also log the units they rewrite (4 bytes each, up to 16384): the
+    // chain that takes over the slice in the next wave copies only those from the initial schedule again, not all of it.
+    const bool touch = c.touch;
+    c.touch_cap = touch ? 16384u : 0u;
+    const size_t o_tlog = take((size_t)c.resident * c.touch_cap * 4), o_tlen = take(touch ? (size_t)c.resident * 4 : 0);
     rc = ensure_chain_ws(p, off, st);
     if (rc) return rc;
     char* base = static_cast<char*>(p->d_chain_ws);
@@ -1086,6 +1136,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     c.hb0 = c.grow ? (uint32_t*)(base + o_hb0) : nullptr; c.hb_tmp = c.grow ? (uint32_t*)(base + o_hbt) : nullptr;
     c.full0 = (uint32_t*)(base + o_full); c.snap = snapshots ? (uint32_t*)(base + o_snap) : nullptr;
     c.undo_log = c.psmem ? nullptr : (uint64_t*)(base + o_ulog); c.undo_len = c.psmem ? nullptr : (uint32_t*)(base + o_ulen);
+    c.touch_log = touch ? (uint32_t*)(base + o_tlog) : nullptr; c.touch_len = touch ? (uint32_t*)(base + o_tlen) : nullptr;
 
     // initial schedule in both layouts
     if (a->init_mode == KVP_INIT_USER) {
@@ -1219,7 +1270,7 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     for (uint32_t first = 0; first < a->chains; first += c.resident, ++waves) {
         const uint32_t count = a->chains - first < c.resident ? a->chains - first : c.resident;
         if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr, c.snap,
-                             c.undo_log != nullptr))) {
+                             c.undo_log != nullptr, waves > 0))) {
             cleanup(); return rc;
         }
         if (c.undo_log) {

@@ -242,11 +242,13 @@ extern "C" int kvp_get_info(const kvp_problem* p, kvp_info* info)
 
 namespace {
 
-// Rows [j0, j1) of the acceptance table. Entries whose exponent is beyond 22.5 > ln(2^32) are zero whatever the
-// last bits of exp() are, so exp() is not called for them.
-void accept_rows(const double* temps, const uint32_t* shifts, uint32_t j0, uint32_t j1, uint32_t* table)
+// The rows rows[i0..i1) of the acceptance table. Entries whose exponent is beyond 22.5 > ln(2^32) are zero whatever
+// the last bits of exp() are, so exp() is not called for them.
+void accept_rows(const double* temps, const uint32_t* shifts, const uint32_t* rows, uint32_t i0, uint32_t i1,
+                 uint32_t* table)
 {
-    for (uint32_t j = j0; j < j1; ++j) {
+    for (uint32_t i = i0; i < i1; ++i) {
+        const uint32_t j = rows[i];
         const double C = temps[j] >= 1.0 ? temps[j] : 1.0;     // also maps NaN to 1
         const double bin = (double)(1ull << shifts[j]);
         for (uint32_t q = 0; q < KVP_TABLE_Q; ++q) {
@@ -267,30 +269,42 @@ void accept_rows(const double* temps, const uint32_t* shifts, uint32_t j0, uint3
 extern "C" int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint32_t* shifts)
 {
     if (!temps || !table || !shifts || !levels) return KVP_ERR_ARG;
+    // A level whose (clamped) temperature equals that of the level before it has the same row: a ladder that has
+    // cooled below one tick repeats its last row, often for a third of its levels. Only the others are computed.
+    std::vector<uint32_t> rows;
+    rows.reserve(levels);
+    double prev = 0.0;
     for (uint32_t j = 0; j < levels; ++j) {
         const double C = temps[j] >= 1.0 ? temps[j] : 1.0;
         uint32_t sh = 0;
         while ((double)KVP_TABLE_Q * (double)(1ull << sh) < 23.0 * C)
             if (++sh > 40) return KVP_ERR_RANGE;
         shifts[j] = sh;
+        if (j == 0 || C != prev) rows.push_back(j);
+        prev = C;
     }
-    // A ladder of 64 levels is 65,536 calls of exp(), about half a millisecond on one core and a tenth of an
+    const uint32_t nrows = (uint32_t)rows.size();
+    // A ladder of 64 levels is up to 65,536 calls of exp(), about half a millisecond on one core and a tenth of an
     // annealing call on a small problem: the rows are independent, so a few threads share them.
-    uint32_t nthr = levels >= 16 ? std::min<uint32_t>(8u, std::max(1u, std::thread::hardware_concurrency())) : 1u;
+    uint32_t nthr = nrows >= 16 ? std::min<uint32_t>(8u, std::max(1u, std::thread::hardware_concurrency())) : 1u;
     if (nthr > 1) {
         std::vector<std::thread> pool;
-        const uint32_t per = (levels + nthr - 1) / nthr;
+        const uint32_t per = (nrows + nthr - 1) / nthr;
         try {
-            for (uint32_t t = 1; t < nthr && t * per < levels; ++t)
-                pool.emplace_back(accept_rows, temps, shifts, t * per, std::min(levels, (t + 1) * per), table);
+            for (uint32_t t = 1; t < nthr && t * per < nrows; ++t)
+                pool.emplace_back(accept_rows, temps, shifts, rows.data(), t * per, std::min(nrows, (t + 1) * per), table);
         } catch (...) {                                        // no thread to be had: this one does the rest
             const uint32_t done = (uint32_t)pool.size() + 1;
-            accept_rows(temps, shifts, std::min(levels, done * per), levels, table);
+            accept_rows(temps, shifts, rows.data(), std::min(nrows, done * per), nrows, table);
         }
-        accept_rows(temps, shifts, 0, std::min(levels, per), table);
+        accept_rows(temps, shifts, rows.data(), 0, std::min(nrows, per), table);
         for (auto& th : pool) th.join();
     } else {
-        accept_rows(temps, shifts, 0, levels, table);
+        accept_rows(temps, shifts, rows.data(), 0, nrows, table);
+    }
+    for (uint32_t j = 1, i = 1; j < levels; ++j) {             // the repeated rows, each from the row before it
+        if (i < nrows && rows[i] == j) { ++i; continue; }
+        memcpy(table + (size_t)j * KVP_TABLE_Q, table + (size_t)(j - 1) * KVP_TABLE_Q, KVP_TABLE_Q * sizeof(uint32_t));
     }
     return KVP_OK;
 }

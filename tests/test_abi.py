@@ -44,8 +44,13 @@ def test_host_only_entry_points(lib, oracle):
     otable, oshifts = oracle.accept_table(temps)
     assert np.array_equal(table, otable) and np.array_equal(shifts, oshifts)
     # long ladders are built by several host threads, rows split unevenly when the level count is no multiple
-    for levels, c0, alpha in ((64, 54321.0, 0.9), (100, 7.5e6, 0.83), (17, 3.0, 0.5)):
-        temps = c0 * alpha ** np.arange(levels, dtype=np.float64)
+    # (equal neighbours, as in a ladder that has cooled below one tick, share a row: the last case has runs of them
+    # at the start, in the middle and at the end)
+    ladders = [c0 * alpha ** np.arange(levels, dtype=np.float64)
+               for levels, c0, alpha in ((64, 54321.0, 0.9), (100, 7.5e6, 0.83), (17, 3.0, 0.5))]
+    ladders.append(np.array([5.0, 5.0, 0.2, 0.1, 9.0] + [700.0] * 20 + [9.0, 9.0, 0.5, 0.5], np.float64))
+    for temps in ladders:
+        levels = temps.size
         table = np.zeros((levels, 1024), np.uint32)
         shifts = np.zeros(levels, np.uint32)
         assert lib.kvp_accept_table(temps.ctypes.data_as(ctypes.c_void_p), ctypes.c_uint32(levels),

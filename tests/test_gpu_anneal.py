@@ -201,6 +201,30 @@ def test_global_state_winner_paths(kvp, oracle, warps_per_chain):
         assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
 
 
+def test_later_waves_copy_only_what_changed(kvp, oracle, warps_per_chain):
+    """More chains than are resident at once: a chain of a later wave takes over a slice of global scratch that holds
+    the final state of an earlier chain, and copies from the initial schedule only the units which that chain logged
+    as rewritten, or all of it once the log has overflowed (the hot start below). Chains of every wave against the
+    oracle; the counts of applied moves show that the first run stays inside the log and the second goes beyond it."""
+    g, o, cfg, A = named_problem(kvp, oracle, "layer_8b")
+    for kw, overflow in ((dict(chains=5000, moves=2000, seed=7, p0=0.3, levels=4), False),
+                         (dict(chains=2600, moves=160_000, seed=7, p0=0.8, levels=4), True)):
+        gp, op = _params(g, o, **kw)
+        out = g.anneal(gp, want_per_chain=True)
+        n = kw["chains"]
+        changed = [r.n_changed for r in out["per_chain"]]
+        if overflow:
+            assert min(changed) > 16384                 # every log overflowed: one entry or two per applied move
+        else:
+            assert min(changed) > 0 and 2 * max(changed) <= 16384
+        for c in (0, 1, n // 2, n // 2 + 1, n - 2, n - 1):
+            want, _, _ = o.anneal_chains(op, c, 1)
+            assert out["per_chain"][c].astuple() == want[0].astuple(), c
+        w = out["stats"].best_chain
+        ref, _, bst = o.anneal_chains(op, w, 1, want_best=True)
+        assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
+
+
 def test_turn_wait_is_bounded(kvp, oracle, monkeypatch):
     """A hand-over that never comes: the waiting warp gives up after its poll limit (about a second), kvp_anneal
     returns KVP_ERR_TIMEOUT instead of holding the GPU, and the next call on the same problem is exact again."""

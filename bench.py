@@ -33,7 +33,7 @@ UNIT = "move-evals/s"
 ISSUE_PEAK_GWIPS = 148 * 4 * 1.965
 # dram__bytes_read.sum + dram__bytes_write.sum of one chain-kernel launch on this workload (ncu capture summarised in
 # profiles/chain_kernel_single_head.md; set to None whenever the kernel changes until it is captured again)
-CHAIN_KERNEL_DRAM_BYTES = 390400
+CHAIN_KERNEL_DRAM_BYTES = 390144
 # what that capture shows of the integer datapath (fractions of peak over the launch; context beside the timed figure)
 CHAIN_KERNEL_NCU = {"issue_active": 0.665, "alu_pipe": 0.574, "imad_pipe": 0.365, "warp_inst_per_move": 30.4}
 ALG_WARP_INSTR_PER_MOVE = 16.0

@@ -72,8 +72,8 @@ __device__ __forceinline__ void select_reset(SelectSmem& sm)
 //
 // The threshold K (the k-th largest key) is found digit by digit from the top, eight bits per pass: the keys that
 // agree with K in the bits fixed so far are counted per digit in a shared-memory histogram, and one warp walks
-// the histogram from the top until the counts reach what is still needed. The bits above the highest one in which
-// the largest and the smallest key differ are common to all keys and need no pass: three passes on these scores.
+// the histogram from the top until the counts reach what is still needed. The search works on the keys minus the
+// smallest one, so only the bits of (largest - smallest) need a pass: three passes on these scores.
 // FULL: the CTA's UPT * T slots are exactly the n units, so no slot needs a bounds test.
 template <int UPT, bool FULL = false>
 __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const TraceK& k, uint32_t topk, uint32_t gbase,
@@ -88,16 +88,29 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
     mn = __reduce_min_sync(0xFFFFFFFFu, mn);
     if (lane == 0) { atomicMax(&sm.hi, mx); atomicMin(&sm.lo, mn); }
     __syncthreads();
-    int rem = 32 - __clz(sm.hi ^ sm.lo);                     // bits still open; 0 when all keys are equal
-    uint32_t K = rem >= 32 ? 0u : sm.hi & ~((1u << rem) - 1u);
+    // The search runs on key - smallest key: the same order, and the digits then spread over the range the keys
+    // really cover (scores on both sides of zero differ in every leading bit, although they span twenty bits or so:
+    // as raw keys they would need four passes, the first two with nearly all keys in two or three bins).
+    const uint32_t lo = sm.lo;
+    uint32_t kk[UPT];
+#pragma unroll
+    for (int j = 0; j < UPT; ++j) kk[j] = key[j] - lo;
+    int rem = 32 - __clz(sm.hi - lo);                        // bits still open; 0 when all keys are equal
+    uint32_t K = 0u;                                         // the bits above them are zero in every reduced key
     uint32_t need = topk, equal = k.n;                       // all keys equal: every one ties at K
     for (int pass = 0; rem > 0; ++pass) {
         const int w = rem < kDigitBits ? rem : kDigitBits, sh = rem - w;
         uint32_t* hist = sm.hist[pass];
+        if (pass == 0) {                                     // no reduced key has a bit above the open ones: all count
 #pragma unroll
-        for (int j = 0; j < UPT; ++j) {
-            const bool in = (FULL || j * T + tid < k.n) && (rem >= 32 || (key[j] >> rem) == (K >> rem));
-            if (in) atomicAdd(hist + ((key[j] >> sh) & ((1u << w) - 1u)), 1u);
+            for (int j = 0; j < UPT; ++j)
+                if (FULL || j * T + tid < k.n) atomicAdd(hist + (kk[j] >> sh), 1u);
+        } else {
+#pragma unroll
+            for (int j = 0; j < UPT; ++j) {
+                const bool in = (FULL || j * T + tid < k.n) && (kk[j] >> rem) == (K >> rem);
+                if (in) atomicAdd(hist + ((kk[j] >> sh) & ((1u << w) - 1u)), 1u);
+            }
         }
         __syncthreads();
         if (warp == 0) {
@@ -139,8 +152,8 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
     for (int j = 0; j < UPT; ++j) {
         const uint32_t i = j * T + tid;
         const bool ok = FULL || i < k.n;
-        const bool tie = ok && key[j] == K;
-        bool pick = ok && key[j] > K;
+        const bool tie = ok && kk[j] == K;
+        bool pick = ok && kk[j] > K;
         if (!rank_ties) {
             pick = pick || tie;
         } else {

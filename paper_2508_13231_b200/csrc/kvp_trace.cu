@@ -48,10 +48,12 @@ __device__ __forceinline__ uint32_t block_sum(uint32_t v, uint32_t* slot)
 constexpr int kDigitBits = 8;                        // the search fixes this many bits of the threshold per pass
 constexpr int kBins = 1 << kDigitBits;
 constexpr int kPasses = 32 / kDigitBits;
+constexpr uint32_t kListCap = 256;                   // a threshold bin of up to this many keys is finished by ranking
 
 struct SelectSmem {
     uint32_t hist[kPasses][kBins];   // per pass: how many keys with the threshold's higher bits have each digit
-    uint32_t cnt[4];                 // block-wide counts beside the search
+    uint32_t cnt[4];                 // block-wide counts beside the search ([1]: keys in `list`)
+    uint32_t list[kListCap];         // the keys of the threshold's bin after the first pass
     uint32_t warp[32];
     uint32_t run;
     uint32_t hi, lo;                 // largest and smallest key of the step
@@ -142,6 +144,30 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
         __syncthreads();
         K = sm.K; need = sm.need; equal = sm.equal;
         rem = sh;
+        if (pass == 0 && rem > 0 && equal <= kListCap) {
+            // The first digit's bin usually holds a few dozen keys: they go to a shared list and each is ranked against
+            // the others, which settles the remaining bits at once; further histogram passes, in which every thread
+            // tests all of its keys again, are left to bins with many keys (ties).
+#pragma unroll
+            for (int j = 0; j < UPT; ++j)
+                if ((FULL || j * T + tid < k.n) && (kk[j] >> rem) == (K >> rem)) sm.list[atomicAdd(&sm.cnt[1], 1u)] = kk[j];
+            __syncthreads();
+            for (uint32_t c = tid; c < equal; c += T) {
+                const uint32_t v = sm.list[c];
+                uint32_t above = 0, same = 0;
+                for (uint32_t i = 0; i < equal; ++i) {
+                    const uint32_t x = sm.list[i];
+                    above += x > v ? 1u : 0u;
+                    same += x == v ? 1u : 0u;
+                }
+                if (above < need && need <= above + same) {   // v is the need-th largest; equal keys write the same
+                    sm.K = v; sm.need = need - above; sm.equal = same;
+                }
+            }
+            __syncthreads();
+            K = sm.K; need = sm.need; equal = sm.equal;
+            rem = 0;
+        }
     }
     const uint32_t take = need;                              // ties to admit, lowest unit index first
     const bool rank_ties = equal != take;

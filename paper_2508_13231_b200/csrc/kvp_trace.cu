@@ -312,6 +312,24 @@ trace_scores_kernel(const TraceK k, uint32_t U, int32_t* __restrict__ scores)
     }
 }
 
+// Pass 1 for traces of many units: a thread per unit walks the steps, draws and recurrence together, and the threads
+// of a warp write 128 contiguous bytes per step. No shared memory and no barrier; the draws of later steps do not
+// depend on the state, so the unrolled loop overlaps their Philox chains with the recurrence. It needs about a
+// thousand units per SM to fill the machine, which is why fewer units take the segmented kernel above.
+__global__ void __launch_bounds__(256)
+trace_scores_unit_kernel(const TraceK k, uint32_t U, int32_t* __restrict__ scores)
+{
+    const uint32_t u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= U) return;
+    const int32_t b = k.base ? __ldg(k.base + u) : 0;
+    int32_t x = 0;
+#pragma unroll 4
+    for (uint32_t t = 0; t < k.steps; ++t) {
+        x = next_state(k, u, t, x);
+        scores[(size_t)t * U + u] = x + b;
+    }
+}
+
 // Two-pass form, pass 2: the top-k selections of different steps are independent: one CTA per (group, step).
 template <int UPT, bool FULL>
 __global__ void __launch_bounds__(1024)
@@ -386,7 +404,8 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
         int prc = retain_in_pool(dev, score_bytes);          // the next call gets the block back from the pool
         if (prc) return prc;
         KVP_CUDA(cudaMallocAsync(&scores, score_bytes, st));
-        trace_scores_kernel<<<(uint32_t)((U64 + 31) / 32), kScoreThreads, 0, st>>>(k, (uint32_t)U64, scores);
+        if (U64 >= 148u * 1024u) trace_scores_unit_kernel<<<(uint32_t)((U64 + 255) / 256), 256, 0, st>>>(k, (uint32_t)U64, scores);
+        else trace_scores_kernel<<<(uint32_t)((U64 + 31) / 32), kScoreThreads, 0, st>>>(k, (uint32_t)U64, scores);
         dim3 grid(tp->groups, tp->steps);
         // Small CTAs with many units per thread: a selection is a chain of barriers and a serial histogram walk, so
         // what counts is how many of them an SM overlaps (whole call, 640 groups of 4096 units x 64 steps: 1.85 ms

@@ -196,6 +196,11 @@ def run_cost_kernel(args):
 # and the AR(1) update 22, a second Philox and a compare for the burst draw 62 when bursts are on, and the top-k
 # search: the range reduction (2), three histogram passes of a prefix compare, a digit and a shared-memory add per
 # unit (12) and the selection compares (4): 18.
+# Multiplier pipe: 148 SMs x 4 schedulers x 1.965 GHz, a warp-wide 32 x 32 -> 64 bit multiply every four cycles
+# (measured: ncu's pipe-busy cycles of the score pass divided by its multiply instructions) = 9.3e12 multiplies/s.
+WIDE_MUL_PEAK_T = 148 * 4 * 1.965e9 / 4 * 32 / 1e12
+
+
 def trace_alg_thread_instr(bursts):
     return 60 + 22 + (62 if bursts else 0) + 18
 
@@ -203,8 +208,10 @@ def trace_alg_thread_instr(bursts):
 def run_trace_kernel(args):
     """The trace kernel alone (synthetic access sets) on the largest configuration: plain-ALU (issue-slot) roofline.
 
-    long_70b: 640 groups of 4096 units, 64 steps, k = 205, bursts on; two passes (scores, then one selection per
-    group and step). Memory traffic: the int32 score matrix written once and read once (2 * U * S * 4 = 1.3 GB) and
+    long_70b: 640 groups of 4096 units, 64 steps, k = 205, bursts on; two passes (scores by a thread per unit, then one
+    selection per group and step). Besides the issue-slot roofline the line gives the rate of 32 x 32 -> 64 bit
+    multiplies (20 per Philox block, 2 in the AR(1) update) against the multiplier pipe: the score pass keeps that
+    pipe 90% busy, a wide multiply occupying a scheduler's pipe for four cycles per warp (both from ncu). Memory traffic: the int32 score matrix written once and read once (2 * U * S * 4 = 1.3 GB) and
     the output (S * W32 * 4 = 21 MB), reported as GB/s beside the instruction rate.
     """
     import torch
@@ -233,15 +240,19 @@ def run_trace_kernel(args):
         total_ms += e0.elapsed_time(e1)
     ms = total_ms / args.steps
     alg = trace_alg_thread_instr(bool(tp.get("burst_thr"))) / 32.0 * U * S           # warp instructions
+    wide = 42 if tp.get("burst_thr") else 22                                         # 32 x 32 -> 64 bit multiplies per (unit, step)
     achieved = alg / (ms * 1e-3) / 1e9
     print(json.dumps({
-        "kernel": "trace_scores_kernel + trace_select_kernel (kvp_trace_generate)", "metric": "unit_steps_per_sec", "value": U * S / (ms * 1e-3),
+        "kernel": "trace_scores_unit_kernel + trace_select_kernel (kvp_trace_generate)", "metric": "unit_steps_per_sec", "value": U * S / (ms * 1e-3),
         "unit": "unit-steps/s", "ms_per_call": ms, "steps": args.steps,
         "config": {"workload": name, "groups": cfg["groups"], "units_per_group": cfg["units_per_group"], "rows": S,
                    "topk": cfg["topk"], "l2": "flushed with a 256 MB write between timed iterations"},
         "roofline": {"bound": "alu", "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s",
                      "frac": achieved / ISSUE_PEAK_GWIPS, "traffic": None,
                      "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)",
+                     "wide_multiplies": {"achieved": wide * U * S / (ms * 1e-3) / 1e12, "peak": WIDE_MUL_PEAK_T,
+                                         "unit": "T multiplies/s", "frac": wide * U * S / (ms * 1e-3) / 1e12 / WIDE_MUL_PEAK_T,
+                                         "per_unit_step": wide},
                      "memory_gbs": (2 * U * S * 4 + S * W32 * 4 + (U * 4 if base is not None else 0)) / (ms * 1e-3) / 1e9}}))
 
 

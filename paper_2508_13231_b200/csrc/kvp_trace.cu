@@ -1,7 +1,8 @@
 // Trace kernels: synthetic importance per unit and step, top-k per (layer, kv-head) group, packed into uint32
-// bitmaps. Two passes by default: the first writes a score matrix (the draws in parallel over units and steps, the
-// AR(1) recurrence, sequential in time, by one lane per unit); then one CTA per (group, step) finds the k-th largest
-// score digit by digit with shared-memory histograms, ties going to the lower unit index. A fused single-pass form
+// bitmaps. Two passes by default: the first writes a score matrix (large traces: a thread per unit walks the steps;
+// small ones: the draws in parallel over units and steps, the AR(1) recurrence, sequential in time, by one lane per
+// unit); then one CTA per (group, step) finds the k-th largest score: the first eight bits of its range by a
+// shared-memory histogram, the rest by ranking the keys of that bin, ties going to the lower unit index. A fused single-pass form
 // (one CTA per group walking the steps, state in registers) serves layered or growing traces and those whose score
 // matrix would exceed the scratch budget.
 #include "kvp_common.cuh"

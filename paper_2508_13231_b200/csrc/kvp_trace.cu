@@ -172,36 +172,40 @@ __device__ __forceinline__ void select_step(const uint32_t (&key)[UPT], const Tr
     }
     const uint32_t take = need;                              // ties to admit, lowest unit index first
     const bool rank_ties = equal != take;
-    if (tid == 0) sm.run = 0;
-    __syncthreads();
     uint32_t* row = k.out + (size_t)t * k.W32;
-#pragma unroll
-    for (int j = 0; j < UPT; ++j) {
+    auto emit = [&](int j, bool pick) {
         const uint32_t i = j * T + tid;
-        const bool ok = FULL || i < k.n;
-        const bool tie = ok && kk[j] == K;
-        bool pick = ok && kk[j] > K;
-        if (!rank_ties) {
-            pick = pick || tie;
-        } else {
-            // units of round j are consecutive over the CTA, so index order = (round, thread) order
-            const uint32_t tb = __ballot_sync(0xFFFFFFFFu, tie);
-            if (lane == 0) sm.warp[warp] = __popc(tb);
-            __syncthreads();
-            uint32_t before = sm.run;
-            for (uint32_t w = 0; w < warp; ++w) before += sm.warp[w];
-            before += __popc(tb & ((1u << lane) - 1u));
-            pick = pick || (tie && before < take);
-            __syncthreads();
-            if (tid == 0) { uint32_t s = 0; for (uint32_t w = 0; w < (T >> 5); ++w) s += sm.warp[w]; sm.run += s; }
-            __syncthreads();
-        }
         if (k.aligned) {
             const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
             if (lane == 0 && (FULL || j * T + (tid & ~31u) < k.n)) row[(gbase + j * T + tid) >> 5] = bits;
         } else if (pick) {
             atomicOr(row + ((gbase + i) >> 5), 1u << ((gbase + i) & 31));
         }
+    };
+    if (!rank_ties) {                                        // the usual case, kept apart so that its loop stays small
+#pragma unroll
+        for (int j = 0; j < UPT; ++j) emit(j, (FULL || j * T + tid < k.n) && kk[j] >= K);
+        return;
+    }
+    if (tid == 0) sm.run = 0;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < UPT; ++j) {
+        const uint32_t i = j * T + tid;
+        const bool ok = FULL || i < k.n;
+        const bool tie = ok && kk[j] == K;
+        // units of round j are consecutive over the CTA, so index order = (round, thread) order
+        const uint32_t tb = __ballot_sync(0xFFFFFFFFu, tie);
+        if (lane == 0) sm.warp[warp] = __popc(tb);
+        __syncthreads();
+        uint32_t before = sm.run;
+        for (uint32_t w = 0; w < warp; ++w) before += sm.warp[w];
+        before += __popc(tb & ((1u << lane) - 1u));
+        const bool pick = (ok && kk[j] > K) || (tie && before < take);
+        __syncthreads();
+        if (tid == 0) { uint32_t s = 0; for (uint32_t w = 0; w < (T >> 5); ++w) s += sm.warp[w]; sm.run += s; }
+        __syncthreads();
+        emit(j, pick);
     }
 }
 

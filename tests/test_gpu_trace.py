@@ -40,7 +40,8 @@ def test_trace_full_size_sampled_groups(kvp, oracle, name, groups):
 
 
 @pytest.mark.parametrize("G,n,S,k", [(3, 40, 12, 7), (1, 16, 5, 16), (5, 100, 9, 1), (2, 1024, 6, 100),
-                                     (2, 2048 + 64, 4, 33), (1, 8192, 3, 500), (7, 33, 40, 5)])
+                                     (2, 2048 + 64, 4, 33), (1, 8192, 3, 500), (7, 33, 40, 5),
+                                     (151, 1030, 3, 70)])  # enough units for the score kernel with a thread per unit
 @pytest.mark.parametrize("flags", [0, 1])          # two passes over a score matrix / single fused pass
 def test_trace_ragged_shapes(kvp, oracle, G, n, S, k, flags):
     rng = np.random.default_rng(G * 1000 + n)

@@ -263,10 +263,11 @@ int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint
  * proposals in turn; the results are those of the sequential chain either way. The environment variable
  * KVP_WARPS_PER_CHAIN=1|2 overrides the choice (tuning and tests). The only device-side wait of the library is a
  * warp's wait for its turn; it is bounded, and a chain whose wait runs out makes the call return KVP_ERR_TIMEOUT
- * (the outputs are then undefined). Two more variables are hooks of the test-suite and nothing else:
- * KVP_TEST_DROP_TURN=1 withholds one hand-over per chain so that the bounded wait runs out (about a second), and
+ * (the outputs are then undefined). Three more variables are hooks of the test-suite and nothing else:
+ * KVP_TEST_DROP_TURN=1 withholds one hand-over per chain so that the bounded wait runs out (about a second),
  * KVP_TEST_SPLIT_QUEUE=n sends batches with more than n work items down the rarely taken two-halves path of the
- * half-size work queue.
+ * half-size work queue, and KVP_TEST_RESIDENT=n lets at most n chains whose schedules live in global memory run at
+ * a time, so that a small job comes in several waves (later waves reuse the slices of earlier ones).
  */
 int kvp_anneal(kvp_problem* p, const kvp_anneal_params* params, uint32_t* best_schedule,
                uint64_t* best_ticks, double* best_seconds, kvp_anneal_stats* stats, void* stream);

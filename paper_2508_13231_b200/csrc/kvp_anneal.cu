@@ -1093,6 +1093,11 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             size_t cap_r = (size_t)per_sm * sms;
             size_t r = a->chains < cap_r ? a->chains : cap_r;
             if (r > fit) r = fit;
+            // KVP_TEST_RESIDENT=n (tests only): at most n chains at a time, so that small jobs come in several waves
+            if (const char* e = getenv("KVP_TEST_RESIDENT")) {
+                const long v = atol(e);
+                if (v >= 1 && (size_t)v < r) r = (size_t)v;
+            }
             const uint32_t waves = (uint32_t)((a->chains + r - 1) / r);
             c.resident = (a->chains + waves - 1) / waves;              // equal waves
             // a wave is spread over all SMs: CTAs of ceil(resident / SMs) chains where one CTA per SM holds them

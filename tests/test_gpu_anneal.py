@@ -225,6 +225,22 @@ def test_later_waves_copy_only_what_changed(kvp, oracle, warps_per_chain):
         assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
 
 
+@pytest.mark.parametrize("resident", ["1", "3", "4"])
+def test_small_job_in_several_waves(kvp, oracle, monkeypatch, resident, warps_per_chain):
+    """Schedules in global memory, at most `resident` chains at a time (test hook): every chain but the first ones
+    starts from a slice that an earlier chain left behind and restores only what that chain logged as rewritten.
+    All chains, the bound and the winner's schedule against the oracle, at a hot and a cold start, with the stop
+    rule, and with a winner that an early wave produced."""
+    monkeypatch.setenv("KVP_TEST_RESIDENT", resident)
+    U, S, cap = 3000, 300, 700
+    A = wl.random_access(U, S, 0.2, seed=21)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    for kw in (dict(chains=10, moves=3000, levels=6, p0=0.5, seed=1), dict(chains=7, moves=4000, levels=5, p0=1e-3, seed=2),
+               dict(chains=9, moves=6400, levels=64, p0=0.3, seed=3, early_stop_permille=20)):
+        gp, op = _params(g, o, **kw)
+        _check_against_oracle(g, o, gp, op)
+
+
 def test_turn_wait_is_bounded(kvp, oracle, monkeypatch):
     """A hand-over that never comes: the waiting warp gives up after its poll limit (about a second), kvp_anneal
     returns KVP_ERR_TIMEOUT instead of holding the GPU, and the next call on the same problem is exact again."""

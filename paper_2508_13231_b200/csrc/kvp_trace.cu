@@ -414,9 +414,11 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
         dim3 grid(tp->groups, tp->steps);
         // Small CTAs with many units per thread: a selection is a chain of barriers and a serial histogram walk, so
         // what counts is how many of them an SM overlaps (whole call, 640 groups of 4096 units x 64 steps: 1.85 ms
-        // with 1024 threads, 1.70 ms with 256; 256 groups of 2048 x 128 steps: 0.84 against 0.61 ms with 128).
+        // with 1024 threads, 1.70 ms with 256; 256 groups of 2048 x 128 steps: 0.84 against 0.61 ms with 128). Since the
+        // search needs one histogram pass only, eight units per thread are a little faster than sixteen (1.05 against
+        // 1.07 ms and 0.359 against 0.363 ms on these two shapes).
         int su = 1;
-        while (su < 16 && (n + su - 1) / su > 128) su *= 2;
+        while (su < 8 && (n + su - 1) / su > 128) su *= 2;
         const uint32_t ST = ((n + su - 1) / su + 31) / 32 * 32;
         const bool full = (uint64_t)su * ST == n;             // every slot of the CTA holds a unit
 #define KVP_SELECT(UPT)                                                                              \
@@ -426,8 +428,7 @@ extern "C" int kvp_trace_generate(const kvp_trace_params* tp, uint32_t* access_b
             case 1: KVP_SELECT(1); break;
             case 2: KVP_SELECT(2); break;
             case 4: KVP_SELECT(4); break;
-            case 8: KVP_SELECT(8); break;
-            default: KVP_SELECT(16); break;
+            default: KVP_SELECT(8); break;
         }
 #undef KVP_SELECT
         cudaError_t le = cudaGetLastError();

@@ -15,7 +15,10 @@
  * bandwidths, the Unlimited-HBM closed form, the aggregate-bandwidth lower
  * bound, the free-migration per-step optimum, brute force over every static
  * placement and over every dynamic schedule of tiny instances, the published
- * Philox4x32-10 known-answer vectors, incremental-vs-full cost agreement.
+ * Philox4x32-10 known-answer vectors, incremental-vs-full cost agreement;
+ * the proposal decoder against the distribution its definition fixes (swap
+ * share, run-length classes, uniform and independent s0, u, v, w) and against
+ * proposals decoded by hand from the published Philox blocks.
  * Growing cache (kvpo_set_births; tests/test_oracle_growing.py): a hand-worked
  * instance with H^w / E^w decided by the schedule, the all-HBM and all-DRAM
  * closed forms, the exact reduction to the fixed-population model with the
@@ -394,6 +397,23 @@ static move_t decode_move(const kvpo_problem *p, const kvpo_anneal_params *ap,
     mv.v = (uint32_t)(((uint64_t)r[2] * p->U) >> 32);
     mv.w = r[3];
     return mv;
+}
+
+/*
+ * Test access to the proposal decoder: the proposals of moves m_begin ..
+ * m_begin+count-1 of `chain` under counter tag `tag`, as the annealer draws them.
+ *   out [count][6] = {swap, s0, len, u, v, w}
+ */
+int kvpo_decode_moves(const kvpo_problem *p, const kvpo_anneal_params *ap, uint32_t chain, uint32_t tag,
+                      uint64_t m_begin, uint32_t count, uint32_t *out)
+{
+    if (!p || !ap || !out) return KVPO_ERR_ARG;
+    for (uint32_t i = 0; i < count; ++i) {
+        move_t mv = decode_move(p, ap, m_begin + i, chain, tag);
+        uint32_t *o = out + (size_t)i * 6;
+        o[0] = (uint32_t)mv.swap; o[1] = mv.s0; o[2] = mv.len; o[3] = mv.u; o[4] = mv.v; o[5] = mv.w;
+    }
+    return KVPO_OK;
 }
 
 typedef struct {

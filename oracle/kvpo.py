@@ -216,6 +216,14 @@ class Problem:
         return dict(best_schedule=best, best_ticks=int(bt.value), best_seconds=int(bt.value) * self.seconds_per_tick,
                     best_chain=int(bc.value), per_chain=list(res))
 
+    def decode_moves(self, ap, chain, m_begin, count, tag=1):
+        """The proposals of moves m_begin .. m_begin+count-1 of `chain` -> uint32 [count][6] = (swap, s0, len, u, v, w).
+        tag 1 = the annealer's moves, 2 = the calibration proposals."""
+        out = np.zeros((count, 6), np.uint32)
+        _chk(lib().kvpo_decode_moves(self._h, C.byref(ap), C.c_uint32(chain), C.c_uint32(tag), C.c_uint64(m_begin),
+                                     C.c_uint32(count), _u32p(out)), "decode_moves")
+        return out
+
     def check_total(self, P, ticks):
         return lib().kvpo_check_total(self._h, _u32p(self._sched(P)), C.c_uint64(ticks)) == 0
 

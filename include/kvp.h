@@ -100,7 +100,11 @@ int kvp_create(kvp_problem** out, uint32_t units, uint64_t bytes_per_unit, uint3
 
 /* Frees the handle and every device buffer it owns, in stream order behind the last call made on the
  * problem (that stream must still exist). NULL is allowed. Device memory comes from CUDA's stream-ordered
- * allocator; the library sets the default pool's release threshold to 1 GiB on first use of a device. */
+ * allocator. Process-wide side effect: the library raises the release threshold of the device's default memory
+ * pool to the largest block it has asked for on that device so far plus 1 GiB (about 42 GB after an annealing
+ * call on a 2.6M-unit x 64-step problem), so that the next problem of the same size gets its workspace back
+ * without a trip to the driver; the pool keeps that much freed memory after kvp_destroy, where other users of
+ * cudaMalloc in the process cannot see it until the pool is trimmed (cudaMemPoolTrimTo). */
 void kvp_destroy(kvp_problem* p);
 
 /* Fills *info (host). */
@@ -144,7 +148,8 @@ int kvp_eval_counts(kvp_problem* p, const uint32_t* schedules, uint32_t n,
  * process exits. It calls no allocating routine, neither of CUDA nor of any other library.
  *
  * Limit: n * steps * 16 bytes <= KVP_NOALLOC_SCRATCH_BYTES, i.e. n * steps <= 65536; a larger batch is
- * refused with KVP_ERR_RANGE and nothing is launched (split it, or use kvp_eval).
+ * refused with KVP_ERR_RANGE and nothing is launched (split it, or use kvp_eval). Every batch inside the limit is
+ * served, also the 32,769 to 65,536 one- or two-step schedules that need more than one launch.
  * First call on a device: looks up the device address of the array (once per device, with that device
  * current). Make that first call outside any stream capture.
  * Sharing: every call on a device uses the same array and overwrites what the previous call left there
@@ -260,14 +265,10 @@ int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint
  *   (entry i belongs to chain first_chain + i)
  * Synchronises `stream` before returning.
  * A job of few chains (at most 8 per SM) is served by two warps per chain that take the chain's batches of 32
- * proposals in turn; the results are those of the sequential chain either way. The environment variable
- * KVP_WARPS_PER_CHAIN=1|2 overrides the choice (tuning and tests). The only device-side wait of the library is a
- * warp's wait for its turn; it is bounded, and a chain whose wait runs out makes the call return KVP_ERR_TIMEOUT
- * (the outputs are then undefined). Three more variables are hooks of the test-suite and nothing else:
- * KVP_TEST_DROP_TURN=1 withholds one hand-over per chain so that the bounded wait runs out (about a second),
- * KVP_TEST_SPLIT_QUEUE=n sends batches with more than n work items down the rarely taken two-halves path of the
- * half-size work queue, and KVP_TEST_RESIDENT=n lets at most n chains whose schedules live in global memory run at
- * a time, so that a small job comes in several waves (later waves reuse the slices of earlier ones).
+ * proposals in turn; the results are those of the sequential chain either way. The only device-side wait of the
+ * library is a warp's wait for its turn; it is bounded, and a chain whose wait runs out makes the call return
+ * KVP_ERR_TIMEOUT (the outputs are then undefined). The library reads no environment variable; the switches that
+ * the test-suite needs are set with kvp_set_test_hooks (end of this header).
  */
 int kvp_anneal(kvp_problem* p, const kvp_anneal_params* params, uint32_t* best_schedule,
                uint64_t* best_ticks, double* best_seconds, kvp_anneal_stats* stats, void* stream);
@@ -318,13 +319,15 @@ typedef struct {
     const uint32_t* birth;/* (device) [groups*units_per_group] or NULL               */
 } kvp_trace_params;
 
-#define KVP_TRACE_SINGLE_PASS 1u /* never allocate the [steps][units] int32 score matrix (the default does for traces
-                                    of fewer than 148 groups when it is at most 1 GiB; stream-ordered, freed on
-                                    return); much slower for few groups */
+#define KVP_TRACE_SINGLE_PASS 1u /* never allocate the [steps][units] int32 score matrix. By default every trace whose
+                                    matrix is at most 1 GiB, and that is neither layered nor growing, is generated in
+                                    two passes through such a matrix (stream-ordered scratch, freed on return); the
+                                    single-pass form is slower, much slower for few groups */
 
 /*
  * kvp_trace_generate -- fill access_bitmaps (device) [steps][ceil(U/32)] with the
  * top-k sets described above. Asynchronous on `stream`.
+ * Limits: units_per_group <= 8192, 1 <= topk <= units_per_group (KVP_ERR_RANGE / KVP_ERR_ARG otherwise).
  */
 int kvp_trace_generate(const kvp_trace_params* params, uint32_t* access_bitmaps, void* stream);
 
@@ -408,6 +411,22 @@ int kvp_wr_anneal(const uint64_t* table, uint32_t w_max, uint32_t n_ratio, const
 /* Philox4x32-10 (Salmon et al., SC'11) on the host; exposed so that callers can
  * reproduce which proposal a given (seed, chain, move) pair is. */
 void kvp_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
+
+/*
+ * ---- test only ----
+ * Switches of the test-suite (and of tuning runs); process-wide, read at the start of every kvp_anneal /
+ * kvp_anneal_chain_state. No production caller needs them. All zero = the library's normal behaviour; NULL resets.
+ */
+typedef struct {
+    uint32_t warps_per_chain;   /* 1 or 2: serve every chain with that many warps, whatever the job size         */
+    uint32_t drop_turn;         /* 1: withhold one hand-over per chain so that the bounded wait for the turn
+                                   runs out (about a second) and the call returns KVP_ERR_TIMEOUT               */
+    uint32_t split_queue_plus1; /* n + 1: batches with more than n work items take the rarely reached two-halves
+                                   path of the half-size work queue                                              */
+    uint32_t resident;          /* n: at most n chains whose schedules live in global memory run at a time, so
+                                   that a small job comes in several waves                                       */
+} kvp_test_hooks;
+void kvp_set_test_hooks(const kvp_test_hooks* hooks);
 
 const char* kvp_strerror(int code);
 /* Text of the last CUDA error seen by the calling thread ("" if none). */

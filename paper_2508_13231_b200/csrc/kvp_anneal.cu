@@ -22,6 +22,8 @@ namespace kvp {
 
 namespace {
 
+kvp_test_hooks g_hooks = {0u, 0u, 0u, 0u};   // kvp_set_test_hooks; read once per call
+
 struct ChainParams {
     const uint32_t* Acol;        // [U][S32]
     const StepC* stepc;          // [S]
@@ -1028,13 +1030,11 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     c.touch = false;
     const size_t pbytes = (size_t)p->U * p->S32 * 4;
     // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
-    // chains then keeps twice as many warps in flight. KVP_WARPS_PER_CHAIN=1|2 overrides the choice (for tuning).
+    // chains then keeps twice as many warps in flight. kvp_set_test_hooks can override the choice (tests, tuning).
     const uint32_t chains_per_sm = (a->chains + sms - 1) / sms;
     uint32_t W = chains_per_sm <= 8 ? 2u : 1u;
-    if (const char* e = getenv("KVP_WARPS_PER_CHAIN")) {
-        if (e[0] == '1' && !e[1]) W = 1;
-        if (e[0] == '2' && !e[1]) W = 2;
-    }
+    const kvp_test_hooks hooks = g_hooks;
+    if (hooks.warps_per_chain == 1 || hooks.warps_per_chain == 2) W = hooks.warps_per_chain;
     c.psmem = fixed_bytes(1) + pbytes <= budget / 2;
     if (c.psmem) {
         uint32_t want = chains_per_sm < 1 ? 1 : chains_per_sm;
@@ -1093,11 +1093,8 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             size_t cap_r = (size_t)per_sm * sms;
             size_t r = a->chains < cap_r ? a->chains : cap_r;
             if (r > fit) r = fit;
-            // KVP_TEST_RESIDENT=n (tests only): at most n chains at a time, so that small jobs come in several waves
-            if (const char* e = getenv("KVP_TEST_RESIDENT")) {
-                const long v = atol(e);
-                if (v >= 1 && (size_t)v < r) r = (size_t)v;
-            }
+            // test hook: at most n chains at a time, so that small jobs come in several waves
+            if (hooks.resident >= 1 && (size_t)hooks.resident < r) r = hooks.resident;
             const uint32_t waves = (uint32_t)((a->chains + r - 1) / r);
             c.resident = (a->chains + waves - 1) / waves;              // equal waves
             // a wave is spread over all SMs: CTAs of ceil(resident / SMs) chains where one CTA per SM holds them
@@ -1180,16 +1177,13 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     prm.table = c.table; prm.shifts = c.shifts; prm.ws = c.slots; prm.K = p->K; prm.full0 = c.full0;
     prm.birth = p->d_birth; prm.hb0 = c.hb0;
     prm.err = reinterpret_cast<uint32_t*>(c.small + 16);
-    // KVP_TEST_DROP_TURN=1 (tests of the bounded wait only): one hand-over per chain is withheld, the waiting warp
-    // gives up after its poll limit (about a second) and the call returns KVP_ERR_TIMEOUT
-    if (const char* e = getenv("KVP_TEST_DROP_TURN")) prm.drop_first_turn = e[0] == '1' && !e[1];
-    // KVP_TEST_SPLIT_QUEUE=n (tests only): batches with more than n < 496 queue items already take the two-halves
-    // path of the half-size work queue, which ordinary inputs almost never reach
+    // test hook (tests of the bounded wait only): one hand-over per chain is withheld, the waiting warp gives up
+    // after its poll limit (about a second) and the call returns KVP_ERR_TIMEOUT
+    prm.drop_first_turn = hooks.drop_turn ? 1u : 0u;
+    // test hook: batches with more than n < 496 queue items already take the two-halves path of the half-size work
+    // queue, which ordinary inputs almost never reach
     prm.split_at = kQueueCap / 2;
-    if (const char* e = getenv("KVP_TEST_SPLIT_QUEUE")) {
-        const long v = atol(e);
-        if (v >= 0 && v < (long)(kQueueCap / 2)) prm.split_at = (uint32_t)v;
-    }
+    if (hooks.split_queue_plus1 >= 1 && hooks.split_queue_plus1 - 1 < kQueueCap / 2) prm.split_at = hooks.split_queue_plus1 - 1;
     KVP_CUDA(cudaMemsetAsync(prm.err, 0, 4, st));
     prm.U = p->U; prm.S = p->S; prm.S32 = p->S32; prm.cap = p->cap;
     prm.levels = a->levels; prm.p_swap_256 = a->p_swap_256; prm.len_choices = a->max_len_log2 + 1;
@@ -1259,11 +1253,15 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     int rc = validate(p, a);
     if (rc) return rc;
     KVP_CUDA(cudaSetDevice(p->device));
-    cudaEvent_t ev[4];
-    for (auto& e : ev) KVP_CUDA(cudaEventCreate(&e));
-    auto cleanup = [&]() { for (auto& e : ev) cudaEventDestroy(e); };
+    struct Events {                                       // destroyed on every way out of the call
+        cudaEvent_t e[4];
+        int n = 0;
+        ~Events() { for (int i = 0; i < n; ++i) cudaEventDestroy(e[i]); }
+        cudaEvent_t operator[](int i) const { return e[i]; }
+    } ev;
+    for (; ev.n < 4; ++ev.n) KVP_CUDA(cudaEventCreate(&ev.e[ev.n]));
     KVP_CUDA(cudaEventRecord(ev[0], st));
-    if ((rc = prepare(p, a, st, c))) { cleanup(); return rc; }
+    if ((rc = prepare(p, a, st, c))) return rc;
     KVP_CUDA(cudaEventRecord(ev[1], st));
 
     // the chains, one wave of resident chains after the other
@@ -1275,9 +1273,8 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     for (uint32_t first = 0; first < a->chains; first += c.resident, ++waves) {
         const uint32_t count = a->chains - first < c.resident ? a->chains - first : c.resident;
         if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr, c.snap,
-                             c.undo_log != nullptr, waves > 0))) {
-            cleanup(); return rc;
-        }
+                             c.undo_log != nullptr, waves > 0)))
+            return rc;
         if (c.undo_log) {
             // Best so far over the chains that have finished; if it belongs to this wave, walk that chain back to
             // its best state while its scratch slice still holds its final state.
@@ -1286,7 +1283,7 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
             ++c.launches;
             KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
             KVP_CUDA(cudaStreamSynchronize(st));
-            if (red.pad) { cleanup(); return KVP_ERR_TIMEOUT; }
+            if (red.pad) return KVP_ERR_TIMEOUT;
             if (red.best_chain >= first && red.best_move != ~0ull) {
                 uint32_t len = 0;
                 KVP_CUDA(cudaMemcpyAsync(&len, c.undo_len + (red.best_chain - first), 4, cudaMemcpyDeviceToHost, st));
@@ -1314,23 +1311,22 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
         ++c.launches;
         KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
         KVP_CUDA(cudaStreamSynchronize(st));
-        if (red.pad) { cleanup(); return KVP_ERR_TIMEOUT; }
+        if (red.pad) return KVP_ERR_TIMEOUT;
     }
     const uint64_t upto = red.best_move == ~0ull ? 0 : red.best_move + 1;
     if (upto && (c.snap || dumped_chain == red.best_chain)) {
         const uint32_t* col = c.snap ? c.snap + (size_t)red.best_chain * p->U * p->S32 : c.dumpcol;
-        if ((rc = launch_bit_transpose(col, p->U, p->S32, p->S, c.sched, p->W32, st))) { cleanup(); return rc; }
+        if ((rc = launch_bit_transpose(col, p->U, p->S32, p->S, c.sched, p->W32, st))) return rc;
         ++c.launches;
         red.best_chain += a->first_chain;                  // the reduction works on call-local indices
     } else {
         red.best_chain += a->first_chain;
-        if ((rc = replay_to_sched(p, c, red.best_chain, upto, c.results + a->chains))) { cleanup(); return rc; }
+        if ((rc = replay_to_sched(p, c, red.best_chain, upto, c.results + a->chains))) return rc;
     }
-    if ((rc = launch_counts(p, c.sched, 1, c.counts0, c.hb_tmp, st, &c.launches))) { cleanup(); return rc; }
+    if ((rc = launch_counts(p, c.sched, 1, c.counts0, c.hb_tmp, st, &c.launches))) return rc;
     if ((rc = launch_finish(p, c.counts0, c.hb_tmp, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2),
-                            c.small + 1, st))) {
-        cleanup(); return rc;
-    }
+                            c.small + 1, st)))
+        return rc;
     ++c.launches;
     if (best_schedule)
         KVP_CUDA(cudaMemcpyAsync(best_schedule, c.sched, (size_t)p->S * p->W32 * 4, cudaMemcpyDeviceToDevice, st));
@@ -1357,7 +1353,6 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
         cudaEventElapsedTime(&stats->ms_finish, ev[2], ev[3]);
         stats->kernel_launches = c.launches;
     }
-    cleanup();
     return ok ? KVP_OK : KVP_ERR_INTERNAL;
 }
 
@@ -1384,4 +1379,10 @@ extern "C" int kvp_anneal_chain_state(kvp_problem* p, const kvp_anneal_params* a
     KVP_CUDA(cudaMemcpyAsync(&gave_up, c.prm.err, 4, cudaMemcpyDeviceToHost, st));
     KVP_CUDA(cudaStreamSynchronize(st));
     return gave_up ? KVP_ERR_TIMEOUT : KVP_OK;
+}
+
+extern "C" void kvp_set_test_hooks(const kvp_test_hooks* hooks)
+{
+    if (hooks) g_hooks = *hooks;
+    else memset(&g_hooks, 0, sizeof g_hooks);
 }

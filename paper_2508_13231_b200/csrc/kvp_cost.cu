@@ -351,7 +351,10 @@ int launch_counts(const kvp_problem* p, const uint32_t* schedules, uint32_t n, u
     // partial wave costs little; every chunk re-reads one halo row (1/SC more traffic, mostly from L2).
     uint32_t SC = p->S;
     while (SC > 8 && (uint64_t)col_ctas * ((p->S + SC - 1) / SC) * nz < 148u * 8u * 4u) SC = (SC + 1) / 2;
-    if (SC > 512) SC = 512;
+    // the per-step accumulators of a chunk live in dynamic shared memory: keep them within the 48 KB a kernel gets
+    // without opting in (NS * WIDE_WARPS * SC entries of 8 bytes, 12 with births)
+    const uint32_t sc_max = (uint32_t)((48u * 1024u) / (NS * WIDE_WARPS * (sizeof(uint2) + (grow ? 4 : 0))));
+    if (SC > sc_max) SC = sc_max;
     dim3 grid(col_ctas, (p->S + SC - 1) / SC, nz);
     const size_t smem = (size_t)NS * WIDE_WARPS * SC * (sizeof(uint2) + (grow ? 4 : 0));
     const int T = WIDE_WARPS * 32;
@@ -393,6 +396,7 @@ extern "C" int kvp_eval_counts(kvp_problem* p, const uint32_t* schedules, uint32
     if (p->dL) return KVP_ERR_ARG;                       // four cardinalities do not describe a growing cache
     if ((reinterpret_cast<uintptr_t>(counts) & 15) != 0) return KVP_ERR_ARG;
     KVP_CUDA(cudaSetDevice(p->device));
+    p->last_stream = static_cast<cudaStream_t>(stream);
     const size_t sched_words = (size_t)p->S * p->W32;
     for (uint32_t i = 0; i < n; i += kBatchSlice) {
         const uint32_t m = n - i < kBatchSlice ? n - i : kBatchSlice;
@@ -465,9 +469,22 @@ extern "C" int kvp_eval_noalloc(kvp_problem* p, const uint32_t* schedules, uint3
     int rc = noalloc_scratch(p->device, &counts);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
     // The array still holds the previous call's numbers. launch_counts either overwrites every entry it
-    // owns (narrow rows) or clears them on the stream before accumulating (wide rows).
-    if ((rc = kvp::launch_counts(p, schedules, n, counts, nullptr, st, nullptr))) return rc;
-    return kvp::launch_finish(p, counts, nullptr, n, step_ticks, total_ticks, step_seconds, total_seconds, bad_step, nullptr,
-                              st);
+    // owns (narrow rows) or clears them on the stream before accumulating (wide rows). The schedule index is a
+    // grid dimension, so a batch of more than kBatchSlice schedules (possible within the limit only for one or two
+    // steps) goes in slices, each with its own part of the array.
+    const size_t sched_words = (size_t)p->S * p->W32;
+    for (uint32_t i = 0; i < n; i += kBatchSlice) {
+        const uint32_t m = n - i < kBatchSlice ? n - i : kBatchSlice;
+        const size_t so = (size_t)i * p->S;
+        uint32_t* part = counts + so * 4;
+        if ((rc = kvp::launch_counts(p, schedules + i * sched_words, m, part, nullptr, st, nullptr))) return rc;
+        if ((rc = kvp::launch_finish(p, part, nullptr, m, step_ticks ? step_ticks + so : nullptr, total_ticks + i,
+                                     step_seconds ? step_seconds + so : nullptr,
+                                     total_seconds ? total_seconds + i : nullptr, bad_step ? bad_step + i : nullptr,
+                                     nullptr, st)))
+            return rc;
+    }
+    return KVP_OK;
 }

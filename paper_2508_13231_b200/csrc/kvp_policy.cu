@@ -346,6 +346,7 @@ extern "C" int kvp_policy_reactive(kvp_problem* p, uint32_t init_mode, uint32_t*
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;        // stamps are 16 bits and live in shared memory
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
     uint32_t T = (p->U + 31) / 32 * 32;
     if (T > 1024) T = 1024;
     const uint32_t rounds = (p->W32 * 32 + T - 1) / T;
@@ -371,6 +372,7 @@ extern "C" int kvp_policy_page(kvp_problem* p, uint32_t page_units, uint32_t* sc
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
     const uint32_t E = p->U / page_units, EW32 = (E + 31) / 32;
     uint32_t T = (E + 31) / 32 * 32;
     if (T > 1024) T = 1024;
@@ -393,6 +395,7 @@ extern "C" int kvp_policy_lookahead(kvp_problem* p, uint32_t init_mode, const ui
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
     uint32_t T = (p->U + 31) / 32 * 32;
     if (T > 1024) T = 1024;
     const uint32_t rounds = (p->W32 * 32 + T - 1) / T;
@@ -424,6 +427,7 @@ extern "C" int kvp_wr_grid(kvp_problem* p, uint32_t init_mode, uint32_t w_max, u
     if (p->U > kPolicyMaxUnits) return KVP_ERR_RANGE;
     KVP_CUDA(cudaSetDevice(p->device));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    p->last_stream = st;
     const uint32_t total = w_max * n_ratio;
     const size_t sched_bytes = (size_t)p->S * p->W32 * 4;
     uint32_t chunk = (uint32_t)(((size_t)1 << 30) / sched_bytes);    // at most 1 GiB of schedules at a time
@@ -481,8 +485,12 @@ extern "C" int kvp_wr_anneal(const uint64_t* table, uint32_t w_max, uint32_t n_r
     const size_t acc_bytes = acc.size() * 4, sh_bytes = (shifts.size() * 4 + 255) & ~(size_t)255;
     const size_t res_bytes = (size_t)wp->chains * sizeof(kvp_wr_result);
     KVP_CUDA(cudaMallocAsync(&dev, acc_bytes + sh_bytes + res_bytes, st));
-    KVP_CUDA(cudaMemcpyAsync(dev, acc.data(), acc_bytes, cudaMemcpyHostToDevice, st));
-    KVP_CUDA(cudaMemcpyAsync(dev + acc_bytes, shifts.data(), shifts.size() * 4, cudaMemcpyHostToDevice, st));
+    cudaError_t ce = cudaMemcpyAsync(dev, acc.data(), acc_bytes, cudaMemcpyHostToDevice, st);
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(dev + acc_bytes, shifts.data(), shifts.size() * 4, cudaMemcpyHostToDevice, st);
+    if (ce != cudaSuccess) {
+        cudaFreeAsync(dev, st);
+        KVP_CUDA(ce);
+    }
     WRK k;
     k.table = table; k.acc = (const uint32_t*)dev; k.shifts = (const uint32_t*)(dev + acc_bytes);
     k.w_max = w_max; k.n_ratio = n_ratio; k.chains = wp->chains; k.levels = wp->levels;

@@ -24,6 +24,7 @@ EXPORTS = [
     "kvp_create", "kvp_destroy", "kvp_get_info", "kvp_eval", "kvp_eval_counts", "kvp_eval_noalloc", "kvp_accept_table", "kvp_anneal",
     "kvp_anneal_chain_state", "kvp_trace_generate", "kvp_philox4x32_10", "kvp_strerror", "kvp_last_cuda_error",
     "kvp_policy_lookahead", "kvp_policy_reactive", "kvp_policy_page", "kvp_wr_grid", "kvp_wr_anneal", "kvp_set_births",
+    "kvp_set_test_hooks",
 ]
 
 
@@ -99,6 +100,11 @@ class TraceParams(C.Structure):
     ]
 
 
+class TestHooks(C.Structure):
+    _fields_ = [("warps_per_chain", C.c_uint32), ("drop_turn", C.c_uint32), ("split_queue_plus1", C.c_uint32),
+                ("resident", C.c_uint32)]
+
+
 _handle = None
 
 
@@ -113,6 +119,7 @@ def _lib():
         h.kvp_last_cuda_error.restype = C.c_char_p
         h.kvp_destroy.restype = None
         h.kvp_philox4x32_10.restype = None
+        h.kvp_set_test_hooks.restype = None
         _handle = h
     return _handle
 
@@ -135,6 +142,12 @@ def _ptr(t, dtype=None):
 def _stream(stream=None):
     s = torch.cuda.current_stream() if stream is None else stream
     return C.c_void_p(s.cuda_stream)
+
+
+def set_test_hooks(warps_per_chain=0, drop_turn=0, split_queue=None, resident=0):
+    """kvp_set_test_hooks (test-suite and tuning only; process-wide). Called without arguments it resets everything."""
+    h = TestHooks(int(warps_per_chain), int(drop_turn), 0 if split_queue is None else int(split_queue) + 1, int(resident))
+    _lib().kvp_set_test_hooks(C.byref(h))
 
 
 def philox(ctr, key):

@@ -20,11 +20,11 @@ def kvp():
     return kvp
 
 
-@pytest.fixture(params=["1", "2"])
-def warps_per_chain(request, monkeypatch):
+@pytest.fixture(params=[1, 2])
+def warps_per_chain(request, hooks):
     """Both forms of the chain kernel: one warp per chain, and two warps that take a chain's batches in turn."""
-    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", request.param)
-    return int(request.param)
+    hooks(warps_per_chain=request.param)
+    return request.param
 
 
 def _params(g, o, **kw):
@@ -225,13 +225,13 @@ def test_later_waves_copy_only_what_changed(kvp, oracle, warps_per_chain):
         assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
 
 
-@pytest.mark.parametrize("resident", ["1", "3", "4"])
-def test_small_job_in_several_waves(kvp, oracle, monkeypatch, resident, warps_per_chain):
+@pytest.mark.parametrize("resident", [1, 3, 4])
+def test_small_job_in_several_waves(kvp, oracle, hooks, resident, warps_per_chain):
     """Schedules in global memory, at most `resident` chains at a time (test hook): every chain but the first ones
     starts from a slice that an earlier chain left behind and restores only what that chain logged as rewritten.
     All chains, the bound and the winner's schedule against the oracle, at a hot and a cold start, with the stop
     rule, and with a winner that an early wave produced."""
-    monkeypatch.setenv("KVP_TEST_RESIDENT", resident)
+    hooks(resident=resident)
     U, S, cap = 3000, 300, 700
     A = wl.random_access(U, S, 0.2, seed=21)
     g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
@@ -241,32 +241,31 @@ def test_small_job_in_several_waves(kvp, oracle, monkeypatch, resident, warps_pe
         _check_against_oracle(g, o, gp, op)
 
 
-def test_turn_wait_is_bounded(kvp, oracle, monkeypatch):
+def test_turn_wait_is_bounded(kvp, oracle, hooks):
     """A hand-over that never comes: the waiting warp gives up after its poll limit (about a second), kvp_anneal
     returns KVP_ERR_TIMEOUT instead of holding the GPU, and the next call on the same problem is exact again."""
     g, o, cfg, A = named_problem(kvp, oracle, "tiny")
-    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", "2")
-    monkeypatch.setenv("KVP_TEST_DROP_TURN", "1")
+    hooks(warps_per_chain=2, drop_turn=1)
     with pytest.raises(kvp.KvpError) as e:
         g.anneal(g.make_params(chains=4, moves=1000, seed=0))
     assert e.value.code == kvp.ERR_TIMEOUT
-    monkeypatch.delenv("KVP_TEST_DROP_TURN")
+    hooks(drop_turn=0)
     gp, op = _params(g, o, chains=4, moves=1000, seed=0)
     _check_against_oracle(g, o, gp, op)
 
 
 @pytest.mark.parametrize("name,p0", [("single_head", 1e-6), ("single_head", 0.3), ("layer_8b", 1e-6)])
-def test_two_warp_chains_repeat_exactly(kvp, oracle, monkeypatch, name, p0):
+def test_two_warp_chains_repeat_exactly(kvp, oracle, hooks, name, p0):
     """Two warps per chain evaluate ahead of each other's commits, so their timing varies from run to run; the
     results may not. All chains of the configuration, twenty runs, against one run with one warp per chain (which the
     other tests compare with the oracle), at a cold and at a hot start (many applied moves, many re-evaluations)."""
     g, o, cfg, A = named_problem(kvp, oracle, name)
     moves = min(cfg["moves"], 50_000)
     gp = g.make_params(chains=cfg["chains"], moves=moves, seed=3, p0=p0)
-    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", "1")
+    hooks(warps_per_chain=1)
     ref = g.anneal(gp, want_per_chain=True)
     want = [r.astuple() for r in ref["per_chain"]]
-    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", "2")
+    hooks(warps_per_chain=2)
     for _ in range(20):
         out = g.anneal(gp, want_per_chain=True)
         assert [r.astuple() for r in out["per_chain"]] == want
@@ -274,12 +273,12 @@ def test_two_warp_chains_repeat_exactly(kvp, oracle, monkeypatch, name, p0):
         assert torch.equal(out["best_schedule"], ref["best_schedule"])
 
 
-@pytest.mark.parametrize("split", ["0", "20", "64"])
-def test_work_queue_in_two_halves(kvp, oracle, monkeypatch, split, warps_per_chain):
+@pytest.mark.parametrize("split", [0, 20, 64])
+def test_work_queue_in_two_halves(kvp, oracle, hooks, split, warps_per_chain):
     """Chains in shared memory with the access bitmap staged beside them keep half a work queue and work a batch
     with more items than it holds off in two halves. Ordinary inputs never fill it, so the hook lowers the limit:
     dense accesses, a churning initial schedule and a hot start give batches of a few hundred items."""
-    monkeypatch.setenv("KVP_TEST_SPLIT_QUEUE", split)
+    hooks(split_queue=split)
     U, S, cap = 64, 200, 32
     A = wl.random_access(U, S, 0.5, seed=9)
     g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))

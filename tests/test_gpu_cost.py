@@ -140,3 +140,22 @@ def test_long_horizons(kvp, oracle):
     ref = o2.anneal(o2.make_params(**kw))
     assert [r.astuple() for r in got["per_chain"]] == [r.astuple() for r in ref["per_chain"]]
     assert np.array_equal(to_np(got["best_schedule"]), ref["best_schedule"])
+
+
+def test_many_long_schedules_keep_the_step_chunks_inside_shared_memory(kvp, oracle):
+    """A batch that already fills the GPU with whole-horizon step chunks: 9,500 schedules of 2,176 units x 512
+    steps (1.3 GB). The per-step accumulators of a chunk live in shared memory; the chunk length is capped so that they
+    fit without opting in to more than 48 KB. Sampled schedules against the oracle."""
+    U, S, cap, n = 2176, 512, 500, 9500
+    A = wl.random_access(U, S, 0.1, seed=77)
+    g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))
+    gen = torch.Generator(device="cuda"); gen.manual_seed(9)
+    w32 = U // 32
+    sched = torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, w32), dtype=torch.int32, device="cuda", generator=gen)
+    for _ in range(2):
+        sched &= torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, w32), dtype=torch.int32, device="cuda", generator=gen)
+    ev = g.eval(sched, want_steps=False, want_seconds=False)
+    torch.cuda.synchronize()
+    for i in (0, 1, 4749, 4750, n - 2, n - 1):
+        ref = o.eval(to_np(sched[i]))
+        assert int(ev["total_ticks"][i]) == ref["total_ticks"] and int(ev["bad_step"][i]) == ref["bad_step"], i

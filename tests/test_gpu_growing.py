@@ -17,11 +17,11 @@ def kvp():
     return kvp
 
 
-@pytest.fixture(params=["1", "2"])
-def warps_per_chain(request, monkeypatch):
+@pytest.fixture(params=[1, 2])
+def warps_per_chain(request, hooks):
     """Both forms of the chain kernel: one warp per chain, and two warps that take a chain's batches in turn."""
-    monkeypatch.setenv("KVP_WARPS_PER_CHAIN", request.param)
-    return int(request.param)
+    hooks(warps_per_chain=request.param)
+    return request.param
 
 
 def _birth_dev(birth):

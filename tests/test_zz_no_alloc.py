@@ -29,12 +29,13 @@ def _outputs(n, S):
 # one shape per counting kernel: rows of 8 words (sub-warp groups) and rows of 512 words (warp per chunk,
 # accumulated with atomics into scratch that the call must clear itself)
 @pytest.mark.parametrize("U,S,n1,n2", [(256, 512, 5, 3), (16384, 64, 6, 9), (1000, 33, 40, 2)])
-def test_noalloc_matches_eval_twice_in_a_row(U, S, n1, n2):
+def test_noalloc_matches_eval_twice_in_a_row(oracle, U, S, n1, n2):
     from paper_2508_13231_b200 import kvp
     cap = U // 4
     A = wl.random_access(U, S, 0.2, seed=U)
-    prob = kvp.Problem(U, 8192, S, to_dev(A), cap, 8000 * GB, 900 * GB, 900 * GB,
-                       hw=np.arange(S) % 2, ew=np.arange(S) % 3)
+    hw, ew = np.arange(S) % 2, np.arange(S) % 3
+    prob = kvp.Problem(U, 8192, S, to_dev(A), cap, 8000 * GB, 900 * GB, 900 * GB, hw=hw, ew=ew)
+    ref = oracle.Problem(U, 8192, S, A, cap, 8000 * GB, 900 * GB, 900 * GB, hw=hw, ew=ew)
     for call, n in enumerate((n1, n2)):
         scheds = wl.random_schedules(U, S, cap, n, seed=100 + call, churn=0.1)
         bits = wl.unpack_bits(scheds[-1], U); bits[S // 2, :cap + 1] = 1       # one schedule over capacity
@@ -50,6 +51,12 @@ def test_noalloc_matches_eval_twice_in_a_row(U, S, n1, n2):
         assert int(got["bad_step"][-1]) == S // 2
         assert torch.allclose(got["step_seconds"], want["step_seconds"], rtol=1e-9, atol=0)
         assert torch.allclose(got["total_seconds"], want["total_seconds"], rtol=1e-9, atol=0)
+        # and directly against the oracle, so that this file stands on its own: first and last schedule of the batch
+        for i in (0, n - 1):
+            o = ref.eval(scheds[i])
+            assert np.array_equal(got["step_ticks"][i].cpu().numpy().view(np.uint64), o["step_ticks"]), (call, i)
+            assert int(got["total_ticks"][i]) == o["total_ticks"] and int(got["bad_step"][i]) == o["bad_step"]
+            assert float(got["total_seconds"][i]) == pytest.approx(o["total_seconds"], rel=1e-9)
 
 
 def test_noalloc_refuses_batches_beyond_its_scratch():
@@ -69,3 +76,29 @@ def test_noalloc_refuses_batches_beyond_its_scratch():
     prob.eval_noalloc(scheds[:n_ok], **ok)
     torch.cuda.synchronize()
     assert torch.equal(ok["total_ticks"], prob.eval(scheds[:n_ok])["total_ticks"])
+
+
+def test_noalloc_serves_the_largest_batch_its_scratch_admits(oracle):
+    """One-step schedules: the limit admits 65,536 of them, more than one launch can index, so the call goes in
+    slices. Compared with kvp_eval on all of them and with the oracle on a few, twice in a row."""
+    from paper_2508_13231_b200 import kvp
+    U, S, cap = 96, 1, 40
+    A = wl.random_access(U, S, 0.3, seed=5)
+    prob = kvp.Problem(U, 8192, S, to_dev(A), cap, 8000 * GB, 900 * GB, 900 * GB)
+    ref = oracle.Problem(U, 8192, S, A, cap, 8000 * GB, 900 * GB, 900 * GB)
+    n = kvp.NOALLOC_SCRATCH_BYTES // 16
+    assert n == 65536
+    rng = np.random.Generator(np.random.PCG64(11))
+    scheds = (rng.integers(0, 2 ** 32, (n, S, 3), dtype=np.uint64) & rng.integers(0, 2 ** 32, (n, S, 3), dtype=np.uint64)
+              & rng.integers(0, 2 ** 32, (n, S, 3), dtype=np.uint64)).astype(np.uint32)
+    dev = to_dev(scheds)
+    want = prob.eval(dev)
+    for call in range(2):
+        got = _outputs(n, S)
+        prob.eval_noalloc(dev, **got)
+        torch.cuda.synchronize()
+        assert torch.equal(got["step_ticks"], want["step_ticks"]) and torch.equal(got["total_ticks"], want["total_ticks"])
+        assert torch.equal(got["bad_step"], want["bad_step"])
+        for i in (0, 32767, 32768, 50000, n - 1):
+            o = ref.eval(scheds[i])
+            assert int(got["total_ticks"][i]) == o["total_ticks"] and int(got["bad_step"][i]) == o["bad_step"], i

@@ -1,13 +1,18 @@
-"""Benchmark of the whole hot path on the `single_head` configuration.
+"""Benchmark of the whole hot path on the largest configuration, `long_70b` (2,621,440 units x 64 steps,
+8192 chains x 1,000,000 moves).
 
 One step = trace kernel -> kvp_create (layout kernels) -> cost kernel on a small batch of schedules ->
-kvp_anneal (initial cost, calibration, all chains, cross-chain reduction, winner replay and re-score).
+kvp_anneal (initial cost, calibration, all chains, cross-chain reduction, winner's schedule and re-score).
 Metric: simulated-annealing move evaluations per second (chains x moves / step time), whole job.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME] [--kernel K]
 
-N > 1 is launched with torch.distributed.run, one rank per GPU; the chains of an N x 1024-chain job are
-split over the ranks (chains are independent; the only exchange is a final 8-byte MIN on the host side).
+The default line also carries, as extra keys measured in the same run: the same step on `single_head` at the
+configured near-greedy start and at the paper's p0 = 0.8, the cost and trace kernels alone on long_70b rows
+(`kernels`), and the time-to-bound figures.
+N > 1: one rank per GPU (started through torch.distributed.run if the script is not already under it); the chains of
+an N x 8192-chain job are split over the ranks (chains are independent; the only exchange is the MIN over one
+(ticks, chain) pair per rank, once per step, inside the timed region).
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 """
 import argparse
@@ -22,21 +27,17 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-WORKLOAD = "single_head"
+WORKLOAD = "long_70b"
 METRIC = "sa_move_evals_per_sec"
 UNIT = "move-evals/s"
 # Issue-slot roofline of the chain kernel: 148 SMs x 4 warp schedulers x 1.965 GHz, one warp instruction per
-# scheduler and cycle. Algorithmic work per move evaluation with one proposal per lane: 16 warp instructions
-# (per 32 moves: Philox and decode ~105, window extraction and word-parallel bit logic ~100, work-queue scan
-# and push ~100, about 35 (lane, step) cost evaluations of ~70 thread instructions each in two warp rounds
-# ~150, Metropolis and in-order commit ~50).
+# scheduler and cycle. Algorithmic work per move evaluation: 16 warp instructions (per 32 moves: Philox and decode
+# ~105, window extraction and word-parallel bit logic ~100, work-queue scan and push ~100, about 35 (lane, step)
+# cost evaluations of ~70 thread instructions each in two warp rounds ~150, Metropolis and in-order commit ~50).
 ISSUE_PEAK_GWIPS = 148 * 4 * 1.965
-# dram__bytes_read.sum + dram__bytes_write.sum of one chain-kernel launch on this workload (ncu capture summarised in
-# profiles/chain_kernel_single_head.md; set to None whenever the kernel changes until it is captured again)
-CHAIN_KERNEL_DRAM_BYTES = 390144
-# what that capture shows of the integer datapath (fractions of peak over the launch; context beside the timed figure)
-CHAIN_KERNEL_NCU = {"issue_active": 0.665, "alu_pipe": 0.574, "imad_pipe": 0.365, "warp_inst_per_move": 30.4}
 ALG_WARP_INSTR_PER_MOVE = 16.0
+PEAK_SOURCE_ALU = "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"
+FLUSH_NOTE = "flushed with a 256 MB write between timed iterations"
 
 
 def _clock_sampler(stop, samples):
@@ -74,8 +75,110 @@ def _clock_summary(samples):
             "reasons": sorted({n for s in samples for n in s[2]})}
 
 
+def _hbm_peak():
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        return float(peaks["hbm_gbs"]), "measured copy bandwidth of this pool's B200s (driver-written peaks file)"
+    except Exception:
+        return 6650.0, "fallback 6.65 TB/s (no measured peaks file)"
+
+
+def _thinned_schedules(torch, n, S, W32, seed):
+    """n random schedules on the device, about 6% of the bits set (three ANDed draws): below every configuration's
+    capacity on average; the capacity check only sets a flag and costs nothing."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    sched = torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, W32), dtype=torch.int32, device="cuda", generator=g)
+    for _ in range(3):
+        sched &= torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, W32), dtype=torch.int32, device="cuda", generator=g)
+    return sched
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# The CPU oracle as a timed baseline (never on the product path): worker functions for a spawn pool.
+
+def _o_groups(args):
+    name, seed, lo, n = args
+    from oracle import kvpo
+    from paper_2508_13231_b200 import workloads as wl
+    return kvpo.trace_generate(**wl.trace_params(name, seed), group_begin=lo, group_count=n)
+
+
+def _o_chains(args):
+    """Problem set-up, temperature ladder and `count` chains from `first`, each for `upto` moves of the full budget."""
+    name, path, first, count, upto, seed = args
+    import numpy as np
+    from oracle import kvpo
+    from paper_2508_13231_b200 import workloads as wl
+    cfg = wl.CONFIGS[name]
+    A = np.ascontiguousarray(np.load(path, mmap_mode="r"))
+    o = kvpo.Problem(wl.units(cfg), cfg["bytes_per_unit"], cfg["steps"], A, cfg["cap"], *cfg["bw"])
+    ap = o.make_params(chains=cfg["chains"], moves=cfg["moves"], seed=seed, p0=cfg["p0"])
+    res, _, _ = o.anneal_chains(ap, first, count, upto_moves=upto)
+    return sum(r.moves_done for r in res)
+
+
+def _oracle_trace(name, seed, procs):
+    """The oracle's access bitmap, the groups spread over `procs` processes -> (array, seconds)."""
+    import multiprocessing as mp
+    from paper_2508_13231_b200 import workloads as wl
+    t0 = time.perf_counter()
+    G = wl.CONFIGS[name]["groups"]
+    if procs <= 1 or G < 2 * procs:
+        A = _o_groups((name, seed, 0, G))
+    else:
+        step = max(1, (G + 4 * procs - 1) // (4 * procs))
+        with mp.get_context("spawn").Pool(procs) as pool:
+            parts = pool.map(_o_groups, [(name, seed, lo, min(step, G - lo)) for lo in range(0, G, step)])
+        A = parts[0]
+        for part in parts[1:]:
+            A |= part
+    return A, time.perf_counter() - t0
+
+
+def _sample_plan(cfg):
+    """How much of a configuration one oracle process is given: chains and moves per chain (of the full budget)."""
+    from paper_2508_13231_b200 import workloads as wl
+    big = wl.units(cfg) * cfg["steps"] > (1 << 24)            # set-up of a chain costs seconds: few chains, short
+    if big:
+        return 2, min(cfg["moves"], 50_000)
+    return max(1, min(cfg["chains"], 96)), cfg["moves"]
+
+
+def cpu_baseline(name):
+    """Oracle timed on this machine's host cores on a bounded sample of the benchmark workload: every core runs the
+    same number of chains (independent processes), after the access bitmap was generated by the oracle on all cores."""
+    import multiprocessing as mp
+    import tempfile
+    import numpy as np
+    from oracle import kvpo
+    from paper_2508_13231_b200 import workloads as wl
+    kvpo.build()
+    cfg = wl.CONFIGS[name]
+    cores = os.cpu_count() or 1
+    procs = max(1, min(cores, 32))
+    A, trace_s = _oracle_trace(name, 0, procs)
+    fd, path = tempfile.mkstemp(suffix=".npy")
+    os.close(fd)
+    try:
+        np.save(path, A)
+        per, upto = _sample_plan(cfg)
+        jobs = [(name, path, i * per, per, upto, 0) for i in range(procs) if (i + 1) * per <= cfg["chains"]]
+        t0 = time.perf_counter()
+        with mp.get_context("spawn").Pool(len(jobs)) as pool:
+            moves = sum(pool.map(_o_chains, jobs))
+        dt = time.perf_counter() - t0
+    finally:
+        os.remove(path)
+    return {"value": moves / dt, "unit": UNIT, "cores": len(jobs), "host_cores": cores, "kind": "oracle",
+            "per_core": moves / dt / len(jobs),
+            "sample": f"{len(jobs)} processes x {per} chains (chains 0..{len(jobs) * per - 1} of {cfg['chains']}), the first "
+                      f"{upto} of {cfg['moves']} moves each, problem set-up and temperature ladder included: {dt:.1f} s; "
+                      f"before that the whole access bitmap by the oracle on {procs} processes: {trace_s:.1f} s"}
+
+
 def run_reference(args):
-    """The oracle as it stands, on host cores, on a bounded sample of the same workload."""
+    """The oracle as it stands, on host cores, each step a bounded sample of the benchmark workload (one thread)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -83,18 +186,28 @@ def run_reference(args):
     from oracle import kvpo
     from paper_2508_13231_b200 import workloads as wl
     kvpo.build()
-    cfg = wl.CONFIGS[WORKLOAD]
-    tp = wl.trace_params(WORKLOAD, seed=0)
-    sample_chains = 8
-    U = wl.units(cfg)
+    name = args.workload
+    cfg = wl.CONFIGS[name]
+    tp = wl.trace_params(name, seed=0)
+    U, S, G = wl.units(cfg), cfg["steps"], cfg["groups"]
+    per, upto = _sample_plan(cfg)
+    big = U * S > (1 << 24)
+    sample_groups = max(1, G // 64) if big else G
+    # the access bitmap the chains run on is generated once, outside the steps (for the large configurations on all
+    # cores); every step still generates a share of the groups as its sample of the trace stage
+    A, trace_s = _oracle_trace(name, 0, max(1, min(os.cpu_count() or 1, 32)) if big else 1)
+    rng = np.random.Generator(np.random.PCG64(5))
+    sched = (rng.integers(0, 2 ** 32, (S, (U + 31) // 32), dtype=np.uint64) & rng.integers(0, 2 ** 32, (S, (U + 31) // 32), dtype=np.uint64)
+             & rng.integers(0, 2 ** 32, (S, (U + 31) // 32), dtype=np.uint64) & rng.integers(0, 2 ** 32, (S, (U + 31) // 32), dtype=np.uint64)).astype(np.uint32)
+    if U % 32:
+        sched[:, -1] &= np.uint32((1 << (U % 32)) - 1)
 
     def step(seed):
-        A = kvpo.trace_generate(**dict(tp, seed=seed))
-        o = kvpo.Problem(U, cfg["bytes_per_unit"], cfg["steps"], A, cfg["cap"], *cfg["bw"])
-        for P in wl.random_schedules(U, cfg["steps"], cfg["cap"], 2, seed=seed):
-            o.eval(P)
-        ap = o.make_params(chains=sample_chains, moves=cfg["moves"], seed=seed, p0=cfg["p0"])
-        res, _, _ = o.anneal_chains(ap, 0, sample_chains)
+        kvpo.trace_generate(**dict(tp, seed=seed), group_begin=0, group_count=sample_groups)
+        o = kvpo.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"])
+        o.eval(sched)
+        ap = o.make_params(chains=cfg["chains"], moves=cfg["moves"], seed=seed, p0=cfg["p0"])
+        res, _, _ = o.anneal_chains(ap, 0, per, upto_moves=upto)
         return sum(r.moves_done for r in res)
 
     for w in range(args.warmup):
@@ -105,90 +218,69 @@ def run_reference(args):
         moves += step(k)
     dt = time.perf_counter() - t0
     value = moves / dt
-    sample = (f"{sample_chains} of {cfg['chains']} chains x {cfg['moves']} moves per step (plus the full trace, "
-              f"problem set-up and 2 schedule evaluations), single thread")
+    sample = (f"per step: trace of {sample_groups} of {G} groups, problem set-up, one schedule evaluation, chains 0..{per - 1} "
+              f"of {cfg['chains']} for the first {upto} of {cfg['moves']} moves; single thread "
+              f"(the access bitmap itself was generated once before the steps in {trace_s:.1f} s)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1000 * dt / max(1, args.steps), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32/uint64 ticks", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "chains": sample_chains, "moves": cfg["moves"]},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "config": {"workload": name, "chains": per, "moves": upto},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def cpu_baseline(cfg, tp):
-    """Oracle timed on this machine's host: a bounded sample of the benchmark workload, one thread."""
-    from oracle import kvpo
-    from paper_2508_13231_b200 import workloads as wl
-    kvpo.build()
-    sample_chains = 768
-    t0 = time.perf_counter()
-    A = kvpo.trace_generate(**tp)
-    o = kvpo.Problem(wl.units(cfg), cfg["bytes_per_unit"], cfg["steps"], A, cfg["cap"], *cfg["bw"])
-    ap = o.make_params(chains=sample_chains, moves=cfg["moves"], seed=0, p0=cfg["p0"])
-    res, _, _ = o.anneal_chains(ap, 0, sample_chains)
-    dt = time.perf_counter() - t0
-    return {"value": sum(r.moves_done for r in res) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"chains 0..{sample_chains - 1} of {cfg['chains']}, all {cfg['moves']} moves each, plus trace "
-                      f"and set-up; {dt:.1f} s on one thread"}
+# ----------------------------------------------------------------------------------------------------------------
+# Single kernels on full-size rows
+
+def _timed_calls(torch, fn, steps, warmup):
+    """Mean device time of fn(k) over `steps` calls (CUDA events on the current stream), L2 flushed before each."""
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    for w in range(max(3, warmup)):
+        fn(1000 + w)
+    torch.cuda.synchronize()
+    total_ms = 0.0
+    for k in range(steps):
+        flush.fill_(k & 255)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn(k)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        total_ms += e0.elapsed_time(e1)
+    return total_ms / steps
 
 
-def run_cost_kernel(args):
+def cost_kernel_record(steps, warmup):
     """The cost kernel alone (Eq. 1-5 over a batch of schedules) on the rows of the largest configuration: HBM roofline.
 
-    A batch of schedules of long_70b (81,920 words per row, 64 rows, 20 MB each) is scored by kvp_eval; the
+    A batch of 96 schedules of long_70b (81,920 words per row, 64 rows, 20 MB each) is scored by kvp_eval; the
     batch plus the access bitmap is larger than L2. Algorithmic bytes: every placement word once and the access
     bitmap once per batch (it stays in L2 across the batch), (n + 1) * S * W32 * 4.
     """
-    import numpy as np
     import torch
     from paper_2508_13231_b200 import kvp, workloads as wl
-    torch.cuda.set_device(0)
     name, n = "long_70b", 96
     cfg = wl.CONFIGS[name]
     tp = wl.trace_params(name, seed=0)
     U, S, W32 = wl.units(cfg), cfg["steps"], wl.words_per_row(cfg)
     A = kvp.trace_generate(**{k: v for k, v in tp.items() if k != "base"}, base=None)
     prob = kvp.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"])
-    g = torch.Generator(device="cuda"); g.manual_seed(1)
-    # random words thinned to ~6% density (three ANDed draws halve it each time; 1/8 would exceed the capacity check,
-    # which only sets a flag and costs nothing)
-    sched = torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, W32), dtype=torch.int32, device="cuda", generator=g)
-    for _ in range(3):
-        sched &= torch.randint(-2 ** 31, 2 ** 31 - 1, (n, S, W32), dtype=torch.int32, device="cuda", generator=g)
-    stream = torch.cuda.current_stream()
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    for _ in range(max(3, args.warmup)):
-        prob.eval(sched, want_steps=False, want_seconds=False)
-    torch.cuda.synchronize()
-    total_ms = 0.0
-    for k in range(args.steps):
-        flush.fill_(k & 255)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        prob.eval(sched, want_steps=False, want_seconds=False)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        total_ms += e0.elapsed_time(e1)
-    ms = total_ms / args.steps
+    sched = _thinned_schedules(torch, n, S, W32, seed=1)
+    ms = _timed_calls(torch, lambda k: prob.eval(sched, want_steps=False, want_seconds=False), steps, warmup)
+    prob.close()
+    del sched
     alg_bytes = (n + 1) * S * W32 * 4
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except Exception:
-        pass
-    peak, src = (peaks["hbm_gbs"], "measured copy bandwidth (MEASURED_PEAKS.json)") if "hbm_gbs" in peaks else \
-        (6650.0, "fallback 6.65 TB/s")
+    peak, src = _hbm_peak()
     achieved = alg_bytes / (ms * 1e-3) / 1e9
-    print(json.dumps({
-        "kernel": "count_wide_kernel+finish_kernel (kvp_eval)", "metric": "schedules_scored_per_sec",
-        "value": n / (ms * 1e-3), "unit": "schedules/s", "ms_per_call": ms, "steps": args.steps,
-        "config": {"workload": name, "batch": n, "words_per_row": W32, "rows": S,
-                   "l2": "flushed with a 256 MB write between timed iterations"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "algorithmic_bytes": alg_bytes, "peak_source": src}}))
+    return {"kernel": "count_wide_kernel+finish_kernel (kvp_eval)", "metric": "schedules_scored_per_sec",
+            "value": n / (ms * 1e-3), "unit": "schedules/s", "ms_per_call": ms, "steps": steps,
+            "config": {"workload": name, "batch": n, "words_per_row": W32, "rows": S, "l2": FLUSH_NOTE},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "algorithmic_bytes": alg_bytes, "peak_source": src}}
 
 
 # Algorithmic thread instructions of the trace kernels per (unit, step): one Philox4x32-10 for the noise (10 rounds
@@ -205,55 +297,37 @@ def trace_alg_thread_instr(bursts):
     return 60 + 22 + (62 if bursts else 0) + 18
 
 
-def run_trace_kernel(args):
-    """The trace kernel alone (synthetic access sets) on the largest configuration: plain-ALU (issue-slot) roofline.
+def trace_kernel_record(steps, warmup):
+    """The trace kernels alone (synthetic access sets) on the largest configuration: plain-ALU (issue-slot) roofline.
 
     long_70b: 640 groups of 4096 units, 64 steps, k = 205, bursts on; two passes (scores by a thread per unit, then one
-    selection per group and step). Besides the issue-slot roofline the line gives the rate of 32 x 32 -> 64 bit
-    multiplies (20 per Philox block, 2 in the AR(1) update) against the multiplier pipe: the score pass keeps that
-    pipe 90% busy, a wide multiply occupying a scheduler's pipe for four cycles per warp (both from ncu). Memory traffic: the int32 score matrix written once and read once (2 * U * S * 4 = 1.3 GB) and
-    the output (S * W32 * 4 = 21 MB), reported as GB/s beside the instruction rate.
+    selection per group and step). Besides the issue-slot roofline the record gives the rate of 32 x 32 -> 64 bit
+    multiplies (20 per Philox block, 2 in the AR(1) update) against the multiplier pipe. Memory traffic: the int32
+    score matrix written once and read once (2 * U * S * 4 = 1.3 GB) and the output (S * W32 * 4 = 21 MB), reported
+    as GB/s beside the instruction rate.
     """
     import torch
     from paper_2508_13231_b200 import kvp, workloads as wl
-    torch.cuda.set_device(0)
     name = "long_70b"
     cfg = wl.CONFIGS[name]
     tp = wl.trace_params(name, seed=0)
     U, S, W32 = wl.units(cfg), cfg["steps"], wl.words_per_row(cfg)
     base = torch.from_numpy(tp["base"]).cuda() if tp["base"] is not None else None
     targs = {k: v for k, v in tp.items() if k not in ("base", "seed")}
-    stream = torch.cuda.current_stream()
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    for w in range(max(3, args.warmup)):
-        kvp.trace_generate(**targs, seed=100 + w, base=base)
-    torch.cuda.synchronize()
-    total_ms = 0.0
-    for k in range(args.steps):
-        flush.fill_(k & 255)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        kvp.trace_generate(**targs, seed=k, base=base)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        total_ms += e0.elapsed_time(e1)
-    ms = total_ms / args.steps
+    ms = _timed_calls(torch, lambda k: kvp.trace_generate(**targs, seed=k, base=base), steps, warmup)
     alg = trace_alg_thread_instr(bool(tp.get("burst_thr"))) / 32.0 * U * S           # warp instructions
-    wide = 42 if tp.get("burst_thr") else 22                                         # 32 x 32 -> 64 bit multiplies per (unit, step)
+    wide = 42 if tp.get("burst_thr") else 22                                         # wide multiplies per (unit, step)
     achieved = alg / (ms * 1e-3) / 1e9
-    print(json.dumps({
-        "kernel": "trace_scores_unit_kernel + trace_select_kernel (kvp_trace_generate)", "metric": "unit_steps_per_sec", "value": U * S / (ms * 1e-3),
-        "unit": "unit-steps/s", "ms_per_call": ms, "steps": args.steps,
-        "config": {"workload": name, "groups": cfg["groups"], "units_per_group": cfg["units_per_group"], "rows": S,
-                   "topk": cfg["topk"], "l2": "flushed with a 256 MB write between timed iterations"},
-        "roofline": {"bound": "alu", "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s",
-                     "frac": achieved / ISSUE_PEAK_GWIPS, "traffic": None,
-                     "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)",
-                     "wide_multiplies": {"achieved": wide * U * S / (ms * 1e-3) / 1e12, "peak": WIDE_MUL_PEAK_T,
-                                         "unit": "T multiplies/s", "frac": wide * U * S / (ms * 1e-3) / 1e12 / WIDE_MUL_PEAK_T,
-                                         "per_unit_step": wide},
-                     "memory_gbs": (2 * U * S * 4 + S * W32 * 4 + (U * 4 if base is not None else 0)) / (ms * 1e-3) / 1e9}}))
+    return {"kernel": "trace_scores_unit_kernel + trace_select_kernel (kvp_trace_generate)", "metric": "unit_steps_per_sec",
+            "value": U * S / (ms * 1e-3), "unit": "unit-steps/s", "ms_per_call": ms, "steps": steps,
+            "config": {"workload": name, "groups": cfg["groups"], "units_per_group": cfg["units_per_group"], "rows": S,
+                       "topk": cfg["topk"], "l2": FLUSH_NOTE},
+            "roofline": {"bound": "alu", "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s",
+                         "frac": achieved / ISSUE_PEAK_GWIPS, "traffic": None, "peak_source": PEAK_SOURCE_ALU,
+                         "wide_multiplies": {"achieved": wide * U * S / (ms * 1e-3) / 1e12, "peak": WIDE_MUL_PEAK_T,
+                                             "unit": "T multiplies/s",
+                                             "frac": wide * U * S / (ms * 1e-3) / 1e12 / WIDE_MUL_PEAK_T, "per_unit_step": wide},
+                         "memory_gbs": (2 * U * S * 4 + S * W32 * 4 + (U * 4 if base is not None else 0)) / (ms * 1e-3) / 1e9}}
 
 
 def run_growing(args):
@@ -277,11 +351,7 @@ def run_growing(args):
     chains, moves = cfg["chains"], cfg["moves"]
     stream = torch.cuda.current_stream()
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    g = torch.Generator(device="cuda"); g.manual_seed(3)
-    w32 = (U + 31) // 32
-    scheds = torch.randint(-2 ** 31, 2 ** 31 - 1, (4, S, w32), dtype=torch.int32, device="cuda", generator=g)
-    for _ in range(3):                                        # ~6% density, below the capacity
-        scheds &= torch.randint(-2 ** 31, 2 ** 31 - 1, (4, S, w32), dtype=torch.int32, device="cuda", generator=g)
+    scheds = _thinned_schedules(torch, 4, S, (U + 31) // 32, seed=3)
 
     def step(seed):
         A = kvp.trace_generate(**targs, seed=seed, base=base, layers=cfg["layers"], birth=birth)
@@ -309,11 +379,11 @@ def run_growing(args):
     achieved = ALG_WARP_INSTR_PER_MOVE * chains * moves / (cms * 1e-3) / 1e9
     line = {"metric": METRIC, "value": chains * moves / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": args.steps,
             "config": {"workload": name, "units": U, "steps": S, "layers": cfg["layers"], "chains": chains, "moves": moves,
-                       "p0": cfg["p0"], "l2": "flushed with a 256 MB write between timed iterations"},
-            "roofline": {"bound": "alu", "kernel": "chain_kernel<global, growing>", "achieved": achieved,
-                         "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
-                         "traffic": None, "ms_per_launch": cms,
-                         "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"},
+                       "p0": cfg["p0"], "l2": FLUSH_NOTE},
+            "roofline": {"bound": "alu", "kernel": "chain kernel, schedules in global memory, growing cache",
+                         "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s",
+                         "frac": achieved / ISSUE_PEAK_GWIPS, "traffic": None, "ms_per_launch": cms,
+                         "peak_source": PEAK_SOURCE_ALU},
             "anneal_ms": {"init": out["stats"].ms_init, "chains": out["stats"].ms_chains, "finish": out["stats"].ms_finish},
             "bound_ticks": out["best_ticks"], "init_ticks": out["stats"].init_ticks}
     if not args.no_cpu_baseline:
@@ -324,131 +394,220 @@ def run_growing(args):
         n = 2
         res, _, _ = o.anneal_chains(o.make_params(chains=chains, moves=moves, seed=0, p0=cfg["p0"]), 0, n)
         dt = time.perf_counter() - t0
-        line["cpu_baseline"] = {"value": sum(r.moves_done for r in res) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+        line["cpu_baseline"] = {"value": sum(r.moves_done for r in res) / dt, "unit": UNIT, "cores": 1,
+                                "host_cores": os.cpu_count(), "kind": "oracle",
                                 "sample": f"chains 0..{n - 1} of {chains}, all {moves} moves each, plus trace and "
                                           f"set-up; {dt:.1f} s on one thread"}
     print(json.dumps(line))
 
 
-def time_to_bound(kvp, cfg, targs, base_dev, U, S):
-    """Outside the timed region: wall time of kvp_anneal (all of its kernels, warm) to reach the bound.
+def time_to_bound(prob, cfg):
+    """Wall time of kvp_anneal (all of its kernels, warm) to reach the bound, on a problem that exists already.
 
     full: the whole budget, the stop rule off. early_stop: the same call with the paper's rule on (a chain stops at
     a level boundary when its best improved by less than 0.1% since the previous one). smallest_budget: the smallest
     of moves/16, /8, /4, /2, moves whose bound is within 0.1% of the full-budget bound, and its wall time.
+    converged says whether doubling the budget from moves/2 to moves still moved the bound by more than 0.1%.
     """
     import torch
-    A = kvp.trace_generate(**targs, seed=0, base=base_dev)
-    prob = kvp.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"])
 
     def run(moves, permille=0):
         prm = prob.make_params(chains=cfg["chains"], moves=moves, seed=0, p0=cfg["p0"], early_stop_permille=permille)
-        prob.anneal(prm, want_schedule=False)                       # warm
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         out = prob.anneal(prm, want_schedule=False)
         torch.cuda.synchronize()
-        return out["best_ticks"], 1e3 * (time.perf_counter() - t0), out["stats"].moves_total
+        return out["best_ticks"], 1e3 * (time.perf_counter() - t0), out["stats"].moves_total, out["stats"].init_ticks
 
-    full_ticks, full_ms, _ = run(cfg["moves"])
-    es_ticks, es_ms, es_moves = run(cfg["moves"], permille=1)
-    res = {"full_budget": {"moves_per_chain": cfg["moves"], "bound_ticks": full_ticks, "ms": full_ms},
-           "early_stop_0.1pct": {"bound_ticks": es_ticks, "ms": es_ms, "moves_executed": es_moves}}
-    for div in (16, 8, 4, 2, 1):
-        ticks, ms, _ = run(cfg["moves"] // div)
-        if (ticks - full_ticks) * 1000 <= full_ticks:
-            res["smallest_budget_within_0.1pct"] = {"moves_per_chain": cfg["moves"] // div, "bound_ticks": ticks, "ms": ms}
+    run(max(1, cfg["moves"] // 16))                                # warm: workspace, kernel attributes
+    full_ticks, full_ms, _, init = run(cfg["moves"])
+    es_ticks, es_ms, es_moves, _ = run(cfg["moves"], permille=1)
+    res = {"init_ticks": init,
+           "full_budget": {"moves_per_chain": cfg["moves"], "bound_ticks": full_ticks, "ms": full_ms},
+           "early_stop_0.1pct": {"bound_ticks": es_ticks, "ms": es_ms, "moves_executed": es_moves},
+           "budgets": {}}
+    for div in (16, 8, 4, 2):
+        ticks, ms, _, _ = run(cfg["moves"] // div)
+        res["budgets"][str(cfg["moves"] // div)] = {"bound_ticks": ticks, "ms": ms}
+    res["budgets"][str(cfg["moves"])] = {"bound_ticks": full_ticks, "ms": full_ms}
+    for m, r in sorted(((int(k), v) for k, v in res["budgets"].items())):
+        if (r["bound_ticks"] - full_ticks) * 1000 <= full_ticks:
+            res["smallest_budget_within_0.1pct"] = {"moves_per_chain": m, **r}
             break
-    prob.close()
+    half = res["budgets"][str(cfg["moves"] // 2)]["bound_ticks"]
+    res["converged"] = bool((half - full_ticks) * 1000 <= full_ticks)
+    res["note"] = ("the bound still improves with the budget: a throughput measurement, not a converged bound"
+                   if not res["converged"] else
+                   "doubling the budget to the full one moves the bound by less than 0.1%")
+    res["improvement_over_initial_permille"] = round((init - full_ticks) * 1000.0 / init, 3)
     return res
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# The whole path
+
+class PathBench:
+    """One named configuration: inputs resident on the device and in pinned host memory, and the step itself."""
+
+    def __init__(self, name, rank, world, p0=None):
+        import numpy as np
+        import torch
+        from paper_2508_13231_b200 import kvp, sharding, workloads as wl
+        self.torch, self.kvp, self.sharding = torch, kvp, sharding
+        self.name, self.rank, self.world = name, rank, world
+        self.cfg = cfg = wl.CONFIGS[name]
+        tp = wl.trace_params(name, seed=0)
+        self.U, self.S, self.W32 = wl.units(cfg), cfg["steps"], wl.words_per_row(cfg)
+        self.chains, self.moves = cfg["chains"], cfg["moves"]
+        self.p0 = cfg["p0"] if p0 is None else p0
+        self.n_eval = 8 if self.U * self.S <= (1 << 24) else 2
+        if self.U <= 65536:
+            sched = torch.from_numpy(wl.random_schedules(self.U, self.S, cfg["cap"], self.n_eval, seed=5).view(np.int32))
+        else:
+            sched = _thinned_schedules(torch, self.n_eval, self.S, self.W32, seed=5).cpu()
+        self.scheds_host = sched.pin_memory()
+        self.base_host = torch.from_numpy(tp["base"]).pin_memory() if tp["base"] is not None else None
+        self.result_host = torch.empty((self.S, self.W32), dtype=torch.int32).pin_memory()
+        self.targs = {k: v for k, v in tp.items() if k not in ("base", "seed")}
+        self.scheds_dev = self.scheds_host.to("cuda")
+        self.base_dev = self.base_host.to("cuda") if self.base_host is not None else None
+        self.flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")     # > 126 MB L2
+        self.launches = 0
+
+    def step(self, seed, base_dev, scheds_dev, dist=None, want_per_chain=False):
+        """One pass of the hot path -> the result dict of kvp_anneal."""
+        kvp, cfg = self.kvp, self.cfg
+        A = kvp.trace_generate(**self.targs, seed=seed, base=base_dev)
+        prob = kvp.Problem(self.U, cfg["bytes_per_unit"], self.S, A, cfg["cap"], *cfg["bw"])
+        prob.eval(scheds_dev, want_steps=False)
+        first, count = self.sharding.chain_range(self.rank, self.world, self.world * self.chains)
+        prm = prob.make_params(chains=count, moves=self.moves, seed=seed, p0=self.p0, first_chain=first)
+        out = prob.anneal(prm, want_per_chain=want_per_chain)
+        if dist is not None:          # the cross-rank part of the reduction: MIN over one (ticks, chain) pair per rank
+            out["global_best"] = self.sharding.combine_best(dist, out["best_ticks"], out["stats"].best_chain, device="cuda")
+        # kernels: 2 trace (scores, select) + 6 create (clean, popcount, transpose, unit counts, histogram,
+        #          static row) + 2 eval (count, finish) + those kvp_anneal reports
+        self.launches = 2 + 6 + 2 + out["stats"].kernel_launches
+        prob.close()
+        return out
+
+    def timed(self, n_steps, e2e, dist=None):
+        """-> (total ms, chain-kernel ms, chain-kernel launches, last result)"""
+        torch = self.torch
+        stream = torch.cuda.current_stream()
+        total_ms, chain_ms, chain_launches, out = 0.0, 0.0, 0, None
+        for k in range(n_steps):
+            self.flush.fill_(k & 255)                                # evict L2 between timed iterations
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            if e2e:
+                b = self.base_host.to("cuda", non_blocking=True) if self.base_host is not None else None
+                sc = self.scheds_host.to("cuda", non_blocking=True)
+                out = self.step(k, b, sc, dist)
+                self.result_host.copy_(out["best_schedule"], non_blocking=True)   # device -> host read of the result
+            else:
+                out = self.step(k, self.base_dev, self.scheds_dev, dist)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            total_ms += e0.elapsed_time(e1)
+            chain_ms += out["stats"].ms_chains
+            chain_launches += out["stats"].chain_launches
+        return total_ms, chain_ms, chain_launches, out
+
+    def warm(self, n, dist=None):
+        for w in range(n):
+            self.step(1000 + w, self.base_dev, self.scheds_dev, dist)
+        self.torch.cuda.synchronize()
+
+    def h2d_bytes(self):
+        return self.scheds_host.numel() * 4 + (self.base_host.numel() * 4 if self.base_host is not None else 0)
+
+    def d2h_bytes(self):
+        return self.result_host.numel() * 4 + 16
+
+    def roofline(self, chain_ms, chain_launches, n_steps, out):
+        """Issue-slot roofline of the chain kernel from the device time the library measured around its launches."""
+        st = out["stats"]
+        per_launch_ms = chain_ms / max(1, chain_launches)
+        moves_per_launch = float(st.moves_total) * n_steps / max(1, chain_launches)
+        achieved = ALG_WARP_INSTR_PER_MOVE * moves_per_launch / (per_launch_ms * 1e-3) / 1e9
+        return {"bound": "alu", "kernel": "chain kernel (%s)" % ("schedules in shared memory" if self.U * self.S <= (1 << 18)
+                                                                  else "schedules in global memory"),
+                "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
+                "traffic": None, "ms_per_launch": per_launch_ms, "launches_per_step": chain_launches / max(1, n_steps),
+                "chains_per_launch": int(st.resident_chains), "algorithmic_warp_instr_per_move": ALG_WARP_INSTR_PER_MOVE,
+                "peak_source": PEAK_SOURCE_ALU}
+
+
+def side_record(name, steps, p0=None):
+    """A smaller configuration measured the same way in the same run (device-resident inputs only)."""
+    b = PathBench(name, 0, 1, p0=p0)
+    b.warm(3)
+    total_ms, chain_ms, launches, out = b.timed(steps, e2e=False)
+    st = out["stats"]
+    extra = b.step(0, b.base_dev, b.scheds_dev, want_per_chain=True)            # untimed: the share of applied moves
+    changed = sum(r.n_changed for r in extra["per_chain"]) / float(extra["stats"].moves_total)
+    rec = {"workload": name, "p0": b.p0, "value": b.chains * b.moves * steps / (total_ms * 1e-3), "unit": UNIT,
+           "ms_per_step": total_ms / steps, "steps": steps, "chains": b.chains, "moves": b.moves,
+           "roofline": b.roofline(chain_ms, launches, steps, out),
+           "state_changing_share": changed, "bound_ticks": out["best_ticks"], "init_ticks": st.init_ticks}
+    return rec
+
+
+def _relaunch_under_torchrun(args):
+    """`python bench.py --gpus N` with N > 1 outside torch.distributed.run: start N ranks on this node."""
+    port = 29500 + (os.getpid() % 2000)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    return subprocess.call(cmd, env=env)
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="kvp", choices=["kvp", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD, help="named configuration of the path benchmark (default: the largest)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="leave out the side records (single_head, kernels, time to bound)")
     ap.add_argument("--kernel", default="path", choices=["path", "cost", "trace", "growing"],
                     help="path: the whole hot path (the benchmark line); cost / trace: that kernel alone on full-size rows; "
                          "growing: the whole path on a growing cache with (token, layer) steps")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
-    if args.kernel == "cost":
-        return run_cost_kernel(args)
-    if args.kernel == "trace":
-        return run_trace_kernel(args)
     if args.kernel == "growing":
         return run_growing(args)
+    if args.kernel in ("cost", "trace"):
+        import torch
+        torch.cuda.set_device(0)
+        rec = cost_kernel_record(args.steps, args.warmup) if args.kernel == "cost" else trace_kernel_record(args.steps, args.warmup)
+        print(json.dumps(rec))
+        return 0
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return _relaunch_under_torchrun(args)
 
-    import numpy as np
     import torch
     import torch.distributed as dist
-    from paper_2508_13231_b200 import kvp, sharding, workloads as wl
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but {world} rank(s) were started")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    cfg = wl.CONFIGS[WORKLOAD]
-    tp = wl.trace_params(WORKLOAD, seed=0)
-    U, S = wl.units(cfg), cfg["steps"]
-    chains, moves = cfg["chains"], cfg["moves"]
-    n_eval = 8
-    scheds_host = torch.from_numpy(wl.random_schedules(U, S, cfg["cap"], n_eval, seed=5).view(np.int32)).pin_memory()
-    base_host = torch.from_numpy(tp["base"]).pin_memory()
-    targs = {k: v for k, v in tp.items() if k not in ("base", "seed")}
-    stream = torch.cuda.current_stream()
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")     # > 126 MB L2
-    launches = [0]
-
-    def step(seed, base_dev, scheds_dev):
-        """One pass of the hot path. Returns (best_ticks, stats, best_schedule)."""
-        A = kvp.trace_generate(**targs, seed=seed, base=base_dev)
-        prob = kvp.Problem(U, cfg["bytes_per_unit"], S, A, cfg["cap"], *cfg["bw"])
-        prob.eval(scheds_dev, want_steps=False)
-        first, count = sharding.chain_range(rank, world, world * chains)
-        prm = prob.make_params(chains=count, moves=moves, seed=seed, p0=cfg["p0"], first_chain=first)
-        out = prob.anneal(prm)
-        # kernels: 2 trace (scores, select) + 6 create (clean, popcount, transpose, unit counts, histogram,
-        #          static row) + 2 eval (count, finish) + those kvp_anneal reports
-        launches[0] = 2 + 6 + 2 + out["stats"].kernel_launches
-        prob.close()
-        return out
-
-    def timed(n_steps, e2e):
-        total_ms, chain_ms, last = 0.0, 0.0, None
-        for k in range(n_steps):
-            flush.fill_(k & 255)                                   # evict L2 between timed iterations
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            if e2e:
-                b = base_host.to("cuda", non_blocking=True)
-                sc = scheds_host.to("cuda", non_blocking=True)
-                out = step(k, b, sc)
-                sched_host = out["best_schedule"].to("cpu")         # device -> host read of the result
-                last = (out, sched_host)
-            else:
-                out = step(k, base_dev, scheds_dev)
-                last = (out, None)
-            e1.record(stream)
-            torch.cuda.synchronize()
-            total_ms += e0.elapsed_time(e1)
-            chain_ms += out["stats"].ms_chains
-        return total_ms, chain_ms, last
-
-    base_dev = base_host.to("cuda")
-    scheds_dev = scheds_host.to("cuda")
-    for w in range(max(3, args.warmup)):
-        step(1000 + w, base_dev, scheds_dev)
-    torch.cuda.synchronize()
+    d = dist if world > 1 else None
+    warmup = max(3, args.warmup)
+    b = PathBench(args.workload, rank, world)
+    b.warm(warmup, d)
 
     def barrier():
         if world > 1:
@@ -466,49 +625,56 @@ def main():
     th = threading.Thread(target=_clock_sampler, args=(stop, samples), daemon=True)
     th.start()
     barrier()
-    total_ms, chain_ms, (out, _) = timed(args.steps, e2e=False)
+    total_ms, chain_ms, chain_launches, out = b.timed(args.steps, e2e=False, dist=d)
     barrier()
     stop.set(); th.join()
     total_ms = max_over_ranks(total_ms)
-    # the cross-rank part of the reduction: two 8-byte MIN reductions over (ticks, chain)
-    if world > 1:
-        sharding.combine_best(dist, out["best_ticks"], out["stats"].best_chain, device="cuda")
     barrier()
-    e2e_ms, _, (out2, sched_host) = timed(args.steps, e2e=True)
+    e2e_ms, _, _, out2 = b.timed(args.steps, e2e=True, dist=d)
     barrier()
     e2e_ms = max_over_ranks(e2e_ms)
 
     if rank == 0:
-        work = float(world) * chains * moves * args.steps
-        value = work / (total_ms * 1e-3)
-        per_launch_ms = chain_ms / args.steps
-        achieved = ALG_WARP_INSTR_PER_MOVE * chains * moves / (per_launch_ms * 1e-3) / 1e9
+        work = float(world) * b.chains * b.moves * args.steps
+        st = out["stats"]
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "metric": METRIC, "value": work / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int32/uint64 ticks", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "units": U, "steps": S, "chains_per_gpu": chains, "moves": moves,
-                       "p0": cfg["p0"], "l2": "flushed with a 256 MB write between timed iterations",
-                       "eval_batch": n_eval},
+            "config": {"workload": b.name, "units": b.U, "steps": b.S, "chains_per_gpu": b.chains, "moves": b.moves,
+                       "p0": b.p0, "start": "near-greedy (p0 of the configuration, not the paper's 0.8; see single_head_p0_0.8)",
+                       "l2": FLUSH_NOTE, "eval_batch": b.n_eval},
             "clocks": _clock_summary(samples),
-            "e2e": {"value": work / (e2e_ms * 1e-3), "unit": UNIT,
-                    "h2d_bytes_per_step": base_host.numel() * 4 + scheds_host.numel() * 4,
-                    "d2h_bytes_per_step": sched_host.numel() * 4 + 16},
-            "gpu_launches": launches[0] * args.steps,
-            "roofline": {"bound": "alu", "kernel": "chain_kernel<smem>", "achieved": achieved,
-                         "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
-                         "traffic": CHAIN_KERNEL_DRAM_BYTES, "ncu": CHAIN_KERNEL_NCU, "ms_per_launch": per_launch_ms,
-                         "peak_source": "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"},
-            "bound_ticks": out["best_ticks"], "init_ticks": out["stats"].init_ticks,
+            "e2e": {"value": work / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": b.h2d_bytes(),
+                    "d2h_bytes_per_step": b.d2h_bytes()},
+            "gpu_launches": b.launches * args.steps,
+            "roofline": b.roofline(chain_ms, chain_launches, args.steps, out),
+            "anneal_ms": {"init": st.ms_init, "chains": st.ms_chains, "finish": st.ms_finish},
+            "bound_ticks": out["best_ticks"], "init_ticks": st.init_ticks,
         }
-        if world == 1:
-            line["time_to_bound"] = time_to_bound(kvp, cfg, targs, base_dev, U, S)
+        if world > 1:
+            line["global_best"] = list(out["global_best"])
+        if world == 1 and not args.no_extras:
+            # further records of the same run: the benchmark configuration's time to bound, the shared-memory
+            # configuration at both start temperatures, and the two streaming kernels alone
+            A = b.kvp.trace_generate(**b.targs, seed=0, base=b.base_dev)
+            prob = b.kvp.Problem(b.U, b.cfg["bytes_per_unit"], b.S, A, b.cfg["cap"], *b.cfg["bw"])
+            line["time_to_bound"] = time_to_bound(prob, b.cfg)
+            prob.close()
+            del A, prob
+            b.scheds_dev = b.flush = None
+            torch.cuda.empty_cache()
+            if b.name != "single_head":
+                line["single_head"] = side_record("single_head", 20)
+            line["single_head_p0_0.8"] = side_record("single_head", 20, p0=0.8)
+            line["kernels"] = {"cost": cost_kernel_record(10, 3), "trace": trace_kernel_record(10, 3)}
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(cfg, tp)
+            line["cpu_baseline"] = cpu_baseline(b.name)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main() or 0)

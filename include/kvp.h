@@ -242,6 +242,8 @@ typedef struct {
     float    ms_init, ms_chains, ms_finish;   /* device time of the three phases (CUDA events)     */
     uint32_t kernel_launches;   /* kernels this call launched                                      */
     kvp_chain_result* per_chain; /* (host) [chains] or NULL                                        */
+    uint32_t chain_launches;    /* launches of the chain kernel (waves of resident chains)         */
+    uint32_t resident_chains;   /* chains per wave                                                 */
 } kvp_anneal_stats;
 
 /*

@@ -1352,6 +1352,7 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
         cudaEventElapsedTime(&stats->ms_chains, ev[1], ev[2]);
         cudaEventElapsedTime(&stats->ms_finish, ev[2], ev[3]);
         stats->kernel_launches = c.launches;
+        stats->chain_launches = waves; stats->resident_chains = c.resident;
     }
     return ok ? KVP_OK : KVP_ERR_INTERNAL;
 }

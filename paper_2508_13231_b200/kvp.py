@@ -72,7 +72,7 @@ class AnnealStats(C.Structure):
         ("best_move", C.c_uint64), ("moves_total", C.c_uint64), ("calib_mean_delta", C.c_uint64), ("temp0", C.c_double),
         ("winner_hits", C.c_uint64), ("winner_accessed", C.c_uint64),
         ("ms_init", C.c_float), ("ms_chains", C.c_float), ("ms_finish", C.c_float), ("kernel_launches", C.c_uint32),
-        ("per_chain", C.POINTER(ChainResult)),
+        ("per_chain", C.POINTER(ChainResult)), ("chain_launches", C.c_uint32), ("resident_chains", C.c_uint32),
     ]
 
 

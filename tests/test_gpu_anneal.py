@@ -164,25 +164,64 @@ def test_anneal_layer_8b_global_state(kvp, oracle):
     assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
 
 
-@pytest.mark.parametrize("name,chains,moves", [("full_8b", 128, 20_000), ("long_70b", 96, 20_000)])
-def test_anneal_full_size_sampled_chains(kvp, oracle, name, chains, moves):
-    # full-size problems, reduced chain count and budget; the oracle recomputes a sample of the chains
+def _spread(chains):
+    """Chain indices that fall into every wave of a job however it is cut: both ends, both sides of every 1/8th
+    boundary (waves are equal parts of the job), and a few in between."""
+    picks = {0, 1, chains - 2, chains - 1}
+    for k in range(1, 8):
+        picks |= {k * chains // 8 - 1, k * chains // 8}
+    picks |= {(k * 2654435761) % chains for k in range(1, 5)}
+    return sorted(picks)
+
+
+@pytest.mark.parametrize("name,moves,p0", [("full_8b", 6000, 1e-6), ("full_8b", 6000, 0.3), ("long_70b", 6000, 1e-6),
+                                            ("long_70b", 6000, 0.3)])
+def test_anneal_full_shape_all_waves(kvp, oracle, name, moves, p0):
+    """The two large configurations at their real shape and chain count (4096 and 8192 chains, which come in several
+    waves of resident chains; later waves take over the scratch of earlier ones), with a reduced move budget so that
+    the oracle can follow: the access bitmap is the oracle's own (and the trace kernel's full-size output is compared
+    with it), about twenty chains spread over every wave plus the winner are recomputed by the oracle on the host
+    cores, all eight per-chain outputs and the winner's schedule bit for bit. Near-greedy and hot start."""
+    from oracle_pool import oracle_chains_sampled, oracle_trace_parallel
     cfg = wl.CONFIGS[name]
-    U, S, cap = wl.units(cfg), cfg["steps"], cfg["cap"]
-    A = to_np(trace_on_gpu(kvp, wl.trace_params(name, seed=0)))
-    g, o = both_problems(kvp, oracle, U, cfg["bytes_per_unit"], S, A, cap, cfg["bw"])
-    kw = dict(chains=chains, moves=moves, seed=0, p0=1e-3)
-    gp, op = _params(g, o, **kw)
-    out = g.anneal(gp, want_per_chain=True)
-    temps, mean = o.temps(op)
-    assert out["stats"].calib_mean_delta == mean
-    for c in (0, chains // 2, chains - 1):
-        want, _, _ = o.anneal_chains(op, c, 1)
-        assert out["per_chain"][c].astuple() == want[0].astuple(), c
-    # properties at full size: the winner's schedule re-scores to the bound and respects Eq. 5
+    U, S, cap, chains = wl.units(cfg), cfg["steps"], cfg["cap"], cfg["chains"]
+    A, path = oracle_trace_parallel(name, 0)
+    assert np.array_equal(to_np(trace_on_gpu(kvp, wl.trace_params(name, seed=0))), A)
+    g = kvp.Problem(U, cfg["bytes_per_unit"], S, to_dev(A), cap, *cfg["bw"])
+    kw = dict(chains=chains, moves=moves, seed=0, p0=p0, levels=8)
+    out = g.anneal(g.make_params(**kw), want_per_chain=True)
+    st = out["stats"]
+    w = st.best_chain
+    assert w == min(range(chains), key=lambda c: (out["per_chain"][c].best_ticks, c))
+    mean, want, best = oracle_chains_sampled(name, path, kw, _spread(chains), want_best=[w])
+    assert st.calib_mean_delta == mean
+    for c, tup in want.items():
+        assert out["per_chain"][c].astuple() == tup, c
+    assert np.array_equal(to_np(out["best_schedule"]), best[w])
+    assert out["best_ticks"] == want[w][0] <= st.init_ticks
+    assert st.moves_total == sum(r.moves_done for r in out["per_chain"])
     ev = g.eval(out["best_schedule"])
     assert int(ev["total_ticks"][0]) == out["best_ticks"] and int(ev["bad_step"][0]) == -1
-    assert out["best_ticks"] <= out["stats"].init_ticks
+    if p0 > 0.1:
+        assert min(r.n_changed for r in out["per_chain"]) > 100       # the hot start rewrites hundreds of units
+
+
+def test_anneal_layer_8b_stated_budget(kvp, oracle):
+    """layer_8b at its stated 1024 chains x 200,000 moves; the oracle recomputes a spread of the chains and the winner."""
+    from oracle_pool import oracle_chains_sampled, oracle_trace_parallel
+    name = "layer_8b"
+    cfg = wl.CONFIGS[name]
+    A, path = oracle_trace_parallel(name, 0)
+    g = kvp.Problem(wl.units(cfg), cfg["bytes_per_unit"], cfg["steps"], to_dev(A), cfg["cap"], *cfg["bw"])
+    kw = dict(chains=cfg["chains"], moves=cfg["moves"], seed=0, p0=cfg["p0"])
+    out = g.anneal(g.make_params(**kw), want_per_chain=True)
+    w = out["stats"].best_chain
+    mean, want, best = oracle_chains_sampled(name, path, kw, _spread(cfg["chains"]), want_best=[w])
+    assert out["stats"].calib_mean_delta == mean
+    for c, tup in want.items():
+        assert out["per_chain"][c].astuple() == tup, c
+    assert np.array_equal(to_np(out["best_schedule"]), best[w]) and out["best_ticks"] == want[w][0]
+    assert out["stats"].moves_total == cfg["chains"] * cfg["moves"]
 
 
 def test_global_state_winner_paths(kvp, oracle, warps_per_chain):

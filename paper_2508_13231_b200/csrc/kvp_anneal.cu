@@ -14,6 +14,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <type_traits>
 #include <vector>
 
 #include "kvp_common.cuh"
@@ -805,6 +806,490 @@ chain_kernel(const ChainParams prm)
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// The wide chain kernel: one warp per chain, kRows proposals per lane, so a batch is 32 * kRows consecutive moves.
+//
+// Most proposals are settled by the placement bits alone: a swap of two units with equal placement over the run
+// changes nothing, a flip into a full step is infeasible (Eq. 5). Every lane first classifies its kRows proposals
+// that way (the Philox draws and the window loads of the rows are independent, so the warp has instruction-level
+// parallelism where the narrow kernel has none). Only the rest, typically a tenth to a third, needs the access
+// windows, the set of steps whose cardinalities change and Eq. 2-4 at those steps: their indices are compacted into
+// a list, and the warp works the list off 32 at a time, one proposal per lane, through the shared work queue of
+// (proposal, step) items. The commit walks the batch in move order and applies every accepted, state-changing
+// proposal it meets until it reaches one whose step range meets that of a move applied since it was evaluated;
+// those are evaluated again, all at once, and the walk goes on from there. The outcome is the sequential chain's.
+constexpr int kRows = 4;
+constexpr uint32_t kWide = 32 * kRows;
+constexpr uint32_t kWideQueueSlots4 = (32 * 31 * 2 + 15) / 16;     // the items of one pass of 32 proposals
+
+template <typename CT> __device__ __forceinline__ uint4 ctr_load(const CT* c, uint32_t t);
+template <> __device__ __forceinline__ uint4 ctr_load<uint4>(const uint4* c, uint32_t t) { return c[t]; }
+template <> __device__ __forceinline__ uint4 ctr_load<ushort4>(const ushort4* c, uint32_t t)
+{
+    const ushort4 v = c[t];
+    return make_uint4(v.x, v.y, v.z, v.w);
+}
+template <typename CT> __device__ __forceinline__ void ctr_store(CT* c, uint32_t t, uint4 v);
+template <> __device__ __forceinline__ void ctr_store<uint4>(uint4* c, uint32_t t, uint4 v) { c[t] = v; }
+template <> __device__ __forceinline__ void ctr_store<ushort4>(ushort4* c, uint32_t t, uint4 v)
+{
+    c[t] = make_ushort4((unsigned short)v.x, (unsigned short)v.y, (unsigned short)v.z, (unsigned short)v.w);
+}
+
+// Where a chain of the wide kernel keeps its state. CT: the four per-step cardinalities as 16-bit fields when the
+// schedule lives in shared memory (then units < 2^16), as 32-bit fields otherwise.
+template <typename CT>
+struct WideView {
+    uint32_t* P;                 // [U][S32] schedule, time-packed (shared or global)
+    CT* ctr;                     // [S] {hr, mi, mo, occ} (shared)
+    uint32_t* full;              // [S32] bit t set iff occ[t] == cap (shared)
+    uint32_t* hb;                // growing cache: [S] units written to HBM at birth (shared)
+    uint4* win;                  // [kWide][2] by proposal: {pk, u, v, -} until it is evaluated, then its windows
+    int* acc;                    // [kWide] by proposal: its cost change being summed
+    uint8_t* nt;                 // [kWide] the proposals that need a cost evaluation, compacted
+    uint16_t* queue;             // [32 * 31] work items (proposal << 5 | window bit) of one pass
+};
+
+// shared-memory words (as uint4 slots) of one chain of the wide kernel besides its schedule
+__host__ __device__ inline uint32_t wide_fixed4(uint32_t S, uint32_t S32, bool grow, bool ctr16, bool touch)
+{
+    return (ctr16 ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (touch ? 1u : 0u) + 2 * kWide +
+           kWide / 4 + kWide / 16 + kWideQueueSlots4;
+}
+
+// What the placement bits alone say about a proposal: does any bit change, and would a flip raise a full step.
+template <bool GROW, typename PPtr, typename FPtr>
+__device__ __forceinline__ void classify(PPtr P, FPtr full, const uint32_t* __restrict__ birth, uint32_t S, uint32_t S32,
+                                         uint32_t pk, uint32_t u, uint32_t v, bool& chg, bool& inf)
+{
+    const bool swap = pk & 1u;
+    const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
+    const uint32_t run = min(s0 + len, S) - s0;
+    const uint32_t M = ((1u << run) - 1u) << 1;
+    const uint32_t Wu = window(P + (size_t)u * S32, S32, s0);
+    uint32_t other = 0xFFFFFFFFu;                                 // a flip toggles every bit of the run
+    if (swap) other = Wu ^ window(P + (size_t)v * S32, S32, s0);
+    uint32_t live = 0xFFFFFFFFu;
+    if (GROW) {
+        uint32_t Lu, Lv, Bu, Bv;
+        alive_born(__ldg(birth + u), s0, Lu, Bu);
+        alive_born(__ldg(birth + (swap ? v : u)), s0, Lv, Bv);
+        live = Lu & Lv;
+    }
+    const uint32_t D = other & M & live;
+    chg = D != 0;
+    inf = false;
+    if (!swap) inf = (~Wu & D & window(full, S32, s0)) != 0;
+}
+
+// N queue items per lane, items base + 32 r + lane: the cost change of one step of one proposal each, added to the
+// proposal's sum.
+template <bool GROW, bool ASMEM, int N, typename CT>
+__device__ __forceinline__ void wide_items(const WideView<CT> cv, const StepC* __restrict__ stepc, const CostK K, uint32_t S,
+                                           uint32_t base, uint32_t count, uint32_t lane)
+{
+    int d[N];
+    uint32_t id[N];
+    bool live[N];
+#pragma unroll
+    for (int r = 0; r < N; ++r) {
+        const uint32_t g = base + 32 * r + lane;
+        live[r] = g < count;
+        const uint32_t item = cv.queue[live[r] ? g : 0u];         // a dead lane repeats item 0 and drops the result
+        id[r] = item >> 5;
+        const uint32_t k = item & 31u;
+        const uint4 w0 = cv.win[id[r] * 2], w1 = cv.win[id[r] * 2 + 1];
+        Windows wn;
+        wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
+        wn.born = w1.w;
+        const uint32_t t = min(wn.s0 + k - 1, S - 1);
+        const StepC sc = ASMEM ? stepc[t] : __ldg(stepc + t);
+        d[r] = item_delta<GROW>(wn, k, ctr_load<CT>(cv.ctr, t), GROW ? cv.hb[t] : 0u, sc, K);
+    }
+#pragma unroll
+    for (int r = 0; r < N; ++r)
+        if (live[r] && d[r]) atomicAdd(cv.acc + id[r], d[r]);
+}
+
+// Per-lane record of the kRows proposals a lane owns in the current batch. Row h of lane l is move m + 32 h + l.
+// inf / acc / chg: one bit per row.
+struct WideMoves {
+    uint32_t pk[kRows], u[kRows], v[kRows], w[kRows];
+    int delta[kRows];
+    uint32_t inf, acc, chg;
+};
+
+// Evaluation of the proposals named by `need` (one lane mask per row) against the current state.
+template <bool GROW, bool ASMEM, typename CT>
+__device__ __forceinline__ void wide_evaluate(const WideView<CT> cv, const uint32_t* __restrict__ Acol,
+                                              const uint32_t* __restrict__ birth, const StepC* __restrict__ stepc,
+                                              const CostK K, uint32_t S, uint32_t S32, const uint32_t* __restrict__ trow,
+                                              uint32_t shift, const uint32_t (&need)[kRows], uint32_t lane, WideMoves& mv)
+{
+    const uint32_t below = (1u << lane) - 1u;
+    // 1. placement bits only; the proposals that need more are listed
+    uint32_t listed = 0;                                          // proposals listed so far (warp-uniform)
+    uint32_t mine = 0;                                            // bit h: this lane's row h is listed
+#pragma unroll
+    for (int h = 0; h < kRows; ++h) {
+        if (!need[h]) continue;                                   // warp-uniform
+        const bool named = (need[h] >> lane) & 1u;
+        bool chg = false, inf = false;
+        if (named) classify<GROW>(cv.P, cv.full, birth, S, S32, mv.pk[h], mv.u[h], mv.v[h], chg, inf);
+        const bool more = named && chg && !inf;
+        if (named) {
+            const uint32_t bit = 1u << h;
+            mv.chg = chg ? mv.chg | bit : mv.chg & ~bit;
+            mv.inf = inf ? mv.inf | bit : mv.inf & ~bit;
+            mv.acc = inf ? mv.acc & ~bit : mv.acc | bit;          // nothing changes: cost change 0, always accepted
+            mv.delta[h] = 0;
+        }
+        const uint32_t mb = __ballot_sync(0xFFFFFFFFu, more);
+        if (more) {
+            const uint32_t id = h * 32 + lane;
+            cv.nt[listed + __popc(mb & below)] = (uint8_t)id;
+            cv.win[id * 2] = make_uint4(mv.pk[h], mv.u[h], mv.v[h], 0u);
+            cv.acc[id] = 0;
+            mine |= 1u << h;
+        }
+        listed += __popc(mb);
+    }
+    if (!listed) return;                                          // warp-uniform
+    __syncwarp();
+    // 2. the listed proposals, 32 at a time, one per lane: windows, the steps whose cost changes, and those (proposal,
+    //    step) items through the shared queue
+    for (uint32_t first = 0; first < listed; first += 32) {
+        const uint32_t g = first + lane;
+        const bool live = g < listed;
+        const uint32_t id = cv.nt[live ? g : first];
+        const uint4 who = cv.win[id * 2];
+        LaneMove lm;
+        lm.pk = who.x; lm.u = who.y; lm.v = who.z; lm.w = 0u; lm.delta = 0; lm.inf = lm.acc = lm.chg = false;
+        Windows wn;
+        const uint32_t tm = lane_windows<GROW>(cv.P, Acol, cv.full, birth, S, S32, lm, wn);
+        __syncwarp();                                             // every lane has read its {pk, u, v}
+        const uint32_t todo = live ? tm : 0u;
+        if (live) {
+            cv.win[id * 2] = make_uint4(wn.Wu, wn.Wv, wn.Nu, wn.Nv);
+            cv.win[id * 2 + 1] = make_uint4(wn.Au, wn.Av, wn.s0, wn.born);
+        }
+        const uint32_t cnt = __popc(todo);
+        uint32_t pos = 0, total = 0;
+#pragma unroll
+        for (int bit = 0; bit < 5; ++bit) {
+            const uint32_t has = __ballot_sync(0xFFFFFFFFu, (cnt >> bit) & 1u);
+            pos += __popc(has & below) << bit;
+            total += __popc(has) << bit;
+        }
+        if (total) {
+#pragma unroll
+            for (uint32_t k = 1; k < 32; ++k) {
+                const uint32_t bit = (todo >> k) & 1u;
+                if (bit) cv.queue[pos] = (uint16_t)((id << 5) | k);
+                pos += bit;
+            }
+            __syncwarp();
+            for (uint32_t base = 0; base < total; base += 64) {
+                if (base + 32 < total) wide_items<GROW, ASMEM, 2>(cv, stepc, K, S, base, total, lane);
+                else wide_items<GROW, ASMEM, 1>(cv, stepc, K, S, base, total, lane);
+            }
+        }
+        __syncwarp();
+    }
+    // 3. the owners take the sums and decide
+#pragma unroll
+    for (int h = 0; h < kRows; ++h)
+        if ((mine >> h) & 1u) {
+            const int d = cv.acc[h * 32 + lane];
+            mv.delta[h] = d;
+            const uint32_t bit = 1u << h;
+            mv.acc = metropolis(d, mv.w[h], trow, shift) ? mv.acc | bit : mv.acc & ~bit;
+        }
+}
+
+// Apply the proposal whose windows are in slot `id` (pk, u, v given): all lanes take part, lane j updates the
+// counters of window bit j, lanes 0 and 1 rewrite the words of the schedule and of the full-step bitmap.
+template <bool GROW, typename CT>
+__device__ __forceinline__ void wide_apply(const WideView<CT> cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
+                                           uint32_t id, uint32_t pk, uint32_t u, uint32_t v)
+{
+    const uint4 w0 = cv.win[id * 2], w1 = cv.win[id * 2 + 1];
+    const uint32_t Wu = w0.x, Wv = w0.y, Nu = w0.z, Nv = w0.w, Au = w1.x, Av = w1.y;
+    const bool swap = pk & 1u;
+    const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
+    const uint32_t run = min(s0 + len, S) - s0;
+    const uint32_t nl = min(s0 + len, S - 1) - s0 + 1;
+    const bool valid = lane >= 1 && lane <= nl;
+    const uint32_t j = valid ? lane : 1u, t = s0 + j - 1;
+    const uint32_t pu = (Wu >> j) & 1u, qu = (Wu >> (j - 1)) & 1u, npu = (Nu >> j) & 1u, nqu = (Nu >> (j - 1)) & 1u;
+    const uint32_t pv = (Wv >> j) & 1u, qv = (Wv >> (j - 1)) & 1u, npv = (Nv >> j) & 1u, nqv = (Nv >> (j - 1)) & 1u;
+    const uint32_t au = (Au >> j) & 1u, av = (Av >> j) & 1u;
+    uint4 c = ctr_load<CT>(cv.ctr, t);
+    c.x += (au & npu) - (au & pu) + (av & npv) - (av & pv);
+    if (GROW) {
+        const uint32_t mu = (w1.w & 255u) == j ? 0u : 1u, mw = ((w1.w >> 8) & 255u) == j ? 0u : 1u;
+        c.y += mu * ((npu & ~nqu) - (pu & ~qu)) + mw * ((npv & ~nqv) - (pv & ~qv));
+        const uint32_t dh = (1u - mu) * (npu - pu) + (1u - mw) * (npv - pv);
+        if (valid && dh) cv.hb[t] += dh;
+    } else {
+        c.y += (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
+    }
+    c.z += (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
+    c.w += npu - pu + npv - pv;
+    if (valid) ctr_store<CT>(cv.ctr, t, c);
+    uint32_t F = __ballot_sync(0xFFFFFFFFu, valid && c.w == cap);   // bit j <-> window bit j
+    uint32_t V = __ballot_sync(0xFFFFFFFFu, valid);
+    if (lane < 2) {
+        uint32_t M = ((1u << run) - 1u) << 1, NU = Nu, NV = Nv, sbit = s0 - 1;
+        if (s0 == 0) { F >>= 1; V >>= 1; M >>= 1; NU >>= 1; NV >>= 1; sbit = 0; }
+        const uint32_t wj = (sbit >> 5) + lane, sh = sbit & 31u;
+        if (wj < S32 && (lane == 0 || sh != 0)) {
+            // lane 0 holds the part of the window that falls into the first word, lane 1 the spill-over
+            const uint32_t Vx = lane ? V >> (32 - sh) : V << sh, Fx = lane ? F >> (32 - sh) : F << sh;
+            const uint32_t Mx = lane ? M >> (32 - sh) : M << sh;
+            const uint32_t NUx = lane ? NU >> (32 - sh) : NU << sh, NVx = lane ? NV >> (32 - sh) : NV << sh;
+            if (Vx) cv.full[wj] = (cv.full[wj] & ~Vx) | (Fx & Vx);
+            if (Mx) {
+                const size_t iu = (size_t)u * S32 + wj;
+                cv.P[iu] = (cv.P[iu] & ~Mx) | (NUx & Mx);
+                if (swap) {
+                    const size_t iv = (size_t)v * S32 + wj;
+                    cv.P[iv] = (cv.P[iv] & ~Mx) | (NVx & Mx);
+                }
+            }
+        }
+    }
+    __syncwarp();
+}
+
+// warp-uniform masks, one per row, indexed by a run-time row number without leaving the registers
+__device__ __forceinline__ uint32_t row_get(const uint32_t (&a)[kRows], uint32_t h)
+{
+    uint32_t r = a[0];
+#pragma unroll
+    for (int k = 1; k < kRows; ++k) r = h == (uint32_t)k ? a[k] : r;
+    return r;
+}
+__device__ __forceinline__ void row_set(uint32_t (&a)[kRows], uint32_t h, uint32_t val)
+{
+#pragma unroll
+    for (int k = 0; k < kRows; ++k) a[k] = h == (uint32_t)k ? val : a[k];
+}
+
+// PSMEM: the schedule lives in shared memory (16-bit counters); otherwise in the chain's slice of global scratch.
+// ASMEM (only with PSMEM): access bitmap and step constants staged in shared memory once per CTA.
+// TOUCH (only without PSMEM): the chain logs the units it rewrites, and may start from a slice that holds the final
+// state of an earlier chain with such a log (ChainParams::restore).
+template <bool PSMEM, bool GROW, bool ASMEM, bool TOUCH>
+__global__ void __launch_bounds__(512)
+wide_chain_kernel(const ChainParams prm)
+{
+    static_assert(!TOUCH || !PSMEM, "touch logs only for schedules in global scratch");
+    static_assert(PSMEM || !ASMEM, "shared access bitmap only beside shared schedules");
+    using CT = typename std::conditional<PSMEM, ushort4, uint4>::type;
+    extern __shared__ uint4 smem4[];
+    const uint32_t lane = threadIdx.x & 31, cic = threadIdx.x >> 5;
+    const uint32_t cpb = blockDim.x >> 5;                         // chains per CTA
+    const uint32_t slot = blockIdx.x * cpb + cic;
+    const bool active = slot < prm.chain_count;
+    if (!ASMEM && !active) return;
+    const uint32_t chain = prm.chain_first + slot;
+    const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
+    const size_t pwords = (size_t)U * S32;
+    const uint32_t c4 = PSMEM ? (S + 1) / 2 : S;                  // uint4 slots of the counters
+    const uint32_t f4 = (S32 + 3) / 4, h4 = GROW ? (S + 3) / 4 : 0u;
+    constexpr uint32_t t4 = TOUCH ? 1u : 0u;
+    const uint32_t fixed4 = wide_fixed4(S, S32, GROW, PSMEM, TOUCH);
+    uint4* const mine4 = smem4 + (size_t)cic * fixed4;
+    WideView<CT> cv;
+    cv.ctr = reinterpret_cast<CT*>(mine4);
+    cv.full = reinterpret_cast<uint32_t*>(mine4 + c4);
+    cv.hb = reinterpret_cast<uint32_t*>(mine4 + c4 + f4);
+    uint32_t* const touched = reinterpret_cast<uint32_t*>(mine4 + c4 + f4 + h4);   // TOUCH: entries in the chain's log
+    cv.win = mine4 + c4 + f4 + h4 + t4;
+    cv.acc = reinterpret_cast<int*>(cv.win + 2 * kWide);
+    cv.nt = reinterpret_cast<uint8_t*>(cv.win + 2 * kWide + kWide / 4);
+    cv.queue = reinterpret_cast<uint16_t*>(cv.win + 2 * kWide + kWide / 4 + kWide / 16);
+    uint32_t* const pool = reinterpret_cast<uint32_t*>(smem4 + (size_t)cpb * fixed4);   // schedules, then A, then constants
+    cv.P = PSMEM ? pool + (size_t)cic * pwords : prm.ws + (size_t)slot * pwords;
+    const uint32_t* Acol = prm.Acol;
+    const StepC* stepc = prm.stepc;
+    if (ASMEM) {
+        const size_t a_off = ((size_t)cpb * pwords + 3) & ~(size_t)3, c_off = (a_off + pwords + 3) & ~(size_t)3;
+        uint32_t* const a_s = pool + a_off;
+        StepC* const c_s = reinterpret_cast<StepC*>(pool + c_off);
+        copy_words(a_s, prm.Acol, pwords, threadIdx.x, blockDim.x);
+        for (uint32_t i = threadIdx.x; i < S; i += blockDim.x) c_s[i] = __ldg(prm.stepc + i);
+        Acol = a_s;
+        stepc = c_s;
+    }
+    if (active) {
+        for (uint32_t i = lane; i < S; i += 32) ctr_store<CT>(cv.ctr, i, __ldg(prm.counters0 + i));
+        for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
+        if (GROW)
+            for (uint32_t i = lane; i < S; i += 32) cv.hb[i] = __ldg(prm.hb0 + i);
+        bool whole = true;
+        if (TOUCH && prm.restore) {
+            const uint32_t n = __ldcg(prm.touch_len + slot);
+            if (n <= prm.touch_cap) {
+                whole = false;
+                const uint32_t* tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
+                for (uint32_t i = lane; i < n; i += 32) {
+                    const size_t o = (size_t)__ldcg(tlog + i) * S32;
+                    for (uint32_t w = 0; w < S32; ++w) cv.P[o + w] = __ldg(prm.Pcol0 + o + w);
+                }
+            }
+        }
+        if (whole) copy_words(cv.P, prm.Pcol0, pwords, lane, 32);
+        if (TOUCH && lane == 0) *touched = 0u;
+    }
+    if (ASMEM) {
+        __syncthreads();
+        if (!active) return;
+    } else {
+        __syncwarp();
+    }
+    uint32_t* snap = prm.snap ? prm.snap + (size_t)slot * pwords : nullptr;
+    uint64_t* ulog = prm.undo_log ? prm.undo_log + (size_t)slot * prm.undo_cap : nullptr;
+
+    uint64_t cur = prm.init_ticks, best = cur, best_move = ~0ull, best_at_boundary = cur;
+    uint64_t n_chg = 0, hash = 0, n_acc = 0, n_inf = 0;
+    bool snap_dirty = false;                                      // the best state is the current one, not yet saved
+    uint32_t ulen = 0;                                            // moves applied since the best state
+
+    uint64_t lvl_start = 0;
+    bool stop = false;
+    for (uint32_t level = 0; level < prm.levels && lvl_start < prm.upto; ++level) {
+        const uint64_t lvl_len = (level + 1 < prm.levels ? min(lvl_start + prm.per_level, prm.upto) : prm.upto) - lvl_start;
+        const uint32_t shift = __ldg(prm.shifts + level);
+        const uint32_t* trow = prm.table + (size_t)level * KVP_TABLE_Q;
+        if (level > 0) {
+            if (prm.early_permille && level >= prm.early_from &&
+                (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille) {
+                stop = true;
+                break;
+            }
+            best_at_boundary = best;
+        }
+        for (uint64_t off = 0; off < lvl_len; off += kWide) {
+            const uint64_t m = lvl_start + off;
+            const uint32_t nb = (uint32_t)min((uint64_t)kWide, lvl_len - off);
+            WideMoves mv;
+            mv.inf = mv.acc = mv.chg = 0u;
+            uint32_t todo[kRows], need[kRows], stale[kRows];
+#pragma unroll
+            for (int h = 0; h < kRows; ++h) {
+                uint32_t r[4];
+                const uint64_t mine = m + 32u * h + lane;
+                philox4x32_10((uint32_t)mine, (uint32_t)(mine >> 32), chain, TAG_MOVE, prm.keys, r);
+                LaneMove lm;
+                decode_move(r, prm.p_swap_256, prm.len_choices, S, U, lm);
+                mv.pk[h] = lm.pk; mv.u[h] = lm.u; mv.v[h] = lm.v; mv.w[h] = lm.w; mv.delta[h] = 0;
+                const uint32_t inrow = nb > 32u * h ? nb - 32u * h : 0u;
+                todo[h] = inrow >= 32 ? 0xFFFFFFFFu : (1u << inrow) - 1u;
+                need[h] = todo[h];
+                stale[h] = 0u;
+            }
+            // Evaluate what is named, then commit in move order as far as the evaluations are still good.
+            for (;;) {
+                wide_evaluate<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+                bool stopped = false;
+                for (uint32_t h = 0; h < kRows && !stopped; ++h) {
+                    uint32_t rem = row_get(todo, h);
+                    if (!rem) continue;
+                    const bool infl = (mv.inf >> h) & 1u, accl = (mv.acc >> h) & 1u, chgl = (mv.chg >> h) & 1u;
+                    const uint32_t infb = __ballot_sync(0xFFFFFFFFu, infl);
+                    const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !infl && accl);
+                    const uint32_t blkb = __ballot_sync(0xFFFFFFFFu, !infl && accl && chgl);
+                    for (;;) {
+                        const uint32_t st = row_get(stale, h) & rem, bl = blkb & rem;
+                        const uint32_t fst = st ? __ffs(st) - 1u : 32u, fbl = bl ? __ffs(bl) - 1u : 32u;
+                        if (fbl < fst) {
+                            // the next state-changing move, evaluated against the state as it is now: apply it
+                            const uint32_t bb = fbl;
+                            const uint32_t done = rem & (0xFFFFFFFFu >> (31 - bb));   // the row's moves up to and including bb
+                            n_inf += __popc(infb & done);
+                            n_acc += __popc(accb & done);
+                            rem &= ~done;
+                            ++n_chg;
+                            uint32_t pk = 0, bu = 0, bv = 0;
+                            int delta = 0;
+#pragma unroll
+                            for (int k = 0; k < kRows; ++k)
+                                if (h == (uint32_t)k) { pk = mv.pk[k]; bu = mv.u[k]; bv = mv.v[k]; delta = mv.delta[k]; }
+                            pk = __shfl_sync(0xFFFFFFFFu, pk, bb); bu = __shfl_sync(0xFFFFFFFFu, bu, bb);
+                            bv = __shfl_sync(0xFFFFFFFFu, bv, bb); delta = __shfl_sync(0xFFFFFFFFu, delta, bb);
+                            const uint64_t after = (uint64_t)((int64_t)cur + delta);
+                            if (snap && snap_dirty && after >= best) {    // leaving the best state: save it first
+                                copy_words(snap, cv.P, pwords, lane);
+                                snap_dirty = false;
+                            }
+                            wide_apply<GROW>(cv, S, S32, prm.cap, lane, h * 32 + bb, pk, bu, bv);
+                            if (TOUCH && prm.touch_log && lane == 0) {    // the units whose words no longer are the initial ones
+                                uint32_t* const tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
+                                const uint32_t n = *touched, two = pk & 1u;
+                                if (n < prm.touch_cap) tlog[n] = bu;
+                                if (two && n + 1u < prm.touch_cap) tlog[n + 1u] = bv;
+                                *touched = min(n + 1u + two, prm.touch_cap + 1u);
+                            }
+                            cur = after;
+                            const uint64_t mb = m + 32u * h + bb;
+                            hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
+                            if (cur < best) { best = cur; best_move = mb; snap_dirty = true; ulen = 0; }
+                            else if (ulog) {                              // every move is its own inverse: remember it
+                                if (ulen < prm.undo_cap && lane == 0) ulog[ulen] = mb;
+                                if (ulen <= prm.undo_cap) ++ulen;
+                            }
+                            // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later
+                            // proposal read steps s0 - 1 .. s0 + len: its evaluation is stale iff the two ranges meet.
+                            const uint32_t s0b = pk >> 8, endb = s0b + ((pk >> 1) & 63u);
+#pragma unroll
+                            for (int k = 0; k < kRows; ++k) {
+                                const uint32_t s0 = mv.pk[k] >> 8, end = s0 + ((mv.pk[k] >> 1) & 63u);
+                                const uint32_t ov = __ballot_sync(0xFFFFFFFFu, s0 <= endb + 1 && s0b <= end);
+                                if ((uint32_t)k == h) stale[k] |= ov & rem;
+                                else if ((uint32_t)k > h) stale[k] |= ov & todo[k];
+                            }
+                        } else if (fst < 32u) {
+                            // a proposal whose evaluation is stale comes first: everything before it is settled
+                            const uint32_t done = rem & ((1u << fst) - 1u);
+                            n_inf += __popc(infb & done);
+                            n_acc += __popc(accb & done);
+                            rem &= ~done;
+                            stopped = true;
+                            break;
+                        } else {
+                            n_inf += __popc(infb & rem);
+                            n_acc += __popc(accb & rem);
+                            rem = 0u;
+                            break;
+                        }
+                    }
+                    row_set(todo, h, rem);
+                }
+                if (!stopped) break;
+#pragma unroll
+                for (int k = 0; k < kRows; ++k) { need[k] = stale[k] & todo[k]; stale[k] = 0u; }
+            }
+        }
+        lvl_start += lvl_len;
+    }
+    const uint64_t m_end = stop ? lvl_start : prm.upto;           // moves done when the chain ended
+    if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
+    if (ulog && lane == 0) prm.undo_len[slot] = ulen;
+    if (TOUCH && prm.touch_log && lane == 0) prm.touch_len[slot] = *touched;
+    if (lane == 0) {
+        kvp_chain_result res;
+        res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m_end;
+        res.n_accepted = n_acc; res.n_changed = n_chg; res.n_infeasible = n_inf; res.traj_hash = hash;
+        prm.results[chain - prm.result_base] = res;
+    }
+    if (prm.dump && slot == 0) {
+        __syncwarp();
+        copy_words(prm.dump, cv.P, pwords, lane);
+    }
+}
+
 // Takes a finished chain's schedule back to its best state: the moves applied after the best were logged, each
 // swap or flip is its own inverse, so applying them again in reverse order undoes them. One warp; only the
 // schedule words are touched (the counters are not needed any more).
@@ -951,6 +1436,7 @@ struct Ctx {
     size_t smem_per_warp;    // shared memory per chain
     size_t smem_shared;      // shared memory of the CTA beside its chains (access bitmap and step constants)
     bool asmem;              // the access bitmap and the step constants are staged in shared memory
+    bool wide;               // the wide kernel (one warp per chain, four proposals per lane)
     std::vector<double> temps;
     uint64_t init_ticks, calib_mean;
     uint32_t launches;
@@ -983,11 +1469,26 @@ ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W, bool
     return asmem ? chain_kernel_pick<true, true, false>(grow, W) : chain_kernel_pick<true, false, false>(grow, W);
 }
 
+ChainKernel wide_kernel_for(bool psmem, bool asmem, bool grow, bool touch)
+{
+    if (!psmem) {
+        if (touch) return grow ? wide_chain_kernel<false, true, false, true> : wide_chain_kernel<false, false, false, true>;
+        return grow ? wide_chain_kernel<false, true, false, false> : wide_chain_kernel<false, false, false, false>;
+    }
+    if (asmem) return grow ? wide_chain_kernel<true, true, true, false> : wide_chain_kernel<true, false, true, false>;
+    return grow ? wide_chain_kernel<true, true, false, false> : wide_chain_kernel<true, false, false, false>;
+}
+
+ChainKernel kernel_of(const Ctx& c, bool psmem, bool asmem, uint32_t W, bool touch)
+{
+    return c.wide ? wide_kernel_for(psmem, asmem, c.grow, touch) : chain_kernel_for(psmem, asmem, c.grow, W, touch);
+}
+
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 {
     const uint32_t grid = (count + c.wpb - 1) / c.wpb;
     const size_t smem = (size_t)c.wpb * c.smem_per_warp + c.smem_shared;
-    chain_kernel_for(c.psmem, c.asmem, c.grow, c.wpc, c.touch)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
+    kernel_of(c, c.psmem, c.asmem, c.wpc, c.touch)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }
@@ -1024,7 +1525,11 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const size_t budget = (size_t)smem_max - 1024;
     // per chain: counters, full-step bitmap and, per warp, the batch's windows, accumulators and work queue
     c.grow = p->dL != nullptr;
-    auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false) {
+    const kvp_test_hooks hooks = g_hooks;
+    c.wide = hooks.warps_per_chain == 0;             // the narrow kernels (one proposal per lane) only on request
+    // `shared`: the schedule is in shared memory (the wide kernel then keeps 16-bit counters)
+    auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false, bool shared = true) {
+        if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared, touch) * 16;
         return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq, touch) * 16;
     };
     c.touch = false;
@@ -1033,9 +1538,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     // chains then keeps twice as many warps in flight. kvp_set_test_hooks can override the choice (tests, tuning).
     const uint32_t chains_per_sm = (a->chains + sms - 1) / sms;
     uint32_t W = chains_per_sm <= 8 ? 2u : 1u;
-    const kvp_test_hooks hooks = g_hooks;
     if (hooks.warps_per_chain == 1 || hooks.warps_per_chain == 2) W = hooks.warps_per_chain;
-    c.psmem = fixed_bytes(1) + pbytes <= budget / 2;
+    if (c.wide) W = 1;
+    c.psmem = fixed_bytes(1) + pbytes <= budget / 2 && (!c.wide || p->U < 65536u);
     if (c.psmem) {
         uint32_t want = chains_per_sm < 1 ? 1 : chains_per_sm;
         if (W == 2 && (want > 8 || (fixed_bytes(2) + pbytes) * want > budget) && (fixed_bytes(1) + pbytes) * want <= budget)
@@ -1056,13 +1561,13 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
         } else {
             c.smem_shared = 0;
         }
-        KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(true, c.asmem, c.grow, W, false), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, true, c.asmem, W, false), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
         // planned without the touch logs first; a job that then needs several waves is planned again with them (one
         // more shared-memory slot per chain)
         for (int pass = 0; pass < 2; ++pass) {
             c.touch = pass == 1;
-            const size_t ctr_bytes = fixed_bytes(W, false, c.touch);
+            const size_t ctr_bytes = fixed_bytes(W, false, c.touch, false);
             if (ctr_bytes > budget) return KVP_ERR_RANGE;
             c.smem_per_warp = ctr_bytes;
             c.smem_shared = 0;
@@ -1070,9 +1575,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             c.wpc = W;
             uint32_t wcap = (uint32_t)(budget / ctr_bytes);            // chains per CTA at most
             if (wcap > 16 / W) wcap = 16 / W;
-            KVP_CUDA(cudaFuncSetAttribute(chain_kernel_for(false, false, c.grow, W, c.touch), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+            KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, false, false, W, c.touch), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
             int ctas = 0;
-            KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, chain_kernel_for(false, false, c.grow, W, c.touch), (int)(wcap * W * 32),
+            KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, kernel_of(c, false, false, W, c.touch), (int)(wcap * W * 32),
                                                                    wcap * c.smem_per_warp));
             if (ctas < 1) return KVP_ERR_RANGE;
             uint32_t per_sm = (uint32_t)ctas * wcap;                   // resident chains per SM, at most 32 warps

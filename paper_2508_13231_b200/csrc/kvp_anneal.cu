@@ -57,6 +57,10 @@ struct ChainParams {
     uint32_t touch_cap;
     uint32_t restore;            // the slices hold the final states of chains that started from the same initial
                                  // schedule and logged what they touched: only those units are copied again
+    uint32_t* cow_out;           // wide kernel, schedules in global scratch: [slots][kCowBits / 32] which buckets of
+                                 // units a slot's slice holds when its chain ends (the rest is the initial schedule)
+    uint32_t cow_shift;          // a bucket is 2^cow_shift consecutive units
+    uint32_t stage_stepc;        // wide kernel without a staged access bitmap: the step constants alone are staged
 };
 
 // Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
@@ -819,6 +823,12 @@ chain_kernel(const ChainParams prm)
 // proposal it meets until it reaches one whose step range meets that of a move applied since it was evaluated;
 // those are evaluated again, all at once, and the walk goes on from there. The outcome is the sequential chain's.
 constexpr int kRows = 4;
+// Largest CTA of the wide kernel with schedules in global scratch; it sets the registers a thread may use (65,536
+// per SM over the resident threads), hence how many chains an SM holds at a time.
+#ifndef KVP_WIDE_GLOBAL_THREADS
+#define KVP_WIDE_GLOBAL_THREADS 512
+#endif
+constexpr int kWideGlobalThreads = KVP_WIDE_GLOBAL_THREADS;
 constexpr uint32_t kWide = 32 * kRows;
 constexpr uint32_t kWideQueueSlots4 = (32 * 31 * 2 + 15) / 16;     // the items of one pass of 32 proposals
 
@@ -836,10 +846,49 @@ template <> __device__ __forceinline__ void ctr_store<ushort4>(ushort4* c, uint3
     c[t] = make_ushort4((unsigned short)v.x, (unsigned short)v.y, (unsigned short)v.z, (unsigned short)v.w);
 }
 
+// The copies off the hot path (a bucket fetched into a slice, a best state saved) as one function each, so that the
+// chain loop stays small enough for the instruction cache.
+__device__ __noinline__ void copy_words_cold(uint32_t* dst, const uint32_t* src, size_t n, uint32_t lane)
+{
+    copy_words(dst, src, n, lane);
+}
+
+// Schedules in global scratch are copy-on-write overlays of the one initial schedule that all chains share: the
+// units come in buckets of 2^shift consecutive units, a chain's slice holds a bucket only once the chain has
+// rewritten a unit of it, and a bitmap in shared memory (at most kCowBits buckets) says which. Chains change few of
+// their units, so nearly every placement window is read from the shared initial schedule, which stays in L2, and
+// not from a private slice that only DRAM can hold; a chain that rewrites everything ends up copying its whole
+// slice once, bucket by bucket.
+constexpr uint32_t kCowBits = 8192;
+constexpr uint32_t kCowSlots4 = kCowBits / 128;
+
 // Where a chain of the wide kernel keeps its state. CT: the four per-step cardinalities as 16-bit fields when the
-// schedule lives in shared memory (then units < 2^16), as 32-bit fields otherwise.
-template <typename CT>
+// schedule lives in shared memory (then units < 2^16), as 32-bit fields otherwise. COW: see above.
+template <typename CT, bool COW>
 struct WideView {
+    const uint32_t* p0;          // COW: [U][S32] the initial schedule
+    uint32_t* have;              // COW: [kCowBits / 32] buckets present in P (shared)
+    uint32_t shift, U, S32;      // COW: bucket size; units; words per unit
+    __device__ __forceinline__ const uint32_t* col(uint32_t u) const
+    {
+        if (COW) {
+            const uint32_t b = u >> shift;
+            return ((have[b >> 5] >> (b & 31u)) & 1u ? P : p0) + (size_t)u * S32;
+        }
+        return P + (size_t)u * S32;
+    }
+    // Before unit u is rewritten: its bucket is copied into the slice if it is not there yet (all lanes, u uniform).
+    __device__ __forceinline__ void own(uint32_t u, uint32_t lane) const
+    {
+        if (!COW) return;
+        const uint32_t b = u >> shift;
+        if ((have[b >> 5] >> (b & 31u)) & 1u) return;
+        const size_t lo = (size_t)(b << shift) * S32, hi = (size_t)min(U, (b + 1u) << shift) * S32;
+        copy_words(P + lo, p0 + lo, hi - lo, lane);
+        __syncwarp();
+        if (lane == 0) have[b >> 5] |= 1u << (b & 31u);
+        __syncwarp();
+    }
     uint32_t* P;                 // [U][S32] schedule, time-packed (shared or global)
     CT* ctr;                     // [S] {hr, mi, mo, occ} (shared)
     uint32_t* full;              // [S32] bit t set iff occ[t] == cap (shared)
@@ -850,42 +899,27 @@ struct WideView {
     uint16_t* queue;             // [32 * 31] work items (proposal << 5 | window bit) of one pass
 };
 
-// shared-memory words (as uint4 slots) of one chain of the wide kernel besides its schedule
-__host__ __device__ inline uint32_t wide_fixed4(uint32_t S, uint32_t S32, bool grow, bool ctr16, bool touch)
-{
-    return (ctr16 ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (touch ? 1u : 0u) + 2 * kWide +
-           kWide / 4 + kWide / 16 + kWideQueueSlots4;
-}
+// The scalars of a chain that only an applied move or a level boundary touches: in shared memory, so that the loop
+// over the batches keeps its registers for the proposals.
+struct WideScalars {
+    uint64_t cur, best, best_move, best_at_boundary, n_chg, hash;
+    uint32_t ulen;               // moves applied since the best state
+    uint32_t snap_dirty;         // the best state is the current one and not saved yet
+    uint32_t pad[2];
+};
+constexpr uint32_t kWideScalars4 = sizeof(WideScalars) / 16;
 
-// What the placement bits alone say about a proposal: does any bit change, and would a flip raise a full step.
-template <bool GROW, typename PPtr, typename FPtr>
-__device__ __forceinline__ void classify(PPtr P, FPtr full, const uint32_t* __restrict__ birth, uint32_t S, uint32_t S32,
-                                         uint32_t pk, uint32_t u, uint32_t v, bool& chg, bool& inf)
+// shared-memory words (as uint4 slots) of one chain of the wide kernel besides its schedule
+__host__ __device__ inline uint32_t wide_fixed4(uint32_t S, uint32_t S32, bool grow, bool shared)
 {
-    const bool swap = pk & 1u;
-    const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
-    const uint32_t run = min(s0 + len, S) - s0;
-    const uint32_t M = ((1u << run) - 1u) << 1;
-    const uint32_t Wu = window(P + (size_t)u * S32, S32, s0);
-    uint32_t other = 0xFFFFFFFFu;                                 // a flip toggles every bit of the run
-    if (swap) other = Wu ^ window(P + (size_t)v * S32, S32, s0);
-    uint32_t live = 0xFFFFFFFFu;
-    if (GROW) {
-        uint32_t Lu, Lv, Bu, Bv;
-        alive_born(__ldg(birth + u), s0, Lu, Bu);
-        alive_born(__ldg(birth + (swap ? v : u)), s0, Lv, Bv);
-        live = Lu & Lv;
-    }
-    const uint32_t D = other & M & live;
-    chg = D != 0;
-    inf = false;
-    if (!swap) inf = (~Wu & D & window(full, S32, s0)) != 0;
+    return (shared ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (shared ? 0u : kCowSlots4) + kWideScalars4 +
+           2 * kWide + kWide / 4 + kWide / 16 + kWideQueueSlots4;
 }
 
 // N queue items per lane, items base + 32 r + lane: the cost change of one step of one proposal each, added to the
 // proposal's sum.
-template <bool GROW, bool ASMEM, int N, typename CT>
-__device__ __forceinline__ void wide_items(const WideView<CT> cv, const StepC* __restrict__ stepc, const CostK K, uint32_t S,
+template <bool GROW, int N, typename CT, bool COW>
+__device__ __forceinline__ void wide_items(const WideView<CT, COW> cv, const StepC* __restrict__ stepc, const CostK K, uint32_t S,
                                            uint32_t base, uint32_t count, uint32_t lane)
 {
     int d[N];
@@ -903,7 +937,7 @@ __device__ __forceinline__ void wide_items(const WideView<CT> cv, const StepC* _
         wn.Wu = w0.x; wn.Wv = w0.y; wn.Nu = w0.z; wn.Nv = w0.w; wn.Au = w1.x; wn.Av = w1.y; wn.s0 = w1.z;
         wn.born = w1.w;
         const uint32_t t = min(wn.s0 + k - 1, S - 1);
-        const StepC sc = ASMEM ? stepc[t] : __ldg(stepc + t);
+        const StepC sc = stepc[t];
         d[r] = item_delta<GROW>(wn, k, ctr_load<CT>(cv.ctr, t), GROW ? cv.hb[t] : 0u, sc, K);
     }
 #pragma unroll
@@ -919,24 +953,90 @@ struct WideMoves {
     uint32_t inf, acc, chg;
 };
 
-// Evaluation of the proposals named by `need` (one lane mask per row) against the current state.
-template <bool GROW, bool ASMEM, typename CT>
-__device__ __forceinline__ void wide_evaluate(const WideView<CT> cv, const uint32_t* __restrict__ Acol,
-                                              const uint32_t* __restrict__ birth, const StepC* __restrict__ stepc,
-                                              const CostK K, uint32_t S, uint32_t S32, const uint32_t* __restrict__ trow,
-                                              uint32_t shift, const uint32_t (&need)[kRows], uint32_t lane, WideMoves& mv)
+// Second half of evaluating a proposal that is known to change bits and to be feasible: given its placement windows
+// (Wu; wv = the window of v for a swap), the access windows, the windows after the move and the set of window bits
+// (steps) whose cardinalities, hence cost, change. Same conventions as lane_windows.
+template <bool GROW>
+__device__ __forceinline__ uint32_t changed_steps(uint32_t Wu, uint32_t wv, const uint32_t* __restrict__ Acol,
+                                                  const uint32_t* __restrict__ birth, uint32_t S, uint32_t S32,
+                                                  uint32_t pk, uint32_t u, uint32_t v, Windows& wn)
+{
+    const bool swap = pk & 1u;
+    const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
+    const uint32_t run = min(s0 + len, S) - s0;                   // steps whose placement bits change hands
+    const uint32_t nl = min(s0 + len, S - 1) - s0 + 1;            // affected steps: the run and the step after it
+    const uint32_t M = ((1u << run) - 1u) << 1;
+    const uint32_t Sb = ((1u << nl) - 1u) << 1;
+    const uint32_t Au = window(Acol + (size_t)u * S32, S32, s0);
+    const uint32_t av = window(Acol + (size_t)(swap ? v : u) * S32, S32, s0);   // a flip reads unit u twice
+    const uint32_t Av = swap ? av : 0u, Wv = swap ? wv : 0u;
+    uint32_t Bu = 0u, Bv = 0u, live = 0xFFFFFFFFu;
+    if (GROW) {
+        uint32_t Lu, Lv;
+        alive_born(__ldg(birth + u), s0, Lu, Bu);
+        alive_born(__ldg(birth + (swap ? v : u)), s0, Lv, Bv);
+        live = Lu & Lv;
+        if (!swap) Bv = 0u;
+    }
+    const uint32_t D = (swap ? (Wu ^ Wv) : 0xFFFFFFFFu) & M & live;      // bits that toggle
+    uint32_t Nu = Wu ^ D, Nv = swap ? (Wv ^ D) : 0u;
+    if (s0 == 0) {                                                // the virtual step -1 follows step 0
+        Nu = (Nu & ~1u) | ((Nu >> 1) & 1u);
+        Nv = (Nv & ~1u) | ((Nv >> 1) & 1u);
+    }
+    wn.Wu = Wu; wn.Wv = Wv; wn.Nu = Nu; wn.Nv = Nv; wn.Au = Au; wn.Av = Av; wn.s0 = s0;
+    wn.born = GROW ? ((Bu ? 31u - __clz(Bu) : 0u) | ((Bv ? 31u - __clz(Bv) : 0u) << 8)) : 0u;
+    const uint32_t hr = (Au ^ Av) & (Wu ^ Nu);                    // a hit is won or lost (v mirrors u in a swap)
+    const uint32_t euo = (Wu ^ (Wu << 1)) & ~Bu, eun = (Nu ^ (Nu << 1)) & ~Bu;
+    const uint32_t evo = (Wv ^ (Wv << 1)) & ~Bv, evn = (Nv ^ (Nv << 1)) & ~Bv;
+    const uint32_t mg = (euo ^ eun) | (euo & eun & (Wu ^ Nu)) | (evo ^ evn) | (evo & evn & (Wv ^ Nv));
+    const uint32_t wr = ((Wu ^ Nu) & Bu) | ((Wv ^ Nv) & Bv);
+    return (hr | mg | wr) & Sb;
+}
+
+// First half of an evaluation, placement bits only: a swap of equal placements changes nothing, a flip into a full
+// step is infeasible (Eq. 5). The proposals of `need` (per lane: bit h = its row h) that need more are listed in cv.nt
+// with their placement windows parked in their slots. `listed`: how many; `mine`: which of this lane's rows.
+// ALL: nearly every row is named (a fresh batch): the window loads of all rows are issued before any is used, named
+// or not (every row holds a drawn proposal, so every address is good). Otherwise rows without a named proposal are
+// skipped.
+template <bool GROW, bool ALL, typename CT, bool COW>
+__device__ __forceinline__ void wide_classify(const WideView<CT, COW> cv, const uint32_t* __restrict__ birth, uint32_t S,
+                                              uint32_t S32, uint32_t need, uint32_t lane, WideMoves& mv, uint32_t& listed,
+                                              uint32_t& mine)
 {
     const uint32_t below = (1u << lane) - 1u;
-    // 1. placement bits only; the proposals that need more are listed
-    uint32_t listed = 0;                                          // proposals listed so far (warp-uniform)
-    uint32_t mine = 0;                                            // bit h: this lane's row h is listed
+    uint32_t Wu[kRows], Wv[kRows], Fw[kRows], Lv[kRows];
+    bool skip[kRows];
 #pragma unroll
     for (int h = 0; h < kRows; ++h) {
-        if (!need[h]) continue;                                   // warp-uniform
-        const bool named = (need[h] >> lane) & 1u;
-        bool chg = false, inf = false;
-        if (named) classify<GROW>(cv.P, cv.full, birth, S, S32, mv.pk[h], mv.u[h], mv.v[h], chg, inf);
-        const bool more = named && chg && !inf;
+        skip[h] = ALL ? false : !__any_sync(0xFFFFFFFFu, (need >> h) & 1u);
+        Wu[h] = Wv[h] = Fw[h] = 0u; Lv[h] = 0xFFFFFFFFu;
+        if (skip[h]) continue;                                    // warp-uniform
+        const uint32_t pk = mv.pk[h], s0 = pk >> 8;
+        const uint32_t ve = (pk & 1u) ? mv.v[h] : mv.u[h];        // a flip reads unit u twice and ignores the copy
+        Wu[h] = window(cv.col(mv.u[h]), S32, s0);
+        Wv[h] = window(cv.col(ve), S32, s0);
+        Fw[h] = window(cv.full, S32, s0);
+        if (GROW) {
+            uint32_t La, Lb, Bu, Bv;
+            alive_born(__ldg(birth + mv.u[h]), s0, La, Bu);
+            alive_born(__ldg(birth + ve), s0, Lb, Bv);
+            Lv[h] = La & Lb;
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < kRows; ++h) {
+        if (skip[h]) continue;
+        const bool named = (need >> h) & 1u;
+        const uint32_t pk = mv.pk[h];
+        const bool swap = pk & 1u;
+        const uint32_t len = (pk >> 1) & 63u, s0 = pk >> 8;
+        const uint32_t run = min(s0 + len, S) - s0;
+        const uint32_t M = ((1u << run) - 1u) << 1;
+        const uint32_t D = (swap ? Wu[h] ^ Wv[h] : 0xFFFFFFFFu) & M & Lv[h];   // a flip toggles every bit of the run
+        const bool chg = D != 0;
+        const bool inf = !swap && (~Wu[h] & D & Fw[h]) != 0;      // a flip may not raise a full step (Eq. 5)
         if (named) {
             const uint32_t bit = 1u << h;
             mv.chg = chg ? mv.chg | bit : mv.chg & ~bit;
@@ -944,30 +1044,47 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT> cv, const uint3
             mv.acc = inf ? mv.acc & ~bit : mv.acc | bit;          // nothing changes: cost change 0, always accepted
             mv.delta[h] = 0;
         }
+        const bool more = named && chg && !inf;
         const uint32_t mb = __ballot_sync(0xFFFFFFFFu, more);
         if (more) {
             const uint32_t id = h * 32 + lane;
             cv.nt[listed + __popc(mb & below)] = (uint8_t)id;
-            cv.win[id * 2] = make_uint4(mv.pk[h], mv.u[h], mv.v[h], 0u);
+            cv.win[id * 2] = make_uint4(pk, mv.u[h], mv.v[h], Wu[h]);
+            cv.win[id * 2 + 1].x = Wv[h];
             cv.acc[id] = 0;
             mine |= 1u << h;
         }
         listed += __popc(mb);
     }
+}
+
+// Evaluation of the proposals named by `need` (per lane: bit h = its row h) against the current state.
+// fresh: a new batch, nearly every row named (see wide_classify).
+template <bool GROW, typename CT, bool COW>
+__device__ __forceinline__ void wide_evaluate(const WideView<CT, COW> cv, const uint32_t* __restrict__ Acol,
+                                              const uint32_t* __restrict__ birth, const StepC* __restrict__ stepc,
+                                              const CostK K, uint32_t S, uint32_t S32, const uint32_t* __restrict__ trow,
+                                              uint32_t shift, uint32_t need, bool fresh, uint32_t lane, WideMoves& mv)
+{
+    const uint32_t below = (1u << lane) - 1u;
+    // 1. placement bits only; the proposals that need more are listed
+    uint32_t listed = 0;                                          // proposals listed (warp-uniform)
+    uint32_t mine = 0;                                            // bit h: this lane's row h is listed
+    if (fresh) wide_classify<GROW, true>(cv, birth, S, S32, need, lane, mv, listed, mine);
+    else wide_classify<GROW, false>(cv, birth, S, S32, need, lane, mv, listed, mine);
     if (!listed) return;                                          // warp-uniform
     __syncwarp();
-    // 2. the listed proposals, 32 at a time, one per lane: windows, the steps whose cost changes, and those (proposal,
-    //    step) items through the shared queue
+    // 2. the listed proposals, 32 at a time, one per lane: access windows, the steps whose cost changes, and those
+    //    (proposal, step) items through the shared queue
     for (uint32_t first = 0; first < listed; first += 32) {
         const uint32_t g = first + lane;
         const bool live = g < listed;
         const uint32_t id = cv.nt[live ? g : first];
         const uint4 who = cv.win[id * 2];
-        LaneMove lm;
-        lm.pk = who.x; lm.u = who.y; lm.v = who.z; lm.w = 0u; lm.delta = 0; lm.inf = lm.acc = lm.chg = false;
+        const uint32_t wv = cv.win[id * 2 + 1].x;
         Windows wn;
-        const uint32_t tm = lane_windows<GROW>(cv.P, Acol, cv.full, birth, S, S32, lm, wn);
-        __syncwarp();                                             // every lane has read its {pk, u, v}
+        const uint32_t tm = changed_steps<GROW>(who.w, wv, Acol, birth, S, S32, who.x, who.y, who.z, wn);
+        __syncwarp();                                             // every lane has read its proposal
         const uint32_t todo = live ? tm : 0u;
         if (live) {
             cv.win[id * 2] = make_uint4(wn.Wu, wn.Wv, wn.Nu, wn.Nv);
@@ -990,8 +1107,8 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT> cv, const uint3
             }
             __syncwarp();
             for (uint32_t base = 0; base < total; base += 64) {
-                if (base + 32 < total) wide_items<GROW, ASMEM, 2>(cv, stepc, K, S, base, total, lane);
-                else wide_items<GROW, ASMEM, 1>(cv, stepc, K, S, base, total, lane);
+                if (base + 32 < total) wide_items<GROW, 2>(cv, stepc, K, S, base, total, lane);
+                else wide_items<GROW, 1>(cv, stepc, K, S, base, total, lane);
             }
         }
         __syncwarp();
@@ -1009,8 +1126,8 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT> cv, const uint3
 
 // Apply the proposal whose windows are in slot `id` (pk, u, v given): all lanes take part, lane j updates the
 // counters of window bit j, lanes 0 and 1 rewrite the words of the schedule and of the full-step bitmap.
-template <bool GROW, typename CT>
-__device__ __forceinline__ void wide_apply(const WideView<CT> cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
+template <bool GROW, typename CT, bool COW>
+__device__ __forceinline__ void wide_apply(const WideView<CT, COW> cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
                                            uint32_t id, uint32_t pk, uint32_t u, uint32_t v)
 {
     const uint4 w0 = cv.win[id * 2], w1 = cv.win[id * 2 + 1];
@@ -1039,6 +1156,8 @@ __device__ __forceinline__ void wide_apply(const WideView<CT> cv, uint32_t S, ui
     if (valid) ctr_store<CT>(cv.ctr, t, c);
     uint32_t F = __ballot_sync(0xFFFFFFFFu, valid && c.w == cap);   // bit j <-> window bit j
     uint32_t V = __ballot_sync(0xFFFFFFFFu, valid);
+    cv.own(u, lane);
+    if (swap) cv.own(v, lane);
     if (lane < 2) {
         uint32_t M = ((1u << run) - 1u) << 1, NU = Nu, NV = Nv, sbit = s0 - 1;
         if (s0 == 0) { F >>= 1; V >>= 1; M >>= 1; NU >>= 1; NV >>= 1; sbit = 0; }
@@ -1062,56 +1181,55 @@ __device__ __forceinline__ void wide_apply(const WideView<CT> cv, uint32_t S, ui
     __syncwarp();
 }
 
-// warp-uniform masks, one per row, indexed by a run-time row number without leaving the registers
-__device__ __forceinline__ uint32_t row_get(const uint32_t (&a)[kRows], uint32_t h)
+// A whole schedule out of a copy-on-write slice: the buckets the slice holds from it, the rest from the initial one.
+__device__ __forceinline__ void copy_merged(uint32_t* __restrict__ dst, const uint32_t* __restrict__ mine,
+                                            const uint32_t* __restrict__ p0, const uint32_t* have, uint32_t shift,
+                                            uint32_t U, uint32_t S32, uint32_t lane)
 {
-    uint32_t r = a[0];
-#pragma unroll
-    for (int k = 1; k < kRows; ++k) r = h == (uint32_t)k ? a[k] : r;
-    return r;
-}
-__device__ __forceinline__ void row_set(uint32_t (&a)[kRows], uint32_t h, uint32_t val)
-{
-#pragma unroll
-    for (int k = 0; k < kRows; ++k) a[k] = h == (uint32_t)k ? val : a[k];
+    const uint32_t nb = (U + (1u << shift) - 1u) >> shift;
+    for (uint32_t b = 0; b < nb; ++b) {
+        const size_t lo = (size_t)(b << shift) * S32, hi = (size_t)min(U, (b + 1u) << shift) * S32;
+        const uint32_t* src = (have[b >> 5] >> (b & 31u)) & 1u ? mine : p0;
+        copy_words_cold(dst + lo, src + lo, hi - lo, lane);
+    }
 }
 
-// PSMEM: the schedule lives in shared memory (16-bit counters); otherwise in the chain's slice of global scratch.
+// PSMEM: the schedule lives in shared memory (16-bit counters); otherwise the chain's slice of global scratch is a
+// copy-on-write overlay of the initial schedule (see kCowBits).
 // ASMEM (only with PSMEM): access bitmap and step constants staged in shared memory once per CTA.
-// TOUCH (only without PSMEM): the chain logs the units it rewrites, and may start from a slice that holds the final
-// state of an earlier chain with such a log (ChainParams::restore).
-template <bool PSMEM, bool GROW, bool ASMEM, bool TOUCH>
-__global__ void __launch_bounds__(512)
+template <bool PSMEM, bool GROW, bool ASMEM>
+__global__ void __launch_bounds__(PSMEM ? 256 : kWideGlobalThreads, 1)
 wide_chain_kernel(const ChainParams prm)
 {
-    static_assert(!TOUCH || !PSMEM, "touch logs only for schedules in global scratch");
     static_assert(PSMEM || !ASMEM, "shared access bitmap only beside shared schedules");
     using CT = typename std::conditional<PSMEM, ushort4, uint4>::type;
+    constexpr bool COW = !PSMEM;
     extern __shared__ uint4 smem4[];
     const uint32_t lane = threadIdx.x & 31, cic = threadIdx.x >> 5;
     const uint32_t cpb = blockDim.x >> 5;                         // chains per CTA
     const uint32_t slot = blockIdx.x * cpb + cic;
     const bool active = slot < prm.chain_count;
-    if (!ASMEM && !active) return;
     const uint32_t chain = prm.chain_first + slot;
     const uint32_t S = prm.S, S32 = prm.S32, U = prm.U;
     const size_t pwords = (size_t)U * S32;
     const uint32_t c4 = PSMEM ? (S + 1) / 2 : S;                  // uint4 slots of the counters
     const uint32_t f4 = (S32 + 3) / 4, h4 = GROW ? (S + 3) / 4 : 0u;
-    constexpr uint32_t t4 = TOUCH ? 1u : 0u;
-    const uint32_t fixed4 = wide_fixed4(S, S32, GROW, PSMEM, TOUCH);
+    constexpr uint32_t o4 = COW ? kCowSlots4 : 0u;
+    const uint32_t fixed4 = wide_fixed4(S, S32, GROW, PSMEM);
     uint4* const mine4 = smem4 + (size_t)cic * fixed4;
-    WideView<CT> cv;
+    WideView<CT, COW> cv;
     cv.ctr = reinterpret_cast<CT*>(mine4);
     cv.full = reinterpret_cast<uint32_t*>(mine4 + c4);
     cv.hb = reinterpret_cast<uint32_t*>(mine4 + c4 + f4);
-    uint32_t* const touched = reinterpret_cast<uint32_t*>(mine4 + c4 + f4 + h4);   // TOUCH: entries in the chain's log
-    cv.win = mine4 + c4 + f4 + h4 + t4;
+    cv.have = reinterpret_cast<uint32_t*>(mine4 + c4 + f4 + h4);
+    WideScalars* const sc = reinterpret_cast<WideScalars*>(mine4 + c4 + f4 + h4 + o4);
+    cv.win = mine4 + c4 + f4 + h4 + o4 + kWideScalars4;
     cv.acc = reinterpret_cast<int*>(cv.win + 2 * kWide);
     cv.nt = reinterpret_cast<uint8_t*>(cv.win + 2 * kWide + kWide / 4);
     cv.queue = reinterpret_cast<uint16_t*>(cv.win + 2 * kWide + kWide / 4 + kWide / 16);
     uint32_t* const pool = reinterpret_cast<uint32_t*>(smem4 + (size_t)cpb * fixed4);   // schedules, then A, then constants
     cv.P = PSMEM ? pool + (size_t)cic * pwords : prm.ws + (size_t)slot * pwords;
+    cv.p0 = prm.Pcol0; cv.shift = prm.cow_shift; cv.U = U; cv.S32 = S32;
     const uint32_t* Acol = prm.Acol;
     const StepC* stepc = prm.stepc;
     if (ASMEM) {
@@ -1122,40 +1240,32 @@ wide_chain_kernel(const ChainParams prm)
         for (uint32_t i = threadIdx.x; i < S; i += blockDim.x) c_s[i] = __ldg(prm.stepc + i);
         Acol = a_s;
         stepc = c_s;
+    } else if (prm.stage_stepc) {                                 // the step constants alone, behind the chains' areas
+        StepC* const c_s = reinterpret_cast<StepC*>(pool + (PSMEM ? (((size_t)cpb * pwords + 3) & ~(size_t)3) : 0));
+        for (uint32_t i = threadIdx.x; i < S; i += blockDim.x) c_s[i] = __ldg(prm.stepc + i);
+        stepc = c_s;
     }
     if (active) {
         for (uint32_t i = lane; i < S; i += 32) ctr_store<CT>(cv.ctr, i, __ldg(prm.counters0 + i));
         for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
         if (GROW)
             for (uint32_t i = lane; i < S; i += 32) cv.hb[i] = __ldg(prm.hb0 + i);
-        bool whole = true;
-        if (TOUCH && prm.restore) {
-            const uint32_t n = __ldcg(prm.touch_len + slot);
-            if (n <= prm.touch_cap) {
-                whole = false;
-                const uint32_t* tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
-                for (uint32_t i = lane; i < n; i += 32) {
-                    const size_t o = (size_t)__ldcg(tlog + i) * S32;
-                    for (uint32_t w = 0; w < S32; ++w) cv.P[o + w] = __ldg(prm.Pcol0 + o + w);
-                }
-            }
+        if (lane == 0) {
+            sc->cur = sc->best = sc->best_at_boundary = prm.init_ticks;
+            sc->best_move = ~0ull; sc->n_chg = 0; sc->hash = 0; sc->ulen = 0u; sc->snap_dirty = 0u;
         }
-        if (whole) copy_words(cv.P, prm.Pcol0, pwords, lane, 32);
-        if (TOUCH && lane == 0) *touched = 0u;
+        if (COW) {
+            for (uint32_t i = lane; i < kCowBits / 32; i += 32) cv.have[i] = 0u;   // the slice holds nothing yet
+        } else {
+            copy_words_cold(cv.P, prm.Pcol0, pwords, lane);
+        }
     }
-    if (ASMEM) {
-        __syncthreads();
-        if (!active) return;
-    } else {
-        __syncwarp();
-    }
+    __syncthreads();
+    if (!active) return;
     uint32_t* snap = prm.snap ? prm.snap + (size_t)slot * pwords : nullptr;
     uint64_t* ulog = prm.undo_log ? prm.undo_log + (size_t)slot * prm.undo_cap : nullptr;
 
-    uint64_t cur = prm.init_ticks, best = cur, best_move = ~0ull, best_at_boundary = cur;
-    uint64_t n_chg = 0, hash = 0, n_acc = 0, n_inf = 0;
-    bool snap_dirty = false;                                      // the best state is the current one, not yet saved
-    uint32_t ulen = 0;                                            // moves applied since the best state
+    uint64_t n_acc = 0, n_inf = 0;                                // per lane: of the proposals this lane owned
 
     uint64_t lvl_start = 0;
     bool stop = false;
@@ -1164,19 +1274,22 @@ wide_chain_kernel(const ChainParams prm)
         const uint32_t shift = __ldg(prm.shifts + level);
         const uint32_t* trow = prm.table + (size_t)level * KVP_TABLE_Q;
         if (level > 0) {
+            const uint64_t best = sc->best, before = sc->best_at_boundary;
             if (prm.early_permille && level >= prm.early_from &&
-                (best_at_boundary - best) * 1000ull < best_at_boundary * (uint64_t)prm.early_permille) {
+                (before - best) * 1000ull < before * (uint64_t)prm.early_permille) {
                 stop = true;
                 break;
             }
-            best_at_boundary = best;
+            __syncwarp();
+            if (lane == 0) sc->best_at_boundary = best;
+            __syncwarp();
         }
         for (uint64_t off = 0; off < lvl_len; off += kWide) {
             const uint64_t m = lvl_start + off;
             const uint32_t nb = (uint32_t)min((uint64_t)kWide, lvl_len - off);
             WideMoves mv;
             mv.inf = mv.acc = mv.chg = 0u;
-            uint32_t todo[kRows], need[kRows], stale[kRows];
+            uint32_t pend = 0u;                                   // bit h: this lane's row h is still to be committed
 #pragma unroll
             for (int h = 0; h < kRows; ++h) {
                 uint32_t r[4];
@@ -1185,33 +1298,42 @@ wide_chain_kernel(const ChainParams prm)
                 LaneMove lm;
                 decode_move(r, prm.p_swap_256, prm.len_choices, S, U, lm);
                 mv.pk[h] = lm.pk; mv.u[h] = lm.u; mv.v[h] = lm.v; mv.w[h] = lm.w; mv.delta[h] = 0;
-                const uint32_t inrow = nb > 32u * h ? nb - 32u * h : 0u;
-                todo[h] = inrow >= 32 ? 0xFFFFFFFFu : (1u << inrow) - 1u;
-                need[h] = todo[h];
-                stale[h] = 0u;
+                if (32u * h + lane < nb) pend |= 1u << h;
             }
+            uint32_t need = pend, stale = 0u;
+            bool first_pass = true;
             // Evaluate what is named, then commit in move order as far as the evaluations are still good.
             for (;;) {
-                wide_evaluate<GROW, ASMEM>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, lane, mv);
+                wide_evaluate<GROW>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, first_pass, lane, mv);
+                first_pass = false;
+                // Nearly always nothing in the batch changes the schedule: every lane counts its own proposals.
+                if (!__any_sync(0xFFFFFFFFu, (mv.acc & mv.chg & ~mv.inf & pend) != 0u)) {
+                    n_inf += __popc(mv.inf & pend);
+                    n_acc += __popc(mv.acc & ~mv.inf & pend);
+                    break;
+                }
                 bool stopped = false;
                 for (uint32_t h = 0; h < kRows && !stopped; ++h) {
-                    uint32_t rem = row_get(todo, h);
+                    uint32_t rem = __ballot_sync(0xFFFFFFFFu, (pend >> h) & 1u);   // the row's lanes still to commit
                     if (!rem) continue;
-                    const bool infl = (mv.inf >> h) & 1u, accl = (mv.acc >> h) & 1u, chgl = (mv.chg >> h) & 1u;
-                    const uint32_t infb = __ballot_sync(0xFFFFFFFFu, infl);
-                    const uint32_t accb = __ballot_sync(0xFFFFFFFFu, !infl && accl);
-                    const uint32_t blkb = __ballot_sync(0xFFFFFFFFu, !infl && accl && chgl);
+                    const bool infl = (mv.inf >> h) & 1u, accl = !infl && ((mv.acc >> h) & 1u);
                     for (;;) {
-                        const uint32_t st = row_get(stale, h) & rem, bl = blkb & rem;
+                        const uint32_t st = __ballot_sync(0xFFFFFFFFu, (stale >> h) & 1u) & rem;
+                        const uint32_t bl = __ballot_sync(0xFFFFFFFFu, accl && ((mv.chg >> h) & 1u)) & rem;
                         const uint32_t fst = st ? __ffs(st) - 1u : 32u, fbl = bl ? __ffs(bl) - 1u : 32u;
+                        // the row's moves that are settled now: up to the next state-changing move (included), or up to
+                        // the first proposal whose evaluation is stale (excluded), or all of them
+                        const uint32_t upto_bit = fbl < fst ? fbl + 1u : fst;
+                        const uint32_t done = upto_bit >= 32u ? rem : rem & ((1u << upto_bit) - 1u);
+                        if ((done >> lane) & 1u) {
+                            n_inf += infl ? 1u : 0u;
+                            n_acc += accl ? 1u : 0u;
+                            pend &= ~(1u << h);
+                        }
+                        rem &= ~done;
                         if (fbl < fst) {
                             // the next state-changing move, evaluated against the state as it is now: apply it
                             const uint32_t bb = fbl;
-                            const uint32_t done = rem & (0xFFFFFFFFu >> (31 - bb));   // the row's moves up to and including bb
-                            n_inf += __popc(infb & done);
-                            n_acc += __popc(accb & done);
-                            rem &= ~done;
-                            ++n_chg;
                             uint32_t pk = 0, bu = 0, bv = 0;
                             int delta = 0;
 #pragma unroll
@@ -1219,74 +1341,69 @@ wide_chain_kernel(const ChainParams prm)
                                 if (h == (uint32_t)k) { pk = mv.pk[k]; bu = mv.u[k]; bv = mv.v[k]; delta = mv.delta[k]; }
                             pk = __shfl_sync(0xFFFFFFFFu, pk, bb); bu = __shfl_sync(0xFFFFFFFFu, bu, bb);
                             bv = __shfl_sync(0xFFFFFFFFu, bv, bb); delta = __shfl_sync(0xFFFFFFFFu, delta, bb);
-                            const uint64_t after = (uint64_t)((int64_t)cur + delta);
-                            if (snap && snap_dirty && after >= best) {    // leaving the best state: save it first
-                                copy_words(snap, cv.P, pwords, lane);
-                                snap_dirty = false;
-                            }
+                            const uint64_t after = (uint64_t)((int64_t)sc->cur + delta);
+                            const bool leaving = snap && sc->snap_dirty && after >= sc->best;
+                            if (leaving) copy_words(snap, cv.P, pwords, lane);   // leaving the best state: save it first
                             wide_apply<GROW>(cv, S, S32, prm.cap, lane, h * 32 + bb, pk, bu, bv);
-                            if (TOUCH && prm.touch_log && lane == 0) {    // the units whose words no longer are the initial ones
-                                uint32_t* const tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
-                                const uint32_t n = *touched, two = pk & 1u;
-                                if (n < prm.touch_cap) tlog[n] = bu;
-                                if (two && n + 1u < prm.touch_cap) tlog[n + 1u] = bv;
-                                *touched = min(n + 1u + two, prm.touch_cap + 1u);
+                            if (lane == 0) {
+                                const uint64_t mb = m + 32u * h + bb;
+                                if (leaving) sc->snap_dirty = 0u;
+                                sc->cur = after;
+                                ++sc->n_chg;
+                                sc->hash = (sc->hash ^ mb) * 0x9E3779B97F4A7C15ull + after;
+                                if (after < sc->best) { sc->best = after; sc->best_move = mb; sc->snap_dirty = 1u; sc->ulen = 0u; }
+                                else if (ulog) {                          // every move is its own inverse: remember it
+                                    const uint32_t ulen = sc->ulen;
+                                    if (ulen < prm.undo_cap) ulog[ulen] = mb;
+                                    if (ulen <= prm.undo_cap) sc->ulen = ulen + 1u;
+                                }
                             }
-                            cur = after;
-                            const uint64_t mb = m + 32u * h + bb;
-                            hash = (hash ^ mb) * 0x9E3779B97F4A7C15ull + cur;
-                            if (cur < best) { best = cur; best_move = mb; snap_dirty = true; ulen = 0; }
-                            else if (ulog) {                              // every move is its own inverse: remember it
-                                if (ulen < prm.undo_cap && lane == 0) ulog[ulen] = mb;
-                                if (ulen <= prm.undo_cap) ++ulen;
-                            }
-                            // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later
+                            __syncwarp();
+                            // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A pending
                             // proposal read steps s0 - 1 .. s0 + len: its evaluation is stale iff the two ranges meet.
                             const uint32_t s0b = pk >> 8, endb = s0b + ((pk >> 1) & 63u);
 #pragma unroll
                             for (int k = 0; k < kRows; ++k) {
                                 const uint32_t s0 = mv.pk[k] >> 8, end = s0 + ((mv.pk[k] >> 1) & 63u);
-                                const uint32_t ov = __ballot_sync(0xFFFFFFFFu, s0 <= endb + 1 && s0b <= end);
-                                if ((uint32_t)k == h) stale[k] |= ov & rem;
-                                else if ((uint32_t)k > h) stale[k] |= ov & todo[k];
+                                if (s0 <= endb + 1 && s0b <= end) stale |= 1u << k;
                             }
+                            stale &= pend;
                         } else if (fst < 32u) {
-                            // a proposal whose evaluation is stale comes first: everything before it is settled
-                            const uint32_t done = rem & ((1u << fst) - 1u);
-                            n_inf += __popc(infb & done);
-                            n_acc += __popc(accb & done);
-                            rem &= ~done;
-                            stopped = true;
+                            stopped = true;                       // a stale evaluation comes first
                             break;
                         } else {
-                            n_inf += __popc(infb & rem);
-                            n_acc += __popc(accb & rem);
-                            rem = 0u;
-                            break;
+                            break;                                // the row is done
                         }
                     }
-                    row_set(todo, h, rem);
                 }
                 if (!stopped) break;
-#pragma unroll
-                for (int k = 0; k < kRows; ++k) { need[k] = stale[k] & todo[k]; stale[k] = 0u; }
+                need = stale & pend;
+                stale = 0u;
             }
         }
         lvl_start += lvl_len;
     }
     const uint64_t m_end = stop ? lvl_start : prm.upto;           // moves done when the chain ended
-    if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
-    if (ulog && lane == 0) prm.undo_len[slot] = ulen;
-    if (TOUCH && prm.touch_log && lane == 0) prm.touch_len[slot] = *touched;
+    // accepted and infeasible proposals were counted by the lanes that owned them
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        n_acc += __shfl_xor_sync(0xFFFFFFFFu, n_acc, off);
+        n_inf += __shfl_xor_sync(0xFFFFFFFFu, n_inf, off);
+    }
+    if (snap && sc->snap_dirty) copy_words_cold(snap, cv.P, pwords, lane);
+    if (ulog && lane == 0) prm.undo_len[slot] = sc->ulen;
+    if (COW && prm.cow_out)                                       // which buckets the slice holds (for the walk back)
+        for (uint32_t i = lane; i < kCowBits / 32; i += 32) prm.cow_out[(size_t)slot * (kCowBits / 32) + i] = cv.have[i];
     if (lane == 0) {
         kvp_chain_result res;
-        res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m_end;
-        res.n_accepted = n_acc; res.n_changed = n_chg; res.n_infeasible = n_inf; res.traj_hash = hash;
+        res.best_ticks = sc->best; res.best_move = sc->best_move; res.final_ticks = sc->cur; res.moves_done = m_end;
+        res.n_accepted = n_acc; res.n_changed = sc->n_chg; res.n_infeasible = n_inf; res.traj_hash = sc->hash;
         prm.results[chain - prm.result_base] = res;
     }
     if (prm.dump && slot == 0) {
         __syncwarp();
-        copy_words(prm.dump, cv.P, pwords, lane);
+        if (COW) copy_merged(prm.dump, cv.P, cv.p0, cv.have, cv.shift, U, S32, lane);
+        else copy_words_cold(prm.dump, cv.P, pwords, lane);
     }
 }
 
@@ -1332,7 +1449,8 @@ undo_kernel(const ChainParams prm, uint32_t slot, uint32_t* __restrict__ dst)
         __syncwarp();
     }
     __syncwarp();
-    copy_words(dst, P, pwords, lane);
+    if (prm.cow_out) copy_merged(dst, P, prm.Pcol0, prm.cow_out + (size_t)slot * (kCowBits / 32), prm.cow_shift, prm.U, S32, lane);
+    else copy_words(dst, P, pwords, lane);
 }
 
 // bit t of full0 is set iff the initial schedule fills the HBM capacity at step t
@@ -1429,6 +1547,8 @@ struct Ctx {
     uint32_t* touch_len;
     uint32_t touch_cap;
     bool touch;              // the chains come in several waves and log the units they rewrite
+    uint32_t* cow_out;       // wide kernel, global variant: bucket bitmaps of the slices, or null
+    uint32_t cow_shift;
     bool psmem;
     uint32_t wpb;            // chains per CTA
     uint32_t wpc;            // warps per chain
@@ -1437,6 +1557,7 @@ struct Ctx {
     size_t smem_shared;      // shared memory of the CTA beside its chains (access bitmap and step constants)
     bool asmem;              // the access bitmap and the step constants are staged in shared memory
     bool wide;               // the wide kernel (one warp per chain, four proposals per lane)
+    bool stage_stepc;        // wide kernel: the step constants are staged in shared memory without the access bitmap
     std::vector<double> temps;
     uint64_t init_ticks, calib_mean;
     uint32_t launches;
@@ -1469,19 +1590,16 @@ ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W, bool
     return asmem ? chain_kernel_pick<true, true, false>(grow, W) : chain_kernel_pick<true, false, false>(grow, W);
 }
 
-ChainKernel wide_kernel_for(bool psmem, bool asmem, bool grow, bool touch)
+ChainKernel wide_kernel_for(bool psmem, bool asmem, bool grow)
 {
-    if (!psmem) {
-        if (touch) return grow ? wide_chain_kernel<false, true, false, true> : wide_chain_kernel<false, false, false, true>;
-        return grow ? wide_chain_kernel<false, true, false, false> : wide_chain_kernel<false, false, false, false>;
-    }
-    if (asmem) return grow ? wide_chain_kernel<true, true, true, false> : wide_chain_kernel<true, false, true, false>;
-    return grow ? wide_chain_kernel<true, true, false, false> : wide_chain_kernel<true, false, false, false>;
+    if (!psmem) return grow ? wide_chain_kernel<false, true, false> : wide_chain_kernel<false, false, false>;
+    if (asmem) return grow ? wide_chain_kernel<true, true, true> : wide_chain_kernel<true, false, true>;
+    return grow ? wide_chain_kernel<true, true, false> : wide_chain_kernel<true, false, false>;
 }
 
 ChainKernel kernel_of(const Ctx& c, bool psmem, bool asmem, uint32_t W, bool touch)
 {
-    return c.wide ? wide_kernel_for(psmem, asmem, c.grow, touch) : chain_kernel_for(psmem, asmem, c.grow, W, touch);
+    return c.wide ? wide_kernel_for(psmem, asmem, c.grow) : chain_kernel_for(psmem, asmem, c.grow, W, touch);
 }
 
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
@@ -1501,6 +1619,7 @@ int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp
     prm.undo_log = with_undo ? c.undo_log : nullptr; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
     prm.touch_log = with_undo ? c.touch_log : nullptr; prm.touch_len = c.touch_len; prm.touch_cap = c.touch_cap;
     prm.restore = with_undo && restore && c.touch_log ? 1u : 0u;
+    prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift; prm.stage_stepc = c.stage_stepc ? 1u : 0u;
     prm.chain_first = first; prm.chain_count = count; prm.result_base = result_base;
     prm.results = results; prm.upto = upto; prm.dump = dump;
     ++c.launches;
@@ -1529,10 +1648,11 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     c.wide = hooks.warps_per_chain == 0;             // the narrow kernels (one proposal per lane) only on request
     // `shared`: the schedule is in shared memory (the wide kernel then keeps 16-bit counters)
     auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false, bool shared = true) {
-        if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared, touch) * 16;
+        if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared) * 16;
         return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq, touch) * 16;
     };
     c.touch = false;
+    c.stage_stepc = false;
     const size_t pbytes = (size_t)p->U * p->S32 * 4;
     // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
     // chains then keeps twice as many warps in flight. kvp_set_test_hooks can override the choice (tests, tuning).
@@ -1547,7 +1667,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             W = 1;                                                 // the second warp's work area does not fit
         c.smem_per_warp = fixed_bytes(W) + pbytes;
         uint32_t wmax = (uint32_t)(budget / c.smem_per_warp);
-        if (wmax > 16 / W) wmax = 16 / W;
+        if (wmax > (c.wide ? 8u : 16u / W)) wmax = c.wide ? 8u : 16u / W;   // the wide kernel is built for CTAs of up to 256 threads
         c.wpb = want > wmax ? wmax : want;
         c.wpc = W;
         c.resident = a->chains;
@@ -1560,6 +1680,12 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             c.smem_shared = with_a - (size_t)c.wpb * c.smem_per_warp;
         } else {
             c.smem_shared = 0;
+            // the wide kernel stages at least the step constants when they fit
+            const size_t with_c = (size_t)c.wpb * c.smem_per_warp + 16 + (size_t)p->S * 16;
+            if (c.wide && with_c <= budget) {
+                c.stage_stepc = true;
+                c.smem_shared = with_c - (size_t)c.wpb * c.smem_per_warp;
+            }
         }
         KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, true, c.asmem, W, false), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
@@ -1573,12 +1699,16 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             c.smem_shared = 0;
             c.asmem = false;
             c.wpc = W;
-            uint32_t wcap = (uint32_t)(budget / ctr_bytes);            // chains per CTA at most
+            // the wide kernel stages the step constants once per CTA when they are small
+            c.stage_stepc = c.wide && (size_t)p->S * 16 <= 32768 && ctr_bytes + (size_t)p->S * 16 <= budget;
+            if (c.stage_stepc) c.smem_shared = (size_t)p->S * 16;
+            uint32_t wcap = (uint32_t)((budget - c.smem_shared) / ctr_bytes);   // chains per CTA at most
             if (wcap > 16 / W) wcap = 16 / W;
+            if (c.wide && wcap > kWideGlobalThreads / 32) wcap = kWideGlobalThreads / 32;
             KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, false, false, W, c.touch), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
             int ctas = 0;
             KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, kernel_of(c, false, false, W, c.touch), (int)(wcap * W * 32),
-                                                                   wcap * c.smem_per_warp));
+                                                                   wcap * c.smem_per_warp + c.smem_shared));
             if (ctas < 1) return KVP_ERR_RANGE;
             uint32_t per_sm = (uint32_t)ctas * wcap;                   // resident chains per SM, at most 32 warps
             if (per_sm * W > 32) per_sm = 32 / W / wcap ? 32 / W / wcap * wcap : wcap;
@@ -1605,9 +1735,12 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
             // a wave is spread over all SMs: CTAs of ceil(resident / SMs) chains where one CTA per SM holds them
             const uint32_t even = (c.resident + sms - 1) / sms;
             c.wpb = even < wcap ? even : wcap;
-            if (a->chains <= c.resident) break;
+            // the wide kernel's slices are overlays of the initial schedule: a later wave just starts an empty one
+            if (a->chains <= c.resident || c.wide) break;
         }
     }
+    c.cow_shift = 0;
+    while (((uint64_t)p->U + (1ull << c.cow_shift) - 1) >> c.cow_shift > kCowBits) ++c.cow_shift;
 
     // workspace layout
     size_t off = 0;
@@ -1633,6 +1766,8 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     const bool touch = c.touch;
     c.touch_cap = touch ? 16384u : 0u;
     const size_t o_tlog = take((size_t)c.resident * c.touch_cap * 4), o_tlen = take(touch ? (size_t)c.resident * 4 : 0);
+    const bool cow = c.wide && !c.psmem;
+    const size_t o_cow = take(cow ? (size_t)c.resident * (kCowBits / 8) : 0);
     rc = ensure_chain_ws(p, off, st);
     if (rc) return rc;
     char* base = static_cast<char*>(p->d_chain_ws);
@@ -1644,6 +1779,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     c.full0 = (uint32_t*)(base + o_full); c.snap = snapshots ? (uint32_t*)(base + o_snap) : nullptr;
     c.undo_log = c.psmem ? nullptr : (uint64_t*)(base + o_ulog); c.undo_len = c.psmem ? nullptr : (uint32_t*)(base + o_ulen);
     c.touch_log = touch ? (uint32_t*)(base + o_tlog) : nullptr; c.touch_len = touch ? (uint32_t*)(base + o_tlen) : nullptr;
+    c.cow_out = cow ? (uint32_t*)(base + o_cow) : nullptr;
 
     // initial schedule in both layouts
     if (a->init_mode == KVP_INIT_USER) {
@@ -1797,6 +1933,7 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
                     ChainParams prm = c.prm;
                     prm.chain_first = a->first_chain + first;
                     prm.undo_log = c.undo_log; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
+                    prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift;
                     if (c.grow) undo_kernel<true><<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
                     else undo_kernel<false><<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
                     KVP_CUDA(cudaGetLastError());

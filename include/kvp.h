@@ -267,8 +267,10 @@ int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint
  *   (entry i belongs to chain first_chain + i)
  * Synchronises `stream` before returning.
  * A job of few chains (at most 8 per SM) is served by two warps per chain that take the chain's batches of 32
- * proposals in turn; the results are those of the sequential chain either way. The only device-side wait of the
- * library is a warp's wait for its turn; it is bounded, and a chain whose wait runs out makes the call return
+ * proposals in turn; a job of many chains by one warp per chain that carries four proposals per lane and keeps the
+ * chains' schedules, when they do not fit shared memory, as copy-on-write overlays of the one initial schedule. The
+ * results are those of the sequential chain either way. The only device-side wait of the library is a warp's wait
+ * for its turn in the two-warp form; it is bounded, and a chain whose wait runs out makes the call return
  * KVP_ERR_TIMEOUT (the outputs are then undefined). The library reads no environment variable; the switches that
  * the test-suite needs are set with kvp_set_test_hooks (end of this header).
  */
@@ -420,7 +422,8 @@ void kvp_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
  * kvp_anneal_chain_state. No production caller needs them. All zero = the library's normal behaviour; NULL resets.
  */
 typedef struct {
-    uint32_t warps_per_chain;   /* 1 or 2: serve every chain with that many warps, whatever the job size         */
+    uint32_t warps_per_chain;   /* 1 or 2: the narrow chain kernel with that many warps per chain; 3: the wide
+                                   chain kernel (one warp, four proposals per lane); whatever the job size       */
     uint32_t drop_turn;         /* 1: withhold one hand-over per chain so that the bounded wait for the turn
                                    runs out (about a second) and the call returns KVP_ERR_TIMEOUT               */
     uint32_t split_queue_plus1; /* n + 1: batches with more than n work items take the rarely reached two-halves

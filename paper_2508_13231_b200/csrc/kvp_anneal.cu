@@ -113,6 +113,42 @@ __device__ __forceinline__ uint32_t window(Ptr col, uint32_t S32, uint32_t s0)
     return s0 ? slid : ((lo << 1) | (lo & 1u));                  // s0 == 0: bit 0 repeats step 0
 }
 
+// The same cut for several columns of one proposal: the position is worked out once.
+struct WinPos {
+    uint32_t w, w2, sh;          // first word, the word after it (clamped), shift
+    bool first;                  // s0 == 0: bit 0 repeats step 0
+};
+__device__ __forceinline__ WinPos window_pos(uint32_t S32, uint32_t s0)
+{
+    WinPos p;
+    const uint32_t b0 = s0 ? s0 - 1 : 0u;
+    p.w = b0 >> 5; p.w2 = min(p.w + 1, S32 - 1); p.sh = b0 & 31u; p.first = s0 == 0;
+    return p;
+}
+// COLV = 2 or 4: every column is exactly that many words (at most 64 or 128 steps) and comes with one vector load: a
+// warp's 32 columns are 32 different lines, and what limits the chains in global memory is the number of such
+// scattered loads. (Every column then starts on an 8- or 16-byte boundary; the arrays themselves are 16-byte
+// aligned.) COLV = 0: columns of any length, the two words they need. The choice is made at compile time: a test of
+// S32 around every load breaks up the straight-line block in which all loads of a batch are issued, and was 1.5x slower.
+template <int COLV, typename Ptr>
+__device__ __forceinline__ uint32_t window_at(Ptr col, const WinPos p)
+{
+    uint32_t lo, hi;
+    if (COLV == 2) {
+        const uint2 q = *reinterpret_cast<const uint2*>(col);
+        lo = p.w ? q.y : q.x;
+        hi = q.y;
+    } else if (COLV == 4) {
+        const uint4 q = *reinterpret_cast<const uint4*>(col);
+        lo = p.w == 0 ? q.x : p.w == 1 ? q.y : p.w == 2 ? q.z : q.w;
+        hi = p.w == 0 ? q.y : p.w == 1 ? q.z : q.w;
+    } else {
+        lo = col[p.w];
+        hi = col[p.w2];
+    }
+    return p.first ? ((lo << 1) | (lo & 1u)) : __funnelshift_r(lo, hi, p.sh);
+}
+
 struct ChainView {               // where a chain's state lives
     uint32_t* P;                 // [U][S32] schedule, time-packed (shared or global)
     uint4* ctr;                  // [S] {hr, mi, mo, occ} (shared)
@@ -207,6 +243,26 @@ __device__ __forceinline__ int item_delta(const Windows& wn, uint32_t k, const u
     const uint32_t mi = c4.y + (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
     const uint32_t mo = c4.z + (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
     return (int)(step_cost(hr, mi, mo, c, K) - step_cost(c4.x, c4.y, c4.z, c, K));
+}
+
+// Cost of the step at window bit k after the proposal (Eq. 2-4), from its windows and the step's present counters.
+template <bool GROW>
+__device__ __forceinline__ uint32_t item_cost_after(const Windows& wn, uint32_t k, const uint4 c4, uint32_t hb, const StepC c,
+                                                    const CostK K)
+{
+    const uint32_t pu = (wn.Wu >> k) & 1u, qu = (wn.Wu >> (k - 1)) & 1u, npu = (wn.Nu >> k) & 1u, nqu = (wn.Nu >> (k - 1)) & 1u;
+    const uint32_t pv = (wn.Wv >> k) & 1u, qv = (wn.Wv >> (k - 1)) & 1u, npv = (wn.Nv >> k) & 1u, nqv = (wn.Nv >> (k - 1)) & 1u;
+    const uint32_t au = (wn.Au >> k) & 1u, av = (wn.Av >> k) & 1u;
+    const uint32_t hr = c4.x + (au & npu) - (au & pu) + (av & npv) - (av & pv);
+    const uint32_t mo = c4.z + (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
+    if (GROW) {
+        const uint32_t mu = (wn.born & 255u) == k ? 0u : 1u, mw = ((wn.born >> 8) & 255u) == k ? 0u : 1u;
+        const uint32_t mi = c4.y + mu * ((npu & ~nqu) - (pu & ~qu)) + mw * ((npv & ~nqv) - (pv & ~qv));
+        const uint32_t hn = hb + (1u - mu) * (npu - pu) + (1u - mw) * (npv - pv);
+        return step_cost_g(hr, mi, mo, hn, c, K);
+    }
+    const uint32_t mi = c4.y + (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
+    return step_cost(hr, mi, mo, c, K);
 }
 
 __device__ __forceinline__ bool metropolis(int delta, uint32_t w, const uint32_t* __restrict__ trow, uint32_t shift)
@@ -864,7 +920,7 @@ constexpr uint32_t kCowSlots4 = kCowBits / 128;
 
 // Where a chain of the wide kernel keeps its state. CT: the four per-step cardinalities as 16-bit fields when the
 // schedule lives in shared memory (then units < 2^16), as 32-bit fields otherwise. COW: see above.
-template <typename CT, bool COW>
+template <typename CT, bool COW, int COLV>
 struct WideView {
     const uint32_t* p0;          // COW: [U][S32] the initial schedule
     uint32_t* have;              // COW: [kCowBits / 32] buckets present in P (shared)
@@ -893,6 +949,7 @@ struct WideView {
     CT* ctr;                     // [S] {hr, mi, mo, occ} (shared)
     uint32_t* full;              // [S32] bit t set iff occ[t] == cap (shared)
     uint32_t* hb;                // growing cache: [S] units written to HBM at birth (shared)
+    uint32_t* fnow;              // [S] the present cost of every step, Eq. 2 (shared)
     uint4* win;                  // [kWide][2] by proposal: {pk, u, v, -} until it is evaluated, then its windows
     int* acc;                    // [kWide] by proposal: its cost change being summed
     uint8_t* nt;                 // [kWide] the proposals that need a cost evaluation, compacted
@@ -912,14 +969,15 @@ constexpr uint32_t kWideScalars4 = sizeof(WideScalars) / 16;
 // shared-memory words (as uint4 slots) of one chain of the wide kernel besides its schedule
 __host__ __device__ inline uint32_t wide_fixed4(uint32_t S, uint32_t S32, bool grow, bool shared)
 {
-    return (shared ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (shared ? 0u : kCowSlots4) + kWideScalars4 +
+    return (shared ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (S + 3) / 4 +
+           (shared ? 0u : kCowSlots4) + kWideScalars4 +
            2 * kWide + kWide / 4 + kWide / 16 + kWideQueueSlots4;
 }
 
 // N queue items per lane, items base + 32 r + lane: the cost change of one step of one proposal each, added to the
 // proposal's sum.
-template <bool GROW, int N, typename CT, bool COW>
-__device__ __forceinline__ void wide_items(const WideView<CT, COW> cv, const StepC* __restrict__ stepc, const CostK K, uint32_t S,
+template <bool GROW, int N, typename CT, bool COW, int COLV>
+__device__ __forceinline__ void wide_items(const WideView<CT, COW, COLV> cv, const StepC* __restrict__ stepc, const CostK K, uint32_t S,
                                            uint32_t base, uint32_t count, uint32_t lane)
 {
     int d[N];
@@ -938,7 +996,7 @@ __device__ __forceinline__ void wide_items(const WideView<CT, COW> cv, const Ste
         wn.born = w1.w;
         const uint32_t t = min(wn.s0 + k - 1, S - 1);
         const StepC sc = stepc[t];
-        d[r] = item_delta<GROW>(wn, k, ctr_load<CT>(cv.ctr, t), GROW ? cv.hb[t] : 0u, sc, K);
+        d[r] = (int)(item_cost_after<GROW>(wn, k, ctr_load<CT>(cv.ctr, t), GROW ? cv.hb[t] : 0u, sc, K) - cv.fnow[t]);
     }
 #pragma unroll
     for (int r = 0; r < N; ++r)
@@ -956,7 +1014,7 @@ struct WideMoves {
 // Second half of evaluating a proposal that is known to change bits and to be feasible: given its placement windows
 // (Wu; wv = the window of v for a swap), the access windows, the windows after the move and the set of window bits
 // (steps) whose cardinalities, hence cost, change. Same conventions as lane_windows.
-template <bool GROW>
+template <bool GROW, int COLV>
 __device__ __forceinline__ uint32_t changed_steps(uint32_t Wu, uint32_t wv, const uint32_t* __restrict__ Acol,
                                                   const uint32_t* __restrict__ birth, uint32_t S, uint32_t S32,
                                                   uint32_t pk, uint32_t u, uint32_t v, Windows& wn)
@@ -967,8 +1025,9 @@ __device__ __forceinline__ uint32_t changed_steps(uint32_t Wu, uint32_t wv, cons
     const uint32_t nl = min(s0 + len, S - 1) - s0 + 1;            // affected steps: the run and the step after it
     const uint32_t M = ((1u << run) - 1u) << 1;
     const uint32_t Sb = ((1u << nl) - 1u) << 1;
-    const uint32_t Au = window(Acol + (size_t)u * S32, S32, s0);
-    const uint32_t av = window(Acol + (size_t)(swap ? v : u) * S32, S32, s0);   // a flip reads unit u twice
+    const WinPos wp = window_pos(S32, s0);
+    const uint32_t Au = window_at<COLV>(Acol + (size_t)u * S32, wp);
+    const uint32_t av = window_at<COLV>(Acol + (size_t)(swap ? v : u) * S32, wp);   // a flip reads unit u twice
     const uint32_t Av = swap ? av : 0u, Wv = swap ? wv : 0u;
     uint32_t Bu = 0u, Bv = 0u, live = 0xFFFFFFFFu;
     if (GROW) {
@@ -1000,8 +1059,8 @@ __device__ __forceinline__ uint32_t changed_steps(uint32_t Wu, uint32_t wv, cons
 // ALL: nearly every row is named (a fresh batch): the window loads of all rows are issued before any is used, named
 // or not (every row holds a drawn proposal, so every address is good). Otherwise rows without a named proposal are
 // skipped.
-template <bool GROW, bool ALL, typename CT, bool COW>
-__device__ __forceinline__ void wide_classify(const WideView<CT, COW> cv, const uint32_t* __restrict__ birth, uint32_t S,
+template <bool GROW, bool ALL, typename CT, bool COW, int COLV>
+__device__ __forceinline__ void wide_classify(const WideView<CT, COW, COLV> cv, const uint32_t* __restrict__ birth, uint32_t S,
                                               uint32_t S32, uint32_t need, uint32_t lane, WideMoves& mv, uint32_t& listed,
                                               uint32_t& mine)
 {
@@ -1014,14 +1073,18 @@ __device__ __forceinline__ void wide_classify(const WideView<CT, COW> cv, const 
         Wu[h] = Wv[h] = Fw[h] = 0u; Lv[h] = 0xFFFFFFFFu;
         if (skip[h]) continue;                                    // warp-uniform
         const uint32_t pk = mv.pk[h], s0 = pk >> 8;
-        const uint32_t ve = (pk & 1u) ? mv.v[h] : mv.u[h];        // a flip reads unit u twice and ignores the copy
-        Wu[h] = window(cv.col(mv.u[h]), S32, s0);
-        Wv[h] = window(cv.col(ve), S32, s0);
-        Fw[h] = window(cv.full, S32, s0);
+        const bool swap = pk & 1u;
+        const WinPos wp = window_pos(S32, s0);
+        Wu[h] = window_at<COLV>(cv.col(mv.u[h]), wp);
+        // the second window: the other unit's placement for a swap, the full-step bitmap for a flip
+        const uint32_t* second = swap ? cv.col(mv.v[h]) : cv.full;
+        const uint32_t w2 = window_at<COLV>(second, wp);
+        Wv[h] = swap ? w2 : Wu[h];
+        Fw[h] = w2;
         if (GROW) {
             uint32_t La, Lb, Bu, Bv;
             alive_born(__ldg(birth + mv.u[h]), s0, La, Bu);
-            alive_born(__ldg(birth + ve), s0, Lb, Bv);
+            alive_born(__ldg(birth + (swap ? mv.v[h] : mv.u[h])), s0, Lb, Bv);
             Lv[h] = La & Lb;
         }
     }
@@ -1060,8 +1123,8 @@ __device__ __forceinline__ void wide_classify(const WideView<CT, COW> cv, const 
 
 // Evaluation of the proposals named by `need` (per lane: bit h = its row h) against the current state.
 // fresh: a new batch, nearly every row named (see wide_classify).
-template <bool GROW, typename CT, bool COW>
-__device__ __forceinline__ void wide_evaluate(const WideView<CT, COW> cv, const uint32_t* __restrict__ Acol,
+template <bool GROW, typename CT, bool COW, int COLV>
+__device__ __forceinline__ void wide_evaluate(const WideView<CT, COW, COLV> cv, const uint32_t* __restrict__ Acol,
                                               const uint32_t* __restrict__ birth, const StepC* __restrict__ stepc,
                                               const CostK K, uint32_t S, uint32_t S32, const uint32_t* __restrict__ trow,
                                               uint32_t shift, uint32_t need, bool fresh, uint32_t lane, WideMoves& mv)
@@ -1083,7 +1146,7 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW> cv, const 
         const uint4 who = cv.win[id * 2];
         const uint32_t wv = cv.win[id * 2 + 1].x;
         Windows wn;
-        const uint32_t tm = changed_steps<GROW>(who.w, wv, Acol, birth, S, S32, who.x, who.y, who.z, wn);
+        const uint32_t tm = changed_steps<GROW, COLV>(who.w, wv, Acol, birth, S, S32, who.x, who.y, who.z, wn);
         __syncwarp();                                             // every lane has read its proposal
         const uint32_t todo = live ? tm : 0u;
         if (live) {
@@ -1099,11 +1162,22 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW> cv, const 
             total += __popc(has) << bit;
         }
         if (total) {
+            if (COW) {
+                // many chains per SM, issue slots scarce: one set bit per lane and trip
+                for (uint32_t td = todo; __any_sync(0xFFFFFFFFu, td != 0u);) {
+                    if (td) {
+                        cv.queue[pos++] = (uint16_t)((id << 5) | (__ffs(td) - 1u));
+                        td &= td - 1u;
+                    }
+                }
+            } else {
+                // few chains per SM, latency scarce: all 31 positions tried, no lane waits on a serial bit scan
 #pragma unroll
-            for (uint32_t k = 1; k < 32; ++k) {
-                const uint32_t bit = (todo >> k) & 1u;
-                if (bit) cv.queue[pos] = (uint16_t)((id << 5) | k);
-                pos += bit;
+                for (uint32_t k = 1; k < 32; ++k) {
+                    const uint32_t bit = (todo >> k) & 1u;
+                    if (bit) cv.queue[pos] = (uint16_t)((id << 5) | k);
+                    pos += bit;
+                }
             }
             __syncwarp();
             for (uint32_t base = 0; base < total; base += 64) {
@@ -1126,8 +1200,9 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW> cv, const 
 
 // Apply the proposal whose windows are in slot `id` (pk, u, v given): all lanes take part, lane j updates the
 // counters of window bit j, lanes 0 and 1 rewrite the words of the schedule and of the full-step bitmap.
-template <bool GROW, typename CT, bool COW>
-__device__ __forceinline__ void wide_apply(const WideView<CT, COW> cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
+template <bool GROW, typename CT, bool COW, int COLV>
+__device__ __forceinline__ void wide_apply(const WideView<CT, COW, COLV> cv, const StepC* __restrict__ stepc, const CostK K,
+                                           uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
                                            uint32_t id, uint32_t pk, uint32_t u, uint32_t v)
 {
     const uint4 w0 = cv.win[id * 2], w1 = cv.win[id * 2 + 1];
@@ -1142,18 +1217,23 @@ __device__ __forceinline__ void wide_apply(const WideView<CT, COW> cv, uint32_t 
     const uint32_t pv = (Wv >> j) & 1u, qv = (Wv >> (j - 1)) & 1u, npv = (Nv >> j) & 1u, nqv = (Nv >> (j - 1)) & 1u;
     const uint32_t au = (Au >> j) & 1u, av = (Av >> j) & 1u;
     uint4 c = ctr_load<CT>(cv.ctr, t);
+    uint32_t hbn = 0u;
     c.x += (au & npu) - (au & pu) + (av & npv) - (av & pv);
     if (GROW) {
         const uint32_t mu = (w1.w & 255u) == j ? 0u : 1u, mw = ((w1.w >> 8) & 255u) == j ? 0u : 1u;
         c.y += mu * ((npu & ~nqu) - (pu & ~qu)) + mw * ((npv & ~nqv) - (pv & ~qv));
         const uint32_t dh = (1u - mu) * (npu - pu) + (1u - mw) * (npv - pv);
-        if (valid && dh) cv.hb[t] += dh;
+        hbn = cv.hb[t] + dh;
+        if (valid && dh) cv.hb[t] = hbn;
     } else {
         c.y += (npu & ~nqu) - (pu & ~qu) + (npv & ~nqv) - (pv & ~qv);
     }
     c.z += (~npu & nqu & 1u) - (~pu & qu & 1u) + (~npv & nqv & 1u) - (~pv & qv & 1u);
     c.w += npu - pu + npv - pv;
-    if (valid) ctr_store<CT>(cv.ctr, t, c);
+    if (valid) {
+        ctr_store<CT>(cv.ctr, t, c);
+        cv.fnow[t] = GROW ? step_cost_g(c.x, c.y, c.z, hbn, stepc[t], K) : step_cost(c.x, c.y, c.z, stepc[t], K);
+    }
     uint32_t F = __ballot_sync(0xFFFFFFFFu, valid && c.w == cap);   // bit j <-> window bit j
     uint32_t V = __ballot_sync(0xFFFFFFFFu, valid);
     cv.own(u, lane);
@@ -1197,11 +1277,13 @@ __device__ __forceinline__ void copy_merged(uint32_t* __restrict__ dst, const ui
 // PSMEM: the schedule lives in shared memory (16-bit counters); otherwise the chain's slice of global scratch is a
 // copy-on-write overlay of the initial schedule (see kCowBits).
 // ASMEM (only with PSMEM): access bitmap and step constants staged in shared memory once per CTA.
-template <bool PSMEM, bool GROW, bool ASMEM>
+// COLV (only without PSMEM): 2 or 4 when every column has exactly that many words, else 0 (see window_at).
+template <bool PSMEM, bool GROW, bool ASMEM, int COLV>
 __global__ void __launch_bounds__(PSMEM ? 256 : kWideGlobalThreads, 1)
 wide_chain_kernel(const ChainParams prm)
 {
     static_assert(PSMEM || !ASMEM, "shared access bitmap only beside shared schedules");
+    static_assert(!PSMEM || COLV == 0, "vector columns only for schedules in global scratch");
     using CT = typename std::conditional<PSMEM, ushort4, uint4>::type;
     constexpr bool COW = !PSMEM;
     extern __shared__ uint4 smem4[];
@@ -1217,13 +1299,15 @@ wide_chain_kernel(const ChainParams prm)
     constexpr uint32_t o4 = COW ? kCowSlots4 : 0u;
     const uint32_t fixed4 = wide_fixed4(S, S32, GROW, PSMEM);
     uint4* const mine4 = smem4 + (size_t)cic * fixed4;
-    WideView<CT, COW> cv;
+    WideView<CT, COW, COLV> cv;
     cv.ctr = reinterpret_cast<CT*>(mine4);
     cv.full = reinterpret_cast<uint32_t*>(mine4 + c4);
     cv.hb = reinterpret_cast<uint32_t*>(mine4 + c4 + f4);
-    cv.have = reinterpret_cast<uint32_t*>(mine4 + c4 + f4 + h4);
-    WideScalars* const sc = reinterpret_cast<WideScalars*>(mine4 + c4 + f4 + h4 + o4);
-    cv.win = mine4 + c4 + f4 + h4 + o4 + kWideScalars4;
+    const uint32_t n4 = (S + 3) / 4;                              // uint4 slots of the present step costs
+    cv.fnow = reinterpret_cast<uint32_t*>(mine4 + c4 + f4 + h4);
+    cv.have = reinterpret_cast<uint32_t*>(mine4 + c4 + f4 + h4 + n4);
+    WideScalars* const sc = reinterpret_cast<WideScalars*>(mine4 + c4 + f4 + h4 + n4 + o4);
+    cv.win = mine4 + c4 + f4 + h4 + n4 + o4 + kWideScalars4;
     cv.acc = reinterpret_cast<int*>(cv.win + 2 * kWide);
     cv.nt = reinterpret_cast<uint8_t*>(cv.win + 2 * kWide + kWide / 4);
     cv.queue = reinterpret_cast<uint16_t*>(cv.win + 2 * kWide + kWide / 4 + kWide / 16);
@@ -1246,10 +1330,15 @@ wide_chain_kernel(const ChainParams prm)
         stepc = c_s;
     }
     if (active) {
-        for (uint32_t i = lane; i < S; i += 32) ctr_store<CT>(cv.ctr, i, __ldg(prm.counters0 + i));
+        for (uint32_t i = lane; i < S; i += 32) {
+            const uint4 c0 = __ldg(prm.counters0 + i);
+            const uint32_t hb0 = GROW ? __ldg(prm.hb0 + i) : 0u;
+            ctr_store<CT>(cv.ctr, i, c0);
+            if (GROW) cv.hb[i] = hb0;
+            cv.fnow[i] = GROW ? step_cost_g(c0.x, c0.y, c0.z, hb0, __ldg(prm.stepc + i), prm.K)
+                              : step_cost(c0.x, c0.y, c0.z, __ldg(prm.stepc + i), prm.K);
+        }
         for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
-        if (GROW)
-            for (uint32_t i = lane; i < S; i += 32) cv.hb[i] = __ldg(prm.hb0 + i);
         if (lane == 0) {
             sc->cur = sc->best = sc->best_at_boundary = prm.init_ticks;
             sc->best_move = ~0ull; sc->n_chg = 0; sc->hash = 0; sc->ulen = 0u; sc->snap_dirty = 0u;
@@ -1344,7 +1433,7 @@ wide_chain_kernel(const ChainParams prm)
                             const uint64_t after = (uint64_t)((int64_t)sc->cur + delta);
                             const bool leaving = snap && sc->snap_dirty && after >= sc->best;
                             if (leaving) copy_words(snap, cv.P, pwords, lane);   // leaving the best state: save it first
-                            wide_apply<GROW>(cv, S, S32, prm.cap, lane, h * 32 + bb, pk, bu, bv);
+                            wide_apply<GROW>(cv, stepc, prm.K, S, S32, prm.cap, lane, h * 32 + bb, pk, bu, bv);
                             if (lane == 0) {
                                 const uint64_t mb = m + 32u * h + bb;
                                 if (leaving) sc->snap_dirty = 0u;
@@ -1557,6 +1646,7 @@ struct Ctx {
     size_t smem_shared;      // shared memory of the CTA beside its chains (access bitmap and step constants)
     bool asmem;              // the access bitmap and the step constants are staged in shared memory
     bool wide;               // the wide kernel (one warp per chain, four proposals per lane)
+    uint32_t S32;            // words per time-packed column
     bool stage_stepc;        // wide kernel: the step constants are staged in shared memory without the access bitmap
     std::vector<double> temps;
     uint64_t init_ticks, calib_mean;
@@ -1590,16 +1680,20 @@ ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W, bool
     return asmem ? chain_kernel_pick<true, true, false>(grow, W) : chain_kernel_pick<true, false, false>(grow, W);
 }
 
-ChainKernel wide_kernel_for(bool psmem, bool asmem, bool grow)
+ChainKernel wide_kernel_for(bool psmem, bool asmem, bool grow, uint32_t S32)
 {
-    if (!psmem) return grow ? wide_chain_kernel<false, true, false> : wide_chain_kernel<false, false, false>;
-    if (asmem) return grow ? wide_chain_kernel<true, true, true> : wide_chain_kernel<true, false, true>;
-    return grow ? wide_chain_kernel<true, true, false> : wide_chain_kernel<true, false, false>;
+    if (!psmem) {
+        if (S32 == 2) return grow ? wide_chain_kernel<false, true, false, 2> : wide_chain_kernel<false, false, false, 2>;
+        if (S32 == 4) return grow ? wide_chain_kernel<false, true, false, 4> : wide_chain_kernel<false, false, false, 4>;
+        return grow ? wide_chain_kernel<false, true, false, 0> : wide_chain_kernel<false, false, false, 0>;
+    }
+    if (asmem) return grow ? wide_chain_kernel<true, true, true, 0> : wide_chain_kernel<true, false, true, 0>;
+    return grow ? wide_chain_kernel<true, true, false, 0> : wide_chain_kernel<true, false, false, 0>;
 }
 
 ChainKernel kernel_of(const Ctx& c, bool psmem, bool asmem, uint32_t W, bool touch)
 {
-    return c.wide ? wide_kernel_for(psmem, asmem, c.grow) : chain_kernel_for(psmem, asmem, c.grow, W, touch);
+    return c.wide ? wide_kernel_for(psmem, asmem, c.grow, c.S32) : chain_kernel_for(psmem, asmem, c.grow, W, touch);
 }
 
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
@@ -1645,7 +1739,12 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     // per chain: counters, full-step bitmap and, per warp, the batch's windows, accumulators and work queue
     c.grow = p->dL != nullptr;
     const kvp_test_hooks hooks = g_hooks;
-    c.wide = hooks.warps_per_chain == 0;             // the narrow kernels (one proposal per lane) only on request
+    c.S32 = p->S32;
+    // Which kernel. Many chains per SM (more than 8, the jobs that fill the registers of an SM with one warp per
+    // chain): the wide kernel, which needs half the instructions per proposal. Few chains per SM: the narrow kernel
+    // with two warps per chain, which hides the latency of a chain's serial parts behind its second warp.
+    // kvp_set_test_hooks can force either (warps_per_chain 1 or 2: narrow; 3: wide).
+    c.wide = hooks.warps_per_chain == 3 || (hooks.warps_per_chain == 0 && (a->chains + sms - 1) / sms > 8);
     // `shared`: the schedule is in shared memory (the wide kernel then keeps 16-bit counters)
     auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false, bool shared = true) {
         if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared) * 16;

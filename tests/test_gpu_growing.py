@@ -17,10 +17,11 @@ def kvp():
     return kvp
 
 
-@pytest.fixture(params=[0, 1, 2], ids=["wide", "narrow1", "narrow2"])
+@pytest.fixture(params=[3, 1, 2], ids=["wide", "narrow1", "narrow2"])
 def warps_per_chain(request, hooks):
-    """The wide chain kernel (the default: one warp per chain, four proposals per lane) and both forms of the narrow
-    one (one proposal per lane; one warp per chain, or two warps that take a chain's batches in turn)."""
+    """The wide chain kernel (one warp per chain, four proposals per lane; the library's choice for jobs of many
+    chains) and both forms of the narrow one (one proposal per lane; one warp per chain, or two warps that take a
+    chain's batches in turn; the choice for few chains)."""
     hooks(warps_per_chain=request.param)
     return request.param
 

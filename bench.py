@@ -35,7 +35,20 @@ UNIT = "move-evals/s"
 # ~105, window extraction and word-parallel bit logic ~100, work-queue scan and push ~100, about 35 (lane, step)
 # cost evaluations of ~70 thread instructions each in two warp rounds ~150, Metropolis and in-order commit ~50).
 ISSUE_PEAK_GWIPS = 148 * 4 * 1.965
-ALG_WARP_INSTR_PER_MOVE = 16.0
+ALG_WARP_INSTR_PER_MOVE = 16.0          # the narrow chain kernel: every proposal is evaluated in full
+# The wide chain kernel settles most proposals by their placement bits alone, so its algorithmic work depends on the
+# workload; the kernel counts what its evaluations amounted to (kvp_anneal_stats) and the numerator is, in warp
+# instructions (thread instructions / 32 of the formulation, counted by hand from the steps it needs):
+#   per move          2.06 : Philox4x32-10 (10 rounds of 2 wide multiplies and 2 three-input XORs) 40, counter 3,
+#                            decoding of swap / run length / first step / two units 18, its share of the commit vote 2
+#   per evaluation    1.65 : unpacking 4, run mask 5, window position 5, two placement columns (overlay lookup, address,
+#                            load, funnel shift) 22, toggled bits, Eq. 5 test, verdict bits 13, listing 4
+#   per listed one    1.75 : slot 2, two access columns 10, windows after the move 6, the steps whose cardinalities
+#                            change 18, window store 2, queue offsets 12, sum and Metropolis test 6
+#   per (proposal, step) item 1.45 : queue 3, windows, counters, constants, present cost 5 loads, bit extraction 10,
+#                            new cardinalities 12, Eq. 2-4 once 13, difference and accumulation 3
+# evaluations = moves + proposals evaluated again after an applied move.
+ALG_WIDE = {"move": 2.06, "evaluation": 1.65, "listed": 1.75, "item": 1.45}
 PEAK_SOURCE_ALU = "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"
 FLUSH_NOTE = "flushed with a 256 MB write between timed iterations"
 
@@ -436,10 +449,17 @@ def time_to_bound(prob, cfg):
             break
     half = res["budgets"][str(cfg["moves"] // 2)]["bound_ticks"]
     res["converged"] = bool((half - full_ticks) * 1000 <= full_ticks)
-    res["note"] = ("the bound still improves with the budget: a throughput measurement, not a converged bound"
-                   if not res["converged"] else
-                   "doubling the budget to the full one moves the bound by less than 0.1%")
-    res["improvement_over_initial_permille"] = round((init - full_ticks) * 1000.0 / init, 3)
+    gain = (init - full_ticks) * 1000.0 / init
+    res["improvement_over_initial_permille"] = round(gain, 3)
+    if gain < 1.0:
+        res["converged"] = False
+        res["note"] = ("the whole budget moves the bound by less than 0.1% from the initial placement, so every budget meets "
+                       "the 0.1% criterion trivially and the bound still falls with the budget: budget-limited, a "
+                       "throughput measurement, not a converged bound")
+    elif not res["converged"]:
+        res["note"] = "the bound still improves with the budget: a throughput measurement, not a converged bound"
+    else:
+        res["note"] = "doubling the budget to the full one moves the bound by less than 0.1%"
     return res
 
 
@@ -449,7 +469,7 @@ def time_to_bound(prob, cfg):
 class PathBench:
     """One named configuration: inputs resident on the device and in pinned host memory, and the step itself."""
 
-    def __init__(self, name, rank, world, p0=None):
+    def __init__(self, name, rank, world, p0=None, chains=None, moves=None):
         import numpy as np
         import torch
         from paper_2508_13231_b200 import kvp, sharding, workloads as wl
@@ -458,7 +478,7 @@ class PathBench:
         self.cfg = cfg = wl.CONFIGS[name]
         tp = wl.trace_params(name, seed=0)
         self.U, self.S, self.W32 = wl.units(cfg), cfg["steps"], wl.words_per_row(cfg)
-        self.chains, self.moves = cfg["chains"], cfg["moves"]
+        self.chains, self.moves = chains or cfg["chains"], moves or cfg["moves"]
         self.p0 = cfg["p0"] if p0 is None else p0
         self.n_eval = 8 if self.U * self.S <= (1 << 24) else 2
         if self.U <= 65536:
@@ -530,14 +550,28 @@ class PathBench:
         """Issue-slot roofline of the chain kernel from the device time the library measured around its launches."""
         st = out["stats"]
         per_launch_ms = chain_ms / max(1, chain_launches)
-        moves_per_launch = float(st.moves_total) * n_steps / max(1, chain_launches)
-        achieved = ALG_WARP_INSTR_PER_MOVE * moves_per_launch / (per_launch_ms * 1e-3) / 1e9
+        moves = float(st.moves_total)                        # of the last step; every step does the same number
+        if st.wide_kernel:
+            alg = (ALG_WIDE["move"] * moves + ALG_WIDE["evaluation"] * (moves + st.work_again) +
+                   ALG_WIDE["listed"] * st.work_listed + ALG_WIDE["item"] * st.work_items) / moves
+            form = {"kernel_form": "wide (one warp per chain, four proposals per lane, placement bits first)",
+                    "work_per_move": {"evaluated_again": st.work_again / moves, "listed": st.work_listed / moves,
+                                      "items": st.work_items / moves},
+                    "frac_against_16_per_move": None}
+        else:
+            alg = ALG_WARP_INSTR_PER_MOVE
+            form = {"kernel_form": "narrow (one proposal per lane, every proposal evaluated in full)"}
+        moves_per_launch = moves * n_steps / max(1, chain_launches)
+        achieved = alg * moves_per_launch / (per_launch_ms * 1e-3) / 1e9
+        if st.wide_kernel:   # the same time against the work of the full-evaluation formulation, for comparison only
+            form["frac_against_16_per_move"] = (ALG_WARP_INSTR_PER_MOVE * moves_per_launch / (per_launch_ms * 1e-3) / 1e9 /
+                                                ISSUE_PEAK_GWIPS)
         return {"bound": "alu", "kernel": "chain kernel (%s)" % ("schedules in shared memory" if self.U * self.S <= (1 << 18)
                                                                   else "schedules in global memory"),
                 "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
                 "traffic": None, "ms_per_launch": per_launch_ms, "launches_per_step": chain_launches / max(1, n_steps),
-                "chains_per_launch": int(st.resident_chains), "algorithmic_warp_instr_per_move": ALG_WARP_INSTR_PER_MOVE,
-                "peak_source": PEAK_SOURCE_ALU}
+                "chains_per_launch": int(st.resident_chains), "algorithmic_warp_instr_per_move": alg,
+                "peak_source": PEAK_SOURCE_ALU, **form}
 
 
 def side_record(name, steps, p0=None):
@@ -572,6 +606,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="kvp", choices=["kvp", "reference"])
     ap.add_argument("--workload", default=WORKLOAD, help="named configuration of the path benchmark (default: the largest)")
+    ap.add_argument("--chains", type=int, default=0, help="override the configuration's chain count (small cases for profiling)")
+    ap.add_argument("--moves", type=int, default=0, help="override the configuration's moves per chain")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="leave out the side records (single_head, kernels, time to bound)")
     ap.add_argument("--kernel", default="path", choices=["path", "cost", "trace", "growing"],
@@ -606,7 +642,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     d = dist if world > 1 else None
     warmup = max(3, args.warmup)
-    b = PathBench(args.workload, rank, world)
+    b = PathBench(args.workload, rank, world, chains=args.chains or None, moves=args.moves or None)
     b.warm(warmup, d)
 
     def barrier():

@@ -244,6 +244,12 @@ typedef struct {
     kvp_chain_result* per_chain; /* (host) [chains] or NULL                                        */
     uint32_t chain_launches;    /* launches of the chain kernel (waves of resident chains)         */
     uint32_t resident_chains;   /* chains per wave                                                 */
+    uint32_t wide_kernel;       /* 1: the wide chain kernel ran (many chains), 0: the narrow one   */
+    uint32_t reserved;
+    /* What the evaluations of the wide kernel amounted to, summed over the chains (0 for the narrow kernel): */
+    uint64_t work_again;        /* proposals evaluated a second time after a move was applied in their batch   */
+    uint64_t work_listed;       /* evaluations that needed more than the placement bits (a cost evaluation)    */
+    uint64_t work_items;        /* (proposal, step) pairs whose step cost (Eq. 2-4) was evaluated              */
 } kvp_anneal_stats;
 
 /*

@@ -61,6 +61,7 @@ struct ChainParams {
                                  // units a slot's slice holds when its chain ends (the rest is the initial schedule)
     uint32_t cow_shift;          // a bucket is 2^cow_shift consecutive units
     uint32_t stage_stepc;        // wide kernel without a staged access bitmap: the step constants alone are staged
+    unsigned long long* work;    // wide kernel: [3] sums over the chains of {n_again, n_listed, n_items}
 };
 
 // Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
@@ -963,6 +964,9 @@ struct WideScalars {
     uint32_t ulen;               // moves applied since the best state
     uint32_t snap_dirty;         // the best state is the current one and not saved yet
     uint32_t pad[2];
+    // what the chain's evaluations amounted to (kvp_anneal_stats): proposals evaluated again after an applied move,
+    // proposals that needed a cost evaluation, (proposal, step) items
+    uint64_t n_again, n_listed, n_items, pad2;
 };
 constexpr uint32_t kWideScalars4 = sizeof(WideScalars) / 16;
 
@@ -1127,7 +1131,8 @@ template <bool GROW, typename CT, bool COW, int COLV>
 __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW, COLV> cv, const uint32_t* __restrict__ Acol,
                                               const uint32_t* __restrict__ birth, const StepC* __restrict__ stepc,
                                               const CostK K, uint32_t S, uint32_t S32, const uint32_t* __restrict__ trow,
-                                              uint32_t shift, uint32_t need, bool fresh, uint32_t lane, WideMoves& mv)
+                                              uint32_t shift, uint32_t need, bool fresh, uint32_t lane, WideMoves& mv,
+                                              WideScalars* sc)
 {
     const uint32_t below = (1u << lane) - 1u;
     // 1. placement bits only; the proposals that need more are listed
@@ -1136,6 +1141,7 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW, COLV> cv, 
     if (fresh) wide_classify<GROW, true>(cv, birth, S, S32, need, lane, mv, listed, mine);
     else wide_classify<GROW, false>(cv, birth, S, S32, need, lane, mv, listed, mine);
     if (!listed) return;                                          // warp-uniform
+    if (lane == 0) sc->n_listed += listed;
     __syncwarp();
     // 2. the listed proposals, 32 at a time, one per lane: access windows, the steps whose cost changes, and those
     //    (proposal, step) items through the shared queue
@@ -1162,6 +1168,7 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW, COLV> cv, 
             total += __popc(has) << bit;
         }
         if (total) {
+            if (lane == 0) sc->n_items += total;
             if (COW) {
                 // many chains per SM, issue slots scarce: one set bit per lane and trip
                 for (uint32_t td = todo; __any_sync(0xFFFFFFFFu, td != 0u);) {
@@ -1342,6 +1349,7 @@ wide_chain_kernel(const ChainParams prm)
         if (lane == 0) {
             sc->cur = sc->best = sc->best_at_boundary = prm.init_ticks;
             sc->best_move = ~0ull; sc->n_chg = 0; sc->hash = 0; sc->ulen = 0u; sc->snap_dirty = 0u;
+            sc->n_again = sc->n_listed = sc->n_items = 0;
         }
         if (COW) {
             for (uint32_t i = lane; i < kCowBits / 32; i += 32) cv.have[i] = 0u;   // the slice holds nothing yet
@@ -1393,7 +1401,7 @@ wide_chain_kernel(const ChainParams prm)
             bool first_pass = true;
             // Evaluate what is named, then commit in move order as far as the evaluations are still good.
             for (;;) {
-                wide_evaluate<GROW>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, first_pass, lane, mv);
+                wide_evaluate<GROW>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, need, first_pass, lane, mv, sc);
                 first_pass = false;
                 // Nearly always nothing in the batch changes the schedule: every lane counts its own proposals.
                 if (!__any_sync(0xFFFFFFFFu, (mv.acc & mv.chg & ~mv.inf & pend) != 0u)) {
@@ -1468,6 +1476,8 @@ wide_chain_kernel(const ChainParams prm)
                 if (!stopped) break;
                 need = stale & pend;
                 stale = 0u;
+                const uint32_t again = __reduce_add_sync(0xFFFFFFFFu, __popc(need));
+                if (lane == 0) sc->n_again += again;
             }
         }
         lvl_start += lvl_len;
@@ -1488,6 +1498,11 @@ wide_chain_kernel(const ChainParams prm)
         res.best_ticks = sc->best; res.best_move = sc->best_move; res.final_ticks = sc->cur; res.moves_done = m_end;
         res.n_accepted = n_acc; res.n_changed = sc->n_chg; res.n_infeasible = n_inf; res.traj_hash = sc->hash;
         prm.results[chain - prm.result_base] = res;
+        if (prm.work) {
+            atomicAdd(prm.work, (unsigned long long)sc->n_again);
+            atomicAdd(prm.work + 1, (unsigned long long)sc->n_listed);
+            atomicAdd(prm.work + 2, (unsigned long long)sc->n_items);
+        }
     }
     if (prm.dump && slot == 0) {
         __syncwarp();
@@ -1917,6 +1932,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     prm.table = c.table; prm.shifts = c.shifts; prm.ws = c.slots; prm.K = p->K; prm.full0 = c.full0;
     prm.birth = p->d_birth; prm.hb0 = c.hb0;
     prm.err = reinterpret_cast<uint32_t*>(c.small + 16);
+    prm.work = nullptr;                                   // set by kvp_anneal for the chains of the search proper
     // test hook (tests of the bounded wait only): one hand-over per chain is withheld, the waiting warp gives up
     // after its poll limit (about a second) and the call returns KVP_ERR_TIMEOUT
     prm.drop_first_turn = hooks.drop_turn ? 1u : 0u;
@@ -2010,6 +2026,9 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     memset(&red, 0, sizeof red);
     uint32_t dumped_chain = 0xFFFFFFFFu;                  // call-local index of the chain whose best state is in dumpcol
     uint32_t waves = 0;
+    unsigned long long* work_dev = reinterpret_cast<unsigned long long*>(c.small + 24);
+    KVP_CUDA(cudaMemsetAsync(work_dev, 0, 24, st));
+    c.prm.work = c.wide ? work_dev : nullptr;
     for (uint32_t first = 0; first < a->chains; first += c.resident, ++waves) {
         const uint32_t count = a->chains - first < c.resident ? a->chains - first : c.resident;
         if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr, c.snap,
@@ -2043,6 +2062,9 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
         }
     }
     KVP_CUDA(cudaEventRecord(ev[2], st));
+    c.prm.work = nullptr;                                 // a replay of the winner is not part of the count
+    unsigned long long work[3] = {0, 0, 0};
+    KVP_CUDA(cudaMemcpyAsync(work, work_dev, sizeof work, cudaMemcpyDeviceToHost, st));
 
     // cross-chain reduction, then the winner's schedule (its own snapshot, its walked-back state, or a replay) and a
     // re-score
@@ -2094,6 +2116,8 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
         cudaEventElapsedTime(&stats->ms_finish, ev[2], ev[3]);
         stats->kernel_launches = c.launches;
         stats->chain_launches = waves; stats->resident_chains = c.resident;
+        stats->wide_kernel = c.wide ? 1u : 0u;
+        stats->work_again = work[0]; stats->work_listed = work[1]; stats->work_items = work[2];
     }
     return ok ? KVP_OK : KVP_ERR_INTERNAL;
 }

@@ -73,6 +73,8 @@ class AnnealStats(C.Structure):
         ("winner_hits", C.c_uint64), ("winner_accessed", C.c_uint64),
         ("ms_init", C.c_float), ("ms_chains", C.c_float), ("ms_finish", C.c_float), ("kernel_launches", C.c_uint32),
         ("per_chain", C.POINTER(ChainResult)), ("chain_launches", C.c_uint32), ("resident_chains", C.c_uint32),
+        ("wide_kernel", C.c_uint32), ("reserved", C.c_uint32),
+        ("work_again", C.c_uint64), ("work_listed", C.c_uint64), ("work_items", C.c_uint64),
     ]
 
 

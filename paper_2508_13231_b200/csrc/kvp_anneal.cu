@@ -1516,11 +1516,10 @@ wide_chain_kernel(const ChainParams prm)
 // schedule words are touched (the counters are not needed any more).
 template <bool GROW>
 __global__ void __launch_bounds__(32)
-undo_kernel(const ChainParams prm, uint32_t slot, uint32_t* __restrict__ dst)
+undo_kernel(const ChainParams prm, uint32_t slot)
 {
     const uint32_t lane = threadIdx.x, S = prm.S, S32 = prm.S32;
-    const size_t pwords = (size_t)prm.U * S32;
-    uint32_t* P = prm.ws + (size_t)slot * pwords;
+    uint32_t* P = prm.ws + (size_t)slot * prm.U * S32;
     const uint64_t* ulog = prm.undo_log + (size_t)slot * prm.undo_cap;
     const uint32_t n = prm.undo_len[slot], chain = prm.chain_first + slot;
     for (uint32_t i = n; i-- > 0;) {
@@ -1552,9 +1551,30 @@ undo_kernel(const ChainParams prm, uint32_t slot, uint32_t* __restrict__ dst)
         }
         __syncwarp();
     }
-    __syncwarp();
-    if (prm.cow_out) copy_merged(dst, P, prm.Pcol0, prm.cow_out + (size_t)slot * (kCowBits / 32), prm.cow_shift, prm.U, S32, lane);
-    else copy_words(dst, P, pwords, lane);
+    // the schedule itself is copied out by gather_slice_kernel, on the whole GPU
+}
+
+// The schedule a slice of global scratch stands for, copied to dst: a plain slice (have == null) word for word; a
+// copy-on-write slice bucket by bucket, from the slice where it holds the bucket and from the initial schedule
+// elsewhere. A warp per bucket (per 1024 words of a plain slice).
+__global__ void __launch_bounds__(256)
+gather_slice_kernel(uint32_t* __restrict__ dst, const uint32_t* __restrict__ mine, const uint32_t* __restrict__ p0,
+                    const uint32_t* __restrict__ have, uint32_t shift, uint32_t U, uint32_t S32)
+{
+    const uint32_t lane = threadIdx.x & 31, warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    if (have) {
+        const uint32_t nb = (U + (1u << shift) - 1u) >> shift;
+        for (uint32_t b = warp; b < nb; b += nwarps) {
+            const size_t lo = (size_t)(b << shift) * S32, hi = (size_t)min(U, (b + 1u) << shift) * S32;
+            const uint32_t* src = (have[b >> 5] >> (b & 31u)) & 1u ? mine : p0;
+            for (size_t i = lo + lane; i < hi; i += 32) dst[i] = src[i];
+        }
+    } else {
+        const size_t n = (size_t)U * S32;
+        for (size_t lo = (size_t)warp * 1024; lo < n; lo += (size_t)nwarps * 1024)
+            for (size_t i = lo + lane; i < min(n, lo + 1024); i += 32) dst[i] = mine[i];
+    }
 }
 
 // bit t of full0 is set iff the initial schedule fills the HBM capacity at step t
@@ -2052,10 +2072,15 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
                     prm.chain_first = a->first_chain + first;
                     prm.undo_log = c.undo_log; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
                     prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift;
-                    if (c.grow) undo_kernel<true><<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
-                    else undo_kernel<false><<<1, 32, 0, st>>>(prm, red.best_chain - first, c.dumpcol);
+                    const uint32_t wslot = red.best_chain - first;
+                    if (c.grow) undo_kernel<true><<<1, 32, 0, st>>>(prm, wslot);
+                    else undo_kernel<false><<<1, 32, 0, st>>>(prm, wslot);
                     KVP_CUDA(cudaGetLastError());
-                    ++c.launches;
+                    gather_slice_kernel<<<148 * 4, 256, 0, st>>>(c.dumpcol, c.slots + (size_t)wslot * p->U * p->S32, c.Pcol0,
+                                                                 c.cow_out ? c.cow_out + (size_t)wslot * (kCowBits / 32) : nullptr,
+                                                                 c.cow_shift, p->U, p->S32);
+                    KVP_CUDA(cudaGetLastError());
+                    c.launches += 2;
                     dumped_chain = red.best_chain;
                 }
             }

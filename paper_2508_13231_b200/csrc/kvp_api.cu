@@ -123,7 +123,8 @@ static int create_impl(kvp_problem* p, const uint32_t* access, const uint32_t* h
     char* base = static_cast<char*>(p->d_block);
     p->dA = (uint32_t*)(base + oA); p->dAcol = (uint32_t*)(base + oAcol); p->d_a = (uint32_t*)(base + oa);
     p->d_stepc = (StepC*)(base + osc); p->d_ucnt = (uint32_t*)(base + ouc); p->d_row_freq = (uint32_t*)(base + orf);
-    if ((rc = ensure_scratch(p, (size_t)(p->S + 1) * 16, st))) return rc;
+    // what launch_static_freq_row needs: histogram, selection, tie counts of the chunks of 1024 units
+    if ((rc = ensure_scratch(p, (size_t)(p->S + 8) * 16 + ((size_t)p->W32 / 32 + 2) * 4, st))) return rc;
     if ((rc = launch_clean_copy(access, p->dA, p->S, p->W32, p->pad_mask, st))) return rc;
     if ((rc = launch_row_popcount(p->dA, p->S, p->W32, p->d_a, st))) return rc;
     if ((rc = launch_bit_transpose(p->dA, p->S, p->W32, p->U, p->dAcol, p->S32, st))) return rc;

@@ -53,23 +53,36 @@ __global__ void unit_counts_kernel(const uint32_t* __restrict__ Acol, uint32_t U
     ucnt[u] = c;
 }
 
-__global__ void histogram_kernel(const uint32_t* __restrict__ ucnt, uint32_t U, uint32_t* __restrict__ hist)
+// Histogram of the per-unit access counts (bins 0..S). Few bins and millions of units: every CTA counts its units in
+// shared memory first (when the bins fit) and adds only its non-empty bins to the global histogram.
+constexpr uint32_t kHistBins = 8192;
+__global__ void __launch_bounds__(1024)
+histogram_kernel(const uint32_t* __restrict__ ucnt, uint32_t U, uint32_t bins, uint32_t* __restrict__ hist)
 {
-    const uint32_t u = blockIdx.x * blockDim.x + threadIdx.x;
-    if (u < U) atomicAdd(hist + ucnt[u], 1u);
+    __shared__ uint32_t local[kHistBins];
+    const bool staged = bins <= kHistBins;
+    if (staged) {
+        for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x) local[b] = 0u;
+        __syncthreads();
+    }
+    for (uint32_t u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x)
+        atomicAdd((staged ? local : hist) + ucnt[u], 1u);
+    if (staged) {
+        __syncthreads();
+        for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x)
+            if (local[b]) atomicAdd(hist + b, local[b]);
+    }
 }
 
-// The `cap` most accessed units, ties to the lower index. One CTA: find the count threshold from the
-// histogram, then walk the units in index order with a running count of the ties already taken.
-// sel = {threshold count, number of ties to take}.
+// The `cap` most accessed units, ties to the lower index, in three steps. First, one CTA finds the count threshold
+// from the histogram: sel = {threshold count, number of ties to take}.
 __global__ void __launch_bounds__(1024)
-static_freq_kernel(const uint32_t* __restrict__ ucnt, const uint32_t* __restrict__ hist, uint32_t U, uint32_t S,
-                   uint32_t cap, uint32_t* __restrict__ row, uint32_t W32)
+static_threshold_kernel(const uint32_t* __restrict__ hist, uint32_t S, uint32_t cap, uint32_t* __restrict__ sel)
 {
-    __shared__ uint32_t s_thr, s_take, s_base, s_found;
+    __shared__ uint32_t s_thr, s_take, s_found;
     __shared__ uint32_t s_warp[32];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) { s_thr = S + 1; s_take = 0; s_base = 0; s_found = 0; }
+    if (threadIdx.x == 0) { s_thr = S + 1; s_take = 0; s_found = 0; }
     __syncthreads();
     // counts run 0..S; descend, 1024 counts at a time (thread i looks at count top - i), until the capacity is reached
     if (cap != 0) {
@@ -100,25 +113,49 @@ static_freq_kernel(const uint32_t* __restrict__ ucnt, const uint32_t* __restrict
             __syncthreads();
         }
     }
-    const uint32_t thr = s_thr, take = s_take;
-    const uint32_t Upad = W32 * 32;
-    for (uint32_t u0 = 0; u0 < Upad; u0 += 1024) {
-        const uint32_t u = u0 + threadIdx.x;
-        const uint32_t c = u < U ? ucnt[u] : 0xFFFFFFFFu;
-        const bool tie = u < U && c == thr;
-        const uint32_t tie_bits = __ballot_sync(0xFFFFFFFFu, tie);
-        if (lane == 0) s_warp[warp] = __popc(tie_bits);
-        __syncthreads();
-        uint32_t before = s_base;
-        for (uint32_t w = 0; w < warp; ++w) before += s_warp[w];
-        before += __popc(tie_bits & ((1u << lane) - 1u));
-        const bool pick = u < U && (c > thr || (tie && before < take));
-        const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
-        if (lane == 0 && u < Upad) row[u >> 5] = bits;
-        __syncthreads();
-        if (threadIdx.x == 0) { uint32_t t = 0; for (int w = 0; w < 32; ++w) t += s_warp[w]; s_base += t; }
-        __syncthreads();
-    }
+    if (threadIdx.x == 0) { sel[0] = s_thr; sel[1] = s_take; }
+}
+
+// Second, every CTA counts the ties (units whose count equals the threshold) among its 1024 units.
+__global__ void __launch_bounds__(1024)
+static_ties_kernel(const uint32_t* __restrict__ ucnt, const uint32_t* __restrict__ sel, uint32_t U, uint32_t* __restrict__ ties)
+{
+    const uint32_t u = blockIdx.x * 1024 + threadIdx.x;
+    const int n = __syncthreads_count(u < U && ucnt[u] == sel[0]);
+    if (threadIdx.x == 0) ties[blockIdx.x] = (uint32_t)n;
+}
+
+// Third, every CTA takes its units above the threshold and as many of its ties as are left after the ties of the CTAs
+// before it (ties go to the lower index).
+__global__ void __launch_bounds__(1024)
+static_pick_kernel(const uint32_t* __restrict__ ucnt, const uint32_t* __restrict__ sel, const uint32_t* __restrict__ ties,
+                   uint32_t U, uint32_t* __restrict__ row, uint32_t W32)
+{
+    __shared__ uint32_t s_warp[32];
+    __shared__ uint32_t s_base;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t thr = sel[0], take = sel[1];
+    uint32_t mine = 0;
+    for (uint32_t j = threadIdx.x; j < blockIdx.x; j += 1024) mine += ties[j];
+    mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if (lane == 0) s_warp[warp] = mine;
+    __syncthreads();
+    if (threadIdx.x == 0) { uint32_t t = 0; for (int w = 0; w < 32; ++w) t += s_warp[w]; s_base = t; }
+    __syncthreads();
+    const uint32_t base = s_base;
+    __syncthreads();
+    const uint32_t u = blockIdx.x * 1024 + threadIdx.x;
+    const uint32_t c = u < U ? ucnt[u] : 0xFFFFFFFFu;
+    const bool tie = u < U && c == thr;
+    const uint32_t tie_bits = __ballot_sync(0xFFFFFFFFu, tie);
+    if (lane == 0) s_warp[warp] = __popc(tie_bits);
+    __syncthreads();
+    uint32_t before = base;
+    for (uint32_t w = 0; w < warp; ++w) before += s_warp[w];
+    before += __popc(tie_bits & ((1u << lane) - 1u));
+    const bool pick = u < U && (c > thr || (tie && before < take));
+    const uint32_t bits = __ballot_sync(0xFFFFFFFFu, pick);
+    if (lane == 0 && u < W32 * 32) row[u >> 5] = bits;
 }
 
 __global__ void static_first_kernel(uint32_t* __restrict__ row, uint32_t W32, uint32_t cap)
@@ -231,11 +268,21 @@ int launch_unit_counts(const uint32_t* Acol, uint32_t U, uint32_t S32, uint32_t*
 // needs (S + 1) * 4 bytes of zeroed scratch for the histogram; uses p->d_scratch
 int launch_static_freq_row(const kvp_problem* p, uint32_t* row, cudaStream_t st)
 {
+    // scratch: the histogram (S + 1 bins), the selection (2 words), the tie counts of the chunks of 1024 units
     uint32_t* hist = static_cast<uint32_t*>(p->d_scratch);
+    uint32_t* sel = hist + ((p->S + 1 + 3) & ~3u);
+    uint32_t* ties = sel + 4;
+    const uint32_t chunks = (p->W32 * 32 + 1023) / 1024;
     KVP_CUDA(cudaMemsetAsync(hist, 0, (size_t)(p->S + 1) * 4, st));
-    histogram_kernel<<<(p->U + 255) / 256, 256, 0, st>>>(p->d_ucnt, p->U, hist);
+    uint32_t hgrid = (p->U + 16383) / 16384;
+    if (hgrid > 1184) hgrid = 1184;
+    histogram_kernel<<<hgrid, 1024, 0, st>>>(p->d_ucnt, p->U, p->S + 1, hist);
     KVP_CUDA(cudaGetLastError());
-    static_freq_kernel<<<1, 1024, 0, st>>>(p->d_ucnt, hist, p->U, p->S, p->cap, row, p->W32);
+    static_threshold_kernel<<<1, 1024, 0, st>>>(hist, p->S, p->cap, sel);
+    KVP_CUDA(cudaGetLastError());
+    static_ties_kernel<<<chunks, 1024, 0, st>>>(p->d_ucnt, sel, p->U, ties);
+    KVP_CUDA(cudaGetLastError());
+    static_pick_kernel<<<chunks, 1024, 0, st>>>(p->d_ucnt, sel, ties, p->U, row, p->W32);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }

@@ -47,6 +47,13 @@ CONFIGS = {
                   bw=(49 * TB // 10, 9 * TB // 10, 5 * TB // 10), rho=0.98, sigma=1.0, zipf=(0.8, 1.4),
                   recency_blocks=0, recency_boost=0.0, burst_p=0.0, burst_jump=0.0,
                   chains=1024, moves=200_000, p0=1e-6),
+    # long_70b cut down to 8 of its 640 groups (same steps, top-k, bursts, capacity share, bandwidths): the chains run the
+    # same kernel instantiation as long_70b (two-word columns in global scratch) on 256 KB of schedule each, small enough
+    # for a profiler to hold a GPU-filling job of thousands of chains in a few hundred MB
+    "profile_70b": dict(groups=8, units_per_group=4096, steps=64, topk=205, bytes_per_unit=16384, cap=3276,
+                        bw=(8 * TB, 45 * TB // 100, 45 * TB // 100), rho=0.95, sigma=1.0, zipf=None,
+                        recency_blocks=0, recency_boost=0.0, burst_p=0.01, burst_jump=4.0,
+                        chains=2368, moves=100_000, p0=1e-6),
 }
 ORDER = ["tiny", "single_head", "layer_8b", "full_8b", "long_70b"]
 

@@ -1058,3 +1058,148 @@ int kvpo_policy_page(const kvpo_problem *p, uint32_t page_units, uint32_t *P)
     free(in); free(cand); free(res);
     return KVPO_OK;
 }
+
+/* ------------------------------------------------------------------ */
+/* Replica exchange (parallel tempering) over the temperature ladder of
+ * Section III-B: instead of one chain cooling through the levels C_0 > C_1 >
+ * ..., a ladder of `rungs` replicas runs side by side, replica r of a ladder
+ * starting on rung r, every replica at the fixed temperature of the rung it
+ * holds; every `every` moves neighbouring rungs may exchange their states
+ * (here: their rung indices, the states stay with the chains). The paper has
+ * no replica exchange; the rule is the standard one for Boltzmann weights
+ * exp(-T/C): rungs j (hotter) and j+1 holding states of cost E_j and E_{j+1}
+ * exchange with probability min(1, exp((1/C_j - 1/C_{j+1}) (E_j - E_{j+1}))).
+ * With d = E_j - E_{j+1}: d <= 0 (the colder rung holds the worse state, or
+ * equal) is always accepted; d > 0 is accepted with exp(-d / C_pair),
+ * 1/C_pair = 1/C_{j+1} - 1/C_j, through the same quantised table as a move
+ * (kvpo_accept_table of the pair temperatures; equal temperatures exchange
+ * always).
+ *
+ * Chains first_chain .. first_chain+chains-1, chains a multiple of rungs:
+ * chain c belongs to ladder c / rungs and starts on rung c % rungs (c counted
+ * from 0, not from first_chain, so that a job can be split by ladders).
+ * Round t = 0, 1, ...: every chain proposes moves t*every .. min((t+1)*every,
+ * moves)-1 at its rung's temperature (table row = rung), then, unless the
+ * budget is used up, the pairs (j, j+1) with j = t (mod 2) try to exchange,
+ * lowest j first. The uniform of pair j of ladder l in round t is word 3 of
+ * Philox(counter (t_lo, t_hi, l*rungs + j, 6), key seed).
+ *   table, shifts  [rungs][1024], [rungs]      : move acceptance per rung
+ *   xalways        [rungs-1]                   : 1 = pair (j, j+1) always exchanges
+ *   xtable, xshifts [rungs-1][1024], [rungs-1] : exchange acceptance per pair
+ *   results [chains]; final_rung [chains]; n_exchanged [chains] (exchanges the chain took part in)
+ *   xlog: NULL or [rounds][ladders][rungs-1][3] = {E_hot, E_cold, accepted(0/1)}, pairs not tried keep accepted = 2
+ *   samples: NULL or [rounds][chains][2] = {rung held during the round, state code after the round's moves}
+ *            (state code = the first two words of the schedule, for instances that small)
+ */
+#define TAG_EXCHANGE 6u
+
+int kvpo_anneal_exchange(const kvpo_problem *p, const kvpo_anneal_params *ap, uint32_t rungs, uint64_t every,
+                         const uint32_t *table, const uint32_t *shifts, const uint32_t *xalways,
+                         const uint32_t *xtable, const uint32_t *xshifts, kvpo_chain_result *results,
+                         uint32_t *final_rung, uint32_t *n_exchanged, uint64_t *xlog, uint64_t *samples)
+{
+    if (!p || !ap || !table || !shifts || !results || !rungs || !every) return KVPO_ERR_ARG;
+    if (!ap->chains || ap->chains % rungs || ap->first_chain % rungs || !ap->moves) return KVPO_ERR_ARG;
+    if (rungs > 1 && (!xalways || !xtable || !xshifts)) return KVPO_ERR_ARG;
+    const uint32_t C = ap->chains, ladders = C / rungs;
+    size_t nw = (size_t)p->S * p->W32;
+    uint32_t *P0 = (uint32_t *)malloc(nw * 4);
+    chain_state *st = (chain_state *)calloc(C, sizeof *st);
+    uint32_t *rung = (uint32_t *)malloc((size_t)C * 4);
+    if (!P0 || !st || !rung) { free(P0); free(st); free(rung); return KVPO_ERR_NOMEM; }
+    int rc = resolve_init(p, ap, P0);
+    for (uint32_t i = 0; i < C && !rc; ++i) {
+        rc = state_init(p, &st[i], P0);
+        memset(&results[i], 0, sizeof results[i]);
+        results[i].best_ticks = st[i].cur;
+        results[i].best_move = UINT64_MAX;
+        rung[i] = (ap->first_chain + i) % rungs;
+        if (n_exchanged) n_exchanged[i] = 0;
+    }
+    uint64_t rounds = (ap->moves + every - 1) / every;
+    for (uint64_t t = 0; t < rounds && !rc; ++t) {
+        uint64_t m0 = t * every, m1 = m0 + every < ap->moves ? m0 + every : ap->moves;
+        for (uint32_t i = 0; i < C; ++i) {
+            uint32_t chain = ap->first_chain + i, lev = rung[i];
+            kvpo_chain_result *r = &results[i];
+            for (uint64_t m = m0; m < m1; ++m) {
+                move_t mv = decode_move(p, ap, m, chain, TAG_MOVE);
+                int64_t delta; int32_t d[32][5]; uint32_t last; int changed;
+                if (evaluate_move(p, &st[i], &mv, &delta, d, &last, &changed)) { ++r->n_infeasible; continue; }
+                int accept;
+                if (delta <= 0) accept = 1;
+                else {
+                    uint64_t q = (uint64_t)delta >> shifts[lev];
+                    accept = q < TABLE_Q && mv.w < table[(size_t)lev * TABLE_Q + q];
+                }
+                if (!accept) continue;
+                ++r->n_accepted;
+                if (!changed) continue;
+                apply_move(p, &st[i], &mv, d, last, delta);
+                ++r->n_changed;
+                r->traj_hash = (r->traj_hash ^ m) * 0x9E3779B97F4A7C15ull + st[i].cur;
+                if (st[i].cur < r->best_ticks) { r->best_ticks = st[i].cur; r->best_move = m; }
+            }
+            r->moves_done = m1;
+            r->final_ticks = st[i].cur;
+            if (samples) {
+                uint64_t code = st[i].P[0];
+                if (nw > 1) code |= (uint64_t)st[i].P[1] << 32;
+                samples[((size_t)t * C + i) * 2] = lev;
+                samples[((size_t)t * C + i) * 2 + 1] = code;
+            }
+        }
+        if (xlog)
+            for (size_t k = 0; k < (size_t)ladders * (rungs - 1); ++k) xlog[((size_t)t * ladders * (rungs - 1) + k) * 3 + 2] = 2;
+        if (m1 >= ap->moves) break;                       /* no exchange after the last round */
+        for (uint32_t l = 0; l < ladders; ++l) {
+            uint32_t gl = ap->first_chain / rungs + l;    /* ladder index in the whole job */
+            /* who holds which rung of this ladder */
+            for (uint32_t j = (uint32_t)(t & 1); j + 1 < rungs; j += 2) {
+                uint32_t hot = 0, cold = 0;
+                for (uint32_t i = l * rungs; i < (l + 1) * rungs; ++i) {
+                    if (rung[i] == j) hot = i;
+                    if (rung[i] == j + 1) cold = i;
+                }
+                uint64_t Eh = st[hot].cur, Ec = st[cold].cur;
+                int accept;
+                if (Eh <= Ec || xalways[j]) accept = 1;   /* the colder rung holds the worse state (or equal) */
+                else {
+                    uint32_t x[4];
+                    philox(ap->seed, (uint32_t)t, (uint32_t)(t >> 32), gl * rungs + j, TAG_EXCHANGE, x);
+                    uint64_t q = (Eh - Ec) >> xshifts[j];
+                    accept = q < TABLE_Q && x[3] < xtable[(size_t)j * TABLE_Q + q];
+                }
+                if (xlog) {
+                    uint64_t *e = xlog + (((size_t)t * ladders + l) * (rungs - 1) + j) * 3;
+                    e[0] = Eh; e[1] = Ec; e[2] = (uint64_t)accept;
+                }
+                if (accept) {
+                    rung[hot] = j + 1; rung[cold] = j;
+                    if (n_exchanged) { ++n_exchanged[hot]; ++n_exchanged[cold]; }
+                }
+            }
+        }
+    }
+    for (uint32_t i = 0; i < C; ++i) {
+        if (final_rung) final_rung[i] = rung[i];
+        state_free(&st[i]);
+    }
+    free(P0); free(st); free(rung);
+    return rc;
+}
+
+/* Pair temperatures of a ladder: 1/C_pair = 1/C_{j+1} - 1/C_j (temperatures below 1 tick count as 1, as in the move
+ * table). always[j] = 1 where the two temperatures are equal (or the pair temperature is beyond 2^40 ticks). */
+int kvpo_exchange_temps(const double *temps, uint32_t rungs, double *pair_temps, uint32_t *always)
+{
+    if (!temps || !rungs || (rungs > 1 && (!pair_temps || !always))) return KVPO_ERR_ARG;
+    for (uint32_t j = 0; j + 1 < rungs; ++j) {
+        double a = temps[j] >= 1.0 ? temps[j] : 1.0, b = temps[j + 1] >= 1.0 ? temps[j + 1] : 1.0;
+        if (b > a) return KVPO_ERR_ARG;                   /* a ladder falls */
+        double inv = 1.0 / b - 1.0 / a;
+        if (!(inv > 0.0) || 1.0 / inv > 1099511627776.0) { always[j] = 1; pair_temps[j] = 1.0; }
+        else { always[j] = 0; pair_temps[j] = 1.0 / inv; }
+    }
+    return KVPO_OK;
+}

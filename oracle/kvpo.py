@@ -224,6 +224,41 @@ class Problem:
                                      C.c_uint32(count), _u32p(out)), "decode_moves")
         return out
 
+    def exchange_tables(self, ap, rungs):
+        """Ladder temperatures, move table and exchange table of a replica-exchange run (ap.levels == rungs).
+        -> dict(temps, table, shifts, pair_temps, xalways, xtable, xshifts)"""
+        assert ap.levels == rungs
+        temps, _ = self.temps(ap)
+        table, shifts = accept_table(temps)
+        pair = np.ones(max(1, rungs - 1), np.float64)
+        always = np.zeros(max(1, rungs - 1), np.uint32)
+        _chk(lib().kvpo_exchange_temps(temps.ctypes.data_as(C.POINTER(C.c_double)), C.c_uint32(rungs),
+                                       pair.ctypes.data_as(C.POINTER(C.c_double)), _u32p(always)), "exchange_temps")
+        xtable, xshifts = accept_table(pair)
+        return dict(temps=temps, table=table, shifts=shifts, pair_temps=pair, xalways=always, xtable=xtable, xshifts=xshifts)
+
+    def anneal_exchange(self, ap, rungs, every, want_log=False, want_samples=False):
+        """Replica exchange: ap.chains chains in ladders of `rungs`, exchanges every `every` moves.
+        -> dict(per_chain, final_rung, n_exchanged, best_ticks, best_chain, xlog [rounds][ladders][rungs-1][3] or None,
+                samples [rounds][chains][2] or None)"""
+        tb = self.exchange_tables(ap, rungs)
+        n = ap.chains
+        res = (ChainResult * n)()
+        final_rung = np.zeros(n, np.uint32)
+        n_ex = np.zeros(n, np.uint32)
+        rounds = (ap.moves + every - 1) // every
+        ladders = n // rungs
+        xlog = np.zeros((rounds, ladders, max(1, rungs - 1), 3), np.uint64) if want_log else None
+        samples = np.zeros((rounds, n, 2), np.uint64) if want_samples else None
+        _chk(lib().kvpo_anneal_exchange(self._h, C.byref(ap), C.c_uint32(rungs), C.c_uint64(every), _u32p(tb["table"]),
+                                        _u32p(tb["shifts"]), _u32p(tb["xalways"]), _u32p(tb["xtable"]), _u32p(tb["xshifts"]),
+                                        res, _u32p(final_rung), _u32p(n_ex), _u64p(xlog), _u64p(samples)), "anneal_exchange")
+        per = list(res)
+        ticks = [r.best_ticks for r in per]
+        bc = int(np.argmin(ticks))
+        return dict(per_chain=per, final_rung=final_rung, n_exchanged=n_ex, best_ticks=int(ticks[bc]),
+                    best_chain=ap.first_chain + bc, xlog=xlog, samples=samples, tables=tb)
+
     def check_total(self, P, ticks):
         return lib().kvpo_check_total(self._h, _u32p(self._sched(P)), C.c_uint64(ticks)) == 0
 

@@ -250,6 +250,9 @@ typedef struct {
     uint64_t work_again;        /* proposals evaluated a second time after a move was applied in their batch   */
     uint64_t work_listed;       /* evaluations that needed more than the placement bits (a cost evaluation)    */
     uint64_t work_items;        /* (proposal, step) pairs whose step cost (Eq. 2-4) was evaluated              */
+    /* kvp_anneal_exchange only: */
+    uint64_t exchanges_tried, exchanges_accepted;
+    uint32_t exchange_rounds, reserved2;
 } kvp_anneal_stats;
 
 /*
@@ -282,6 +285,41 @@ int kvp_accept_table(const double* temps, uint32_t levels, uint32_t* table, uint
  */
 int kvp_anneal(kvp_problem* p, const kvp_anneal_params* params, uint32_t* best_schedule,
                uint64_t* best_ticks, double* best_seconds, kvp_anneal_stats* stats, void* stream);
+
+/*
+ * kvp_anneal_exchange -- replica exchange (parallel tempering) over the temperature ladder of Section III-B. The
+ * paper anneals one chain through falling temperatures; here `rungs` replicas form a ladder, replica r starting on
+ * rung r, every replica running at the fixed temperature C_r of the rung it holds, and every `exchange_every` moves
+ * neighbouring rungs may exchange (the chains keep their schedules, the rungs change hands). The rule is the
+ * standard one for Boltzmann weights exp(-T/C): rungs j (hotter) and j+1 with present costs E_j, E_{j+1} exchange
+ * with probability min(1, exp((1/C_j - 1/C_{j+1}) (E_j - E_{j+1}))): always when the colder rung holds the worse
+ * schedule (or an equal one), else with exp(-d / C_pair), d = E_j - E_{j+1}, 1/C_pair = 1/C_{j+1} - 1/C_j, through
+ * the quantised table of kvp_accept_table at the pair temperatures (kvp_exchange_temps); pairs of equal temperature
+ * exchange always.
+ *   params: as for kvp_anneal with levels == rungs (the ladder: `temps`, or C_0 from p0 and C_{j+1} = alpha C_j),
+ *     chains and first_chain multiples of rungs (chain c belongs to ladder c / rungs, so a job can be split by
+ *     ladders over GPUs or calls), early_stop_permille == 0.
+ *   Round t = 0, 1, ...: every chain proposes its moves t * exchange_every .. (t + 1) * exchange_every - 1 (up to
+ *     `moves`); then, unless the budget is used up, the pairs (j, j+1) with j = t (mod 2) try to exchange. The uniform
+ *     of pair j of ladder l in round t is word 3 of Philox4x32-10(counter (t_lo, t_hi, l * rungs + j, 6), key seed).
+ *   final_rung  (host) [chains] or NULL: the rung each chain holds at the end
+ *   n_exchanged (host) [chains] or NULL: the exchanges each chain took part in
+ *   best_schedule, best_ticks, best_seconds, stats: as for kvp_anneal (per-chain results over all rounds).
+ * Limits: rungs <= 256; rounds * chains <= 2^30 (the rung history is kept); chains whose schedules do not fit shared
+ * memory must all be resident at once (KVP_ERR_RANGE otherwise). Synchronises `stream` before returning.
+ */
+typedef struct {
+    uint32_t rungs;             /* replicas per ladder = temperatures of the ladder, 1..256 */
+    uint32_t reserved;          /* must be 0 */
+    uint64_t exchange_every;    /* moves between exchange rounds, >= 1 */
+} kvp_exchange_params;
+int kvp_anneal_exchange(kvp_problem* p, const kvp_anneal_params* params, const kvp_exchange_params* xp,
+                        uint32_t* best_schedule, uint64_t* best_ticks, double* best_seconds, kvp_anneal_stats* stats,
+                        uint32_t* final_rung, uint32_t* n_exchanged, void* stream);
+
+/* Pair temperatures of a ladder (host arithmetic): 1/pair_temps[j] = 1/temps[j+1] - 1/temps[j] with temperatures below
+ * one tick counted as one; always[j] = 1 where the pair exchanges unconditionally (equal temperatures). */
+int kvp_exchange_temps(const double* temps, uint32_t rungs, double* pair_temps, uint32_t* always);
 
 /*
  * kvp_anneal_chain_state -- replay one chain for its first `upto_moves` proposals

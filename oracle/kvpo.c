@@ -1090,13 +1090,15 @@ int kvpo_policy_page(const kvpo_problem *p, uint32_t page_units, uint32_t *P)
  *   xlog: NULL or [rounds][ladders][rungs-1][3] = {E_hot, E_cold, accepted(0/1)}, pairs not tried keep accepted = 2
  *   samples: NULL or [rounds][chains][2] = {rung held during the round, state code after the round's moves}
  *            (state code = the first two words of the schedule, for instances that small)
+ *   best_states: NULL or [chains][S][W32] = every chain's schedule when it reached its best_ticks
  */
 #define TAG_EXCHANGE 6u
 
 int kvpo_anneal_exchange(const kvpo_problem *p, const kvpo_anneal_params *ap, uint32_t rungs, uint64_t every,
                          const uint32_t *table, const uint32_t *shifts, const uint32_t *xalways,
                          const uint32_t *xtable, const uint32_t *xshifts, kvpo_chain_result *results,
-                         uint32_t *final_rung, uint32_t *n_exchanged, uint64_t *xlog, uint64_t *samples)
+                         uint32_t *final_rung, uint32_t *n_exchanged, uint64_t *xlog, uint64_t *samples,
+                         uint32_t *best_states)
 {
     if (!p || !ap || !table || !shifts || !results || !rungs || !every) return KVPO_ERR_ARG;
     if (!ap->chains || ap->chains % rungs || ap->first_chain % rungs || !ap->moves) return KVPO_ERR_ARG;
@@ -1115,6 +1117,7 @@ int kvpo_anneal_exchange(const kvpo_problem *p, const kvpo_anneal_params *ap, ui
         results[i].best_move = UINT64_MAX;
         rung[i] = (ap->first_chain + i) % rungs;
         if (n_exchanged) n_exchanged[i] = 0;
+        if (best_states && !rc) memcpy(best_states + i * nw, st[i].P, nw * 4);
     }
     uint64_t rounds = (ap->moves + every - 1) / every;
     for (uint64_t t = 0; t < rounds && !rc; ++t) {
@@ -1138,7 +1141,10 @@ int kvpo_anneal_exchange(const kvpo_problem *p, const kvpo_anneal_params *ap, ui
                 apply_move(p, &st[i], &mv, d, last, delta);
                 ++r->n_changed;
                 r->traj_hash = (r->traj_hash ^ m) * 0x9E3779B97F4A7C15ull + st[i].cur;
-                if (st[i].cur < r->best_ticks) { r->best_ticks = st[i].cur; r->best_move = m; }
+                if (st[i].cur < r->best_ticks) {
+                    r->best_ticks = st[i].cur; r->best_move = m;
+                    if (best_states) memcpy(best_states + i * nw, st[i].P, nw * 4);
+                }
             }
             r->moves_done = m1;
             r->final_ticks = st[i].cur;

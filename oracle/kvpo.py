@@ -237,7 +237,7 @@ class Problem:
         xtable, xshifts = accept_table(pair)
         return dict(temps=temps, table=table, shifts=shifts, pair_temps=pair, xalways=always, xtable=xtable, xshifts=xshifts)
 
-    def anneal_exchange(self, ap, rungs, every, want_log=False, want_samples=False):
+    def anneal_exchange(self, ap, rungs, every, want_log=False, want_samples=False, want_best=False):
         """Replica exchange: ap.chains chains in ladders of `rungs`, exchanges every `every` moves.
         -> dict(per_chain, final_rung, n_exchanged, best_ticks, best_chain, xlog [rounds][ladders][rungs-1][3] or None,
                 samples [rounds][chains][2] or None)"""
@@ -250,14 +250,16 @@ class Problem:
         ladders = n // rungs
         xlog = np.zeros((rounds, ladders, max(1, rungs - 1), 3), np.uint64) if want_log else None
         samples = np.zeros((rounds, n, 2), np.uint64) if want_samples else None
+        bst = np.zeros((n, self.steps, self.w32), np.uint32) if want_best else None
         _chk(lib().kvpo_anneal_exchange(self._h, C.byref(ap), C.c_uint32(rungs), C.c_uint64(every), _u32p(tb["table"]),
                                         _u32p(tb["shifts"]), _u32p(tb["xalways"]), _u32p(tb["xtable"]), _u32p(tb["xshifts"]),
-                                        res, _u32p(final_rung), _u32p(n_ex), _u64p(xlog), _u64p(samples)), "anneal_exchange")
+                                        res, _u32p(final_rung), _u32p(n_ex), _u64p(xlog), _u64p(samples), _u32p(bst)), "anneal_exchange")
         per = list(res)
         ticks = [r.best_ticks for r in per]
         bc = int(np.argmin(ticks))
         return dict(per_chain=per, final_rung=final_rung, n_exchanged=n_ex, best_ticks=int(ticks[bc]),
-                    best_chain=ap.first_chain + bc, xlog=xlog, samples=samples, tables=tb)
+                    best_chain=ap.first_chain + bc, xlog=xlog, samples=samples, tables=tb,
+                    best_schedule=bst[bc] if want_best else None)
 
     def check_total(self, P, ticks):
         return lib().kvpo_check_total(self._h, _u32p(self._sched(P)), C.c_uint64(ticks)) == 0

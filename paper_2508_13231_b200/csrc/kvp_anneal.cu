@@ -62,6 +62,16 @@ struct ChainParams {
     uint32_t cow_shift;          // a bucket is 2^cow_shift consecutive units
     uint32_t stage_stepc;        // wide kernel without a staged access bitmap: the step constants alone are staged
     unsigned long long* work;    // wide kernel: [3] sums over the chains of {n_again, n_listed, n_items}
+    // Replica exchange (wide kernel): the call runs rounds round0 .. round1-1; in round t chain c proposes moves
+    // t * exch_every .. (t + 1) * exch_every - 1 (up to `upto`) with the table row of the rung it holds,
+    // rung_hist[t * hist_stride + (c - hist_base)].
+    const uint8_t* rung_hist;    // null: the ordinary cooling schedule by temperature levels
+    uint64_t exch_every;
+    uint32_t round0, round1, hist_stride, hist_base;
+    uint4* state;                // if set: [chains][state4] the chain's persistent shared-memory state (and its
+                                 // schedule, when that lives in shared memory), indexed like rung_hist
+    uint32_t state4;             // uint4 slots per chain in `state`
+    uint32_t resume;             // 1: start from `state` instead of the initial schedule
 };
 
 // Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
@@ -966,9 +976,18 @@ struct WideScalars {
     uint32_t pad[2];
     // what the chain's evaluations amounted to (kvp_anneal_stats): proposals evaluated again after an applied move,
     // proposals that needed a cost evaluation, (proposal, step) items
-    uint64_t n_again, n_listed, n_items, pad2;
+    uint64_t n_again, n_listed, n_items;
+    uint64_t n_acc, n_inf;       // accepted / infeasible proposals of earlier calls on this state (replica exchange)
+    uint64_t pad2;
 };
 constexpr uint32_t kWideScalars4 = sizeof(WideScalars) / 16;
+
+// the part of wide_fixed4 that outlives a batch (what a replica-exchange run saves between its rounds)
+__host__ __device__ inline uint32_t wide_persist4(uint32_t S, uint32_t S32, bool grow, bool shared)
+{
+    return (shared ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (S + 3) / 4 + (shared ? 0u : kCowSlots4) +
+           kWideScalars4;
+}
 
 // shared-memory words (as uint4 slots) of one chain of the wide kernel besides its schedule
 __host__ __device__ inline uint32_t wide_fixed4(uint32_t S, uint32_t S32, bool grow, bool shared)
@@ -1349,13 +1368,22 @@ wide_chain_kernel(const ChainParams prm)
         if (lane == 0) {
             sc->cur = sc->best = sc->best_at_boundary = prm.init_ticks;
             sc->best_move = ~0ull; sc->n_chg = 0; sc->hash = 0; sc->ulen = 0u; sc->snap_dirty = 0u;
-            sc->n_again = sc->n_listed = sc->n_items = 0;
+            sc->n_again = sc->n_listed = sc->n_items = 0; sc->n_acc = sc->n_inf = 0;
         }
         if (COW) {
             for (uint32_t i = lane; i < kCowBits / 32; i += 32) cv.have[i] = 0u;   // the slice holds nothing yet
-        } else {
+        } else if (!(prm.state && prm.resume)) {
             copy_words_cold(cv.P, prm.Pcol0, pwords, lane);
         }
+    }
+    // the persistent part of a chain's shared memory: counters, full-step bitmap, written-to-HBM counts, present step
+    // costs, overlay bitmap, scalars (everything before the per-batch work areas)
+    const uint32_t persist4 = c4 + f4 + h4 + n4 + o4 + kWideScalars4;
+    uint4* const saved = prm.state ? prm.state + (size_t)(chain - prm.hist_base) * prm.state4 : nullptr;
+    if (active && saved && prm.resume) {
+        __syncwarp();
+        for (uint32_t i = lane; i < persist4; i += 32) mine4[i] = saved[i];
+        if (PSMEM) copy_words_cold(cv.P, reinterpret_cast<const uint32_t*>(saved + persist4), pwords, lane);
     }
     __syncthreads();
     if (!active) return;
@@ -1364,13 +1392,17 @@ wide_chain_kernel(const ChainParams prm)
 
     uint64_t n_acc = 0, n_inf = 0;                                // per lane: of the proposals this lane owned
 
-    uint64_t lvl_start = 0;
+    // A segment of moves at one temperature: a level of the cooling schedule, or a round of a replica-exchange run.
+    const bool exchange = prm.rung_hist != nullptr;
+    uint64_t lvl_start = exchange ? (uint64_t)prm.round0 * prm.exch_every : 0;
     bool stop = false;
-    for (uint32_t level = 0; level < prm.levels && lvl_start < prm.upto; ++level) {
-        const uint64_t lvl_len = (level + 1 < prm.levels ? min(lvl_start + prm.per_level, prm.upto) : prm.upto) - lvl_start;
+    for (uint32_t seg = exchange ? prm.round0 : 0u; seg < (exchange ? prm.round1 : prm.levels) && lvl_start < prm.upto; ++seg) {
+        const uint32_t level = exchange ? prm.rung_hist[(size_t)seg * prm.hist_stride + (chain - prm.hist_base)] : seg;
+        const uint64_t lvl_len = exchange ? min(prm.exch_every, prm.upto - lvl_start)
+                                          : (level + 1 < prm.levels ? min(lvl_start + prm.per_level, prm.upto) : prm.upto) - lvl_start;
         const uint32_t shift = __ldg(prm.shifts + level);
         const uint32_t* trow = prm.table + (size_t)level * KVP_TABLE_Q;
-        if (level > 0) {
+        if (!exchange && level > 0) {
             const uint64_t best = sc->best, before = sc->best_at_boundary;
             if (prm.early_permille && level >= prm.early_from &&
                 (before - best) * 1000ull < before * (uint64_t)prm.early_permille) {
@@ -1482,12 +1514,20 @@ wide_chain_kernel(const ChainParams prm)
         }
         lvl_start += lvl_len;
     }
-    const uint64_t m_end = stop ? lvl_start : prm.upto;           // moves done when the chain ended
+    const uint64_t m_end = stop || exchange ? lvl_start : prm.upto;   // moves done when the call ended
     // accepted and infeasible proposals were counted by the lanes that owned them
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         n_acc += __shfl_xor_sync(0xFFFFFFFFu, n_acc, off);
         n_inf += __shfl_xor_sync(0xFFFFFFFFu, n_inf, off);
+    }
+    n_acc += sc->n_acc; n_inf += sc->n_inf;                       // plus those of earlier calls on this state
+    __syncwarp();
+    if (lane == 0) { sc->n_acc = n_acc; sc->n_inf = n_inf; }
+    __syncwarp();
+    if (saved) {                                                  // the next round goes on from here
+        for (uint32_t i = lane; i < persist4; i += 32) saved[i] = mine4[i];
+        if (PSMEM) copy_words_cold(reinterpret_cast<uint32_t*>(saved + persist4), cv.P, pwords, lane);
     }
     if (snap && sc->snap_dirty) copy_words_cold(snap, cv.P, pwords, lane);
     if (ulog && lane == 0) prm.undo_len[slot] = sc->ulen;
@@ -1644,6 +1684,67 @@ reduce_kernel(const kvp_chain_result* __restrict__ res, uint32_t chains, const u
     }
 }
 
+// One exchange round of a replica-exchange run: in every ladder the pairs of neighbouring rungs (j, j+1) with
+// j = t (mod 2) may exchange. The chains keep their states; what changes hands is the rung, i.e. the temperature
+// the chain runs at in the next round. A thread per ladder.
+//   holder [ladders][rungs] : the chain (index within the call) that holds each rung; updated
+//   rung_next [chains]      : the rungs for round t + 1 (the next row of the rung history)
+//   counts                  : {exchanges tried, exchanges accepted}
+struct ExchangeK {
+    const kvp_chain_result* results;   // final_ticks = the chain's present cost
+    uint32_t* holder;
+    uint8_t* rung_next;
+    uint32_t* n_exchanged;
+    unsigned long long* counts;
+    const uint32_t* xalways; const uint32_t* xtable; const uint32_t* xshifts;
+    uint32_t ladders, rungs, first_ladder;
+    uint32_t seed_lo, seed_hi;
+    uint64_t t;
+};
+
+__global__ void __launch_bounds__(128)
+exchange_kernel(const ExchangeK k)
+{
+    const uint32_t l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l >= k.ladders) return;
+    uint32_t* hold = k.holder + (size_t)l * k.rungs;
+    uint32_t tried = 0, done = 0;
+    for (uint32_t j = (uint32_t)(k.t & 1ull); j + 1 < k.rungs; j += 2) {
+        const uint32_t hot = hold[j], cold = hold[j + 1];
+        const uint64_t Eh = k.results[hot].final_ticks, Ec = k.results[cold].final_ticks;
+        bool accept;
+        if (Eh <= Ec || k.xalways[j]) {
+            accept = true;                                // the colder rung holds the worse schedule (or an equal one)
+        } else {
+            uint32_t x[4];
+            philox4x32_10((uint32_t)k.t, (uint32_t)(k.t >> 32), (k.first_ladder + l) * k.rungs + j, TAG_EXCHANGE, k.seed_lo,
+                          k.seed_hi, x);
+            const uint64_t q = (Eh - Ec) >> k.xshifts[j];
+            accept = q < KVP_TABLE_Q && x[3] < k.xtable[(size_t)j * KVP_TABLE_Q + q];
+        }
+        ++tried;
+        if (accept) {
+            hold[j] = cold; hold[j + 1] = hot;
+            ++k.n_exchanged[hot]; ++k.n_exchanged[cold];
+            ++done;
+        }
+    }
+    for (uint32_t j = 0; j < k.rungs; ++j) k.rung_next[hold[j]] = (uint8_t)j;
+    if (tried) {
+        atomicAdd(k.counts, (unsigned long long)tried);
+        atomicAdd(k.counts + 1, (unsigned long long)done);
+    }
+}
+
+__global__ void exchange_init_kernel(uint32_t* holder, uint8_t* rung0, uint32_t* n_exchanged, uint32_t chains, uint32_t rungs)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= chains) return;
+    holder[i] = i;                                        // chain i of the call starts on rung i % rungs of ladder i / rungs
+    rung0[i] = (uint8_t)(i % rungs);
+    n_exchanged[i] = 0u;
+}
+
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // Everything a run needs on the device, carved out of the problem's chain workspace.
@@ -1756,7 +1857,7 @@ int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp
 }
 
 // Initial schedule, its counters and cost, the temperature ladder and the acceptance table.
-int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
+int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c, bool exchange = false)
 {
     int rc = validate(p, a);
     if (rc) return rc;
@@ -1779,7 +1880,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     // chain): the wide kernel, which needs half the instructions per proposal. Few chains per SM: the narrow kernel
     // with two warps per chain, which hides the latency of a chain's serial parts behind its second warp.
     // kvp_set_test_hooks can force either (warps_per_chain 1 or 2: narrow; 3: wide).
-    c.wide = hooks.warps_per_chain == 3 || (hooks.warps_per_chain == 0 && (a->chains + sms - 1) / sms > 8);
+    c.wide = exchange || hooks.warps_per_chain == 3 || (hooks.warps_per_chain == 0 && (a->chains + sms - 1) / sms > 8);
     // `shared`: the schedule is in shared memory (the wide kernel then keeps 16-bit counters)
     auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false, bool shared = true) {
         if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared) * 16;
@@ -1875,6 +1976,8 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c)
     }
     c.cow_shift = 0;
     while (((uint64_t)p->U + (1ull << c.cow_shift) - 1) >> c.cow_shift > kCowBits) ++c.cow_shift;
+    // a replica-exchange run keeps every chain's slice between its rounds: all chains have to be resident at once
+    if (exchange && !c.psmem && a->chains > c.resident) return KVP_ERR_RANGE;
 
     // workspace layout
     size_t off = 0;
@@ -2176,4 +2279,174 @@ extern "C" void kvp_set_test_hooks(const kvp_test_hooks* hooks)
 {
     if (hooks) g_hooks = *hooks;
     else memset(&g_hooks, 0, sizeof g_hooks);
+}
+
+extern "C" int kvp_exchange_temps(const double* temps, uint32_t rungs, double* pair_temps, uint32_t* always)
+{
+    if (!temps || !rungs || (rungs > 1 && (!pair_temps || !always))) return KVP_ERR_ARG;
+    for (uint32_t j = 0; j + 1 < rungs; ++j) {
+        const double a = temps[j] >= 1.0 ? temps[j] : 1.0, b = temps[j + 1] >= 1.0 ? temps[j + 1] : 1.0;
+        if (b > a) return KVP_ERR_ARG;                     // a ladder falls
+        const double inv = 1.0 / b - 1.0 / a;
+        if (!(inv > 0.0) || 1.0 / inv > 1099511627776.0) { always[j] = 1; pair_temps[j] = 1.0; }
+        else { always[j] = 0; pair_temps[j] = 1.0 / inv; }
+    }
+    return KVP_OK;
+}
+
+extern "C" int kvp_anneal_exchange(kvp_problem* p, const kvp_anneal_params* a, const kvp_exchange_params* xp,
+                                   uint32_t* best_schedule, uint64_t* best_ticks, double* best_seconds,
+                                   kvp_anneal_stats* stats, uint32_t* final_rung, uint32_t* n_exchanged, void* stream)
+{
+    Ctx c;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int rc = validate(p, a);
+    if (rc) return rc;
+    if (!xp || !xp->rungs || xp->rungs > 256 || xp->reserved || !xp->exchange_every) return KVP_ERR_ARG;
+    const uint32_t rungs = xp->rungs, chains = a->chains;
+    if (a->levels != rungs || chains % rungs || a->first_chain % rungs || a->early_stop_permille) return KVP_ERR_ARG;
+    const uint64_t rounds64 = (a->moves + xp->exchange_every - 1) / xp->exchange_every;
+    if (rounds64 * chains > (1ull << 30)) return KVP_ERR_RANGE;          // the rung history is kept: one byte per chain and round
+    const uint32_t rounds = (uint32_t)rounds64;
+    KVP_CUDA(cudaSetDevice(p->device));
+    struct Events {
+        cudaEvent_t e[4];
+        int n = 0;
+        ~Events() { for (int i = 0; i < n; ++i) cudaEventDestroy(e[i]); }
+        cudaEvent_t operator[](int i) const { return e[i]; }
+    } ev;
+    for (; ev.n < 4; ++ev.n) KVP_CUDA(cudaEventCreate(&ev.e[ev.n]));
+    KVP_CUDA(cudaEventRecord(ev[0], st));
+    if ((rc = prepare(p, a, st, c, true))) return rc;
+
+    // exchange thresholds of the pairs of neighbouring rungs: the move table's form at the pair temperatures
+    const uint32_t pairs = rungs > 1 ? rungs - 1 : 1;
+    std::vector<double> pair_temps(pairs, 1.0);
+    std::vector<uint32_t> always(pairs, 0u), xtable((size_t)pairs * KVP_TABLE_Q), xshifts(pairs);
+    if ((rc = kvp_exchange_temps(c.temps.data(), rungs, pair_temps.data(), always.data()))) return rc;
+    if ((rc = kvp_accept_table(pair_temps.data(), pairs, xtable.data(), xshifts.data()))) return rc;
+
+    // workspace of the run: rung history, holders, exchange counts, thresholds, the chains' saved states
+    const uint32_t persist4 = wide_persist4(p->S, p->S32, c.grow, c.psmem);
+    const size_t pwords = (size_t)p->U * p->S32;
+    const uint32_t state4 = persist4 + (c.psmem ? (uint32_t)((pwords + 3) / 4) : 0u);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
+    const size_t o_hist = take((size_t)rounds * chains), o_hold = take((size_t)chains * 4), o_nex = take((size_t)chains * 4);
+    const size_t o_cnt = take(16), o_alw = take((size_t)pairs * 4), o_xsh = take((size_t)pairs * 4);
+    const size_t o_xt = take((size_t)pairs * KVP_TABLE_Q * 4), o_state = take((size_t)chains * state4 * 16);
+    char* xw = nullptr;
+    KVP_CUDA(cudaMallocAsync(&xw, off, st));
+    struct Free {                                          // in stream order, on every way out
+        char* ptr; cudaStream_t st;
+        ~Free() { cudaFreeAsync(ptr, st); }
+    } guard{xw, st};
+    uint8_t* hist = (uint8_t*)(xw + o_hist);
+    uint32_t* holder = (uint32_t*)(xw + o_hold);
+    uint32_t* nex = (uint32_t*)(xw + o_nex);
+    unsigned long long* counts = (unsigned long long*)(xw + o_cnt);
+    KVP_CUDA(cudaMemsetAsync(counts, 0, 16, st));
+    KVP_CUDA(cudaMemcpyAsync(xw + o_alw, always.data(), (size_t)pairs * 4, cudaMemcpyHostToDevice, st));
+    KVP_CUDA(cudaMemcpyAsync(xw + o_xsh, xshifts.data(), (size_t)pairs * 4, cudaMemcpyHostToDevice, st));
+    KVP_CUDA(cudaMemcpyAsync(xw + o_xt, xtable.data(), xtable.size() * 4, cudaMemcpyHostToDevice, st));
+    exchange_init_kernel<<<(chains + 255) / 256, 256, 0, st>>>(holder, hist, nex, chains, rungs);
+    KVP_CUDA(cudaGetLastError());
+    ++c.launches;
+    KVP_CUDA(cudaEventRecord(ev[1], st));
+
+    ChainParams prm = c.prm;
+    prm.snap = c.snap; prm.undo_log = nullptr; prm.touch_log = nullptr; prm.restore = 0u;
+    prm.cow_out = nullptr; prm.cow_shift = c.cow_shift; prm.stage_stepc = c.stage_stepc ? 1u : 0u;
+    prm.chain_first = a->first_chain; prm.chain_count = chains; prm.result_base = a->first_chain;
+    prm.results = c.results; prm.upto = a->moves; prm.dump = nullptr;
+    prm.rung_hist = hist; prm.exch_every = xp->exchange_every; prm.hist_stride = chains; prm.hist_base = a->first_chain;
+    prm.state = (uint4*)(xw + o_state); prm.state4 = state4;
+    unsigned long long* work_dev = reinterpret_cast<unsigned long long*>(c.small + 24);
+    KVP_CUDA(cudaMemsetAsync(work_dev, 0, 24, st));
+    ExchangeK xk;
+    xk.results = c.results; xk.holder = holder; xk.n_exchanged = nex; xk.counts = counts;
+    xk.xalways = (const uint32_t*)(xw + o_alw); xk.xtable = (const uint32_t*)(xw + o_xt); xk.xshifts = (const uint32_t*)(xw + o_xsh);
+    xk.ladders = chains / rungs; xk.rungs = rungs; xk.first_ladder = a->first_chain / rungs;
+    xk.seed_lo = (uint32_t)a->seed; xk.seed_hi = (uint32_t)(a->seed >> 32);
+    for (uint32_t t = 0; t < rounds; ++t) {
+        prm.round0 = t; prm.round1 = t + 1; prm.resume = t > 0 ? 1u : 0u;
+        prm.work = t + 1 == rounds ? work_dev : nullptr;   // the counts travel with the saved state; the last round reports
+        if ((rc = launch_chains(c, prm, chains))) return rc;
+        ++c.launches;
+        if (t + 1 < rounds) {
+            xk.t = t; xk.rung_next = hist + (size_t)(t + 1) * chains;
+            exchange_kernel<<<(xk.ladders + 127) / 128, 128, 0, st>>>(xk);
+            KVP_CUDA(cudaGetLastError());
+            ++c.launches;
+        }
+    }
+    KVP_CUDA(cudaEventRecord(ev[2], st));
+
+    ReduceOut* red_dev = reinterpret_cast<ReduceOut*>(c.small + 8);
+    ReduceOut red;
+    reduce_kernel<<<1, 1024, 0, st>>>(c.results, chains, c.prm.err, red_dev);
+    KVP_CUDA(cudaGetLastError());
+    ++c.launches;
+    unsigned long long work[3] = {0, 0, 0}, xcounts[2] = {0, 0};
+    KVP_CUDA(cudaMemcpyAsync(&red, red_dev, sizeof red, cudaMemcpyDeviceToHost, st));
+    KVP_CUDA(cudaMemcpyAsync(work, work_dev, sizeof work, cudaMemcpyDeviceToHost, st));
+    KVP_CUDA(cudaMemcpyAsync(xcounts, counts, sizeof xcounts, cudaMemcpyDeviceToHost, st));
+    KVP_CUDA(cudaStreamSynchronize(st));
+    // the winner's schedule: its snapshot, or a replay of that one chain through the rungs it held
+    const uint64_t upto = red.best_move == ~0ull ? 0 : red.best_move + 1;
+    if (upto == 0) {
+        KVP_CUDA(cudaMemcpyAsync(c.sched, c.P0, (size_t)p->S * p->W32 * 4, cudaMemcpyDeviceToDevice, st));
+    } else if (c.snap) {
+        if ((rc = launch_bit_transpose(c.snap + (size_t)red.best_chain * pwords, p->U, p->S32, p->S, c.sched, p->W32, st))) return rc;
+        ++c.launches;
+    } else {
+        ChainParams rp = prm;
+        rp.snap = nullptr; rp.state = nullptr; rp.resume = 0u; rp.work = nullptr;
+        rp.chain_first = a->first_chain + red.best_chain; rp.chain_count = 1; rp.result_base = rp.chain_first;
+        rp.results = c.results + chains; rp.upto = upto; rp.dump = c.dumpcol;
+        rp.round0 = 0; rp.round1 = rounds;
+        if ((rc = launch_chains(c, rp, 1))) return rc;
+        if ((rc = launch_bit_transpose(c.dumpcol, p->U, p->S32, p->S, c.sched, p->W32, st))) return rc;
+        c.launches += 2;
+    }
+    red.best_chain += a->first_chain;
+    if ((rc = launch_counts(p, c.sched, 1, c.counts0, c.hb_tmp, st, &c.launches))) return rc;
+    if ((rc = launch_finish(p, c.counts0, c.hb_tmp, 1, nullptr, c.small, nullptr, nullptr, (int32_t*)(c.small + 2),
+                            c.small + 1, st)))
+        return rc;
+    ++c.launches;
+    if (best_schedule)
+        KVP_CUDA(cudaMemcpyAsync(best_schedule, c.sched, (size_t)p->S * p->W32 * 4, cudaMemcpyDeviceToDevice, st));
+    uint64_t host_small[4];
+    KVP_CUDA(cudaMemcpyAsync(host_small, c.small, sizeof host_small, cudaMemcpyDeviceToHost, st));
+    if (stats && stats->per_chain)
+        KVP_CUDA(cudaMemcpyAsync(stats->per_chain, c.results, (size_t)chains * sizeof(kvp_chain_result), cudaMemcpyDeviceToHost, st));
+    std::vector<uint8_t> last_row(final_rung ? chains : 0);
+    if (final_rung)
+        KVP_CUDA(cudaMemcpyAsync(last_row.data(), hist + (size_t)(rounds - 1) * chains, chains, cudaMemcpyDeviceToHost, st));
+    if (n_exchanged) KVP_CUDA(cudaMemcpyAsync(n_exchanged, nex, (size_t)chains * 4, cudaMemcpyDeviceToHost, st));
+    KVP_CUDA(cudaEventRecord(ev[3], st));
+    KVP_CUDA(cudaStreamSynchronize(st));
+    if (final_rung)
+        for (uint32_t i = 0; i < chains; ++i) final_rung[i] = last_row[i];
+    const bool ok = host_small[0] == red.best_ticks && (int32_t)(host_small[2] & 0xFFFFFFFFu) < 0;
+    if (best_ticks) *best_ticks = red.best_ticks;
+    if (best_seconds) *best_seconds = (double)red.best_ticks * p->spt;
+    if (stats) {
+        kvp_chain_result* keep = stats->per_chain;
+        memset(stats, 0, sizeof *stats);
+        stats->per_chain = keep;
+        stats->init_ticks = c.init_ticks; stats->best_ticks = red.best_ticks; stats->best_chain = red.best_chain;
+        stats->levels = a->levels; stats->best_move = red.best_move; stats->moves_total = red.moves_total;
+        stats->calib_mean_delta = c.calib_mean; stats->temp0 = c.temps[0];
+        stats->winner_hits = host_small[1]; stats->winner_accessed = p->total_accessed;
+        cudaEventElapsedTime(&stats->ms_init, ev[0], ev[1]);
+        cudaEventElapsedTime(&stats->ms_chains, ev[1], ev[2]);
+        cudaEventElapsedTime(&stats->ms_finish, ev[2], ev[3]);
+        stats->kernel_launches = c.launches;
+        stats->chain_launches = rounds; stats->resident_chains = chains; stats->wide_kernel = 1u;
+        stats->work_again = work[0]; stats->work_listed = work[1]; stats->work_items = work[2];
+        stats->exchange_rounds = rounds; stats->exchanges_tried = xcounts[0]; stats->exchanges_accepted = xcounts[1];
+    }
+    return ok ? KVP_OK : KVP_ERR_INTERNAL;
 }

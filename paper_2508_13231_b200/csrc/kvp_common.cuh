@@ -9,7 +9,7 @@
 namespace kvp {
 
 // Philox counter tags: word 3 of the counter says what a block of random bits is for.
-constexpr uint32_t TAG_MOVE = 1, TAG_CALIB = 2, TAG_NOISE = 3, TAG_BURST = 4;
+constexpr uint32_t TAG_MOVE = 1, TAG_CALIB = 2, TAG_NOISE = 3, TAG_BURST = 4, TAG_EXCHANGE = 6;   // 5: the (W, R) walk
 constexpr uint32_t CALIB_N = 1024;
 
 // Integer weights of Eq. 3-4, premultiplied with the migration flags.

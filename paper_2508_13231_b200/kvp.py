@@ -24,7 +24,7 @@ EXPORTS = [
     "kvp_create", "kvp_destroy", "kvp_get_info", "kvp_eval", "kvp_eval_counts", "kvp_eval_noalloc", "kvp_accept_table", "kvp_anneal",
     "kvp_anneal_chain_state", "kvp_trace_generate", "kvp_philox4x32_10", "kvp_strerror", "kvp_last_cuda_error",
     "kvp_policy_lookahead", "kvp_policy_reactive", "kvp_policy_page", "kvp_wr_grid", "kvp_wr_anneal", "kvp_set_births",
-    "kvp_set_test_hooks",
+    "kvp_set_test_hooks", "kvp_anneal_exchange", "kvp_exchange_temps",
 ]
 
 
@@ -75,7 +75,13 @@ class AnnealStats(C.Structure):
         ("per_chain", C.POINTER(ChainResult)), ("chain_launches", C.c_uint32), ("resident_chains", C.c_uint32),
         ("wide_kernel", C.c_uint32), ("reserved", C.c_uint32),
         ("work_again", C.c_uint64), ("work_listed", C.c_uint64), ("work_items", C.c_uint64),
+        ("exchanges_tried", C.c_uint64), ("exchanges_accepted", C.c_uint64), ("exchange_rounds", C.c_uint32),
+        ("reserved2", C.c_uint32),
     ]
+
+
+class ExchangeParams(C.Structure):
+    _fields_ = [("rungs", C.c_uint32), ("reserved", C.c_uint32), ("exchange_every", C.c_uint64)]
 
 
 class WRParams(C.Structure):
@@ -308,6 +314,21 @@ class Problem:
                                _stream(stream)), "kvp_anneal")
         return dict(best_schedule=best, best_ticks=int(bt.value), best_seconds=float(bs.value), stats=stats,
                     per_chain=list(per) if per is not None else None)
+
+    def anneal_exchange(self, ap, rungs, every, want_schedule=True, stream=None):
+        """kvp_anneal_exchange -> dict(best_schedule, best_ticks, best_seconds, stats, per_chain, final_rung, n_exchanged)."""
+        best = torch.empty((self.steps, self.w32), dtype=torch.int32, device="cuda") if want_schedule else None
+        bt = C.c_uint64(); bs = C.c_double()
+        stats = AnnealStats()
+        per = (ChainResult * ap.chains)()
+        stats.per_chain = C.cast(per, C.POINTER(ChainResult))
+        final_rung = (C.c_uint32 * ap.chains)()
+        n_ex = (C.c_uint32 * ap.chains)()
+        xp = ExchangeParams(int(rungs), 0, int(every))
+        _chk(_lib().kvp_anneal_exchange(self._h, C.byref(ap), C.byref(xp), _ptr(best), C.byref(bt), C.byref(bs),
+                                        C.byref(stats), final_rung, n_ex, _stream(stream)), "kvp_anneal_exchange")
+        return dict(best_schedule=best, best_ticks=int(bt.value), best_seconds=float(bs.value), stats=stats,
+                    per_chain=list(per), final_rung=list(final_rung), n_exchanged=list(n_ex))
 
     def chain_state(self, ap, chain, upto_moves, stream=None):
         """kvp_anneal_chain_state -> (schedule CUDA int32 [S][W32], ChainResult)."""

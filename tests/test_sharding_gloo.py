@@ -92,3 +92,53 @@ def test_three_ranks_winner_on_the_last_rank():
     for g in got:
         assert (g[5], g[6]) == (ref["best_ticks"], ref["best_chain"])
     assert got[2][3] == ref["best_ticks"] and got[0][3] > ref["best_ticks"] and got[1][3] > ref["best_ticks"]
+
+
+def _xrank(rank, world, port, out):
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    o = _problem("apart")
+    first, count = sharding.ladder_range(rank, world, 20, 4)
+    res = o.anneal_exchange(o.make_params(chains=count, first_chain=first, **XKW), 4, 25)
+    ticks, chain = sharding.combine_best(dist, res["best_ticks"], res["best_chain"])
+    out.put((rank, first, count, [r.astuple() for r in res["per_chain"]], res["final_rung"].tolist(), ticks, chain))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+XKW = dict(moves=1500, levels=4, p0=0.4, alpha=0.5, seed=13)
+
+
+def test_ladder_range_keeps_ladders_whole():
+    for total, rungs in ((20, 4), (8, 8), (36, 3)):
+        for world in (1, 2, 3, 5):
+            parts = [sharding.ladder_range(r, world, total, rungs) for r in range(world)]
+            assert parts[0][0] == 0 and sum(c for _, c in parts) == total
+            assert all(f % rungs == 0 and c % rungs == 0 for f, c in parts)
+            assert all(parts[i][0] + parts[i][1] == parts[i + 1][0] for i in range(world - 1))
+
+
+def test_replica_exchange_split_by_ladders_over_two_ranks():
+    """Five ladders of four replicas over two ranks (three and two ladders): every chain, the rungs held at the end
+    and the agreed winner equal those of one process running all twenty chains."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_xrank, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    o = _problem("apart")
+    ref = o.anneal_exchange(o.make_params(chains=20, **XKW), 4, 25)
+    assert [(g[1], g[2]) for g in got] == [(0, 12), (12, 8)]
+    assert got[0][3] + got[1][3] == [r.astuple() for r in ref["per_chain"]]
+    assert got[0][4] + got[1][4] == ref["final_rung"].tolist()
+    assert ref["n_exchanged"].sum() > 0
+    for g in got:
+        assert (g[5], g[6]) == (ref["best_ticks"], ref["best_chain"])

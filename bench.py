@@ -54,7 +54,8 @@ FLUSH_NOTE = "flushed with a 256 MB write between timed iterations"
 
 
 def _clock_sampler(stop, samples):
-    """SM clock and throttle reasons of this rank's GPU through NVML, every 20 ms while the timed region runs."""
+    """SM clock and throttle reasons of this rank's GPU through NVML, every 100 ms while the timed region runs
+    (a shorter period makes the NVML queries contend with the step's own driver calls and shows up in the step time)."""
     try:
         import pynvml
         pynvml.nvmlInit()
@@ -77,7 +78,7 @@ def _clock_sampler(stop, samples):
             samples.append((float(sm), float(smax), [n for b, n in bits.items() if r & b]))
         except Exception:
             pass
-        stop.wait(0.02)
+        stop.wait(0.1)
 
 
 def _clock_summary(samples):

@@ -57,7 +57,7 @@ struct ChainParams {
     uint32_t touch_cap;
     uint32_t restore;            // the slices hold the final states of chains that started from the same initial
                                  // schedule and logged what they touched: only those units are copied again
-    uint32_t* cow_out;           // wide kernel, schedules in global scratch: [slots][kCowBits / 32] which buckets of
+    uint32_t* cow_out;           // wide kernel, schedules in global scratch: [slots][cow_slots4 * 4] which buckets of
                                  // units a slot's slice holds when its chain ends (the rest is the initial schedule)
     uint32_t cow_shift;          // a bucket is 2^cow_shift consecutive units
     uint32_t stage_stepc;        // wide kernel without a staged access bitmap: the step constants alone are staged
@@ -72,6 +72,7 @@ struct ChainParams {
                                  // schedule, when that lives in shared memory), indexed like rung_hist
     uint32_t state4;             // uint4 slots per chain in `state`
     uint32_t resume;             // 1: start from `state` instead of the initial schedule
+    uint32_t cow_slots4;         // wide kernel, schedules in global scratch: uint4 slots of a chain's bucket bitmap
 };
 
 // Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
@@ -922,19 +923,21 @@ __device__ __noinline__ void copy_words_cold(uint32_t* dst, const uint32_t* src,
 
 // Schedules in global scratch are copy-on-write overlays of the one initial schedule that all chains share: the
 // units come in buckets of 2^shift consecutive units, a chain's slice holds a bucket only once the chain has
-// rewritten a unit of it, and a bitmap in shared memory (at most kCowBits buckets) says which. Chains change few of
-// their units, so nearly every placement window is read from the shared initial schedule, which stays in L2, and
-// not from a private slice that only DRAM can hold; a chain that rewrites everything ends up copying its whole
-// slice once, bucket by bucket.
-constexpr uint32_t kCowBits = 8192;
-constexpr uint32_t kCowSlots4 = kCowBits / 128;
+// rewritten a unit of it, and a bitmap in shared memory says which. Chains change few of their units, so nearly
+// every placement window is read from the shared initial schedule, which stays in L2, and not from a private slice
+// that only DRAM can hold; a chain that rewrites everything ends up copying its whole slice once, bucket by bucket.
+// The bitmap takes the shared memory that a full CTA of chains leaves free (kCowBitsMin to kCowBitsMax buckets): a
+// chain of a million moves rewrites thousands of units, and every read of a bucket it owns misses L2, so the buckets
+// should be small (with 8192 buckets of 512 units a chain of the largest configuration owned two thirds of them at
+// its end; with 40,960 of 64 units it owns an eighth).
+constexpr uint32_t kCowBitsMin = 8192, kCowBitsMax = 65536;
 
 // Where a chain of the wide kernel keeps its state. CT: the four per-step cardinalities as 16-bit fields when the
 // schedule lives in shared memory (then units < 2^16), as 32-bit fields otherwise. COW: see above.
 template <typename CT, bool COW, int COLV>
 struct WideView {
     const uint32_t* p0;          // COW: [U][S32] the initial schedule
-    uint32_t* have;              // COW: [kCowBits / 32] buckets present in P (shared)
+    uint32_t* have;              // COW: [cow_slots4 * 4] buckets present in P (shared)
     uint32_t shift, U, S32;      // COW: bucket size; units; words per unit
     __device__ __forceinline__ const uint32_t* col(uint32_t u) const
     {
@@ -973,7 +976,8 @@ struct WideScalars {
     uint64_t cur, best, best_move, best_at_boundary, n_chg, hash;
     uint32_t ulen;               // moves applied since the best state
     uint32_t snap_dirty;         // the best state is the current one and not saved yet
-    uint32_t pad[2];
+    uint32_t qn;                 // items reserved in the work queue during a pass (0 between passes)
+    uint32_t pad;
     // what the chain's evaluations amounted to (kvp_anneal_stats): proposals evaluated again after an applied move,
     // proposals that needed a cost evaluation, (proposal, step) items
     uint64_t n_again, n_listed, n_items;
@@ -983,17 +987,18 @@ struct WideScalars {
 constexpr uint32_t kWideScalars4 = sizeof(WideScalars) / 16;
 
 // the part of wide_fixed4 that outlives a batch (what a replica-exchange run saves between its rounds)
-__host__ __device__ inline uint32_t wide_persist4(uint32_t S, uint32_t S32, bool grow, bool shared)
+// cow4: uint4 slots of the bucket bitmap (schedules in global scratch)
+__host__ __device__ inline uint32_t wide_persist4(uint32_t S, uint32_t S32, bool grow, bool shared, uint32_t cow4)
 {
-    return (shared ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (S + 3) / 4 + (shared ? 0u : kCowSlots4) +
+    return (shared ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (S + 3) / 4 + (shared ? 0u : cow4) +
            kWideScalars4;
 }
 
 // shared-memory words (as uint4 slots) of one chain of the wide kernel besides its schedule
-__host__ __device__ inline uint32_t wide_fixed4(uint32_t S, uint32_t S32, bool grow, bool shared)
+__host__ __device__ inline uint32_t wide_fixed4(uint32_t S, uint32_t S32, bool grow, bool shared, uint32_t cow4)
 {
     return (shared ? (S + 1) / 2 : S) + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (S + 3) / 4 +
-           (shared ? 0u : kCowSlots4) + kWideScalars4 +
+           (shared ? 0u : cow4) + kWideScalars4 +
            2 * kWide + kWide / 4 + kWide / 16 + kWideQueueSlots4;
 }
 
@@ -1153,7 +1158,6 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW, COLV> cv, 
                                               uint32_t shift, uint32_t need, bool fresh, uint32_t lane, WideMoves& mv,
                                               WideScalars* sc)
 {
-    const uint32_t below = (1u << lane) - 1u;
     // 1. placement bits only; the proposals that need more are listed
     uint32_t listed = 0;                                          // proposals listed (warp-uniform)
     uint32_t mine = 0;                                            // bit h: this lane's row h is listed
@@ -1178,23 +1182,21 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW, COLV> cv, 
             cv.win[id * 2] = make_uint4(wn.Wu, wn.Wv, wn.Nu, wn.Nv);
             cv.win[id * 2 + 1] = make_uint4(wn.Au, wn.Av, wn.s0, wn.born);
         }
+        // every lane reserves room for its items in the queue (the order of the items does not matter)
         const uint32_t cnt = __popc(todo);
-        uint32_t pos = 0, total = 0;
-#pragma unroll
-        for (int bit = 0; bit < 5; ++bit) {
-            const uint32_t has = __ballot_sync(0xFFFFFFFFu, (cnt >> bit) & 1u);
-            pos += __popc(has & below) << bit;
-            total += __popc(has) << bit;
-        }
+        uint32_t pos = cnt ? atomicAdd(&sc->qn, cnt) : 0u;
+        __syncwarp();
+        const uint32_t total = sc->qn;
+        __syncwarp();
         if (total) {
-            if (lane == 0) sc->n_items += total;
+            if (lane == 0) { sc->n_items += total; sc->qn = 0u; }
             if (COW) {
-                // many chains per SM, issue slots scarce: one set bit per lane and trip
-                for (uint32_t td = todo; __any_sync(0xFFFFFFFFu, td != 0u);) {
-                    if (td) {
-                        cv.queue[pos++] = (uint16_t)((id << 5) | (__ffs(td) - 1u));
-                        td &= td - 1u;
-                    }
+                // many chains per SM, issue slots scarce: every lane peels its own set bits, highest first (the order
+                // of the items in the queue does not matter: their cost changes are summed)
+                for (uint32_t td = todo; td != 0u;) {
+                    const uint32_t k = 31u - __clz(td);
+                    cv.queue[pos++] = (uint16_t)((id << 5) | k);
+                    td ^= 1u << k;
                 }
             } else {
                 // few chains per SM, latency scarce: all 31 positions tried, no lane waits on a serial bit scan
@@ -1301,7 +1303,7 @@ __device__ __forceinline__ void copy_merged(uint32_t* __restrict__ dst, const ui
 }
 
 // PSMEM: the schedule lives in shared memory (16-bit counters); otherwise the chain's slice of global scratch is a
-// copy-on-write overlay of the initial schedule (see kCowBits).
+// copy-on-write overlay of the initial schedule (see kCowBitsMin).
 // ASMEM (only with PSMEM): access bitmap and step constants staged in shared memory once per CTA.
 // COLV (only without PSMEM): 2 or 4 when every column has exactly that many words, else 0 (see window_at).
 template <bool PSMEM, bool GROW, bool ASMEM, int COLV>
@@ -1322,8 +1324,8 @@ wide_chain_kernel(const ChainParams prm)
     const size_t pwords = (size_t)U * S32;
     const uint32_t c4 = PSMEM ? (S + 1) / 2 : S;                  // uint4 slots of the counters
     const uint32_t f4 = (S32 + 3) / 4, h4 = GROW ? (S + 3) / 4 : 0u;
-    constexpr uint32_t o4 = COW ? kCowSlots4 : 0u;
-    const uint32_t fixed4 = wide_fixed4(S, S32, GROW, PSMEM);
+    const uint32_t o4 = COW ? prm.cow_slots4 : 0u;
+    const uint32_t fixed4 = wide_fixed4(S, S32, GROW, PSMEM, o4);
     uint4* const mine4 = smem4 + (size_t)cic * fixed4;
     WideView<CT, COW, COLV> cv;
     cv.ctr = reinterpret_cast<CT*>(mine4);
@@ -1367,11 +1369,11 @@ wide_chain_kernel(const ChainParams prm)
         for (uint32_t i = lane; i < S32; i += 32) cv.full[i] = __ldg(prm.full0 + i);
         if (lane == 0) {
             sc->cur = sc->best = sc->best_at_boundary = prm.init_ticks;
-            sc->best_move = ~0ull; sc->n_chg = 0; sc->hash = 0; sc->ulen = 0u; sc->snap_dirty = 0u;
+            sc->best_move = ~0ull; sc->n_chg = 0; sc->hash = 0; sc->ulen = 0u; sc->snap_dirty = 0u; sc->qn = 0u;
             sc->n_again = sc->n_listed = sc->n_items = 0; sc->n_acc = sc->n_inf = 0;
         }
         if (COW) {
-            for (uint32_t i = lane; i < kCowBits / 32; i += 32) cv.have[i] = 0u;   // the slice holds nothing yet
+            for (uint32_t i = lane; i < prm.cow_slots4 * 4; i += 32) cv.have[i] = 0u;   // the slice holds nothing yet
         } else if (!(prm.state && prm.resume)) {
             copy_words_cold(cv.P, prm.Pcol0, pwords, lane);
         }
@@ -1532,7 +1534,8 @@ wide_chain_kernel(const ChainParams prm)
     if (snap && sc->snap_dirty) copy_words_cold(snap, cv.P, pwords, lane);
     if (ulog && lane == 0) prm.undo_len[slot] = sc->ulen;
     if (COW && prm.cow_out)                                       // which buckets the slice holds (for the walk back)
-        for (uint32_t i = lane; i < kCowBits / 32; i += 32) prm.cow_out[(size_t)slot * (kCowBits / 32) + i] = cv.have[i];
+        for (uint32_t i = lane; i < prm.cow_slots4 * 4; i += 32)
+            prm.cow_out[(size_t)slot * (prm.cow_slots4 * 4) + i] = cv.have[i];
     if (lane == 0) {
         kvp_chain_result res;
         res.best_ticks = sc->best; res.best_move = sc->best_move; res.final_ticks = sc->cur; res.moves_done = m_end;
@@ -1774,6 +1777,7 @@ struct Ctx {
     bool touch;              // the chains come in several waves and log the units they rewrite
     uint32_t* cow_out;       // wide kernel, global variant: bucket bitmaps of the slices, or null
     uint32_t cow_shift;
+    uint32_t cow_slots4;     // uint4 slots of a chain's bucket bitmap
     bool psmem;
     uint32_t wpb;            // chains per CTA
     uint32_t wpc;            // warps per chain
@@ -1849,7 +1853,8 @@ int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp
     prm.undo_log = with_undo ? c.undo_log : nullptr; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
     prm.touch_log = with_undo ? c.touch_log : nullptr; prm.touch_len = c.touch_len; prm.touch_cap = c.touch_cap;
     prm.restore = with_undo && restore && c.touch_log ? 1u : 0u;
-    prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift; prm.stage_stepc = c.stage_stepc ? 1u : 0u;
+    prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift; prm.cow_slots4 = c.cow_slots4;
+    prm.stage_stepc = c.stage_stepc ? 1u : 0u;
     prm.chain_first = first; prm.chain_count = count; prm.result_base = result_base;
     prm.results = results; prm.upto = upto; prm.dump = dump;
     ++c.launches;
@@ -1883,11 +1888,13 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
     c.wide = exchange || hooks.warps_per_chain == 3 || (hooks.warps_per_chain == 0 && (a->chains + sms - 1) / sms > 8);
     // `shared`: the schedule is in shared memory (the wide kernel then keeps 16-bit counters)
     auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false, bool shared = true) {
-        if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared) * 16;
+        if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared, shared ? 0u : c.cow_slots4) * 16;
         return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq, touch) * 16;
     };
     c.touch = false;
     c.stage_stepc = false;
+    c.cow_slots4 = kCowBitsMin / 128;
+    c.cow_shift = 0;
     const size_t pbytes = (size_t)p->U * p->S32 * 4;
     // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
     // chains then keeps twice as many warps in flight. kvp_set_test_hooks can override the choice (tests, tuning).
@@ -1928,6 +1935,21 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
         // more shared-memory slot per chain)
         for (int pass = 0; pass < 2; ++pass) {
             c.touch = pass == 1;
+            if (c.wide) {
+                // The bucket bitmap of the copy-on-write slices takes what a full CTA of chains leaves of the shared
+                // memory: the smaller the buckets, the fewer reads of a long chain go to its private slice.
+                c.cow_slots4 = 0;
+                const size_t bare = fixed_bytes(W, false, false, false);
+                const size_t stepc_bytes = (size_t)p->S * 16 <= 32768 ? (size_t)p->S * 16 : 0;
+                const size_t share = (budget - stepc_bytes) / (kWideGlobalThreads / 32);
+                size_t bits = share > bare ? (share - bare) / 16 * 128 : 0;
+                if (bits < kCowBitsMin) bits = kCowBitsMin;
+                if (bits > kCowBitsMax) bits = kCowBitsMax;
+                c.cow_shift = 0;
+                while (((uint64_t)p->U + (1ull << c.cow_shift) - 1) >> c.cow_shift > bits) ++c.cow_shift;
+                const uint64_t buckets = ((uint64_t)p->U + (1ull << c.cow_shift) - 1) >> c.cow_shift;
+                c.cow_slots4 = (uint32_t)((buckets + 127) / 128);
+            }
             const size_t ctr_bytes = fixed_bytes(W, false, c.touch, false);
             if (ctr_bytes > budget) return KVP_ERR_RANGE;
             c.smem_per_warp = ctr_bytes;
@@ -1974,8 +1996,6 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
             if (a->chains <= c.resident || c.wide) break;
         }
     }
-    c.cow_shift = 0;
-    while (((uint64_t)p->U + (1ull << c.cow_shift) - 1) >> c.cow_shift > kCowBits) ++c.cow_shift;
     // a replica-exchange run keeps every chain's slice between its rounds: all chains have to be resident at once
     if (exchange && !c.psmem && a->chains > c.resident) return KVP_ERR_RANGE;
 
@@ -2004,7 +2024,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
     c.touch_cap = touch ? 16384u : 0u;
     const size_t o_tlog = take((size_t)c.resident * c.touch_cap * 4), o_tlen = take(touch ? (size_t)c.resident * 4 : 0);
     const bool cow = c.wide && !c.psmem;
-    const size_t o_cow = take(cow ? (size_t)c.resident * (kCowBits / 8) : 0);
+    const size_t o_cow = take(cow ? (size_t)c.resident * c.cow_slots4 * 16 : 0);
     rc = ensure_chain_ws(p, off, st);
     if (rc) return rc;
     char* base = static_cast<char*>(p->d_chain_ws);
@@ -2174,13 +2194,13 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
                     ChainParams prm = c.prm;
                     prm.chain_first = a->first_chain + first;
                     prm.undo_log = c.undo_log; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
-                    prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift;
+                    prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift; prm.cow_slots4 = c.cow_slots4;
                     const uint32_t wslot = red.best_chain - first;
                     if (c.grow) undo_kernel<true><<<1, 32, 0, st>>>(prm, wslot);
                     else undo_kernel<false><<<1, 32, 0, st>>>(prm, wslot);
                     KVP_CUDA(cudaGetLastError());
                     gather_slice_kernel<<<148 * 4, 256, 0, st>>>(c.dumpcol, c.slots + (size_t)wslot * p->U * p->S32, c.Pcol0,
-                                                                 c.cow_out ? c.cow_out + (size_t)wslot * (kCowBits / 32) : nullptr,
+                                                                 c.cow_out ? c.cow_out + (size_t)wslot * (c.cow_slots4 * 4) : nullptr,
                                                                  c.cow_shift, p->U, p->S32);
                     KVP_CUDA(cudaGetLastError());
                     c.launches += 2;
@@ -2327,7 +2347,7 @@ extern "C" int kvp_anneal_exchange(kvp_problem* p, const kvp_anneal_params* a, c
     if ((rc = kvp_accept_table(pair_temps.data(), pairs, xtable.data(), xshifts.data()))) return rc;
 
     // workspace of the run: rung history, holders, exchange counts, thresholds, the chains' saved states
-    const uint32_t persist4 = wide_persist4(p->S, p->S32, c.grow, c.psmem);
+    const uint32_t persist4 = wide_persist4(p->S, p->S32, c.grow, c.psmem, c.cow_slots4);
     const size_t pwords = (size_t)p->U * p->S32;
     const uint32_t state4 = persist4 + (c.psmem ? (uint32_t)((pwords + 3) / 4) : 0u);
     size_t off = 0;
@@ -2356,7 +2376,8 @@ extern "C" int kvp_anneal_exchange(kvp_problem* p, const kvp_anneal_params* a, c
 
     ChainParams prm = c.prm;
     prm.snap = c.snap; prm.undo_log = nullptr; prm.touch_log = nullptr; prm.restore = 0u;
-    prm.cow_out = nullptr; prm.cow_shift = c.cow_shift; prm.stage_stepc = c.stage_stepc ? 1u : 0u;
+    prm.cow_out = nullptr; prm.cow_shift = c.cow_shift; prm.cow_slots4 = c.cow_slots4;
+    prm.stage_stepc = c.stage_stepc ? 1u : 0u;
     prm.chain_first = a->first_chain; prm.chain_count = chains; prm.result_base = a->first_chain;
     prm.results = c.results; prm.upto = a->moves; prm.dump = nullptr;
     prm.rung_hist = hist; prm.exch_every = xp->exchange_every; prm.hist_stride = chains; prm.hist_base = a->first_chain;

@@ -279,9 +279,11 @@ __device__ __forceinline__ uint32_t item_cost_after(const Windows& wn, uint32_t 
 
 __device__ __forceinline__ bool metropolis(int delta, uint32_t w, const uint32_t* __restrict__ trow, uint32_t shift)
 {
-    if (delta <= 0) return true;
-    const uint32_t q = (uint32_t)delta >> shift;
-    return q < KVP_TABLE_Q && w < __ldg(trow + q);                // quantised exp(-delta/C)
+    // branch-free: the threshold is loaded whatever delta is (a clamped index), so that the loads of several
+    // proposals are in flight together instead of each behind its own branch
+    const uint32_t q = (uint32_t)max(delta, 0) >> shift;
+    const uint32_t thr = __ldg(trow + min(q, (uint32_t)KVP_TABLE_Q - 1u));
+    return delta <= 0 || (q < KVP_TABLE_Q && w < thr);            // quantised exp(-delta/C)
 }
 
 // Whole evaluation in one lane (used where there is no warp to share the work with: calibration).
@@ -1137,12 +1139,16 @@ __device__ __forceinline__ void wide_classify(const WideView<CT, COW, COLV> cv, 
         }
         const bool more = named && chg && !inf;
         const uint32_t mb = __ballot_sync(0xFFFFFFFFu, more);
-        if (more) {
-            const uint32_t id = h * 32 + lane;
-            cv.nt[listed + __popc(mb & below)] = (uint8_t)id;
+        const uint32_t id = h * 32 + lane;
+        // the slot of a proposal that is not listed is not looked at again, so a fresh batch parks every row's
+        // windows without a test
+        if (ALL || more) {
             cv.win[id * 2] = make_uint4(pk, mv.u[h], mv.v[h], Wu[h]);
             cv.win[id * 2 + 1].x = Wv[h];
             cv.acc[id] = 0;
+        }
+        if (more) {
+            cv.nt[listed + __popc(mb & below)] = (uint8_t)id;
             mine |= 1u << h;
         }
         listed += __popc(mb);
@@ -1215,15 +1221,28 @@ __device__ __forceinline__ void wide_evaluate(const WideView<CT, COW, COLV> cv, 
         }
         __syncwarp();
     }
-    // 3. the owners take the sums and decide
+    // 3. the owners take the sums and decide. Straight-line over the rows (the sums and the thresholds of all rows
+    //    are loaded before any is used); a row that is not listed reads a stale sum and drops the outcome.
+    int d[kRows];
+    uint32_t thr[kRows];
 #pragma unroll
-    for (int h = 0; h < kRows; ++h)
-        if ((mine >> h) & 1u) {
-            const int d = cv.acc[h * 32 + lane];
-            mv.delta[h] = d;
-            const uint32_t bit = 1u << h;
-            mv.acc = metropolis(d, mv.w[h], trow, shift) ? mv.acc | bit : mv.acc & ~bit;
+    for (int h = 0; h < kRows; ++h) d[h] = cv.acc[h * 32 + lane];
+#pragma unroll
+    for (int h = 0; h < kRows; ++h) {
+        const uint32_t q = (uint32_t)max(d[h], 0) >> shift;
+        thr[h] = __ldg(trow + min(q, (uint32_t)KVP_TABLE_Q - 1u));
+        if (q >= KVP_TABLE_Q) thr[h] = 0u;                        // beyond the table: never accepted
+    }
+#pragma unroll
+    for (int h = 0; h < kRows; ++h) {
+        const bool lst = (mine >> h) & 1u;
+        const bool ok = d[h] <= 0 || mv.w[h] < thr[h];            // quantised exp(-delta/C), as in metropolis()
+        const uint32_t bit = 1u << h;
+        if (lst) {
+            mv.delta[h] = d[h];
+            mv.acc = ok ? mv.acc | bit : mv.acc & ~bit;
         }
+    }
 }
 
 // Apply the proposal whose windows are in slot `id` (pk, u, v given): all lanes take part, lane j updates the
@@ -1882,10 +1901,18 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
     const kvp_test_hooks hooks = g_hooks;
     c.S32 = p->S32;
     // Which kernel. Many chains per SM (more than 8, the jobs that fill the registers of an SM with one warp per
-    // chain): the wide kernel, which needs half the instructions per proposal. Few chains per SM: the narrow kernel
-    // with two warps per chain, which hides the latency of a chain's serial parts behind its second warp.
+    // chain; more than 5 when the schedules fit shared memory): the wide kernel, which needs half the instructions
+    // per proposal. Fewer chains per SM: the narrow kernel with two warps per chain, which hides the latency of a
+    // chain's serial parts behind its second warp. A hot start (C_0 from p0 >= 0.5: a fifth of the proposals change
+    // the schedule and the chain is a sequence of applied moves) on few chains: the narrow kernel with one warp per
+    // chain, whose path through an applied move is the shortest.
     // kvp_set_test_hooks can force either (warps_per_chain 1 or 2: narrow; 3: wide).
-    c.wide = exchange || hooks.warps_per_chain == 3 || (hooks.warps_per_chain == 0 && (a->chains + sms - 1) / sms > 8);
+    const uint32_t chains_per_sm = (a->chains + sms - 1) / sms;
+    const size_t pbytes = (size_t)p->U * p->S32 * 4;
+    const bool hot = !a->temps && a->p0 >= 0.5;
+    const bool wide_in_smem = p->U < 65536u && (size_t)wide_fixed4(p->S, p->S32, c.grow, true, 0u) * 16 + pbytes <= budget / 2;
+    c.wide = exchange || hooks.warps_per_chain == 3 ||
+             (hooks.warps_per_chain == 0 && (chains_per_sm > 8 || (wide_in_smem && chains_per_sm > 5 && !hot)));
     // `shared`: the schedule is in shared memory (the wide kernel then keeps 16-bit counters)
     auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false, bool shared = true) {
         if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared, shared ? 0u : c.cow_slots4) * 16;
@@ -1895,11 +1922,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
     c.stage_stepc = false;
     c.cow_slots4 = kCowBitsMin / 128;
     c.cow_shift = 0;
-    const size_t pbytes = (size_t)p->U * p->S32 * 4;
     // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
     // chains then keeps twice as many warps in flight. kvp_set_test_hooks can override the choice (tests, tuning).
-    const uint32_t chains_per_sm = (a->chains + sms - 1) / sms;
-    uint32_t W = chains_per_sm <= 8 ? 2u : 1u;
+    uint32_t W = chains_per_sm <= 8 && !hot ? 2u : 1u;
     if (hooks.warps_per_chain == 1 || hooks.warps_per_chain == 2) W = hooks.warps_per_chain;
     if (c.wide) W = 1;
     c.psmem = fixed_bytes(1) + pbytes <= budget / 2 && (!c.wide || p->U < 65536u);

@@ -43,12 +43,12 @@ ALG_WARP_INSTR_PER_MOVE = 16.0          # the narrow chain kernel: every proposa
 #                            decoding of swap / run length / first step / two units 18, its share of the commit vote 2
 #   per evaluation    1.65 : unpacking 4, run mask 5, window position 5, two placement columns (overlay lookup, address,
 #                            load, funnel shift) 22, toggled bits, Eq. 5 test, verdict bits 13, listing 4
-#   per listed one    1.75 : slot 2, two access columns 10, windows after the move 6, the steps whose cardinalities
-#                            change 18, window store 2, queue offsets 12, sum and Metropolis test 6
+#   per listed one    1.47 : slot 2, two access columns 10, windows after the move 6, the steps whose cardinalities
+#                            change 18, window store 2, room in the queue 3, sum and Metropolis test 6
 #   per (proposal, step) item 1.45 : queue 3, windows, counters, constants, present cost 5 loads, bit extraction 10,
 #                            new cardinalities 12, Eq. 2-4 once 13, difference and accumulation 3
 # evaluations = moves + proposals evaluated again after an applied move.
-ALG_WIDE = {"move": 2.06, "evaluation": 1.65, "listed": 1.75, "item": 1.45}
+ALG_WIDE = {"move": 2.06, "evaluation": 1.65, "listed": 1.47, "item": 1.45}
 PEAK_SOURCE_ALU = "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"
 FLUSH_NOTE = "flushed with a 256 MB write between timed iterations"
 

@@ -50,6 +50,12 @@ ALG_WARP_INSTR_PER_MOVE = 16.0          # the narrow chain kernel: every proposa
 # evaluations = moves + proposals evaluated again after an applied move.
 ALG_WIDE = {"move": 2.06, "evaluation": 1.65, "listed": 1.47, "item": 1.45}
 PEAK_SOURCE_ALU = "148 SMs x 4 issue slots x 1.965 GHz (unit counts and clocks)"
+# DRAM bytes (read + written) of one chain-kernel launch, from a one-pass profiler capture of the very launches this
+# benchmark times (2048 chains x 1,000,000 moves of long_70b); not measured in the run that prints it, and labelled so.
+# To be taken again whenever the chain kernel or the copy-on-write layout changes.
+PROFILED_DRAM_BYTES_PER_LAUNCH = {("long_70b", 2048, 1_000_000): 15.68e9}
+PROFILED_NOTE = ("dram__bytes_read.sum + dram__bytes_write.sum of one launch (13.26 + 2.42 GB), one-pass ncu capture of "
+                 "the benchmark command; a profile figure, not measured in this run")
 FLUSH_NOTE = "flushed with a 256 MB write between timed iterations"
 
 
@@ -567,10 +573,13 @@ class PathBench:
         if st.wide_kernel:   # the same time against the work of the full-evaluation formulation, for comparison only
             form["frac_against_16_per_move"] = (ALG_WARP_INSTR_PER_MOVE * moves_per_launch / (per_launch_ms * 1e-3) / 1e9 /
                                                 ISSUE_PEAK_GWIPS)
+        traffic = PROFILED_DRAM_BYTES_PER_LAUNCH.get((self.name, int(st.resident_chains), int(self.moves))) if st.wide_kernel else None
+        if traffic is not None:
+            form["traffic_source"] = PROFILED_NOTE
         return {"bound": "alu", "kernel": "chain kernel (%s)" % ("schedules in shared memory" if self.U * self.S <= (1 << 18)
                                                                   else "schedules in global memory"),
                 "achieved": achieved, "peak": ISSUE_PEAK_GWIPS, "unit": "Gwarp-inst/s", "frac": achieved / ISSUE_PEAK_GWIPS,
-                "traffic": None, "ms_per_launch": per_launch_ms, "launches_per_step": chain_launches / max(1, n_steps),
+                "traffic": traffic, "ms_per_launch": per_launch_ms, "launches_per_step": chain_launches / max(1, n_steps),
                 "chains_per_launch": int(st.resident_chains), "algorithmic_warp_instr_per_move": alg,
                 "peak_source": PEAK_SOURCE_ALU, **form}
 

@@ -52,11 +52,6 @@ struct ChainParams {
     uint32_t early_permille, early_from;
     PhiloxKeys keys;             // round keys of the seed
     uint64_t per_level, upto, init_ticks;
-    uint32_t* touch_log;         // if set: [slots][touch_cap] units whose schedule words the slot's chain has rewritten
-    uint32_t* touch_len;         // [slots] how many entries (more than touch_cap: the log overflowed)
-    uint32_t touch_cap;
-    uint32_t restore;            // the slices hold the final states of chains that started from the same initial
-                                 // schedule and logged what they touched: only those units are copied again
     uint32_t* cow_out;           // wide kernel, schedules in global scratch: [slots][cow_slots4 * 4] which buckets of
                                  // units a slot's slice holds when its chain ends (the rest is the initial schedule)
     uint32_t cow_shift;          // a bucket is 2^cow_shift consecutive units
@@ -72,7 +67,8 @@ struct ChainParams {
                                  // schedule, when that lives in shared memory), indexed like rung_hist
     uint32_t state4;             // uint4 slots per chain in `state`
     uint32_t resume;             // 1: start from `state` instead of the initial schedule
-    uint32_t cow_slots4;         // wide kernel, schedules in global scratch: uint4 slots of a chain's bucket bitmap
+    uint32_t cow_slots4;         // schedules in global scratch: uint4 slots of a chain's bucket bitmap; 0 (narrow kernel
+                                 // only): plain slices, each a whole copy of the initial schedule
 };
 
 // Batches: every lane of a chain's warp carries kMPL proposals, so a batch is 32 * kMPL consecutive moves.
@@ -162,7 +158,40 @@ __device__ __forceinline__ uint32_t window_at(Ptr col, const WinPos p)
 }
 
 struct ChainView {               // where a chain's state lives
-    uint32_t* P;                 // [U][S32] schedule, time-packed (shared or global)
+    uint32_t* P;                 // [U][S32] schedule, time-packed (shared, or the chain's slice of global scratch)
+    // COW (a compile-time choice of the kernel): the slice of global scratch is a copy-on-write overlay of the initial
+    // schedule p0 (see kCowBitsMin) and `have` says which buckets of 2^shift units it holds. Otherwise the schedule is
+    // all in P.
+    const uint32_t* p0;
+    uint32_t* have;
+    uint32_t shift, U, S32;
+    bool shared_chain;           // a second warp of the chain reads while this one commits
+    template <bool COW>
+    __device__ __forceinline__ const uint32_t* col(uint32_t u) const
+    {
+        if (COW) {
+            const uint32_t b = u >> shift;
+            // volatile: another warp of the chain may be taking the bucket over meanwhile (it sets the bit after the
+            // copy); a select, not a branch, so that the loads of a batch stay in one straight-line block
+            const uint32_t w = reinterpret_cast<const volatile uint32_t*>(have)[b >> 5];
+            return ((w >> (b & 31u)) & 1u ? P : p0) + (size_t)u * S32;
+        }
+        return P + (size_t)u * S32;
+    }
+    // Before unit u is rewritten (all lanes of the committing warp, u uniform): its bucket is copied into the slice.
+    template <bool COW>
+    __device__ __forceinline__ void own(uint32_t u, uint32_t lane) const
+    {
+        if (!COW) return;
+        const uint32_t b = u >> shift;
+        if ((have[b >> 5] >> (b & 31u)) & 1u) return;
+        const size_t lo = (size_t)(b << shift) * S32, hi = (size_t)min(U, (b + 1u) << shift) * S32;
+        for (size_t i = lo + lane; i < hi; i += 32) P[i] = p0[i];
+        if (shared_chain) __threadfence_block();                  // the copy before the bit, for the chain's other warp
+        __syncwarp();
+        if (lane == 0) have[b >> 5] |= 1u << (b & 31u);
+        __syncwarp();
+    }
     uint4* ctr;                  // [S] {hr, mi, mo, occ} (shared)
     uint32_t* full;              // [S32] bit t set iff occ[t] == cap (shared)
     uint4* win;                  // [kBatch][2] windows of the batch's proposals (shared)
@@ -188,8 +217,9 @@ __device__ __forceinline__ void alive_born(uint32_t b, uint32_t s0, uint32_t& al
 // of window bits (steps) whose cardinalities, hence cost, change.
 // GROW: a move acts only on the steps at which the units it names exist, and a unit that enters HBM in the step
 // it is written was written there (it counts in hb), not migrated.
+// colu, colv: the time-packed placement columns of unit u and of unit v (of u again for a flip).
 template <bool GROW, typename PPtr, typename FPtr>
-__device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restrict__ Acol, FPtr full,
+__device__ __forceinline__ uint32_t lane_windows(PPtr colu, PPtr colv, const uint32_t* __restrict__ Acol, FPtr full,
                                                  const uint32_t* __restrict__ birth, uint32_t S, uint32_t S32,
                                                  LaneMove& mv, Windows& wn)
 {
@@ -201,8 +231,8 @@ __device__ __forceinline__ uint32_t lane_windows(PPtr P, const uint32_t* __restr
     const uint32_t Sb = ((1u << nl) - 1u) << 1;
     // branch-free: a flip reads unit u twice and ignores the second copy, a swap ignores the full-step window
     const size_t ub = (size_t)mv.u * S32, vb = (size_t)(swap ? mv.v : mv.u) * S32;
-    const uint32_t Wu = window(P + ub, S32, s0), Au = window(Acol + ub, S32, s0);
-    const uint32_t wv = window(P + vb, S32, s0), av = window(Acol + vb, S32, s0);
+    const uint32_t Wu = window(colu, S32, s0), Au = window(Acol + ub, S32, s0);
+    const uint32_t wv = window(colv, S32, s0), av = window(Acol + vb, S32, s0);
     const uint32_t Wv = swap ? wv : 0u, Av = swap ? av : 0u;
     const uint32_t Fw = window(full, S32, s0);
     uint32_t Bu = 0u, Bv = 0u, live = 0xFFFFFFFFu;
@@ -294,7 +324,8 @@ __device__ __forceinline__ void eval_lane(PPtr P, const uint32_t* __restrict__ A
                                           const uint32_t* __restrict__ trow, uint32_t shift, LaneMove& mv)
 {
     Windows wn;
-    uint32_t todo = lane_windows<GROW>(P, Acol, full, birth, S, S32, mv, wn);
+    uint32_t todo = lane_windows<GROW>(P + (size_t)mv.u * S32, P + (size_t)((mv.pk & 1u) ? mv.v : mv.u) * S32, Acol, full, birth, S,
+                                       S32, mv, wn);
     int delta = 0;
     while (todo) {
         const uint32_t k = __ffs(todo) - 1;
@@ -342,7 +373,7 @@ __device__ __forceinline__ void eval_items(const ChainView cv, const StepC* __re
 // ALL: every lane prepares its proposal whether `need` names it or not (its items are dropped if not), so that this
 // part is straight-line code; `side_work` is then scheduled into it by the compiler (the draw of the next batch: a
 // long chain of dependent integer operations that fills the issue slots the window loads leave empty).
-template <bool GROW, bool ASMEM, bool ALL, typename SideWork>
+template <bool GROW, bool ASMEM, bool ALL, bool COW, typename SideWork>
 __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* __restrict__ Acol,
                                            const uint32_t* __restrict__ birth,
                                            const StepC* __restrict__ stepc, const CostK K, uint32_t S, uint32_t S32,
@@ -358,7 +389,8 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
         if (ALL || named) {
             const uint32_t slot = h * 32 + lane;
             Windows wn;
-            const uint32_t tm = lane_windows<GROW>(cv.P, Acol, cv.full, birth, S, S32, mv[h], wn);
+            const uint32_t tm = lane_windows<GROW>(cv.col<COW>(mv[h].u), cv.col<COW>((mv[h].pk & 1u) ? mv[h].v : mv[h].u), Acol, cv.full,
+                                                   birth, S, S32, mv[h], wn);
             todo[h] = named ? tm : 0u;
             cv.win[slot * 2] = make_uint4(wn.Wu, wn.Wv, wn.Nu, wn.Nv);
             cv.win[slot * 2 + 1] = make_uint4(wn.Au, wn.Av, wn.s0, wn.born);
@@ -424,7 +456,7 @@ __device__ __forceinline__ void eval_batch(const ChainView cv, const uint32_t* _
 
 // Apply the proposal in window slot `slot` (pk, u, v given): all lanes take part, lane j updates the counters
 // of window bit j, lanes 0 and 1 rewrite the words of the schedule and of the full-step bitmap.
-template <bool GROW>
+template <bool GROW, bool COW>
 __device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint32_t S32, uint32_t cap, uint32_t lane,
                                            uint32_t slot, uint32_t pk, uint32_t u, uint32_t v)
 {
@@ -454,6 +486,8 @@ __device__ __forceinline__ void apply_move(const ChainView cv, uint32_t S, uint3
     if (valid) cv.ctr[t] = c;
     uint32_t F = __ballot_sync(0xFFFFFFFFu, valid && c.w == cap);   // bit j <-> window bit j
     uint32_t V = __ballot_sync(0xFFFFFFFFu, valid);
+    cv.own<COW>(u, lane);
+    if (swap) cv.own<COW>(v, lane);
     if (lane < 2) {
         uint32_t M = ((1u << run) - 1u) << 1, NU = Nu, NV = Nv, sbit = s0 - 1;
         if (s0 == 0) { F >>= 1; V >>= 1; M >>= 1; NU >>= 1; NV >>= 1; sbit = 0; }
@@ -501,6 +535,37 @@ __device__ __forceinline__ void copy_words(uint32_t* __restrict__ dst, const uin
     }
 }
 
+// The copies off the hot path (a bucket fetched into a slice, a best state saved) as one function each, so that the
+// chain loop stays small enough for the instruction cache.
+__device__ __noinline__ void copy_words_cold(uint32_t* dst, const uint32_t* src, size_t n, uint32_t lane)
+{
+    copy_words(dst, src, n, lane);
+}
+
+// Schedules in global scratch are copy-on-write overlays of the one initial schedule that all chains share: the
+// units come in buckets of 2^shift consecutive units, a chain's slice holds a bucket only once the chain has
+// rewritten a unit of it, and a bitmap in shared memory says which. Chains change few of their units, so nearly
+// every placement window is read from the shared initial schedule, which stays in L2, and not from a private slice
+// that only DRAM can hold; a chain that rewrites everything ends up copying its whole slice once, bucket by bucket.
+// The bitmap takes the shared memory that a full CTA of chains leaves free (kCowBitsMin to kCowBitsMax buckets): a
+// chain of a million moves rewrites thousands of units, and every read of a bucket it owns misses L2, so the buckets
+// should be small (with 8192 buckets of 512 units a chain of the largest configuration owned two thirds of them at
+// its end; with 40,960 of 64 units it owns an eighth).
+constexpr uint32_t kCowBitsMin = 8192, kCowBitsMax = 65536;
+
+// A whole schedule out of a copy-on-write slice: the buckets the slice holds from it, the rest from the initial one.
+__device__ __forceinline__ void copy_merged(uint32_t* __restrict__ dst, const uint32_t* __restrict__ mine,
+                                            const uint32_t* __restrict__ p0, const uint32_t* have, uint32_t shift,
+                                            uint32_t U, uint32_t S32, uint32_t lane)
+{
+    const uint32_t nb = (U + (1u << shift) - 1u) >> shift;
+    for (uint32_t b = 0; b < nb; ++b) {
+        const size_t lo = (size_t)(b << shift) * S32, hi = (size_t)min(U, (b + 1u) << shift) * S32;
+        const uint32_t* src = (have[b >> 5] >> (b & 31u)) & 1u ? mine : p0;
+        copy_words_cold(dst + lo, src + lo, hi - lo, lane);
+    }
+}
+
 // Hand-over block of a chain that is served by more than one warp (shared memory, one per chain).
 // The warps of a chain take the batches in turn: warp w owns batches w, w + W, w + 2W, ... It evaluates a batch
 // against whatever state it finds (another warp may be committing an earlier batch meanwhile), then waits for its
@@ -532,22 +597,23 @@ __device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p) { return 
 __device__ __forceinline__ void st_volatile_u32(uint32_t* p, uint32_t v) { *reinterpret_cast<volatile uint32_t*>(p) = v; }
 
 // shared-memory words (as uint4 slots) of one chain besides its schedule
-__host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool grow, uint32_t W, bool halfq, bool touch)
+// cow4: uint4 slots of the bucket bitmap of a copy-on-write slice (schedules in global scratch), else 0
+__host__ __device__ inline uint32_t chain_fixed4(uint32_t S, uint32_t S32, bool grow, uint32_t W, bool halfq, uint32_t cow4)
 {
-    return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + (touch ? 1u : 0u) + (W > 1 ? kShareSlots4 : 0u) +
-           W * priv_slots4(halfq);
+    return S + (S32 + 3) / 4 + (grow ? (S + 3) / 4 : 0u) + cow4 + (W > 1 ? kShareSlots4 : 0u) + W * priv_slots4(halfq);
 }
 
 // ASMEM (only with PSMEM): the access bitmap and the per-step constants, which every chain of the CTA reads, are
 // staged in shared memory once per CTA. With the schedules in shared memory the L1 cache is down to its minimum and
 // cannot hold them.
-// TOUCH (only without PSMEM): the chain logs the units it rewrites, and may start from a slice that holds the final
-// state of an earlier chain with such a log (ChainParams::restore).
-template <bool PSMEM, bool GROW, int W, bool ASMEM, bool TOUCH>
+// Without PSMEM the chain's slice of global scratch is a copy-on-write overlay of the initial schedule when
+// prm.cow_slots4 is set (jobs whose slices add up to gigabytes: the chains then start without copying anything), else a
+// plain copy of it (small slices: the copy costs nothing and an applied move is cheaper without the take-over).
+template <bool PSMEM, bool GROW, int W, bool ASMEM, bool COW>
 __global__ void __launch_bounds__(512)
 chain_kernel(const ChainParams prm)
 {
-    static_assert(!TOUCH || !PSMEM, "touch logs only for schedules in global scratch");
+    static_assert(!COW || !PSMEM, "overlays only for schedules in global scratch");
     static_assert(W >= 1 && W <= kMaxW && (W & (W - 1)) == 0, "warps per chain");
     static_assert(PSMEM || !ASMEM, "shared access bitmap only beside shared schedules");
     extern __shared__ uint4 smem4[];
@@ -563,21 +629,22 @@ chain_kernel(const ChainParams prm)
     const size_t pwords = (size_t)U * S32;
     const uint32_t f4 = (S32 + 3) / 4;                            // uint4 slots of the full-step bitmap
     const uint32_t h4 = GROW ? (S + 3) / 4 : 0u;                  // uint4 slots of the written-to-HBM counts
-    const uint32_t fixed4 = chain_fixed4(S, S32, GROW, W, ASMEM, TOUCH);
-    constexpr uint32_t t4 = TOUCH ? 1u : 0u;
+    const uint32_t o4 = COW ? prm.cow_slots4 : 0u;                 // the slice is a copy-on-write overlay
+    const uint32_t fixed4 = chain_fixed4(S, S32, GROW, W, ASMEM, o4);
     uint4* const mine4 = smem4 + (size_t)cic * fixed4;
     ChainView cv;
     cv.ctr = mine4;
     cv.full = reinterpret_cast<uint32_t*>(mine4 + S);
     cv.hb = reinterpret_cast<uint32_t*>(mine4 + S + f4);
-    uint32_t* const touched = reinterpret_cast<uint32_t*>(mine4 + S + f4 + h4);   // TOUCH: entries in the chain's log
-    ChainShare* const sh = reinterpret_cast<ChainShare*>(mine4 + S + f4 + h4 + t4);
-    uint4* const priv4 = mine4 + S + f4 + h4 + t4 + (W > 1 ? kShareSlots4 : 0u) + sub * priv_slots4(ASMEM);
+    uint32_t* const cowmap = reinterpret_cast<uint32_t*>(mine4 + S + f4 + h4);   // buckets the slice holds
+    ChainShare* const sh = reinterpret_cast<ChainShare*>(mine4 + S + f4 + h4 + o4);
+    uint4* const priv4 = mine4 + S + f4 + h4 + o4 + (W > 1 ? kShareSlots4 : 0u) + sub * priv_slots4(ASMEM);
     cv.win = priv4;
     cv.acc = reinterpret_cast<int*>(priv4 + kWinSlots4);
     cv.queue = reinterpret_cast<uint16_t*>(priv4 + kWinSlots4 + kAccSlots4);
     uint32_t* const pool = reinterpret_cast<uint32_t*>(smem4 + (size_t)cpb * fixed4);   // schedules, then A, then constants
     cv.P = PSMEM ? pool + (size_t)cic * pwords : prm.ws + (size_t)slot * pwords;
+    cv.p0 = prm.Pcol0; cv.have = COW ? cowmap : nullptr; cv.shared_chain = W > 1; cv.shift = prm.cow_shift; cv.U = U; cv.S32 = S32;
     const uint32_t* Acol = prm.Acol;
     const StepC* stepc = prm.stepc;
     if (ASMEM) {
@@ -595,20 +662,9 @@ chain_kernel(const ChainParams prm)
         if (GROW)
             for (uint32_t i = tid; i < S; i += 32 * W) cv.hb[i] = __ldg(prm.hb0 + i);
         for (uint32_t i = lane; i < kWinSlots4; i += 32) cv.win[i] = make_uint4(0u, 0u, 0u, 0u);
-        bool whole = true;
-        if (TOUCH && prm.restore) {
-            const uint32_t n = __ldcg(prm.touch_len + slot);
-            if (n <= prm.touch_cap) {
-                whole = false;
-                const uint32_t* tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
-                for (uint32_t i = tid; i < n; i += 32 * W) {
-                    const size_t o = (size_t)__ldcg(tlog + i) * S32;
-                    for (uint32_t w = 0; w < S32; ++w) cv.P[o + w] = __ldg(prm.Pcol0 + o + w);
-                }
-            }
-        }
-        if (whole) copy_words(cv.P, prm.Pcol0, pwords, tid, 32 * W);
-        if (TOUCH && tid == 0) *touched = 0u;
+        if (!COW) copy_words(cv.P, prm.Pcol0, pwords, tid, 32 * W);
+        else
+            for (uint32_t i = tid; i < prm.cow_slots4 * 4; i += 32 * W) cowmap[i] = 0u;   // the slice holds nothing yet
         if (W > 1 && tid == 0) {
             sh->cur = sh->best = sh->best_at_boundary = prm.init_ticks;
             sh->best_move = ~0ull; sh->n_chg = 0; sh->hash = 0;
@@ -709,7 +765,7 @@ chain_kernel(const ChainParams prm)
             need[0] = todo[0];
             // the proposals of this warp's next batch of the level are drawn while this batch's windows are loaded
             // (drawn, and dropped, even where the level has no further batch for this warp)
-            eval_batch<GROW, ASMEM, true>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv,
+            eval_batch<GROW, ASMEM, true, COW>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv,
                                           [&]() {
                                               uint32_t r[4];
                                               const uint64_t mine = m + (uint64_t)W * kBatch + lane;
@@ -772,7 +828,7 @@ chain_kernel(const ChainParams prm)
 #pragma unroll
                 for (int h = 0; h < kMPL; ++h) any_need |= need[h];
                 if (any_need)
-                    eval_batch<GROW, ASMEM, false>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv,
+                    eval_batch<GROW, ASMEM, false, COW>(cv, Acol, prm.birth, stepc, prm.K, S, S32, trow, shift, prm.split_at, need, lane, mv,
                                                    []() {});
                 bool applied = false;
 #pragma unroll
@@ -803,17 +859,10 @@ chain_kernel(const ChainParams prm)
                         copy_words(snap, cv.P, pwords, lane);
                         snap_dirty = false;
                     }
-                    apply_move<GROW>(cv, S, S32, prm.cap, lane, h * 32 + bb, pk, bu, bv);
+                    apply_move<GROW, COW>(cv, S, S32, prm.cap, lane, h * 32 + bb, pk, bu, bv);
                     // The applied move rewrote steps s0b .. s0b + len_b (bits, counters, full flags). A later
                     // proposal read steps s0 - 1 .. s0 + len: it has to be evaluated again iff the two ranges meet.
                     const uint32_t s0b = pk >> 8, endb = s0b + ((pk >> 1) & 63u);
-                    if (TOUCH && prm.touch_log && lane == 0) {   // the units whose words no longer are the initial ones
-                        uint32_t* const tlog = prm.touch_log + (size_t)slot * prm.touch_cap;
-                        const uint32_t n = *touched, two = pk & 1u;
-                        if (n < prm.touch_cap) tlog[n] = bu;
-                        if (two && n + 1u < prm.touch_cap) tlog[n + 1u] = bv;
-                        *touched = min(n + 1u + two, prm.touch_cap + 1u);
-                    }
                     if (W > 1) {                                  // tell the warps that are evaluating later batches
                         if (lane == 0) {
                             sh->applog[napp % kLog] = s0b | (endb << 16);
@@ -859,7 +908,9 @@ chain_kernel(const ChainParams prm)
     }
     if (snap && snap_dirty) copy_words(snap, cv.P, pwords, lane);
     if (ulog && lane == 0) prm.undo_len[slot] = ulen;
-    if (TOUCH && prm.touch_log && lane == 0) prm.touch_len[slot] = *touched;
+    if (COW && prm.cow_out)                                    // which buckets the slice holds (for the walk back)
+        for (uint32_t i = lane; i < prm.cow_slots4 * 4; i += 32)
+            prm.cow_out[(size_t)slot * (prm.cow_slots4 * 4) + i] = cowmap[i];
     if (lane == 0) {
         kvp_chain_result res;
         res.best_ticks = best; res.best_move = best_move; res.final_ticks = cur; res.moves_done = m_end;
@@ -868,7 +919,8 @@ chain_kernel(const ChainParams prm)
     }
     if (prm.dump && slot == 0) {
         __syncwarp();
-        copy_words(prm.dump, cv.P, pwords, lane);
+        if (!COW) copy_words(prm.dump, cv.P, pwords, lane);
+        else copy_merged(prm.dump, cv.P, prm.Pcol0, cowmap, prm.cow_shift, U, S32, lane);
     }
     if (W > 1 && stop) {                                          // ended by the stop rule: release the next owner
         __syncwarp();
@@ -915,24 +967,6 @@ template <> __device__ __forceinline__ void ctr_store<ushort4>(ushort4* c, uint3
 {
     c[t] = make_ushort4((unsigned short)v.x, (unsigned short)v.y, (unsigned short)v.z, (unsigned short)v.w);
 }
-
-// The copies off the hot path (a bucket fetched into a slice, a best state saved) as one function each, so that the
-// chain loop stays small enough for the instruction cache.
-__device__ __noinline__ void copy_words_cold(uint32_t* dst, const uint32_t* src, size_t n, uint32_t lane)
-{
-    copy_words(dst, src, n, lane);
-}
-
-// Schedules in global scratch are copy-on-write overlays of the one initial schedule that all chains share: the
-// units come in buckets of 2^shift consecutive units, a chain's slice holds a bucket only once the chain has
-// rewritten a unit of it, and a bitmap in shared memory says which. Chains change few of their units, so nearly
-// every placement window is read from the shared initial schedule, which stays in L2, and not from a private slice
-// that only DRAM can hold; a chain that rewrites everything ends up copying its whole slice once, bucket by bucket.
-// The bitmap takes the shared memory that a full CTA of chains leaves free (kCowBitsMin to kCowBitsMax buckets): a
-// chain of a million moves rewrites thousands of units, and every read of a bucket it owns misses L2, so the buckets
-// should be small (with 8192 buckets of 512 units a chain of the largest configuration owned two thirds of them at
-// its end; with 40,960 of 64 units it owns an eighth).
-constexpr uint32_t kCowBitsMin = 8192, kCowBitsMax = 65536;
 
 // Where a chain of the wide kernel keeps its state. CT: the four per-step cardinalities as 16-bit fields when the
 // schedule lives in shared memory (then units < 2^16), as 32-bit fields otherwise. COW: see above.
@@ -1306,19 +1340,6 @@ __device__ __forceinline__ void wide_apply(const WideView<CT, COW, COLV> cv, con
         }
     }
     __syncwarp();
-}
-
-// A whole schedule out of a copy-on-write slice: the buckets the slice holds from it, the rest from the initial one.
-__device__ __forceinline__ void copy_merged(uint32_t* __restrict__ dst, const uint32_t* __restrict__ mine,
-                                            const uint32_t* __restrict__ p0, const uint32_t* have, uint32_t shift,
-                                            uint32_t U, uint32_t S32, uint32_t lane)
-{
-    const uint32_t nb = (U + (1u << shift) - 1u) >> shift;
-    for (uint32_t b = 0; b < nb; ++b) {
-        const size_t lo = (size_t)(b << shift) * S32, hi = (size_t)min(U, (b + 1u) << shift) * S32;
-        const uint32_t* src = (have[b >> 5] >> (b & 31u)) & 1u ? mine : p0;
-        copy_words_cold(dst + lo, src + lo, hi - lo, lane);
-    }
 }
 
 // PSMEM: the schedule lives in shared memory (16-bit counters); otherwise the chain's slice of global scratch is a
@@ -1790,10 +1811,6 @@ struct Ctx {
     uint64_t* undo_log;      // undo logs (global variant), or null
     uint32_t* undo_len;
     uint32_t undo_cap;
-    uint32_t* touch_log;     // touched-unit logs (global variant), or null
-    uint32_t* touch_len;
-    uint32_t touch_cap;
-    bool touch;              // the chains come in several waves and log the units they rewrite
     uint32_t* cow_out;       // wide kernel, global variant: bucket bitmaps of the slices, or null
     uint32_t cow_shift;
     uint32_t cow_slots4;     // uint4 slots of a chain's bucket bitmap
@@ -1826,16 +1843,16 @@ int validate(const kvp_problem* p, const kvp_anneal_params* a)
 
 typedef void (*ChainKernel)(const ChainParams);
 
-template <bool PSMEM, bool ASMEM, bool TOUCH>
+template <bool PSMEM, bool ASMEM, bool COW>
 ChainKernel chain_kernel_pick(bool grow, uint32_t W)
 {
-    if (W == 2) return grow ? chain_kernel<PSMEM, true, 2, ASMEM, TOUCH> : chain_kernel<PSMEM, false, 2, ASMEM, TOUCH>;
-    return grow ? chain_kernel<PSMEM, true, 1, ASMEM, TOUCH> : chain_kernel<PSMEM, false, 1, ASMEM, TOUCH>;
+    if (W == 2) return grow ? chain_kernel<PSMEM, true, 2, ASMEM, COW> : chain_kernel<PSMEM, false, 2, ASMEM, COW>;
+    return grow ? chain_kernel<PSMEM, true, 1, ASMEM, COW> : chain_kernel<PSMEM, false, 1, ASMEM, COW>;
 }
 
-ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W, bool touch)
+ChainKernel chain_kernel_for(bool psmem, bool asmem, bool grow, uint32_t W, bool cow)
 {
-    if (!psmem) return touch ? chain_kernel_pick<false, false, true>(grow, W) : chain_kernel_pick<false, false, false>(grow, W);
+    if (!psmem) return cow ? chain_kernel_pick<false, false, true>(grow, W) : chain_kernel_pick<false, false, false>(grow, W);
     return asmem ? chain_kernel_pick<true, true, false>(grow, W) : chain_kernel_pick<true, false, false>(grow, W);
 }
 
@@ -1850,28 +1867,26 @@ ChainKernel wide_kernel_for(bool psmem, bool asmem, bool grow, uint32_t S32)
     return grow ? wide_chain_kernel<true, true, false, 0> : wide_chain_kernel<true, false, false, 0>;
 }
 
-ChainKernel kernel_of(const Ctx& c, bool psmem, bool asmem, uint32_t W, bool touch)
+ChainKernel kernel_of(const Ctx& c, bool psmem, bool asmem, uint32_t W)
 {
-    return c.wide ? wide_kernel_for(psmem, asmem, c.grow, c.S32) : chain_kernel_for(psmem, asmem, c.grow, W, touch);
+    return c.wide ? wide_kernel_for(psmem, asmem, c.grow, c.S32) : chain_kernel_for(psmem, asmem, c.grow, W, c.cow_slots4 != 0);
 }
 
 int launch_chains(const Ctx& c, const ChainParams& prm, uint32_t count)
 {
     const uint32_t grid = (count + c.wpb - 1) / c.wpb;
     const size_t smem = (size_t)c.wpb * c.smem_per_warp + c.smem_shared;
-    kernel_of(c, c.psmem, c.asmem, c.wpc, c.touch)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
+    kernel_of(c, c.psmem, c.asmem, c.wpc)<<<grid, c.wpb * c.wpc * 32, smem, c.st>>>(prm);
     KVP_CUDA(cudaGetLastError());
     return KVP_OK;
 }
 
 int run_chains(Ctx& c, uint32_t first, uint32_t count, uint32_t result_base, kvp_chain_result* results, uint64_t upto,
-               uint32_t* dump, uint32_t* snap, bool with_undo = false, bool restore = false)
+               uint32_t* dump, uint32_t* snap, bool with_undo = false)
 {
     ChainParams prm = c.prm;
     prm.snap = snap;
     prm.undo_log = with_undo ? c.undo_log : nullptr; prm.undo_len = c.undo_len; prm.undo_cap = c.undo_cap;
-    prm.touch_log = with_undo ? c.touch_log : nullptr; prm.touch_len = c.touch_len; prm.touch_cap = c.touch_cap;
-    prm.restore = with_undo && restore && c.touch_log ? 1u : 0u;
     prm.cow_out = c.cow_out; prm.cow_shift = c.cow_shift; prm.cow_slots4 = c.cow_slots4;
     prm.stage_stepc = c.stage_stepc ? 1u : 0u;
     prm.chain_first = first; prm.chain_count = count; prm.result_base = result_base;
@@ -1914,13 +1929,12 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
     c.wide = exchange || hooks.warps_per_chain == 3 ||
              (hooks.warps_per_chain == 0 && (chains_per_sm > 8 || (wide_in_smem && chains_per_sm > 5 && !hot)));
     // `shared`: the schedule is in shared memory (the wide kernel then keeps 16-bit counters)
-    auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool touch = false, bool shared = true) {
+    auto fixed_bytes = [&](uint32_t W, bool halfq = false, bool shared = true) {
         if (c.wide) return (size_t)wide_fixed4(p->S, p->S32, c.grow, shared, shared ? 0u : c.cow_slots4) * 16;
-        return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq, touch) * 16;
+        return (size_t)chain_fixed4(p->S, p->S32, c.grow, W, halfq, shared ? 0u : c.cow_slots4) * 16;
     };
-    c.touch = false;
     c.stage_stepc = false;
-    c.cow_slots4 = kCowBitsMin / 128;
+    c.cow_slots4 = 0;
     c.cow_shift = 0;
     // Two warps per chain while that leaves an SM at most 16 warps (the registers allow no more): a job of few
     // chains then keeps twice as many warps in flight. kvp_set_test_hooks can override the choice (tests, tuning).
@@ -1954,19 +1968,28 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
                 c.smem_shared = with_c - (size_t)c.wpb * c.smem_per_warp;
             }
         }
-        KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, true, c.asmem, W, false), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, true, c.asmem, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
     } else {
-        // planned without the touch logs first; a job that then needs several waves is planned again with them (one
-        // more shared-memory slot per chain)
-        for (int pass = 0; pass < 2; ++pass) {
-            c.touch = pass == 1;
-            if (c.wide) {
-                // The bucket bitmap of the copy-on-write slices takes what a full CTA of chains leaves of the shared
-                // memory: the smaller the buckets, the fewer reads of a long chain go to its private slice.
-                c.cow_slots4 = 0;
-                const size_t bare = fixed_bytes(W, false, false, false);
-                const size_t stepc_bytes = (size_t)p->S * 16 <= 32768 ? (size_t)p->S * 16 : 0;
-                const size_t share = (budget - stepc_bytes) / (kWideGlobalThreads / 32);
+        {
+            // Copy-on-write slices: always for the wide kernel; for the narrow kernel where whole copies of the initial
+            // schedule would add up to gigabytes (growing_8b: 1024 x 17 MB, a third of the kernel's time), not where
+            // they are small (layer_8b: 1024 x 512 KB), because a take-over lengthens the path through an applied move
+            // (layer_8b 14.0 -> 16.0 ms with it).
+            const size_t per_sm_max = c.wide ? kWideGlobalThreads / 32 : 16 / W;
+            const size_t most = a->chains < per_sm_max * sms ? a->chains : per_sm_max * sms;
+            const bool overlay = c.wide || most * col_bytes >= ((size_t)4 << 30);
+            c.cow_slots4 = 0;
+            c.cow_shift = 0;
+            if (overlay) {
+                // The bucket bitmap takes what a full CTA of chains leaves of the shared memory: the smaller the
+                // buckets, the fewer reads of a long chain go to its private slice.
+                const size_t bare = fixed_bytes(W, false, false);
+                const size_t stepc_bytes = c.wide && (size_t)p->S * 16 <= 32768 ? (size_t)p->S * 16 : 0;
+                uint32_t per_cta = c.wide ? kWideGlobalThreads / 32 : 16 / W;     // chains of a full CTA
+                if (chains_per_sm < per_cta) per_cta = chains_per_sm ? chains_per_sm : 1u;
+                if ((budget - stepc_bytes) / bare < per_cta) per_cta = (uint32_t)((budget - stepc_bytes) / bare);
+                if (per_cta < 1) return KVP_ERR_RANGE;
+                const size_t share = (budget - stepc_bytes) / per_cta;
                 size_t bits = share > bare ? (share - bare) / 16 * 128 : 0;
                 if (bits < kCowBitsMin) bits = kCowBitsMin;
                 if (bits > kCowBitsMax) bits = kCowBitsMax;
@@ -1975,7 +1998,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
                 const uint64_t buckets = ((uint64_t)p->U + (1ull << c.cow_shift) - 1) >> c.cow_shift;
                 c.cow_slots4 = (uint32_t)((buckets + 127) / 128);
             }
-            const size_t ctr_bytes = fixed_bytes(W, false, c.touch, false);
+            const size_t ctr_bytes = fixed_bytes(W, false, false);
             if (ctr_bytes > budget) return KVP_ERR_RANGE;
             c.smem_per_warp = ctr_bytes;
             c.smem_shared = 0;
@@ -1987,9 +2010,9 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
             uint32_t wcap = (uint32_t)((budget - c.smem_shared) / ctr_bytes);   // chains per CTA at most
             if (wcap > 16 / W) wcap = 16 / W;
             if (c.wide && wcap > kWideGlobalThreads / 32) wcap = kWideGlobalThreads / 32;
-            KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, false, false, W, c.touch), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+            KVP_CUDA(cudaFuncSetAttribute(kernel_of(c, false, false, W), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
             int ctas = 0;
-            KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, kernel_of(c, false, false, W, c.touch), (int)(wcap * W * 32),
+            KVP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&ctas, kernel_of(c, false, false, W), (int)(wcap * W * 32),
                                                                    wcap * c.smem_per_warp + c.smem_shared));
             if (ctas < 1) return KVP_ERR_RANGE;
             uint32_t per_sm = (uint32_t)ctas * wcap;                   // resident chains per SM, at most 32 warps
@@ -2017,8 +2040,6 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
             // a wave is spread over all SMs: CTAs of ceil(resident / SMs) chains where one CTA per SM holds them
             const uint32_t even = (c.resident + sms - 1) / sms;
             c.wpb = even < wcap ? even : wcap;
-            // the wide kernel's slices are overlays of the initial schedule: a later wave just starts an empty one
-            if (a->chains <= c.resident || c.wide) break;
         }
     }
     // a replica-exchange run keeps every chain's slice between its rounds: all chains have to be resident at once
@@ -2045,10 +2066,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
     const size_t o_ulog = take((size_t)c.resident * c.undo_cap * 8), o_ulen = take(c.psmem ? 0 : (size_t)c.resident * 4);
     // Where the chains come in several waves they also log the units they rewrite (4 bytes each, up to 16384): the
     // chain that takes over the slice in the next wave copies only those from the initial schedule again, not all of it.
-    const bool touch = c.touch;
-    c.touch_cap = touch ? 16384u : 0u;
-    const size_t o_tlog = take((size_t)c.resident * c.touch_cap * 4), o_tlen = take(touch ? (size_t)c.resident * 4 : 0);
-    const bool cow = c.wide && !c.psmem;
+    const bool cow = !c.psmem && c.cow_slots4 != 0;
     const size_t o_cow = take(cow ? (size_t)c.resident * c.cow_slots4 * 16 : 0);
     rc = ensure_chain_ws(p, off, st);
     if (rc) return rc;
@@ -2060,7 +2078,6 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
     c.hb0 = c.grow ? (uint32_t*)(base + o_hb0) : nullptr; c.hb_tmp = c.grow ? (uint32_t*)(base + o_hbt) : nullptr;
     c.full0 = (uint32_t*)(base + o_full); c.snap = snapshots ? (uint32_t*)(base + o_snap) : nullptr;
     c.undo_log = c.psmem ? nullptr : (uint64_t*)(base + o_ulog); c.undo_len = c.psmem ? nullptr : (uint32_t*)(base + o_ulen);
-    c.touch_log = touch ? (uint32_t*)(base + o_tlog) : nullptr; c.touch_len = touch ? (uint32_t*)(base + o_tlen) : nullptr;
     c.cow_out = cow ? (uint32_t*)(base + o_cow) : nullptr;
 
     // initial schedule in both layouts
@@ -2200,7 +2217,7 @@ extern "C" int kvp_anneal(kvp_problem* p, const kvp_anneal_params* a, uint32_t* 
     for (uint32_t first = 0; first < a->chains; first += c.resident, ++waves) {
         const uint32_t count = a->chains - first < c.resident ? a->chains - first : c.resident;
         if ((rc = run_chains(c, a->first_chain + first, count, a->first_chain, c.results, a->moves, nullptr, c.snap,
-                             c.undo_log != nullptr, waves > 0)))
+                             c.undo_log != nullptr)))
             return rc;
         if (c.undo_log) {
             // Best so far over the chains that have finished; if it belongs to this wave, walk that chain back to
@@ -2400,7 +2417,7 @@ extern "C" int kvp_anneal_exchange(kvp_problem* p, const kvp_anneal_params* a, c
     KVP_CUDA(cudaEventRecord(ev[1], st));
 
     ChainParams prm = c.prm;
-    prm.snap = c.snap; prm.undo_log = nullptr; prm.touch_log = nullptr; prm.restore = 0u;
+    prm.snap = c.snap; prm.undo_log = nullptr;
     prm.cow_out = nullptr; prm.cow_shift = c.cow_shift; prm.cow_slots4 = c.cow_slots4;
     prm.stage_stepc = c.stage_stepc ? 1u : 0u;
     prm.chain_first = a->first_chain; prm.chain_count = chains; prm.result_base = a->first_chain;

@@ -206,6 +206,19 @@ def test_anneal_full_shape_all_waves(kvp, oracle, name, moves, p0):
     assert int(ev["total_ticks"][0]) == out["best_ticks"] and int(ev["bad_step"][0]) == -1
     if p0 > 0.1:
         assert min(r.n_changed for r in out["per_chain"]) > 100       # the hot start rewrites hundreds of units
+    if name == "full_8b":
+        # the same job on the narrow kernel, one and two warps per chain: slices of this size are copy-on-write overlays
+        # of the initial schedule there too, the chains come in more waves, and the winner is walked back in its overlay
+        for warps in (1, 2):
+            kvp.set_test_hooks(warps_per_chain=warps)
+            try:
+                again = g.anneal(g.make_params(**kw), want_per_chain=True)
+            finally:
+                kvp.set_test_hooks()
+            assert not again["stats"].wide_kernel and again["stats"].chain_launches >= (2, 4)[warps - 1]
+            assert [r.astuple() for r in again["per_chain"]] == [r.astuple() for r in out["per_chain"]]
+            assert again["stats"].best_chain == w and again["best_ticks"] == out["best_ticks"]
+            assert np.array_equal(to_np(again["best_schedule"]), best[w])
 
 
 def test_anneal_layer_8b_stated_budget(kvp, oracle):

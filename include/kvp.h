@@ -474,6 +474,8 @@ typedef struct {
                                    path of the half-size work queue                                              */
     uint32_t resident;          /* n: at most n chains whose schedules live in global memory run at a time, so
                                    that a small job comes in several waves                                       */
+    uint32_t overlay;           /* narrow chain kernel, schedules in global memory: 1 = copy-on-write slices, 2 =
+                                   plain slices, whatever the size of the job (0: by size)                       */
 } kvp_test_hooks;
 void kvp_set_test_hooks(const kvp_test_hooks* hooks);
 

@@ -23,7 +23,7 @@ namespace kvp {
 
 namespace {
 
-kvp_test_hooks g_hooks = {0u, 0u, 0u, 0u};   // kvp_set_test_hooks; read once per call
+kvp_test_hooks g_hooks = {0u, 0u, 0u, 0u, 0u};   // kvp_set_test_hooks; read once per call
 
 struct ChainParams {
     const uint32_t* Acol;        // [U][S32]
@@ -1977,7 +1977,7 @@ int prepare(kvp_problem* p, const kvp_anneal_params* a, cudaStream_t st, Ctx& c,
             // (layer_8b 14.0 -> 16.0 ms with it).
             const size_t per_sm_max = c.wide ? kWideGlobalThreads / 32 : 16 / W;
             const size_t most = a->chains < per_sm_max * sms ? a->chains : per_sm_max * sms;
-            const bool overlay = c.wide || most * col_bytes >= ((size_t)4 << 30);
+            const bool overlay = c.wide || (hooks.overlay ? hooks.overlay == 1 : most * col_bytes >= ((size_t)4 << 30));
             c.cow_slots4 = 0;
             c.cow_shift = 0;
             if (overlay) {

@@ -110,7 +110,7 @@ class TraceParams(C.Structure):
 
 class TestHooks(C.Structure):
     _fields_ = [("warps_per_chain", C.c_uint32), ("drop_turn", C.c_uint32), ("split_queue_plus1", C.c_uint32),
-                ("resident", C.c_uint32)]
+                ("resident", C.c_uint32), ("overlay", C.c_uint32)]
 
 
 _handle = None
@@ -152,9 +152,10 @@ def _stream(stream=None):
     return C.c_void_p(s.cuda_stream)
 
 
-def set_test_hooks(warps_per_chain=0, drop_turn=0, split_queue=None, resident=0):
+def set_test_hooks(warps_per_chain=0, drop_turn=0, split_queue=None, resident=0, overlay=0):
     """kvp_set_test_hooks (test-suite and tuning only; process-wide). Called without arguments it resets everything."""
-    h = TestHooks(int(warps_per_chain), int(drop_turn), 0 if split_queue is None else int(split_queue) + 1, int(resident))
+    h = TestHooks(int(warps_per_chain), int(drop_turn), 0 if split_queue is None else int(split_queue) + 1, int(resident),
+                  int(overlay))
     _lib().kvp_set_test_hooks(C.byref(h))
 
 

@@ -255,22 +255,23 @@ def test_global_state_winner_paths(kvp, oracle, warps_per_chain):
         assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
 
 
-def test_later_waves_copy_only_what_changed(kvp, oracle, warps_per_chain):
+@pytest.mark.parametrize("overlay", [1, 2], ids=["overlay", "plain"])
+def test_later_waves_start_afresh(kvp, oracle, hooks, warps_per_chain, overlay):
     """More chains than are resident at once: a chain of a later wave takes over a slice of global scratch that holds
-    the final state of an earlier chain, and copies from the initial schedule only the units which that chain logged
-    as rewritten, or all of it once the log has overflowed (the hot start below). Chains of every wave against the
-    oracle; the counts of applied moves show that the first run stays inside the log and the second goes beyond it."""
+    the final state of an earlier chain. With copy-on-write slices it starts from an empty overlay of the initial
+    schedule, with plain slices from a fresh copy (the narrow kernel has both forms, test hook; the wide kernel always
+    the first). Chains of every wave against the oracle, after a warm start with few rewritten units and after a hot
+    one that rewrites most of them."""
+    hooks(overlay=overlay)
     g, o, cfg, A = named_problem(kvp, oracle, "layer_8b")
-    for kw, overflow in ((dict(chains=5000, moves=2000, seed=7, p0=0.3, levels=4), False),
-                         (dict(chains=2600, moves=160_000, seed=7, p0=0.8, levels=4), True)):
+    for kw, hot in ((dict(chains=5000, moves=2000, seed=7, p0=0.3, levels=4), False),
+                    (dict(chains=2600, moves=160_000, seed=7, p0=0.8, levels=4), True)):
         gp, op = _params(g, o, **kw)
         out = g.anneal(gp, want_per_chain=True)
         n = kw["chains"]
         changed = [r.n_changed for r in out["per_chain"]]
-        if overflow:
-            assert min(changed) > 16384                 # every log overflowed: one entry or two per applied move
-        else:
-            assert min(changed) > 0 and 2 * max(changed) <= 16384
+        assert min(changed) > (16384 if hot else 0)     # hot: more applied moves than the problem has units
+        assert out["stats"].chain_launches >= 2
         for c in (0, 1, n // 2, n // 2 + 1, n - 2, n - 1):
             want, _, _ = o.anneal_chains(op, c, 1)
             assert out["per_chain"][c].astuple() == want[0].astuple(), c
@@ -279,13 +280,15 @@ def test_later_waves_copy_only_what_changed(kvp, oracle, warps_per_chain):
         assert np.array_equal(to_np(out["best_schedule"]), bst[0]) and out["best_ticks"] == ref[0].best_ticks
 
 
+@pytest.mark.parametrize("overlay", [1, 2], ids=["overlay", "plain"])
 @pytest.mark.parametrize("resident", [1, 3, 4])
-def test_small_job_in_several_waves(kvp, oracle, hooks, resident, warps_per_chain):
+def test_small_job_in_several_waves(kvp, oracle, hooks, resident, warps_per_chain, overlay):
     """Schedules in global memory, at most `resident` chains at a time (test hook): every chain but the first ones
-    starts from a slice that an earlier chain left behind and restores only what that chain logged as rewritten.
-    All chains, the bound and the winner's schedule against the oracle, at a hot and a cold start, with the stop
-    rule, and with a winner that an early wave produced."""
-    hooks(resident=resident)
+    starts in a slice that an earlier chain left behind, as a copy-on-write overlay of the initial schedule or as a
+    plain copy of it (test hook; the narrow kernel has both forms). All chains, the bound and the winner's schedule
+    (walked back in its slice) against the oracle, at a hot and a cold start, with the stop rule, and with a winner
+    that an early wave produced."""
+    hooks(resident=resident, overlay=overlay)
     U, S, cap = 3000, 300, 700
     A = wl.random_access(U, S, 0.2, seed=21)
     g, o = both_problems(kvp, oracle, U, 8192, S, A, cap, (8000 * GB, 900 * GB, 900 * GB))

@@ -1,8 +1,11 @@
-// Annealing kernels: one or two warps per chain, one proposal per lane.
+// Annealing kernels. Two of them, chosen per job (see prepare()): the narrow chain kernel described here (one or two
+// warps per chain, one proposal per lane) and the wide one further down (one warp per chain, four proposals per lane,
+// most proposals settled by their placement bits alone).
 //
 // State of a chain: the schedule in time-packed form (for every unit a bit string over the steps), either
-// in shared memory (small problems) or in a private slice of global scratch, plus the four per-step
-// cardinalities {hr, mi, mo, occ} in shared memory and the running total T.
+// in shared memory (small problems) or in a private slice of global scratch (a plain copy of the initial schedule,
+// or a copy-on-write overlay of the one all chains share), plus the four per-step cardinalities {hr, mi, mo, occ}
+// in shared memory and the running total T.
 //
 // A proposal (one Philox4x32-10 block, a pure function of seed, chain and move index) names a run of at most
 // 30 consecutive steps and one or two units. Only the run's steps and the step after it change cost. Proposals
